@@ -1,0 +1,421 @@
+/*
+ * CPU oracle for the MoE verification layer -- TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain, fp64 statement of what the verification-pass
+ * MoE layer computes for gamma draft-tree tokens.  Only the test-suite, the
+ * smoke check and the bench's CPU-baseline leg may call it; the product
+ * (CUDA) path shares no code with it and must never route through it.
+ *
+ * What it follows:
+ *   - Sec. 1 / Sec. 3 of the paper: a router assigns every token a top-k
+ *     subset S_l(x_t) of the E experts of layer l.
+ *   - Eq. 1: verification touches the union  E_verify = U_t S_l(x_t); its
+ *     cardinality (the paper's "average active experts" metric, Table 1/3
+ *     captions) is what this oracle reports as n_active.
+ *   - Sec. 3 ("verification can reuse expert weights"): every expert of the
+ *     union is applied to all tokens routed to it, so a weight row is decoded
+ *     once and reused.
+ *   - Fig. 1(c): one FP8 DeepSeek-V3.1 expert is 3*7168*2048 bytes = 44.04 MB;
+ *     oracle_expert_code_bytes() reproduces that figure.
+ * The paper does not print the expert FFN; the form used here is the gated
+ * SwiGLU FFN  down( silu(gate x) * (up x) )  without biases, routed outputs
+ * combined with the renormalised top-k router weights, plus always-on shared
+ * experts with weight 1 (Table 13: "256 routed + 1 shared").
+ *
+ * Everything is evaluated in double precision directly from the raw input
+ * bytes with the decoders below.  There is no blocking, fusion or reordering:
+ * loops run in the order of the definition.  OpenMP (optional) only splits
+ * independent output rows between threads.
+ *
+ * Every function here is pinned by tests that do not depend on this file's
+ * own arithmetic (library decoders, float64 matmul, brute force, closed
+ * forms); none is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORC_W_FP32 = 0, ORC_W_BF16 = 1, ORC_W_FP8E4M3_B128 = 2, ORC_W_MXFP4 = 3 };
+enum { ORC_ACT_FP32 = 0, ORC_ACT_BF16 = 1 };
+enum { ORC_SCORE_SOFTMAX = 0, ORC_SCORE_SIGMOID = 1 };
+
+typedef struct {
+  int32_t H, I, E, top_k, n_shared;
+  int32_t wfmt, afmt, score;
+  double routed_scale;
+} oracle_cfg;
+
+/* All pointers are HOST pointers.  Layouts (K = contraction dim, contiguous):
+ *   w_gate, w_up [E, I, H]; w_down [E, H, I]
+ *   fp32 / bf16        : plain elements
+ *   fp8 e4m3 + b128    : 1 byte per element, scales fp32 [E, ceil(N/128), ceil(K/128)]
+ *   mxfp4              : byte i of a row = elements 2i (low nibble), 2i+1 (high nibble);
+ *                        scales u8 e8m0 [E, N, K/32]
+ *   shared experts use the same layouts with leading dim n_shared.            */
+typedef struct {
+  const float *router_w; /* [E,H] fp32 */
+  const void *w_gate, *w_up, *w_down;
+  const void *s_gate, *s_up, *s_down;
+  const void *sh_gate, *sh_up, *sh_down;
+  const void *sh_s_gate, *sh_s_up, *sh_s_down;
+} oracle_layer;
+
+/* ---------------------------------------------------------------- decoders */
+
+/* bf16 is the upper half of an IEEE binary32. */
+double oracle_decode_bf16(uint16_t b) {
+  uint32_t u = ((uint32_t)b) << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+/* e4m3 "fn": 1 sign, 4 exponent (bias 7), 3 mantissa bits; no infinities;
+ * exponent 15 with mantissa 7 is NaN; exponent 0 is subnormal (m * 2^-9). */
+double oracle_decode_e4m3(uint8_t b) {
+  int s = b >> 7, e = (b >> 3) & 15, m = b & 7;
+  double v;
+  if (e == 15 && m == 7) return NAN;
+  if (e == 0)
+    v = ldexp((double)m, -9);
+  else
+    v = ldexp(1.0 + (double)m / 8.0, e - 7);
+  return s ? -v : v;
+}
+
+/* e2m1: 1 sign, 2 exponent (bias 1), 1 mantissa bit -> 0, .5, 1, 1.5, 2, 3, 4, 6 */
+double oracle_decode_e2m1(uint8_t nib) {
+  int s = (nib >> 3) & 1, e = (nib >> 1) & 3, m = nib & 1;
+  double v = (e == 0) ? 0.5 * (double)m : ldexp(1.0 + 0.5 * (double)m, e - 1);
+  return s ? -v : v;
+}
+
+/* e8m0: unsigned power-of-two scale 2^(b-127); 0xFF is NaN. */
+double oracle_decode_e8m0(uint8_t b) {
+  if (b == 0xFF) return NAN;
+  return ldexp(1.0, (int)b - 127);
+}
+
+static double decode_act(const void *x, int afmt, size_t idx) {
+  if (afmt == ORC_ACT_FP32) return (double)((const float *)x)[idx];
+  return oracle_decode_bf16(((const uint16_t *)x)[idx]);
+}
+
+/* Decode row n of the [N,K] matrix of expert e into out[K]. */
+static void decode_row(int wfmt, const void *w, const void *s, int64_t e, int64_t N, int64_t K,
+                       int64_t n, double *out) {
+  if (wfmt == ORC_W_FP32) {
+    const float *p = (const float *)w + (e * N + n) * K;
+    for (int64_t k = 0; k < K; ++k) out[k] = (double)p[k];
+  } else if (wfmt == ORC_W_BF16) {
+    const uint16_t *p = (const uint16_t *)w + (e * N + n) * K;
+    for (int64_t k = 0; k < K; ++k) out[k] = oracle_decode_bf16(p[k]);
+  } else if (wfmt == ORC_W_FP8E4M3_B128) {
+    const uint8_t *p = (const uint8_t *)w + (e * N + n) * K;
+    int64_t nb = (N + 127) / 128, kb = (K + 127) / 128;
+    const float *sc = (const float *)s + (e * nb + n / 128) * kb;
+    for (int64_t k = 0; k < K; ++k) out[k] = oracle_decode_e4m3(p[k]) * (double)sc[k / 128];
+  } else { /* MXFP4 */
+    const uint8_t *p = (const uint8_t *)w + (e * N + n) * (K / 2);
+    const uint8_t *sc = (const uint8_t *)s + (e * N + n) * (K / 32);
+    for (int64_t k = 0; k < K; ++k) {
+      uint8_t byte = p[k >> 1];
+      uint8_t nib = (k & 1) ? (uint8_t)(byte >> 4) : (uint8_t)(byte & 15);
+      out[k] = oracle_decode_e2m1(nib) * oracle_decode_e8m0(sc[k / 32]);
+    }
+  }
+}
+
+/* Exposed so tests can pin the row decoder against library casts. */
+void oracle_decode_weight_row(int32_t wfmt, const void *w, const void *s, int64_t e, int64_t N,
+                              int64_t K, int64_t n, double *out) {
+  decode_row(wfmt, w, s, e, N, K, n, out);
+}
+
+/* Bytes of weight codes of one expert (3 matrices of I*H elements) -- Fig. 1(c). */
+int64_t oracle_expert_code_bytes(const oracle_cfg *c) {
+  int64_t el = 3 * (int64_t)c->H * c->I;
+  switch (c->wfmt) {
+    case ORC_W_FP32: return el * 4;
+    case ORC_W_BF16: return el * 2;
+    case ORC_W_FP8E4M3_B128: return el;
+    default: return el / 2;
+  }
+}
+
+/* Bytes of scale factors of one expert. */
+int64_t oracle_expert_scale_bytes(const oracle_cfg *c) {
+  int64_t H = c->H, I = c->I;
+  if (c->wfmt == ORC_W_FP8E4M3_B128) {
+    int64_t hb = (H + 127) / 128, ib = (I + 127) / 128;
+    return 3 * hb * ib * 4;
+  }
+  if (c->wfmt == ORC_W_MXFP4) return 3 * H * I / 32;
+  return 0;
+}
+
+/* ------------------------------------------------------------------ router */
+
+/* logits[t,e] = sum_h x[t,h] * Wr[e,h], summed in index order (Sec. 1: "a
+ * router assigns each token to a small top-k subset of experts"). */
+void oracle_router_logits(const oracle_cfg *c, const void *x, const float *router_w, int32_t gamma,
+                          double *logits) {
+  int64_t H = c->H, E = c->E;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < gamma; ++t)
+    for (int64_t e = 0; e < E; ++e) {
+      double acc = 0.0;
+      for (int64_t h = 0; h < H; ++h)
+        acc += decode_act(x, c->afmt, (size_t)(t * H + h)) * (double)router_w[e * H + h];
+      logits[t * E + e] = acc;
+    }
+}
+
+/* Top-k on the raw logits: order experts by (logit descending, id ascending)
+ * and keep the first k.  Weights over the selected experts:
+ *   softmax: w_j = exp(l_j - l_max) / sum_{j<k} exp(l_j - l_max)
+ *   sigmoid: s_j = 1/(1+exp(-l_j)),  w_j = c * s_j / (sum_j s_j + 1e-20)
+ * gap[t] = l_(k) - l_(k+1) (inf when k == E): the decision margin of token t. */
+void oracle_topk(const oracle_cfg *c, const double *logits, int32_t gamma, int32_t *ids, double *w,
+                 double *gap) {
+  int E = c->E, k = c->top_k;
+  for (int t = 0; t < gamma; ++t) {
+    const double *l = logits + (int64_t)t * E;
+    char *taken = (char *)calloc((size_t)E, 1);
+    for (int j = 0; j < k; ++j) {
+      int best = -1;
+      for (int e = 0; e < E; ++e) {
+        if (taken[e]) continue;
+        if (best < 0 || l[e] > l[best]) best = e; /* strict '>' keeps the lower id on ties */
+      }
+      taken[best] = 1;
+      ids[t * k + j] = best;
+    }
+    if (gap) {
+      int nxt = -1;
+      for (int e = 0; e < E; ++e) {
+        if (taken[e]) continue;
+        if (nxt < 0 || l[e] > l[nxt]) nxt = e;
+      }
+      gap[t] = (nxt < 0) ? INFINITY : l[ids[t * k + k - 1]] - l[nxt];
+    }
+    free(taken);
+    if (c->score == ORC_SCORE_SOFTMAX) {
+      double lmax = l[ids[t * k]], den = 0.0;
+      for (int j = 0; j < k; ++j) den += exp(l[ids[t * k + j]] - lmax);
+      for (int j = 0; j < k; ++j) w[t * k + j] = exp(l[ids[t * k + j]] - lmax) / den;
+    } else {
+      double den = 0.0;
+      for (int j = 0; j < k; ++j) den += 1.0 / (1.0 + exp(-l[ids[t * k + j]]));
+      for (int j = 0; j < k; ++j)
+        w[t * k + j] = c->routed_scale * (1.0 / (1.0 + exp(-l[ids[t * k + j]]))) / (den + 1e-20);
+    }
+  }
+}
+
+/* Eq. 1: the union of the per-token expert sets, and the token->expert
+ * grouping.  union_ids ascending [U]; offsets [U+1] exclusive scan of the
+ * per-expert token counts in that order; perm[A] lists the assignments
+ * a = t*k + j sorted by expert id, ties kept in increasing a (stable);
+ * inv_perm[a] is the position of a in perm.  Returns U. */
+int32_t oracle_union_perm(int32_t E, int32_t k, int32_t gamma, const int32_t *ids,
+                          int32_t *union_ids, int32_t *offsets, int32_t *perm, int32_t *inv_perm) {
+  int A = gamma * k, U = 0, pos = 0;
+  for (int e = 0; e < E; ++e) {
+    int cnt = 0;
+    for (int a = 0; a < A; ++a)
+      if (ids[a] == e) {
+        if (perm) perm[pos] = a;
+        if (inv_perm) inv_perm[a] = pos;
+        ++pos;
+        ++cnt;
+      }
+    if (cnt) {
+      if (union_ids) union_ids[U] = e;
+      if (offsets) offsets[U] = pos - cnt;
+      ++U;
+    }
+  }
+  if (offsets) offsets[U] = pos;
+  return U;
+}
+
+/* --------------------------------------------------------------- expert FFN */
+
+/* Apply expert e (of the tensor set wg/wu/wd with scales sg/su/sd) to m
+ * tokens: xs[m][H] -> out[m][H] with out = Wd * ( silu(Wg x) * (Wu x) ),
+ * silu(z) = z / (1 + exp(-z)).  Each weight row is decoded once. */
+static void expert_ffn(const oracle_cfg *c, const void *wg, const void *wu, const void *wd,
+                       const void *sg, const void *su, const void *sd, int64_t e, int m,
+                       const double *xs, double *out) {
+  int64_t H = c->H, I = c->I;
+  double *hbuf = (double *)malloc(sizeof(double) * (size_t)m * (size_t)I);
+#pragma omp parallel
+  {
+    double *rg = (double *)malloc(sizeof(double) * (size_t)(H > I ? H : I));
+    double *ru = (double *)malloc(sizeof(double) * (size_t)H);
+#pragma omp for schedule(static)
+    for (int64_t i = 0; i < I; ++i) {
+      decode_row(c->wfmt, wg, sg, e, I, H, i, rg);
+      decode_row(c->wfmt, wu, su, e, I, H, i, ru);
+      for (int r = 0; r < m; ++r) {
+        const double *xv = xs + (int64_t)r * H;
+        double g = 0.0, p = 0.0;
+        for (int64_t h = 0; h < H; ++h) g += rg[h] * xv[h];
+        for (int64_t h = 0; h < H; ++h) p += ru[h] * xv[h];
+        hbuf[(int64_t)r * I + i] = g / (1.0 + exp(-g)) * p;
+      }
+    }
+#pragma omp for schedule(static)
+    for (int64_t n = 0; n < H; ++n) {
+      decode_row(c->wfmt, wd, sd, e, H, I, n, rg);
+      for (int r = 0; r < m; ++r) {
+        const double *hv = hbuf + (int64_t)r * I;
+        double o = 0.0;
+        for (int64_t i = 0; i < I; ++i) o += rg[i] * hv[i];
+        out[(int64_t)r * H + n] = o;
+      }
+    }
+    free(rg);
+    free(ru);
+  }
+  free(hbuf);
+}
+
+/* Exposed single-expert FFN on already-decoded double inputs (pins). */
+void oracle_expert_ffn(const oracle_cfg *c, const oracle_layer *L, int32_t shared, int32_t e,
+                       int32_t m, const double *xs, double *out) {
+  if (shared)
+    expert_ffn(c, L->sh_gate, L->sh_up, L->sh_down, L->sh_s_gate, L->sh_s_up, L->sh_s_down, e, m,
+               xs, out);
+  else
+    expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, e, m, xs, out);
+}
+
+/* ------------------------------------------------------------- whole layer */
+
+/* The routed MoE layer over gamma tokens.
+ *   y64[t,:] = sum_j w[t,j] * FFN_{ids[t,j]}(x_t) + sum_s FFN_shared_s(x_t)
+ * evaluated expert by expert over the union (Eq. 1), each expert applied to
+ * all of its tokens at once.  override_w (may be NULL) replaces the router
+ * weights in the combine (used to test linearity in the combine weights).
+ * skip_ffn != 0 stops after routing/grouping (y64 untouched).
+ * Any output pointer may be NULL.  Returns U, or -1 on bad arguments. */
+int32_t oracle_moe_verify(const oracle_cfg *c, const oracle_layer *L, const void *x, int32_t gamma,
+                          const double *override_w, int32_t skip_ffn, double *y64,
+                          int32_t *topk_ids, double *topk_w, int32_t *union_ids, int32_t *offsets,
+                          int32_t *perm, int32_t *inv_perm, double *gap, double *logits_out) {
+  if (!c || !L || !x || gamma < 1 || c->top_k < 1 || c->top_k > c->E) return -1;
+  int64_t H = c->H;
+  int E = c->E, k = c->top_k, A = gamma * k;
+  double *logits = (double *)malloc(sizeof(double) * (size_t)gamma * (size_t)E);
+  int32_t *ids = (int32_t *)malloc(sizeof(int32_t) * (size_t)A);
+  double *w = (double *)malloc(sizeof(double) * (size_t)A);
+  int32_t *uni = (int32_t *)malloc(sizeof(int32_t) * (size_t)E);
+  int32_t *off = (int32_t *)malloc(sizeof(int32_t) * (size_t)(E + 1));
+  int32_t *pm = (int32_t *)malloc(sizeof(int32_t) * (size_t)A);
+  int32_t *ipm = (int32_t *)malloc(sizeof(int32_t) * (size_t)A);
+
+  oracle_router_logits(c, x, L->router_w, gamma, logits);
+  oracle_topk(c, logits, gamma, ids, w, gap);
+  int U = oracle_union_perm(E, k, gamma, ids, uni, off, pm, ipm);
+
+  if (logits_out) memcpy(logits_out, logits, sizeof(double) * (size_t)gamma * (size_t)E);
+  if (topk_ids) memcpy(topk_ids, ids, sizeof(int32_t) * (size_t)A);
+  if (topk_w) memcpy(topk_w, w, sizeof(double) * (size_t)A);
+  if (union_ids) memcpy(union_ids, uni, sizeof(int32_t) * (size_t)U);
+  if (offsets) memcpy(offsets, off, sizeof(int32_t) * (size_t)(U + 1));
+  if (perm) memcpy(perm, pm, sizeof(int32_t) * (size_t)A);
+  if (inv_perm) memcpy(inv_perm, ipm, sizeof(int32_t) * (size_t)A);
+
+  if (!skip_ffn && y64) {
+    const double *cw = override_w ? override_w : w;
+    double *xd = (double *)malloc(sizeof(double) * (size_t)gamma * (size_t)H);
+    for (int64_t i = 0; i < (int64_t)gamma * H; ++i) xd[i] = decode_act(x, c->afmt, (size_t)i);
+    double *xs = (double *)malloc(sizeof(double) * (size_t)gamma * (size_t)H);
+    double *os = (double *)malloc(sizeof(double) * (size_t)gamma * (size_t)H);
+    memset(y64, 0, sizeof(double) * (size_t)gamma * (size_t)H);
+    for (int u = 0; u < U; ++u) {
+      int m = off[u + 1] - off[u];
+      for (int r = 0; r < m; ++r) {
+        int t = pm[off[u] + r] / k;
+        memcpy(xs + (int64_t)r * H, xd + (int64_t)t * H, sizeof(double) * (size_t)H);
+      }
+      expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, uni[u], m, xs,
+                 os);
+      for (int r = 0; r < m; ++r) {
+        int a = pm[off[u] + r], t = a / k;
+        for (int64_t n = 0; n < H; ++n) y64[(int64_t)t * H + n] += cw[a] * os[(int64_t)r * H + n];
+      }
+    }
+    for (int s = 0; s < c->n_shared; ++s) {
+      expert_ffn(c, L->sh_gate, L->sh_up, L->sh_down, L->sh_s_gate, L->sh_s_up, L->sh_s_down, s,
+                 gamma, xd, os);
+      for (int64_t i = 0; i < (int64_t)gamma * H; ++i) y64[i] += os[i];
+    }
+    free(xd);
+    free(xs);
+    free(os);
+  }
+  free(logits);
+  free(ids);
+  free(w);
+  free(uni);
+  free(off);
+  free(pm);
+  free(ipm);
+  return U;
+}
+
+/* Brute-force dense evaluation (tiny inputs only): every one of the E experts
+ * is applied to every token and weighted by the gate g[t,e], which is the
+ * router weight if e is among the token's top-k and 0 otherwise; shared
+ * experts are added with weight 1.  No union, no grouping, no permutation. */
+int32_t oracle_moe_dense(const oracle_cfg *c, const oracle_layer *L, const void *x, int32_t gamma,
+                         double *y64) {
+  if (!c || !L || !x || !y64 || gamma < 1) return -1;
+  int64_t H = c->H;
+  int E = c->E, k = c->top_k;
+  double *logits = (double *)malloc(sizeof(double) * (size_t)gamma * (size_t)E);
+  int32_t *ids = (int32_t *)malloc(sizeof(int32_t) * (size_t)gamma * (size_t)k);
+  double *w = (double *)malloc(sizeof(double) * (size_t)gamma * (size_t)k);
+  double *gate = (double *)calloc((size_t)gamma * (size_t)E, sizeof(double));
+  oracle_router_logits(c, x, L->router_w, gamma, logits);
+  oracle_topk(c, logits, gamma, ids, w, NULL);
+  for (int t = 0; t < gamma; ++t)
+    for (int j = 0; j < k; ++j) gate[(int64_t)t * E + ids[t * k + j]] = w[t * k + j];
+  double *xd = (double *)malloc(sizeof(double) * (size_t)H);
+  double *o = (double *)malloc(sizeof(double) * (size_t)H);
+  memset(y64, 0, sizeof(double) * (size_t)gamma * (size_t)H);
+  for (int t = 0; t < gamma; ++t) {
+    for (int64_t h = 0; h < H; ++h) xd[h] = decode_act(x, c->afmt, (size_t)(t * H + h));
+    for (int e = 0; e < E; ++e) {
+      expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, e, 1, xd, o);
+      for (int64_t n = 0; n < H; ++n) y64[(int64_t)t * H + n] += gate[(int64_t)t * E + e] * o[n];
+    }
+    for (int s = 0; s < c->n_shared; ++s) {
+      expert_ffn(c, L->sh_gate, L->sh_up, L->sh_down, L->sh_s_gate, L->sh_s_up, L->sh_s_down, s, 1,
+                 xd, o);
+      for (int64_t n = 0; n < H; ++n) y64[(int64_t)t * H + n] += o[n];
+    }
+  }
+  free(logits);
+  free(ids);
+  free(w);
+  free(gate);
+  free(xd);
+  free(o);
+  return 0;
+}
+
+int32_t oracle_num_threads(void) {
+#ifdef _OPENMP
+  return (int32_t)omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
