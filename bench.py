@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE verification layer (one "step" = one moev_verify call: router
+top-k -> expert union/grouping -> grouped SwiGLU expert FFN -> weighted combine).
+
+Default workload: the DeepSeek-V3.1-shaped FP8 layer at gamma = 64 with scattered routing
+(H=7168, I=2048, 256 routed + 1 shared expert, top-8 sigmoid), four distinct layers' weights
+(45 GB) rotated call by call so no weight byte can be an L2 hit.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload NAME] [--sweep]
+
+N > 1 (under torchrun) runs N independent replicas, one per GPU (the path has no exchange
+step); value is the aggregate over replicas, time the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import synth  # noqa: E402
+
+METRIC = "moe_verify_expert_weight_bandwidth"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+
+# workload name -> (shape, gamma, routing, kwargs)
+WORKLOADS = {
+    "deepseek_fp8_g64_scattered": ("deepseek", 64, "scattered", {}),
+    "deepseek_fp8_g64_clustered": ("deepseek", 64, "clustered", {}),
+    "qwen_bf16_g16": ("qwen", 16, "iid", {}),
+    "qwen_bf16_g32": ("qwen", 32, "iid", {}),
+    "qwen_bf16_g64": ("qwen", 64, "iid", {}),
+    "gptoss_mxfp4_g8": ("gptoss", 8, "iid", {}),
+    "gptoss_mxfp4_g16": ("gptoss", 16, "iid", {}),
+    "gptoss_mxfp4_g32": ("gptoss", 32, "iid", {}),
+    "gptoss_mxfp4_g64": ("gptoss", 64, "iid", {}),
+    "tiny_fp32_g8": ("tiny", 8, "iid", {}),
+}
+DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
+
+# DRAM bytes per launch of the dominant kernel from the committed ncu captures
+# (profiles/*.md), keyed by (workload, impl name); absent = not captured.
+NCU_TRAFFIC_BYTES: dict = {}
+
+ROUTING = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
+           "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+                mask = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def start(self):
+        if self.nv:
+            self._thr = threading.Thread(target=self._run, daemon=True)
+            self._thr.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def build_workload(name: str, n_layers: int, device, rank: int = 0):
+    base, gamma, routing, kw = WORKLOADS[name]
+    shape = synth.SHAPES[base]
+    layers = []
+    for l in range(n_layers):
+        lid = rank * 1000 + l
+        w = synth.make_expert_weights(shape, layer=lid, device=device)
+        wr, x = ROUTING[routing](shape, gamma, layer=lid, device=device, **kw)
+        layers.append({"weights": w, "router_w": wr, "x": x})
+    return shape, gamma, layers
+
+
+def layers_that_fit(shape: synth.Shape, want: int = 4) -> int:
+    per_layer = (shape.E + shape.n_shared) * shape.bytes_per_expert()
+    free, _ = torch.cuda.mem_get_info()
+    return max(1, min(want, int((free * 0.85) // per_layer)))
+
+
+def ocfg_of(shape):
+    import oracle
+    return oracle.Config(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, shape.wfmt,
+                         shape.afmt, shape.score, shape.routed_scale)
+
+
+def time_oracle_sample(shape, layer, gamma_sample: int, repeats: int = 1):
+    """The CPU oracle, as it stands, on the first gamma_sample tokens of one layer's input
+    with that layer's full weights.  Returns (GB/s of expert-weight bytes, seconds, U, cores)."""
+    import oracle
+    host = synth.layer_to_numpy(layer["router_w"], layer["weights"])
+    xs = synth.to_numpy(layer["x"][:gamma_sample].contiguous())
+    best, U = None, 0
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        res = oracle.moe_verify(ocfg_of(shape), host, xs, gamma_sample)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+        U = res.n_active
+    nbytes = (U + shape.n_shared) * shape.bytes_per_expert()
+    return nbytes / best / 1e9, best, U, oracle.num_threads()
+
+
+def run_reference(args):
+    """--impl reference: the oracle on the host cores, on a bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    base, gamma, routing, kw = WORKLOADS[args.workload]
+    shape = synth.SHAPES[base]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    shape_, gamma, layers = build_workload(args.workload, 1, dev)
+    import oracle
+    host = synth.layer_to_numpy(layers[0]["router_w"], layers[0]["weights"])
+    gs = 1  # one token per step: k routed experts + shared
+    cfg = ocfg_of(shape)
+    steps, warm = max(1, min(args.steps, 5)), max(0, min(args.warmup, 1))
+    tot_b, tot_t = 0, 0.0
+    for i in range(warm + steps):
+        xs = synth.to_numpy(layers[0]["x"][i % gamma:i % gamma + gs].contiguous())
+        t0 = time.perf_counter()
+        res = oracle.moe_verify(cfg, host, xs, gs)
+        dt = time.perf_counter() - t0
+        if i >= warm:
+            tot_t += dt
+            tot_b += (res.n_active + shape.n_shared) * shape.bytes_per_expert()
+    val = tot_b / tot_t / 1e9
+    sample = f"{gs} token(s) of the workload per step, full layer weights, {steps} steps"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warm, "ms_per_step": 1e3 * tot_t / steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": args.workload, "gamma": gamma},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(),
+                             "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import paper_2607_12696_b200 as moev
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    base = WORKLOADS[args.workload][0]
+    shape = synth.SHAPES[base]
+    n_layers = layers_that_fit(shape, args.layers)
+    shape, gamma, layers = build_workload(args.workload, n_layers, dev, rank)
+    impl = {"auto": moev.IMPL_AUTO, "simt": moev.IMPL_SIMT, "tcgen05": moev.IMPL_TCGEN05}[args.kernels]
+    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, gamma, shape.wfmt,
+                          shape.afmt, shape.score, impl, shape.routed_scale)
+    v = moev.MoeVerifier(cfg)
+    packed = []
+    for L in layers:
+        d = {"router_w": L["router_w"]}
+        d.update({k: t for k, t in L["weights"].items() if t is not None})
+        packed.append((moev.binding.make_layer(d), d))
+    outs = [v.alloc_out(gamma, diagnostics=False) for _ in layers]
+    Wb = moev.expert_bytes(cfg)
+
+    def step(i):
+        l = i % n_layers
+        v.verify(packed[l][0], layers[l]["x"], gamma, outs[l])
+
+    for i in range(args.warmup):
+        step(i)
+    v.status_sync()
+    U = [int(o["n_active"].item()) for o in outs]
+    if args.warmup < n_layers:  # make sure every layer's U is known
+        for l in range(n_layers):
+            step(l)
+        torch.cuda.synchronize()
+        U = [int(o["n_active"].item()) for o in outs]
+    bytes_step = [(u + shape.n_shared) * Wb for u in U]
+
+    def barrier():
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing
+    v.profile_enable(True)
+    sampler = ClockSampler(local)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    sampler.start()
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    kern_us, kern_calls = v.profile_read()
+    v.profile_enable(False)
+    v.status_sync()
+    tot_bytes = sum(bytes_step[i % n_layers] for i in range(args.steps))
+
+    # ---- end to end through the host-buffer entry point
+    xh = [L["x"].cpu().pin_memory() for L in layers]
+    yh = [torch.empty_like(t).pin_memory() for t in xh]
+    nh = torch.zeros(1, dtype=torch.int32).pin_memory()
+    for i in range(min(3, args.warmup)):
+        v.verify_host(packed[i % n_layers][0], xh[i % n_layers], gamma, yh[i % n_layers], nh)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        l = i % n_layers
+        v.verify_host(packed[l][0], xh[l], gamma, yh[l], nh)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    act_b = 4 if shape.afmt == synth.ACT_FP32 else 2
+    h2d, d2h = gamma * shape.H * act_b, gamma * shape.H * act_b + 4
+
+    # ---- aggregate over replicas: max time, summed bytes
+    if dist:
+        t = torch.tensor([ms_total, e2e_s * 1e3], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        b = torch.tensor([float(tot_bytes)], device=dev, dtype=torch.float64)
+        dist.all_reduce(b, op=dist.ReduceOp.SUM)
+        ms_total, e2e_ms, all_bytes = float(t[0]), float(t[1]), float(b[0])
+    else:
+        e2e_ms, all_bytes = e2e_s * 1e3, float(tot_bytes)
+
+    if rank == 0:
+        value = all_bytes / (ms_total * 1e-3) / 1e9
+        peak, peak_src = measured_peaks()
+        impl_name = {1: "simt", 2: "tcgen05"}[v.resolved_impl()]
+        mean_bytes = tot_bytes / args.steps
+        if impl_name == "simt":  # two kernels; the first (gate/up) streams 2/3 of the bytes
+            k_name, k_bytes, k_us = "ffn_gateup_simt", mean_bytes * 2.0 / 3.0, kern_us[0]
+        else:
+            k_name, k_bytes, k_us = "grouped_ffn_tcgen05", mean_bytes, kern_us[0]
+        achieved = k_bytes / (k_us * 1e-6) / 1e9 if k_us > 0 else None
+        cpu = None
+        if not args.no_cpu_baseline:
+            cv, cs, cu, cores = time_oracle_sample(shape, layers[0], args.cpu_tokens)
+            cpu = {"value": cv, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"first {args.cpu_tokens} of the {gamma} tokens of layer 0 (U={cu}"
+                             f"+{shape.n_shared} experts streamed), full layer weights, {cs:.2f} s"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "mxfp4"}[shape.wfmt],
+            "data": "synthetic",
+            "config": {"workload": args.workload, "gamma": gamma, "H": shape.H, "I": shape.I,
+                       "E": shape.E, "top_k": shape.top_k, "n_shared": shape.n_shared,
+                       "unique_experts_per_layer": U, "layers_rotated": n_layers,
+                       "l2_policy": "weights of %d layers (%.1f GB) rotated per call, > L2" % (
+                           n_layers, n_layers * (shape.E + shape.n_shared) * Wb / 1e9),
+                       "bytes_per_expert": Wb, "kernels": impl_name, "parallelism": "replicas"},
+            "latency_us": 1e3 * ms_total / args.steps,
+            "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": (achieved / peak) if achieved else None,
+                         "traffic": NCU_TRAFFIC_BYTES.get((args.workload, impl_name)),
+                         "kernel": k_name, "kernel_us": k_us, "kernel_bytes": k_bytes,
+                         "second_kernel_us": kern_us[1], "launches_timed": kern_calls,
+                         "peak_source": peak_src + " (of %s)" % peak_src},
+            "cpu_baseline": cpu,
+            "e2e": {"value": all_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": e2e_ms / args.steps,
+                    "note": "host x -> device, layer, y + n_active -> host each step; expert "
+                            "weights are layer parameters and stay resident"},
+            "gpu_launches": v.launches_per_call() * args.steps,
+            "clocks": clocks,
+        }
+        print(json.dumps(line))
+    v.close()
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--layers", type=int, default=4)
+    ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tcgen05"])
+    ap.add_argument("--cpu-tokens", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

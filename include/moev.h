@@ -1,0 +1,186 @@
+/*
+ * moev.h -- C ABI of the B200 (sm_100a) MoE verification layer.
+ *
+ * One call, moev_verify(), runs the MoE expert layer of the target model's
+ * verification pass over the gamma tokens of a speculative draft tree:
+ *
+ *   router top-k per token  ->  expert union + token->expert grouping
+ *   ->  grouped gated-SwiGLU expert FFN over the union, each active expert's
+ *       weights read from HBM once  ->  routing-weighted combine,
+ *
+ * and reports the per-layer active-expert count.
+ *
+ * Paper passages the operations follow:
+ *   - Sec. 1: "a router assigns each token to a small top-k subset of experts".
+ *   - Eq. 1 (Sec. 3): the verification footprint is the union over the gamma
+ *     verified tokens of their expert sets; its size -- not gamma -- drives the
+ *     cost, because the verifier fetches every expert of the union from HBM and
+ *     reuses it for all tokens routed to it.
+ *   - Table 1 / Table 3 metric "average active experts": the size of that union
+ *     per MoE layer per verification step (n_active here; shared experts are not
+ *     counted, as the autoregressive rows of Table 1 show).
+ *   - Table 13: experts per layer, top-k and the always-on shared expert.
+ *   - Fig. 1(c): bytes of one expert (moev_expert_bytes).
+ * The paper does not print the expert FFN; it is the bias-free gated SwiGLU
+ *   FFN_e(x) = W_down,e ( silu(W_gate,e x) * (W_up,e x) ),  silu(z) = z/(1+exp(-z)),
+ *   y_t = sum_j w[t,j] FFN_{ids[t,j]}(x_t) + sum_s FFN_shared,s(x_t).
+ *
+ * Conventions
+ *   - No exceptions, aborts or traps cross this boundary: every entry point
+ *     returns a moev_status; moev_last_error() gives the text of the last failure.
+ *   - Unless a parameter says HOST, pointers are DEVICE pointers, borrowed for the
+ *     duration of the call; the library never frees or retains caller memory.
+ *   - moev_verify() is asynchronous on the given CUDA stream, allocates nothing
+ *     and never synchronises; outputs are valid once the stream reaches that point.
+ *   - One context per host thread / stream (calls on one context must not overlap).
+ */
+#ifndef MOEV_H_
+#define MOEV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moev_ctx moev_ctx; /* opaque; owns the device workspace */
+
+typedef enum {
+  MOEV_OK = 0,
+  MOEV_EINVAL = 1,       /* bad argument (null, out of range, misaligned, shape granularity) */
+  MOEV_EUNSUPPORTED = 2, /* device is not sm_100 */
+  MOEV_ECUDA = 3,        /* a CUDA runtime/driver call failed; see moev_last_error */
+  MOEV_ENOMEM = 4,       /* workspace allocation failed in moev_create */
+  MOEV_ETIMEOUT = 5      /* a bounded device-side wait expired (reported by moev_status_sync) */
+} moev_status;
+
+/* Expert-weight storage formats (K = contraction dimension, always contiguous). */
+typedef enum {
+  MOEV_W_FP32 = 0,         /* float32 */
+  MOEV_W_BF16 = 1,         /* bfloat16 */
+  MOEV_W_FP8E4M3_B128 = 2, /* e4m3fn codes + float32 scale per 128x128 block: W = code * s */
+  MOEV_W_MXFP4 = 3         /* e2m1 codes, two per byte (even k in the low nibble) + e8m0
+                              scale per 32 along K: W = code * 2^(s-127) */
+} moev_wfmt;
+
+typedef enum { MOEV_ACT_FP32 = 0, MOEV_ACT_BF16 = 1 } moev_afmt;
+
+/* Router weights over the k selected experts (selection itself is always on raw logits,
+ * descending, exact ties to the lower expert id):
+ *   SOFTMAX: w_j = exp(l_j - l_max) / sum_{j<k} exp(l_j - l_max)
+ *   SIGMOID: s_j = 1/(1+exp(-l_j)),  w_j = routed_scale * s_j / (sum_j s_j + 1e-20)      */
+typedef enum { MOEV_SCORE_SOFTMAX = 0, MOEV_SCORE_SIGMOID = 1 } moev_score;
+
+/* Which expert-FFN kernels moev_verify uses. */
+typedef enum {
+  MOEV_IMPL_AUTO = 0,   /* tensor-core (TMA + tcgen05) path when the shape allows, else SIMT */
+  MOEV_IMPL_SIMT = 1,   /* CUDA-core kernels (all formats, all shapes) */
+  MOEV_IMPL_TCGEN05 = 2 /* tensor-core path; MOEV_EINVAL if the shape does not allow it */
+} moev_impl;
+
+typedef struct {
+  int32_t H;          /* hidden size; multiple of 32 */
+  int32_t I;          /* expert intermediate size; multiple of 32 */
+  int32_t E;          /* routed experts, 1..512 */
+  int32_t top_k;      /* 1..min(E,32) */
+  int32_t n_shared;   /* always-on shared experts (weight 1), >= 0 */
+  int32_t max_tokens; /* largest gamma this context will be asked to verify, 1..1024 */
+  int32_t wfmt;       /* moev_wfmt */
+  int32_t afmt;       /* moev_afmt: type of x and y */
+  int32_t score;      /* moev_score */
+  int32_t impl;       /* moev_impl */
+  float routed_scale; /* c in the SIGMOID rule; ignored for SOFTMAX */
+} moev_config;
+
+/* One layer's parameters.  Layouts, row-major, last index contiguous:
+ *   router_w            [E, H]  float32
+ *   w_gate, w_up        [E, I, H]   in wfmt     (K = H)
+ *   w_down              [E, H, I]   in wfmt     (K = I)
+ *   s_*   FP8 : float32 [E, ceil(N/128), ceil(K/128)]   (N = rows of the matrix)
+ *         MXFP4: uint8  [E, N, K/32]                     else NULL
+ *   sh_*  the same for the n_shared shared experts (leading dim n_shared), NULL if none.
+ * Every pointer must be 16-byte aligned. */
+typedef struct {
+  const float* router_w;
+  const void *w_gate, *w_up, *w_down;
+  const void *s_gate, *s_up, *s_down;
+  const void *sh_gate, *sh_up, *sh_down;
+  const void *sh_s_gate, *sh_s_up, *sh_s_down;
+} moev_layer;
+
+/* Outputs.  y and n_active are required; the others are diagnostics and may be NULL.
+ *   y          [gamma, H] in afmt
+ *   topk_ids   [gamma, k] int32   expert ids in descending-logit order
+ *   topk_w     [gamma, k] float32 router weights
+ *   union_ids  [E]        int32   first U entries: active experts, ascending (Eq. 1)
+ *   offsets    [E+1]      int32   first U+1 entries: exclusive scan of tokens per active expert
+ *   perm       [gamma*k]  int32   assignments a = t*k+j stably sorted by expert id
+ *   n_active   [1]        int32   U = size of the union (shared experts not counted)       */
+typedef struct {
+  void* y;
+  int32_t* topk_ids;
+  float* topk_w;
+  int32_t* union_ids;
+  int32_t* offsets;
+  int32_t* perm;
+  int32_t* n_active;
+} moev_out;
+
+/* Create a context for one layer shape on the current CUDA device; allocates the device
+ * workspace (router logits, grouping tables, fp32 intermediates).  MOEV_EINVAL on a bad
+ * config, MOEV_EUNSUPPORTED when the device is not compute capability 10.x, MOEV_ENOMEM /
+ * MOEV_ECUDA on allocation failure.  *out is NULL on failure. */
+moev_status moev_create(const moev_config* cfg, moev_ctx** out);
+
+/* Free the workspace.  The caller must have synchronised the streams it used. */
+moev_status moev_destroy(moev_ctx* ctx);
+
+/* Verify gamma tokens (1 <= gamma <= max_tokens): x [gamma, H] in afmt (device).
+ * Enqueues the whole path on cuda_stream (a cudaStream_t, may be NULL for the default
+ * stream) and returns without waiting.  Invalid arguments are rejected with MOEV_EINVAL
+ * before anything is launched. */
+moev_status moev_verify(moev_ctx* ctx, const moev_layer* layer, const void* x, int32_t gamma,
+                        const moev_out* out, void* cuda_stream);
+
+/* The same path for callers whose activations live in HOST memory: x_host [gamma, H]
+ * (pinned memory recommended) is copied to the device, the layer runs, and y_host
+ * [gamma, H] plus *n_active_host are copied back, all on cuda_stream; the call waits for
+ * the stream before returning so the host buffers are valid.  Weights stay on the device. */
+moev_status moev_verify_host(moev_ctx* ctx, const moev_layer* layer, const void* x_host,
+                             int32_t gamma, void* y_host, int32_t* n_active_host,
+                             void* cuda_stream);
+
+/* Wait for cuda_stream and read the device status word: MOEV_OK, or MOEV_ETIMEOUT if a
+ * bounded device-side wait gave up (the outputs of that call are then undefined). */
+moev_status moev_status_sync(moev_ctx* ctx, void* cuda_stream);
+
+/* Text of the last error on this context ("" if none).  Owned by the context. */
+const char* moev_last_error(const moev_ctx* ctx);
+
+/* Bytes of one expert's three matrices including scale factors (Fig. 1(c): the FP8
+ * DeepSeek-V3.1 expert is 3*7168*2048 = 44 040 192 code bytes, + 10 752 scale bytes). */
+size_t moev_expert_bytes(const moev_config* cfg);
+
+/* Code bytes only (the paper's 44.04 MB figure). */
+size_t moev_expert_code_bytes(const moev_config* cfg);
+
+/* Number of kernels one moev_verify call launches on this context (for launch accounting),
+ * and which FFN implementation it resolved to (a moev_impl value, never AUTO). */
+int32_t moev_launches_per_call(const moev_ctx* ctx);
+int32_t moev_resolved_impl(const moev_ctx* ctx);
+
+/* Device time of the expert-FFN kernels (the weight-streaming part of the call), measured
+ * with CUDA events recorded on the call's stream.  moev_profile_enable(ctx, 1) turns the
+ * event records on (at most 512 calls are kept between reads), 0 off.  moev_profile_read
+ * waits for the stream, writes mean_us[0..1] -- the mean duration in microseconds of the
+ * first and of the second FFN kernel of a call (the SIMT path has two: gate/up and down; a
+ * fused path reports 0 for the second) -- and the number of calls averaged, then resets. */
+moev_status moev_profile_enable(moev_ctx* ctx, int32_t on);
+moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[2]*/,
+                              int32_t* calls);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOEV_H_ */

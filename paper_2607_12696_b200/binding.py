@@ -1,0 +1,218 @@
+"""ctypes binding with the same names as the C ABI (see include/moev.h)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmoev.so")
+
+W_FP32, W_BF16, W_FP8E4M3_B128, W_MXFP4 = 0, 1, 2, 3
+ACT_FP32, ACT_BF16 = 0, 1
+SCORE_SOFTMAX, SCORE_SIGMOID = 0, 1
+IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
+STATUS = {0: "MOEV_OK", 1: "MOEV_EINVAL", 2: "MOEV_EUNSUPPORTED", 3: "MOEV_ECUDA",
+          4: "MOEV_ENOMEM", 5: "MOEV_ETIMEOUT"}
+
+EXPORTS = ("moev_create", "moev_destroy", "moev_verify", "moev_verify_host", "moev_status_sync",
+           "moev_last_error", "moev_expert_bytes", "moev_expert_code_bytes",
+           "moev_launches_per_call", "moev_resolved_impl", "moev_profile_enable",
+           "moev_profile_read")
+
+
+class MoevError(RuntimeError):
+    def __init__(self, status: int, text: str = ""):
+        self.status = status
+        super().__init__(f"{STATUS.get(status, status)}: {text}")
+
+
+class _Config(C.Structure):
+    _fields_ = [("H", C.c_int32), ("I", C.c_int32), ("E", C.c_int32), ("top_k", C.c_int32),
+                ("n_shared", C.c_int32), ("max_tokens", C.c_int32), ("wfmt", C.c_int32),
+                ("afmt", C.c_int32), ("score", C.c_int32), ("impl", C.c_int32),
+                ("routed_scale", C.c_float)]
+
+
+_LAYER_FIELDS = ("router_w", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down",
+                 "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down")
+_OUT_FIELDS = ("y", "topk_ids", "topk_w", "union_ids", "offsets", "perm", "n_active")
+
+
+class _Layer(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _LAYER_FIELDS]
+
+
+class _Out(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in _OUT_FIELDS]
+
+
+@dataclass
+class MoevConfig:
+    H: int
+    I: int
+    E: int
+    top_k: int
+    n_shared: int = 0
+    max_tokens: int = 128
+    wfmt: int = W_BF16
+    afmt: int = ACT_BF16
+    score: int = SCORE_SOFTMAX
+    impl: int = IMPL_AUTO
+    routed_scale: float = 1.0
+
+    def c(self) -> _Config:
+        return _Config(self.H, self.I, self.E, self.top_k, self.n_shared, self.max_tokens,
+                       self.wfmt, self.afmt, self.score, self.impl, self.routed_scale)
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _LIB_PATH
+
+
+def lib() -> C.CDLL:
+    """Load libmoev.so; raises (never falls back) when it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError(f"{_LIB_PATH} not found: build it with "
+                              "`python -m paper_2607_12696_b200.build` (there is no CPU fallback)")
+        L = C.CDLL(_LIB_PATH)
+        L.moev_create.restype = C.c_int
+        L.moev_create.argtypes = [C.POINTER(_Config), C.POINTER(C.c_void_p)]
+        L.moev_destroy.restype = C.c_int
+        L.moev_destroy.argtypes = [C.c_void_p]
+        L.moev_verify.restype = C.c_int
+        L.moev_verify.argtypes = [C.c_void_p, C.POINTER(_Layer), C.c_void_p, C.c_int32,
+                                  C.POINTER(_Out), C.c_void_p]
+        L.moev_verify_host.restype = C.c_int
+        L.moev_verify_host.argtypes = [C.c_void_p, C.POINTER(_Layer), C.c_void_p, C.c_int32,
+                                       C.c_void_p, C.c_void_p, C.c_void_p]
+        L.moev_status_sync.restype = C.c_int
+        L.moev_status_sync.argtypes = [C.c_void_p, C.c_void_p]
+        L.moev_last_error.restype = C.c_char_p
+        L.moev_last_error.argtypes = [C.c_void_p]
+        L.moev_expert_bytes.restype = C.c_size_t
+        L.moev_expert_bytes.argtypes = [C.POINTER(_Config)]
+        L.moev_expert_code_bytes.restype = C.c_size_t
+        L.moev_expert_code_bytes.argtypes = [C.POINTER(_Config)]
+        L.moev_launches_per_call.restype = C.c_int32
+        L.moev_launches_per_call.argtypes = [C.c_void_p]
+        L.moev_resolved_impl.restype = C.c_int32
+        L.moev_resolved_impl.argtypes = [C.c_void_p]
+        L.moev_profile_enable.restype = C.c_int
+        L.moev_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.moev_profile_read.restype = C.c_int
+        L.moev_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_double),
+                                        C.POINTER(C.c_int32)]
+        _lib = L
+    return _lib
+
+
+def expert_bytes(cfg: MoevConfig) -> int:
+    c = cfg.c()
+    return lib().moev_expert_bytes(C.byref(c))
+
+
+def expert_code_bytes(cfg: MoevConfig) -> int:
+    c = cfg.c()
+    return lib().moev_expert_code_bytes(C.byref(c))
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def make_layer(tensors: dict) -> _Layer:
+    """Pack device tensors (keys = moev_layer field names; missing/None = NULL)."""
+    L = _Layer()
+    for n in _LAYER_FIELDS:
+        t = tensors.get(n)
+        if t is not None:
+            assert t.is_cuda and t.is_contiguous(), f"{n} must be a contiguous CUDA tensor"
+        setattr(L, n, _ptr(t))
+    return L
+
+
+class MoeVerifier:
+    """Owns one ``moev_ctx``.  ``verify`` enqueues on torch's current stream."""
+
+    def __init__(self, cfg: MoevConfig):
+        self.cfg = cfg
+        self._h = C.c_void_p()
+        c = cfg.c()
+        st = lib().moev_create(C.byref(c), C.byref(self._h))
+        if st != 0:
+            self._h = None
+            raise MoevError(st, "moev_create failed")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().moev_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int):
+        if st != 0:
+            raise MoevError(st, lib().moev_last_error(self._h).decode())
+
+    @staticmethod
+    def _stream():
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    def alloc_out(self, gamma: int, diagnostics: bool = True) -> dict:
+        cfg, dev = self.cfg, "cuda"
+        out = {"y": torch.empty(gamma, cfg.H, device=dev,
+                                dtype=torch.float32 if cfg.afmt == ACT_FP32 else torch.bfloat16),
+               "n_active": torch.zeros(1, dtype=torch.int32, device=dev)}
+        if diagnostics:
+            out.update(topk_ids=torch.full((gamma, cfg.top_k), -1, dtype=torch.int32, device=dev),
+                       topk_w=torch.zeros(gamma, cfg.top_k, dtype=torch.float32, device=dev),
+                       union_ids=torch.full((cfg.E,), -1, dtype=torch.int32, device=dev),
+                       offsets=torch.full((cfg.E + 1,), -1, dtype=torch.int32, device=dev),
+                       perm=torch.full((gamma * cfg.top_k,), -1, dtype=torch.int32, device=dev))
+        return out
+
+    def verify(self, layer: _Layer, x: torch.Tensor, gamma: int, out: dict):
+        """moev_verify: asynchronous on the current stream; ``out`` maps moev_out fields to tensors."""
+        O = _Out()
+        for n in _OUT_FIELDS:
+            setattr(O, n, _ptr(out.get(n)))
+        self._check(lib().moev_verify(self._h, C.byref(layer), _ptr(x), gamma, C.byref(O),
+                                      self._stream()))
+
+    def verify_host(self, layer: _Layer, x_host: torch.Tensor, gamma: int, y_host: torch.Tensor,
+                    n_active_host: torch.Tensor):
+        """moev_verify_host: host x in, host y / n_active out (synchronous)."""
+        assert not x_host.is_cuda and not y_host.is_cuda and not n_active_host.is_cuda
+        self._check(lib().moev_verify_host(self._h, C.byref(layer), x_host.data_ptr(), gamma,
+                                           y_host.data_ptr(), n_active_host.data_ptr(),
+                                           self._stream()))
+
+    def status_sync(self):
+        self._check(lib().moev_status_sync(self._h, self._stream()))
+
+    def launches_per_call(self) -> int:
+        return lib().moev_launches_per_call(self._h)
+
+    def resolved_impl(self) -> int:
+        return lib().moev_resolved_impl(self._h)
+
+    def profile_enable(self, on: bool):
+        self._check(lib().moev_profile_enable(self._h, int(on)))
+
+    def profile_read(self):
+        us = (C.c_double * 2)()
+        n = C.c_int32()
+        self._check(lib().moev_profile_read(self._h, self._stream(), us, C.byref(n)))
+        return [us[0], us[1]], n.value

@@ -1,0 +1,79 @@
+// Shared device helpers for the MoE verification kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_fp4.h>
+#include <cuda_fp8.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/moev.h"
+
+namespace moev {
+
+constexpr int kMaxE = 512;       // routed experts per layer
+constexpr int kMaxTopK = 32;     // one lane per selected expert
+constexpr int kStatusOk = 0;
+constexpr int kStatusTimeout = 1;
+
+// Device-side tables produced by the routing kernels and consumed by the FFN kernels.
+// slot = position in expert-sorted assignment order (0..A), then shared-expert slots
+// A + s*gamma + t.  All pointers live in the context workspace.
+struct Tables {
+  double* logits;      // [gamma, E]
+  int32_t* topk_ids;   // [gamma, k]
+  float* topk_w;       // [gamma, k]
+  int32_t* union_ids;  // [E]
+  int32_t* offsets;    // [E+1]
+  int32_t* perm;       // [A]
+  int32_t* slot_token; // [A]   token index of the assignment in this slot
+  float* slot_w;       // [A]   its routing weight
+  int32_t* n_active;   // [1]
+  int32_t* status;     // [1]   kStatusOk / kStatusTimeout
+};
+
+struct LayerPtrs {
+  const void *w_gate, *w_up, *w_down;
+  const void *s_gate, *s_up, *s_down;
+  const void *sh_gate, *sh_up, *sh_down;
+  const void *sh_s_gate, *sh_s_up, *sh_s_down;
+};
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// e8m0 scale byte -> float 2^(b-127)  (b = 0 is the subnormal 2^-127)
+__device__ __forceinline__ float e8m0_to_float(uint32_t b) {
+  return __uint_as_float(b == 0 ? 0x00400000u : (b << 23));
+}
+
+// Load 8 consecutive activations x[idx .. idx+8) as floats (idx multiple of 8).
+template <int AFMT>
+__device__ __forceinline__ void load_act8(const void* x, size_t idx, float (&v)[8]) {
+  if (AFMT == MOEV_ACT_FP32) {
+    const float4* p = reinterpret_cast<const float4*>(static_cast<const float*>(x) + idx);
+    float4 a = __ldg(p), b = __ldg(p + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  } else {
+    uint4 q = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(x) + idx));
+    uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+}
+
+}  // namespace moev

@@ -1,0 +1,322 @@
+// Host side of the C ABI declared in include/moev.h: context, validation, launches.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+#include "ffn_simt.cuh"
+#include "router.cuh"
+
+using namespace moev;
+
+namespace {
+constexpr int kProfSlots = 512;
+}
+
+struct moev_ctx {
+  moev_config cfg;
+  int device = -1;
+  int resolved_impl = MOEV_IMPL_SIMT;
+  Tables T{};
+  float* hbuf = nullptr;  // [(max_tokens*k + n_shared*max_tokens), I] fp32
+  float* y32 = nullptr;   // [max_tokens, H] fp32 combine accumulator
+  void* x_stage = nullptr;  // device staging for moev_verify_host
+  void* y_stage = nullptr;
+  int32_t* host_word = nullptr;  // pinned scratch for status / n_active reads
+  bool profile = false;
+  cudaEvent_t ev[kProfSlots][3];
+  int prof_n = 0;
+  bool prof_events_ready = false;
+  char err[512] = {0};
+};
+
+namespace {
+
+moev_status fail(moev_ctx* c, moev_status st, const char* fmt, ...) {
+  if (c) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(c->err, sizeof(c->err), fmt, ap);
+    va_end(ap);
+  }
+  return st;
+}
+
+bool cfg_ok(const moev_config* c, char* why, size_t n) {
+#define BAD(cond, msg) if (cond) { snprintf(why, n, "%s", msg); return false; }
+  BAD(!c, "config is null");
+  BAD(c->H < 32 || c->H % 32, "H must be a positive multiple of 32");
+  BAD(c->I < 32 || c->I % 32, "I must be a positive multiple of 32");
+  BAD(c->E < 1 || c->E > kMaxE, "E must be in 1..512");
+  BAD(c->top_k < 1 || c->top_k > c->E || c->top_k > kMaxTopK, "top_k must be in 1..min(E,32)");
+  BAD(c->n_shared < 0 || c->n_shared > 64, "n_shared must be in 0..64");
+  BAD(c->max_tokens < 1 || c->max_tokens > 1024, "max_tokens must be in 1..1024");
+  BAD((long long)c->max_tokens * c->top_k > 8192, "max_tokens * top_k must be <= 8192");
+  BAD(c->wfmt < 0 || c->wfmt > MOEV_W_MXFP4, "unknown weight format");
+  BAD(c->afmt < 0 || c->afmt > MOEV_ACT_BF16, "unknown activation format");
+  BAD(c->score < 0 || c->score > MOEV_SCORE_SIGMOID, "unknown score function");
+  BAD(c->impl < 0 || c->impl > MOEV_IMPL_TCGEN05, "unknown impl");
+  BAD((size_t)c->H * 4 > 200 * 1024, "H too large for the router kernel's shared memory");
+#undef BAD
+  return true;
+}
+
+size_t code_bytes(const moev_config* c) {
+  size_t el = 3 * (size_t)c->H * c->I;
+  switch (c->wfmt) {
+    case MOEV_W_FP32: return el * 4;
+    case MOEV_W_BF16: return el * 2;
+    case MOEV_W_FP8E4M3_B128: return el;
+    default: return el / 2;
+  }
+}
+size_t scale_bytes(const moev_config* c) {
+  size_t H = c->H, I = c->I;
+  if (c->wfmt == MOEV_W_FP8E4M3_B128) return 3 * ((H + 127) / 128) * ((I + 127) / 128) * 4;
+  if (c->wfmt == MOEV_W_MXFP4) return 3 * H * I / 32;
+  return 0;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+cudaError_t dmalloc(T** p, size_t count) {
+  return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+}
+
+size_t route_smem(const moev_config& c, int gamma) {
+  return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4;
+}
+
+template <int WFMT, int AFMT>
+void launch_simt_ffn(moev_ctx* c, const LayerPtrs& L, const void* x, int gamma, cudaStream_t st,
+                     cudaEvent_t* ev) {
+  const moev_config& g = c->cfg;
+  const int rows = 64;
+  dim3 g1(g.E + g.n_shared, (g.I + rows - 1) / rows), g2(g.E + g.n_shared, (g.H + rows - 1) / rows);
+  if (ev) cudaEventRecord(ev[0], st);
+  ffn_gateup_simt<WFMT, AFMT><<<g1, 256, 0, st>>>(L, c->T, x, c->hbuf, gamma, g.H, g.I, g.top_k,
+                                                   g.n_shared, rows);
+  if (ev) cudaEventRecord(ev[1], st);
+  ffn_down_simt<WFMT><<<g2, 256, 0, st>>>(L, c->T, c->hbuf, c->y32, gamma, g.H, g.I, g.top_k,
+                                           g.n_shared, rows);
+  if (ev) cudaEventRecord(ev[2], st);
+}
+
+template <int AFMT>
+void launch_simt_ffn_w(moev_ctx* c, const LayerPtrs& L, const void* x, int gamma, cudaStream_t st,
+                       cudaEvent_t* ev) {
+  switch (c->cfg.wfmt) {
+    case MOEV_W_FP32: launch_simt_ffn<MOEV_W_FP32, AFMT>(c, L, x, gamma, st, ev); break;
+    case MOEV_W_BF16: launch_simt_ffn<MOEV_W_BF16, AFMT>(c, L, x, gamma, st, ev); break;
+    case MOEV_W_FP8E4M3_B128: launch_simt_ffn<MOEV_W_FP8E4M3_B128, AFMT>(c, L, x, gamma, st, ev); break;
+    default: launch_simt_ffn<MOEV_W_MXFP4, AFMT>(c, L, x, gamma, st, ev); break;
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t moev_expert_code_bytes(const moev_config* cfg) { return cfg ? code_bytes(cfg) : 0; }
+size_t moev_expert_bytes(const moev_config* cfg) { return cfg ? code_bytes(cfg) + scale_bytes(cfg) : 0; }
+
+moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
+  if (!out) return MOEV_EINVAL;
+  *out = nullptr;
+  char why[256];
+  if (!cfg_ok(cfg, why, sizeof(why))) return MOEV_EINVAL;
+  int dev = -1;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    cudaGetLastError();
+    return MOEV_ECUDA;
+  }
+  if (prop.major != 10) return MOEV_EUNSUPPORTED;
+  if (cfg->impl == MOEV_IMPL_TCGEN05) return MOEV_EINVAL;  // tensor-core path not built for this shape
+  moev_ctx* c = new (std::nothrow) moev_ctx();
+  if (!c) return MOEV_ENOMEM;
+  c->cfg = *cfg;
+  c->device = dev;
+  c->resolved_impl = MOEV_IMPL_SIMT;
+  const size_t G = cfg->max_tokens, E = cfg->E, K = cfg->top_k, A = G * K;
+  const size_t slots = A + (size_t)cfg->n_shared * G;
+  const size_t act_b = cfg->afmt == MOEV_ACT_FP32 ? 4 : 2;
+  bool ok = true;
+  ok = ok && dmalloc(&c->T.logits, G * E) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.union_ids, E) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.offsets, E + 1) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.perm, A) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.slot_token, A) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.slot_w, A) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.n_active, 1) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.status, 1) == cudaSuccess;
+  ok = ok && dmalloc(&c->hbuf, slots * cfg->I) == cudaSuccess;
+  ok = ok && dmalloc(&c->y32, G * cfg->H) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->x_stage, G * cfg->H * act_b) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->y_stage, G * cfg->H * act_b) == cudaSuccess;
+  ok = ok && cudaMallocHost(reinterpret_cast<void**>(&c->host_word), 4 * sizeof(int32_t)) == cudaSuccess;
+  if (ok) ok = cudaMemset(c->T.status, 0, sizeof(int32_t)) == cudaSuccess;
+  // opt in to large dynamic shared memory where the shape needs it
+  if (ok) {
+    size_t rs = (size_t)cfg->H * 4, gs = route_smem(*cfg, cfg->max_tokens);
+    if (rs > 48 * 1024) {
+      ok = ok && cudaFuncSetAttribute(router_logits_kernel<MOEV_ACT_FP32>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(router_logits_kernel<MOEV_ACT_BF16>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs) == cudaSuccess;
+    }
+    if (gs > 48 * 1024)
+      ok = ok && cudaFuncSetAttribute(route_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)gs) == cudaSuccess;
+  }
+  if (!ok) {
+    cudaError_t e = cudaGetLastError();
+    moev_status st = (e == cudaErrorMemoryAllocation) ? MOEV_ENOMEM : MOEV_ECUDA;
+    moev_destroy(c);
+    return st;
+  }
+  *out = c;
+  return MOEV_OK;
+}
+
+moev_status moev_destroy(moev_ctx* c) {
+  if (!c) return MOEV_EINVAL;
+  cudaFree(c->T.logits); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
+  cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
+  cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->hbuf); cudaFree(c->y32);
+  cudaFree(c->x_stage); cudaFree(c->y_stage);
+  if (c->host_word) cudaFreeHost(c->host_word);
+  if (c->prof_events_ready)
+    for (int i = 0; i < kProfSlots; ++i)
+      for (int j = 0; j < 3; ++j) cudaEventDestroy(c->ev[i][j]);
+  cudaGetLastError();
+  delete c;
+  return MOEV_OK;
+}
+
+const char* moev_last_error(const moev_ctx* c) { return c ? c->err : "null context"; }
+int32_t moev_launches_per_call(const moev_ctx* c) { return c ? 5 : 0; }
+int32_t moev_resolved_impl(const moev_ctx* c) { return c ? c->resolved_impl : 0; }
+
+moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int32_t gamma,
+                        const moev_out* out, void* cuda_stream) {
+  if (!c) return MOEV_EINVAL;
+  const moev_config& g = c->cfg;
+  if (!layer || !x || !out) return fail(c, MOEV_EINVAL, "null layer, x or out");
+  if (gamma < 1 || gamma > g.max_tokens)
+    return fail(c, MOEV_EINVAL, "gamma=%d outside 1..max_tokens=%d", gamma, g.max_tokens);
+  if (!out->y || !out->n_active) return fail(c, MOEV_EINVAL, "out->y and out->n_active are required");
+  const bool scaled = g.wfmt == MOEV_W_FP8E4M3_B128 || g.wfmt == MOEV_W_MXFP4;
+  if (!layer->router_w || !layer->w_gate || !layer->w_up || !layer->w_down)
+    return fail(c, MOEV_EINVAL, "null router or expert weight pointer");
+  if (scaled && (!layer->s_gate || !layer->s_up || !layer->s_down))
+    return fail(c, MOEV_EINVAL, "weight format needs scale tensors");
+  if (g.n_shared > 0) {
+    if (!layer->sh_gate || !layer->sh_up || !layer->sh_down)
+      return fail(c, MOEV_EINVAL, "n_shared > 0 but shared expert weights are null");
+    if (scaled && (!layer->sh_s_gate || !layer->sh_s_up || !layer->sh_s_down))
+      return fail(c, MOEV_EINVAL, "shared experts need scale tensors");
+  }
+  const void* ptrs[] = {layer->router_w, layer->w_gate, layer->w_up, layer->w_down, layer->s_gate,
+                        layer->s_up, layer->s_down, layer->sh_gate, layer->sh_up, layer->sh_down,
+                        layer->sh_s_gate, layer->sh_s_up, layer->sh_s_down, x, out->y};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return fail(c, MOEV_EINVAL, "pointer %p is not 16-byte aligned", p);
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  LayerPtrs L{layer->w_gate, layer->w_up, layer->w_down, layer->s_gate, layer->s_up, layer->s_down,
+              layer->sh_gate, layer->sh_up, layer->sh_down, layer->sh_s_gate, layer->sh_s_up,
+              layer->sh_s_down};
+  RouteOut O{out->topk_ids, out->topk_w, out->union_ids, out->offsets, out->perm, out->n_active};
+  const size_t y_elems = (size_t)gamma * g.H;
+
+  if (g.afmt == MOEV_ACT_FP32)
+    router_logits_kernel<MOEV_ACT_FP32><<<g.E, 256, (size_t)g.H * 4, st>>>(
+        x, layer->router_w, c->T.logits, c->y32, gamma, g.H, g.E, y_elems);
+  else
+    router_logits_kernel<MOEV_ACT_BF16><<<g.E, 256, (size_t)g.H * 4, st>>>(
+        x, layer->router_w, c->T.logits, c->y32, gamma, g.H, g.E, y_elems);
+  route_group_kernel<<<1, 1024, route_smem(g, gamma), st>>>(c->T, O, gamma, g.E, g.top_k, g.score,
+                                                            g.routed_scale);
+  cudaEvent_t* ev = nullptr;
+  if (c->profile && c->prof_n < kProfSlots) ev = c->ev[c->prof_n++];
+  if (g.afmt == MOEV_ACT_FP32) launch_simt_ffn_w<MOEV_ACT_FP32>(c, L, x, gamma, st, ev);
+  else launch_simt_ffn_w<MOEV_ACT_BF16>(c, L, x, gamma, st, ev);
+  const int fin_blocks = (int)((y_elems / 4 + 255) / 256);
+  if (g.afmt == MOEV_ACT_FP32) finalize_kernel<MOEV_ACT_FP32><<<fin_blocks, 256, 0, st>>>(c->y32, out->y, y_elems);
+  else finalize_kernel<MOEV_ACT_BF16><<<fin_blocks, 256, 0, st>>>(c->y32, out->y, y_elems);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "kernel launch failed: %s", cudaGetErrorString(e));
+  return MOEV_OK;
+}
+
+moev_status moev_verify_host(moev_ctx* c, const moev_layer* layer, const void* x_host, int32_t gamma,
+                             void* y_host, int32_t* n_active_host, void* cuda_stream) {
+  if (!c) return MOEV_EINVAL;
+  if (!x_host || !y_host || !n_active_host) return fail(c, MOEV_EINVAL, "null host buffer");
+  if (gamma < 1 || gamma > c->cfg.max_tokens)
+    return fail(c, MOEV_EINVAL, "gamma=%d outside 1..max_tokens=%d", gamma, c->cfg.max_tokens);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t bytes = (size_t)gamma * c->cfg.H * (c->cfg.afmt == MOEV_ACT_FP32 ? 4 : 2);
+  cudaError_t e = cudaMemcpyAsync(c->x_stage, x_host, bytes, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "H2D copy failed: %s", cudaGetErrorString(e));
+  moev_out o{};
+  o.y = c->y_stage;
+  o.n_active = c->T.n_active;
+  moev_status s = moev_verify(c, layer, c->x_stage, gamma, &o, cuda_stream);
+  if (s != MOEV_OK) return s;
+  e = cudaMemcpyAsync(y_host, c->y_stage, bytes, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(n_active_host, c->T.n_active, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "D2H copy / sync failed: %s", cudaGetErrorString(e));
+  return MOEV_OK;
+}
+
+moev_status moev_status_sync(moev_ctx* c, void* cuda_stream) {
+  if (!c) return MOEV_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(c->host_word, c->T.status, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "status read failed: %s", cudaGetErrorString(e));
+  if (c->host_word[0] == kStatusTimeout) return fail(c, MOEV_ETIMEOUT, "a bounded device-side wait expired");
+  return MOEV_OK;
+}
+
+moev_status moev_profile_enable(moev_ctx* c, int32_t on) {
+  if (!c) return MOEV_EINVAL;
+  if (on && !c->prof_events_ready) {
+    for (int i = 0; i < kProfSlots; ++i)
+      for (int j = 0; j < 3; ++j)
+        if (cudaEventCreate(&c->ev[i][j]) != cudaSuccess)
+          return fail(c, MOEV_ECUDA, "cudaEventCreate failed");
+    c->prof_events_ready = true;
+  }
+  c->profile = on != 0;
+  c->prof_n = 0;
+  return MOEV_OK;
+}
+
+moev_status moev_profile_read(moev_ctx* c, void* cuda_stream, double* mean_us, int32_t* calls) {
+  if (!c || !mean_us || !calls) return MOEV_EINVAL;
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "sync failed: %s", cudaGetErrorString(e));
+  double s0 = 0, s1 = 0;
+  for (int i = 0; i < c->prof_n; ++i) {
+    float a = 0, b = 0;
+    cudaEventElapsedTime(&a, c->ev[i][0], c->ev[i][1]);
+    cudaEventElapsedTime(&b, c->ev[i][1], c->ev[i][2]);
+    s0 += a; s1 += b;
+  }
+  *calls = c->prof_n;
+  mean_us[0] = c->prof_n ? 1e3 * s0 / c->prof_n : 0.0;
+  mean_us[1] = c->prof_n ? 1e3 * s1 / c->prof_n : 0.0;
+  c->prof_n = 0;
+  return MOEV_OK;
+}
+
+}  // extern "C"

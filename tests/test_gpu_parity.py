@@ -1,0 +1,137 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU fp64 oracle, element by
+element on the same seeded inputs.  Integer results bit-exact; router weights 1e-5;
+outputs max_t(max_i|y-ref| / max_i|ref|) <= 1e-2 (fp32/bf16/fp8) or 3e-2 (mxfp4)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_12696_b200 as moev
+import synth
+from gpu_common import compare, device_layer, gcfg, ocfg, parity_case, run_gpu
+from helpers import small_shape
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [moev.IMPL_SIMT, moev.IMPL_AUTO]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_tiny_config(impl):
+    parity_case(synth.SHAPES["tiny"], 8, impl=impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("gamma", [1, 16, 33])
+def test_qwen_shaped_reduced(impl, gamma):
+    shape = small_shape("qwen", H=1024, I=384, E=32)
+    parity_case(shape, gamma, impl=impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("routing", ["scattered", "clustered"])
+def test_deepseek_shaped_reduced(impl, routing):
+    shape = small_shape("deepseek", H=1024, I=512, E=64)
+    err, ref = parity_case(shape, 32, routing=routing, impl=impl)
+    assert 8 <= ref.n_active <= 64
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("gamma", [1, 8, 19])
+def test_gptoss_shaped_reduced_ragged(impl, gamma):
+    # 736 = 5.75 * 128 and 352 = 2.75 * 128: several tiles and a ragged tail in both dims
+    shape = small_shape("gptoss", H=736, I=352, E=32)
+    parity_case(shape, gamma, impl=impl)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("gamma,U", [(1, 8), (8, 8), (8, 64), (32, 40), (128, 8), (128, 64)])
+def test_exact_union_cases(impl, gamma, U):
+    """Degenerate groupings: all tokens on the same k experts (m_e = gamma), every expert
+    used, one token only."""
+    shape = small_shape("deepseek", H=512, I=256, E=64)
+    err, ref = parity_case(shape, gamma, routing="exact", impl=impl, U=U)
+    assert ref.n_active == U
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_topk_equals_E_and_two_shared(impl):
+    shape = small_shape("deepseek", H=256, I=128, E=8, top_k=8, n_shared=2)
+    err, ref = parity_case(shape, 5, routing="scattered", impl=impl)
+    assert ref.n_active == 8
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_exact_logit_ties_break_to_lower_id(impl):
+    shape = small_shape("qwen", H=256, I=128, E=32, top_k=4)
+    w = synth.make_expert_weights(shape, device="cuda")
+    wr, x = synth.make_scattered_routing(shape, 6, device="cuda")
+    x = x.clone()
+    x[:, :32] = 0.0          # all 32 logits tie at 0 -> ids must be 0,1,2,3
+    x[3, 7] = 1.0            # one clear winner, then ties
+    res = run_gpu(shape, wr, w, x, 6, impl)
+    ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), 6)
+    assert list(ref.topk_ids[0]) == [0, 1, 2, 3] and list(ref.topk_ids[3]) == [7, 0, 1, 2]
+    compare(shape, res, ref, 6)
+
+
+def test_context_reuse_and_smaller_gamma():
+    """One context, several calls with different gamma: workspace state must not leak."""
+    shape = small_shape("qwen", H=512, I=256, E=16, top_k=4)
+    v = moev.MoeVerifier(gcfg(shape, 64))
+    w = synth.make_expert_weights(shape, device="cuda")
+    for gamma in (64, 3, 17, 64):
+        wr, x = synth.make_iid_routing(shape, gamma, device="cuda", layer=gamma)
+        res = run_gpu(shape, wr, w, x, gamma, verifier=v)
+        ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), gamma)
+        compare(shape, res, ref, gamma)
+    v.close()
+
+
+def test_verify_host_matches_verify():
+    shape = small_shape("deepseek", H=512, I=256, E=32)
+    v = moev.MoeVerifier(gcfg(shape, 16))
+    w = synth.make_expert_weights(shape, device="cuda")
+    wr, x = synth.make_scattered_routing(shape, 16, device="cuda")
+    layer, keep = device_layer(wr, w)
+    out = v.alloc_out(16)
+    v.verify(layer, x, 16, out)
+    torch.cuda.synchronize()
+    xh = x.cpu().pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    nh = torch.zeros(1, dtype=torch.int32).pin_memory()
+    v.verify_host(layer, xh, 16, yh, nh)
+    assert int(nh[0]) == int(out["n_active"][0])
+    ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), 16)
+    from helpers import rel_err
+    assert rel_err(yh.float().numpy(), ref.y) <= 1e-2
+    v.close()
+
+
+def test_invalid_arguments_are_rejected_before_launch():
+    shape = small_shape("qwen", H=256, I=128, E=16, top_k=4)
+    with pytest.raises(moev.MoevError) as e:
+        moev.MoeVerifier(moev.MoevConfig(H=250, I=128, E=16, top_k=4))
+    assert e.value.status == 1
+    with pytest.raises(moev.MoevError):
+        moev.MoeVerifier(moev.MoevConfig(H=256, I=128, E=16, top_k=17))
+    v = moev.MoeVerifier(gcfg(shape, 8))
+    w = synth.make_expert_weights(shape, device="cuda")
+    wr, x = synth.make_iid_routing(shape, 8, device="cuda")
+    layer, keep = device_layer(wr, w)
+    out = v.alloc_out(8)
+    for gamma in (0, 9):
+        with pytest.raises(moev.MoevError) as e:
+            v.verify(layer, x, gamma, out)
+        assert e.value.status == 1
+    with pytest.raises(moev.MoevError):  # misaligned x
+        v.verify(layer, x.view(-1)[1:257], 1, out)
+    bad = dict(keep)
+    bad.pop("w_up")
+    with pytest.raises(moev.MoevError):
+        v.verify(moev.binding.make_layer(bad), x, 8, out)
+    with pytest.raises(moev.MoevError):
+        v.verify(layer, x, 8, {"y": out["y"]})  # n_active missing
+    v.verify(layer, x, 8, out)  # still usable afterwards
+    v.status_sync()
+    v.close()
