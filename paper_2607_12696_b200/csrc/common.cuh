@@ -16,6 +16,15 @@ constexpr int kMaxTopK = 32;     // one lane per selected expert
 constexpr int kStatusOk = 0;
 constexpr int kStatusTimeout = 1;
 
+// One unit of tensor-core FFN work: an expert and a contiguous run of at most MC of its
+// assignment slots (experts with more tokens are split into several units).
+struct __align__(16) Unit {
+  int32_t expert;  // expert id (routed) or shared-expert index
+  int32_t slot0;   // first slot (shared: A + s*gamma + first token)
+  int32_t m;       // tokens in this unit
+  int32_t shared;  // 1 for a shared expert
+};
+
 // Device-side tables produced by the routing kernels and consumed by the FFN kernels.
 // slot = position in expert-sorted assignment order (0..A), then shared-expert slots
 // A + s*gamma + t.  All pointers live in the context workspace.
@@ -29,6 +38,9 @@ struct Tables {
   int32_t* slot_token; // [A]   token index of the assignment in this slot
   float* slot_w;       // [A]   its routing weight
   int32_t* n_active;   // [1]
+  float* tok_scale;    // [gamma] power of two bringing the token's max |x| into [64,128)
+  Unit* units;         // [max_units]
+  int32_t* n_units;    // [1]
   int32_t* status;     // [1]   kStatusOk / kStatusTimeout
 };
 

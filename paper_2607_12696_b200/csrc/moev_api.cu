@@ -6,13 +6,23 @@
 
 #include "common.cuh"
 #include "ffn_simt.cuh"
+#include "ffn_tc.cuh"
 #include "router.cuh"
 
 using namespace moev;
 
 namespace {
 constexpr int kProfSlots = 512;
-}
+constexpr int kTmapCache = 8;
+
+// The six TMA descriptors of one layer (gate, up, down, shared gate, up, down) and the
+// pointers they were encoded for.
+struct TmapSet {
+  const void* key[6] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  CUtensorMap map[6];
+  bool valid = false;
+};
+}  // namespace
 
 struct moev_ctx {
   moev_config cfg;
@@ -24,6 +34,10 @@ struct moev_ctx {
   void* x_stage = nullptr;  // device staging for moev_verify_host
   void* y_stage = nullptr;
   int32_t* host_word = nullptr;  // pinned scratch for status / n_active reads
+  TmapSet tmaps[kTmapCache];
+  int tmap_next = 0;
+  int n_sm = 0;
+  int unit_cap = 1 << 20;
   bool profile = false;
   cudaEvent_t ev[kProfSlots][3];
   int prof_n = 0;
@@ -89,6 +103,90 @@ size_t route_smem(const moev_config& c, int gamma) {
   return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4;
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// Can the tensor-core kernel run this shape?  (Otherwise AUTO resolves to the SIMT kernels.)
+bool tc_eligible(const moev_config& c) {
+  if (c.afmt != MOEV_ACT_BF16) return false;
+  if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
+  if (c.H % 128 || c.I % 128) return false;
+  const int bk = c.wfmt == MOEV_W_BF16 ? 64 : 128;
+  if (c.H / bk < 4 || c.H / 128 > 128 || c.H / bk > 128 * (128 / bk)) return false;
+  return true;
+}
+
+// [n_mat, N, K] weight tensor -> 3-D tiled map with a 128-row x 128-byte box, 128B swizzle.
+bool encode_weight_map(CUtensorMap* m, const moev_config& c, const void* ptr, int n_mat, int N, int K) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const bool bf16 = c.wfmt == MOEV_W_BF16;
+  const cuuint64_t es = bf16 ? 2 : 1;
+  cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)N, (cuuint64_t)n_mat};
+  cuuint64_t strides[2] = {(cuuint64_t)K * es, (cuuint64_t)K * es * (cuuint64_t)N};
+  cuuint32_t box[3] = {(cuuint32_t)(128 / es), 128, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 3,
+                  const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Find or build the descriptors of this layer (cache keyed by the six weight pointers).
+const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
+  const void* key[6] = {L->w_gate, L->w_up, L->w_down, L->sh_gate, L->sh_up, L->sh_down};
+  for (int i = 0; i < kTmapCache; ++i)
+    if (c->tmaps[i].valid && memcmp(c->tmaps[i].key, key, sizeof(key)) == 0) return &c->tmaps[i];
+  TmapSet& t = c->tmaps[c->tmap_next];
+  c->tmap_next = (c->tmap_next + 1) % kTmapCache;
+  t.valid = false;
+  const moev_config& g = c->cfg;
+  bool ok = encode_weight_map(&t.map[0], g, L->w_gate, g.E, g.I, g.H) &&
+            encode_weight_map(&t.map[1], g, L->w_up, g.E, g.I, g.H) &&
+            encode_weight_map(&t.map[2], g, L->w_down, g.E, g.H, g.I);
+  if (ok && g.n_shared > 0)
+    ok = encode_weight_map(&t.map[3], g, L->sh_gate, g.n_shared, g.I, g.H) &&
+         encode_weight_map(&t.map[4], g, L->sh_up, g.n_shared, g.I, g.H) &&
+         encode_weight_map(&t.map[5], g, L->sh_down, g.n_shared, g.H, g.I);
+  else if (ok) { t.map[3] = t.map[0]; t.map[4] = t.map[1]; t.map[5] = t.map[2]; }
+  if (!ok) return nullptr;
+  memcpy(t.key, key, sizeof(key));
+  t.valid = true;
+  return &t;
+}
+
+template <int WFMT>
+void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const void* x, int gamma,
+                   cudaStream_t st, cudaEvent_t* ev) {
+  const moev_config& g = c->cfg;
+  tc::Params P{};
+  P.units = c->T.units; P.n_units = c->T.n_units; P.slot_token = c->T.slot_token; P.slot_w = c->T.slot_w;
+  P.tok_scale = c->T.tok_scale; P.x = x; P.y32 = c->y32;
+  P.s_gate = static_cast<const float*>(L->s_gate); P.s_up = static_cast<const float*>(L->s_up);
+  P.s_down = static_cast<const float*>(L->s_down);
+  P.sh_s_gate = static_cast<const float*>(L->sh_s_gate); P.sh_s_up = static_cast<const float*>(L->sh_s_up);
+  P.sh_s_down = static_cast<const float*>(L->sh_s_down);
+  P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
+  if (ev) cudaEventRecord(ev[0], st);
+  tc::grouped_ffn_tc_kernel<WFMT><<<c->n_sm, tc::kThreads, tc::kSmemBytes, st>>>(
+      tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
+  if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); }
+}
+
 template <int WFMT, int AFMT>
 void launch_simt_ffn(moev_ctx* c, const LayerPtrs& L, const void* x, int gamma, cudaStream_t st,
                      cudaEvent_t* ev) {
@@ -134,12 +232,16 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     return MOEV_ECUDA;
   }
   if (prop.major != 10) return MOEV_EUNSUPPORTED;
-  if (cfg->impl == MOEV_IMPL_TCGEN05) return MOEV_EINVAL;  // tensor-core path not built for this shape
+  const bool tc_ok = tc_eligible(*cfg) && encode_tiled_fn() != nullptr;
+  if (cfg->impl == MOEV_IMPL_TCGEN05 && !tc_ok) return MOEV_EINVAL;  // shape not served by the tensor-core kernel
   moev_ctx* c = new (std::nothrow) moev_ctx();
   if (!c) return MOEV_ENOMEM;
   c->cfg = *cfg;
   c->device = dev;
-  c->resolved_impl = MOEV_IMPL_SIMT;
+  c->n_sm = prop.multiProcessorCount;
+  c->resolved_impl = (cfg->impl != MOEV_IMPL_SIMT && tc_ok) ? MOEV_IMPL_TCGEN05 : MOEV_IMPL_SIMT;
+  if (c->resolved_impl == MOEV_IMPL_TCGEN05)
+    c->unit_cap = cfg->wfmt == MOEV_W_BF16 ? tc::Fmt<MOEV_W_BF16>::kMC : tc::Fmt<MOEV_W_FP8E4M3_B128>::kMC;
   const size_t G = cfg->max_tokens, E = cfg->E, K = cfg->top_k, A = G * K;
   const size_t slots = A + (size_t)cfg->n_shared * G;
   const size_t act_b = cfg->afmt == MOEV_ACT_FP32 ? 4 : 2;
@@ -154,6 +256,13 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && dmalloc(&c->T.slot_w, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.n_active, 1) == cudaSuccess;
   ok = ok && dmalloc(&c->T.status, 1) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.tok_scale, G) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.n_units, 1) == cudaSuccess;
+  {
+    const size_t cap = c->unit_cap;
+    const size_t max_units = E + A / cap + (size_t)cfg->n_shared * (G / cap + 1) + 8;
+    ok = ok && dmalloc(&c->T.units, max_units) == cudaSuccess;
+  }
   ok = ok && dmalloc(&c->hbuf, slots * cfg->I) == cudaSuccess;
   ok = ok && dmalloc(&c->y32, G * cfg->H) == cudaSuccess;
   ok = ok && cudaMalloc(&c->x_stage, G * cfg->H * act_b) == cudaSuccess;
@@ -172,6 +281,12 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     if (gs > 48 * 1024)
       ok = ok && cudaFuncSetAttribute(route_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)gs) == cudaSuccess;
+    if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
+      ok = ok && cudaFuncSetAttribute(tc::grouped_ffn_tc_kernel<MOEV_W_BF16>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(tc::grouped_ffn_tc_kernel<MOEV_W_FP8E4M3_B128>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) == cudaSuccess;
+    }
   }
   if (!ok) {
     cudaError_t e = cudaGetLastError();
@@ -187,7 +302,8 @@ moev_status moev_destroy(moev_ctx* c) {
   if (!c) return MOEV_EINVAL;
   cudaFree(c->T.logits); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
-  cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->hbuf); cudaFree(c->y32);
+  cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale);
+  cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->hbuf); cudaFree(c->y32);
   cudaFree(c->x_stage); cudaFree(c->y_stage);
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)
@@ -199,7 +315,9 @@ moev_status moev_destroy(moev_ctx* c) {
 }
 
 const char* moev_last_error(const moev_ctx* c) { return c ? c->err : "null context"; }
-int32_t moev_launches_per_call(const moev_ctx* c) { return c ? 5 : 0; }
+int32_t moev_launches_per_call(const moev_ctx* c) {
+  return c ? (c->resolved_impl == MOEV_IMPL_TCGEN05 ? 4 : 5) : 0;
+}
 int32_t moev_resolved_impl(const moev_ctx* c) { return c ? c->resolved_impl : 0; }
 
 moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int32_t gamma,
@@ -227,6 +345,11 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   for (const void* p : ptrs)
     if (p && !aligned16(p)) return fail(c, MOEV_EINVAL, "pointer %p is not 16-byte aligned", p);
 
+  const TmapSet* tm = nullptr;
+  if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
+    tm = get_tmaps(c, layer);
+    if (!tm) return fail(c, MOEV_ECUDA, "cuTensorMapEncodeTiled failed for this layer's weight tensors");
+  }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   LayerPtrs L{layer->w_gate, layer->w_up, layer->w_down, layer->s_gate, layer->s_up, layer->s_down,
               layer->sh_gate, layer->sh_up, layer->sh_down, layer->sh_s_gate, layer->sh_s_up,
@@ -236,15 +359,18 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
 
   if (g.afmt == MOEV_ACT_FP32)
     router_logits_kernel<MOEV_ACT_FP32><<<g.E, 256, (size_t)g.H * 4, st>>>(
-        x, layer->router_w, c->T.logits, c->y32, gamma, g.H, g.E, y_elems);
+        x, layer->router_w, c->T.logits, c->y32, c->T.tok_scale, gamma, g.H, g.E, y_elems);
   else
     router_logits_kernel<MOEV_ACT_BF16><<<g.E, 256, (size_t)g.H * 4, st>>>(
-        x, layer->router_w, c->T.logits, c->y32, gamma, g.H, g.E, y_elems);
+        x, layer->router_w, c->T.logits, c->y32, c->T.tok_scale, gamma, g.H, g.E, y_elems);
   route_group_kernel<<<1, 1024, route_smem(g, gamma), st>>>(c->T, O, gamma, g.E, g.top_k, g.score,
-                                                            g.routed_scale);
+                                                            g.routed_scale, g.n_shared, c->unit_cap);
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->prof_n < kProfSlots) ev = c->ev[c->prof_n++];
-  if (g.afmt == MOEV_ACT_FP32) launch_simt_ffn_w<MOEV_ACT_FP32>(c, L, x, gamma, st, ev);
+  if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
+    if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);
+    else launch_tc_ffn<MOEV_W_FP8E4M3_B128>(c, tm, layer, x, gamma, st, ev);
+  } else if (g.afmt == MOEV_ACT_FP32) launch_simt_ffn_w<MOEV_ACT_FP32>(c, L, x, gamma, st, ev);
   else launch_simt_ffn_w<MOEV_ACT_BF16>(c, L, x, gamma, st, ev);
   const int fin_blocks = (int)((y_elems / 4 + 255) / 256);
   if (g.afmt == MOEV_ACT_FP32) finalize_kernel<MOEV_ACT_FP32><<<fin_blocks, 256, 0, st>>>(c->y32, out->y, y_elems);
@@ -283,7 +409,10 @@ moev_status moev_status_sync(moev_ctx* c, void* cuda_stream) {
   cudaError_t e = cudaMemcpyAsync(c->host_word, c->T.status, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "status read failed: %s", cudaGetErrorString(e));
-  if (c->host_word[0] == kStatusTimeout) return fail(c, MOEV_ETIMEOUT, "a bounded device-side wait expired");
+  if (c->host_word[0] == kStatusTimeout) {
+    cudaMemsetAsync(c->T.status, 0, sizeof(int32_t), st);
+    return fail(c, MOEV_ETIMEOUT, "a bounded device-side wait expired");
+  }
   return MOEV_OK;
 }
 

@@ -9,14 +9,17 @@ namespace moev {
 // logits[t,e] = sum_h x[t,h] * Wr[e,h], accumulated in fp64 so the top-k decision matches
 // an fp64 evaluation whenever the decision margin exceeds ~1e-12.  One CTA per expert row
 // (the router matrix is read from HBM once); x is re-read through L2.  Each CTA also zeroes
-// its slice of the fp32 combine accumulator y32 and (CTA 0) resets the status word.
+// its slice of the fp32 combine accumulator y32 and computes the power-of-two scale of the
+// tokens it owns.
 template <int AFMT>
 __global__ void __launch_bounds__(256) router_logits_kernel(const void* __restrict__ x,
                                                             const float* __restrict__ router_w,
                                                             double* __restrict__ logits,
-                                                            float* __restrict__ y32, int gamma,
+                                                            float* __restrict__ y32,
+                                                            float* __restrict__ tok_scale, int gamma,
                                                             int H, int E, size_t y32_elems) {
   extern __shared__ float wr_s[];
+  __shared__ float amax_s[8];
   const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float4* src = reinterpret_cast<const float4*>(router_w + (size_t)e * H);
   for (int i = tid; i < H / 4; i += 256) reinterpret_cast<float4*>(wr_s)[i] = __ldg(src + i);
@@ -39,6 +42,27 @@ __global__ void __launch_bounds__(256) router_logits_kernel(const void* __restri
     acc = warp_sum(acc);
     if (lane == 0) logits[(size_t)t * E + e] = acc;
   }
+  // tokens t = e, e+E, ...: 2^p with max|x_t| * 2^p in [64,128) (used by the fp8 operand split)
+  for (int t = e; t < gamma; t += E) {
+    float am = 0.f;
+    for (int h = tid * 8; h < H; h += 256 * 8) {
+      float v[8];
+      load_act8<AFMT>(x, (size_t)t * H + h, v);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) am = fmaxf(am, fabsf(v[i]));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
+    __syncthreads();
+    if (lane == 0) amax_s[warp] = am;
+    __syncthreads();
+    if (tid == 0) {
+      for (int w = 1; w < 8; ++w) am = fmaxf(am, amax_s[w]);
+      int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
+      ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
+      tok_scale[t] = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
+    }
+  }
 }
 
 struct RouteOut {  // optional caller-visible copies (may be null)
@@ -57,7 +81,8 @@ struct RouteOut {  // optional caller-visible copies (may be null)
 // assignments in order with ballots and writes the stable permutation.
 // Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A].
 __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O, int gamma, int E,
-                                                           int k, int score, float routed_scale) {
+                                                           int k, int score, float routed_scale,
+                                                           int n_shared, int unit_cap) {
   extern __shared__ int32_t sm[];
   const int A = gamma * k;
   int32_t* cnt = sm;
@@ -65,7 +90,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   int32_t* uidx = sm + 2 * E;
   int32_t* ids_s = sm + 3 * E;
   float* w_s = reinterpret_cast<float*>(sm + 3 * E + A);
-  __shared__ int32_t warp_tot_cnt[32], warp_tot_flag[32];
+  __shared__ int32_t warp_tot_cnt[32], warp_tot_flag[32], warp_tot_unit[32], n_union_s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
 
   for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
@@ -153,11 +178,38 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       T.offsets[U] = A;
       if (O.offsets) O.offsets[U] = A;
       *T.n_active = U;
+      n_union_s = U;
       if (O.n_active) *O.n_active = U;
-      *T.status = kStatusOk;
     }
   }
   __syncthreads();
+
+  // ---- phase 2b: work units for the tensor-core FFN: expert u of the union (then the shared
+  // experts) is cut into ceil(m / unit_cap) runs of at most unit_cap slots
+  {
+    const int U = n_union_s;
+    int e = 0, slot0 = 0, m = 0, shared = 0;
+    if (tid < U) { e = T.union_ids[tid]; slot0 = T.offsets[tid]; m = cnt[e]; }
+    else if (tid < U + n_shared) { shared = 1; e = tid - U; slot0 = A + e * gamma; m = gamma; }
+    int nch = (m + unit_cap - 1) / unit_cap, sc = nch;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      int a = __shfl_up_sync(0xffffffffu, sc, o);
+      if (lane >= o) sc += a;
+    }
+    if (lane == 31) warp_tot_unit[warp] = sc;
+    __syncthreads();
+    int base = 0;
+    for (int w = 0; w < warp; ++w) base += warp_tot_unit[w];
+    int first = base + sc - nch;
+    for (int c = 0; c < nch; ++c) {
+      Unit un;
+      un.expert = e; un.slot0 = slot0 + c * unit_cap;
+      un.m = min(unit_cap, m - c * unit_cap); un.shared = shared;
+      T.units[first + c] = un;
+    }
+    if (tid == blockDim.x - 1) *T.n_units = base + sc;
+  }
 
   // ---- phase 3: stable permutation, one warp per expert
   for (int e = warp; e < E; e += nwarps) {
