@@ -45,6 +45,10 @@ WORKLOADS = {
     "gptoss_mxfp4_g32": ("gptoss", 32, "iid", {}),
     "gptoss_mxfp4_g64": ("gptoss", 64, "iid", {}),
     "tiny_fp32_g8": ("tiny", 8, "iid", {}),
+    # profiling-size cases (a few GB on the device, still far larger than L2): the DeepSeek-
+    # and Qwen-shaped layers with 64 experts
+    "deepseek_fp8_E64_g16_profile": ("deepseek", 16, "scattered", {"_E": 64}),
+    "qwen_bf16_E64_g16_profile": ("qwen", 16, "iid", {"_E": 64}),
 }
 DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 
@@ -112,9 +116,16 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+def workload_shape(name: str) -> synth.Shape:
+    base, _, _, kw = WORKLOADS[name]
+    shape = synth.SHAPES[base]
+    return shape.scaled(E=kw["_E"]) if "_E" in kw else shape
+
+
 def build_workload(name: str, n_layers: int, device, rank: int = 0):
     base, gamma, routing, kw = WORKLOADS[name]
-    shape = synth.SHAPES[base]
+    shape = workload_shape(name)
+    kw = {k: v for k, v in kw.items() if not k.startswith("_")}
     layers = []
     for l in range(n_layers):
         lid = rank * 1000 + l
@@ -158,8 +169,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    base, gamma, routing, kw = WORKLOADS[args.workload]
-    shape = synth.SHAPES[base]
+    shape = workload_shape(args.workload)
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     shape_, gamma, layers = build_workload(args.workload, 1, dev)
     import oracle
@@ -200,8 +210,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
 
-    base = WORKLOADS[args.workload][0]
-    shape = synth.SHAPES[base]
+    shape = workload_shape(args.workload)
     n_layers = layers_that_fit(shape, args.layers)
     shape, gamma, layers = build_workload(args.workload, n_layers, dev, rank)
     impl = {"auto": moev.IMPL_AUTO, "simt": moev.IMPL_SIMT, "tcgen05": moev.IMPL_TCGEN05}[args.kernels]
@@ -286,9 +295,9 @@ def run_ours(args):
         impl_name = {1: "simt", 2: "tcgen05"}[v.resolved_impl()]
         mean_bytes = tot_bytes / args.steps
         if impl_name == "simt":  # two kernels; the first (gate/up) streams 2/3 of the bytes
-            k_name, k_bytes, k_us = "ffn_gateup_simt", mean_bytes * 2.0 / 3.0, kern_us[0]
+            k_name, k_bytes, k_us = "ffn_gateup_simt", mean_bytes * 2.0 / 3.0, kern_us[3]
         else:
-            k_name, k_bytes, k_us = "grouped_ffn_tcgen05", mean_bytes, kern_us[0]
+            k_name, k_bytes, k_us = "grouped_ffn_tc_kernel", mean_bytes, kern_us[3]
         achieved = k_bytes / (k_us * 1e-6) / 1e9 if k_us > 0 else None
         cpu = None
         if not args.no_cpu_baseline:
@@ -314,7 +323,10 @@ def run_ours(args):
                          "frac": (achieved / peak) if achieved else None,
                          "traffic": NCU_TRAFFIC_BYTES.get((args.workload, impl_name)),
                          "kernel": k_name, "kernel_us": k_us, "kernel_bytes": k_bytes,
-                         "second_kernel_us": kern_us[1], "launches_timed": kern_calls,
+                         "launches_timed": kern_calls,
+                         "per_kernel_us": {"router_partial": kern_us[0], "topk_refine": kern_us[1],
+                                           "route_group": kern_us[2], "ffn_1": kern_us[3],
+                                           "ffn_2": kern_us[4], "finalize": kern_us[5]},
                          "peak_source": peak_src + " (of %s)" % peak_src},
             "cpu_baseline": cpu,
             "e2e": {"value": all_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,

@@ -170,14 +170,15 @@ size_t moev_expert_code_bytes(const moev_config* cfg);
 int32_t moev_launches_per_call(const moev_ctx* ctx);
 int32_t moev_resolved_impl(const moev_ctx* ctx);
 
-/* Device time of the expert-FFN kernels (the weight-streaming part of the call), measured
- * with CUDA events recorded on the call's stream.  moev_profile_enable(ctx, 1) turns the
- * event records on (at most 512 calls are kept between reads), 0 off.  moev_profile_read
- * waits for the stream, writes mean_us[0..1] -- the mean duration in microseconds of the
- * first and of the second FFN kernel of a call (the SIMT path has two: gate/up and down; a
- * fused path reports 0 for the second) -- and the number of calls averaged, then resets. */
+/* Per-kernel device time of a call, measured with CUDA events recorded on the call's
+ * stream between its kernels.  moev_profile_enable(ctx, 1) turns the event records on (at
+ * most 512 calls are kept between reads), 0 off.  moev_profile_read waits for the stream and
+ * writes mean_us[0..5], the mean duration in microseconds of: router partial logits, top-k
+ * with exact refinement, grouping (union / permutation), first FFN kernel (the fused
+ * tensor-core kernel, or SIMT gate/up), second FFN kernel (SIMT down; 0 on the fused path),
+ * finalize; then the number of calls averaged, and resets the accumulator. */
 moev_status moev_profile_enable(moev_ctx* ctx, int32_t on);
-moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[2]*/,
+moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[6]*/,
                               int32_t* calls);
 
 #ifdef __cplusplus

@@ -212,7 +212,7 @@ class MoeVerifier:
         self._check(lib().moev_profile_enable(self._h, int(on)))
 
     def profile_read(self):
-        us = (C.c_double * 2)()
+        us = (C.c_double * 6)()
         n = C.c_int32()
         self._check(lib().moev_profile_read(self._h, self._stream(), us, C.byref(n)))
-        return [us[0], us[1]], n.value
+        return [us[i] for i in range(6)], n.value

@@ -29,7 +29,6 @@ struct __align__(16) Unit {
 // slot = position in expert-sorted assignment order (0..A), then shared-expert slots
 // A + s*gamma + t.  All pointers live in the context workspace.
 struct Tables {
-  double* logits;      // [gamma, E]
   int32_t* topk_ids;   // [gamma, k]
   float* topk_w;       // [gamma, k]
   int32_t* union_ids;  // [E]

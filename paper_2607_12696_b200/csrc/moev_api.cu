@@ -31,6 +31,10 @@ struct moev_ctx {
   Tables T{};
   float* hbuf = nullptr;  // [(max_tokens*k + n_shared*max_tokens), I] fp32
   float* y32 = nullptr;   // [max_tokens, H] fp32 combine accumulator
+  float* part = nullptr;     // [n_slices, max_tokens, E] split-K partial router logits
+  float* part_x2 = nullptr;  // [n_slices, max_tokens]
+  float* part_w2 = nullptr;  // [n_slices] max over experts of the slice's squared row norm
+  int n_slices = 0;
   void* x_stage = nullptr;  // device staging for moev_verify_host
   void* y_stage = nullptr;
   int32_t* host_word = nullptr;  // pinned scratch for status / n_active reads
@@ -39,7 +43,7 @@ struct moev_ctx {
   int n_sm = 0;
   int unit_cap = 1 << 20;
   bool profile = false;
-  cudaEvent_t ev[kProfSlots][3];
+  cudaEvent_t ev[kProfSlots][7];  // before/after each kernel of a call
   int prof_n = 0;
   bool prof_events_ready = false;
   char err[512] = {0};
@@ -71,7 +75,6 @@ bool cfg_ok(const moev_config* c, char* why, size_t n) {
   BAD(c->afmt < 0 || c->afmt > MOEV_ACT_BF16, "unknown activation format");
   BAD(c->score < 0 || c->score > MOEV_SCORE_SIGMOID, "unknown score function");
   BAD(c->impl < 0 || c->impl > MOEV_IMPL_TCGEN05, "unknown impl");
-  BAD((size_t)c->H * 4 > 200 * 1024, "H too large for the router kernel's shared memory");
 #undef BAD
   return true;
 }
@@ -181,10 +184,9 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.sh_s_gate = static_cast<const float*>(L->sh_s_gate); P.sh_s_up = static_cast<const float*>(L->sh_s_up);
   P.sh_s_down = static_cast<const float*>(L->sh_s_down);
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
-  if (ev) cudaEventRecord(ev[0], st);
   tc::grouped_ffn_tc_kernel<WFMT><<<c->n_sm, tc::kThreads, tc::kSmemBytes, st>>>(
       tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
-  if (ev) { cudaEventRecord(ev[1], st); cudaEventRecord(ev[2], st); }
+  if (ev) cudaEventRecord(ev[4], st);
 }
 
 template <int WFMT, int AFMT>
@@ -193,13 +195,12 @@ void launch_simt_ffn(moev_ctx* c, const LayerPtrs& L, const void* x, int gamma, 
   const moev_config& g = c->cfg;
   const int rows = 64;
   dim3 g1(g.E + g.n_shared, (g.I + rows - 1) / rows), g2(g.E + g.n_shared, (g.H + rows - 1) / rows);
-  if (ev) cudaEventRecord(ev[0], st);
   ffn_gateup_simt<WFMT, AFMT><<<g1, 256, 0, st>>>(L, c->T, x, c->hbuf, gamma, g.H, g.I, g.top_k,
                                                    g.n_shared, rows);
-  if (ev) cudaEventRecord(ev[1], st);
+  if (ev) cudaEventRecord(ev[4], st);
   ffn_down_simt<WFMT><<<g2, 256, 0, st>>>(L, c->T, c->hbuf, c->y32, gamma, g.H, g.I, g.top_k,
                                            g.n_shared, rows);
-  if (ev) cudaEventRecord(ev[2], st);
+  if (ev) cudaEventRecord(ev[5], st);
 }
 
 template <int AFMT>
@@ -246,7 +247,10 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   const size_t slots = A + (size_t)cfg->n_shared * G;
   const size_t act_b = cfg->afmt == MOEV_ACT_FP32 ? 4 : 2;
   bool ok = true;
-  ok = ok && dmalloc(&c->T.logits, G * E) == cudaSuccess;
+  c->n_slices = (cfg->H + kRouterKS - 1) / kRouterKS;
+  ok = ok && dmalloc(&c->part, (size_t)c->n_slices * G * E) == cudaSuccess;
+  ok = ok && dmalloc(&c->part_x2, (size_t)c->n_slices * G) == cudaSuccess;
+  ok = ok && dmalloc(&c->part_w2, (size_t)c->n_slices) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.union_ids, E) == cudaSuccess;
@@ -271,13 +275,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   if (ok) ok = cudaMemset(c->T.status, 0, sizeof(int32_t)) == cudaSuccess;
   // opt in to large dynamic shared memory where the shape needs it
   if (ok) {
-    size_t rs = (size_t)cfg->H * 4, gs = route_smem(*cfg, cfg->max_tokens);
-    if (rs > 48 * 1024) {
-      ok = ok && cudaFuncSetAttribute(router_logits_kernel<MOEV_ACT_FP32>,
-                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs) == cudaSuccess;
-      ok = ok && cudaFuncSetAttribute(router_logits_kernel<MOEV_ACT_BF16>,
-                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rs) == cudaSuccess;
-    }
+    size_t gs = route_smem(*cfg, cfg->max_tokens);
     if (gs > 48 * 1024)
       ok = ok && cudaFuncSetAttribute(route_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)gs) == cudaSuccess;
@@ -300,7 +298,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
 
 moev_status moev_destroy(moev_ctx* c) {
   if (!c) return MOEV_EINVAL;
-  cudaFree(c->T.logits); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
+  cudaFree(c->part); cudaFree(c->part_x2); cudaFree(c->part_w2); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale);
   cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->hbuf); cudaFree(c->y32);
@@ -308,7 +306,7 @@ moev_status moev_destroy(moev_ctx* c) {
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)
     for (int i = 0; i < kProfSlots; ++i)
-      for (int j = 0; j < 3; ++j) cudaEventDestroy(c->ev[i][j]);
+      for (int j = 0; j < 7; ++j) cudaEventDestroy(c->ev[i][j]);
   cudaGetLastError();
   delete c;
   return MOEV_OK;
@@ -316,7 +314,7 @@ moev_status moev_destroy(moev_ctx* c) {
 
 const char* moev_last_error(const moev_ctx* c) { return c ? c->err : "null context"; }
 int32_t moev_launches_per_call(const moev_ctx* c) {
-  return c ? (c->resolved_impl == MOEV_IMPL_TCGEN05 ? 4 : 5) : 0;
+  return c ? (c->resolved_impl == MOEV_IMPL_TCGEN05 ? 5 : 6) : 0;
 }
 int32_t moev_resolved_impl(const moev_ctx* c) { return c ? c->resolved_impl : 0; }
 
@@ -357,16 +355,29 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   RouteOut O{out->topk_ids, out->topk_w, out->union_ids, out->offsets, out->perm, out->n_active};
   const size_t y_elems = (size_t)gamma * g.H;
 
-  if (g.afmt == MOEV_ACT_FP32)
-    router_logits_kernel<MOEV_ACT_FP32><<<g.E, 256, (size_t)g.H * 4, st>>>(
-        x, layer->router_w, c->T.logits, c->y32, c->T.tok_scale, gamma, g.H, g.E, y_elems);
-  else
-    router_logits_kernel<MOEV_ACT_BF16><<<g.E, 256, (size_t)g.H * 4, st>>>(
-        x, layer->router_w, c->T.logits, c->y32, c->T.tok_scale, gamma, g.H, g.E, y_elems);
-  route_group_kernel<<<1, 1024, route_smem(g, gamma), st>>>(c->T, O, gamma, g.E, g.top_k, g.score,
-                                                            g.routed_scale, g.n_shared, c->unit_cap);
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->prof_n < kProfSlots) ev = c->ev[c->prof_n++];
+  if (ev) cudaEventRecord(ev[0], st);
+  const size_t refine_smem = (size_t)g.E * 16;
+  if (g.afmt == MOEV_ACT_FP32)
+    router_partial_kernel<MOEV_ACT_FP32><<<c->n_slices, 256, 0, st>>>(x, layer->router_w, c->part, c->part_x2,
+                                                                      c->part_w2, gamma, g.H, g.E);
+  else
+    router_partial_kernel<MOEV_ACT_BF16><<<c->n_slices, 256, 0, st>>>(x, layer->router_w, c->part, c->part_x2,
+                                                                      c->part_w2, gamma, g.H, g.E);
+  if (ev) cudaEventRecord(ev[1], st);
+  if (g.afmt == MOEV_ACT_FP32)
+    topk_refine_kernel<MOEV_ACT_FP32><<<gamma, 256, refine_smem, st>>>(
+        c->T, O, x, layer->router_w, c->part, c->part_x2, c->part_w2, c->y32, gamma, g.H, g.E, g.top_k,
+        c->n_slices, g.score, g.routed_scale);
+  else
+    topk_refine_kernel<MOEV_ACT_BF16><<<gamma, 256, refine_smem, st>>>(
+        c->T, O, x, layer->router_w, c->part, c->part_x2, c->part_w2, c->y32, gamma, g.H, g.E, g.top_k,
+        c->n_slices, g.score, g.routed_scale);
+  if (ev) cudaEventRecord(ev[2], st);
+  route_group_kernel<<<1, 1024, route_smem(g, gamma), st>>>(c->T, O, gamma, g.E, g.top_k, g.n_shared,
+                                                            c->unit_cap);
+  if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);
     else launch_tc_ffn<MOEV_W_FP8E4M3_B128>(c, tm, layer, x, gamma, st, ev);
@@ -375,6 +386,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   const int fin_blocks = (int)((y_elems / 4 + 255) / 256);
   if (g.afmt == MOEV_ACT_FP32) finalize_kernel<MOEV_ACT_FP32><<<fin_blocks, 256, 0, st>>>(c->y32, out->y, y_elems);
   else finalize_kernel<MOEV_ACT_BF16><<<fin_blocks, 256, 0, st>>>(c->y32, out->y, y_elems);
+  if (ev) cudaEventRecord(ev[6], st);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "kernel launch failed: %s", cudaGetErrorString(e));
   return MOEV_OK;
@@ -420,7 +432,7 @@ moev_status moev_profile_enable(moev_ctx* c, int32_t on) {
   if (!c) return MOEV_EINVAL;
   if (on && !c->prof_events_ready) {
     for (int i = 0; i < kProfSlots; ++i)
-      for (int j = 0; j < 3; ++j)
+      for (int j = 0; j < 7; ++j)
         if (cudaEventCreate(&c->ev[i][j]) != cudaSuccess)
           return fail(c, MOEV_ECUDA, "cudaEventCreate failed");
     c->prof_events_ready = true;
@@ -434,16 +446,19 @@ moev_status moev_profile_read(moev_ctx* c, void* cuda_stream, double* mean_us, i
   if (!c || !mean_us || !calls) return MOEV_EINVAL;
   cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(cuda_stream));
   if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "sync failed: %s", cudaGetErrorString(e));
-  double s0 = 0, s1 = 0;
-  for (int i = 0; i < c->prof_n; ++i) {
-    float a = 0, b = 0;
-    cudaEventElapsedTime(&a, c->ev[i][0], c->ev[i][1]);
-    cudaEventElapsedTime(&b, c->ev[i][1], c->ev[i][2]);
-    s0 += a; s1 += b;
-  }
+  // intervals: router partials | top-k refine | grouping | FFN kernel 1 | FFN kernel 2 (SIMT) | finalize
+  const bool two = c->resolved_impl == MOEV_IMPL_SIMT;
+  const int from[6] = {0, 1, 2, 3, 4, two ? 5 : 4}, to[6] = {1, 2, 3, 4, 5, 6};
+  double sum[6] = {0, 0, 0, 0, 0, 0};
+  for (int i = 0; i < c->prof_n; ++i)
+    for (int j = 0; j < 6; ++j) {
+      if (j == 4 && !two) continue;
+      float ms = 0;
+      cudaEventElapsedTime(&ms, c->ev[i][from[j]], c->ev[i][to[j]]);
+      sum[j] += ms;
+    }
   *calls = c->prof_n;
-  mean_us[0] = c->prof_n ? 1e3 * s0 / c->prof_n : 0.0;
-  mean_us[1] = c->prof_n ? 1e3 * s1 / c->prof_n : 0.0;
+  for (int j = 0; j < 6; ++j) mean_us[j] = c->prof_n ? 1e3 * sum[j] / c->prof_n : 0.0;
   c->prof_n = 0;
   return MOEV_OK;
 }

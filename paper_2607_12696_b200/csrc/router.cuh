@@ -1,67 +1,123 @@
-// Routing kernels: router logits (fp64 accumulation), per-token top-k + router weights,
-// expert union (Eq. 1), per-expert histogram, offsets and the stable token->expert
-// permutation.  Integer outputs are exact; see the notes at each kernel.
+// Routing kernels.
+//   1. router_partial_kernel  split-K fp32 partial logits (the router matrix and x are each
+//                             read once), plus partial squared norms for the error bound;
+//   2. topk_refine_kernel     one CTA per token: sums the partials, takes every expert whose
+//                             fp32 logit could reach the top-k given a rigorous rounding-error
+//                             bound, re-evaluates exactly those logits in fp64 and ranks them
+//                             (larger logit first, exact ties to the lower id), then the router
+//                             weights in fp64;
+//   3. route_group_kernel     one CTA: expert union (Eq. 1), per-expert histogram, offsets,
+//                             stable token->expert permutation, FFN work units.
+// The selected ids therefore equal the ids an all-fp64 evaluation selects whenever the fp64
+// decision margin exceeds the fp64 rounding error (~1e-12); integer tables are exact.
 #pragma once
 #include "common.cuh"
 
 namespace moev {
 
-// logits[t,e] = sum_h x[t,h] * Wr[e,h], accumulated in fp64 so the top-k decision matches
-// an fp64 evaluation whenever the decision margin exceeds ~1e-12.  One CTA per expert row
-// (the router matrix is read from HBM once); x is re-read through L2.  Each CTA also zeroes
-// its slice of the fp32 combine accumulator y32 and computes the power-of-two scale of the
-// tokens it owns.
+constexpr int kRouterKS = 32;  // K extent of one split-K slice
+
+// bf16 bit pattern -> double without the fp64 conversion unit (exact for normal numbers;
+// zeros / subnormals / non-finite take the conversion instruction).
+__device__ __forceinline__ double bf16_bits_to_double(uint32_t b) {
+  if ((b & 0x7F80u) == 0u || (b & 0x7F80u) == 0x7F80u) return (double)__uint_as_float(b << 16);
+  uint32_t hi = ((b & 0x8000u) << 16) | (((b & 0x7FFFu) << 13) + (896u << 20));
+  return __hiloint2double((int)hi, 0);
+}
+
 template <int AFMT>
-__global__ void __launch_bounds__(256) router_logits_kernel(const void* __restrict__ x,
-                                                            const float* __restrict__ router_w,
-                                                            double* __restrict__ logits,
-                                                            float* __restrict__ y32,
-                                                            float* __restrict__ tok_scale, int gamma,
-                                                            int H, int E, size_t y32_elems) {
-  extern __shared__ float wr_s[];
-  __shared__ float amax_s[8];
-  const int e = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const float4* src = reinterpret_cast<const float4*>(router_w + (size_t)e * H);
-  for (int i = tid; i < H / 4; i += 256) reinterpret_cast<float4*>(wr_s)[i] = __ldg(src + i);
-  // zero this CTA's slice of y32 (float4 granularity; y32_elems is a multiple of 4)
-  {
-    size_t n4 = y32_elems / 4, per = (n4 + gridDim.x - 1) / gridDim.x;
-    size_t lo = (size_t)e * per, hi = lo + per < n4 ? lo + per : n4;
-    for (size_t i = lo + tid; i < hi; i += 256)
-      reinterpret_cast<float4*>(y32)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+__device__ __forceinline__ float load_act1(const void* x, size_t idx) {
+  if (AFMT == MOEV_ACT_FP32) return __ldg(static_cast<const float*>(x) + idx);
+  return bf16_bits_to_float(__ldg(static_cast<const uint16_t*>(x) + idx));
+}
+
+// part[c, t, e] = sum_{h in slice c} x[t,h] * Wr[e,h]  (fp32, sequential over the slice)
+// part_x2[c, t] = sum_{h in slice c} x[t,h]^2,  part_w2max[c] = max_e sum_{h in slice c} Wr[e,h]^2
+// (so that sum_c part_w2max[c] >= max_e ||Wr[e,:]||^2).
+// Grid: one CTA per K slice of kRouterKS columns; 256 threads, thread (ty, tx) owns the 8 x 8
+// block of tokens 8*ty.. and experts tx + 32*j of each 64-token x 256-expert tile.
+template <int AFMT>
+__global__ void __launch_bounds__(256) router_partial_kernel(const void* __restrict__ x,
+                                                             const float* __restrict__ router_w,
+                                                             float* __restrict__ part,
+                                                             float* __restrict__ part_x2,
+                                                             float* __restrict__ part_w2max, int gamma,
+                                                             int H, int E) {
+  constexpr int KS = kRouterKS;
+  __shared__ float wmax_s[8];
+  float w2max = 0.f;
+  __shared__ float x_s[KS][64 + 4];    // [k][token]
+  __shared__ float w_s[KS][256 + 1];   // [k][expert]
+  const int c = blockIdx.x, tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+  const int k0 = c * KS, kn = min(KS, H - k0);
+  for (int e0 = 0; e0 < E; e0 += 256) {
+    __syncthreads();
+    // router tile -> shared, transposed; also the squared row norms of this slice
+    for (int i = tid; i < 256 * (KS / 4); i += 256) {
+      int er = i / (KS / 4), kq = (i % (KS / 4)) * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (e0 + er < E && kq < kn) v = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)(e0 + er) * H + k0 + kq));
+      w_s[kq][er] = v.x; w_s[kq + 1][er] = v.y; w_s[kq + 2][er] = v.z; w_s[kq + 3][er] = v.w;
+    }
+    __syncthreads();
+    if (e0 + tid < E) {
+      float s2 = 0.f;
+      for (int k = 0; k < KS; ++k) s2 = fmaf(w_s[k][tid], w_s[k][tid], s2);
+      w2max = fmaxf(w2max, s2);
+    }
+    for (int t0 = 0; t0 < gamma; t0 += 64) {
+      __syncthreads();
+      for (int i = tid; i < 64 * KS; i += 256) {
+        int tr = i / KS, k = i % KS;
+        float v = (t0 + tr < gamma && k < kn) ? load_act1<AFMT>(x, (size_t)(t0 + tr) * H + k0 + k) : 0.f;
+        x_s[k][tr] = v;
+      }
+      __syncthreads();
+      if (e0 == 0 && tid < 64 && t0 + tid < gamma) {
+        float s2 = 0.f;
+        for (int k = 0; k < KS; ++k) s2 = fmaf(x_s[k][tid], x_s[k][tid], s2);
+        part_x2[(size_t)c * gamma + t0 + tid] = s2;
+      }
+      float acc[8][8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+#pragma unroll 4
+      for (int k = 0; k < KS; ++k) {
+        float xv[8], wv[8];
+        float4 xa = *reinterpret_cast<const float4*>(&x_s[k][ty * 8]);
+        float4 xb = *reinterpret_cast<const float4*>(&x_s[k][ty * 8 + 4]);
+        xv[0] = xa.x; xv[1] = xa.y; xv[2] = xa.z; xv[3] = xa.w;
+        xv[4] = xb.x; xv[5] = xb.y; xv[6] = xb.z; xv[7] = xb.w;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) wv[j] = w_s[k][tx + 32 * j];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(xv[i], wv[j], acc[i][j]);
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        int t = t0 + ty * 8 + i;
+        if (t < gamma) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            int e = e0 + tx + 32 * j;
+            if (e < E) part[((size_t)c * gamma + t) * E + e] = acc[i][j];
+          }
+        }
+      }
+    }
   }
+  // max over experts of the squared norm of this slice of the router rows
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) w2max = fmaxf(w2max, __shfl_xor_sync(0xffffffffu, w2max, o));
+  if (tx == 0) wmax_s[ty] = w2max;
   __syncthreads();
-  for (int t = warp; t < gamma; t += 8) {
-    double acc = 0.0;
-    for (int h = lane * 8; h < H; h += 256) {
-      float v[8];
-      load_act8<AFMT>(x, (size_t)t * H + h, v);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc = fma((double)v[i], (double)wr_s[h + i], acc);
-    }
-    acc = warp_sum(acc);
-    if (lane == 0) logits[(size_t)t * E + e] = acc;
-  }
-  // tokens t = e, e+E, ...: 2^p with max|x_t| * 2^p in [64,128) (used by the fp8 operand split)
-  for (int t = e; t < gamma; t += E) {
-    float am = 0.f;
-    for (int h = tid * 8; h < H; h += 256 * 8) {
-      float v[8];
-      load_act8<AFMT>(x, (size_t)t * H + h, v);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) am = fmaxf(am, fabsf(v[i]));
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
-    __syncthreads();
-    if (lane == 0) amax_s[warp] = am;
-    __syncthreads();
-    if (tid == 0) {
-      for (int w = 1; w < 8; ++w) am = fmaxf(am, amax_s[w]);
-      int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
-      ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
-      tok_scale[t] = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
-    }
+  if (tid == 0) {
+    for (int w = 1; w < 8; ++w) w2max = fmaxf(w2max, wmax_s[w]);
+    part_w2max[c] = w2max;
   }
 }
 
@@ -74,56 +130,193 @@ struct RouteOut {  // optional caller-visible copies (may be null)
   int32_t* n_active;
 };
 
-// One CTA (1024 threads).  Phase 1: one warp per token selects the top-k experts by k
-// rounds of warp arg-max on (logit, id) keys -- larger logit first, exact ties to the lower
-// id -- and computes the router weights in fp64.  Phase 2: block scan over the E per-expert
-// counts gives the ascending union and the offsets.  Phase 3: one warp per expert walks the
-// assignments in order with ballots and writes the stable permutation.
-// Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A].
-__global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O, int gamma, int E,
-                                                           int k, int score, float routed_scale,
-                                                           int n_shared, int unit_cap) {
-  extern __shared__ int32_t sm[];
-  const int A = gamma * k;
-  int32_t* cnt = sm;
-  int32_t* excl = sm + E;
-  int32_t* uidx = sm + 2 * E;
-  int32_t* ids_s = sm + 3 * E;
-  float* w_s = reinterpret_cast<float*>(sm + 3 * E + A);
-  __shared__ int32_t warp_tot_cnt[32], warp_tot_flag[32], warp_tot_unit[32], n_union_s;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+// One CTA (256 threads) per token.  Shared memory: l32[E] floats | cand[E] ints | L[E] doubles.
+template <int AFMT>
+__global__ void __launch_bounds__(256) topk_refine_kernel(Tables T, RouteOut O, const void* __restrict__ x,
+                                                          const float* __restrict__ router_w,
+                                                          const float* __restrict__ part,
+                                                          const float* __restrict__ part_x2,
+                                                          const float* __restrict__ part_w2max,
+                                                          float* __restrict__ y32, int gamma, int H, int E,
+                                                          int k, int n_slices, int score, float routed_scale) {
+  extern __shared__ double sm_d[];
+  double* L = sm_d;                                    // [E] refined logits of the candidates
+  float* l32 = reinterpret_cast<float*>(sm_d + E);     // [E]
+  int32_t* cand = reinterpret_cast<int32_t*>(l32 + E); // [E]
+  __shared__ double red[8][8];
+  __shared__ float redf[8];
+  __shared__ float thr_s;
+  __shared__ int ncand_s;
+  const int t = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
+  // zero this token's row of the fp32 combine accumulator
+  for (int i = tid; i < H / 4; i += 256)
+    reinterpret_cast<float4*>(y32 + (size_t)t * H)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  // ---- fp32 logits of this token and the norms for the error bound
+  for (int e = tid; e < E; e += 256) {
+    const float* pp = part + (size_t)t * E + e;
+    const size_t cs = (size_t)gamma * E;
+    float s = 0.f;
+    int c = 0;
+    for (; c + 8 <= n_slices; c += 8) {
+      float v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) v[i] = __ldg(pp + (size_t)(c + i) * cs);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) s += v[i];
+    }
+    for (; c < n_slices; ++c) s += __ldg(pp + (size_t)c * cs);
+    l32[e] = s;
+  }
+  float x2 = 0.f, w2 = 0.f;
+  for (int c = tid; c < n_slices; c += 256) {
+    x2 += part_x2[(size_t)c * gamma + t];
+    w2 += part_w2max[c];
+  }
+  x2 = warp_sum(x2);
+  w2 = warp_sum(w2);
+  if (lane == 0) { redf[warp] = x2; red[warp][0] = (double)w2; }
   __syncthreads();
-
-  // ---- phase 1: top-k per token
-  constexpr int PL = kMaxE / 32;
-  for (int t = warp; t < gamma; t += nwarps) {
-    double v[PL];
+  if (warp == 0) {
+    float xs = 0.f, wm = 0.f;
+    for (int w = 0; w < 8; ++w) { xs += redf[w]; wm += (float)red[w][0]; }
+    // |fp32 logit - exact| <= gamma_n * sum|x w| <= n u ||x|| ||w||, n = roundings on the longest path
+    // (slice length + number of slices + the norm sums' own error, covered by the factor 1.25)
+    const float n_round = (float)(kRouterKS + n_slices + 4);
+    const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
+    // ---- fp32 top-k: value of the k-th largest logit
+    constexpr int PL = kMaxE / 32;
+    float v[PL];
     uint32_t taken = 0;
 #pragma unroll
     for (int i = 0; i < PL; ++i) {
       int e = i * 32 + lane;
-      if (e < E) v[i] = T.logits[(size_t)t * E + e];
-      else { v[i] = 0.0; taken |= 1u << i; }
+      if (e < E) v[i] = l32[e];
+      else { v[i] = 0.f; taken |= 1u << i; }
     }
-    double sel_v = 0.0;
-    int sel_e = -1;
+    float kth = 0.f;
     for (int j = 0; j < k; ++j) {
-      double bv = 0.0;
-      int be = 0x7fffffff;  // "no candidate"
+      float bv = 0.f;
+      int be = 0x7fffffff;
 #pragma unroll
       for (int i = 0; i < PL; ++i)
         if (!((taken >> i) & 1u) && (be == 0x7fffffff || v[i] > bv)) { bv = v[i]; be = i * 32 + lane; }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
-        double ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        float ov = __shfl_xor_sync(0xffffffffu, bv, o);
         int oe = __shfl_xor_sync(0xffffffffu, be, o);
         bool better = (oe != 0x7fffffff) && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be));
         if (better) { bv = ov; be = oe; }
       }
       if ((be & 31) == lane) taken |= 1u << (be >> 5);
-      if (lane == j) { sel_v = bv; sel_e = be; }
+      kth = bv;
+    }
+    // ---- candidates: every expert whose exact logit may be >= the exact k-th largest
+    const float thr = kth - 2.f * eps;
+    int n = 0;
+    for (int e0 = 0; e0 < E; e0 += 32) {
+      int e = e0 + lane;
+      bool in = e < E && l32[e] >= thr;
+      uint32_t m = __ballot_sync(0xffffffffu, in);
+      if (in) cand[n + __popc(m & ((1u << lane) - 1u))] = e;
+      n += __popc(m);
+    }
+    if (lane == 0) { ncand_s = n; thr_s = thr; }
+  }
+  __syncthreads();
+  const int ncand = ncand_s;
+
+  // ---- exact (fp64) logits of the candidates, 8 at a time; every thread owns chunks of 8 columns
+  float amax = 0.f;
+  for (int c0 = 0; c0 < ncand; c0 += 8) {
+    double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const int nc = min(8, ncand - c0);
+    for (int h8 = tid; h8 < H / 8; h8 += 256) {
+      double xv[8];
+      if constexpr (AFMT == MOEV_ACT_BF16) {
+        uint4 v = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + h8);
+        uint32_t wd[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          xv[2 * i] = bf16_bits_to_double(wd[i] & 0xffffu);
+          xv[2 * i + 1] = bf16_bits_to_double(wd[i] >> 16);
+          if (c0 == 0) amax = fmaxf(amax, fmaxf(fabsf(__uint_as_float(wd[i] << 16)), fabsf(__uint_as_float(wd[i] & 0xffff0000u))));
+        }
+      } else {
+        float f[8];
+        load_act8<AFMT>(x, (size_t)t * H + 8 * (size_t)h8, f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { xv[i] = (double)f[i]; if (c0 == 0) amax = fmaxf(amax, fabsf(f[i])); }
+      }
+      float4 wa[8], wb[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        if (q < nc) {
+          const float4* wp = reinterpret_cast<const float4*>(router_w + (size_t)cand[c0 + q] * H) + 2 * h8;
+          wa[q] = __ldg(wp);
+          wb[q] = __ldg(wp + 1);
+        }
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        if (q < nc) {
+          acc[q] = fma(xv[0], (double)wa[q].x, acc[q]); acc[q] = fma(xv[1], (double)wa[q].y, acc[q]);
+          acc[q] = fma(xv[2], (double)wa[q].z, acc[q]); acc[q] = fma(xv[3], (double)wa[q].w, acc[q]);
+          acc[q] = fma(xv[4], (double)wb[q].x, acc[q]); acc[q] = fma(xv[5], (double)wb[q].y, acc[q]);
+          acc[q] = fma(xv[6], (double)wb[q].z, acc[q]); acc[q] = fma(xv[7], (double)wb[q].w, acc[q]);
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      double a = warp_sum(acc[q]);
+      if (lane == 0) red[warp][q] = a;
+    }
+    __syncthreads();
+    if (tid < nc) {
+      double a = 0.0;
+      for (int w = 0; w < 8; ++w) a += red[w][tid];
+      L[c0 + tid] = a;
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  if (lane == 0) redf[warp] = amax;
+  __syncthreads();
+
+  // ---- exact ranking of the candidates and the router weights (warp 0)
+  if (warp == 0) {
+    if (lane == 0) {
+      float am = 0.f;
+      for (int w = 0; w < 8; ++w) am = fmaxf(am, redf[w]);
+      int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
+      ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
+      T.tok_scale[t] = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
+    }
+    double sel_v = 0.0;
+    int sel_e = -1;
+    // candidates are stored in ascending id; lane owns candidates lane, lane+32, ...
+    uint32_t taken = 0;  // bit i: candidate lane + 32 i already selected (ncand <= 512 -> 16 bits)
+    for (int j = 0; j < k; ++j) {
+      double bv = 0.0;
+      int be = 0x7fffffff, bi = -1;
+      for (int i = 0; lane + 32 * i < ncand; ++i) {
+        if ((taken >> i) & 1u) continue;
+        double val = L[lane + 32 * i];
+        int e = cand[lane + 32 * i];
+        if (be == 0x7fffffff || val > bv) { bv = val; be = e; bi = i; }
+      }
+      double wv = bv;
+      int we = be;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        double ov = __shfl_xor_sync(0xffffffffu, wv, o);
+        int oe = __shfl_xor_sync(0xffffffffu, we, o);
+        bool better = (oe != 0x7fffffff) && (we == 0x7fffffff || ov > wv || (ov == wv && oe < we));
+        if (better) { wv = ov; we = oe; }
+      }
+      if (we == be && bi >= 0) taken |= 1u << bi;
+      if (lane == j) { sel_v = wv; sel_e = we; }
     }
     double wgt = 0.0;
     if (score == MOEV_SCORE_SOFTMAX) {
@@ -132,20 +325,43 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       double den = warp_sum(ex);
       wgt = ex / den;
     } else {
-      double s = lane < k ? 1.0 / (1.0 + exp(-sel_v)) : 0.0;
-      double den = warp_sum(s);
-      wgt = (double)routed_scale * s / (den + 1e-20);
+      double sg = lane < k ? 1.0 / (1.0 + exp(-sel_v)) : 0.0;
+      double den = warp_sum(sg);
+      wgt = (double)routed_scale * sg / (den + 1e-20);
     }
     if (lane < k) {
       int a = t * k + lane;
-      ids_s[a] = sel_e;
-      w_s[a] = (float)wgt;
       T.topk_ids[a] = sel_e;
       T.topk_w[a] = (float)wgt;
       if (O.topk_ids) O.topk_ids[a] = sel_e;
       if (O.topk_w) O.topk_w[a] = (float)wgt;
-      atomicAdd(&cnt[sel_e], 1);
     }
+  }
+}
+
+// One CTA (1024 threads): per-expert histogram of the selected ids, block scan over the E
+// counts (ascending union and offsets), FFN work units, then one warp per expert walks the
+// assignments in order with ballots and writes the stable permutation.
+// Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A].
+__global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O, int gamma, int E,
+                                                           int k, int n_shared, int unit_cap) {
+  extern __shared__ int32_t sm[];
+  const int A = gamma * k;
+  int32_t* cnt = sm;
+  int32_t* excl = sm + E;
+  int32_t* uidx = sm + 2 * E;
+  int32_t* ids_s = sm + 3 * E;
+  float* w_s = reinterpret_cast<float*>(sm + 3 * E + A);
+  __shared__ int32_t warp_tot_cnt[32], warp_tot_flag[32], warp_tot_unit[32], n_union_s;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
+  __syncthreads();
+  for (int a = tid; a < A; a += blockDim.x) {
+    int e = T.topk_ids[a];
+    ids_s[a] = e;
+    w_s[a] = T.topk_w[a];
+    atomicAdd(&cnt[e], 1);
   }
   __syncthreads();
 
@@ -211,22 +427,28 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
     if (tid == blockDim.x - 1) *T.n_units = base + sc;
   }
 
-  // ---- phase 3: stable permutation, one warp per expert
-  for (int e = warp; e < E; e += nwarps) {
-    if (cnt[e] == 0) continue;
-    int base = excl[e];
+  // ---- phase 3: stable permutation.  Warp 0 walks the assignments in order, 32 at a time;
+  // uidx[] is reused as the running count of slots already handed out per expert.
+  __syncthreads();
+  for (int e = tid; e < E; e += blockDim.x) uidx[e] = 0;
+  __syncthreads();
+  if (warp == 0) {
     for (int a0 = 0; a0 < A; a0 += 32) {
-      int a = a0 + lane;
-      bool match = a < A && ids_s[a] == e;
-      uint32_t m = __ballot_sync(0xffffffffu, match);
-      if (match) {
-        int pos = base + __popc(m & ((1u << lane) - 1u));
+      const int a = a0 + lane;
+      const bool valid = a < A;
+      const int e = valid ? ids_s[a] : -1 - lane;  // distinct dummies for idle lanes
+      const uint32_t same = __match_any_sync(0xffffffffu, e);
+      if (valid) {
+        const int before = __popc(same & ((1u << lane) - 1u));
+        const int pos = excl[e] + uidx[e] + before;
         T.perm[pos] = a;
         T.slot_token[pos] = a / k;
         T.slot_w[pos] = w_s[a];
         if (O.perm) O.perm[pos] = a;
       }
-      base += __popc(m);
+      __syncwarp();
+      if (valid && (same & ((1u << lane) - 1u)) == 0) uidx[e] += __popc(same);  // lowest lane of each group
+      __syncwarp();
     }
   }
 }
