@@ -40,6 +40,7 @@ struct Tables {
   float* tok_scale;    // [gamma] power of two bringing the token's max |x| into [64,128)
   Unit* units;         // [max_units]
   int32_t* n_units;    // [1]
+  int32_t* task_counter; // [1] dynamic task scheduler of the tensor-core FFN, zeroed per call
   int32_t* status;     // [1]   kStatusOk / kStatusTimeout
 };
 

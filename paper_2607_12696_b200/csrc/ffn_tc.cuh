@@ -1,19 +1,22 @@
 // Tensor-core grouped expert FFN for sm_100a: one persistent, warp-specialised kernel.
 //
-// Work decomposition.  A *unit* is (expert, chunk of at most MC of its tokens); a *task* is
-// (unit, 128-row slice of the intermediate dimension I).  Tasks are dealt round-robin to the
-// persistent CTAs (one per SM).  For its task a CTA
+// Work decomposition.  A *unit* is (expert, run of at most MC of its tokens); a *task* is
+// (unit, 128-row slice of the intermediate dimension I).  Tasks are handed out dynamically
+// (one atomic counter) to the persistent CTAs, one per SM; ids are ordered so that the two
+// slices 2s, 2s+1 of a unit are taken back to back by two CTAs, which then read the two
+// 128-byte halves of the same 256-byte runs of W_down at about the same time.  For its task
+// a CTA
 //   1. streams the 128 x H slices of W_gate and W_up through a TMA ring (K chunks of 128 bytes)
 //      and accumulates  G = Wg_slice * X^T,  P = Wu_slice * X^T  in TMEM with tcgen05.mma
 //      (weights are the M operand, the unit's tokens the N operand);
 //   2. the epilogue warps read G and P from TMEM, form h = silu(G) * P and write it to shared
 //      memory as the N operand of the down projection;
 //   3. streams the H x 128 column slice of W_down (128 x 128 tiles) through the same ring and
-//      computes each 128-row tile of  O = Wd[:, slice] * h  into a double-buffered TMEM
-//      accumulator; the epilogue scales by the routing weight and reduce-adds into the fp32
-//      output accumulator y32 (split-K over the I slices).
+//      computes each 128-row tile of  O = Wd[:, slice] * h  into TMEM accumulators (two ring
+//      stages in flight); the epilogue scales by the routing weight and reduce-adds into the
+//      fp32 output accumulator y32 (split-K over the I slices).
 // Every weight byte of an active expert is fetched from HBM by exactly one TMA load per unit
-// (units of one expert run back to back on neighbouring CTAs, so extra chunks hit L2).
+// (units of one expert are adjacent in task order, so extra token runs hit L2).
 //
 // Formats.  BF16 weights: kind::f16 with the bf16 activations as they are.  FP8 (e4m3 with
 // fp32 scales per 128 x 128 block): kind::f8f6f4 on the untouched weight bytes; the bf16
@@ -23,9 +26,9 @@
 // epilogue; h is split the same way and the down-projection block scale (again one scalar per
 // 128 x 128 tile) is applied in the epilogue.
 //
-// Warps: 0 = TMA producer, 1 = MMA issuer, 2..5 = epilogue (TMEM lane quarters), 6..9 =
-// activation producers.  All mbarrier waits are bounded; on expiry the CTA raises an abort
-// flag, writes the timeout status word and every role leaves its loop.
+// Warps: 0 = TMA producer + task scheduler, 1 = MMA issuer, 2..5 = epilogue (TMEM lane
+// quarters), 6..9 = activation producers.  All mbarrier waits are bounded; on expiry the CTA
+// raises an abort flag, writes the timeout status word and every role leaves its loop.
 #pragma once
 #include <cuda.h>
 
@@ -40,16 +43,19 @@ constexpr int kStages = 5;                  // weight ring
 constexpr int kStageBytes = 32 * 1024;      // two 128 x 128-byte tiles
 constexpr int kBSlots = 3;                  // activation-operand ring
 constexpr int kNMax = 64;                   // widest N operand
-constexpr int kTmemCols = 256;              // G 64 | P 64 | O[0] 64 | O[1] 64
+constexpr int kTaskQ = 4;                   // depth of the task-id queue between the roles
+constexpr int kTmemCols = 512;              // G 64 | P 64 | O[2 stages][<=2 tiles] 64 each
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // 2 s per wait
 
-// tiles (fp8: 160 + 48 + 8 KB, bf16: 160 + 24 + 16 KB) + 1 KB alignment slack + 4 KB control block
+// tiles (fp8: 160 + 48 + 8 KB, bf16: 160 + 24 + 16 KB) + 1 KB alignment slack + 8 KB control block
 constexpr int kTileBytes = kStages * kStageBytes + 56 * 1024;
-constexpr int kSmemBytes = kTileBytes + 1024 + 4096;
+constexpr int kCtlBytes = 8 * 1024;
+constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
 
 struct Params {
   const Unit* units;
   const int32_t* n_units;
+  int32_t* task_counter;      // zeroed by the grouping kernel of the same call
   const int32_t* slot_token;  // [A]
   const float* slot_w;        // [A]
   const float* tok_scale;     // [gamma]  2^p_t, brings a token's amax into [64,128)
@@ -59,6 +65,9 @@ struct Params {
   const float *sh_s_gate, *sh_s_up, *sh_s_down;  // fp8 block scales (shared)
   int32_t* status;
   int32_t gamma, H, I, A;
+#ifdef MOEV_TC_STATS
+  unsigned long long* stats;  // [grid][8] cycles the MMA thread spent per wait class (debug builds)
+#endif
 };
 
 struct Smem {
@@ -66,20 +75,23 @@ struct Smem {
   uint64_t b_full[kBSlots], b_empty[kBSlots];
   uint64_t acc_full, acc_empty, h_full, h_empty;
   uint64_t d_full[2], d_empty[2];
-  uint64_t ep_bar, pr_bar;  // group barriers (128 threads each), bounded like every other wait
+  uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
+  uint64_t ep_bar;  // epilogue group barrier (128 threads), bounded like every other wait
+  volatile int32_t tq_task[kTaskQ];
   uint32_t tmem_base;
   volatile int abort_flag;
-  // activation-producer private
-  int32_t p_tok[kNMax];
-  float p_tscale[kNMax];
-  float p_sg[128], p_su[128];      // per K chunk: block scale * 2^p (fp8)
-  float p_wmax[2][4];
-  float pscale_inv[2][2];          // [task parity][gate, up]: 2^-p, read by the epilogue
-  // epilogue private
-  int32_t e_tok[kNMax];
-  float e_f[kNMax];                // routing weight (* 2^(e_r-6) for fp8)
-  float e_inv[kNMax];              // 1 / tok_scale
-  float e_sd[128];                 // down block scale per H tile (fp8)
+  // activation-producer tables, double-buffered by task parity; every producer warp writes
+  // all entries itself (identical values), so no cross-warp synchronisation is needed
+  int32_t p_tok[2][kNMax];
+  float p_tscale[2][kNMax];
+  float p_sg[2][128], p_su[2][128];  // per K chunk: block scale * 2^-p (fp8)
+  float pscale_inv[2][2];            // [task parity][gate, up]: 2^p, read by the epilogue
+  // epilogue tables, same scheme
+  int32_t e_tok[2][kNMax];
+  float e_w[2][kNMax];               // routing weight
+  float e_inv[2][kNMax];             // 1 / tok_scale
+  float e_sd[2][128];                // down block scale per H tile (fp8)
+  float e_f[kNMax];                  // routing weight * 2^(e_r - 6) (fp8), identical writes by all warps
   uint32_t e_amax[4][32];
 };
 
@@ -90,33 +102,36 @@ __device__ __forceinline__ float pow2i(int n) {  // 2^n, n clamped to the normal
   n = n < -126 ? -126 : (n > 127 ? 127 : n);
   return __uint_as_float((uint32_t)(n + 127) << 23);
 }
+__device__ __forceinline__ int safe_exponent(float a) {
+  int e = (a > 0.f && a < 3.0e38f) ? exponent_of(a) : 0;
+  return e < -100 ? -100 : (e > 100 ? 100 : e);
+}
 
-// Split 16 floats into e4m3 hi and lo (= (v - hi) * 16) codes, 16 bytes each.
-__device__ __forceinline__ void split_e4m3(const float (&v)[16], uint4& hi, uint4& lo) {
-  uint32_t h[4], l[4];
+// Split 4 floats into e4m3 hi and lo (= (v - hi) * 16) codes, 4 bytes each.
+__device__ __forceinline__ void split4_e4m3(const float (&v)[4], uint32_t& hi, uint32_t& lo) {
+  hi = 0; lo = 0;
 #pragma unroll
-  for (int w = 0; w < 4; ++w) {
-    uint32_t hw = 0, lw = 0;
-#pragma unroll
-    for (int p = 0; p < 2; ++p) {
-      float a = v[4 * w + 2 * p], b = v[4 * w + 2 * p + 1];
-      __nv_fp8x2_storage_t hc = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
-      __half2_raw hr = __nv_cvt_fp8x2_to_halfraw2(hc, __NV_E4M3);
-      float2 hf = __half22float2(*reinterpret_cast<__half2*>(&hr));
-      __nv_fp8x2_storage_t lc = __nv_cvt_float2_to_fp8x2(make_float2((a - hf.x) * 16.f, (b - hf.y) * 16.f),
-                                                         __NV_SATFINITE, __NV_E4M3);
-      hw |= (uint32_t)hc << (16 * p);
-      lw |= (uint32_t)lc << (16 * p);
-    }
-    h[w] = hw;
-    l[w] = lw;
+  for (int p = 0; p < 2; ++p) {
+    float a = v[2 * p], b = v[2 * p + 1];
+    __nv_fp8x2_storage_t hc = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
+    __half2_raw hr = __nv_cvt_fp8x2_to_halfraw2(hc, __NV_E4M3);
+    float2 hf = __half22float2(*reinterpret_cast<__half2*>(&hr));
+    __nv_fp8x2_storage_t lc = __nv_cvt_float2_to_fp8x2(make_float2((a - hf.x) * 16.f, (b - hf.y) * 16.f),
+                                                       __NV_SATFINITE, __NV_E4M3);
+    hi |= (uint32_t)hc << (16 * p);
+    lo |= (uint32_t)lc << (16 * p);
   }
-  hi = make_uint4(h[0], h[1], h[2], h[3]);
-  lo = make_uint4(l[0], l[1], l[2], l[3]);
 }
 
 // byte offset of 16-byte chunk c of row r in a [rows x 128 B] tile with the 128-byte swizzle
 __device__ __forceinline__ uint32_t sw128(int r, int c) { return (uint32_t)r * 128u + (uint32_t)((c ^ (r & 7)) << 4); }
+
+// Wait used by the multi-thread roles: the outcome is made warp-uniform (and the warp
+// reconverged) so that the .sync.aligned tcgen05 instructions that follow see all 32 lanes.
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abortp, int* status) {
+  bool ok = ptx::bounded_wait(bar, parity, abortp, status, kStatusTimeout, kWaitBudgetNs);
+  return __all_sync(0xffffffffu, ok);
+}
 
 // Barrier among the 128 threads of one role group, built on an mbarrier so that it is bounded.
 __device__ __forceinline__ bool group_sync(uint64_t* bar, uint32_t& phase, volatile int* abortp, int* status) {
@@ -126,12 +141,13 @@ __device__ __forceinline__ bool group_sync(uint64_t* bar, uint32_t& phase, volat
   return __all_sync(0xffffffffu, ok);
 }
 
-// Wait used by the multi-thread roles: the outcome is made warp-uniform (and the warp
-// reconverged) so that the .sync.aligned tcgen05 instructions that follow see all 32 lanes.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abortp, int* status) {
-  bool ok = ptx::bounded_wait(bar, parity, abortp, status, kStatusTimeout, kWaitBudgetNs);
-  return __all_sync(0xffffffffu, ok);
-}
+#ifdef MOEV_TC_STATS
+#define MOEV_STAT_BEGIN() long long _t0 = clock64()
+#define MOEV_STAT_END(i) st_acc[i] += (unsigned long long)(clock64() - _t0)
+#else
+#define MOEV_STAT_BEGIN()
+#define MOEV_STAT_END(i)
+#endif
 
 template <int WFMT>
 struct Fmt;
@@ -162,6 +178,31 @@ __device__ __forceinline__ void issue_mma(uint32_t d, uint64_t a, uint64_t b, ui
   else ptx::mma_f8f6f4(d, a, b, idesc, acc);
 }
 
+// Task id -> (unit index, slice).  Ids enumerate (slice pair, unit, half) with the half
+// fastest; slice = 2 * pair + half may fall past the end when the slice count is odd.
+struct TaskDesc { int unit, slice; bool valid; };
+__device__ __forceinline__ TaskDesc decode_task(int id, int n_units, int n_slices) {
+  TaskDesc t;
+  const int pair = id >> 1;
+  t.unit = pair % n_units;
+  t.slice = (pair / n_units) * 2 + (id & 1);
+  t.valid = t.slice < n_slices;
+  return t;
+}
+
+// Consumer side of the task queue: returns the next task id, -1 when the work is done and
+// -2 when the wait was abandoned.
+__device__ __forceinline__ int next_task(Smem& S, uint32_t& q, volatile int* abortp, int* status, bool whole_warp) {
+  const int slot = q % kTaskQ;
+  bool ok = whole_warp ? warp_wait(&S.tq_full[slot], (q / kTaskQ) & 1, abortp, status)
+                       : ptx::bounded_wait(&S.tq_full[slot], (q / kTaskQ) & 1, abortp, status, kStatusTimeout, kWaitBudgetNs);
+  if (!ok) return -2;
+  const int id = S.tq_task[slot];
+  ptx::mbar_arrive(&S.tq_empty[slot]);
+  ++q;
+  return id;
+}
+
 template <int WFMT>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_constant__ CUtensorMap tm_up,
@@ -170,6 +211,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
                       const Params P) {
   using F = Fmt<WFMT>;
   constexpr bool kFp8 = WFMT == MOEV_W_FP8E4M3_B128;
+  constexpr int TPS = F::kDownTilesPerStage;
   extern __shared__ uint8_t smem_raw[];
   // 1024-byte alignment for the swizzled tiles
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -178,7 +220,8 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   constexpr int kBSlotBytes = F::kBSlotBytes;
   uint8_t* h_tile = b_ring + kBSlots * kBSlotBytes;
   static_assert(kStages * kStageBytes + kBSlots * F::kBSlotBytes + F::kHTileBytes <= kTileBytes, "tile budget");
-  static_assert(sizeof(Smem) <= 4096, "control block budget");
+  static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
+  static_assert(128 + 2 * TPS * 64 <= kTmemCols, "TMEM budget");
   Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -186,6 +229,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   const int KC = H / F::kBK;        // K chunks of the gate/up phase
   const int HT = H / 128;           // 128-row tiles of the down phase
   const int n_slices = I / 128;
+  const int n_dstage = (HT + TPS - 1) / TPS;
 
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 1); }
@@ -193,7 +237,8 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     ptx::mbar_init(&S.acc_full, 1); ptx::mbar_init(&S.acc_empty, 128);
     ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 1);
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 1); ptx::mbar_init(&S.d_empty[i], 128); }
-    ptx::mbar_init(&S.ep_bar, 128); ptx::mbar_init(&S.pr_bar, 128);
+    for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 257); }
+    ptx::mbar_init(&S.ep_bar, 128);
     S.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -206,18 +251,36 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   ptx::tc_fence_after();
   const uint32_t tmem = S.tmem_base;
   const int n_units = *P.n_units;
-  const int n_tasks = n_units * n_slices;
+  const int n_ids = n_units * ((n_slices + 1) & ~1);
   volatile int* abortp = &S.abort_flag;
 
   if (warp == 0) {
-    // ===================================================== TMA producer (one lane)
+    // ===================================================== TMA producer + scheduler (one lane)
     if (lane == 0) {
       ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
-      uint32_t it = 0;  // ring use counter
+      uint32_t it = 0, q = 0;
       bool ok = true;
-      for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x) {
-        const Unit u = P.units[task % n_units];
-        const int slice = task / n_units;
+      while (ok) {
+        // fetch the next valid task id and publish it to the other roles
+        int id;
+        TaskDesc td;
+        td.unit = 0; td.slice = 0; td.valid = false;
+        do {
+          id = atomicAdd(P.task_counter, 1);
+          if (id >= n_ids) { id = -1; break; }
+          td = decode_task(id, n_units, n_slices);
+        } while (!td.valid);
+        {
+          const int slot = q % kTaskQ;
+          ok = ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          if (!ok) break;
+          S.tq_task[slot] = id;
+          ptx::mbar_arrive(&S.tq_full[slot]);
+          ++q;
+        }
+        if (id < 0) break;
+        const Unit u = P.units[td.unit];
+        const int slice = td.slice;
         const CUtensorMap* mg = u.shared ? &tm_sh_gate : &tm_gate;
         const CUtensorMap* mu = u.shared ? &tm_sh_up : &tm_up;
         const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
@@ -230,7 +293,6 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           ptx::tma_load_3d(dst, mg, &S.w_full[s], kc * F::kBK, slice * 128, u.expert, ptx::kPolicyEvictFirst);
           ptx::tma_load_3d(dst + 16384, mu, &S.w_full[s], kc * F::kBK, slice * 128, u.expert, ptx::kPolicyEvictFirst);
         }
-        const int n_dstage = (HT + F::kDownTilesPerStage - 1) / F::kDownTilesPerStage;
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
           const int s = it % kStages;
           ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
@@ -253,21 +315,34 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   } else if (warp == 1) {
     // ===================================================== MMA issuer (one lane)
     if (lane == 0) {
-      uint32_t it = 0, bit = 0, tcount = 0, htc = 0;
+      uint32_t it = 0, bit = 0, tcount = 0, dsc = 0, q = 0;
       bool ok = true;
-      for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x, ++tcount) {
-        const Unit u = P.units[task % n_units];
+#ifdef MOEV_TC_STATS
+      unsigned long long st_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      const long long st_begin = clock64();
+#endif
+      for (;; ++tcount) {
+        const int id = next_task(S, q, abortp, P.status, false);
+        if (id < 0) break;
+        const TaskDesc td = decode_task(id, n_units, n_slices);
+        const Unit u = P.units[td.unit];
         const int ncols = u.m * F::kColsPerTok;
         const uint32_t N = (uint32_t)((ncols + 15) & ~15);
         const uint32_t idesc = ptx::instr_desc(F::kKindFmt, F::kKindFmt, N);
         const uint32_t d_gate = tmem, d_up = tmem + 64;
-        ok = ptx::bounded_wait(&S.acc_empty, (tcount & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+        { MOEV_STAT_BEGIN();
+          ok = ptx::bounded_wait(&S.acc_empty, (tcount & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          MOEV_STAT_END(3); }
         if (!ok) break;
         ptx::tc_fence_after();
         for (int kc = 0; kc < KC && ok; ++kc, ++it, ++bit) {
           const int s = it % kStages, sb = bit % kBSlots;
-          ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs) &&
-               ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          { MOEV_STAT_BEGIN();
+            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(1); }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(2); }
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t wa = ptx::smem_u32(w_ring + s * kStageBytes);
@@ -284,26 +359,35 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         }
         if (!ok) break;
         ptx::mma_commit(&S.acc_full);
-        ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+        { MOEV_STAT_BEGIN();
+          ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          MOEV_STAT_END(4); }
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t ha = ptx::smem_u32(h_tile);
-        for (int ht = 0; ht < HT && ok; ++ht, ++htc) {
-          const int db = htc & 1;
+        for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc, ++it) {
+          const int db = dsc & 1;
           const int s = it % kStages;
-          const bool first_in_stage = kFp8 ? ((ht & 1) == 0) : true;
-          if (first_in_stage)
+          { MOEV_STAT_BEGIN();
             ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-          ok = ok && ptx::bounded_wait(&S.d_empty[db], ((htc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(5); }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.d_empty[db], ((dsc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(6); }
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t wa = ptx::smem_u32(w_ring + s * kStageBytes) + (kFp8 ? (ht & 1) * 16384 : 0);
-          const uint32_t d_down = tmem + 128 + db * 64;
+          const uint32_t wa = ptx::smem_u32(w_ring + s * kStageBytes);
           if constexpr (kFp8) {
+            const int nt = (2 * ds + 1 < HT) ? 2 : 1;
+            for (int tl = 0; tl < nt; ++tl) {
+              const uint32_t d_down = tmem + 128 + (db * TPS + tl) * 64;
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              issue_mma<WFMT>(d_down, ptx::smem_desc_sw128(wa + j * 32), ptx::smem_desc_sw128(ha + j * 32), idesc, j ? 1u : 0u);
+              for (int j = 0; j < 4; ++j)
+                issue_mma<WFMT>(d_down, ptx::smem_desc_sw128(wa + tl * 16384 + j * 32),
+                                ptx::smem_desc_sw128(ha + j * 32), idesc, j ? 1u : 0u);
+            }
           } else {
+            const uint32_t d_down = tmem + 128 + db * 64;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
@@ -312,43 +396,48 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
                                 ptx::smem_desc_sw128(ha + hf * 8192 + j * 32), idesc, (hf | j) ? 1u : 0u);
           }
           ptx::mma_commit(&S.d_full[db]);
-          const bool last_in_stage = kFp8 ? ((ht & 1) == 1 || ht == HT - 1) : true;
-          if (last_in_stage) { ptx::mma_commit(&S.w_empty[s]); ++it; }
+          ptx::mma_commit(&S.w_empty[s]);
         }
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
       }
+#ifdef MOEV_TC_STATS
+      st_acc[0] = (unsigned long long)(clock64() - st_begin);
+      st_acc[7] = tcount;
+      if (P.stats)
+        for (int i = 0; i < 8; ++i) P.stats[(size_t)blockIdx.x * 8 + i] = st_acc[i];
+#endif
     }
   } else if (warp < 6) {
     // ===================================================== epilogue warps (TMEM lane quarter = warp % 4)
-    const int q = warp & 3;           // warps 2,3,4,5 -> quarters 2,3,0,1
-    const int et = tid - 64;          // 0..127 within the epilogue group
-    const uint32_t lane_base = (uint32_t)(q * 32) << 16;
-    const int row = q * 32 + lane;    // row of the 128-row tile this thread owns
-    uint32_t tcount = 0, htc = 0, gph = 0;
+    const int qd = warp & 3;          // warps 2,3,4,5 -> quarters 2,3,0,1
+    const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
+    const int row = qd * 32 + lane;   // row of the 128-row tile this thread owns
+    uint32_t tcount = 0, dsc = 0, gph = 0, q = 0;
     bool ok = true;
-    for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x, ++tcount) {
-      const Unit u = P.units[task % n_units];
-      const int slice = task / n_units;
+    for (;; ++tcount) {
+      const int id = next_task(S, q, abortp, P.status, true);
+      if (id < 0) break;
+      const TaskDesc td = decode_task(id, n_units, n_slices);
+      const Unit u = P.units[td.unit];
+      const int slice = td.slice;
       const int m = u.m;
-      // previous task's down epilogues are finished by all four warps before the tables change
-      if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
-      if (et < m) {
+      const int par = tcount & 1;
+      // tables of this task: every warp writes all entries it will read (identical values)
+      for (int r = lane; r < m; r += 32) {
         int tok;
         float w;
-        if (u.shared) { tok = u.slot0 - (P.A + u.expert * P.gamma) + et; w = 1.f; }
-        else { tok = P.slot_token[u.slot0 + et]; w = P.slot_w[u.slot0 + et]; }
-        S.e_tok[et] = tok;
-        S.e_f[et] = w;
-        S.e_inv[et] = kFp8 ? 1.f / P.tok_scale[tok] : 1.f;
+        if (u.shared) { tok = u.slot0 - (P.A + u.expert * P.gamma) + r; w = 1.f; }
+        else { tok = P.slot_token[u.slot0 + r]; w = P.slot_w[u.slot0 + r]; }
+        S.e_tok[par][r] = tok;
+        S.e_w[par][r] = w;
+        S.e_inv[par][r] = kFp8 ? 1.f / P.tok_scale[tok] : 1.f;
       }
       if constexpr (kFp8) {
-        if (et < HT) {
-          const float* sd = u.shared ? P.sh_s_down : P.s_down;
-          S.e_sd[et] = sd[((size_t)u.expert * HT + et) * n_slices + slice];
-        }
+        const float* sd = u.shared ? P.sh_s_down : P.s_down;
+        for (int ht = lane; ht < HT; ht += 32) S.e_sd[par][ht] = sd[((size_t)u.expert * HT + ht) * n_slices + slice];
       }
-      if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
+      __syncwarp();
       ok = warp_wait(&S.acc_full, tcount & 1, abortp, P.status);
       if (!ok) break;
       ptx::tc_fence_after();
@@ -357,7 +446,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       if (!ok) break;
 
       if constexpr (kFp8) {
-        const float ig = S.pscale_inv[tcount & 1][0], iu = S.pscale_inv[tcount & 1][1];
+        const float ig = S.pscale_inv[par][0], iu = S.pscale_inv[par][1];
         float hv[32];
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 16) {
@@ -369,7 +458,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
               const int tr = c0 / 2 + r;
-              float inv = tr < m ? S.e_inv[tr] : 0.f;
+              float inv = tr < m ? S.e_inv[par][tr] : 0.f;
               float gg = (__uint_as_float(g[2 * r]) + __uint_as_float(g[2 * r + 1]) * 0.0625f) * (inv * ig);
               float pp = (__uint_as_float(p[2 * r]) + __uint_as_float(p[2 * r + 1]) * 0.0625f) * (inv * iu);
               hv[tr] = tr < m ? gg / (1.f + __expf(-gg)) * pp : 0.f;
@@ -394,9 +483,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         for (int r = 0; r < 32; ++r) {
           if (r < m) {
             uint32_t mx = max(max(S.e_amax[0][r], S.e_amax[1][r]), max(S.e_amax[2][r], S.e_amax[3][r]));
-            float amax = __uint_as_float(mx);
-            int er = (amax > 0.f && amax < 3.0e38f) ? exponent_of(amax) : 0;
-            er = er < -100 ? -100 : (er > 100 ? 100 : er);
+            const int er = safe_exponent(__uint_as_float(mx));
             float v = hv[r] * pow2i(6 - er);
             __nv_fp8_storage_t hc = __nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
             __half_raw hr = __nv_cvt_fp8_to_halfraw(hc, __NV_E4M3);
@@ -404,9 +491,10 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             __nv_fp8_storage_t lc = __nv_cvt_float_to_fp8((v - hf) * 16.f, __NV_SATFINITE, __NV_E4M3);
             h_tile[sw128(2 * r, row >> 4) + (row & 15)] = hc;
             h_tile[sw128(2 * r + 1, row >> 4) + (row & 15)] = lc;
-            if (et == r) S.e_f[r] *= pow2i(er - 6);  // one writer per token
+            if (lane == (r & 31)) S.e_f[r] = S.e_w[par][r] * pow2i(er - 6);  // same value from every warp
           }
         }
+        __syncwarp();
       } else {
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 16) {
@@ -434,147 +522,186 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       }
       ptx::fence_proxy_async_smem();
       ptx::mbar_arrive(&S.h_full);
-      if constexpr (kFp8) {  // e_f updates visible to all epilogue threads
-        if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
-      }
 
-      // ---- down-projection epilogues: one 128-row tile of the output per iteration
-      for (int ht = 0; ht < HT && ok; ++ht, ++htc) {
-        const int db = htc & 1;
-        ok = warp_wait(&S.d_full[db], (htc >> 1) & 1, abortp, P.status);
+      // ---- down-projection epilogues: one ring stage (TPS 128-row tiles) per iteration
+      const int ncols = m * F::kColsPerTok;
+      for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc) {
+        const int db = dsc & 1;
+        ok = warp_wait(&S.d_full[db], (dsc >> 1) & 1, abortp, P.status);
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t d_down = tmem + lane_base + 128 + db * 64;
-        float* ycol = P.y32 + (size_t)ht * 128 + row;
-        const float sd = kFp8 ? S.e_sd[ht] : 1.f;
-        const int ncols = m * F::kColsPerTok;
+        const int nt = kFp8 ? ((2 * ds + 1 < HT) ? 2 : 1) : 1;
+        for (int tl = 0; tl < nt; ++tl) {
+          const int ht = ds * TPS + tl;
+          const uint32_t d_down = tmem + lane_base + 128 + (db * TPS + tl) * 64;
+          float* ycol = P.y32 + (size_t)ht * 128 + row;
+          const float sd = kFp8 ? S.e_sd[par][ht] : 1.f;
 #pragma unroll
-        for (int c0 = 0; c0 < 64; c0 += 16) {
-          if (c0 < ncols) {
-            uint32_t o[16];
-            ptx::tmem_ld16(d_down + c0, o);
-            ptx::tmem_ld_wait();
-            if (c0 + 16 >= ncols) {  // last column chunk read: release the accumulator early
-              ptx::tc_fence_before();
-              ptx::mbar_arrive(&S.d_empty[db]);
-            }
-            if constexpr (kFp8) {
-#pragma unroll
-              for (int r = 0; r < 8; ++r) {
-                const int tr = c0 / 2 + r;
-                if (tr < m) {
-                  float val = (__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f) * (sd * S.e_f[tr]);
-                  ptx::red_add_f32(ycol + (size_t)S.e_tok[tr] * H, val);
-                }
+          for (int c0 = 0; c0 < 64; c0 += 16) {
+            if (c0 < ncols) {
+              uint32_t o[16];
+              ptx::tmem_ld16(d_down + c0, o);
+              ptx::tmem_ld_wait();
+              if (tl == nt - 1 && c0 + 16 >= ncols) {  // last read of this stage's accumulators
+                ptx::tc_fence_before();
+                ptx::mbar_arrive(&S.d_empty[db]);
               }
-            } else {
+              if constexpr (kFp8) {
 #pragma unroll
-              for (int r = 0; r < 16; ++r) {
-                const int tr = c0 + r;
-                if (tr < m) ptx::red_add_f32(ycol + (size_t)S.e_tok[tr] * H, __uint_as_float(o[r]) * S.e_f[tr]);
+                for (int r = 0; r < 8; ++r) {
+                  const int tr = c0 / 2 + r;
+                  if (tr < m) {
+                    float val = (__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f) * (sd * S.e_f[tr]);
+                    ptx::red_add_f32(ycol + (size_t)S.e_tok[par][tr] * H, val);
+                  }
+                }
+              } else {
+#pragma unroll
+                for (int r = 0; r < 16; ++r) {
+                  const int tr = c0 + r;
+                  if (tr < m) ptx::red_add_f32(ycol + (size_t)S.e_tok[par][tr] * H, __uint_as_float(o[r]) * S.e_w[par][tr]);
+                }
               }
             }
           }
         }
       }
+      if (!ok) break;
     }
   } else {
-    // ===================================================== activation producers (128 threads)
+    // ===================================================== activation producers (4 warps)
+    const int pw = warp - 6;               // producer warp 0..3
     const int pt = tid - 192;              // 0..127
-    const int r_local = pt >> 3, c = pt & 7;  // token row within a pass, 16-byte chunk of the 128-byte row
-    uint32_t bit = 0, tcount = 0, gph = 0;
+    uint32_t bit = 0, tcount = 0, q = 0;
     bool ok = true;
     const uint16_t* xb = static_cast<const uint16_t*>(P.x);
-    for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x, ++tcount) {
-      const Unit u = P.units[task % n_units];
-      const int slice = task / n_units;
+    for (;; ++tcount) {
+      const int id = next_task(S, q, abortp, P.status, true);
+      if (id < 0) break;
+      const TaskDesc td = decode_task(id, n_units, n_slices);
+      const Unit u = P.units[td.unit];
+      const int slice = td.slice;
       const int m = u.m;
-      // everyone is done with the previous task's tables
-      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) break;
-      if (pt < m) {
-        int tok = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma) + pt) : P.slot_token[u.slot0 + pt];
-        S.p_tok[pt] = tok;
-        S.p_tscale[pt] = kFp8 ? P.tok_scale[tok] : 1.f;
+      const int par = tcount & 1;
+      // tables of this task; every warp writes every entry (identical values), then reads its own
+      for (int r = lane; r < m; r += 32) {
+        int tok = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma) + r) : P.slot_token[u.slot0 + r];
+        S.p_tok[par][r] = tok;
+        S.p_tscale[par][r] = kFp8 ? P.tok_scale[tok] : 1.f;
       }
       if constexpr (kFp8) {
         // block scales of this task's row block, one per K chunk; common power of two from their max
         const float* sg = (u.shared ? P.sh_s_gate : P.s_gate) + ((size_t)u.expert * n_slices + slice) * KC;
         const float* su = (u.shared ? P.sh_s_up : P.s_up) + ((size_t)u.expert * n_slices + slice) * KC;
-        float vg = pt < KC ? sg[pt] : 0.f, vu = pt < KC ? su[pt] : 0.f;
-        uint32_t mg = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(vg)));
-        uint32_t mu = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(vu)));
-        if (lane == 0) { S.p_wmax[0][warp - 6] = __uint_as_float(mg); S.p_wmax[1][warp - 6] = __uint_as_float(mu); }
-        if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) break;
-        float amg = fmaxf(fmaxf(S.p_wmax[0][0], S.p_wmax[0][1]), fmaxf(S.p_wmax[0][2], S.p_wmax[0][3]));
-        float amu = fmaxf(fmaxf(S.p_wmax[1][0], S.p_wmax[1][1]), fmaxf(S.p_wmax[1][2], S.p_wmax[1][3]));
-        int eg = (amg > 0.f && amg < 3.0e38f) ? exponent_of(amg) : 0;
-        int eu = (amu > 0.f && amu < 3.0e38f) ? exponent_of(amu) : 0;
-        eg = eg < -100 ? -100 : (eg > 100 ? 100 : eg);
-        eu = eu < -100 ? -100 : (eu > 100 ? 100 : eu);
-        if (pt < KC) { S.p_sg[pt] = vg * pow2i(-eg); S.p_su[pt] = vu * pow2i(-eu); }
-        if (pt == 0) { S.pscale_inv[tcount & 1][0] = pow2i(eg); S.pscale_inv[tcount & 1][1] = pow2i(eu); }
-      }
-      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) break;
-
-      const int passes = (m + 15) >> 4;
-      // x rows of the first pass are fetched one K chunk ahead (L2 latency off the critical path)
-      constexpr int kXBytes = kFp8 ? 256 : 128;  // bytes of one token row per K chunk
-      uint4 n0 = make_uint4(0, 0, 0, 0), n1 = n0;
-      const uint8_t* xrow0 = nullptr;
-      if (r_local < m) {
-        xrow0 = reinterpret_cast<const uint8_t*>(xb + (size_t)S.p_tok[r_local] * H) + c * (kFp8 ? 32 : 16);
-        n0 = __ldg(reinterpret_cast<const uint4*>(xrow0));
-        if constexpr (kFp8) n1 = __ldg(reinterpret_cast<const uint4*>(xrow0) + 1);
-      }
-      for (int kc = 0; kc < KC && ok; ++kc, ++bit) {
-        const int sb = bit % kBSlots;
-        uint4 c0q = n0, c1q = n1;
-        if (xrow0 && kc + 1 < KC) {
-          const uint4* nx = reinterpret_cast<const uint4*>(xrow0 + (size_t)(kc + 1) * kXBytes);
-          n0 = __ldg(nx);
-          if constexpr (kFp8) n1 = __ldg(nx + 1);
+        float vg[4], vu[4];
+        float mg = 0.f, mu = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int kc = lane + 32 * i;
+          vg[i] = kc < KC ? __ldg(sg + kc) : 0.f;
+          vu[i] = kc < KC ? __ldg(su + kc) : 0.f;
+          mg = fmaxf(mg, fabsf(vg[i]));
+          mu = fmaxf(mu, fabsf(vu[i]));
         }
-        ok = warp_wait(&S.b_empty[sb], ((bit / kBSlots) & 1) ^ 1, abortp, P.status);
-        if (!ok) break;
-        uint8_t* tile = b_ring + sb * kBSlotBytes;
-        for (int ps = 0; ps < passes; ++ps) {
-          const int r = ps * 16 + r_local;
-          if (r < m) {
-            if (ps > 0) {
-              const uint4* src = reinterpret_cast<const uint4*>(
-                  reinterpret_cast<const uint8_t*>(xb + (size_t)S.p_tok[r] * H) + c * (kFp8 ? 32 : 16) + (size_t)kc * kXBytes);
-              c0q = __ldg(src);
-              if constexpr (kFp8) c1q = __ldg(src + 1);
+        mg = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mg)));
+        mu = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mu)));
+        const int eg = safe_exponent(mg), eu = safe_exponent(mu);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int kc = lane + 32 * i;
+          if (kc < KC) { S.p_sg[par][kc] = vg[i] * pow2i(-eg); S.p_su[par][kc] = vu[i] * pow2i(-eu); }
+        }
+        if (lane == 0) { S.pscale_inv[par][0] = pow2i(eg); S.pscale_inv[par][1] = pow2i(eu); }
+      }
+      __syncwarp();
+
+      if constexpr (kFp8) {
+        // warp pw converts token rows pw, pw+4, ...; lane owns 4 consecutive elements of the
+        // 128-element chunk.  All rows of the next chunk are fetched before this one is converted.
+        constexpr int kMaxPass = Fmt<MOEV_W_FP8E4M3_B128>::kMC / 4;
+        const int passes = (m - pw + 3) >> 2;  // rows pw + 4 i < m
+        uint2 nxt[kMaxPass];
+        const uint8_t* xrow[kMaxPass];
+#pragma unroll
+        for (int i = 0; i < kMaxPass; ++i) {
+          nxt[i] = make_uint2(0, 0);
+          xrow[i] = nullptr;
+          if (i < passes) {
+            xrow[i] = reinterpret_cast<const uint8_t*>(xb + (size_t)S.p_tok[par][pw + 4 * i] * H) + lane * 8;
+            nxt[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i]));
+          }
+        }
+        for (int kc = 0; kc < KC && ok; ++kc, ++bit) {
+          const int sb = bit % kBSlots;
+          uint2 cur[kMaxPass];
+#pragma unroll
+          for (int i = 0; i < kMaxPass; ++i) {
+            cur[i] = nxt[i];
+            if (i < passes && kc + 1 < KC) nxt[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + (size_t)(kc + 1) * 256));
+          }
+          ok = warp_wait(&S.b_empty[sb], ((bit / kBSlots) & 1) ^ 1, abortp, P.status);
+          if (!ok) break;
+          uint8_t* tile = b_ring + sb * kBSlotBytes;
+          const float sgc = S.p_sg[par][kc], suc = S.p_su[par][kc];
+#pragma unroll
+          for (int i = 0; i < kMaxPass; ++i) {
+            if (i < passes) {
+              const int r = pw + 4 * i;
+              const float ts = S.p_tscale[par][r];
+              float v[4], f[4];
+              v[0] = __uint_as_float(cur[i].x << 16) * ts;
+              v[1] = __uint_as_float(cur[i].x & 0xffff0000u) * ts;
+              v[2] = __uint_as_float(cur[i].y << 16) * ts;
+              v[3] = __uint_as_float(cur[i].y & 0xffff0000u) * ts;
+              uint32_t hi, lo;
+              const uint32_t off_hi = sw128(2 * r, lane >> 2) + (lane & 3) * 4;
+              const uint32_t off_lo = sw128(2 * r + 1, lane >> 2) + (lane & 3) * 4;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) f[e] = v[e] * sgc;
+              split4_e4m3(f, hi, lo);
+              *reinterpret_cast<uint32_t*>(tile + off_hi) = hi;
+              *reinterpret_cast<uint32_t*>(tile + off_lo) = lo;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) f[e] = v[e] * suc;
+              split4_e4m3(f, hi, lo);
+              *reinterpret_cast<uint32_t*>(tile + 8192 + off_hi) = hi;
+              *reinterpret_cast<uint32_t*>(tile + 8192 + off_lo) = lo;
             }
-            if constexpr (kFp8) {
-              const float ts = S.p_tscale[r];
-              uint32_t wds[8] = {c0q.x, c0q.y, c0q.z, c0q.w, c1q.x, c1q.y, c1q.z, c1q.w};
-              float v[16], f[16];
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                v[2 * i] = __uint_as_float(wds[i] << 16) * ts;
-                v[2 * i + 1] = __uint_as_float(wds[i] & 0xffff0000u) * ts;
-              }
-              uint4 hi, lo;
-              const float sgc = S.p_sg[kc], suc = S.p_su[kc];
-#pragma unroll
-              for (int i = 0; i < 16; ++i) f[i] = v[i] * sgc;
-              split_e4m3(f, hi, lo);
-              *reinterpret_cast<uint4*>(tile + sw128(2 * r, c)) = hi;
-              *reinterpret_cast<uint4*>(tile + sw128(2 * r + 1, c)) = lo;
-#pragma unroll
-              for (int i = 0; i < 16; ++i) f[i] = v[i] * suc;
-              split_e4m3(f, hi, lo);
-              *reinterpret_cast<uint4*>(tile + 8192 + sw128(2 * r, c)) = hi;
-              *reinterpret_cast<uint4*>(tile + 8192 + sw128(2 * r + 1, c)) = lo;
-            } else {
+          }
+          ptx::fence_proxy_async_smem();
+          ptx::mbar_arrive(&S.b_full[sb]);
+        }
+      } else {
+        // bf16: plain copy of the token rows; thread (row r_local within a pass, 16-byte chunk c)
+        const int r_local = pt >> 3, c = pt & 7;
+        const int passes = (m + 15) >> 4;
+        uint4 n0 = make_uint4(0, 0, 0, 0);
+        const uint8_t* xrow0 = nullptr;
+        if (r_local < m) {
+          xrow0 = reinterpret_cast<const uint8_t*>(xb + (size_t)S.p_tok[par][r_local] * H) + c * 16;
+          n0 = __ldg(reinterpret_cast<const uint4*>(xrow0));
+        }
+        for (int kc = 0; kc < KC && ok; ++kc, ++bit) {
+          const int sb = bit % kBSlots;
+          uint4 c0q = n0;
+          if (xrow0 && kc + 1 < KC) n0 = __ldg(reinterpret_cast<const uint4*>(xrow0 + (size_t)(kc + 1) * 128));
+          ok = warp_wait(&S.b_empty[sb], ((bit / kBSlots) & 1) ^ 1, abortp, P.status);
+          if (!ok) break;
+          uint8_t* tile = b_ring + sb * kBSlotBytes;
+          for (int ps = 0; ps < passes; ++ps) {
+            const int r = ps * 16 + r_local;
+            if (r < m) {
+              if (ps > 0)
+                c0q = __ldg(reinterpret_cast<const uint4*>(
+                    reinterpret_cast<const uint8_t*>(xb + (size_t)S.p_tok[par][r] * H) + c * 16 + (size_t)kc * 128));
               *reinterpret_cast<uint4*>(tile + sw128(r, c)) = c0q;
             }
           }
+          ptx::fence_proxy_async_smem();
+          ptx::mbar_arrive(&S.b_full[sb]);
         }
-        ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(&S.b_full[sb]);
       }
+      if (!ok) break;
     }
   }
 

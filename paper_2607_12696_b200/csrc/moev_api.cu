@@ -35,6 +35,9 @@ struct moev_ctx {
   float* part_x2 = nullptr;  // [n_slices, max_tokens]
   float* part_w2 = nullptr;  // [n_slices] max over experts of the slice's squared row norm
   int n_slices = 0;
+#ifdef MOEV_TC_STATS
+  unsigned long long* tc_stats = nullptr;  // [n_sm][8], debug builds only
+#endif
   void* x_stage = nullptr;  // device staging for moev_verify_host
   void* y_stage = nullptr;
   int32_t* host_word = nullptr;  // pinned scratch for status / n_active reads
@@ -177,12 +180,15 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
                    cudaStream_t st, cudaEvent_t* ev) {
   const moev_config& g = c->cfg;
   tc::Params P{};
-  P.units = c->T.units; P.n_units = c->T.n_units; P.slot_token = c->T.slot_token; P.slot_w = c->T.slot_w;
+  P.units = c->T.units; P.n_units = c->T.n_units; P.task_counter = c->T.task_counter; P.slot_token = c->T.slot_token; P.slot_w = c->T.slot_w;
   P.tok_scale = c->T.tok_scale; P.x = x; P.y32 = c->y32;
   P.s_gate = static_cast<const float*>(L->s_gate); P.s_up = static_cast<const float*>(L->s_up);
   P.s_down = static_cast<const float*>(L->s_down);
   P.sh_s_gate = static_cast<const float*>(L->sh_s_gate); P.sh_s_up = static_cast<const float*>(L->sh_s_up);
   P.sh_s_down = static_cast<const float*>(L->sh_s_down);
+#ifdef MOEV_TC_STATS
+  P.stats = c->tc_stats;
+#endif
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
   tc::grouped_ffn_tc_kernel<WFMT><<<c->n_sm, tc::kThreads, tc::kSmemBytes, st>>>(
       tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
@@ -262,6 +268,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && dmalloc(&c->T.status, 1) == cudaSuccess;
   ok = ok && dmalloc(&c->T.tok_scale, G) == cudaSuccess;
   ok = ok && dmalloc(&c->T.n_units, 1) == cudaSuccess;
+  ok = ok && dmalloc(&c->T.task_counter, 1) == cudaSuccess;
   {
     const size_t cap = c->unit_cap;
     const size_t max_units = E + A / cap + (size_t)cfg->n_shared * (G / cap + 1) + 8;
@@ -273,6 +280,9 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && cudaMalloc(&c->y_stage, G * cfg->H * act_b) == cudaSuccess;
   ok = ok && cudaMallocHost(reinterpret_cast<void**>(&c->host_word), 4 * sizeof(int32_t)) == cudaSuccess;
   if (ok) ok = cudaMemset(c->T.status, 0, sizeof(int32_t)) == cudaSuccess;
+#ifdef MOEV_TC_STATS
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->tc_stats), (size_t)c->n_sm * 8 * sizeof(unsigned long long)) == cudaSuccess;
+#endif
   // opt in to large dynamic shared memory where the shape needs it
   if (ok) {
     size_t gs = route_smem(*cfg, cfg->max_tokens);
@@ -301,7 +311,7 @@ moev_status moev_destroy(moev_ctx* c) {
   cudaFree(c->part); cudaFree(c->part_x2); cudaFree(c->part_w2); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale);
-  cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->hbuf); cudaFree(c->y32);
+  cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->T.task_counter); cudaFree(c->hbuf); cudaFree(c->y32);
   cudaFree(c->x_stage); cudaFree(c->y_stage);
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)
@@ -427,6 +437,16 @@ moev_status moev_status_sync(moev_ctx* c, void* cuda_stream) {
   }
   return MOEV_OK;
 }
+
+#ifdef MOEV_TC_STATS
+// Debug builds: copy the per-CTA wait-cycle counters of the last tensor-core FFN launch.
+int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*8]*/) {
+  if (!c || !host_out) return -1;
+  cudaDeviceSynchronize();
+  cudaMemcpy(host_out, c->tc_stats, (size_t)c->n_sm * 8 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+  return c->n_sm;
+}
+#endif
 
 moev_status moev_profile_enable(moev_ctx* c, int32_t on) {
   if (!c) return MOEV_EINVAL;

@@ -424,7 +424,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       un.m = min(unit_cap, m - c * unit_cap); un.shared = shared;
       T.units[first + c] = un;
     }
-    if (tid == blockDim.x - 1) *T.n_units = base + sc;
+    if (tid == blockDim.x - 1) { *T.n_units = base + sc; *T.task_counter = 0; }
   }
 
   // ---- phase 3: stable permutation.  Warp 0 walks the assignments in order, 32 at a time;
