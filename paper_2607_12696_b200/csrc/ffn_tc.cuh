@@ -66,7 +66,7 @@ struct Params {
   int32_t* status;
   int32_t gamma, H, I, A;
 #ifdef MOEV_TC_STATS
-  unsigned long long* stats;  // [grid][8] cycles the MMA thread spent per wait class (debug builds)
+  unsigned long long* stats;  // [grid][12] cycles the MMA thread spent per wait / issue class (debug builds)
 #endif
 };
 
@@ -172,10 +172,11 @@ struct Fmt<MOEV_W_FP8E4M3_B128> {
   static constexpr int kHTileBytes = 8 * 1024;   // one [64 x 128 B] tile
 };
 
+// a_lo / b_lo: descriptor lower halves (ptx::desc_lo_sw128); +2 per 32 bytes along K.
 template <int WFMT>
-__device__ __forceinline__ void issue_mma(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-  if constexpr (WFMT == MOEV_W_BF16) ptx::mma_f16(d, a, b, idesc, acc);
-  else ptx::mma_f8f6f4(d, a, b, idesc, acc);
+__device__ __forceinline__ void issue_mma(uint32_t d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t acc) {
+  if constexpr (WFMT == MOEV_W_BF16) ptx::mma_f16_lohi(d, a_lo, b_lo, ptx::kDescHiSw128, idesc, acc);
+  else ptx::mma_f8f6f4_lohi(d, a_lo, b_lo, ptx::kDescHiSw128, idesc, acc);
 }
 
 // Task id -> (unit index, slice).  Ids enumerate (slice pair, unit, half) with the half
@@ -260,25 +261,29 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
       uint32_t it = 0, q = 0;
       bool ok = true;
-      while (ok) {
-        // fetch the next valid task id and publish it to the other roles
+      // Task ids are published one task ahead of the loads, so the other roles can prepare
+      // their tables (and the first activation tiles) while this task still streams.
+      auto fetch_publish = [&](TaskDesc& td) -> int {
         int id;
-        TaskDesc td;
         td.unit = 0; td.slice = 0; td.valid = false;
         do {
           id = atomicAdd(P.task_counter, 1);
           if (id >= n_ids) { id = -1; break; }
           td = decode_task(id, n_units, n_slices);
         } while (!td.valid);
-        {
-          const int slot = q % kTaskQ;
-          ok = ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-          if (!ok) break;
-          S.tq_task[slot] = id;
-          ptx::mbar_arrive(&S.tq_full[slot]);
-          ++q;
-        }
-        if (id < 0) break;
+        const int slot = q % kTaskQ;
+        ok = ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+        if (!ok) return -2;
+        S.tq_task[slot] = id;
+        ptx::mbar_arrive(&S.tq_full[slot]);
+        ++q;
+        return id;
+      };
+      TaskDesc td, td_next;
+      int id = fetch_publish(td);
+      while (ok && id >= 0) {
+        const int id_next = fetch_publish(td_next);
+        if (!ok) break;
         const Unit u = P.units[td.unit];
         const int slice = td.slice;
         const CUtensorMap* mg = u.shared ? &tm_sh_gate : &tm_gate;
@@ -310,6 +315,8 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             ptx::tma_load_3d(dst + 16384, md, &S.w_full[s], slice * 128 + 64, ds * 128, u.expert, ptx::kPolicyEvictFirst);
           }
         }
+        id = id_next;
+        td = td_next;
       }
     }
   } else if (warp == 1) {
@@ -317,8 +324,11 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     if (lane == 0) {
       uint32_t it = 0, bit = 0, tcount = 0, dsc = 0, q = 0;
       bool ok = true;
+      const uint32_t w_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(w_ring));
+      const uint32_t b_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(b_ring));
+      const uint32_t h_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(h_tile));
 #ifdef MOEV_TC_STATS
-      unsigned long long st_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      unsigned long long st_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
       const long long st_begin = clock64();
 #endif
       for (;; ++tcount) {
@@ -345,17 +355,22 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             MOEV_STAT_END(2); }
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t wa = ptx::smem_u32(w_ring + s * kStageBytes);
-          const uint32_t ba = ptx::smem_u32(b_ring + sb * kBSlotBytes);
+          const uint32_t wa = w_lo0 + s * (kStageBytes >> 4);
+          const uint32_t ba = b_lo0 + sb * (kBSlotBytes >> 4);
+          const uint32_t acc0 = kc ? 1u : 0u;
+          { MOEV_STAT_BEGIN();
+          issue_mma<WFMT>(d_gate, wa, ba, idesc, acc0);
+          issue_mma<WFMT>(d_up, wa + 1024, ba + (kFp8 ? 512 : 0), idesc, acc0);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t acc = (kc | j) ? 1u : 0u;
-            issue_mma<WFMT>(d_gate, ptx::smem_desc_sw128(wa + j * 32), ptx::smem_desc_sw128(ba + j * 32), idesc, acc);
-            issue_mma<WFMT>(d_up, ptx::smem_desc_sw128(wa + 16384 + j * 32),
-                            ptx::smem_desc_sw128(ba + (kFp8 ? 8192 : 0) + j * 32), idesc, acc);
+          for (int j = 1; j < 4; ++j) {
+            issue_mma<WFMT>(d_gate, wa + 2 * j, ba + 2 * j, idesc, 1u);
+            issue_mma<WFMT>(d_up, wa + 1024 + 2 * j, ba + (kFp8 ? 512 : 0) + 2 * j, idesc, 1u);
           }
+          MOEV_STAT_END(8); }
+          { MOEV_STAT_BEGIN();
           ptx::mma_commit(&S.w_empty[s]);
           ptx::mma_commit(&S.b_empty[sb]);
+          MOEV_STAT_END(9); }
         }
         if (!ok) break;
         ptx::mma_commit(&S.acc_full);
@@ -364,7 +379,6 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           MOEV_STAT_END(4); }
         if (!ok) break;
         ptx::tc_fence_after();
-        const uint32_t ha = ptx::smem_u32(h_tile);
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc, ++it) {
           const int db = dsc & 1;
           const int s = it % kStages;
@@ -376,15 +390,15 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             MOEV_STAT_END(6); }
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t wa = ptx::smem_u32(w_ring + s * kStageBytes);
+          const uint32_t wa = w_lo0 + s * (kStageBytes >> 4);
+          MOEV_STAT_BEGIN();
           if constexpr (kFp8) {
             const int nt = (2 * ds + 1 < HT) ? 2 : 1;
             for (int tl = 0; tl < nt; ++tl) {
               const uint32_t d_down = tmem + 128 + (db * TPS + tl) * 64;
 #pragma unroll
               for (int j = 0; j < 4; ++j)
-                issue_mma<WFMT>(d_down, ptx::smem_desc_sw128(wa + tl * 16384 + j * 32),
-                                ptx::smem_desc_sw128(ha + j * 32), idesc, j ? 1u : 0u);
+                issue_mma<WFMT>(d_down, wa + tl * 1024 + 2 * j, h_lo0 + 2 * j, idesc, j ? 1u : 0u);
             }
           } else {
             const uint32_t d_down = tmem + 128 + db * 64;
@@ -392,11 +406,13 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
               for (int j = 0; j < 4; ++j)
-                issue_mma<WFMT>(d_down, ptx::smem_desc_sw128(wa + hf * 16384 + j * 32),
-                                ptx::smem_desc_sw128(ha + hf * 8192 + j * 32), idesc, (hf | j) ? 1u : 0u);
+                issue_mma<WFMT>(d_down, wa + hf * 1024 + 2 * j, h_lo0 + hf * 512 + 2 * j, idesc, (hf | j) ? 1u : 0u);
           }
+          MOEV_STAT_END(10);
+          { MOEV_STAT_BEGIN();
           ptx::mma_commit(&S.d_full[db]);
           ptx::mma_commit(&S.w_empty[s]);
+          MOEV_STAT_END(11); }
         }
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
@@ -405,7 +421,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
       if (P.stats)
-        for (int i = 0; i < 8; ++i) P.stats[(size_t)blockIdx.x * 8 + i] = st_acc[i];
+        for (int i = 0; i < 12; ++i) P.stats[(size_t)blockIdx.x * 12 + i] = st_acc[i];
 #endif
     }
   } else if (warp < 6) {
@@ -531,6 +547,38 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         if (!ok) break;
         ptx::tc_fence_after();
         const int nt = kFp8 ? ((2 * ds + 1 < HT) ? 2 : 1) : 1;
+        if (ncols <= 16) {
+          // common case (few tokens): fetch every tile of the stage, release the accumulators,
+          // then do the reductions
+          uint32_t o[TPS][16];
+#pragma unroll
+          for (int tl = 0; tl < TPS; ++tl)
+            if (tl < nt) ptx::tmem_ld16(tmem + lane_base + 128 + (db * TPS + tl) * 64, o[tl]);
+          ptx::tmem_ld_wait();
+          ptx::tc_fence_before();
+          ptx::mbar_arrive(&S.d_empty[db]);
+#pragma unroll
+          for (int tl = 0; tl < TPS; ++tl) {
+            if (tl < nt) {
+              const int ht = ds * TPS + tl;
+              float* ycol = P.y32 + (size_t)ht * 128 + row;
+              if constexpr (kFp8) {
+                const float sd = S.e_sd[par][ht];
+#pragma unroll
+                for (int r = 0; r < 8; ++r)
+                  if (r < m) {
+                    float val = (__uint_as_float(o[tl][2 * r]) + __uint_as_float(o[tl][2 * r + 1]) * 0.0625f) * (sd * S.e_f[r]);
+                    ptx::red_add_f32(ycol + (size_t)S.e_tok[par][r] * H, val);
+                  }
+              } else {
+#pragma unroll
+                for (int r = 0; r < 16; ++r)
+                  if (r < m) ptx::red_add_f32(ycol + (size_t)S.e_tok[par][r] * H, __uint_as_float(o[tl][r]) * S.e_w[par][r]);
+              }
+            }
+          }
+          continue;
+        }
         for (int tl = 0; tl < nt; ++tl) {
           const int ht = ds * TPS + tl;
           const uint32_t d_down = tmem + lane_base + 128 + (db * TPS + tl) * 64;

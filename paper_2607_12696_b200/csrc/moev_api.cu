@@ -36,7 +36,7 @@ struct moev_ctx {
   float* part_w2 = nullptr;  // [n_slices] max over experts of the slice's squared row norm
   int n_slices = 0;
 #ifdef MOEV_TC_STATS
-  unsigned long long* tc_stats = nullptr;  // [n_sm][8], debug builds only
+  unsigned long long* tc_stats = nullptr;  // [n_sm][12], debug builds only
 #endif
   void* x_stage = nullptr;  // device staging for moev_verify_host
   void* y_stage = nullptr;
@@ -281,7 +281,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && cudaMallocHost(reinterpret_cast<void**>(&c->host_word), 4 * sizeof(int32_t)) == cudaSuccess;
   if (ok) ok = cudaMemset(c->T.status, 0, sizeof(int32_t)) == cudaSuccess;
 #ifdef MOEV_TC_STATS
-  ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->tc_stats), (size_t)c->n_sm * 8 * sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->tc_stats), (size_t)c->n_sm * 12 * sizeof(unsigned long long)) == cudaSuccess;
 #endif
   // opt in to large dynamic shared memory where the shape needs it
   if (ok) {
@@ -440,10 +440,10 @@ moev_status moev_status_sync(moev_ctx* c, void* cuda_stream) {
 
 #ifdef MOEV_TC_STATS
 // Debug builds: copy the per-CTA wait-cycle counters of the last tensor-core FFN launch.
-int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*8]*/) {
+int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*12]*/) {
   if (!c || !host_out) return -1;
   cudaDeviceSynchronize();
-  cudaMemcpy(host_out, c->tc_stats, (size_t)c->n_sm * 8 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+  cudaMemcpy(host_out, c->tc_stats, (size_t)c->n_sm * 12 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
   return c->n_sm;
 }
 #endif
