@@ -52,9 +52,11 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 
-# DRAM bytes per launch of the dominant kernel from the committed ncu captures
-# (profiles/*.md), keyed by (workload, impl name); absent = not captured.
-NCU_TRAFFIC_BYTES: dict = {}
+# DRAM (read + write) bytes per algorithmic byte of the dominant kernel, from the committed ncu
+# capture of a smaller case of the same kernel (profiles/grouped_ffn_tc_fp8_E64_g16.md:
+# 2.443169 GB + 3.97 MB against 2.422802 GB); traffic grows in proportion to the experts
+# streamed, so the full-size launch is scaled by the same ratio.  Absent = not captured.
+NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.443169e9 + 3.97184e6) / 2.422801920e9}
 
 ROUTING = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
            "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing}
@@ -198,6 +200,17 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def aggregate_over_ranks(dist, device, ms_total: float, e2e_ms: float, nbytes: float):
+    """Whole-job figures for N replicas: max time over ranks, bytes summed over ranks."""
+    if dist is None:
+        return ms_total, e2e_ms, nbytes
+    t = torch.tensor([ms_total, e2e_ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    b = torch.tensor([float(nbytes)], device=device, dtype=torch.float64)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(t[0]), float(t[1]), float(b[0])
+
+
 def run_ours(args):
     import paper_2607_12696_b200 as moev
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -280,14 +293,7 @@ def run_ours(args):
     h2d, d2h = gamma * shape.H * act_b, gamma * shape.H * act_b + 4
 
     # ---- aggregate over replicas: max time, summed bytes
-    if dist:
-        t = torch.tensor([ms_total, e2e_s * 1e3], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        b = torch.tensor([float(tot_bytes)], device=dev, dtype=torch.float64)
-        dist.all_reduce(b, op=dist.ReduceOp.SUM)
-        ms_total, e2e_ms, all_bytes = float(t[0]), float(t[1]), float(b[0])
-    else:
-        e2e_ms, all_bytes = e2e_s * 1e3, float(tot_bytes)
+    ms_total, e2e_ms, all_bytes = aggregate_over_ranks(dist, dev, ms_total, e2e_s * 1e3, float(tot_bytes))
 
     if rank == 0:
         value = all_bytes / (ms_total * 1e-3) / 1e9
@@ -299,17 +305,19 @@ def run_ours(args):
         else:
             k_name, k_bytes, k_us = "grouped_ffn_tc_kernel", mean_bytes, kern_us[3]
         achieved = k_bytes / (k_us * 1e-6) / 1e9 if k_us > 0 else None
+        dtype_name = {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "mxfp4"}[shape.wfmt]
         cpu = None
         if not args.no_cpu_baseline:
-            cv, cs, cu, cores = time_oracle_sample(shape, layers[0], args.cpu_tokens)
+            n_cpu = args.cpu_tokens if args.cpu_tokens > 0 else gamma
+            cv, cs, cu, cores = time_oracle_sample(shape, layers[0], n_cpu)
             cpu = {"value": cv, "unit": UNIT, "cores": cores, "kind": "oracle",
-                   "sample": f"first {args.cpu_tokens} of the {gamma} tokens of layer 0 (U={cu}"
+                   "sample": f"first {n_cpu} of the {gamma} tokens of layer 0 (U={cu}"
                              f"+{shape.n_shared} experts streamed), full layer weights, {cs:.2f} s"}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
-            "dtype": {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "mxfp4"}[shape.wfmt],
+            "dtype": dtype_name,
             "data": "synthetic",
             "config": {"workload": args.workload, "gamma": gamma, "H": shape.H, "I": shape.I,
                        "E": shape.E, "top_k": shape.top_k, "n_shared": shape.n_shared,
@@ -321,7 +329,8 @@ def run_ours(args):
             "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": (achieved / peak) if achieved else None,
-                         "traffic": NCU_TRAFFIC_BYTES.get((args.workload, impl_name)),
+                         "traffic": (k_bytes * NCU_TRAFFIC_RATIO[(dtype_name, impl_name)]
+                                     if (dtype_name, impl_name) in NCU_TRAFFIC_RATIO else None),
                          "kernel": k_name, "kernel_us": k_us, "kernel_bytes": k_bytes,
                          "launches_timed": kern_calls,
                          "per_kernel_us": {"router_partial": kern_us[0], "topk_refine": kern_us[1],
@@ -353,7 +362,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--layers", type=int, default=4)
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tcgen05"])
-    ap.add_argument("--cpu-tokens", type=int, default=2)
+    ap.add_argument("--cpu-tokens", type=int, default=0, help="tokens of layer 0 the oracle is timed on (0 = all gamma)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
