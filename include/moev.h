@@ -181,6 +181,35 @@ moev_status moev_profile_enable(moev_ctx* ctx, int32_t on);
 moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[6]*/,
                               int32_t* calls);
 
+/* Router top-k without any allocation.  (The paper has no counterpart: this entry point
+ * exists for the integration constraints of some callers, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is forbidden or unavailable -- inside a
+ * memory-pool-managed serving process that has handed all device memory to its own allocator,
+ * in a latency-critical thread that may not take the allocator's lock, or before a framework
+ * has set up its caching allocator.  Such callers cannot create a moev_ctx (moev_create
+ * allocates the workspace), but may still want the routing decision of a layer.
+ *
+ * Computes, for the gamma tokens x [gamma, H] (afmt of cfg), the same topk_ids [gamma, k] and
+ * topk_w [gamma, k] that moev_verify writes, using cfg->H, E, top_k, afmt, score,
+ * routed_scale and max_tokens (gamma <= max_tokens); all pointers are DEVICE pointers owned by
+ * the caller.  The split-K partial logits live in a fixed 20 MiB array compiled into the
+ * library (held by every GPU that loads it until the process exits) instead of a context
+ * workspace; moev_route_topk_static_scratch_floats() returns how many of its 5 242 880 floats a
+ * problem needs, and problems that need more are rejected with MOEV_EINVAL.  The call itself
+ * calls no cudaMalloc/cudaFree and no allocating library routine; it enqueues two kernels on
+ * cuda_stream and returns without waiting.
+ *
+ * The first call on a device looks up the device address of the array (once per device, with
+ * that device current); make that first call before starting any stream capture.  All calls
+ * share the one array: nothing in it has to be cleared between calls (each call overwrites
+ * what it reads), but two calls whose kernels overlap on the GPU (different streams, or
+ * several host threads) race on it and give undefined results -- serialise them. */
+moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w, const void* x,
+                                   int32_t gamma, int32_t* topk_ids, float* topk_w,
+                                   void* cuda_stream);
+size_t moev_route_topk_static_scratch_floats(int32_t H, int32_t E, int32_t gamma);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,7 +20,7 @@ STATUS = {0: "MOEV_OK", 1: "MOEV_EINVAL", 2: "MOEV_EUNSUPPORTED", 3: "MOEV_ECUDA
 EXPORTS = ("moev_create", "moev_destroy", "moev_verify", "moev_verify_host", "moev_status_sync",
            "moev_last_error", "moev_expert_bytes", "moev_expert_code_bytes",
            "moev_launches_per_call", "moev_resolved_impl", "moev_profile_enable",
-           "moev_profile_read")
+           "moev_profile_read", "moev_route_topk_static", "moev_route_topk_static_scratch_floats")
 
 
 class MoevError(RuntimeError):
@@ -110,6 +110,11 @@ def lib() -> C.CDLL:
         L.moev_profile_read.restype = C.c_int
         L.moev_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_double),
                                         C.POINTER(C.c_int32)]
+        L.moev_route_topk_static.restype = C.c_int
+        L.moev_route_topk_static.argtypes = [C.POINTER(_Config), C.c_void_p, C.c_void_p, C.c_int32,
+                                             C.c_void_p, C.c_void_p, C.c_void_p]
+        L.moev_route_topk_static_scratch_floats.restype = C.c_size_t
+        L.moev_route_topk_static_scratch_floats.argtypes = [C.c_int32, C.c_int32, C.c_int32]
         _lib = L
     return _lib
 
@@ -122,6 +127,25 @@ def expert_bytes(cfg: MoevConfig) -> int:
 def expert_code_bytes(cfg: MoevConfig) -> int:
     c = cfg.c()
     return lib().moev_expert_code_bytes(C.byref(c))
+
+
+def route_topk_static(cfg: MoevConfig, router_w: torch.Tensor, x: torch.Tensor, gamma: int,
+                      topk_ids: torch.Tensor, topk_w: torch.Tensor):
+    """moev_route_topk_static: router top-k for callers that may not allocate device memory.
+
+    Needs no context; the scratch is the fixed array inside the library, shared by all calls
+    (do not overlap calls on the GPU).  Asynchronous on torch's current stream."""
+    c = cfg.c()
+    st = lib().moev_route_topk_static(C.byref(c), router_w.data_ptr(), x.data_ptr(), gamma,
+                                      topk_ids.data_ptr(), topk_w.data_ptr(),
+                                      C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if st != 0:
+        raise MoevError(st, "moev_route_topk_static rejected the call (arguments, or the problem "
+                            "exceeds the fixed scratch array)")
+
+
+def static_scratch_floats(H: int, E: int, gamma: int) -> int:
+    return lib().moev_route_topk_static_scratch_floats(H, E, gamma)
 
 
 def _ptr(t):

@@ -66,7 +66,7 @@ struct Params {
   int32_t* status;
   int32_t gamma, H, I, A;
 #ifdef MOEV_TC_STATS
-  unsigned long long* stats;  // [grid][12] cycles the MMA thread spent per wait / issue class (debug builds)
+  unsigned long long* stats;  // [grid][16] cycles the MMA thread spent per wait / issue class (debug builds)
 #endif
 };
 
@@ -328,7 +328,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       const uint32_t b_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(b_ring));
       const uint32_t h_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(h_tile));
 #ifdef MOEV_TC_STATS
-      unsigned long long st_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+      unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
       const long long st_begin = clock64();
 #endif
       for (;; ++tcount) {
@@ -352,7 +352,12 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             MOEV_STAT_END(1); }
           { MOEV_STAT_BEGIN();
             ok = ok && ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            MOEV_STAT_END(2); }
+#ifdef MOEV_TC_STATS
+            { unsigned long long dt = (unsigned long long)(clock64() - _t0);
+              if (kc < 3) st_acc[12] += dt; else st_acc[2] += dt;
+              if (dt > 400) { st_acc[13] += 1; st_acc[14] += dt; } }
+#endif
+            }
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t wa = w_lo0 + s * (kStageBytes >> 4);
@@ -421,7 +426,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
       if (P.stats)
-        for (int i = 0; i < 12; ++i) P.stats[(size_t)blockIdx.x * 12 + i] = st_acc[i];
+        for (int i = 0; i < 16; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
 #endif
     }
   } else if (warp < 6) {

@@ -36,7 +36,7 @@ struct moev_ctx {
   float* part_w2 = nullptr;  // [n_slices] max over experts of the slice's squared row norm
   int n_slices = 0;
 #ifdef MOEV_TC_STATS
-  unsigned long long* tc_stats = nullptr;  // [n_sm][12], debug builds only
+  unsigned long long* tc_stats = nullptr;  // [n_sm][16], debug builds only
 #endif
   void* x_stage = nullptr;  // device staging for moev_verify_host
   void* y_stage = nullptr;
@@ -281,7 +281,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && cudaMallocHost(reinterpret_cast<void**>(&c->host_word), 4 * sizeof(int32_t)) == cudaSuccess;
   if (ok) ok = cudaMemset(c->T.status, 0, sizeof(int32_t)) == cudaSuccess;
 #ifdef MOEV_TC_STATS
-  ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->tc_stats), (size_t)c->n_sm * 12 * sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->tc_stats), (size_t)c->n_sm * 16 * sizeof(unsigned long long)) == cudaSuccess;
 #endif
   // opt in to large dynamic shared memory where the shape needs it
   if (ok) {
@@ -438,12 +438,93 @@ moev_status moev_status_sync(moev_ctx* c, void* cuda_stream) {
   return MOEV_OK;
 }
 
+// ---------------------------------------------------------------------------------------
+// Allocation-free router top-k.  The split-K router kernels need scratch memory for their
+// partial logits; callers that must not (or cannot) allocate device memory get that scratch
+// from this fixed array instead.  It lives in every GPU context that loads the library until
+// the process exits.  In host code `g_static_scratch` is only a handle for the runtime: the
+// device address is obtained once per device with cudaGetSymbolAddress.
+constexpr size_t kStaticScratchFloats = 5u * 1024u * 1024u;  // 20 MiB
+static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float* g_static_scratch_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the static scratch array on the current device (set up on first use).
+cudaError_t static_scratch_address(float** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!g_static_scratch_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_scratch_ptr[dev] = static_cast<float*>(p);
+  }
+  *out = g_static_scratch_ptr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+
+size_t moev_route_topk_static_scratch_floats(int32_t H, int32_t E, int32_t gamma) {
+  const size_t ns = (size_t)(H + kRouterKS - 1) / kRouterKS;
+  // partial logits | squared-norm partials of x | per-slice router norm bound | token scales | y32 rows
+  return ns * gamma * E + ns * gamma + ns + (size_t)gamma + (size_t)gamma * H + 64;
+}
+
+moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w, const void* x,
+                                   int32_t gamma, int32_t* topk_ids, float* topk_w, void* cuda_stream) {
+  char why[256];
+  if (!cfg_ok(cfg, why, sizeof(why))) return MOEV_EINVAL;
+  if (!router_w || !x || !topk_ids || !topk_w || gamma < 1 || gamma > cfg->max_tokens) return MOEV_EINVAL;
+  if (!aligned16(router_w) || !aligned16(x)) return MOEV_EINVAL;
+  if (moev_route_topk_static_scratch_floats(cfg->H, cfg->E, gamma) > kStaticScratchFloats)
+    return MOEV_EINVAL;  // the problem does not fit the fixed scratch array
+  float* base = nullptr;
+  if (static_scratch_address(&base) != cudaSuccess) {
+    cudaGetLastError();
+    return MOEV_ECUDA;
+  }
+  const size_t ns = (size_t)(cfg->H + kRouterKS - 1) / kRouterKS;
+  // carve the array (every region starts on a 256-byte boundary)
+  auto up64 = [](size_t n) { return (n + 63) & ~size_t(63); };
+  float* part = base;
+  float* part_x2 = part + up64(ns * gamma * cfg->E);
+  float* part_w2 = part_x2 + up64(ns * gamma);
+  float* tok_scale = part_w2 + up64(ns);
+  float* y32 = tok_scale + up64((size_t)gamma);
+  if ((size_t)(y32 - base) + (size_t)gamma * cfg->H > kStaticScratchFloats) return MOEV_EINVAL;
+  Tables T{};
+  T.topk_ids = topk_ids;
+  T.topk_w = topk_w;
+  T.tok_scale = tok_scale;
+  RouteOut O{};
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t refine_smem = (size_t)cfg->E * 16;
+  // Nothing has to start at zero: every partial that is read is written by the first kernel of
+  // the same call, and the y32 rows are cleared (not accumulated into) by the second.
+  if (cfg->afmt == MOEV_ACT_FP32) {
+    router_partial_kernel<MOEV_ACT_FP32><<<(int)ns, 256, 0, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E);
+    topk_refine_kernel<MOEV_ACT_FP32><<<gamma, 256, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns,
+                                                                       cfg->score, cfg->routed_scale);
+  } else {
+    router_partial_kernel<MOEV_ACT_BF16><<<(int)ns, 256, 0, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E);
+    topk_refine_kernel<MOEV_ACT_BF16><<<gamma, 256, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns,
+                                                                       cfg->score, cfg->routed_scale);
+  }
+  return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
+}
+
 #ifdef MOEV_TC_STATS
 // Debug builds: copy the per-CTA wait-cycle counters of the last tensor-core FFN launch.
-int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*12]*/) {
+int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*16]*/) {
   if (!c || !host_out) return -1;
   cudaDeviceSynchronize();
-  cudaMemcpy(host_out, c->tc_stats, (size_t)c->n_sm * 12 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
+  cudaMemcpy(host_out, c->tc_stats, (size_t)c->n_sm * 16 * sizeof(unsigned long long), cudaMemcpyDeviceToHost);
   return c->n_sm;
 }
 #endif
