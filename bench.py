@@ -353,6 +353,75 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Unique-expert sweep at the DeepSeek FP8 shape: routing built so that the union is exactly
+    U, for gamma in {1, 8, 32, 128}; 4 layers' weights rotated per call.  Prints one JSON line
+    per cell plus a linear fit latency = a + b U per gamma (rank 0, one GPU)."""
+    import paper_2607_12696_b200 as moev
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    shape = synth.SHAPES["deepseek"]
+    n_layers = layers_that_fit(shape, args.layers)
+    weights = [synth.make_expert_weights(shape, layer=l, device=dev) for l in range(n_layers)]
+    gammas, unions = [1, 8, 32, 128], [8, 16, 32, 64, 128, 256]
+    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, max(gammas), shape.wfmt,
+                          shape.afmt, shape.score, moev.IMPL_AUTO, shape.routed_scale)
+    v = moev.MoeVerifier(cfg)
+    Wb = moev.expert_bytes(cfg)
+    peak, peak_src = measured_peaks()
+    fits = {}
+    for gamma in gammas:
+        pts = []
+        for U in unions:
+            cell = {"sweep": "unique_experts", "gamma": gamma, "U": U}
+            if not synth.union_feasible(shape, gamma, U):
+                cell["latency_us"] = "n/a"
+                print(json.dumps(cell))
+                continue
+            packed, xs, outs = [], [], []
+            for l in range(n_layers):
+                wr, x = synth.make_exact_union_routing(shape, gamma, U, layer=l, device=dev)
+                d = {"router_w": wr}
+                d.update({k: t for k, t in weights[l].items() if t is not None})
+                packed.append((moev.binding.make_layer(d), d))
+                xs.append(x)
+                outs.append(v.alloc_out(gamma, diagnostics=False))
+            for i in range(max(args.warmup, n_layers)):
+                v.verify(packed[i % n_layers][0], xs[i % n_layers], gamma, outs[i % n_layers])
+            torch.cuda.synchronize()
+            assert all(int(o["n_active"].item()) == U for o in outs)
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(args.steps)]
+            v.profile_enable(True)
+            for i, (e0, e1) in enumerate(evs):
+                l = i % n_layers
+                e0.record()
+                v.verify(packed[l][0], xs[l], gamma, outs[l])
+                e1.record()
+            torch.cuda.synchronize()
+            kern_us, _ = v.profile_read()
+            v.profile_enable(False)
+            lat = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+            med = lat[len(lat) // 2]
+            nbytes = (U + shape.n_shared) * Wb
+            cell.update(latency_us=med, latency_min_us=lat[0], latency_p90_us=lat[int(0.9 * len(lat))],
+                        ffn_kernel_us=kern_us[3], bytes=nbytes, gbs=nbytes / med / 1e3,
+                        frac_of_8TBps=nbytes / med / 1e3 / NOMINAL_HBM_GBS, frac_of_measured=nbytes / med / 1e3 / peak,
+                        roofline_us_8TBps=nbytes / 8e6)
+            print(json.dumps(cell))
+            pts.append((U, med))
+        if len(pts) >= 2:
+            u = np.array([p[0] for p in pts], dtype=np.float64)
+            t = np.array([p[1] for p in pts], dtype=np.float64)
+            b, a = np.polyfit(u, t, 1)
+            r2 = 1.0 - ((t - (a + b * u)) ** 2).sum() / max(((t - t.mean()) ** 2).sum(), 1e-30)
+            fits[gamma] = {"a_us": a, "b_us_per_expert": b, "r2": r2,
+                           "roofline_b_us_per_expert_8TBps": Wb / 8e6}
+    print(json.dumps({"sweep": "unique_experts", "fit_latency_us = a + b*U": fits,
+                      "layers_rotated": n_layers, "peak_source": peak_src}))
+    v.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -364,6 +433,7 @@ def main():
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--cpu-tokens", type=int, default=0, help="tokens of layer 0 the oracle is timed on (0 = all gamma)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="unique-expert sweep (DeepSeek FP8 shape) instead of the bench line")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -371,7 +441,10 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-        run_ours(args)
+        if args.sweep:
+            run_sweep(args)
+        else:
+            run_ours(args)
 
 
 if __name__ == "__main__":
