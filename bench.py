@@ -49,6 +49,8 @@ WORKLOADS = {
     # and Qwen-shaped layers with 64 experts
     "deepseek_fp8_E64_g16_profile": ("deepseek", 16, "scattered", {"_E": 64}),
     "qwen_bf16_E64_g16_profile": ("qwen", 16, "iid", {"_E": 64}),
+    # routing kernels at the full router shape (256 experts, gamma 64) with thin experts (0.7 GB)
+    "deepseek_router_profile": ("deepseek", 64, "scattered", {"_I": 128}),
 }
 DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 
@@ -121,7 +123,11 @@ class ClockSampler:
 def workload_shape(name: str) -> synth.Shape:
     base, _, _, kw = WORKLOADS[name]
     shape = synth.SHAPES[base]
-    return shape.scaled(E=kw["_E"]) if "_E" in kw else shape
+    if "_E" in kw:
+        shape = shape.scaled(E=kw["_E"])
+    if "_I" in kw:
+        shape = shape.scaled(I=kw["_I"])
+    return shape
 
 
 def build_workload(name: str, n_layers: int, device, rank: int = 0):
@@ -258,8 +264,8 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing
-    v.profile_enable(True)
+    # ---- device-resident timing (the number: no per-kernel event records, kernels overlap their
+    # launch latencies through programmatic dependent launch)
     sampler = ClockSampler(local)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
@@ -271,10 +277,15 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     ms_total = ev0.elapsed_time(ev1)
-    kern_us, kern_calls = v.profile_read()
-    v.profile_enable(False)
     v.status_sync()
     tot_bytes = sum(bytes_step[i % n_layers] for i in range(args.steps))
+    # ---- the same steps again with CUDA events recorded between the kernels of every call:
+    # per-kernel durations for the roofline of the dominant kernel
+    v.profile_enable(True)
+    for i in range(min(args.steps, 500)):
+        step(i)
+    kern_us, kern_calls = v.profile_read()
+    v.profile_enable(False)
 
     # ---- end to end through the host-buffer entry point
     xh = [L["x"].cpu().pin_memory() for L in layers]

@@ -213,6 +213,7 @@ __global__ void __launch_bounds__(256) ffn_down_simt(LayerPtrs L, Tables T, cons
 // y32 (fp32) -> y in the activation format
 template <int AFMT>
 __global__ void finalize_kernel(const float* __restrict__ y32, void* __restrict__ y, size_t n) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the FFN kernel's reductions are complete
   size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= n) return;
   float4 v = *reinterpret_cast<const float4*>(y32 + i);

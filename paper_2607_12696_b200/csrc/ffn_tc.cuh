@@ -251,6 +251,9 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = S.tmem_base;
+  // everything above overlapped the tail of the grouping kernel; its tables are needed from here
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n_units = *P.n_units;
   const int n_ids = n_units * ((n_slices + 1) & ~1);
   volatile int* abortp = &S.abort_flag;

@@ -33,8 +33,9 @@ struct moev_ctx {
   float* y32 = nullptr;   // [max_tokens, H] fp32 combine accumulator
   float* part = nullptr;     // [n_slices, max_tokens, E] split-K partial router logits
   float* part_x2 = nullptr;  // [n_slices, max_tokens]
-  float* part_w2 = nullptr;  // [n_slices] max over experts of the slice's squared row norm
+  float* part_w2 = nullptr;  // [n_slices, expert tiles] max over the tile's experts of the slice's squared row norm
   int n_slices = 0;
+  int ks = 32;  // columns per split-K slice of the router
 #ifdef MOEV_TC_STATS
   unsigned long long* tc_stats = nullptr;  // [n_sm][16], debug builds only
 #endif
@@ -175,6 +176,25 @@ const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
   return &t;
 }
 
+// Launch with (or without) the programmatic-dependent-launch attribute: the kernel may start
+// while its predecessor in the stream drains; it calls griddepcontrol.wait before touching the
+// predecessor's results.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                     Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 template <int WFMT>
 void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const void* x, int gamma,
                    cudaStream_t st, cudaEvent_t* ev) {
@@ -190,8 +210,8 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.stats = c->tc_stats;
 #endif
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
-  tc::grouped_ffn_tc_kernel<WFMT><<<c->n_sm, tc::kThreads, tc::kSmemBytes, st>>>(
-      tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
+  launch_k(tc::grouped_ffn_tc_kernel<WFMT>, dim3(c->n_sm), dim3(tc::kThreads), tc::kSmemBytes, st, ev == nullptr,
+           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
   if (ev) cudaEventRecord(ev[4], st);
 }
 
@@ -253,10 +273,11 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   const size_t slots = A + (size_t)cfg->n_shared * G;
   const size_t act_b = cfg->afmt == MOEV_ACT_FP32 ? 4 : 2;
   bool ok = true;
-  c->n_slices = (cfg->H + kRouterKS - 1) / kRouterKS;
+  c->ks = router_slice_width(cfg->H, prop.multiProcessorCount);
+  c->n_slices = (cfg->H + c->ks - 1) / c->ks;
   ok = ok && dmalloc(&c->part, (size_t)c->n_slices * G * E) == cudaSuccess;
   ok = ok && dmalloc(&c->part_x2, (size_t)c->n_slices * G) == cudaSuccess;
-  ok = ok && dmalloc(&c->part_w2, (size_t)c->n_slices) == cudaSuccess;
+  ok = ok && dmalloc(&c->part_w2, (size_t)c->n_slices * ((E + kRouterETile - 1) / kRouterETile)) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.union_ids, E) == cudaSuccess;
@@ -286,6 +307,10 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   // opt in to large dynamic shared memory where the shape needs it
   if (ok) {
     size_t gs = route_smem(*cfg, cfg->max_tokens);
+    ok = ok && cudaFuncSetAttribute(router_partial_kernel<MOEV_ACT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)router_partial_smem(kRouterMaxKS)) == cudaSuccess;
+    ok = ok && cudaFuncSetAttribute(router_partial_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)router_partial_smem(kRouterMaxKS)) == cudaSuccess;
     if (gs > 48 * 1024)
       ok = ok && cudaFuncSetAttribute(route_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)gs) == cudaSuccess;
@@ -369,24 +394,26 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   if (c->profile && c->prof_n < kProfSlots) ev = c->ev[c->prof_n++];
   if (ev) cudaEventRecord(ev[0], st);
   const size_t refine_smem = (size_t)g.E * 16;
+  const bool pdl = ev == nullptr;  // event records between the kernels would serialise them anyway
+  const size_t rp_smem = router_partial_smem(c->ks);
   if (g.afmt == MOEV_ACT_FP32)
-    router_partial_kernel<MOEV_ACT_FP32><<<c->n_slices, 256, 0, st>>>(x, layer->router_w, c->part, c->part_x2,
-                                                                      c->part_w2, gamma, g.H, g.E);
+    launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, false, x, layer->router_w,
+             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
   else
-    router_partial_kernel<MOEV_ACT_BF16><<<c->n_slices, 256, 0, st>>>(x, layer->router_w, c->part, c->part_x2,
-                                                                      c->part_w2, gamma, g.H, g.E);
+    launch_k(router_partial_kernel<MOEV_ACT_BF16>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, false, x, layer->router_w,
+             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
   if (ev) cudaEventRecord(ev[1], st);
   if (g.afmt == MOEV_ACT_FP32)
-    topk_refine_kernel<MOEV_ACT_FP32><<<gamma, 256, refine_smem, st>>>(
-        c->T, O, x, layer->router_w, c->part, c->part_x2, c->part_w2, c->y32, gamma, g.H, g.E, g.top_k,
-        c->n_slices, g.score, g.routed_scale);
+    launch_k(topk_refine_kernel<MOEV_ACT_FP32>, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x,
+             layer->router_w, (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma,
+             g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale);
   else
-    topk_refine_kernel<MOEV_ACT_BF16><<<gamma, 256, refine_smem, st>>>(
-        c->T, O, x, layer->router_w, c->part, c->part_x2, c->part_w2, c->y32, gamma, g.H, g.E, g.top_k,
-        c->n_slices, g.score, g.routed_scale);
+    launch_k(topk_refine_kernel<MOEV_ACT_BF16>, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x,
+             layer->router_w, (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma,
+             g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale);
   if (ev) cudaEventRecord(ev[2], st);
-  route_group_kernel<<<1, 1024, route_smem(g, gamma), st>>>(c->T, O, gamma, g.E, g.top_k, g.n_shared,
-                                                            c->unit_cap);
+  launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
+           g.n_shared, c->unit_cap);
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);
@@ -394,8 +421,10 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   } else if (g.afmt == MOEV_ACT_FP32) launch_simt_ffn_w<MOEV_ACT_FP32>(c, L, x, gamma, st, ev);
   else launch_simt_ffn_w<MOEV_ACT_BF16>(c, L, x, gamma, st, ev);
   const int fin_blocks = (int)((y_elems / 4 + 255) / 256);
-  if (g.afmt == MOEV_ACT_FP32) finalize_kernel<MOEV_ACT_FP32><<<fin_blocks, 256, 0, st>>>(c->y32, out->y, y_elems);
-  else finalize_kernel<MOEV_ACT_BF16><<<fin_blocks, 256, 0, st>>>(c->y32, out->y, y_elems);
+  if (g.afmt == MOEV_ACT_FP32)
+    launch_k(finalize_kernel<MOEV_ACT_FP32>, dim3(fin_blocks), dim3(256), 0, st, pdl, (const float*)c->y32, out->y, y_elems);
+  else
+    launch_k(finalize_kernel<MOEV_ACT_BF16>, dim3(fin_blocks), dim3(256), 0, st, pdl, (const float*)c->y32, out->y, y_elems);
   if (ev) cudaEventRecord(ev[6], st);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "kernel launch failed: %s", cudaGetErrorString(e));
@@ -445,6 +474,7 @@ moev_status moev_status_sync(moev_ctx* c, void* cuda_stream) {
 // the process exits.  In host code `g_static_scratch` is only a handle for the runtime: the
 // device address is obtained once per device with cudaGetSymbolAddress.
 constexpr size_t kStaticScratchFloats = 5u * 1024u * 1024u;  // 20 MiB
+constexpr int kStaticKS = 32;  // split-K slice width of the static-scratch path (fixed, so its footprint is device-independent)
 static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 
 namespace {
@@ -469,9 +499,9 @@ cudaError_t static_scratch_address(float** out) {
 }  // namespace
 
 size_t moev_route_topk_static_scratch_floats(int32_t H, int32_t E, int32_t gamma) {
-  const size_t ns = (size_t)(H + kRouterKS - 1) / kRouterKS;
+  const size_t ns = (size_t)(H + kStaticKS - 1) / kStaticKS;
   // partial logits | squared-norm partials of x | per-slice router norm bound | token scales | y32 rows
-  return ns * gamma * E + ns * gamma + ns + (size_t)gamma + (size_t)gamma * H + 64;
+  return ns * gamma * E + ns * gamma + ns * ((E + 63) / 64) + (size_t)gamma + (size_t)gamma * H + 4 * 64;
 }
 
 moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w, const void* x,
@@ -487,13 +517,14 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
     cudaGetLastError();
     return MOEV_ECUDA;
   }
-  const size_t ns = (size_t)(cfg->H + kRouterKS - 1) / kRouterKS;
+  const int ks = kStaticKS;
+  const size_t ns = (size_t)(cfg->H + ks - 1) / ks;
   // carve the array (every region starts on a 256-byte boundary)
   auto up64 = [](size_t n) { return (n + 63) & ~size_t(63); };
   float* part = base;
   float* part_x2 = part + up64(ns * gamma * cfg->E);
   float* part_w2 = part_x2 + up64(ns * gamma);
-  float* tok_scale = part_w2 + up64(ns);
+  float* tok_scale = part_w2 + up64(ns * ((cfg->E + kRouterETile - 1) / kRouterETile));
   float* y32 = tok_scale + up64((size_t)gamma);
   if ((size_t)(y32 - base) + (size_t)gamma * cfg->H > kStaticScratchFloats) return MOEV_EINVAL;
   Tables T{};
@@ -505,15 +536,16 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
   const size_t refine_smem = (size_t)cfg->E * 16;
   // Nothing has to start at zero: every partial that is read is written by the first kernel of
   // the same call, and the y32 rows are cleared (not accumulated into) by the second.
+  const size_t rp_smem = router_partial_smem(ks);  // 17 KB: below the default dynamic limit, no attribute needed
   if (cfg->afmt == MOEV_ACT_FP32) {
-    router_partial_kernel<MOEV_ACT_FP32><<<(int)ns, 256, 0, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E);
-    topk_refine_kernel<MOEV_ACT_FP32><<<gamma, 256, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
-                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns,
+    router_partial_kernel<MOEV_ACT_FP32><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
+    topk_refine_kernel<MOEV_ACT_FP32><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
                                                                        cfg->score, cfg->routed_scale);
   } else {
-    router_partial_kernel<MOEV_ACT_BF16><<<(int)ns, 256, 0, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E);
-    topk_refine_kernel<MOEV_ACT_BF16><<<gamma, 256, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
-                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns,
+    router_partial_kernel<MOEV_ACT_BF16><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
+    topk_refine_kernel<MOEV_ACT_BF16><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
                                                                        cfg->score, cfg->routed_scale);
   }
   return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;

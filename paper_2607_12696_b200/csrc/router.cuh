@@ -15,7 +15,15 @@
 
 namespace moev {
 
-constexpr int kRouterKS = 32;  // K extent of one split-K slice
+constexpr int kRouterMaxKS = 64;  // largest K extent of one split-K slice
+
+// K extent of a slice: the hidden dimension is cut into about one slice per SM (one wave of
+// CTAs), in multiples of 4 columns.
+inline int router_slice_width(int H, int n_sm) {
+  int ks = (H + n_sm - 1) / n_sm;
+  ks = (ks + 3) & ~3;
+  return ks < 4 ? 4 : (ks > kRouterMaxKS ? kRouterMaxKS : ks);
+}
 
 // bf16 bit pattern -> double without the fp64 conversion unit (exact for normal numbers;
 // zeros / subnormals / non-finite take the conversion instruction).
@@ -25,6 +33,16 @@ __device__ __forceinline__ double bf16_bits_to_double(uint32_t b) {
   return __hiloint2double((int)hi, 0);
 }
 
+// fp32 -> double by integer operations (exact; zeros / subnormals / non-finite take the
+// conversion instruction)
+__device__ __forceinline__ double f32_to_double_int(float f) {
+  const uint32_t b = __float_as_uint(f);
+  const uint32_t e = (b >> 23) & 0xFFu;
+  if (e == 0u || e == 0xFFu) return (double)f;
+  const uint32_t hi = (b & 0x80000000u) | (((b & 0x7FFFFFFFu) >> 3) + (896u << 20));
+  return __hiloint2double((int)hi, (int)(b << 29));
+}
+
 template <int AFMT>
 __device__ __forceinline__ float load_act1(const void* x, size_t idx) {
   if (AFMT == MOEV_ACT_FP32) return __ldg(static_cast<const float*>(x) + idx);
@@ -32,92 +50,96 @@ __device__ __forceinline__ float load_act1(const void* x, size_t idx) {
 }
 
 // part[c, t, e] = sum_{h in slice c} x[t,h] * Wr[e,h]  (fp32, sequential over the slice)
-// part_x2[c, t] = sum_{h in slice c} x[t,h]^2,  part_w2max[c] = max_e sum_{h in slice c} Wr[e,h]^2
-// (so that sum_c part_w2max[c] >= max_e ||Wr[e,:]||^2).
-// Grid: one CTA per K slice of kRouterKS columns; 256 threads, thread (ty, tx) owns the 8 x 8
-// block of tokens 8*ty.. and experts tx + 32*j of each 64-token x 256-expert tile.
+// part_x2[c, t] = sum_{h in slice c} x[t,h]^2,
+// part_w2max[c, j] = max over the experts of tile j of sum_{h in slice c} Wr[e,h]^2
+// (so that sum_c max_j part_w2max[c, j] >= max_e ||Wr[e,:]||^2).
+// Grid: (K slices of ks columns, tiles of 64 experts); ks a multiple of 4, <= kRouterMaxKS.
+// 256 threads; thread (ty, tx) owns tokens 4 ty .. 4 ty + 3 and experts tx + 16 j of each
+// 64-token x 64-expert tile.  Small CTAs (several per SM) hide the load latencies.
+constexpr int kRouterETile = 64;
+inline size_t router_partial_smem(int ks) { return (size_t)ks * (68 + 65) * sizeof(float); }
+
 template <int AFMT>
 __global__ void __launch_bounds__(256) router_partial_kernel(const void* __restrict__ x,
                                                              const float* __restrict__ router_w,
                                                              float* __restrict__ part,
                                                              float* __restrict__ part_x2,
                                                              float* __restrict__ part_w2max, int gamma,
-                                                             int H, int E) {
-  constexpr int KS = kRouterKS;
+                                                             int H, int E, int KS) {
   __shared__ float wmax_s[8];
-  float w2max = 0.f;
-  __shared__ float x_s[KS][64 + 4];    // [k][token]
-  __shared__ float w_s[KS][256 + 1];   // [k][expert]
-  const int c = blockIdx.x, tid = threadIdx.x, tx = tid & 31, ty = tid >> 5;
+  extern __shared__ __align__(16) float rp_smem[];
+  float (*x_s)[64 + 4] = reinterpret_cast<float (*)[64 + 4]>(rp_smem);            // [k][token]
+  float (*w_s)[64 + 1] = reinterpret_cast<float (*)[64 + 1]>(rp_smem + KS * 68);  // [k][expert]
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int c = blockIdx.x, e0 = blockIdx.y * kRouterETile;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4, lane = tid & 31, warp = tid >> 5;
   const int k0 = c * KS, kn = min(KS, H - k0);
-  for (int e0 = 0; e0 < E; e0 += 256) {
-    __syncthreads();
-    // router tile -> shared, transposed; also the squared row norms of this slice
-    for (int i = tid; i < 256 * (KS / 4); i += 256) {
-      int er = i / (KS / 4), kq = (i % (KS / 4)) * 4;
+  // router tile -> shared, transposed
+  // (16 lanes per expert row, one float4 each; no integer division in the index arithmetic)
+  for (int er = tid >> 4; er < kRouterETile; er += 16) {
+    const int kq = (tid & 15) * 4;
+    if (kq < KS) {
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (e0 + er < E && kq < kn) v = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)(e0 + er) * H + k0 + kq));
       w_s[kq][er] = v.x; w_s[kq + 1][er] = v.y; w_s[kq + 2][er] = v.z; w_s[kq + 3][er] = v.w;
     }
+  }
+  __syncthreads();
+  float w2max = 0.f;
+  if (tid < kRouterETile && e0 + tid < E) {
+    float s2 = 0.f;
+    for (int k = 0; k < KS; ++k) s2 = fmaf(w_s[k][tid], w_s[k][tid], s2);
+    w2max = s2;
+  }
+  for (int t0 = 0; t0 < gamma; t0 += 64) {
     __syncthreads();
-    if (e0 + tid < E) {
-      float s2 = 0.f;
-      for (int k = 0; k < KS; ++k) s2 = fmaf(w_s[k][tid], w_s[k][tid], s2);
-      w2max = fmaxf(w2max, s2);
-    }
-    for (int t0 = 0; t0 < gamma; t0 += 64) {
-      __syncthreads();
-      for (int i = tid; i < 64 * KS; i += 256) {
-        int tr = i / KS, k = i % KS;
+    for (int tr = warp; tr < 64; tr += 8)
+      for (int k = lane; k < KS; k += 32) {
         float v = (t0 + tr < gamma && k < kn) ? load_act1<AFMT>(x, (size_t)(t0 + tr) * H + k0 + k) : 0.f;
         x_s[k][tr] = v;
       }
-      __syncthreads();
-      if (e0 == 0 && tid < 64 && t0 + tid < gamma) {
-        float s2 = 0.f;
-        for (int k = 0; k < KS; ++k) s2 = fmaf(x_s[k][tid], x_s[k][tid], s2);
-        part_x2[(size_t)c * gamma + t0 + tid] = s2;
-      }
-      float acc[8][8];
+    __syncthreads();
+    if (blockIdx.y == 0 && tid < 64 && t0 + tid < gamma) {
+      float s2 = 0.f;
+      for (int k = 0; k < KS; ++k) s2 = fmaf(x_s[k][tid], x_s[k][tid], s2);
+      part_x2[(size_t)c * gamma + t0 + tid] = s2;
+    }
+    float acc[4][4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < 4; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 #pragma unroll 4
-      for (int k = 0; k < KS; ++k) {
-        float xv[8], wv[8];
-        float4 xa = *reinterpret_cast<const float4*>(&x_s[k][ty * 8]);
-        float4 xb = *reinterpret_cast<const float4*>(&x_s[k][ty * 8 + 4]);
-        xv[0] = xa.x; xv[1] = xa.y; xv[2] = xa.z; xv[3] = xa.w;
-        xv[4] = xb.x; xv[5] = xb.y; xv[6] = xb.z; xv[7] = xb.w;
+    for (int k = 0; k < KS; ++k) {
+      float4 xa = *reinterpret_cast<const float4*>(&x_s[k][ty * 4]);
+      float xv[4] = {xa.x, xa.y, xa.z, xa.w}, wv[4];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) wv[j] = w_s[k][tx + 32 * j];
+      for (int j = 0; j < 4; ++j) wv[j] = w_s[k][tx + 16 * j];
 #pragma unroll
-        for (int i = 0; i < 8; ++i)
+      for (int i = 0; i < 4; ++i)
 #pragma unroll
-          for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(xv[i], wv[j], acc[i][j]);
-      }
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(xv[i], wv[j], acc[i][j]);
+    }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        int t = t0 + ty * 8 + i;
-        if (t < gamma) {
+    for (int i = 0; i < 4; ++i) {
+      int t = t0 + ty * 4 + i;
+      if (t < gamma) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            int e = e0 + tx + 32 * j;
-            if (e < E) part[((size_t)c * gamma + t) * E + e] = acc[i][j];
-          }
+        for (int j = 0; j < 4; ++j) {
+          int e = e0 + tx + 16 * j;
+          if (e < E) part[((size_t)c * gamma + t) * E + e] = acc[i][j];
         }
       }
     }
   }
-  // max over experts of the squared norm of this slice of the router rows
+  // max over this tile's experts of the squared norm of this slice of the router rows
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) w2max = fmaxf(w2max, __shfl_xor_sync(0xffffffffu, w2max, o));
-  if (tx == 0) wmax_s[ty] = w2max;
+  if (lane == 0) wmax_s[warp] = w2max;
   __syncthreads();
   if (tid == 0) {
     for (int w = 1; w < 8; ++w) w2max = fmaxf(w2max, wmax_s[w]);
-    part_w2max[c] = w2max;
+    part_w2max[(size_t)c * gridDim.y + blockIdx.y] = w2max;
   }
 }
 
@@ -130,60 +152,76 @@ struct RouteOut {  // optional caller-visible copies (may be null)
   int32_t* n_active;
 };
 
-// One CTA (256 threads) per token.  Shared memory: l32[E] floats | cand[E] ints | L[E] doubles.
+// One CTA (kRefineThreads threads) per token.  Shared memory: L[E] doubles | l32[E] floats | cand[E] ints.
+constexpr int kRefineThreads = 512;
+constexpr int kRefineWarps = kRefineThreads / 32;
+constexpr int kRefineCand = 12;  // candidates re-evaluated per pass over the token's row
+
 template <int AFMT>
-__global__ void __launch_bounds__(256) topk_refine_kernel(Tables T, RouteOut O, const void* __restrict__ x,
-                                                          const float* __restrict__ router_w,
-                                                          const float* __restrict__ part,
-                                                          const float* __restrict__ part_x2,
-                                                          const float* __restrict__ part_w2max,
-                                                          float* __restrict__ y32, int gamma, int H, int E,
-                                                          int k, int n_slices, int score, float routed_scale) {
+__global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, RouteOut O, const void* __restrict__ x,
+                                                                     const float* __restrict__ router_w,
+                                                                     const float* __restrict__ part,
+                                                                     const float* __restrict__ part_x2,
+                                                                     const float* __restrict__ part_w2max,
+                                                                     float* __restrict__ y32, int gamma, int H, int E,
+                                                                     int k, int n_slices, int ks, int score,
+                                                                     float routed_scale) {
   extern __shared__ double sm_d[];
   double* L = sm_d;                                    // [E] refined logits of the candidates
   float* l32 = reinterpret_cast<float*>(sm_d + E);     // [E]
   int32_t* cand = reinterpret_cast<int32_t*>(l32 + E); // [E]
-  __shared__ double red[8][8];
-  __shared__ float redf[8];
-  __shared__ float thr_s;
+  __shared__ double red[kRefineWarps][kRefineCand];
+  __shared__ float redf[kRefineWarps], redw[kRefineWarps];
   __shared__ int ncand_s;
   const int t = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  asm volatile("griddepcontrol.wait;" ::: "memory");               // router partials are complete
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   // zero this token's row of the fp32 combine accumulator
-  for (int i = tid; i < H / 4; i += 256)
+  for (int i = tid; i < H / 4; i += kRefineThreads)
     reinterpret_cast<float4*>(y32 + (size_t)t * H)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  // ---- fp32 logits of this token and the norms for the error bound
-  for (int e = tid; e < E; e += 256) {
-    const float* pp = part + (size_t)t * E + e;
+  // ---- fp32 logits of this token (two threads per expert when the block is wide enough)
+  {
+    const int split = (2 * E <= kRefineThreads) ? 2 : 1;
     const size_t cs = (size_t)gamma * E;
-    float s = 0.f;
-    int c = 0;
-    for (; c + 8 <= n_slices; c += 8) {
-      float v[8];
+    for (int base = 0; base < E * split; base += kRefineThreads) {  // one trip when split == 2
+      const int idx = base + tid;
+      const bool act = idx < E * split;
+      const int e = act ? idx / split : 0, half = idx % split;
+      const float* pp = part + (size_t)t * E + e;
+      float s = 0.f;
+      int c = act ? half : n_slices;
+      for (; c + 15 * split < n_slices; c += 16 * split) {
+        float v[16];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) v[i] = __ldg(pp + (size_t)(c + i) * cs);
+        for (int i = 0; i < 16; ++i) v[i] = __ldg(pp + (size_t)(c + i * split) * cs);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) s += v[i];
+        for (int i = 0; i < 16; ++i) s += v[i];
+      }
+      for (; c < n_slices; c += split) s += __ldg(pp + (size_t)c * cs);
+      if (split == 2) s += __shfl_xor_sync(0xffffffffu, s, 1);  // all lanes reach this point
+      if (act && half == 0) l32[e] = s;
     }
-    for (; c < n_slices; ++c) s += __ldg(pp + (size_t)c * cs);
-    l32[e] = s;
   }
   float x2 = 0.f, w2 = 0.f;
-  for (int c = tid; c < n_slices; c += 256) {
+  const int n_et = (E + kRouterETile - 1) / kRouterETile;
+  for (int c = tid; c < n_slices; c += kRefineThreads) {
     x2 += part_x2[(size_t)c * gamma + t];
-    w2 += part_w2max[c];
+    float m = 0.f;
+    for (int j = 0; j < n_et; ++j) m = fmaxf(m, part_w2max[(size_t)c * n_et + j]);
+    w2 += m;
   }
   x2 = warp_sum(x2);
   w2 = warp_sum(w2);
-  if (lane == 0) { redf[warp] = x2; red[warp][0] = (double)w2; }
+  if (lane == 0) { redf[warp] = x2; redw[warp] = w2; }
   __syncthreads();
   if (warp == 0) {
     float xs = 0.f, wm = 0.f;
-    for (int w = 0; w < 8; ++w) { xs += redf[w]; wm += (float)red[w][0]; }
+    for (int w = 0; w < kRefineWarps; ++w) { xs += redf[w]; wm += redw[w]; }
     // |fp32 logit - exact| <= gamma_n * sum|x w| <= n u ||x|| ||w||, n = roundings on the longest path
     // (slice length + number of slices + the norm sums' own error, covered by the factor 1.25)
-    const float n_round = (float)(kRouterKS + n_slices + 4);
+    const float n_round = (float)(ks + n_slices + 4);
     const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
     // ---- fp32 top-k: value of the k-th largest logit
     constexpr int PL = kMaxE / 32;
@@ -222,59 +260,56 @@ __global__ void __launch_bounds__(256) topk_refine_kernel(Tables T, RouteOut O, 
       if (in) cand[n + __popc(m & ((1u << lane) - 1u))] = e;
       n += __popc(m);
     }
-    if (lane == 0) { ncand_s = n; thr_s = thr; }
+    if (lane == 0) ncand_s = n;
   }
   __syncthreads();
   const int ncand = ncand_s;
 
-  // ---- exact (fp64) logits of the candidates, 8 at a time; every thread owns chunks of 8 columns
+  // ---- exact (fp64) logits of the candidates, kRefineCand at a time; a thread owns groups of 4 columns
   float amax = 0.f;
-  for (int c0 = 0; c0 < ncand; c0 += 8) {
-    double acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    const int nc = min(8, ncand - c0);
-    for (int h8 = tid; h8 < H / 8; h8 += 256) {
-      double xv[8];
-      if constexpr (AFMT == MOEV_ACT_BF16) {
-        uint4 v = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + h8);
-        uint32_t wd[4] = {v.x, v.y, v.z, v.w};
+  for (int c0 = 0; c0 < ncand; c0 += kRefineCand) {
+    double acc[kRefineCand];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+    for (int q = 0; q < kRefineCand; ++q) acc[q] = 0.0;
+    const int nc = min(kRefineCand, ncand - c0);
+    for (int h4 = tid; h4 < H / 4; h4 += kRefineThreads) {
+      double xv[4];
+      if constexpr (AFMT == MOEV_ACT_BF16) {
+        uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + h4);
+        uint32_t wd[2] = {v.x, v.y};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
           xv[2 * i] = bf16_bits_to_double(wd[i] & 0xffffu);
           xv[2 * i + 1] = bf16_bits_to_double(wd[i] >> 16);
           if (c0 == 0) amax = fmaxf(amax, fmaxf(fabsf(__uint_as_float(wd[i] << 16)), fabsf(__uint_as_float(wd[i] & 0xffff0000u))));
         }
       } else {
-        float f[8];
-        load_act8<AFMT>(x, (size_t)t * H + 8 * (size_t)h8, f);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { xv[i] = (double)f[i]; if (c0 == 0) amax = fmaxf(amax, fabsf(f[i])); }
+        float4 f = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + h4);
+        xv[0] = (double)f.x; xv[1] = (double)f.y; xv[2] = (double)f.z; xv[3] = (double)f.w;
+        if (c0 == 0) amax = fmaxf(amax, fmaxf(fmaxf(fabsf(f.x), fabsf(f.y)), fmaxf(fabsf(f.z), fabsf(f.w))));
       }
-      float4 wa[8], wb[8];
+      float4 wv[kRefineCand];
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
-        if (q < nc) {
-          const float4* wp = reinterpret_cast<const float4*>(router_w + (size_t)cand[c0 + q] * H) + 2 * h8;
-          wa[q] = __ldg(wp);
-          wb[q] = __ldg(wp + 1);
-        }
+      for (int q = 0; q < kRefineCand; ++q)
+        if (q < nc) wv[q] = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)cand[c0 + q] * H) + h4);
 #pragma unroll
-      for (int q = 0; q < 8; ++q)
+      for (int q = 0; q < kRefineCand; ++q)
         if (q < nc) {
-          acc[q] = fma(xv[0], (double)wa[q].x, acc[q]); acc[q] = fma(xv[1], (double)wa[q].y, acc[q]);
-          acc[q] = fma(xv[2], (double)wa[q].z, acc[q]); acc[q] = fma(xv[3], (double)wa[q].w, acc[q]);
-          acc[q] = fma(xv[4], (double)wb[q].x, acc[q]); acc[q] = fma(xv[5], (double)wb[q].y, acc[q]);
-          acc[q] = fma(xv[6], (double)wb[q].z, acc[q]); acc[q] = fma(xv[7], (double)wb[q].w, acc[q]);
+          acc[q] = fma(xv[0], (double)wv[q].x, acc[q]); acc[q] = fma(xv[1], (double)wv[q].y, acc[q]);
+          acc[q] = fma(xv[2], (double)wv[q].z, acc[q]); acc[q] = fma(xv[3], (double)wv[q].w, acc[q]);
         }
     }
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      double a = warp_sum(acc[q]);
-      if (lane == 0) red[warp][q] = a;
+    for (int q = 0; q < kRefineCand; ++q) {
+      if (q < nc) {
+        double a = warp_sum(acc[q]);
+        if (lane == 0) red[warp][q] = a;
+      }
     }
     __syncthreads();
     if (tid < nc) {
       double a = 0.0;
-      for (int w = 0; w < 8; ++w) a += red[w][tid];
+      for (int w = 0; w < kRefineWarps; ++w) a += red[w][tid];
       L[c0 + tid] = a;
     }
     __syncthreads();
@@ -288,7 +323,7 @@ __global__ void __launch_bounds__(256) topk_refine_kernel(Tables T, RouteOut O, 
   if (warp == 0) {
     if (lane == 0) {
       float am = 0.f;
-      for (int w = 0; w < 8; ++w) am = fmaxf(am, redf[w]);
+      for (int w = 0; w < kRefineWarps; ++w) am = fmaxf(am, redf[w]);
       int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
       ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
       T.tok_scale[t] = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
@@ -354,6 +389,8 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   float* w_s = reinterpret_cast<float*>(sm + 3 * E + A);
   __shared__ int32_t warp_tot_cnt[32], warp_tot_flag[32], warp_tot_unit[32], n_union_s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  asm volatile("griddepcontrol.wait;" ::: "memory");               // top-k tables are complete
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
   __syncthreads();
