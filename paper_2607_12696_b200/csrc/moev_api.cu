@@ -7,6 +7,7 @@
 #include "common.cuh"
 #include "ffn_simt.cuh"
 #include "ffn_tc.cuh"
+#include "ffn_tc_mx.cuh"
 #include "router.cuh"
 
 using namespace moev;
@@ -129,6 +130,8 @@ EncodeTiledFn encode_tiled_fn() {
 // Can the tensor-core kernel run this shape?  (Otherwise AUTO resolves to the SIMT kernels.)
 bool tc_eligible(const moev_config& c) {
   if (c.afmt != MOEV_ACT_BF16) return false;
+  if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: K axes in half chunks of 64, >= 4 chunks per row
+    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 512 && c.I >= 128;
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
   if (c.H % 128 || c.I % 128) return false;
   const int bk = c.wfmt == MOEV_W_BF16 ? 64 : 128;
@@ -153,6 +156,22 @@ bool encode_weight_map(CUtensorMap* m, const moev_config& c, const void* ptr, in
   return r == CUDA_SUCCESS;
 }
 
+// MXFP4: [n_mat, N, K] 4-bit codes -> 4-D map {128 elements, half chunks of 64 (stride 32 bytes),
+// rows, matrices} with the "16 x U4 in 16 bytes" element type (expands into the padded layout
+// kind::mxf8f6f4 reads), 128B swizzle.
+bool encode_weight_map_mx(CUtensorMap* m, const void* ptr, int n_mat, int N, int K) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {128, (cuuint64_t)(K / 64 - 1), (cuuint64_t)N, (cuuint64_t)n_mat};
+  cuuint64_t strides[3] = {32, (cuuint64_t)K / 2, (cuuint64_t)K / 2 * (cuuint64_t)N};
+  cuuint32_t box[4] = {128, 1, 128, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 4, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
 // Find or build the descriptors of this layer (cache keyed by the six weight pointers).
 const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
   const void* key[6] = {L->w_gate, L->w_up, L->w_down, L->sh_gate, L->sh_up, L->sh_down};
@@ -162,13 +181,15 @@ const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
   c->tmap_next = (c->tmap_next + 1) % kTmapCache;
   t.valid = false;
   const moev_config& g = c->cfg;
-  bool ok = encode_weight_map(&t.map[0], g, L->w_gate, g.E, g.I, g.H) &&
-            encode_weight_map(&t.map[1], g, L->w_up, g.E, g.I, g.H) &&
-            encode_weight_map(&t.map[2], g, L->w_down, g.E, g.H, g.I);
+  auto enc = [&](CUtensorMap* m, const void* ptr, int n_mat, int N, int K) {
+    if (reinterpret_cast<uintptr_t>(ptr) & 31u) return false;  // the 4-bit element type needs 32-byte alignment
+    return g.wfmt == MOEV_W_MXFP4 ? encode_weight_map_mx(m, ptr, n_mat, N, K) : encode_weight_map(m, g, ptr, n_mat, N, K);
+  };
+  bool ok = enc(&t.map[0], L->w_gate, g.E, g.I, g.H) && enc(&t.map[1], L->w_up, g.E, g.I, g.H) &&
+            enc(&t.map[2], L->w_down, g.E, g.H, g.I);
   if (ok && g.n_shared > 0)
-    ok = encode_weight_map(&t.map[3], g, L->sh_gate, g.n_shared, g.I, g.H) &&
-         encode_weight_map(&t.map[4], g, L->sh_up, g.n_shared, g.I, g.H) &&
-         encode_weight_map(&t.map[5], g, L->sh_down, g.n_shared, g.H, g.I);
+    ok = enc(&t.map[3], L->sh_gate, g.n_shared, g.I, g.H) && enc(&t.map[4], L->sh_up, g.n_shared, g.I, g.H) &&
+         enc(&t.map[5], L->sh_down, g.n_shared, g.H, g.I);
   else if (ok) { t.map[3] = t.map[0]; t.map[4] = t.map[1]; t.map[5] = t.map[2]; }
   if (!ok) return nullptr;
   memcpy(t.key, key, sizeof(key));
@@ -211,6 +232,22 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
 #endif
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
   launch_k(tc::grouped_ffn_tc_kernel<WFMT>, dim3(c->n_sm), dim3(tc::kThreads), tc::kSmemBytes, st, ev == nullptr,
+           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
+  if (ev) cudaEventRecord(ev[4], st);
+}
+
+void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const void* x, int gamma, cudaStream_t st,
+                   cudaEvent_t* ev) {
+  const moev_config& g = c->cfg;
+  tcmx::Params P{};
+  P.units = c->T.units; P.n_units = c->T.n_units; P.task_counter = c->T.task_counter;
+  P.slot_token = c->T.slot_token; P.slot_w = c->T.slot_w; P.tok_scale = c->T.tok_scale; P.x = x; P.y32 = c->y32;
+  P.s_gate = static_cast<const uint8_t*>(L->s_gate); P.s_up = static_cast<const uint8_t*>(L->s_up);
+  P.s_down = static_cast<const uint8_t*>(L->s_down);
+  P.sh_s_gate = static_cast<const uint8_t*>(L->sh_s_gate); P.sh_s_up = static_cast<const uint8_t*>(L->sh_s_up);
+  P.sh_s_down = static_cast<const uint8_t*>(L->sh_s_down);
+  P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
+  launch_k(tcmx::grouped_ffn_mx_kernel, dim3(c->n_sm), dim3(tcmx::kThreads), tcmx::kSmemBytes, st, ev == nullptr,
            tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
   if (ev) cudaEventRecord(ev[4], st);
 }
@@ -268,7 +305,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   c->n_sm = prop.multiProcessorCount;
   c->resolved_impl = (cfg->impl != MOEV_IMPL_SIMT && tc_ok) ? MOEV_IMPL_TCGEN05 : MOEV_IMPL_SIMT;
   if (c->resolved_impl == MOEV_IMPL_TCGEN05)
-    c->unit_cap = cfg->wfmt == MOEV_W_BF16 ? tc::Fmt<MOEV_W_BF16>::kMC : tc::Fmt<MOEV_W_FP8E4M3_B128>::kMC;
+    c->unit_cap = cfg->wfmt == MOEV_W_BF16 ? tc::Fmt<MOEV_W_BF16>::kMC
+                  : cfg->wfmt == MOEV_W_MXFP4 ? tcmx::kMC : tc::Fmt<MOEV_W_FP8E4M3_B128>::kMC;
   const size_t G = cfg->max_tokens, E = cfg->E, K = cfg->top_k, A = G * K;
   const size_t slots = A + (size_t)cfg->n_shared * G;
   const size_t act_b = cfg->afmt == MOEV_ACT_FP32 ? 4 : 2;
@@ -319,6 +357,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(tc::grouped_ffn_tc_kernel<MOEV_W_FP8E4M3_B128>,
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(tcmx::grouped_ffn_mx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      tcmx::kSmemBytes) == cudaSuccess;
     }
   }
   if (!ok) {
@@ -417,6 +457,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);
+    else if (g.wfmt == MOEV_W_MXFP4) launch_mx_ffn(c, tm, layer, x, gamma, st, ev);
     else launch_tc_ffn<MOEV_W_FP8E4M3_B128>(c, tm, layer, x, gamma, st, ev);
   } else if (g.afmt == MOEV_ACT_FP32) launch_simt_ffn_w<MOEV_ACT_FP32>(c, L, x, gamma, st, ev);
   else launch_simt_ffn_w<MOEV_ACT_BF16>(c, L, x, gamma, st, ev);
