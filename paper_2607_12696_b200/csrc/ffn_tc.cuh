@@ -26,8 +26,9 @@
 // epilogue; h is split the same way and the down-projection block scale (again one scalar per
 // 128 x 128 tile) is applied in the epilogue.
 //
-// Warps: 0 = TMA producer + task scheduler, 1 = MMA issuer, 2..5 = epilogue (TMEM lane
-// quarters), 6..9 = activation producers.  All mbarrier waits are bounded; on expiry the CTA
+// Warps: 0 = TMA producer + task scheduler, 1 and 10 = MMA issuers (gate chain / up chain,
+// and alternate W_down tiles: one thread cannot issue MMAs fast enough to keep up with the
+// weight stream), 2..5 = epilogue (TMEM lane quarters), 6..9 = activation producers.  All mbarrier waits are bounded; on expiry the CTA
 // raises an abort flag, writes the timeout status word and every role leaves its loop.
 #pragma once
 #include <cuda.h>
@@ -38,7 +39,7 @@
 namespace moev {
 namespace tc {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;  // 11 warps
 constexpr int kStages = 5;                  // weight ring
 constexpr int kStageBytes = 32 * 1024;      // two 128 x 128-byte tiles
 constexpr int kBSlots = 3;                  // activation-operand ring
@@ -233,12 +234,13 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   const int n_dstage = (HT + TPS - 1) / TPS;
 
   if (tid == 0) {
-    for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 1); }
-    for (int i = 0; i < kBSlots; ++i) { ptx::mbar_init(&S.b_full[i], 128); ptx::mbar_init(&S.b_empty[i], 1); }
-    ptx::mbar_init(&S.acc_full, 1); ptx::mbar_init(&S.acc_empty, 128);
-    ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 1);
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 1); ptx::mbar_init(&S.d_empty[i], 128); }
-    for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 257); }
+    // barriers the MMA issuers complete by tcgen05.commit count 2: one arrival per issuer
+    for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
+    for (int i = 0; i < kBSlots; ++i) { ptx::mbar_init(&S.b_full[i], 128); ptx::mbar_init(&S.b_empty[i], 2); }
+    ptx::mbar_init(&S.acc_full, 2); ptx::mbar_init(&S.acc_empty, 128);
+    ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 2);
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 128); }
+    for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     S.abort_flag = 0;
     ptx::fence_mbar_init();
@@ -322,8 +324,9 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         td = td_next;
       }
     }
-  } else if (warp == 1) {
-    // ===================================================== MMA issuer (one lane)
+  } else if (warp == 1 || warp == 10) {
+    // ===================================================== MMA issuers (one lane each)
+    const int issuer = warp == 1 ? 0 : 1;  // 0: gate chain and even W_down tiles, 1: up chain and odd tiles
     if (lane == 0) {
       uint32_t it = 0, bit = 0, tcount = 0, dsc = 0, q = 0;
       bool ok = true;
@@ -367,13 +370,11 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           const uint32_t ba = b_lo0 + sb * (kBSlotBytes >> 4);
           const uint32_t acc0 = kc ? 1u : 0u;
           { MOEV_STAT_BEGIN();
-          issue_mma<WFMT>(d_gate, wa, ba, idesc, acc0);
-          issue_mma<WFMT>(d_up, wa + 1024, ba + (kFp8 ? 512 : 0), idesc, acc0);
+          const uint32_t dacc = issuer ? d_up : d_gate;
+          const uint32_t wa_i = wa + (issuer ? 1024 : 0), ba_i = ba + ((issuer && kFp8) ? 512 : 0);
+          issue_mma<WFMT>(dacc, wa_i, ba_i, idesc, acc0);
 #pragma unroll
-          for (int j = 1; j < 4; ++j) {
-            issue_mma<WFMT>(d_gate, wa + 2 * j, ba + 2 * j, idesc, 1u);
-            issue_mma<WFMT>(d_up, wa + 1024 + 2 * j, ba + (kFp8 ? 512 : 0) + 2 * j, idesc, 1u);
-          }
+          for (int j = 1; j < 4; ++j) issue_mma<WFMT>(dacc, wa_i + 2 * j, ba_i + 2 * j, idesc, 1u);
           MOEV_STAT_END(8); }
           { MOEV_STAT_BEGIN();
           ptx::mma_commit(&S.w_empty[s]);
@@ -402,13 +403,14 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           MOEV_STAT_BEGIN();
           if constexpr (kFp8) {
             const int nt = (2 * ds + 1 < HT) ? 2 : 1;
-            for (int tl = 0; tl < nt; ++tl) {
+            const int tl = issuer;  // each issuer owns one tile of the stage
+            if (tl < nt) {
               const uint32_t d_down = tmem + 128 + (db * TPS + tl) * 64;
 #pragma unroll
               for (int j = 0; j < 4; ++j)
                 issue_mma<WFMT>(d_down, wa + tl * 1024 + 2 * j, h_lo0 + 2 * j, idesc, j ? 1u : 0u);
             }
-          } else {
+          } else if ((ds & 1) == issuer) {  // one tile per stage: the issuers alternate stages
             const uint32_t d_down = tmem + 128 + db * 64;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf)
@@ -428,7 +430,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #ifdef MOEV_TC_STATS
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
-      if (P.stats)
+      if (P.stats && issuer == 0)
         for (int i = 0; i < 16; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
 #endif
     }

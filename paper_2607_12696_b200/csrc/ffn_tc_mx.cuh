@@ -39,7 +39,7 @@ using tc::safe_exponent;
 using tc::pow2i;
 using tc::split4_e4m3;
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 352;  // 11 warps: TMA, MMA issuer 0, 4 epilogue, 4 producers, MMA issuer 1
 constexpr int kBSlots = 3;
 constexpr int kBSlotBytes = 8 * 1024 + 1024;  // [64 x 128 B] activation tile | gate scale atom | up scale atom
 constexpr int kDsfSlots = 4;                  // down-phase scale-factor ring (two 512-byte atoms per slot)
@@ -50,7 +50,7 @@ constexpr int kTmemCols = 512;
 constexpr int kColSfGate = 384;   // 4 slots x 4 columns
 constexpr int kColSfUp = 400;     // 4 slots x 4 columns
 constexpr int kColSfDown = 416;   // 4 slots x 2 tiles x 4 columns
-constexpr int kColSfB = 448;      // unit scales of the activation operand (4 columns)
+constexpr int kColSfB = 448;      // unit scales of the activation operand (4 columns per MMA issuer)
 constexpr int kSfRing = 4;
 constexpr int kTileBytes = kStages * kStageBytes + kBSlots * kBSlotBytes + kHTileBytes + kDsfSlots * 1024 + 512;
 constexpr int kCtlBytes = 8 * 1024;
@@ -69,6 +69,9 @@ struct Params {
   const uint8_t *sh_s_gate, *sh_s_up, *sh_s_down;
   int32_t* status;
   int32_t gamma, H, I, A;
+#ifdef MOEV_TC_STATS
+  unsigned long long* stats;  // [grid][16] cycles MMA issuer 0 spent per wait / issue class (debug builds)
+#endif
 };
 
 struct Smem {
@@ -179,13 +182,14 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   const int kb_gu = H / 32, kb_dn = I / 32;  // scale blocks per row
 
   if (tid == 0) {
-    for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 1); }
-    for (int i = 0; i < kBSlots; ++i) { ptx::mbar_init(&S.b_full[i], 128); ptx::mbar_init(&S.b_empty[i], 1); }
-    for (int i = 0; i < kDsfSlots; ++i) { ptx::mbar_init(&S.dsf_full[i], 128); ptx::mbar_init(&S.dsf_empty[i], 1); }
-    ptx::mbar_init(&S.acc_full, 1); ptx::mbar_init(&S.acc_empty, 128);
-    ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 1);
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 1); ptx::mbar_init(&S.d_empty[i], 128); }
-    for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 257); }
+    // barriers completed by tcgen05.commit count 2: one arrival per MMA issuer
+    for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
+    for (int i = 0; i < kBSlots; ++i) { ptx::mbar_init(&S.b_full[i], 128); ptx::mbar_init(&S.b_empty[i], 2); }
+    for (int i = 0; i < kDsfSlots; ++i) { ptx::mbar_init(&S.dsf_full[i], 128); ptx::mbar_init(&S.dsf_empty[i], 2); }
+    ptx::mbar_init(&S.acc_full, 2); ptx::mbar_init(&S.acc_empty, 128);
+    ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 2);
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 128); }
+    for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     S.abort_flag = 0;
     ptx::fence_mbar_init();
@@ -263,14 +267,21 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         td = td_next;
       }
     }
-  } else if (warp == 1) {
-    // ===================================================== MMA issuer (one lane)
+  } else if (warp == 1 || warp == 10) {
+    // ===================================================== MMA issuers (one lane each): issuer 0 runs the gate chain
+    // and the even W_down tiles, issuer 1 the up chain and the odd tiles
+    const int issuer = warp == 1 ? 0 : 1;
     if (lane == 0) {
       uint32_t it = 0, bit = 0, tcount = 0, dsc = 0, q = 0;
       bool ok = true;
       const uint32_t w_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(w_ring));
       const uint32_t h_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(h_tile));
-      sf_copy(tmem + kColSfB, ptx::smem_u32(sfb_unit));  // unit activation scales, once
+#ifdef MOEV_TC_STATS
+      unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+      const long long st_begin = clock64();
+#endif
+      const uint32_t sfb_col = tmem + kColSfB + 4 * issuer;
+      sf_copy(sfb_col, ptx::smem_u32(sfb_unit));  // unit activation scales, once per issuer
       for (;; ++tcount) {
         const int id = next_task(S, q, abortp, P.status, false);
         if (id < 0) break;
@@ -278,51 +289,63 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         const Unit u = P.units[td.unit];
         const uint32_t N = (uint32_t)((2 * u.m + 15) & ~15);
         const uint32_t d_gate = tmem, d_up = tmem + 64;
-        ok = ptx::bounded_wait(&S.acc_empty, (tcount & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+        { MOEV_STAT_BEGIN();
+          ok = ptx::bounded_wait(&S.acc_empty, (tcount & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          MOEV_STAT_END(3); }
         if (!ok) break;
         ptx::tc_fence_after();
         for (int kc = 0; kc < KC && ok; ++kc, ++it, ++bit) {
           const int s = it % kStages, sb = bit % kBSlots, sf = bit % kSfRing;
-          ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs) &&
-               ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          { MOEV_STAT_BEGIN();
+            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(1); }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(2); }
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t bslot = ptx::smem_u32(b_ring + sb * kBSlotBytes);
-          sf_copy(tmem + kColSfGate + 4 * sf, bslot + 8192);
-          sf_copy(tmem + kColSfUp + 4 * sf, bslot + 8192 + 512);
-          const uint32_t wa = w_lo0 + s * (kStageBytes >> 4);
+          const uint32_t sfa_col = tmem + (issuer ? kColSfUp : kColSfGate) + 4 * sf;
+          sf_copy(sfa_col, bslot + 8192 + 512 * issuer);
+          const uint32_t wa = w_lo0 + s * (kStageBytes >> 4) + 1024 * issuer;
           const uint32_t ba = ptx::desc_lo_sw128(bslot);
+          const uint32_t dacc = issuer ? d_up : d_gate;
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t acc = (kc | j) ? 1u : 0u;
-            const uint32_t idesc = idesc_mx(N, j);
-            mma_mx(d_gate, wa + 2 * j, ba + 2 * j, idesc, acc, tmem + kColSfGate + 4 * sf, tmem + kColSfB);
-            mma_mx(d_up, wa + 1024 + 2 * j, ba + 2 * j, idesc, acc, tmem + kColSfUp + 4 * sf, tmem + kColSfB);
-          }
+          for (int j = 0; j < 4; ++j)
+            mma_mx(dacc, wa + 2 * j, ba + 2 * j, idesc_mx(N, j), (kc | j) ? 1u : 0u, sfa_col, sfb_col);
           ptx::mma_commit(&S.w_empty[s]);
           ptx::mma_commit(&S.b_empty[sb]);
         }
         if (!ok) break;
         ptx::mma_commit(&S.acc_full);
-        ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+        { MOEV_STAT_BEGIN();
+          ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          MOEV_STAT_END(4); }
         if (!ok) break;
         ptx::tc_fence_after();
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc, ++it) {
           const int db = dsc & 1, s = it % kStages, sfs = dsc % kDsfSlots;
-          ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs) &&
-               ptx::bounded_wait(&S.dsf_full[sfs], (dsc / kDsfSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs) &&
-               ptx::bounded_wait(&S.d_empty[db], ((dsc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          { MOEV_STAT_BEGIN();
+            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(5); }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.dsf_full[sfs], (dsc / kDsfSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(12); }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.d_empty[db], ((dsc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(6); }
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t wa = w_lo0 + s * (kStageBytes >> 4);
           const int nt = (2 * ds + 1 < HT) ? 2 : 1;
-          for (int tl = 0; tl < nt; ++tl) {
+          const int tl = issuer;
+          if (tl < nt) {
             const uint32_t sfcol = tmem + kColSfDown + (sfs * 2 + tl) * 4;
             sf_copy(sfcol, ptx::smem_u32(dsf_ring + sfs * 1024 + tl * 512));
             const uint32_t d_down = tmem + 128 + (db * 2 + tl) * 64;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-              mma_mx(d_down, wa + tl * 1024 + 2 * j, h_lo0 + 2 * j, idesc_mx(N, j), j ? 1u : 0u, sfcol, tmem + kColSfB);
+              mma_mx(d_down, wa + tl * 1024 + 2 * j, h_lo0 + 2 * j, idesc_mx(N, j), j ? 1u : 0u, sfcol, sfb_col);
           }
           ptx::mma_commit(&S.d_full[db]);
           ptx::mma_commit(&S.w_empty[s]);
@@ -331,6 +354,12 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
       }
+#ifdef MOEV_TC_STATS
+      st_acc[0] = (unsigned long long)(clock64() - st_begin);
+      st_acc[7] = tcount;
+      if (P.stats && issuer == 0)
+        for (int i = 0; i < 16; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
+#endif
     }
   } else if (warp < 6) {
     // ===================================================== epilogue warps (TMEM lane quarter = warp % 4)

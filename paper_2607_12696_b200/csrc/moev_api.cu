@@ -247,6 +247,9 @@ void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.sh_s_gate = static_cast<const uint8_t*>(L->sh_s_gate); P.sh_s_up = static_cast<const uint8_t*>(L->sh_s_up);
   P.sh_s_down = static_cast<const uint8_t*>(L->sh_s_down);
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
+#ifdef MOEV_TC_STATS
+  P.stats = c->tc_stats;
+#endif
   launch_k(tcmx::grouped_ffn_mx_kernel, dim3(c->n_sm), dim3(tcmx::kThreads), tcmx::kSmemBytes, st, ev == nullptr,
            tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
   if (ev) cudaEventRecord(ev[4], st);
