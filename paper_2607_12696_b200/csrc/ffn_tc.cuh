@@ -678,15 +678,18 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         // 128-element chunk.  All rows of the next chunk are fetched before this one is converted.
         constexpr int kMaxPass = Fmt<MOEV_W_FP8E4M3_B128>::kMC / 4;
         const int passes = (m - pw + 3) >> 2;  // rows pw + 4 i < m
-        uint2 nxt[kMaxPass];
+        // x is fetched three K chunks ahead (a chunk lasts less than one trip to L2)
+        uint2 n0[kMaxPass], n1[kMaxPass], n2[kMaxPass];
         const uint8_t* xrow[kMaxPass];
 #pragma unroll
         for (int i = 0; i < kMaxPass; ++i) {
-          nxt[i] = make_uint2(0, 0);
+          n0[i] = n1[i] = n2[i] = make_uint2(0, 0);
           xrow[i] = nullptr;
           if (i < passes) {
             xrow[i] = reinterpret_cast<const uint8_t*>(xb + (size_t)S.p_tok[par][pw + 4 * i] * H) + lane * 8;
-            nxt[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i]));
+            n0[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i]));
+            if (1 < KC) n1[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + 256));
+            if (2 < KC) n2[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + 512));
           }
         }
         for (int kc = 0; kc < KC && ok; ++kc, ++bit) {
@@ -694,8 +697,10 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           uint2 cur[kMaxPass];
 #pragma unroll
           for (int i = 0; i < kMaxPass; ++i) {
-            cur[i] = nxt[i];
-            if (i < passes && kc + 1 < KC) nxt[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + (size_t)(kc + 1) * 256));
+            cur[i] = n0[i];
+            n0[i] = n1[i];
+            n1[i] = n2[i];
+            if (i < passes && kc + 3 < KC) n2[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + (size_t)(kc + 3) * 256));
           }
           ok = warp_wait(&S.b_empty[sb], ((bit / kBSlots) & 1) ^ 1, abortp, P.status);
           if (!ok) break;

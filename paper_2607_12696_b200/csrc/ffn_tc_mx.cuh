@@ -27,7 +27,6 @@ namespace moev {
 namespace tcmx {
 
 using tc::kStageBytes;
-using tc::kStages;
 using tc::kTaskQ;
 using tc::kWaitBudgetNs;
 using tc::TaskDesc;
@@ -40,6 +39,7 @@ using tc::pow2i;
 using tc::split4_e4m3;
 
 constexpr int kThreads = 352;  // 11 warps: TMA, MMA issuer 0, 4 epilogue, 4 producers, MMA issuer 1
+constexpr int kStages = 4;   // weight ring: a 32 KB stage holds 16 KB of packed weights
 constexpr int kBSlots = 3;
 constexpr int kBSlotBytes = 8 * 1024 + 1024;  // [64 x 128 B] activation tile | gate scale atom | up scale atom
 constexpr int kDsfSlots = 4;                  // down-phase scale-factor ring (two 512-byte atoms per slot)
@@ -52,7 +52,9 @@ constexpr int kColSfUp = 400;     // 4 slots x 4 columns
 constexpr int kColSfDown = 416;   // 4 slots x 2 tiles x 4 columns
 constexpr int kColSfB = 448;      // unit scales of the activation operand (4 columns per MMA issuer)
 constexpr int kSfRing = 4;
-constexpr int kTileBytes = kStages * kStageBytes + kBSlots * kBSlotBytes + kHTileBytes + kDsfSlots * 1024 + 512;
+// staged gate / up scale blocks of a task's 128-row slice: [task parity][gate, up][128 rows x K/32 bytes]
+constexpr int kScStageBytes = 11776;  // >= 128 * (H / 32) bytes, H <= 2944
+constexpr int kTileBytes = kStages * kStageBytes + kBSlots * kBSlotBytes + kHTileBytes + kDsfSlots * 1024 + 512 + 4 * kScStageBytes;
 constexpr int kCtlBytes = 8 * 1024;
 constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
 
@@ -81,7 +83,7 @@ struct Smem {
   uint64_t acc_full, acc_empty, h_full, h_empty;
   uint64_t d_full[2], d_empty[2];
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
-  uint64_t ep_bar;
+  uint64_t ep_bar, pr_bar;
   volatile int32_t tq_task[kTaskQ];
   uint32_t tmem_base;
   volatile int abort_flag;
@@ -150,11 +152,10 @@ __device__ __forceinline__ int next_task(Smem& S, uint32_t& q, volatile int* abo
 // packed little-endian; rows or blocks outside the matrix get the unit scale 127.
 __device__ __forceinline__ uint32_t load_scale4(const uint8_t* s, int e, int n_rows, int kblocks, int row, int kb0) {
   if (row >= n_rows) return 0x7F7F7F7Fu;
-  const uint8_t* p = s + ((size_t)e * n_rows + row) * kblocks + kb0;
-  uint32_t v = 0;
-#pragma unroll
-  for (int i = 0; i < 4; ++i) v |= (uint32_t)(kb0 + i < kblocks ? __ldg(p + i) : (uint8_t)127) << (8 * i);
-  return v;
+  // kblocks = K / 32 is even (K % 64 == 0) and kb0 is even, so the four bytes are 2-byte aligned
+  // and lie inside the row (kb0 + 4 <= kblocks for every chunk coordinate)
+  const uint16_t* p = reinterpret_cast<const uint16_t*>(s + ((size_t)e * n_rows + row) * kblocks + kb0);
+  return (uint32_t)__ldg(p) | ((uint32_t)__ldg(p + 1) << 16);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -169,6 +170,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   uint8_t* h_tile = b_ring + kBSlots * kBSlotBytes;  // 27 KB after a 1 KB-aligned start: still 1 KB aligned
   uint8_t* dsf_ring = h_tile + kHTileBytes;
   uint8_t* sfb_unit = dsf_ring + kDsfSlots * 1024;
+  uint8_t* sc_stage = sfb_unit + 512;  // 16-byte aligned
   static_assert((kBSlots * kBSlotBytes) % 1024 == 0, "h tile alignment");
   static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
   Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
@@ -191,6 +193,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 128); }
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
+    ptx::mbar_init(&S.pr_bar, 128);
     S.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -358,7 +361,8 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
       if (P.stats && issuer == 0)
-        for (int i = 0; i < 16; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
+        for (int i = 0; i < 16; ++i)
+          if (i < 8 || i >= 12) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
 #endif
     }
   } else if (warp < 6) {
@@ -511,13 +515,33 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     // ===================================================== producers (4 warps): activation tiles and scale atoms
     const int pw = warp - 6;
     const int pt = tid - 192;  // 0..127: the weight-tile row whose scale bytes this thread moves
-    uint32_t bit = 0, tcount = 0, dsc = 0, q = 0;
+    uint32_t bit = 0, tcount = 0, dsc = 0, q = 0, gph = 0;
     bool ok = true;
     const uint16_t* xb = static_cast<const uint16_t*>(P.x);
     const uint32_t sf_off = (uint32_t)(pt & 31) * 16u + (uint32_t)(pt >> 5) * 4u;  // this row's word in a scale atom
-    for (;; ++tcount) {
-      const int id = next_task(S, q, abortp, P.status, true);
-      if (id < 0) break;
+    // Gate / up scale bytes of a task's slice are one contiguous block per matrix; they are
+    // staged in shared memory with 16-byte asynchronous copies (one latency per task, no
+    // divergent loads in the chunk loop).  The copy for the next task is issued before this
+    // task's down-phase work.
+    auto stage_scales = [&](int id, int par) {
+      const TaskDesc td = decode_task(id, n_units, n_slices);
+      const Unit u = P.units[td.unit];
+      const uint8_t* sg = u.shared ? P.sh_s_gate : P.s_gate;
+      const uint8_t* su = u.shared ? P.sh_s_up : P.s_up;
+      const int rows = min(128, I - td.slice * 128);
+      const int n16 = rows * kb_gu / 16;  // kb_gu % 2 == 0 and rows % 64 == 0: a whole number of 16-byte pieces
+      const size_t off = ((size_t)u.expert * I + (size_t)td.slice * 128) * kb_gu;
+      uint8_t* dg = sc_stage + (par * 2 + 0) * kScStageBytes;
+      uint8_t* du = sc_stage + (par * 2 + 1) * kScStageBytes;
+      for (int i = pt; i < n16; i += 128) {
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(dg + i * 16)), "l"(sg + off + (size_t)i * 16) : "memory");
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(du + i * 16)), "l"(su + off + (size_t)i * 16) : "memory");
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    int id = next_task(S, q, abortp, P.status, true);
+    if (id >= 0) stage_scales(id, 0);
+    for (; id >= 0; ++tcount) {
       const TaskDesc td = decode_task(id, n_units, n_slices);
       const Unit u = P.units[td.unit];
       const int slice = td.slice;
@@ -529,9 +553,13 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         S.p_tscale[par][r] = P.tok_scale[tok];
       }
       __syncwarp();
-      const uint8_t* sg = u.shared ? P.sh_s_gate : P.s_gate;
-      const uint8_t* su = u.shared ? P.sh_s_up : P.s_up;
       const uint8_t* sd = u.shared ? P.sh_s_down : P.s_down;
+      // this task's staged scales have landed (every thread waits for its own copies, then all meet)
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) break;
+      const uint8_t* stg = sc_stage + (par * 2 + 0) * kScStageBytes;
+      const uint8_t* stu = sc_stage + (par * 2 + 1) * kScStageBytes;
+      const bool row_ok = slice * 128 + pt < I;
 
       // ---- gate/up phase: per K chunk the activation tile (hi/lo of x * 2^p_t) and the two scale atoms
       constexpr int kMaxPass = kMC / 4;
@@ -546,28 +574,35 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         const bool valid = e0 >= kc * 128 && e0 < H;  // a ragged tail chunk re-reads 64 elements that must be zero
         return valid ? __ldg(reinterpret_cast<const uint2*>(xrow[i] + e0)) : make_uint2(0u, 0u);
       };
-      uint2 nxt[kMaxPass];
-      uint32_t nsg, nsu;
+      // x is fetched three K chunks ahead (a chunk lasts less than one trip to L2)
+      uint2 n0[kMaxPass], n1[kMaxPass], n2[kMaxPass];
 #pragma unroll
-      for (int i = 0; i < kMaxPass; ++i) nxt[i] = (i < passes) ? load_x(i, 0) : make_uint2(0u, 0u);
-      {
-        const int kb0 = half_chunk_coord(0, H) * 2;
-        nsg = load_scale4(sg, u.expert, I, kb_gu, slice * 128 + pt, kb0);
-        nsu = load_scale4(su, u.expert, I, kb_gu, slice * 128 + pt, kb0);
+      for (int i = 0; i < kMaxPass; ++i) {
+        n0[i] = n1[i] = n2[i] = make_uint2(0u, 0u);
+        if (i < passes) {
+          n0[i] = load_x(i, 0);
+          if (1 < KC) n1[i] = load_x(i, 1);
+          if (2 < KC) n2[i] = load_x(i, 2);
+        }
       }
       for (int kc = 0; kc < KC && ok; ++kc, ++bit) {
         const int sb = bit % kBSlots;
         uint2 cur[kMaxPass];
-        const uint32_t csg = nsg, csu = nsu;
 #pragma unroll
         for (int i = 0; i < kMaxPass; ++i) {
-          cur[i] = nxt[i];
-          if (i < passes && kc + 1 < KC) nxt[i] = load_x(i, kc + 1);
+          cur[i] = n0[i];
+          n0[i] = n1[i];
+          n1[i] = n2[i];
+          if (i < passes && kc + 3 < KC) n2[i] = load_x(i, kc + 3);
         }
-        if (kc + 1 < KC) {
-          const int kb0 = half_chunk_coord((kc + 1) * 128, H) * 2;
-          nsg = load_scale4(sg, u.expert, I, kb_gu, slice * 128 + pt, kb0);
-          nsu = load_scale4(su, u.expert, I, kb_gu, slice * 128 + pt, kb0);
+        // this row's four scale bytes of the chunk, from the staged block (2-byte aligned)
+        uint32_t csg = 0x7F7F7F7Fu, csu = 0x7F7F7F7Fu;
+        if (row_ok) {
+          const int bo = pt * kb_gu + half_chunk_coord(kc * 128, H) * 2;
+          const uint16_t* pg = reinterpret_cast<const uint16_t*>(stg + bo);
+          const uint16_t* pu = reinterpret_cast<const uint16_t*>(stu + bo);
+          csg = (uint32_t)pg[0] | ((uint32_t)pg[1] << 16);
+          csu = (uint32_t)pu[0] | ((uint32_t)pu[1] << 16);
         }
         ok = warp_wait(&S.b_empty[sb], ((bit / kBSlots) & 1) ^ 1, abortp, P.status);
         if (!ok) break;
@@ -595,16 +630,31 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       }
       if (!ok) break;
 
-      // ---- down phase: scale atoms of the W_down tiles of every ring stage
+      // ---- the next task is known by now (ids are published one task ahead): start staging its scales
+      const int id_next = next_task(S, q, abortp, P.status, true);
+      if (id_next == -2) { ok = false; break; }
+      if (id_next >= 0) stage_scales(id_next, par ^ 1);
+
+      // ---- down phase: scale atoms of the W_down tiles of every ring stage (gathered: the four
+      // bytes of a row are 2-byte aligned and rows are K/32 bytes apart)
       const int kbd = half_chunk_coord(slice * 128, I) * 2;
-      uint32_t nd0 = load_scale4(sd, u.expert, H, kb_dn, pt, kbd);
-      uint32_t nd1 = load_scale4(sd, u.expert, H, kb_dn, 128 + pt, kbd);
+      uint32_t da[4], db2[4];  // stages ds .. ds + 3 (rotated)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        da[i] = db2[i] = 0x7F7F7F7Fu;
+        if (i < n_dstage) {
+          da[i] = load_scale4(sd, u.expert, H, kb_dn, (2 * i) * 128 + pt, kbd);
+          db2[i] = load_scale4(sd, u.expert, H, kb_dn, (2 * i + 1) * 128 + pt, kbd);
+        }
+      }
       for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc) {
         const int sfs = dsc % kDsfSlots;
-        const uint32_t c0v = nd0, c1v = nd1;
-        if (ds + 1 < n_dstage) {
-          nd0 = load_scale4(sd, u.expert, H, kb_dn, (2 * ds + 2) * 128 + pt, kbd);
-          nd1 = load_scale4(sd, u.expert, H, kb_dn, (2 * ds + 3) * 128 + pt, kbd);
+        const uint32_t c0v = da[0], c1v = db2[0];
+#pragma unroll
+        for (int i = 0; i < 3; ++i) { da[i] = da[i + 1]; db2[i] = db2[i + 1]; }
+        if (ds + 4 < n_dstage) {
+          da[3] = load_scale4(sd, u.expert, H, kb_dn, (2 * ds + 8) * 128 + pt, kbd);
+          db2[3] = load_scale4(sd, u.expert, H, kb_dn, (2 * ds + 9) * 128 + pt, kbd);
         }
         ok = warp_wait(&S.dsf_empty[sfs], ((dsc / kDsfSlots) & 1) ^ 1, abortp, P.status);
         if (!ok) break;
@@ -614,6 +664,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         ptx::mbar_arrive(&S.dsf_full[sfs]);
       }
       if (!ok) break;
+      id = id_next;
     }
   }
 

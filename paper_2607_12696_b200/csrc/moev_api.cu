@@ -131,7 +131,8 @@ EncodeTiledFn encode_tiled_fn() {
 bool tc_eligible(const moev_config& c) {
   if (c.afmt != MOEV_ACT_BF16) return false;
   if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: K axes in half chunks of 64, >= 4 chunks per row
-    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 512 && c.I >= 128;
+    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 512 && c.I >= 128 &&
+           128 * (c.H / 32) <= tcmx::kScStageBytes;  // a slice's gate/up scale block is staged in shared memory
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
   if (c.H % 128 || c.I % 128) return false;
   const int bk = c.wfmt == MOEV_W_BF16 ? 64 : 128;
