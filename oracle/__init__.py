@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
         _lib.oracle_moe_verify.restype = C.c_int32
         _lib.oracle_moe_dense.restype = C.c_int32
         _lib.oracle_num_threads.restype = C.c_int32
+        _lib.oracle_select_drafts.restype = C.c_int32
     return _lib
 
 
@@ -229,3 +230,22 @@ def moe_dense(cfg: Config, layer: dict, x: np.ndarray, gamma: int) -> np.ndarray
     if rc != 0:
         raise ValueError("oracle_moe_dense: bad arguments")
     return y
+
+
+def select_drafts(parent, P, pred, gamma: int, eps: float = 1e-6, buffer0=None, global_cost: bool = False):
+    """Algorithm 1 on a draft tree.  pred: uint32 [n, W] bitmaps.  Returns (selected, costs, buffer)."""
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    P = np.ascontiguousarray(P, dtype=np.float32)
+    pred = np.ascontiguousarray(pred, dtype=np.uint32)
+    n, W = pred.shape
+    if buffer0 is not None:
+        buffer0 = np.ascontiguousarray(buffer0, dtype=np.uint32)
+    sel = np.full(gamma, -1, dtype=np.int32)
+    costs = np.zeros(gamma, dtype=np.int32)
+    buf = np.zeros(W, dtype=np.uint32)
+    cnt = lib().oracle_select_drafts(C.c_int32(n), C.c_int32(W), _p(parent), _p(P), _p(pred), _p(buffer0),
+                                     C.c_int32(gamma), C.c_float(eps), C.c_int32(int(global_cost)), _p(sel),
+                                     _p(costs), _p(buf))
+    if cnt < 0:
+        raise ValueError("oracle_select_drafts: bad arguments")
+    return sel[:cnt].copy(), costs[:cnt].copy(), buf

@@ -419,3 +419,68 @@ int32_t oracle_num_threads(void) {
   return 1;
 #endif
 }
+
+/* ------------------------------------------------- cost-aware draft selection */
+
+/* Algorithm 1 (cost-aware draft selection), Eqs. 7-10 -- the step that runs before the
+ * verification pass and shrinks its expert union.
+ *
+ * Tree of n nodes in topological order (parent[i] < i, parent[root] = -1); P[i] is the
+ * cumulative draft probability of node i; pred[i] is the predicted expert set of node i
+ * over all MoE layers as a bitmap of W 32-bit words (bit (l*E + e) = pair (l, e), Eq. 4);
+ * buffer0 is the initial expert buffer B_0 (W words, may be NULL = empty).
+ *   E_traj(i)  = OR of pred over the path root -> i                      (Eq. 7)
+ *   dCost(i|B) = | E_traj(i) \ B |                                       (Eq. 8)
+ *   score(i)   = P(i) / (dCost + eps)                                    (Eq. 9)
+ * gamma rounds: score every unselected node, take the arg-max (exact ties: the lowest
+ * index, so a parent precedes its children), add it to S and OR its E_traj into B.
+ * global_cost != 0 is the ablation variant of Eq. 10: the cost is |E_traj(i)| and the
+ * buffer is not updated.  Scores are evaluated in IEEE binary32 (one rounded add, one
+ * rounded divide), the precision in which the arg-max is decided.
+ * Outputs: selected[gamma] node indices in selection order; costs[gamma] the cost each had
+ * when chosen (may be NULL); buffer_out (W words, may be NULL) the final buffer.
+ * Returns the number selected (min(gamma, n)) or -1 on bad arguments. */
+int32_t oracle_select_drafts(int32_t n, int32_t W, const int32_t *parent, const float *P,
+                             const uint32_t *pred, const uint32_t *buffer0, int32_t gamma,
+                             float eps, int32_t global_cost, int32_t *selected, int32_t *costs,
+                             uint32_t *buffer_out) {
+  if (n < 1 || W < 1 || gamma < 1 || !parent || !P || !pred || !selected) return -1;
+  uint32_t *traj = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)n * (size_t)W);
+  uint32_t *B = (uint32_t *)calloc((size_t)W, sizeof(uint32_t));
+  char *taken = (char *)calloc((size_t)n, 1);
+  if (buffer0) memcpy(B, buffer0, sizeof(uint32_t) * (size_t)W);
+  for (int i = 0; i < n; ++i) {
+    if (parent[i] >= i) { free(traj); free(B); free(taken); return -1; }
+    for (int w = 0; w < W; ++w)
+      traj[(size_t)i * W + w] =
+          pred[(size_t)i * W + w] | (parent[i] >= 0 ? traj[(size_t)parent[i] * W + w] : 0u);
+  }
+  int count = 0;
+  while (count < gamma && count < n) {
+    int best = -1, best_cost = 0;
+    float best_score = 0.f;
+    for (int i = 0; i < n; ++i) {
+      if (taken[i]) continue;
+      int cost = 0;
+      for (int w = 0; w < W; ++w) {
+        uint32_t v = traj[(size_t)i * W + w];
+        if (!global_cost) v &= ~B[w];
+        while (v) { v &= v - 1; ++cost; }
+      }
+      volatile float den = (float)cost + eps; /* rounded to binary32 before the divide */
+      float score = P[i] / den;
+      if (best < 0 || score > best_score) { best = i; best_score = score; best_cost = cost; }
+    }
+    taken[best] = 1;
+    selected[count] = best;
+    if (costs) costs[count] = best_cost;
+    if (!global_cost)
+      for (int w = 0; w < W; ++w) B[w] |= traj[(size_t)best * W + w];
+    ++count;
+  }
+  if (buffer_out) memcpy(buffer_out, B, sizeof(uint32_t) * (size_t)W);
+  free(traj);
+  free(B);
+  free(taken);
+  return count;
+}

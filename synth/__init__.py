@@ -272,3 +272,43 @@ def layer_to_numpy(router_w: torch.Tensor, weights: dict) -> dict:
     for kname, v in weights.items():
         d[kname] = to_numpy(v)
     return d
+
+
+# ----------------------------------------------------------- draft trees (selection stage)
+
+def make_draft_tree(n_layers: int, E: int, K: int, depth: int = 3, branch: int = 2, seed_tag="tree",
+                    p_reuse: float = 0.7):
+    """A draft tree like the paper's setup (``depth`` drafting steps, top-``branch`` children
+    per node, root = the bonus token) with cumulative draft probabilities and predicted expert
+    sets (K experts per layer per node).  A child keeps each of its parent's predicted experts
+    with probability ``p_reuse`` (expert locality along a path) and redraws the rest.
+    Returns (parent int32 [n], P float32 [n], pred uint32 [n, ceil(n_layers*E/32)])."""
+    rs = np.random.RandomState(stream_seed(seed_tag, n_layers, E, K, depth, branch) % (2 ** 31))
+    parent, P, sets = [-1], [1.0], []
+    sets.append([rs.choice(E, K, replace=False) for _ in range(n_layers)])
+    frontier = [0]
+    for _ in range(depth):
+        nxt = []
+        for node in frontier:
+            probs = np.sort(rs.dirichlet(np.ones(branch + 1)))[::-1][:branch]
+            for b in range(branch):
+                parent.append(node)
+                P.append(P[node] * float(probs[b]))
+                child = []
+                for l in range(n_layers):
+                    keep = [e for e in sets[node][l] if rs.rand() < p_reuse]
+                    pool = [e for e in range(E) if e not in keep]
+                    extra = rs.choice(pool, K - len(keep), replace=False) if len(keep) < K else []
+                    child.append(np.array(list(keep) + list(extra), dtype=np.int64))
+                sets.append(child)
+                nxt.append(len(parent) - 1)
+        frontier = nxt
+    n = len(parent)
+    W = _cdiv(n_layers * E, 32)
+    pred = np.zeros((n, W), dtype=np.uint32)
+    for i in range(n):
+        for l in range(n_layers):
+            for e in sets[i][l]:
+                bit = l * E + int(e)
+                pred[i, bit >> 5] |= np.uint32(1 << (bit & 31))
+    return np.array(parent, dtype=np.int32), np.array(P, dtype=np.float32), pred
