@@ -181,6 +181,30 @@ moev_status moev_profile_enable(moev_ctx* ctx, int32_t on);
 moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[6]*/,
                               int32_t* calls);
 
+/* Cost-aware draft selection: Algorithm 1 of the paper (Sec. 4.2, Eqs. 7-10), the step that
+ * runs between drafting and verification and decides which gamma draft-tree nodes are verified.
+ *   n, parent [n]   draft tree in topological order: parent[i] < i, parent[root] = -1
+ *   P [n]           cumulative draft probability of every node (float32)
+ *   pred [n, W]     predicted expert set of every node as a bitmap over (layer, expert) pairs,
+ *                   bit l*E + e, W = ceil(L*E / 32) 32-bit words (Eq. 4)
+ *   buffer0 [W]     initial expert buffer B_0, or NULL for the empty set
+ *   E_traj(i) = OR of pred along root -> i (Eq. 7);  cost = |E_traj(i) \ B| (Eq. 8);
+ *   score = P(i) / (cost + eps) (Eq. 9), evaluated in binary32;  gamma rounds of arg-max
+ *   (exact ties: the lowest index, so a parent precedes its children), each followed by
+ *   B |= E_traj(chosen).  global_cost != 0 selects the ablation variant of Eq. 10: cost =
+ *   |E_traj(i)|, buffer not updated.
+ * Outputs: selected [gamma] (first min(gamma, n) entries, in selection order), costs [gamma]
+ * (cost of each choice when it was made; may be NULL), buffer_out [W] (final B; may be NULL),
+ * n_selected [1] (may be NULL).  traj_workspace [n, W] is caller-provided scratch.  All
+ * pointers are DEVICE pointers; one kernel is enqueued on cuda_stream; nothing is allocated.
+ * MOEV_EINVAL for n outside 1..65536, W < 1, gamma < 1, eps <= 0, null required pointers, or a
+ * bitmap too large for shared memory (W > ~50 000 words). */
+moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, const float* P,
+                               const uint32_t* pred, const uint32_t* buffer0, int32_t gamma, float eps,
+                               int32_t global_cost, uint32_t* traj_workspace, int32_t* selected,
+                               int32_t* costs, uint32_t* buffer_out, int32_t* n_selected,
+                               void* cuda_stream);
+
 /* Router top-k without any allocation.  (The paper has no counterpart: this entry point
  * exists for the integration constraints of some callers, not for the method.)
  *

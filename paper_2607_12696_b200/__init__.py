@@ -8,4 +8,4 @@ is missing or fails to load, importing :mod:`paper_2607_12696_b200.binding` rais
 from .binding import (ACT_BF16, ACT_FP32, IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05, SCORE_SIGMOID,  # noqa: F401
                       SCORE_SOFTMAX, W_BF16, W_FP32, W_FP8E4M3_B128, W_MXFP4, MoevConfig,
                       MoevError, MoeVerifier, expert_bytes, expert_code_bytes, lib, lib_path,
-                      route_topk_static, static_scratch_floats)
+                      route_topk_static, select_drafts, static_scratch_floats)

@@ -20,7 +20,7 @@ STATUS = {0: "MOEV_OK", 1: "MOEV_EINVAL", 2: "MOEV_EUNSUPPORTED", 3: "MOEV_ECUDA
 EXPORTS = ("moev_create", "moev_destroy", "moev_verify", "moev_verify_host", "moev_status_sync",
            "moev_last_error", "moev_expert_bytes", "moev_expert_code_bytes",
            "moev_launches_per_call", "moev_resolved_impl", "moev_profile_enable",
-           "moev_profile_read", "moev_route_topk_static", "moev_route_topk_static_scratch_floats")
+           "moev_profile_read", "moev_route_topk_static", "moev_route_topk_static_scratch_floats", "moev_select_drafts")
 
 
 class MoevError(RuntimeError):
@@ -115,6 +115,9 @@ def lib() -> C.CDLL:
                                              C.c_void_p, C.c_void_p, C.c_void_p]
         L.moev_route_topk_static_scratch_floats.restype = C.c_size_t
         L.moev_route_topk_static_scratch_floats.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+        L.moev_select_drafts.restype = C.c_int
+        L.moev_select_drafts.argtypes = [C.c_int32, C.c_int32] + [C.c_void_p] * 4 + [C.c_int32, C.c_float, C.c_int32] + \
+                                        [C.c_void_p] * 6
         _lib = L
     return _lib
 
@@ -142,6 +145,26 @@ def route_topk_static(cfg: MoevConfig, router_w: torch.Tensor, x: torch.Tensor, 
     if st != 0:
         raise MoevError(st, "moev_route_topk_static rejected the call (arguments, or the problem "
                             "exceeds the fixed scratch array)")
+
+
+def select_drafts(parent: torch.Tensor, P: torch.Tensor, pred: torch.Tensor, gamma: int, eps: float = 1e-6,
+                  buffer0: torch.Tensor = None, global_cost: bool = False):
+    """moev_select_drafts: Algorithm 1 on device tensors (parent int32 [n], P float32 [n], pred
+    int32/uint32 bitmaps [n, W]).  Returns device tensors (selected [gamma], costs [gamma],
+    buffer [W], n_selected [1]); asynchronous on the current stream."""
+    n, W = pred.shape
+    dev = pred.device
+    traj = torch.empty(n, W, dtype=torch.int32, device=dev)
+    selected = torch.full((gamma,), -1, dtype=torch.int32, device=dev)
+    costs = torch.zeros(gamma, dtype=torch.int32, device=dev)
+    buf = torch.zeros(W, dtype=torch.int32, device=dev)
+    nsel = torch.zeros(1, dtype=torch.int32, device=dev)
+    st = lib().moev_select_drafts(n, W, parent.data_ptr(), P.data_ptr(), pred.data_ptr(), _ptr(buffer0), gamma,
+                                  eps, int(global_cost), traj.data_ptr(), selected.data_ptr(), costs.data_ptr(),
+                                  buf.data_ptr(), nsel.data_ptr(), C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if st != 0:
+        raise MoevError(st, "moev_select_drafts rejected the call")
+    return selected, costs, buf, nsel
 
 
 def static_scratch_floats(H: int, E: int, gamma: int) -> int:

@@ -9,6 +9,7 @@
 #include "ffn_tc.cuh"
 #include "ffn_tc_mx.cuh"
 #include "router.cuh"
+#include "select.cuh"
 
 using namespace moev;
 
@@ -593,6 +594,25 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
                                                                        gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
                                                                        cfg->score, cfg->routed_scale);
   }
+  return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
+}
+
+moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, const float* P, const uint32_t* pred,
+                               const uint32_t* buffer0, int32_t gamma, float eps, int32_t global_cost,
+                               uint32_t* traj_workspace, int32_t* selected, int32_t* costs, uint32_t* buffer_out,
+                               int32_t* n_selected, void* cuda_stream) {
+  if (n < 1 || n > 65536 || W < 1 || gamma < 1 || !parent || !P || !pred || !traj_workspace || !selected)
+    return MOEV_EINVAL;
+  if (!(eps > 0.f)) return MOEV_EINVAL;  // eps avoids the division by zero (Eq. 9)
+  const size_t smem = ((size_t)W + 96 + (size_t)(n + 31) / 32) * sizeof(uint32_t);
+  if (smem > 200 * 1024) return MOEV_EINVAL;
+  if (smem > 48 * 1024 &&
+      cudaFuncSetAttribute(select_drafts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    cudaGetLastError();
+    return MOEV_ECUDA;
+  }
+  select_drafts_kernel<<<1, 1024, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
+      n, W, parent, P, pred, buffer0, gamma, eps, global_cost, traj_workspace, selected, costs, buffer_out, n_selected);
   return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
 }
 

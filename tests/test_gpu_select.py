@@ -1,0 +1,64 @@
+"""GPU parity of the cost-aware draft selection kernel (Algorithm 1) against the oracle:
+selected nodes, their costs and the final expert buffer must be bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_12696_b200 as moev
+import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(parent, P, pred, gamma, eps=1e-6, buffer0=None, global_cost=False):
+    dev = "cuda"
+    tp = torch.from_numpy(parent).to(dev)
+    tP = torch.from_numpy(P).to(dev)
+    tpred = torch.from_numpy(pred.view(np.int32)).to(dev)
+    tb = None if buffer0 is None else torch.from_numpy(buffer0.view(np.int32)).to(dev)
+    sel, costs, buf, nsel = moev.select_drafts(tp, tP, tpred, gamma, eps, tb, global_cost)
+    torch.cuda.synchronize()
+    k = int(nsel.item())
+    return sel.cpu().numpy()[:k], costs.cpu().numpy()[:k], buf.cpu().numpy().view(np.uint32)
+
+
+@pytest.mark.parametrize("L,E,K,depth,branch,gamma", [
+    (58, 256, 8, 3, 2, 4),      # DeepSeek-V3.1-sized footprint, the paper's tree (3 steps x top-2) and budget
+    (94, 128, 8, 3, 2, 4),      # Qwen3-235B-sized
+    (36, 128, 4, 3, 2, 4),      # GPT-OSS-sized
+    (58, 256, 8, 5, 2, 16),     # deeper tree, larger budget
+    (4, 32, 4, 6, 3, 64),       # 1093 nodes: more nodes than threads' warps, many rounds
+    (1, 16, 2, 2, 2, 100)])     # budget larger than the tree
+def test_selection_matches_oracle(L, E, K, depth, branch, gamma):
+    parent, P, pred = synth.make_draft_tree(L, E, K, depth=depth, branch=branch)
+    for glob in (False, True):
+        s_ref, c_ref, b_ref = oracle.select_drafts(parent, P, pred, gamma, eps=1e-6, global_cost=glob)
+        s, c, b = _run(parent, P, pred, gamma, global_cost=glob)
+        np.testing.assert_array_equal(s, s_ref)
+        np.testing.assert_array_equal(c, c_ref)
+        np.testing.assert_array_equal(b, b_ref)
+
+
+def test_selection_with_initial_buffer_and_ties():
+    parent, P, pred = synth.make_draft_tree(8, 64, 4, depth=4)
+    b0 = np.random.RandomState(3).randint(0, 2 ** 32, size=pred.shape[1], dtype=np.uint64).astype(np.uint32)
+    P = np.round(P * 8) / 8                      # coarse probabilities: many exact score ties
+    P[0] = 1.0
+    P = P.astype(np.float32)
+    s_ref, c_ref, b_ref = oracle.select_drafts(parent, P, pred, 12, eps=0.5, buffer0=b0)
+    s, c, b = _run(parent, P, pred, 12, eps=0.5, buffer0=b0)
+    np.testing.assert_array_equal(s, s_ref)
+    np.testing.assert_array_equal(c, c_ref)
+    np.testing.assert_array_equal(b, b_ref)
+
+
+def test_selection_rejects_bad_arguments():
+    parent, P, pred = synth.make_draft_tree(2, 16, 2, depth=2)
+    tp = torch.from_numpy(parent).cuda()
+    tP = torch.from_numpy(P).cuda()
+    tpred = torch.from_numpy(pred.view(np.int32)).cuda()
+    with pytest.raises(moev.MoevError):
+        moev.select_drafts(tp, tP, tpred, 0)
+    with pytest.raises(moev.MoevError):
+        moev.select_drafts(tp, tP, tpred, 2, eps=0.0)
