@@ -266,6 +266,10 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
       uint32_t it = 0, q = 0;
       bool ok = true;
+#ifdef MOEV_TC_STATS
+      unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+      const long long st_begin = clock64();
+#endif
       // Task ids are published one task ahead of the loads, so the other roles can prepare
       // their tables (and the first activation tiles) while this task still streams.
       auto fetch_publish = [&](TaskDesc& td) -> int {
@@ -296,7 +300,9 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
         for (int kc = 0; kc < KC && ok; ++kc, ++it) {
           const int s = it % kStages;
+          { MOEV_STAT_BEGIN();
           ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          MOEV_STAT_END(13); }
           if (!ok) break;
           uint8_t* dst = w_ring + s * kStageBytes;
           ptx::mbar_arrive_expect_tx(&S.w_full[s], kStageBytes);
@@ -305,7 +311,9 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         }
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
           const int s = it % kStages;
+          { MOEV_STAT_BEGIN();
           ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          MOEV_STAT_END(14); }
           if (!ok) break;
           uint8_t* dst = w_ring + s * kStageBytes;
           if constexpr (kFp8) {
@@ -323,6 +331,11 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         id = id_next;
         td = td_next;
       }
+#ifdef MOEV_TC_STATS
+      st_acc[15] = (unsigned long long)(clock64() - st_begin);
+      if (P.stats)
+        for (int i = 13; i < 16; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
+#endif
     }
   } else if (warp == 1 || warp == 10) {
     // ===================================================== MMA issuers (one lane each)
@@ -361,7 +374,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #ifdef MOEV_TC_STATS
             { unsigned long long dt = (unsigned long long)(clock64() - _t0);
               if (kc < 3) st_acc[12] += dt; else st_acc[2] += dt;
-              if (dt > 400) { st_acc[13] += 1; st_acc[14] += dt; } }
+            }
 #endif
             }
           if (!ok) break;
@@ -431,7 +444,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
       if (P.stats && issuer == 0)
-        for (int i = 0; i < 16; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
+        for (int i = 0; i < 13; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
 #endif
     }
   } else if (warp < 6) {

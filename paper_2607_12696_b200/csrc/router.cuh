@@ -437,13 +437,15 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   }
   __syncthreads();
 
-  // ---- phase 2b: work units for the tensor-core FFN: expert u of the union (then the shared
-  // experts) is cut into ceil(m / unit_cap) runs of at most unit_cap slots
+  // ---- phase 2b: work units for the tensor-core FFN: the shared experts, then expert u of the
+  // union, each cut into ceil(m / unit_cap) runs of at most unit_cap slots.  The shared experts
+  // see every token, so their tasks are the longest; first in unit order, they are never the
+  // last tasks handed out
   {
     const int U = n_union_s;
     int e = 0, slot0 = 0, m = 0, shared = 0;
-    if (tid < U) { e = T.union_ids[tid]; slot0 = T.offsets[tid]; m = cnt[e]; }
-    else if (tid < U + n_shared) { shared = 1; e = tid - U; slot0 = A + e * gamma; m = gamma; }
+    if (tid < n_shared) { shared = 1; e = tid; slot0 = A + e * gamma; m = gamma; }
+    else if (tid < U + n_shared) { e = T.union_ids[tid - n_shared]; slot0 = T.offsets[tid - n_shared]; m = cnt[e]; }
     int nch = (m + unit_cap - 1) / unit_cap, sc = nch;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
