@@ -15,6 +15,10 @@
 //      computes each 128-row tile of  O = Wd[:, slice] * h  into TMEM accumulators (two ring
 //      stages in flight); the epilogue scales by the routing weight and reduce-adds into the
 //      fp32 output accumulator y32 (split-K over the I slices).
+// The phases of consecutive tasks are software-pipelined: the weight stream and the MMAs run in
+// the order GU(0), GU(1), D(0), GU(2), D(1), ... (GU = gate/up phase, D = down phase), with two
+// G/P accumulator pairs in TMEM, so step 2 of a task overlaps the gate/up phase of the next one
+// and the tensor pipe and the weight stream never wait for the SwiGLU epilogue.
 // Every weight byte of an active expert is fetched from HBM by exactly one TMA load per unit
 // (units of one expert are adjacent in task order, so extra token runs hit L2).
 //
@@ -45,7 +49,7 @@ constexpr int kStageBytes = 32 * 1024;      // two 128 x 128-byte tiles
 constexpr int kBSlots = 3;                  // activation-operand ring
 constexpr int kNMax = 64;                   // widest N operand
 constexpr int kTaskQ = 4;                   // depth of the task-id queue between the roles
-constexpr int kTmemCols = 512;              // G 64 | P 64 | O[2 stages][<=2 tiles] 64 each
+constexpr int kTmemCols = 512;              // (G 64 | P 64) x 2 task parities | O[2 stages][<=2 tiles] 64 each
 constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // 2 s per wait
 
 // tiles (fp8: 160 + 48 + 8 KB, bf16: 160 + 24 + 16 KB) + 1 KB alignment slack + 8 KB control block
@@ -74,7 +78,7 @@ struct Params {
 struct Smem {
   uint64_t w_full[kStages], w_empty[kStages];
   uint64_t b_full[kBSlots], b_empty[kBSlots];
-  uint64_t acc_full, acc_empty, h_full, h_empty;
+  uint64_t acc_full[2], acc_empty[2], h_full, h_empty;
   uint64_t d_full[2], d_empty[2];
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar;  // epilogue group barrier (128 threads), bounded like every other wait
@@ -86,7 +90,6 @@ struct Smem {
   int32_t p_tok[2][kNMax];
   float p_tscale[2][kNMax];
   float p_sg[2][128], p_su[2][128];  // per K chunk: block scale * 2^-p (fp8)
-  float pscale_inv[2][2];            // [task parity][gate, up]: 2^p, read by the epilogue
   // epilogue tables, same scheme
   int32_t e_tok[2][kNMax];
   float e_w[2][kNMax];               // routing weight
@@ -223,7 +226,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   uint8_t* h_tile = b_ring + kBSlots * kBSlotBytes;
   static_assert(kStages * kStageBytes + kBSlots * F::kBSlotBytes + F::kHTileBytes <= kTileBytes, "tile budget");
   static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
-  static_assert(128 + 2 * TPS * 64 <= kTmemCols, "TMEM budget");
+  static_assert(256 + 2 * TPS * 64 <= kTmemCols, "TMEM budget");
   Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -237,7 +240,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     // barriers the MMA issuers complete by tcgen05.commit count 2: one arrival per issuer
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
     for (int i = 0; i < kBSlots; ++i) { ptx::mbar_init(&S.b_full[i], 128); ptx::mbar_init(&S.b_empty[i], 2); }
-    ptx::mbar_init(&S.acc_full, 2); ptx::mbar_init(&S.acc_empty, 128);
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.acc_full[i], 2); ptx::mbar_init(&S.acc_empty[i], 128); }
     ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 2);
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 128); }
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
@@ -288,16 +291,10 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         ++q;
         return id;
       };
-      TaskDesc td, td_next;
-      int id = fetch_publish(td);
-      while (ok && id >= 0) {
-        const int id_next = fetch_publish(td_next);
-        if (!ok) break;
-        const Unit u = P.units[td.unit];
-        const int slice = td.slice;
+      auto load_gu = [&](const TaskDesc& t) {
+        const Unit u = P.units[t.unit];
         const CUtensorMap* mg = u.shared ? &tm_sh_gate : &tm_gate;
         const CUtensorMap* mu = u.shared ? &tm_sh_up : &tm_up;
-        const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
         for (int kc = 0; kc < KC && ok; ++kc, ++it) {
           const int s = it % kStages;
           { MOEV_STAT_BEGIN();
@@ -306,9 +303,14 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           if (!ok) break;
           uint8_t* dst = w_ring + s * kStageBytes;
           ptx::mbar_arrive_expect_tx(&S.w_full[s], kStageBytes);
-          ptx::tma_load_3d(dst, mg, &S.w_full[s], kc * F::kBK, slice * 128, u.expert, ptx::kPolicyEvictFirst);
-          ptx::tma_load_3d(dst + 16384, mu, &S.w_full[s], kc * F::kBK, slice * 128, u.expert, ptx::kPolicyEvictFirst);
+          ptx::tma_load_3d(dst, mg, &S.w_full[s], kc * F::kBK, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
+          ptx::tma_load_3d(dst + 16384, mu, &S.w_full[s], kc * F::kBK, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
         }
+      };
+      auto load_down = [&](const TaskDesc& t) {
+        const Unit u = P.units[t.unit];
+        const int slice = t.slice;
+        const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
           const int s = it % kStages;
           { MOEV_STAT_BEGIN();
@@ -328,8 +330,27 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             ptx::tma_load_3d(dst + 16384, md, &S.w_full[s], slice * 128 + 64, ds * 128, u.expert, ptx::kPolicyEvictFirst);
           }
         }
-        id = id_next;
-        td = td_next;
+      };
+      // Stream order GU(0), GU(1), D(0), GU(2), D(1), ...; task t + 2 is published between the
+      // loads of GU(t + 1) and D(t), one down phase before its own loads begin.
+      TaskDesc td, td_next, td_nn;
+      int id = fetch_publish(td);
+      int id_next = -1;
+      if (ok && id >= 0) {
+        id_next = fetch_publish(td_next);
+        if (ok) load_gu(td);
+      }
+      while (ok && id >= 0) {
+        int id_nn = -1;
+        if (id_next >= 0) {
+          load_gu(td_next);
+          if (!ok) break;
+          id_nn = fetch_publish(td_nn);
+          if (!ok) break;
+        }
+        load_down(td);
+        id = id_next; td = td_next;
+        id_next = id_nn; td_next = td_nn;
       }
 #ifdef MOEV_TC_STATS
       st_acc[15] = (unsigned long long)(clock64() - st_begin);
@@ -350,19 +371,19 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
       const long long st_begin = clock64();
 #endif
-      for (;; ++tcount) {
-        const int id = next_task(S, q, abortp, P.status, false);
-        if (id < 0) break;
+      auto idesc_of = [&](int id) -> uint32_t {
         const TaskDesc td = decode_task(id, n_units, n_slices);
-        const Unit u = P.units[td.unit];
-        const int ncols = u.m * F::kColsPerTok;
-        const uint32_t N = (uint32_t)((ncols + 15) & ~15);
-        const uint32_t idesc = ptx::instr_desc(F::kKindFmt, F::kKindFmt, N);
-        const uint32_t d_gate = tmem, d_up = tmem + 64;
+        const int ncols = P.units[td.unit].m * F::kColsPerTok;
+        return ptx::instr_desc(F::kKindFmt, F::kKindFmt, (uint32_t)((ncols + 15) & ~15));
+      };
+      // gate/up phase of the g-th task of this CTA into accumulator pair g & 1
+      auto gate_up = [&](uint32_t g, uint32_t idesc) {
+        const uint32_t pb = g & 1u;
+        const uint32_t dacc = tmem + pb * 128 + (issuer ? 64 : 0);
         { MOEV_STAT_BEGIN();
-          ok = ptx::bounded_wait(&S.acc_empty, (tcount & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          ok = ptx::bounded_wait(&S.acc_empty[pb], ((g >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
           MOEV_STAT_END(3); }
-        if (!ok) break;
+        if (!ok) return;
         ptx::tc_fence_after();
         for (int kc = 0; kc < KC && ok; ++kc, ++it, ++bit) {
           const int s = it % kStages, sb = bit % kBSlots;
@@ -371,19 +392,13 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             MOEV_STAT_END(1); }
           { MOEV_STAT_BEGIN();
             ok = ok && ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-#ifdef MOEV_TC_STATS
-            { unsigned long long dt = (unsigned long long)(clock64() - _t0);
-              if (kc < 3) st_acc[12] += dt; else st_acc[2] += dt;
-            }
-#endif
-            }
+            MOEV_STAT_END(2); }
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t wa = w_lo0 + s * (kStageBytes >> 4);
           const uint32_t ba = b_lo0 + sb * (kBSlotBytes >> 4);
           const uint32_t acc0 = kc ? 1u : 0u;
           { MOEV_STAT_BEGIN();
-          const uint32_t dacc = issuer ? d_up : d_gate;
           const uint32_t wa_i = wa + (issuer ? 1024 : 0), ba_i = ba + ((issuer && kFp8) ? 512 : 0);
           issue_mma<WFMT>(dacc, wa_i, ba_i, idesc, acc0);
 #pragma unroll
@@ -394,8 +409,21 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           ptx::mma_commit(&S.b_empty[sb]);
           MOEV_STAT_END(9); }
         }
-        if (!ok) break;
-        ptx::mma_commit(&S.acc_full);
+        if (ok) ptx::mma_commit(&S.acc_full[pb]);
+      };
+      int id = next_task(S, q, abortp, P.status, false);
+      uint32_t idesc = 0;
+      if (id >= 0) { idesc = idesc_of(id); gate_up(0, idesc); }
+      for (; ok && id >= 0; ++tcount) {
+        // gate/up phase of the next task first: it overlaps the SwiGLU step of this one
+        const int id_next = next_task(S, q, abortp, P.status, false);
+        if (id_next == -2) break;
+        uint32_t idesc_next = 0;
+        if (id_next >= 0) {
+          idesc_next = idesc_of(id_next);
+          gate_up(tcount + 1, idesc_next);
+          if (!ok) break;
+        }
         { MOEV_STAT_BEGIN();
           ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
           MOEV_STAT_END(4); }
@@ -418,13 +446,13 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             const int nt = (2 * ds + 1 < HT) ? 2 : 1;
             const int tl = issuer;  // each issuer owns one tile of the stage
             if (tl < nt) {
-              const uint32_t d_down = tmem + 128 + (db * TPS + tl) * 64;
+              const uint32_t d_down = tmem + 256 + (db * TPS + tl) * 64;
 #pragma unroll
               for (int j = 0; j < 4; ++j)
                 issue_mma<WFMT>(d_down, wa + tl * 1024 + 2 * j, h_lo0 + 2 * j, idesc, j ? 1u : 0u);
             }
           } else if ((ds & 1) == issuer) {  // one tile per stage: the issuers alternate stages
-            const uint32_t d_down = tmem + 128 + db * 64;
+            const uint32_t d_down = tmem + 256 + db * 64;
 #pragma unroll
             for (int hf = 0; hf < 2; ++hf)
 #pragma unroll
@@ -439,6 +467,8 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         }
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
+        id = id_next;
+        idesc = idesc_next;
       }
 #ifdef MOEV_TC_STATS
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
@@ -472,12 +502,21 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         S.e_w[par][r] = w;
         S.e_inv[par][r] = kFp8 ? 1.f / P.tok_scale[tok] : 1.f;
       }
+      float ig = 1.f, iu = 1.f;  // fp8: the common powers of two the producers took out of the gate / up block scales
       if constexpr (kFp8) {
         const float* sd = u.shared ? P.sh_s_down : P.s_down;
         for (int ht = lane; ht < HT; ht += 32) S.e_sd[par][ht] = sd[((size_t)u.expert * HT + ht) * n_slices + slice];
+        const float* sg = (u.shared ? P.sh_s_gate : P.s_gate) + ((size_t)u.expert * n_slices + slice) * KC;
+        const float* su = (u.shared ? P.sh_s_up : P.s_up) + ((size_t)u.expert * n_slices + slice) * KC;
+        float mg = 0.f, mu = 0.f;
+        for (int kc = lane; kc < KC; kc += 32) { mg = fmaxf(mg, fabsf(__ldg(sg + kc))); mu = fmaxf(mu, fabsf(__ldg(su + kc))); }
+        mg = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mg)));
+        mu = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mu)));
+        ig = pow2i(safe_exponent(mg));
+        iu = pow2i(safe_exponent(mu));
       }
       __syncwarp();
-      ok = warp_wait(&S.acc_full, tcount & 1, abortp, P.status);
+      ok = warp_wait(&S.acc_full[par], (tcount >> 1) & 1, abortp, P.status);
       if (!ok) break;
       ptx::tc_fence_after();
       // h tile must be free: all down MMAs of the previous task have completed
@@ -485,14 +524,14 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       if (!ok) break;
 
       if constexpr (kFp8) {
-        const float ig = S.pscale_inv[par][0], iu = S.pscale_inv[par][1];
+        const uint32_t gp = tmem + lane_base + par * 128;
         float hv[32];
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 16) {
           if (c0 < 2 * m) {
             uint32_t g[16], p[16];
-            ptx::tmem_ld16(tmem + lane_base + c0, g);
-            ptx::tmem_ld16(tmem + lane_base + 64 + c0, p);
+            ptx::tmem_ld16(gp + c0, g);
+            ptx::tmem_ld16(gp + 64 + c0, p);
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
@@ -508,7 +547,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           }
         }
         ptx::tc_fence_before();
-        ptx::mbar_arrive(&S.acc_empty);  // G and P are in registers: the MMA warp may start the next task
+        ptx::mbar_arrive(&S.acc_empty[par]);  // G and P are in registers: the MMA warp may start the next task
         // per-token power-of-two scale from the amax over the 128 rows of the slice
 #pragma unroll
         for (int r = 0; r < 32; ++r) {
@@ -539,8 +578,8 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         for (int c0 = 0; c0 < 64; c0 += 16) {
           if (c0 < m) {
             uint32_t g[16], p[16];
-            ptx::tmem_ld16(tmem + lane_base + c0, g);
-            ptx::tmem_ld16(tmem + lane_base + 64 + c0, p);
+            ptx::tmem_ld16(tmem + lane_base + par * 128 + c0, g);
+            ptx::tmem_ld16(tmem + lane_base + par * 128 + 64 + c0, p);
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int r = 0; r < 16; ++r) {
@@ -557,7 +596,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           }
         }
         ptx::tc_fence_before();
-        ptx::mbar_arrive(&S.acc_empty);
+        ptx::mbar_arrive(&S.acc_empty[par]);
       }
       ptx::fence_proxy_async_smem();
       ptx::mbar_arrive(&S.h_full);
@@ -576,7 +615,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           uint32_t o[TPS][16];
 #pragma unroll
           for (int tl = 0; tl < TPS; ++tl)
-            if (tl < nt) ptx::tmem_ld16(tmem + lane_base + 128 + (db * TPS + tl) * 64, o[tl]);
+            if (tl < nt) ptx::tmem_ld16(tmem + lane_base + 256 + (db * TPS + tl) * 64, o[tl]);
           ptx::tmem_ld_wait();
           ptx::tc_fence_before();
           ptx::mbar_arrive(&S.d_empty[db]);
@@ -604,7 +643,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         }
         for (int tl = 0; tl < nt; ++tl) {
           const int ht = ds * TPS + tl;
-          const uint32_t d_down = tmem + lane_base + 128 + (db * TPS + tl) * 64;
+          const uint32_t d_down = tmem + lane_base + 256 + (db * TPS + tl) * 64;
           float* ycol = P.y32 + (size_t)ht * 128 + row;
           const float sd = kFp8 ? S.e_sd[par][ht] : 1.f;
 #pragma unroll
@@ -682,7 +721,6 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           const int kc = lane + 32 * i;
           if (kc < KC) { S.p_sg[par][kc] = vg[i] * pow2i(-eg); S.p_su[par][kc] = vu[i] * pow2i(-eu); }
         }
-        if (lane == 0) { S.pscale_inv[par][0] = pow2i(eg); S.pscale_inv[par][1] = pow2i(eu); }
       }
       __syncwarp();
 
