@@ -56,9 +56,9 @@ DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 
 # DRAM (read + write) bytes per algorithmic byte of the dominant kernel, from the committed ncu
 # capture of a smaller case of the same kernel (profiles/grouped_ffn_tc_fp8_E64_g16.md:
-# 2.443169 GB + 3.97 MB against 2.422802 GB); traffic grows in proportion to the experts
+# 2.458471 GB + 4.67 MB against 2.422802 GB); traffic grows in proportion to the experts
 # streamed, so the full-size launch is scaled by the same ratio.  Absent = not captured.
-NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.443169e9 + 3.97184e6) / 2.422801920e9}
+NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.458471e9 + 4.670208e6) / 2.422801920e9}
 
 ROUTING = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
            "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing}
