@@ -38,6 +38,8 @@ struct Tables {
   float* slot_w;       // [A]   its routing weight
   int32_t* n_active;   // [1]
   float* tok_scale;    // [gamma] power of two bringing the token's max |x| into [64,128)
+  uint8_t* xq;         // [gamma, 2, xq_stride] e4m3 hi / lo terms of x * tok_scale (MXFP4 tensor-core path), or null
+  int32_t xq_stride;   // bytes per row: H, plus a 128-byte tail block when H % 128 != 0
   Unit* units;         // [max_units]
   int32_t* n_units;    // [1]
   int32_t* task_counter; // [1] dynamic task scheduler of the tensor-core FFN, zeroed per call
@@ -62,6 +64,22 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
+}
+
+// Split 4 floats into e4m3 hi and lo (= (v - hi) * 16) codes, 4 bytes each.
+__device__ __forceinline__ void split4_e4m3(const float (&v)[4], uint32_t& hi, uint32_t& lo) {
+  hi = 0; lo = 0;
+#pragma unroll
+  for (int p = 0; p < 2; ++p) {
+    float a = v[2 * p], b = v[2 * p + 1];
+    __nv_fp8x2_storage_t hc = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
+    __half2_raw hr = __nv_cvt_fp8x2_to_halfraw2(hc, __NV_E4M3);
+    float2 hf = __half22float2(*reinterpret_cast<__half2*>(&hr));
+    __nv_fp8x2_storage_t lc = __nv_cvt_float2_to_fp8x2(make_float2((a - hf.x) * 16.f, (b - hf.y) * 16.f),
+                                                       __NV_SATFINITE, __NV_E4M3);
+    hi |= (uint32_t)hc << (16 * p);
+    lo |= (uint32_t)lc << (16 * p);
+  }
 }
 
 // e8m0 scale byte -> float 2^(b-127)  (b = 0 is the subnormal 2^-127)

@@ -111,22 +111,6 @@ __device__ __forceinline__ int safe_exponent(float a) {
   return e < -100 ? -100 : (e > 100 ? 100 : e);
 }
 
-// Split 4 floats into e4m3 hi and lo (= (v - hi) * 16) codes, 4 bytes each.
-__device__ __forceinline__ void split4_e4m3(const float (&v)[4], uint32_t& hi, uint32_t& lo) {
-  hi = 0; lo = 0;
-#pragma unroll
-  for (int p = 0; p < 2; ++p) {
-    float a = v[2 * p], b = v[2 * p + 1];
-    __nv_fp8x2_storage_t hc = __nv_cvt_float2_to_fp8x2(make_float2(a, b), __NV_SATFINITE, __NV_E4M3);
-    __half2_raw hr = __nv_cvt_fp8x2_to_halfraw2(hc, __NV_E4M3);
-    float2 hf = __half22float2(*reinterpret_cast<__half2*>(&hr));
-    __nv_fp8x2_storage_t lc = __nv_cvt_float2_to_fp8x2(make_float2((a - hf.x) * 16.f, (b - hf.y) * 16.f),
-                                                       __NV_SATFINITE, __NV_E4M3);
-    hi |= (uint32_t)hc << (16 * p);
-    lo |= (uint32_t)lc << (16 * p);
-  }
-}
-
 // byte offset of 16-byte chunk c of row r in a [rows x 128 B] tile with the 128-byte swizzle
 __device__ __forceinline__ uint32_t sw128(int r, int c) { return (uint32_t)r * 128u + (uint32_t)((c ^ (r & 7)) << 4); }
 

@@ -5,13 +5,22 @@
 //     which expands every 8 packed bytes into a 16-byte container -- the shared-memory layout
 //     tcgen05.mma kind::mxf8f6f4 reads; a 128-row x 128-element tile is 8 KB in HBM and 16 KB
 //     in shared memory;
-//   * the e8m0 block scales are applied by the tensor core (block_scale): the producers copy
-//     the four scale bytes of each row of a K chunk into the 512-byte scale-factor layout
-//     (byte (r % 32) * 16 + (r / 32) * 4 + kblock), the MMA thread moves it to TMEM with
-//     tcgen05.cp, and every K = 32 MMA selects its byte with the scale-factor id of the
-//     instruction descriptor.  The activation side uses unit scales;
+//   * the e8m0 block scales are applied by the tensor core (block_scale); every K = 32 MMA
+//     selects its scale byte with the scale-factor id of the instruction descriptor.  The scale
+//     factors of a 128-row x 128-element tile are four 32-bit TMEM columns (lane r % 32 of
+//     every lane quarter, column r / 32, byte = K block).  For the gate and up tiles the
+//     The producer warps write them straight into TMEM (tcgen05.st, each warp its own lane
+//     quarter) from scale bytes staged in shared memory once per task (gate/up: one contiguous
+//     block per matrix, copied asynchronously; W_down: a gather of one word per row).  The
+//     activation side uses unit scales, placed once by tcgen05.cp;
+//   * one activation tile and one set of scale-factor columns per weight-ring stage, so the
+//     stage's w_empty barrier (tcgen05.commit) releases all of them: the MMA threads issue
+//     four MMAs and one commit per gate/up stage, nothing else;
 //   * because the scales ride with the weights, the activation operand (two e4m3 terms of
-//     x * 2^p_t) is the same for gate and up;
+//     x * 2^p_t) is the same for gate and up and for every expert: the routing kernels write it
+//     once per token to a [gamma, 2, H] byte array, and the TMA thread loads the two rows of each
+//     of the unit's tokens straight into the swizzled operand tile of the stage (2-D tiled
+//     loads completing on the stage's w_full barrier);
 //   * H and I need only be multiples of 64: the K axis is addressed in half chunks of 64
 //     elements (tensor-map stride 32 bytes), so a ragged tail chunk re-reads the previous half
 //     chunk, whose activations are zeroed; rows past the end of a matrix are zero-filled by TMA
@@ -36,26 +45,29 @@ using tc::warp_wait;
 using tc::group_sync;
 using tc::safe_exponent;
 using tc::pow2i;
-using tc::split4_e4m3;
 
 constexpr int kThreads = 352;  // 11 warps: TMA, MMA issuer 0, 4 epilogue, 4 producers, MMA issuer 1
-constexpr int kStages = 4;   // weight ring: a 32 KB stage holds 16 KB of packed weights
-constexpr int kBSlots = 3;
-constexpr int kBSlotBytes = 8 * 1024 + 1024;  // [64 x 128 B] activation tile | gate scale atom | up scale atom
-constexpr int kDsfSlots = 4;                  // down-phase scale-factor ring (two 512-byte atoms per slot)
-constexpr int kMC = 32;                       // tokens per unit (hi/lo -> N <= 64)
-constexpr int kHTileBytes = 8 * 1024;
+constexpr int kStages = 5;   // weight ring: a 32 KB stage holds 16 KB of packed weights
+constexpr int kMC = 16;                       // tokens per unit (hi/lo -> N <= 32)
+constexpr int kBTileBytes = 4 * 1024;         // [32 x 128 B] activation tile, one per weight-ring stage
+constexpr int kHTileBytes = 4 * 1024;
 constexpr int kTmemCols = 512;
-// TMEM columns: G 0 | P 64 | O 128.. (2 stages x 2 tiles x 64) | scale factors from 384
-constexpr int kColSfGate = 384;   // 4 slots x 4 columns
-constexpr int kColSfUp = 400;     // 4 slots x 4 columns
-constexpr int kColSfDown = 416;   // 4 slots x 2 tiles x 4 columns
-constexpr int kColSfB = 448;      // unit scales of the activation operand (4 columns per MMA issuer)
-constexpr int kSfRing = 4;
-// staged gate / up scale blocks of a task's 128-row slice: [task parity][gate, up][128 rows x K/32 bytes]
-constexpr int kScStageBytes = 11776;  // >= 128 * (H / 32) bytes, H <= 2944
-constexpr int kTileBytes = kStages * kStageBytes + kBSlots * kBSlotBytes + kHTileBytes + kDsfSlots * 1024 + 512 + 4 * kScStageBytes;
-constexpr int kCtlBytes = 8 * 1024;
+// TMEM columns: (G 32 | P 32) x 2 task parities | O 128.. (kDBuf stages x 2 tiles x 32) | scale factors from 384.
+// Every weight-ring stage has its own activation tile and scale-factor columns, so one barrier
+// (w_empty of the stage) releases all of them.
+constexpr int kColD = 128;
+constexpr int kDBuf = 4;          // down-phase accumulator ring (stages)
+constexpr int kColSfGate = 384;                        // kStages slots x 4 columns
+constexpr int kColSfUp = kColSfGate + 4 * kStages;     // kStages slots x 4 columns
+constexpr int kColSfDown = kColSfUp + 4 * kStages;     // kStages slots x 2 tiles x 4 columns
+constexpr int kColSfB = kColSfDown + 8 * kStages;      // unit scales of the activation operand (4 columns per MMA issuer)
+static_assert(kColSfB + 8 <= kTmemCols, "TMEM budget");
+// staged scale bytes of a task: [gate, up][128 rows x K/32 bytes] of its 128-row slice, and one
+// 32-bit word (the four K blocks of the slice) per W_down row
+constexpr int kScStageBytes = 11776;  // >= 128 * (H / 32) bytes and >= 4 * 128 * ceil(H / 128), H <= 2944
+constexpr int kDownWords = kScStageBytes / 4 / 128;  // 128-row tiles of W_down whose row words fit
+constexpr int kTileBytes = kStages * kStageBytes + kStages * kBTileBytes + kHTileBytes + 512 + 3 * kScStageBytes;
+constexpr int kCtlBytes = 2 * 1024;
 constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
 
 struct Params {
@@ -78,22 +90,19 @@ struct Params {
 
 struct Smem {
   uint64_t w_full[kStages], w_empty[kStages];
-  uint64_t b_full[kBSlots], b_empty[kBSlots];
-  uint64_t dsf_full[kDsfSlots], dsf_empty[kDsfSlots];
-  uint64_t acc_full, acc_empty, h_full, h_empty;
-  uint64_t d_full[2], d_empty[2];
+  uint64_t aux_full[kStages];  // activation tile + gate/up scale factors (gate/up stage) or W_down scale atoms (down stage)
+  uint64_t acc_full[2], acc_empty[2], h_full, h_empty;
+  uint64_t d_full[kDBuf], d_empty[kDBuf];
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar, pr_bar;
   volatile int32_t tq_task[kTaskQ];
   uint32_t tmem_base;
   volatile int abort_flag;
-  int32_t p_tok[2][64];
-  float p_tscale[2][64];
-  int32_t e_tok[2][64];
-  float e_w[2][64];
-  float e_inv[2][64];
-  float e_f[64];
-  uint32_t e_amax[4][32];
+  int32_t e_tok[2][kMC];
+  float e_w[2][kMC];
+  float e_inv[2][kMC];
+  float e_f[kMC];
+  uint32_t e_amax[4][kMC];
 };
 
 // Half-chunk coordinate (units of 64 elements) of the 128-element K chunk that starts at
@@ -119,6 +128,15 @@ __device__ __forceinline__ void sf_copy(uint32_t tmem_col_addr, uint32_t smem_ad
   d |= (uint64_t)1 << 46;   // descriptor version
   asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(tmem_col_addr), "l"(d) : "memory");
 }
+
+// Four 32-bit columns of this warp's TMEM lane quarter from registers: lane l writes TMEM lane
+// (quarter base + l).  Used for the scale factors of the gate/up weight tiles, which have the
+// same layout as sf_copy produces when every warp writes its own quarter.
+__device__ __forceinline__ void tmem_st4(uint32_t taddr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // D (+)= A(e2m1, scaled per row and 32-element K block) * B(e4m3, unit scales)
 __device__ __forceinline__ void mma_mx(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate,
@@ -162,17 +180,19 @@ __global__ void __launch_bounds__(kThreads, 1)
 grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_constant__ CUtensorMap tm_up,
                       const __grid_constant__ CUtensorMap tm_down, const __grid_constant__ CUtensorMap tm_sh_gate,
                       const __grid_constant__ CUtensorMap tm_sh_up, const __grid_constant__ CUtensorMap tm_sh_down,
-                      const Params P) {
+                      const __grid_constant__ CUtensorMap tm_xq, const Params P) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* w_ring = base;
-  uint8_t* b_ring = w_ring + kStages * kStageBytes;
-  uint8_t* h_tile = b_ring + kBSlots * kBSlotBytes;  // 27 KB after a 1 KB-aligned start: still 1 KB aligned
-  uint8_t* dsf_ring = h_tile + kHTileBytes;
-  uint8_t* sfb_unit = dsf_ring + kDsfSlots * 1024;
-  uint8_t* sc_stage = sfb_unit + 512;  // 16-byte aligned
-  static_assert((kBSlots * kBSlotBytes) % 1024 == 0, "h tile alignment");
+  uint8_t* b_tiles = w_ring + kStages * kStageBytes;
+  uint8_t* h_tile = b_tiles + kStages * kBTileBytes;
+  uint8_t* sfb_unit = h_tile + kHTileBytes;
+  uint8_t* sc_stage = sfb_unit + 512;  // 16-byte aligned: gate block | up block | W_down row words
+  uint32_t* dsc_stage = reinterpret_cast<uint32_t*>(sc_stage + 2 * kScStageBytes);
+  static_assert(kBTileBytes % 1024 == 0 && kHTileBytes % 1024 == 0, "tile alignment");
+  static_assert(kDownWords * 128 * 4 <= kScStageBytes, "W_down scale words");
   static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
   Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -185,12 +205,13 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 
   if (tid == 0) {
     // barriers completed by tcgen05.commit count 2: one arrival per MMA issuer
-    for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
-    for (int i = 0; i < kBSlots; ++i) { ptx::mbar_init(&S.b_full[i], 128); ptx::mbar_init(&S.b_empty[i], 2); }
-    for (int i = 0; i < kDsfSlots; ++i) { ptx::mbar_init(&S.dsf_full[i], 128); ptx::mbar_init(&S.dsf_empty[i], 2); }
-    ptx::mbar_init(&S.acc_full, 2); ptx::mbar_init(&S.acc_empty, 128);
-    ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 2);
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 128); }
+    for (int i = 0; i < kStages; ++i) {
+      ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); ptx::mbar_init(&S.aux_full[i], 4);
+    }
+    // barriers completed by a 4-warp role group count 4: one elected arrival per warp
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.acc_full[i], 2); ptx::mbar_init(&S.acc_empty[i], 4); }
+    ptx::mbar_init(&S.h_full, 4); ptx::mbar_init(&S.h_empty, 2);
+    for (int i = 0; i < kDBuf; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 4); }
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     ptx::mbar_init(&S.pr_bar, 128);
@@ -213,10 +234,15 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   const int n_ids = n_units * ((n_slices + 1) & ~1);
   volatile int* abortp = &S.abort_flag;
 
+  // Phase order of the weight stream, the MMAs and the producers (GU = gate/up phase, D = down
+  // phase of the CTA's t-th task): GU(0), GU(1), D(0), GU(2), D(1), ...  The SwiGLU step of a
+  // task overlaps the gate/up phase of the next one.  `it` counts ring stages in that order in
+  // every role.
+
   if (warp == 0) {
     // ===================================================== TMA producer + scheduler (one lane)
     if (lane == 0) {
-      ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
+      ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down); ptx::prefetch_tmap(&tm_xq);
       uint32_t it = 0, q = 0;
       bool ok = true;
       auto fetch_publish = [&](TaskDesc& td) -> int {
@@ -235,27 +261,37 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         ++q;
         return id;
       };
-      TaskDesc td, td_next;
-      int id = fetch_publish(td);
-      while (ok && id >= 0) {
-        const int id_next = fetch_publish(td_next);
-        if (!ok) break;
-        const Unit u = P.units[td.unit];
-        const int slice = td.slice;
+      auto load_gu = [&](const TaskDesc& t) {
+        const Unit u = P.units[t.unit];
         const CUtensorMap* mg = u.shared ? &tm_sh_gate : &tm_gate;
         const CUtensorMap* mu = u.shared ? &tm_sh_up : &tm_up;
-        const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
+        const int m = u.m;
+        const int tok0 = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma)) : -1;  // shared experts: consecutive tokens
+        const int32_t* toks = P.slot_token + (u.shared ? 0 : u.slot0);
         for (int kc = 0; kc < KC && ok; ++kc, ++it) {
           const int s = it % kStages;
           ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
           if (!ok) break;
           uint8_t* dst = w_ring + s * kStageBytes;
           const int cc = half_chunk_coord(kc * 128, H);
-          ptx::mbar_arrive_expect_tx(&S.w_full[s], 2 * 8192);  // the transaction count is in packed (HBM) bytes
-          tma_load_4d(dst, mg, &S.w_full[s], 0, cc, slice * 128, u.expert, ptx::kPolicyEvictFirst);
-          tma_load_4d(dst + 16384, mu, &S.w_full[s], 0, cc, slice * 128, u.expert, ptx::kPolicyEvictFirst);
+          // the transaction count is in packed (HBM) bytes for the weights; 2 x 128 bytes per token
+          ptx::mbar_arrive_expect_tx(&S.w_full[s], 2 * 8192 + 256 * m);
+          tma_load_4d(dst, mg, &S.w_full[s], 0, cc, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
+          tma_load_4d(dst + 16384, mu, &S.w_full[s], 0, cc, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
+          // activation operand: rows 2r (hi) and 2r + 1 (lo) of the stage's tile; a ragged last
+          // chunk takes the tail block (zeros under the re-read half of the weight chunk)
+          const int xcol = (kc * 128 + 128 <= H) ? kc * 128 : H;
+          uint8_t* bt = b_tiles + s * kBTileBytes;
+          for (int r = 0; r < m; ++r) {
+            const int tok = tok0 >= 0 ? tok0 + r : __ldg(toks + r);
+            ptx::tma_load_2d(bt + r * 256, &tm_xq, &S.w_full[s], xcol, 2 * tok, ptx::kPolicyEvictNormal);
+          }
         }
-        const int cd = half_chunk_coord(slice * 128, I);
+      };
+      auto load_down = [&](const TaskDesc& t) {
+        const Unit u = P.units[t.unit];
+        const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
+        const int cd = half_chunk_coord(t.slice * 128, I);
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
           const int s = it % kStages;
           ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
@@ -266,8 +302,26 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           tma_load_4d(dst, md, &S.w_full[s], 0, cd, (2 * ds) * 128, u.expert, ptx::kPolicyEvictFirst);
           if (nt == 2) tma_load_4d(dst + 16384, md, &S.w_full[s], 0, cd, (2 * ds + 1) * 128, u.expert, ptx::kPolicyEvictFirst);
         }
-        id = id_next;
-        td = td_next;
+      };
+      // task t + 2 is published between the loads of GU(t + 1) and D(t)
+      TaskDesc td, td_next, td_nn;
+      int id = fetch_publish(td);
+      int id_next = -1;
+      if (ok && id >= 0) {
+        id_next = fetch_publish(td_next);
+        if (ok) load_gu(td);
+      }
+      while (ok && id >= 0) {
+        int id_nn = -1;
+        if (id_next >= 0) {
+          load_gu(td_next);
+          if (!ok) break;
+          id_nn = fetch_publish(td_nn);
+          if (!ok) break;
+        }
+        load_down(td);
+        id = id_next; td = td_next;
+        id_next = id_nn; td_next = td_nn;
       }
     }
   } else if (warp == 1 || warp == 10) {
@@ -275,9 +329,10 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     // and the even W_down tiles, issuer 1 the up chain and the odd tiles
     const int issuer = warp == 1 ? 0 : 1;
     if (lane == 0) {
-      uint32_t it = 0, bit = 0, tcount = 0, dsc = 0, q = 0;
+      uint32_t it = 0, tcount = 0, dsc = 0, q = 0;
       bool ok = true;
       const uint32_t w_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(w_ring));
+      const uint32_t b_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(b_tiles));
       const uint32_t h_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(h_tile));
 #ifdef MOEV_TC_STATS
       unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
@@ -285,84 +340,99 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #endif
       const uint32_t sfb_col = tmem + kColSfB + 4 * issuer;
       sf_copy(sfb_col, ptx::smem_u32(sfb_unit));  // unit activation scales, once per issuer
-      for (;; ++tcount) {
-        const int id = next_task(S, q, abortp, P.status, false);
-        if (id < 0) break;
+      auto n_of = [&](int id) -> uint32_t {
         const TaskDesc td = decode_task(id, n_units, n_slices);
-        const Unit u = P.units[td.unit];
-        const uint32_t N = (uint32_t)((2 * u.m + 15) & ~15);
-        const uint32_t d_gate = tmem, d_up = tmem + 64;
+        return (uint32_t)((2 * P.units[td.unit].m + 15) & ~15);
+      };
+      auto gate_up = [&](uint32_t g, uint32_t N) {
+        const uint32_t pb = g & 1u;
+        const uint32_t dacc = tmem + pb * 64 + (issuer ? 32 : 0);
         { MOEV_STAT_BEGIN();
-          ok = ptx::bounded_wait(&S.acc_empty, (tcount & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          ok = ptx::bounded_wait(&S.acc_empty[pb], ((g >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
           MOEV_STAT_END(3); }
-        if (!ok) break;
+        if (!ok) return;
         ptx::tc_fence_after();
-        for (int kc = 0; kc < KC && ok; ++kc, ++it, ++bit) {
-          const int s = it % kStages, sb = bit % kBSlots, sf = bit % kSfRing;
+        for (int kc = 0; kc < KC && ok; ++kc, ++it) {
+          const int s = it % kStages;
           { MOEV_STAT_BEGIN();
             ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             MOEV_STAT_END(1); }
           { MOEV_STAT_BEGIN();
-            ok = ok && ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            ok = ok && ptx::bounded_wait(&S.aux_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             MOEV_STAT_END(2); }
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t bslot = ptx::smem_u32(b_ring + sb * kBSlotBytes);
-          const uint32_t sfa_col = tmem + (issuer ? kColSfUp : kColSfGate) + 4 * sf;
-          sf_copy(sfa_col, bslot + 8192 + 512 * issuer);
+          { MOEV_STAT_BEGIN();
+          const uint32_t sfa_col = tmem + (issuer ? kColSfUp : kColSfGate) + 4 * s;
           const uint32_t wa = w_lo0 + s * (kStageBytes >> 4) + 1024 * issuer;
-          const uint32_t ba = ptx::desc_lo_sw128(bslot);
-          const uint32_t dacc = issuer ? d_up : d_gate;
+          const uint32_t ba = b_lo0 + s * (kBTileBytes >> 4);
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             mma_mx(dacc, wa + 2 * j, ba + 2 * j, idesc_mx(N, j), (kc | j) ? 1u : 0u, sfa_col, sfb_col);
+          MOEV_STAT_END(8); }
+          { MOEV_STAT_BEGIN();
           ptx::mma_commit(&S.w_empty[s]);
-          ptx::mma_commit(&S.b_empty[sb]);
+          MOEV_STAT_END(9); }
         }
-        if (!ok) break;
-        ptx::mma_commit(&S.acc_full);
+        if (ok) ptx::mma_commit(&S.acc_full[pb]);
+      };
+      int id = next_task(S, q, abortp, P.status, false);
+      uint32_t N = 0;
+      if (id >= 0) { N = n_of(id); gate_up(0, N); }
+      for (; ok && id >= 0; ++tcount) {
+        const int id_next = next_task(S, q, abortp, P.status, false);
+        if (id_next == -2) break;
+        uint32_t N_next = 0;
+        if (id_next >= 0) {
+          N_next = n_of(id_next);
+          gate_up(tcount + 1, N_next);
+          if (!ok) break;
+        }
         { MOEV_STAT_BEGIN();
           ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
           MOEV_STAT_END(4); }
         if (!ok) break;
         ptx::tc_fence_after();
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc, ++it) {
-          const int db = dsc & 1, s = it % kStages, sfs = dsc % kDsfSlots;
+          const int db = dsc % kDBuf, s = it % kStages;
           { MOEV_STAT_BEGIN();
             ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             MOEV_STAT_END(5); }
           { MOEV_STAT_BEGIN();
-            ok = ok && ptx::bounded_wait(&S.dsf_full[sfs], (dsc / kDsfSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            ok = ok && ptx::bounded_wait(&S.aux_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             MOEV_STAT_END(12); }
           { MOEV_STAT_BEGIN();
-            ok = ok && ptx::bounded_wait(&S.d_empty[db], ((dsc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            ok = ok && ptx::bounded_wait(&S.d_empty[db], ((dsc / kDBuf) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             MOEV_STAT_END(6); }
           if (!ok) break;
           ptx::tc_fence_after();
+          { MOEV_STAT_BEGIN();
           const uint32_t wa = w_lo0 + s * (kStageBytes >> 4);
           const int nt = (2 * ds + 1 < HT) ? 2 : 1;
           const int tl = issuer;
           if (tl < nt) {
-            const uint32_t sfcol = tmem + kColSfDown + (sfs * 2 + tl) * 4;
-            sf_copy(sfcol, ptx::smem_u32(dsf_ring + sfs * 1024 + tl * 512));
-            const uint32_t d_down = tmem + 128 + (db * 2 + tl) * 64;
+            const uint32_t sfcol = tmem + kColSfDown + (s * 2 + tl) * 4;
+            const uint32_t d_down = tmem + kColD + (db * 2 + tl) * 32;
 #pragma unroll
             for (int j = 0; j < 4; ++j)
               mma_mx(d_down, wa + tl * 1024 + 2 * j, h_lo0 + 2 * j, idesc_mx(N, j), j ? 1u : 0u, sfcol, sfb_col);
           }
+          MOEV_STAT_END(10); }
+          { MOEV_STAT_BEGIN();
           ptx::mma_commit(&S.d_full[db]);
           ptx::mma_commit(&S.w_empty[s]);
-          ptx::mma_commit(&S.dsf_empty[sfs]);
+          MOEV_STAT_END(11); }
         }
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
+        id = id_next;
+        N = N_next;
       }
 #ifdef MOEV_TC_STATS
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
       if (P.stats && issuer == 0)
-        for (int i = 0; i < 16; ++i)
-          if (i < 8 || i >= 12) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
+        for (int i = 0; i < 13; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
 #endif
     }
   } else if (warp < 6) {
@@ -390,19 +460,21 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         S.e_inv[par][r] = 1.f / P.tok_scale[tok];
       }
       __syncwarp();
-      ok = warp_wait(&S.acc_full, tcount & 1, abortp, P.status);
+      ok = warp_wait(&S.acc_full[par], (tcount >> 1) & 1, abortp, P.status);
       if (!ok) break;
       ptx::tc_fence_after();
+      // h tile must be free: all down MMAs of the previous task have completed
       ok = warp_wait(&S.h_empty, (tcount & 1) ^ 1, abortp, P.status);
       if (!ok) break;
 
-      float hv[32];
+      float hv[kMC];
+      const uint32_t gp = tmem + lane_base + par * 64;
 #pragma unroll
-      for (int c0 = 0; c0 < 64; c0 += 16) {
+      for (int c0 = 0; c0 < 32; c0 += 16) {
         if (c0 < 2 * m) {
           uint32_t g[16], p[16];
-          ptx::tmem_ld16(tmem + lane_base + c0, g);
-          ptx::tmem_ld16(tmem + lane_base + 64 + c0, p);
+          ptx::tmem_ld16(gp + c0, g);
+          ptx::tmem_ld16(gp + 32 + c0, p);
           ptx::tmem_ld_wait();
 #pragma unroll
           for (int r = 0; r < 8; ++r) {
@@ -418,14 +490,15 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         }
       }
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&S.acc_empty);
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&S.acc_empty[par]);
       // rows of the slice past the end of I carry zero weights, hence h = 0 there already.
       // K position of this row's h in the down operand: a ragged last slice is loaded one half
       // chunk early, so its 64 valid rows sit at K 64..127 and K 0..63 must be zero.
       const bool ragged = slice * 128 + 128 > I;
       const int kpos = ragged ? ((row + 64) & 127) : row;
 #pragma unroll
-      for (int r = 0; r < 32; ++r) {
+      for (int r = 0; r < kMC; ++r) {
         if (r < m) {
           uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hv[r])));
           if (lane == 0) S.e_amax[warp - 2][r] = mx;
@@ -433,7 +506,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       }
       if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
 #pragma unroll
-      for (int r = 0; r < 32; ++r) {
+      for (int r = 0; r < kMC; ++r) {
         if (r < m) {
           uint32_t mx = max(max(S.e_amax[0][r], S.e_amax[1][r]), max(S.e_amax[2][r], S.e_amax[3][r]));
           const int er = safe_exponent(__uint_as_float(mx));
@@ -447,83 +520,62 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           if (lane == (r & 31)) S.e_f[r] = S.e_w[par][r] * pow2i(er - 6);
         }
       }
-      __syncwarp();
       ptx::fence_proxy_async_smem();
-      ptx::mbar_arrive(&S.h_full);
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&S.h_full);
 
       const int ncols = 2 * m;
       for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc) {
-        const int db = dsc & 1;
-        ok = warp_wait(&S.d_full[db], (dsc >> 1) & 1, abortp, P.status);
+        const int db = dsc % kDBuf;
+        ok = warp_wait(&S.d_full[db], (dsc / kDBuf) & 1, abortp, P.status);
         if (!ok) break;
         ptx::tc_fence_after();
         const int nt = (2 * ds + 1 < HT) ? 2 : 1;
-        if (ncols <= 16) {
-          uint32_t o[2][16];
+        // fetch the accumulators of both tiles of the stage, release them, then do the reductions
+        uint32_t o[2][32];
 #pragma unroll
-          for (int tl = 0; tl < 2; ++tl)
-            if (tl < nt) ptx::tmem_ld16(tmem + lane_base + 128 + (db * 2 + tl) * 64, o[tl]);
-          ptx::tmem_ld_wait();
-          ptx::tc_fence_before();
-          ptx::mbar_arrive(&S.d_empty[db]);
-#pragma unroll
-          for (int tl = 0; tl < 2; ++tl) {
-            const int hrow = (ds * 2 + tl) * 128 + row;
-            if (tl < nt && hrow < H) {
-              float* ycol = P.y32 + hrow;
-#pragma unroll
-              for (int r = 0; r < 8; ++r)
-                if (r < m) {
-                  float val = (__uint_as_float(o[tl][2 * r]) + __uint_as_float(o[tl][2 * r + 1]) * 0.0625f) * S.e_f[r];
-                  ptx::red_add_f32(ycol + (size_t)S.e_tok[par][r] * H, val);
-                }
-            }
+        for (int tl = 0; tl < 2; ++tl)
+          if (tl < nt) {
+            ptx::tmem_ld16(tmem + lane_base + kColD + (db * 2 + tl) * 32, *reinterpret_cast<uint32_t(*)[16]>(&o[tl][0]));
+            if (ncols > 16)
+              ptx::tmem_ld16(tmem + lane_base + kColD + (db * 2 + tl) * 32 + 16, *reinterpret_cast<uint32_t(*)[16]>(&o[tl][16]));
           }
-          continue;
-        }
-        for (int tl = 0; tl < nt; ++tl) {
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&S.d_empty[db]);
+#pragma unroll
+        for (int tl = 0; tl < 2; ++tl) {
           const int hrow = (ds * 2 + tl) * 128 + row;
-          const uint32_t d_down = tmem + lane_base + 128 + (db * 2 + tl) * 64;
-          float* ycol = P.y32 + hrow;
+          if (tl < nt && hrow < H) {
+            float* ycol = P.y32 + hrow;
 #pragma unroll
-          for (int c0 = 0; c0 < 64; c0 += 16) {
-            if (c0 < ncols) {
-              uint32_t o[16];
-              ptx::tmem_ld16(d_down + c0, o);
-              ptx::tmem_ld_wait();
-              if (tl == nt - 1 && c0 + 16 >= ncols) {
-                ptx::tc_fence_before();
-                ptx::mbar_arrive(&S.d_empty[db]);
+            for (int r = 0; r < kMC; ++r)
+              if (r < m) {
+                float val = (__uint_as_float(o[tl][2 * r]) + __uint_as_float(o[tl][2 * r + 1]) * 0.0625f) * S.e_f[r];
+                ptx::red_add_f32(ycol + (size_t)S.e_tok[par][r] * H, val);
               }
-              if (hrow < H) {
-#pragma unroll
-                for (int r = 0; r < 8; ++r) {
-                  const int tr = c0 / 2 + r;
-                  if (tr < m) {
-                    float val = (__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f) * S.e_f[tr];
-                    ptx::red_add_f32(ycol + (size_t)S.e_tok[par][tr] * H, val);
-                  }
-                }
-              }
-            }
           }
         }
       }
       if (!ok) break;
     }
   } else {
-    // ===================================================== producers (4 warps): activation tiles and scale atoms
-    const int pw = warp - 6;
-    const int pt = tid - 192;  // 0..127: the weight-tile row whose scale bytes this thread moves
-    uint32_t bit = 0, tcount = 0, dsc = 0, q = 0, gph = 0;
+    // ===================================================== producers (4 warps): activation tiles and scale factors
+    const int pt = tid - 192;  // 0..127: the W_down tile row whose scale bytes this thread moves
+    uint32_t it = 0, q = 0, gph = 0;
     bool ok = true;
-    const uint16_t* xb = static_cast<const uint16_t*>(P.x);
-    const uint32_t sf_off = (uint32_t)(pt & 31) * 16u + (uint32_t)(pt >> 5) * 4u;  // this row's word in a scale atom
+    const uint32_t tm_quarter = tmem + ((uint32_t)((warp & 3) * 32) << 16);          // this warp's TMEM lane quarter
+    auto wait_slot = [&]() -> bool {  // every buffer of ring stage `it` is free once the stage's previous MMAs are done
+      return warp_wait(&S.w_empty[it % kStages], ((it / kStages) & 1) ^ 1, abortp, P.status);
+    };
     // Gate / up scale bytes of a task's slice are one contiguous block per matrix; they are
     // staged in shared memory with 16-byte asynchronous copies (one latency per task, no
-    // divergent loads in the chunk loop).  The copy for the next task is issued before this
-    // task's down-phase work.
-    auto stage_scales = [&](int id, int par) {
+    // divergent loads in the chunk loop).  One buffer: the copy for the next gate/up phase is
+    // issued when every producer thread has finished the current one (its last reads of the
+    // buffer), and lands during the down phase in between.
+    auto stage_scales = [&](int id) {
+      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) return;
       const TaskDesc td = decode_task(id, n_units, n_slices);
       const Unit u = P.units[td.unit];
       const uint8_t* sg = u.shared ? P.sh_s_gate : P.s_gate;
@@ -531,140 +583,133 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       const int rows = min(128, I - td.slice * 128);
       const int n16 = rows * kb_gu / 16;  // kb_gu % 2 == 0 and rows % 64 == 0: a whole number of 16-byte pieces
       const size_t off = ((size_t)u.expert * I + (size_t)td.slice * 128) * kb_gu;
-      uint8_t* dg = sc_stage + (par * 2 + 0) * kScStageBytes;
-      uint8_t* du = sc_stage + (par * 2 + 1) * kScStageBytes;
+      uint8_t* dg = sc_stage;
+      uint8_t* du = sc_stage + kScStageBytes;
       for (int i = pt; i < n16; i += 128) {
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(dg + i * 16)), "l"(sg + off + (size_t)i * 16) : "memory");
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_u32(du + i * 16)), "l"(su + off + (size_t)i * 16) : "memory");
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    int id = next_task(S, q, abortp, P.status, true);
-    if (id >= 0) stage_scales(id, 0);
-    for (; id >= 0; ++tcount) {
+    // ---- gate/up phase of the g-th task: per K chunk the scale factors of the gate and up tiles, into TMEM
+    // While it runs, gate_up also gathers the W_down scale words of task id_dn (whose down phase
+    // follows) into shared memory: one row word per K chunk and thread, four chunks in flight
+    // (the number of K chunks equals the number of 128-row tiles of W_down).
+    auto gate_up = [&](int id, int id_dn) {
       const TaskDesc td = decode_task(id, n_units, n_slices);
-      const Unit u = P.units[td.unit];
-      const int slice = td.slice;
-      const int m = u.m;
-      const int par = tcount & 1;
-      for (int r = lane; r < m; r += 32) {
-        int tok = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma) + r) : P.slot_token[u.slot0 + r];
-        S.p_tok[par][r] = tok;
-        S.p_tscale[par][r] = P.tok_scale[tok];
+      const uint8_t* sd = nullptr;
+      int dn_e = 0, kbd = 0;
+      if (id_dn >= 0) {
+        const TaskDesc tdn = decode_task(id_dn, n_units, n_slices);
+        const Unit un = P.units[tdn.unit];
+        sd = un.shared ? P.sh_s_down : P.s_down;
+        dn_e = un.expert;
+        kbd = half_chunk_coord(tdn.slice * 128, I) * 2;
       }
-      __syncwarp();
-      const uint8_t* sd = u.shared ? P.sh_s_down : P.s_down;
+      uint32_t dw0 = 0, dw1 = 0, dw2 = 0, dw3 = 0;
       // this task's staged scales have landed (every thread waits for its own copies, then all meet)
       asm volatile("cp.async.wait_group 0;" ::: "memory");
-      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) break;
-      const uint8_t* stg = sc_stage + (par * 2 + 0) * kScStageBytes;
-      const uint8_t* stu = sc_stage + (par * 2 + 1) * kScStageBytes;
-      const bool row_ok = slice * 128 + pt < I;
+      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) return;
+      const uint8_t* stg = sc_stage;
+      const uint8_t* stu = sc_stage + kScStageBytes;
+      const int rows = min(128, I - td.slice * 128);
 
-      // ---- gate/up phase: per K chunk the activation tile (hi/lo of x * 2^p_t) and the two scale atoms
-      constexpr int kMaxPass = kMC / 4;
-      const int passes = (m - pw + 3) >> 2;
-      const uint16_t* xrow[kMaxPass];
-#pragma unroll
-      for (int i = 0; i < kMaxPass; ++i) xrow[i] = (i < passes) ? xb + (size_t)S.p_tok[par][pw + 4 * i] * H : nullptr;
-      auto load_x = [&](int i, int kc) -> uint2 {
-        // this lane's 4 elements of the chunk: K positions 4 lane .. 4 lane + 3 hold elements e0 ..
-        const int cc = half_chunk_coord(kc * 128, H);
-        const int e0 = cc * 64 + lane * 4;
-        const bool valid = e0 >= kc * 128 && e0 < H;  // a ragged tail chunk re-reads 64 elements that must be zero
-        return valid ? __ldg(reinterpret_cast<const uint2*>(xrow[i] + e0)) : make_uint2(0u, 0u);
-      };
-      // x is fetched three K chunks ahead (a chunk lasts less than one trip to L2)
-      uint2 n0[kMaxPass], n1[kMaxPass], n2[kMaxPass];
-#pragma unroll
-      for (int i = 0; i < kMaxPass; ++i) {
-        n0[i] = n1[i] = n2[i] = make_uint2(0u, 0u);
-        if (i < passes) {
-          n0[i] = load_x(i, 0);
-          if (1 < KC) n1[i] = load_x(i, 1);
-          if (2 < KC) n2[i] = load_x(i, 2);
+      for (int kc = 0; kc < KC && ok; ++kc, ++it) {
+        const int s = it % kStages;
+        if (sd) {
+          if (kc >= 4) dsc_stage[(kc - 4) * 128 + pt] = dw0;
+          dw0 = dw1; dw1 = dw2; dw2 = dw3;
+          dw3 = load_scale4(sd, dn_e, H, kb_dn, kc * 128 + pt, kbd);  // rows >= H: unit scale
         }
-      }
-      for (int kc = 0; kc < KC && ok; ++kc, ++bit) {
-        const int sb = bit % kBSlots;
-        uint2 cur[kMaxPass];
+        // scale bytes of the chunk for the four tile rows lane, lane + 32, .. (one TMEM column
+        // each), from the staged block (2-byte aligned); rows past the matrix get the unit scale
+        uint32_t cg[4], cu[4];
+        const int bo = half_chunk_coord(kc * 128, H) * 2;
 #pragma unroll
-        for (int i = 0; i < kMaxPass; ++i) {
-          cur[i] = n0[i];
-          n0[i] = n1[i];
-          n1[i] = n2[i];
-          if (i < passes && kc + 3 < KC) n2[i] = load_x(i, kc + 3);
-        }
-        // this row's four scale bytes of the chunk, from the staged block (2-byte aligned)
-        uint32_t csg = 0x7F7F7F7Fu, csu = 0x7F7F7F7Fu;
-        if (row_ok) {
-          const int bo = pt * kb_gu + half_chunk_coord(kc * 128, H) * 2;
-          const uint16_t* pg = reinterpret_cast<const uint16_t*>(stg + bo);
-          const uint16_t* pu = reinterpret_cast<const uint16_t*>(stu + bo);
-          csg = (uint32_t)pg[0] | ((uint32_t)pg[1] << 16);
-          csu = (uint32_t)pu[0] | ((uint32_t)pu[1] << 16);
-        }
-        ok = warp_wait(&S.b_empty[sb], ((bit / kBSlots) & 1) ^ 1, abortp, P.status);
-        if (!ok) break;
-        uint8_t* tile = b_ring + sb * kBSlotBytes;
-#pragma unroll
-        for (int i = 0; i < kMaxPass; ++i) {
-          if (i < passes) {
-            const int r = pw + 4 * i;
-            const float ts = S.p_tscale[par][r];
-            float v[4];
-            v[0] = __uint_as_float(cur[i].x << 16) * ts;
-            v[1] = __uint_as_float(cur[i].x & 0xffff0000u) * ts;
-            v[2] = __uint_as_float(cur[i].y << 16) * ts;
-            v[3] = __uint_as_float(cur[i].y & 0xffff0000u) * ts;
-            uint32_t hi, lo;
-            split4_e4m3(v, hi, lo);
-            *reinterpret_cast<uint32_t*>(tile + sw128(2 * r, lane >> 2) + (lane & 3) * 4) = hi;
-            *reinterpret_cast<uint32_t*>(tile + sw128(2 * r + 1, lane >> 2) + (lane & 3) * 4) = lo;
+        for (int i = 0; i < 4; ++i) {
+          const int r = lane + 32 * i;
+          cg[i] = cu[i] = 0x7F7F7F7Fu;
+          if (r < rows) {
+            const uint16_t* pg = reinterpret_cast<const uint16_t*>(stg + r * kb_gu + bo);
+            const uint16_t* pu = reinterpret_cast<const uint16_t*>(stu + r * kb_gu + bo);
+            cg[i] = (uint32_t)pg[0] | ((uint32_t)pg[1] << 16);
+            cu[i] = (uint32_t)pu[0] | ((uint32_t)pu[1] << 16);
           }
         }
-        *reinterpret_cast<uint32_t*>(tile + 8192 + sf_off) = csg;
-        *reinterpret_cast<uint32_t*>(tile + 8192 + 512 + sf_off) = csu;
-        ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(&S.b_full[sb]);
-      }
-      if (!ok) break;
-
-      // ---- the next task is known by now (ids are published one task ahead): start staging its scales
-      const int id_next = next_task(S, q, abortp, P.status, true);
-      if (id_next == -2) { ok = false; break; }
-      if (id_next >= 0) stage_scales(id_next, par ^ 1);
-
-      // ---- down phase: scale atoms of the W_down tiles of every ring stage (gathered: the four
-      // bytes of a row are 2-byte aligned and rows are K/32 bytes apart)
-      const int kbd = half_chunk_coord(slice * 128, I) * 2;
-      uint32_t da[4], db2[4];  // stages ds .. ds + 3 (rotated)
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        da[i] = db2[i] = 0x7F7F7F7Fu;
-        if (i < n_dstage) {
-          da[i] = load_scale4(sd, u.expert, H, kb_dn, (2 * i) * 128 + pt, kbd);
-          db2[i] = load_scale4(sd, u.expert, H, kb_dn, (2 * i + 1) * 128 + pt, kbd);
-        }
-      }
-      for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc) {
-        const int sfs = dsc % kDsfSlots;
-        const uint32_t c0v = da[0], c1v = db2[0];
-#pragma unroll
-        for (int i = 0; i < 3; ++i) { da[i] = da[i + 1]; db2[i] = db2[i + 1]; }
-        if (ds + 4 < n_dstage) {
-          da[3] = load_scale4(sd, u.expert, H, kb_dn, (2 * ds + 8) * 128 + pt, kbd);
-          db2[3] = load_scale4(sd, u.expert, H, kb_dn, (2 * ds + 9) * 128 + pt, kbd);
-        }
-        ok = warp_wait(&S.dsf_empty[sfs], ((dsc / kDsfSlots) & 1) ^ 1, abortp, P.status);
+        ok = wait_slot();
         if (!ok) break;
-        *reinterpret_cast<uint32_t*>(dsf_ring + sfs * 1024 + sf_off) = c0v;
-        *reinterpret_cast<uint32_t*>(dsf_ring + sfs * 1024 + 512 + sf_off) = c1v;
-        ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(&S.dsf_full[sfs]);
+        ptx::tc_fence_after();
+        tmem_st4(tm_quarter + kColSfGate + 4 * s, cg[0], cg[1], cg[2], cg[3]);
+        tmem_st4(tm_quarter + kColSfUp + 4 * s, cu[0], cu[1], cu[2], cu[3]);
+        tmem_st_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&S.aux_full[s]);
       }
-      if (!ok) break;
-      id = id_next;
+      if (sd && ok) {
+        dsc_stage[(KC - 4) * 128 + pt] = dw0; dsc_stage[(KC - 3) * 128 + pt] = dw1;
+        dsc_stage[(KC - 2) * 128 + pt] = dw2; dsc_stage[(KC - 1) * 128 + pt] = dw3;
+      }
+    };
+    // ---- down phase: scale atoms of the W_down tiles of every ring stage (gathered: the four
+    // bytes of a row are 2-byte aligned and rows are K/32 bytes apart)
+    // ---- down phase: scale factors of the W_down tiles of every ring stage.  The four scale bytes
+    // of a row (its K blocks inside the slice) are 2-byte aligned and rows are I/32 bytes apart: a
+    // gather, done during the preceding gate/up phase (above) or, when none precedes, here.
+    auto fetch_down_words = [&](int id) {
+      const TaskDesc td = decode_task(id, n_units, n_slices);
+      const Unit u = P.units[td.unit];
+      const uint8_t* sd = u.shared ? P.sh_s_down : P.s_down;
+      const int kbd = half_chunk_coord(td.slice * 128, I) * 2;
+      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) return;  // all reads of the previous block are over
+      for (int i = 0; i < HT; ++i) dsc_stage[i * 128 + pt] = load_scale4(sd, u.expert, H, kb_dn, i * 128 + pt, kbd);
+    };
+    auto down = [&]() {
+      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) return;  // the task's words are all in place
+      for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
+        const int s = it % kStages;
+        const int nt = (2 * ds + 1 < HT) ? 2 : 1;
+        uint32_t c0[4], c1[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          c0[i] = dsc_stage[(2 * ds) * 128 + lane + 32 * i];
+          c1[i] = nt == 2 ? dsc_stage[(2 * ds + 1) * 128 + lane + 32 * i] : 0x7F7F7F7Fu;
+        }
+        ok = wait_slot();
+        if (!ok) break;
+        ptx::tc_fence_after();
+        tmem_st4(tm_quarter + kColSfDown + (s * 2) * 4, c0[0], c0[1], c0[2], c0[3]);
+        tmem_st4(tm_quarter + kColSfDown + (s * 2 + 1) * 4, c1[0], c1[1], c1[2], c1[3]);
+        tmem_st_wait();
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&S.aux_full[s]);
+      }
+    };
+    int cur = next_task(S, q, abortp, P.status, true);
+    if (cur >= 0) {
+      stage_scales(cur);
+      if (ok) gate_up(cur, -1);
+      int nxt = ok ? next_task(S, q, abortp, P.status, true) : -2;
+      if (nxt == -2) ok = false;
+      if (ok && nxt >= 0) stage_scales(nxt);
+      while (ok) {
+        int nn = -1;
+        if (nxt >= 0) {
+          gate_up(nxt, cur);
+          if (!ok) break;
+          nn = next_task(S, q, abortp, P.status, true);
+          if (nn == -2) { ok = false; break; }
+          if (nn >= 0) stage_scales(nn);
+        } else {
+          fetch_down_words(cur);
+        }
+        if (!ok) break;
+        down();
+        if (nxt < 0) break;
+        cur = nxt;
+        nxt = nn;
+      }
     }
   }
 

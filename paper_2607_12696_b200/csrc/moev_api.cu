@@ -46,6 +46,7 @@ struct moev_ctx {
   int32_t* host_word = nullptr;  // pinned scratch for status / n_active reads
   TmapSet tmaps[kTmapCache];
   int tmap_next = 0;
+  CUtensorMap tm_xq;  // MXFP4 tensor-core path: the [2 * max_tokens, xq_stride] byte array T.xq, box 128 x 2
   int n_sm = 0;
   int unit_cap = 1 << 20;
   bool profile = false;
@@ -133,7 +134,8 @@ bool tc_eligible(const moev_config& c) {
   if (c.afmt != MOEV_ACT_BF16) return false;
   if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: K axes in half chunks of 64, >= 4 chunks per row
     return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 512 && c.I >= 128 &&
-           128 * (c.H / 32) <= tcmx::kScStageBytes;  // a slice's gate/up scale block is staged in shared memory
+           128 * (c.H / 32) <= tcmx::kScStageBytes &&  // a slice's gate/up scale block is staged in shared memory,
+           (c.H + 127) / 128 <= tcmx::kDownWords;         // and one word per W_down row
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
   if (c.H % 128 || c.I % 128) return false;
   const int bk = c.wfmt == MOEV_W_BF16 ? 64 : 128;
@@ -253,7 +255,7 @@ void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.stats = c->tc_stats;
 #endif
   launch_k(tcmx::grouped_ffn_mx_kernel, dim3(c->n_sm), dim3(tcmx::kThreads), tcmx::kSmemBytes, st, ev == nullptr,
-           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
+           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], c->tm_xq, P);
   if (ev) cudaEventRecord(ev[4], st);
 }
 
@@ -338,6 +340,23 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     const size_t max_units = E + A / cap + (size_t)cfg->n_shared * (G / cap + 1) + 8;
     ok = ok && dmalloc(&c->T.units, max_units) == cudaSuccess;
   }
+  if (c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_MXFP4) {
+    // quantised activations (two e4m3 terms per element), loaded by TMA as the MMA's N operand
+    c->T.xq_stride = cfg->H + (cfg->H % 128 ? 128 : 0);
+    ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->T.xq), 2 * G * (size_t)c->T.xq_stride) == cudaSuccess;
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (ok && fn) {
+      cuuint64_t dims[2] = {(cuuint64_t)c->T.xq_stride, (cuuint64_t)(2 * G)};
+      cuuint64_t strides[1] = {(cuuint64_t)c->T.xq_stride};
+      cuuint32_t box[2] = {128, 2};
+      cuuint32_t estr[2] = {1, 1};
+      ok = fn(&c->tm_xq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c->T.xq, dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    } else {
+      ok = false;
+    }
+  }
   ok = ok && dmalloc(&c->hbuf, slots * cfg->I) == cudaSuccess;
   ok = ok && dmalloc(&c->y32, G * cfg->H) == cudaSuccess;
   ok = ok && cudaMalloc(&c->x_stage, G * cfg->H * act_b) == cudaSuccess;
@@ -380,7 +399,7 @@ moev_status moev_destroy(moev_ctx* c) {
   if (!c) return MOEV_EINVAL;
   cudaFree(c->part); cudaFree(c->part_x2); cudaFree(c->part_w2); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
-  cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale);
+  cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
   cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->T.task_counter); cudaFree(c->hbuf); cudaFree(c->y32);
   cudaFree(c->x_stage); cudaFree(c->y_stage);
   if (c->host_word) cudaFreeHost(c->host_word);

@@ -319,6 +319,42 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   if (lane == 0) redf[warp] = amax;
   __syncthreads();
 
+  // ---- MXFP4 tensor-core path: the two e4m3 terms (hi + lo / 16) of x * 2^p_t, the activation
+  // operand of every expert of this call, are formed once per token here (warps other than the
+  // ranking warp).  A ragged last K chunk reads its operand from a tail block after the row:
+  // 64 zeros, then the last 64 elements.
+  if (AFMT == MOEV_ACT_BF16 && T.xq != nullptr && warp > 0) {
+    float am = 0.f;
+    for (int w = 0; w < kRefineWarps; ++w) am = fmaxf(am, redf[w]);
+    int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
+    ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
+    const float ts = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
+    const uint16_t* xr = static_cast<const uint16_t*>(x) + (size_t)t * H;
+    uint8_t* hi_row = T.xq + (size_t)(2 * t) * T.xq_stride;
+    uint8_t* lo_row = hi_row + T.xq_stride;
+    const bool tail = T.xq_stride > H;
+    const int n4 = H / 4 + (tail ? 32 : 0);  // groups of 4 elements, then the 128-byte tail block
+    for (int i = tid - 32; i < n4; i += kRefineThreads - 32) {
+      int src = i * 4, dst = i * 4;
+      bool zero = false;
+      if (i >= H / 4) {
+        const int j = i - H / 4;  // 0..31 within the tail block
+        dst = H + j * 4;
+        zero = j < 16;
+        src = H - 64 + (j - 16) * 4;
+      }
+      uint32_t hi = 0, lo = 0;
+      if (!zero) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(xr + src));
+        float v[4] = {__uint_as_float(q.x << 16) * ts, __uint_as_float(q.x & 0xffff0000u) * ts,
+                      __uint_as_float(q.y << 16) * ts, __uint_as_float(q.y & 0xffff0000u) * ts};
+        split4_e4m3(v, hi, lo);
+      }
+      *reinterpret_cast<uint32_t*>(hi_row + dst) = hi;
+      *reinterpret_cast<uint32_t*>(lo_row + dst) = lo;
+    }
+  }
+
   // ---- exact ranking of the candidates and the router weights (warp 0)
   if (warp == 0) {
     if (lane == 0) {
