@@ -433,6 +433,75 @@ def run_sweep(args):
     v.close()
 
 
+def run_select_demo(args):
+    """Closing the loop of the paper on this path: cost-aware draft selection (Algorithm 1) in
+    front of the verification layer, against acceptance-only selection (the same kernel with
+    empty footprints, i.e. ranking by cumulative draft probability).  A binary draft tree of
+    depth 7 (255 nodes) with expert locality along paths; each node's predicted expert set is
+    its true single-layer routing (the paper's oracle-expert-set setting); gamma = 64 nodes are
+    selected and verified on the DeepSeek-V3.1-shaped FP8 layer.  Prints one JSON line."""
+    import paper_2607_12696_b200 as moev
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    shape = synth.SHAPES["deepseek"]
+    gamma, depth = 64, 7
+    n_layers = layers_that_fit(shape, 2)
+    weights = [synth.make_expert_weights(shape, layer=l, device=dev) for l in range(n_layers)]
+    parent, P, pred = synth.make_draft_tree(1, shape.E, shape.top_k, depth=depth, branch=2, seed_tag="demo-tree",
+                                            p_reuse=args.p_reuse)
+    wr, x_all = synth.make_tree_verify_inputs(shape, parent, pred, device=dev)
+    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, gamma, shape.wfmt,
+                          shape.afmt, shape.score, moev.IMPL_AUTO, shape.routed_scale)
+    v = moev.MoeVerifier(cfg)
+    Wb = moev.expert_bytes(cfg)
+    packed = []
+    for l in range(n_layers):
+        d = {"router_w": wr}
+        d.update({k: t for k, t in weights[l].items() if t is not None})
+        packed.append((moev.binding.make_layer(d), d))
+    t_parent = torch.from_numpy(parent).to(dev)
+    t_P = torch.from_numpy(P).to(dev)
+    t_pred = torch.from_numpy(pred.view(np.int32)).to(dev)
+    result = {"demo": "draft selection -> verification layer", "tree_nodes": int(len(parent)), "gamma": gamma,
+              "p_reuse": args.p_reuse, "workload": "deepseek_fp8, oracle expert sets, 1 layer", "layers_rotated": n_layers}
+    for name, bitmaps in (("acceptance_only", torch.zeros_like(t_pred)), ("cost_aware", t_pred)):
+        out = None
+        for _ in range(3):
+            out = moev.select_drafts(t_parent, t_P, bitmaps, gamma, 1e-6, out=out)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(20):
+            out = moev.select_drafts(t_parent, t_P, bitmaps, gamma, 1e-6, out=out)
+        e1.record()
+        sel = out[0]
+        torch.cuda.synchronize()
+        sel_us = e0.elapsed_time(e1) * 1e3 / 20
+        idx = sel.long()
+        x = x_all[idx].contiguous()
+        outs = [v.alloc_out(gamma, diagnostics=False) for _ in range(n_layers)]
+        for i in range(max(args.warmup, n_layers)):
+            v.verify(packed[i % n_layers][0], x, gamma, outs[i % n_layers])
+        torch.cuda.synchronize()
+        U = int(outs[0]["n_active"].item())
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        for i, (a, b) in enumerate(evs):
+            a.record()
+            v.verify(packed[i % n_layers][0], x, gamma, outs[i % n_layers])
+            b.record()
+        torch.cuda.synchronize()
+        lat = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+        med = lat[len(lat) // 2]
+        result[name] = {"active_experts": U, "verify_latency_us": med, "selection_us": sel_us,
+                        "sum_draft_prob": float(t_P[idx].sum().item()),
+                        "expert_bytes": (U + shape.n_shared) * Wb,
+                        "gbs": (U + shape.n_shared) * Wb / med / 1e3}
+    a, c = result["acceptance_only"], result["cost_aware"]
+    result["active_expert_reduction"] = 1.0 - c["active_experts"] / a["active_experts"]
+    result["verify_latency_ratio"] = c["verify_latency_us"] / a["verify_latency_us"]
+    print(json.dumps(result))
+    v.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -445,6 +514,9 @@ def main():
     ap.add_argument("--cpu-tokens", type=int, default=0, help="tokens of layer 0 the oracle is timed on (0 = all gamma)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="unique-expert sweep (DeepSeek FP8 shape) instead of the bench line")
+    ap.add_argument("--select-demo", action="store_true",
+                    help="cost-aware vs acceptance-only draft selection in front of the verification layer")
+    ap.add_argument("--p-reuse", type=float, default=0.7, help="expert locality along a tree path (select demo)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -454,6 +526,8 @@ def main():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
         if args.sweep:
             run_sweep(args)
+        elif args.select_demo:
+            run_select_demo(args)
         else:
             run_ours(args)
 

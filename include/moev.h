@@ -197,8 +197,8 @@ moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us 
  * (cost of each choice when it was made; may be NULL), buffer_out [W] (final B; may be NULL),
  * n_selected [1] (may be NULL).  traj_workspace [n, W] is caller-provided scratch.  All
  * pointers are DEVICE pointers; one kernel is enqueued on cuda_stream; nothing is allocated.
- * MOEV_EINVAL for n outside 1..65536, W < 1, gamma < 1, eps <= 0, null required pointers, or a
- * bitmap too large for shared memory (W > ~50 000 words). */
+ * MOEV_EINVAL for n outside 1..4096, W < 1, gamma < 1, eps <= 0, null required pointers, or
+ * tables too large for shared memory (3 n + 4 W words above ~50 000). */
 moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, const float* P,
                                const uint32_t* pred, const uint32_t* buffer0, int32_t gamma, float eps,
                                int32_t global_cost, uint32_t* traj_workspace, int32_t* selected,

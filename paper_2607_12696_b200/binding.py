@@ -148,23 +148,26 @@ def route_topk_static(cfg: MoevConfig, router_w: torch.Tensor, x: torch.Tensor, 
 
 
 def select_drafts(parent: torch.Tensor, P: torch.Tensor, pred: torch.Tensor, gamma: int, eps: float = 1e-6,
-                  buffer0: torch.Tensor = None, global_cost: bool = False):
+                  buffer0: torch.Tensor = None, global_cost: bool = False, out: tuple = None):
     """moev_select_drafts: Algorithm 1 on device tensors (parent int32 [n], P float32 [n], pred
     int32/uint32 bitmaps [n, W]).  Returns device tensors (selected [gamma], costs [gamma],
-    buffer [W], n_selected [1]); asynchronous on the current stream."""
+    buffer [W], n_selected [1], workspace [n, W]); asynchronous on the current stream.  Pass the
+    tuple a previous call returned as ``out`` to reuse its tensors (no allocation)."""
     n, W = pred.shape
     dev = pred.device
-    traj = torch.empty(n, W, dtype=torch.int32, device=dev)
-    selected = torch.full((gamma,), -1, dtype=torch.int32, device=dev)
-    costs = torch.zeros(gamma, dtype=torch.int32, device=dev)
-    buf = torch.zeros(W, dtype=torch.int32, device=dev)
-    nsel = torch.zeros(1, dtype=torch.int32, device=dev)
+    if out is None:
+        out = (torch.full((gamma,), -1, dtype=torch.int32, device=dev),
+               torch.zeros(gamma, dtype=torch.int32, device=dev),
+               torch.zeros(W, dtype=torch.int32, device=dev),
+               torch.zeros(1, dtype=torch.int32, device=dev),
+               torch.empty(n, W, dtype=torch.int32, device=dev))
+    selected, costs, buf, nsel, traj = out
     st = lib().moev_select_drafts(n, W, parent.data_ptr(), P.data_ptr(), pred.data_ptr(), _ptr(buffer0), gamma,
                                   eps, int(global_cost), traj.data_ptr(), selected.data_ptr(), costs.data_ptr(),
                                   buf.data_ptr(), nsel.data_ptr(), C.c_void_p(torch.cuda.current_stream().cuda_stream))
     if st != 0:
         raise MoevError(st, "moev_select_drafts rejected the call")
-    return selected, costs, buf, nsel
+    return out
 
 
 def static_scratch_floats(H: int, E: int, gamma: int) -> int:

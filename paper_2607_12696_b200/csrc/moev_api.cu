@@ -620,18 +620,26 @@ moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, cons
                                const uint32_t* buffer0, int32_t gamma, float eps, int32_t global_cost,
                                uint32_t* traj_workspace, int32_t* selected, int32_t* costs, uint32_t* buffer_out,
                                int32_t* n_selected, void* cuda_stream) {
-  if (n < 1 || n > 65536 || W < 1 || gamma < 1 || !parent || !P || !pred || !traj_workspace || !selected)
+  if (n < 1 || n > kSelMaxNodes || W < 1 || gamma < 1 || !parent || !P || !pred || !traj_workspace || !selected)
     return MOEV_EINVAL;
   if (!(eps > 0.f)) return MOEV_EINVAL;  // eps avoids the division by zero (Eq. 9)
-  const size_t smem = ((size_t)W + 96 + (size_t)(n + 31) / 32) * sizeof(uint32_t);
-  if (smem > 200 * 1024) return MOEV_EINVAL;
+  const size_t fixed = select_fixed_smem_words(n, W) * sizeof(uint32_t);
+  constexpr size_t kBudget = 200 * 1024;
+  if (fixed > kBudget) return MOEV_EINVAL;
+  // the footprints are copied to shared memory when they fit beside the tables
+  const size_t traj_bytes = (size_t)n * (size_t)(W | 1) * sizeof(uint32_t);
+  const int in_smem = fixed + traj_bytes <= kBudget;
+  const size_t smem = fixed + (in_smem ? traj_bytes : 0);
   if (smem > 48 * 1024 &&
-      cudaFuncSetAttribute(select_drafts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+      cudaFuncSetAttribute(select_drafts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBudget) != cudaSuccess) {
     cudaGetLastError();
     return MOEV_ECUDA;
   }
-  select_drafts_kernel<<<1, 1024, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
-      n, W, parent, P, pred, buffer0, gamma, eps, global_cost, traj_workspace, selected, costs, buffer_out, n_selected);
+  int threads = (n + 31) & ~31;
+  threads = threads < 128 ? 128 : (threads > kSelThreads ? kSelThreads : threads);
+  select_drafts_kernel<<<1, threads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
+      n, W, parent, P, pred, buffer0, gamma, eps, global_cost, in_smem, traj_workspace, selected, costs, buffer_out,
+      n_selected);
   return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
 }
 

@@ -312,3 +312,20 @@ def make_draft_tree(n_layers: int, E: int, K: int, depth: int = 3, branch: int =
                 bit = l * E + int(e)
                 pred[i, bit >> 5] |= np.uint32(1 << (bit & 31))
     return np.array(parent, dtype=np.int32), np.array(P, dtype=np.float32), pred
+
+
+def make_tree_verify_inputs(shape: Shape, parent: np.ndarray, pred: np.ndarray, device="cpu",
+                            seed_tag="treex"):
+    """Hidden states for the nodes of a draft tree whose single-layer expert sets are given as
+    bitmaps (``pred`` uint32 [n, ceil(E/32)], exactly top_k bits per node): through the logit
+    carrier, node i routes to exactly the experts of its bitmap (logits 4 - 0.25 j for its j-th
+    expert in ascending id, -4 elsewhere).  Returns (router_w [E,H], x [n,H])."""
+    n, E, k = len(parent), shape.E, shape.top_k
+    logits = np.full((n, E), -4.0, dtype=np.float32)
+    for i in range(n):
+        ids = [e for e in range(E) if (int(pred[i, e >> 5]) >> (e & 31)) & 1]
+        assert len(ids) == k, "one top-k set per node"
+        for j, e in enumerate(ids):
+            logits[i, e] = 4.0 - 0.25 * j
+    gx = _gen(device, shape.name, seed_tag, "x", n)
+    return _carrier(shape, torch.from_numpy(logits), device, gx)

@@ -17,7 +17,7 @@ def _run(parent, P, pred, gamma, eps=1e-6, buffer0=None, global_cost=False):
     tP = torch.from_numpy(P).to(dev)
     tpred = torch.from_numpy(pred.view(np.int32)).to(dev)
     tb = None if buffer0 is None else torch.from_numpy(buffer0.view(np.int32)).to(dev)
-    sel, costs, buf, nsel = moev.select_drafts(tp, tP, tpred, gamma, eps, tb, global_cost)
+    sel, costs, buf, nsel, _ = moev.select_drafts(tp, tP, tpred, gamma, eps, tb, global_cost)
     torch.cuda.synchronize()
     k = int(nsel.item())
     return sel.cpu().numpy()[:k], costs.cpu().numpy()[:k], buf.cpu().numpy().view(np.uint32)
@@ -62,3 +62,35 @@ def test_selection_rejects_bad_arguments():
         moev.select_drafts(tp, tP, tpred, 0)
     with pytest.raises(moev.MoevError):
         moev.select_drafts(tp, tP, tpred, 2, eps=0.0)
+
+
+def test_selection_then_verify_union_matches_buffer():
+    """End to end with the verification layer: when the predicted sets are the nodes' true routing
+    (single layer), the expert buffer the selection ends with is exactly the union the router
+    kernels report for the selected tokens."""
+    shape = synth.SHAPES["tiny"]
+    parent, P, pred = synth.make_draft_tree(1, shape.E, shape.top_k, depth=4, branch=2, seed_tag="e2e-tree")
+    wr, x_all = synth.make_tree_verify_inputs(shape, parent, pred, device="cuda")
+    gamma = 8
+    tp, tP = torch.from_numpy(parent).cuda(), torch.from_numpy(P).cuda()
+    tpred = torch.from_numpy(pred.view(np.int32)).cuda()
+    sel, costs, buf, nsel, _ = moev.select_drafts(tp, tP, tpred, gamma, 1e-6)
+    torch.cuda.synchronize()
+    w = synth.make_expert_weights(shape, layer=0, device="cuda")
+    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, gamma, shape.wfmt, shape.afmt,
+                          shape.score, moev.IMPL_AUTO, shape.routed_scale)
+    v = moev.MoeVerifier(cfg)
+    d = {"router_w": wr}
+    d.update({k: t for k, t in w.items() if t is not None})
+    L = moev.binding.make_layer(d)
+    out = v.alloc_out(gamma, diagnostics=True)
+    v.verify(L, x_all[sel.long()].contiguous(), gamma, out)
+    v.status_sync()
+    U = int(out["n_active"].item())
+    bits = buf.cpu().numpy().view(np.uint32)
+    assert U == int(sum(bin(int(b)).count("1") for b in bits))
+    union = out["union_ids"].cpu().numpy()[:U]
+    expect = [e for e in range(shape.E) if (int(bits[e >> 5]) >> (e & 31)) & 1]
+    np.testing.assert_array_equal(union, np.array(expect, dtype=np.int32))
+    assert int(costs.sum().item()) == U          # marginal costs add up to the final footprint
+    v.close()
