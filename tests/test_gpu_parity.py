@@ -45,6 +45,16 @@ def test_gptoss_shaped_reduced_ragged(impl, gamma):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("gamma,U,n_shared", [(40, 4, 0), (33, 8, 0), (21, 12, 1), (64, 4, 2)])
+def test_gptoss_shaped_many_tokens_per_expert(impl, gamma, U, n_shared):
+    """MXFP4 with more tokens per expert than one work unit holds (runs of 16), with and
+    without shared experts, on ragged dimensions."""
+    shape = small_shape("gptoss", H=736, I=352, E=32, n_shared=n_shared)
+    err, ref = parity_case(shape, gamma, routing="exact", impl=impl, U=U)
+    assert ref.n_active == U
+
+
+@pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("gamma,U", [(1, 8), (8, 8), (8, 64), (32, 40), (128, 8), (128, 64)])
 def test_exact_union_cases(impl, gamma, U):
     """Degenerate groupings: all tokens on the same k experts (m_e = gamma), every expert
