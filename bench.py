@@ -58,7 +58,9 @@ DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 # capture of a smaller case of the same kernel (profiles/grouped_ffn_tc_fp8_E64_g16.md:
 # 2.458471 GB + 4.67 MB against 2.422802 GB); traffic grows in proportion to the experts
 # streamed, so the full-size launch is scaled by the same ratio.  Absent = not captured.
-NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.458471e9 + 4.670208e6) / 2.422801920e9}
+NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.458471e9 + 4.670208e6) / 2.422801920e9,
+                     # profiles/grouped_ffn_mx_gptoss_g64.md: 1.855084 GB + 3.81 MB against 1.454112 GB
+                     ("mxfp4", "tcgen05"): (1.855084e9 + 3.813376e6) / 1.454112e9}
 
 ROUTING = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
            "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing}
@@ -314,7 +316,8 @@ def run_ours(args):
         if impl_name == "simt":  # two kernels; the first (gate/up) streams 2/3 of the bytes
             k_name, k_bytes, k_us = "ffn_gateup_simt", mean_bytes * 2.0 / 3.0, kern_us[3]
         else:
-            k_name, k_bytes, k_us = "grouped_ffn_tc_kernel", mean_bytes, kern_us[3]
+            k_name = "grouped_ffn_mx_kernel" if shape.wfmt == synth.W_MXFP4 else "grouped_ffn_tc_kernel"
+            k_bytes, k_us = mean_bytes, kern_us[3]
         achieved = k_bytes / (k_us * 1e-6) / 1e9 if k_us > 0 else None
         dtype_name = {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "mxfp4"}[shape.wfmt]
         cpu = None
