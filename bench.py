@@ -289,6 +289,24 @@ def run_ours(args):
     kern_us, kern_calls = v.profile_read()
     v.profile_enable(False)
 
+    # ---- the rotated layers as one pipelined call per n_layers steps (independent inputs): the
+    # next layer's router fills the tail of the previous layer's expert kernel
+    pipe_us = None
+    if n_layers > 1:
+        Ls, xs_, os_ = [p[0] for p in packed], [L["x"] for L in layers], outs
+        for _ in range(2):
+            v.verify_pipeline(Ls, xs_, gamma, os_)
+        n_calls = max(1, args.steps // n_layers)
+        pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        pe0.record()
+        for _ in range(n_calls):
+            v.verify_pipeline(Ls, xs_, gamma, os_)
+        pe1.record()
+        barrier()
+        pipe_us = pe0.elapsed_time(pe1) * 1e3 / (n_calls * n_layers)
+        v.status_sync()
+
     # ---- end to end through the host-buffer entry point
     xh = [L["x"].cpu().pin_memory() for L in layers]
     yh = [torch.empty_like(t).pin_memory() for t in xh]
@@ -331,6 +349,9 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
+            "pipelined": (None if pipe_us is None else
+                          {"us_per_layer": pipe_us, "layers_per_call": n_layers,
+                           "gbs": mean_bytes / pipe_us / 1e3, "note": "moev_verify_pipeline, independent inputs per layer"}),
             "dtype": dtype_name,
             "data": "synthetic",
             "config": {"workload": args.workload, "gamma": gamma, "H": shape.H, "I": shape.I,

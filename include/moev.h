@@ -181,6 +181,20 @@ moev_status moev_profile_enable(moev_ctx* ctx, int32_t on);
 moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[6]*/,
                               int32_t* calls);
 
+/* Several independent layers in one call (multi-layer pipelining; the paper has no counterpart:
+ * its prototype runs layer by layer).  Equivalent to n_layers calls of moev_verify on the same
+ * stream with layers[l], x[l], outs[l] and the same gamma, except that the first kernel of layer
+ * l + 1 is enqueued as a programmatic dependent launch: its CTAs occupy the SMs that layer l's
+ * expert kernel has already left, so the router of the next layer overlaps the tail of the
+ * previous one.  The inputs x[l] must not depend on the outputs of earlier layers of the same
+ * call (independent requests, or hidden states that are already available); results are the same
+ * as those of separate calls.  layers / x / outs are HOST arrays of n_layers entries whose
+ * pointers are DEVICE pointers.  Errors as moev_verify; nothing is enqueued for layers after the
+ * first failing one. */
+moev_status moev_verify_pipeline(moev_ctx* ctx, int32_t n_layers, const moev_layer* layers,
+                                 const void* const* x, int32_t gamma, const moev_out* outs,
+                                 void* cuda_stream);
+
 /* Cost-aware draft selection: Algorithm 1 of the paper (Sec. 4.2, Eqs. 7-10), the step that
  * runs between drafting and verification and decides which gamma draft-tree nodes are verified.
  *   n, parent [n]   draft tree in topological order: parent[i] < i, parent[root] = -1

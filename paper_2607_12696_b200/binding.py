@@ -20,7 +20,8 @@ STATUS = {0: "MOEV_OK", 1: "MOEV_EINVAL", 2: "MOEV_EUNSUPPORTED", 3: "MOEV_ECUDA
 EXPORTS = ("moev_create", "moev_destroy", "moev_verify", "moev_verify_host", "moev_status_sync",
            "moev_last_error", "moev_expert_bytes", "moev_expert_code_bytes",
            "moev_launches_per_call", "moev_resolved_impl", "moev_profile_enable",
-           "moev_profile_read", "moev_route_topk_static", "moev_route_topk_static_scratch_floats", "moev_select_drafts")
+           "moev_profile_read", "moev_route_topk_static", "moev_route_topk_static_scratch_floats", "moev_select_drafts",
+           "moev_verify_pipeline")
 
 
 class MoevError(RuntimeError):
@@ -90,6 +91,9 @@ def lib() -> C.CDLL:
         L.moev_verify.restype = C.c_int
         L.moev_verify.argtypes = [C.c_void_p, C.POINTER(_Layer), C.c_void_p, C.c_int32,
                                   C.POINTER(_Out), C.c_void_p]
+        L.moev_verify_pipeline.restype = C.c_int
+        L.moev_verify_pipeline.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_Layer), C.POINTER(C.c_void_p), C.c_int32,
+                                           C.POINTER(_Out), C.c_void_p]
         L.moev_verify_host.restype = C.c_int
         L.moev_verify_host.argtypes = [C.c_void_p, C.POINTER(_Layer), C.c_void_p, C.c_int32,
                                        C.c_void_p, C.c_void_p, C.c_void_p]
@@ -240,6 +244,19 @@ class MoeVerifier:
             setattr(O, n, _ptr(out.get(n)))
         self._check(lib().moev_verify(self._h, C.byref(layer), _ptr(x), gamma, C.byref(O),
                                       self._stream()))
+
+    def verify_pipeline(self, layers: list, xs: list, gamma: int, outs: list):
+        """moev_verify_pipeline: independent layers back to back, the router of each overlapping
+        the tail of the previous layer's expert kernel."""
+        n = len(layers)
+        assert len(xs) == n and len(outs) == n
+        LA = (_Layer * n)(*layers)
+        XA = (C.c_void_p * n)(*[x.data_ptr() for x in xs])
+        OA = (_Out * n)()
+        for i, out in enumerate(outs):
+            for f in _OUT_FIELDS:
+                setattr(OA[i], f, _ptr(out.get(f)))
+        self._check(lib().moev_verify_pipeline(self._h, n, LA, XA, gamma, OA, self._stream()))
 
     def verify_host(self, layer: _Layer, x_host: torch.Tensor, gamma: int, y_host: torch.Tensor,
                     n_active_host: torch.Tensor):

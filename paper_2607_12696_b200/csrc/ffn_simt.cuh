@@ -213,6 +213,8 @@ __global__ void __launch_bounds__(256) ffn_down_simt(LayerPtrs L, Tables T, cons
 // y32 (fp32) -> y in the activation format
 template <int AFMT>
 __global__ void finalize_kernel(const float* __restrict__ y32, void* __restrict__ y, size_t n) {
+  // a dependent launch (the first kernel of the next layer of a pipelined call) may be scheduled from here on
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the FFN kernel's reductions are complete
   size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= n) return;

@@ -50,6 +50,7 @@ struct moev_ctx {
   int n_sm = 0;
   int unit_cap = 1 << 20;
   bool profile = false;
+  bool chain = false;  // next moev_verify is a later layer of a pipelined call: its first kernel is a dependent launch
   cudaEvent_t ev[kProfSlots][7];  // before/after each kernel of a call
   int prof_n = 0;
   bool prof_events_ready = false;
@@ -461,10 +462,10 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   const bool pdl = ev == nullptr;  // event records between the kernels would serialise them anyway
   const size_t rp_smem = router_partial_smem(c->ks);
   if (g.afmt == MOEV_ACT_FP32)
-    launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, false, x, layer->router_w,
+    launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain, x, layer->router_w,
              c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
   else
-    launch_k(router_partial_kernel<MOEV_ACT_BF16>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, false, x, layer->router_w,
+    launch_k(router_partial_kernel<MOEV_ACT_BF16>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain, x, layer->router_w,
              c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
   if (ev) cudaEventRecord(ev[1], st);
   if (g.afmt == MOEV_ACT_FP32)
@@ -494,6 +495,19 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "kernel launch failed: %s", cudaGetErrorString(e));
   return MOEV_OK;
+}
+
+moev_status moev_verify_pipeline(moev_ctx* c, int32_t n_layers, const moev_layer* layers, const void* const* x,
+                                 int32_t gamma, const moev_out* outs, void* cuda_stream) {
+  if (!c) return MOEV_EINVAL;
+  if (n_layers < 1 || !layers || !x || !outs) return fail(c, MOEV_EINVAL, "null argument or n_layers < 1");
+  moev_status s = MOEV_OK;
+  for (int32_t l = 0; l < n_layers && s == MOEV_OK; ++l) {
+    c->chain = l > 0;
+    s = moev_verify(c, &layers[l], x[l], gamma, &outs[l], cuda_stream);
+  }
+  c->chain = false;
+  return s;
 }
 
 moev_status moev_verify_host(moev_ctx* c, const moev_layer* layer, const void* x_host, int32_t gamma,

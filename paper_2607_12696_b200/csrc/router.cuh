@@ -141,6 +141,12 @@ __global__ void __launch_bounds__(256) router_partial_kernel(const void* __restr
     for (int w = 1; w < 8; ++w) w2max = fmaxf(w2max, wmax_s[w]);
     part_w2max[(size_t)c * gridDim.y + blockIdx.y] = w2max;
   }
+  // In a pipelined multi-layer call this kernel is launched as a programmatic dependent of the
+  // previous layer's last kernel and fills the SMs that layer's FFN kernel has already left.  It
+  // touches nothing the previous layer still uses, but it must not complete before that layer has:
+  // the kernels after it (which do reuse the workspace) wait only for this one.  Without the
+  // launch attribute the instruction returns at once.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 struct RouteOut {  // optional caller-visible copies (may be null)

@@ -85,6 +85,33 @@ def test_exact_logit_ties_break_to_lower_id(impl):
     compare(shape, res, ref, 6)
 
 
+@pytest.mark.parametrize("base,kw", [("deepseek", dict(H=1024, I=512, E=64)), ("gptoss", dict(H=736, I=352, E=32)),
+                                     ("qwen", dict(H=1024, I=384, E=32))])
+def test_pipelined_layers_match_oracle(base, kw):
+    """moev_verify_pipeline: three independent layers in one call (the router of layer l + 1
+    overlaps the tail of layer l) give each layer's oracle result; run twice back to back."""
+    shape = small_shape(base, **kw)
+    gamma, n = 24, 3
+    v = moev.MoeVerifier(gcfg(shape, gamma))
+    layers, keep, xs, refs = [], [], [], []
+    for l in range(n):
+        w = synth.make_expert_weights(shape, layer=l, device="cuda")
+        wr, x = synth.make_scattered_routing(shape, gamma, layer=l, device="cuda") if shape.E <= shape.H and base != "qwen" \
+            else synth.make_iid_routing(shape, gamma, layer=l, device="cuda")
+        L, d = device_layer(wr, w)
+        layers.append(L); keep.append(d); xs.append(x)
+        refs.append(oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), gamma))
+    for rep in range(2):
+        outs = [v.alloc_out(gamma) for _ in range(n)]
+        v.verify_pipeline(layers, xs, gamma, outs)
+        v.status_sync()
+        torch.cuda.synchronize()
+        for l in range(n):
+            res = {k: (t.float() if t.dtype == torch.bfloat16 else t).cpu().numpy() for k, t in outs[l].items()}
+            compare(shape, res, refs[l], gamma)
+    v.close()
+
+
 def test_context_reuse_and_smaller_gamma():
     """One context, several calls with different gamma: workspace state must not leak."""
     shape = small_shape("qwen", H=512, I=256, E=16, top_k=4)
