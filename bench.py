@@ -45,6 +45,11 @@ WORKLOADS = {
     "gptoss_mxfp4_g32": ("gptoss", 32, "iid", {}),
     "gptoss_mxfp4_g64": ("gptoss", 64, "iid", {}),
     "tiny_fp32_g8": ("tiny", 8, "iid", {}),
+    # batched verification (B requests x gamma tree tokens in one call) and skewed routing
+    "deepseek_fp8_b4g64_scattered": ("deepseek", 256, "scattered", {}),
+    "deepseek_fp8_b8g64_scattered": ("deepseek", 512, "scattered", {}),
+    "deepseek_fp8_b4g64_zipf": ("deepseek", 256, "zipf", {"alpha": 1.0}),
+    "deepseek_fp8_b8g64_zipf": ("deepseek", 512, "zipf", {"alpha": 1.0}),
     # profiling-size cases (a few GB on the device, still far larger than L2): the DeepSeek-
     # and Qwen-shaped layers with 64 experts
     "deepseek_fp8_E64_g16_profile": ("deepseek", 16, "scattered", {"_E": 64}),
@@ -63,7 +68,8 @@ NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.458471e9 + 4.670208e6) / 2.4228
                      ("mxfp4", "tcgen05"): (1.855084e9 + 3.813376e6) / 1.454112e9}
 
 ROUTING = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
-           "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing}
+           "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing,
+           "zipf": synth.make_zipf_routing}
 
 
 def measured_peaks():

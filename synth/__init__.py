@@ -226,6 +226,20 @@ def make_clustered_routing(shape: Shape, gamma: int, p_copy: float = 0.7, layer:
     return _carrier(shape, logits, device, gx)
 
 
+def make_zipf_routing(shape: Shape, gamma: int, alpha: float = 1.0, layer: int = 0, device="cpu",
+                      seed_tag="zipf"):
+    """Skewed routing (a few hot experts, as in batched verification of similar requests): expert
+    of popularity rank r (ranks assigned by a seeded permutation) gets the logit offset
+    -alpha * ln(1 + r) on top of iid N(0,1) noise; bf16-rounded, through the logit carrier."""
+    g = _gen("cpu", shape.name, layer, seed_tag, "logits", gamma)
+    noise = torch.randn(gamma, shape.E, generator=g)
+    rs = np.random.RandomState(stream_seed(shape.name, layer, seed_tag, "rank") % (2 ** 31))
+    rank = torch.from_numpy(rs.permutation(shape.E).astype(np.float32))
+    logits = (noise - alpha * torch.log1p(rank)[None, :]).to(torch.bfloat16).to(torch.float32)
+    gx = _gen(device, shape.name, layer, seed_tag, "x", gamma)
+    return _carrier(shape, logits, device, gx)
+
+
 def union_feasible(shape: Shape, gamma: int, U: int) -> bool:
     return shape.top_k <= U <= min(shape.E, gamma * shape.top_k)
 

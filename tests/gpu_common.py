@@ -64,7 +64,8 @@ def parity_case(shape, gamma, routing="iid", impl=moev.IMPL_AUTO, layer_id=0, **
     dev = "cuda"
     w = synth.make_expert_weights(shape, layer=layer_id, device=dev)
     fn = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
-          "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing}[routing]
+          "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing,
+          "zipf": synth.make_zipf_routing}[routing]
     wr, x = fn(shape, gamma, layer=layer_id, device=dev, **kw)
     res = run_gpu(shape, wr, w, x, gamma, impl)
     ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), gamma)

@@ -64,6 +64,18 @@ def test_exact_union_cases(impl, gamma, U):
     assert ref.n_active == U
 
 
+@pytest.mark.parametrize("base,kw,gamma", [("deepseek", dict(H=512, I=256, E=64), 512),
+                                           ("gptoss", dict(H=736, I=352, E=32), 200),
+                                           ("qwen", dict(H=512, I=256, E=32), 260)])
+def test_batched_verification_skewed_routing(base, kw, gamma):
+    """Many rows per call (several requests' trees at once) with Zipf-skewed routing: hot
+    experts receive hundreds of tokens (many work units each), cold ones none."""
+    shape = small_shape(base, **kw)
+    err, ref = parity_case(shape, gamma, routing="zipf", alpha=1.5)
+    counts = np.bincount(ref.topk_ids.reshape(-1), minlength=shape.E)
+    assert counts.max() >= gamma // 2 and ref.n_active <= shape.E
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_topk_equals_E_and_two_shared(impl):
     shape = small_shape("deepseek", H=256, I=128, E=8, top_k=8, n_shared=2)

@@ -388,3 +388,16 @@ def test_byte_model_matches_paper_figures():
         s = synth.SHAPES[name]
         assert s.code_bytes_per_expert() == oracle.expert_code_bytes(_ocfg(s))
         assert s.scale_bytes_per_expert() == oracle.expert_scale_bytes(_ocfg(s))
+
+
+def test_zipf_routing_is_skewed_and_has_a_margin():
+    """The skewed generator concentrates assignments on few experts; logits are exact through
+    the carrier, so the oracle's ids are the top-k of the constructed logits."""
+    shape = small_shape("deepseek", H=256, I=128, E=64)
+    wr, x = synth.make_zipf_routing(shape, 128, alpha=1.5)
+    res = oracle.moe_verify(_ocfg(shape), {"router_w": synth.to_numpy(wr)}, synth.to_numpy(x), 128, skip_ffn=True)
+    counts = np.bincount(res.topk_ids.reshape(-1), minlength=shape.E)
+    assert counts.max() >= 64 and (counts == 0).sum() >= 1
+    logits = x[:, :shape.E].float().numpy().astype(np.float64)
+    np.testing.assert_array_equal(np.sort(res.topk_ids, axis=1),
+                                  np.sort(np.argsort(-logits, axis=1, kind="stable")[:, :shape.top_k], axis=1))
