@@ -110,8 +110,9 @@ cudaError_t dmalloc(T** p, size_t count) {
   return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
 }
 
+bool route_use_bitmap(const moev_config& c, int gamma) { return route_bitmap_bytes(c.E, gamma) <= kRouteBitmapBudget; }
 size_t route_smem(const moev_config& c, int gamma) {
-  return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4;
+  return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + (route_use_bitmap(c, gamma) ? route_bitmap_bytes(c.E, gamma) : 0);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -370,6 +371,10 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   // opt in to large dynamic shared memory where the shape needs it
   if (ok) {
     size_t gs = route_smem(*cfg, cfg->max_tokens);
+    {  // the largest gamma that still uses the token bitmaps may need more than max_tokens does
+      const int g_bm = (int)(kRouteBitmapBudget / (4 * (size_t)cfg->E)) * 32;
+      if (g_bm < cfg->max_tokens && g_bm >= 1) gs = gs > route_smem(*cfg, g_bm) ? gs : route_smem(*cfg, g_bm);
+    }
     ok = ok && cudaFuncSetAttribute(router_partial_kernel<MOEV_ACT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)router_partial_smem(kRouterMaxKS)) == cudaSuccess;
     ok = ok && cudaFuncSetAttribute(router_partial_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -478,7 +483,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
              g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale);
   if (ev) cudaEventRecord(ev[2], st);
   launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
-           g.n_shared, c->unit_cap);
+           g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma));
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);
@@ -658,6 +663,9 @@ moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, cons
 }
 
 #ifdef MOEV_TC_STATS
+extern "C" int32_t moev_debug_rt_stats(long long* host_out /*[32]*/) {
+  return cudaMemcpyFromSymbol(host_out, g_rt_stats, sizeof(long long) * 32) == cudaSuccess ? 0 : -1;
+}
 // Debug builds: copy the per-CTA wait-cycle counters of the last tensor-core FFN launch.
 int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*16]*/) {
   if (!c || !host_out) return -1;

@@ -149,6 +149,13 @@ __global__ void __launch_bounds__(256) router_partial_kernel(const void* __restr
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+#ifdef MOEV_TC_STATS
+__device__ long long g_rt_stats[32];  // debug builds: phase timestamps of the routing kernels (CTA 0)
+#define MOEV_RT_MARK(i) do { __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) g_rt_stats[i] = clock64(); } while (0)
+#else
+#define MOEV_RT_MARK(i)
+#endif
+
 struct RouteOut {  // optional caller-visible copies (may be null)
   int32_t* topk_ids;
   float* topk_w;
@@ -183,10 +190,12 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   asm volatile("griddepcontrol.wait;" ::: "memory");               // router partials are complete
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  MOEV_RT_MARK(0);
   // zero this token's row of the fp32 combine accumulator
   for (int i = tid; i < H / 4; i += kRefineThreads)
     reinterpret_cast<float4*>(y32 + (size_t)t * H)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 
+  MOEV_RT_MARK(1);
   // ---- fp32 logits of this token (two threads per expert when the block is wide enough)
   {
     const int split = (2 * E <= kRefineThreads) ? 2 : 1;
@@ -210,6 +219,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       if (act && half == 0) l32[e] = s;
     }
   }
+  MOEV_RT_MARK(2);
   float x2 = 0.f, w2 = 0.f;
   const int n_et = (E + kRouterETile - 1) / kRouterETile;
   for (int c = tid; c < n_slices; c += kRefineThreads) {
@@ -270,6 +280,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   }
   __syncthreads();
   const int ncand = ncand_s;
+  MOEV_RT_MARK(3);
 
   // ---- exact (fp64) logits of the candidates, kRefineCand at a time; a thread owns groups of 4 columns
   float amax = 0.f;
@@ -320,6 +331,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     }
     __syncthreads();
   }
+  MOEV_RT_MARK(4);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
   if (lane == 0) redf[warp] = amax;
@@ -361,6 +373,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     }
   }
 
+  MOEV_RT_MARK(5);
   // ---- exact ranking of the candidates and the router weights (warp 0)
   if (warp == 0) {
     if (lane == 0) {
@@ -414,14 +427,18 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       if (O.topk_w) O.topk_w[a] = (float)wgt;
     }
   }
+  MOEV_RT_MARK(6);
 }
 
 // One CTA (1024 threads): per-expert histogram of the selected ids, block scan over the E
 // counts (ascending union and offsets), FFN work units, then one warp per expert walks the
 // assignments in order with ballots and writes the stable permutation.
-// Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A].
+// Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A] | (use_bitmap) token bitmaps [E][ceil(gamma/32)].
+// Bytes beyond the bitmaps' budget: the caller passes use_bitmap = 0 and one warp orders the slots.
+inline size_t route_bitmap_bytes(int E, int gamma) { return (size_t)E * ((gamma + 31) / 32) * 4; }
+constexpr size_t kRouteBitmapBudget = 96 * 1024;
 __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O, int gamma, int E,
-                                                           int k, int n_shared, int unit_cap) {
+                                                           int k, int n_shared, int unit_cap, int use_bitmap) {
   extern __shared__ int32_t sm[];
   const int A = gamma * k;
   int32_t* cnt = sm;
@@ -434,6 +451,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   asm volatile("griddepcontrol.wait;" ::: "memory");               // top-k tables are complete
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  MOEV_RT_MARK(8);
   for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
   __syncthreads();
   for (int a = tid; a < A; a += blockDim.x) {
@@ -444,6 +462,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   }
   __syncthreads();
 
+  MOEV_RT_MARK(9);
   // ---- phase 2: exclusive scans over experts (E <= 512 <= blockDim)
   {
     int c = tid < E ? cnt[tid] : 0, f = c > 0 ? 1 : 0;
@@ -479,6 +498,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   }
   __syncthreads();
 
+  MOEV_RT_MARK(10);
   // ---- phase 2b: work units for the tensor-core FFN: the shared experts, then expert u of the
   // union, each cut into ceil(m / unit_cap) runs of at most unit_cap slots.  The shared experts
   // see every token, so their tasks are the longest; first in unit order, they are never the
@@ -508,9 +528,37 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
     if (tid == blockDim.x - 1) { *T.n_units = base + sc; *T.task_counter = 0; }
   }
 
-  // ---- phase 3: stable permutation.  Warp 0 walks the assignments in order, 32 at a time;
-  // uidx[] is reused as the running count of slots already handed out per expert.
+  MOEV_RT_MARK(11);
+  // ---- phase 3: stable permutation.  A token selects an expert at most once, so the slot of
+  // assignment (t, e) inside e's run is the number of tokens below t that selected e: a prefix
+  // population count over e's token bitmap, one thread per assignment.
   __syncthreads();
+  if (use_bitmap) {
+    const int TW = (gamma + 31) / 32;
+    uint32_t* tb = reinterpret_cast<uint32_t*>(sm + 3 * E + 2 * A);  // [E][TW]
+    for (int i = tid; i < E * TW; i += blockDim.x) tb[i] = 0u;
+    __syncthreads();
+    for (int a = tid; a < A; a += blockDim.x) {
+      const int t = a / k;
+      atomicOr(&tb[ids_s[a] * TW + (t >> 5)], 1u << (t & 31));
+    }
+    __syncthreads();
+    for (int a = tid; a < A; a += blockDim.x) {
+      const int t = a / k, e = ids_s[a];
+      const uint32_t* row = tb + e * TW;
+      int rank = __popc(row[t >> 5] & ((1u << (t & 31)) - 1u));
+      for (int w = 0; w < (t >> 5); ++w) rank += __popc(row[w]);
+      const int pos = excl[e] + rank;
+      T.perm[pos] = a;
+      T.slot_token[pos] = t;
+      T.slot_w[pos] = w_s[a];
+      if (O.perm) O.perm[pos] = a;
+    }
+    MOEV_RT_MARK(12);
+    return;
+  }
+  // Fallback for very large gamma: warp 0 walks the assignments in order, 32 at a time; uidx[]
+  // is reused as the running count of slots already handed out per expert.
   for (int e = tid; e < E; e += blockDim.x) uidx[e] = 0;
   __syncthreads();
   if (warp == 0) {
@@ -532,6 +580,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       __syncwarp();
     }
   }
+  MOEV_RT_MARK(12);
 }
 
 }  // namespace moev
