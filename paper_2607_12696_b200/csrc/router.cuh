@@ -49,6 +49,13 @@ __device__ __forceinline__ float load_act1(const void* x, size_t idx) {
   return bf16_bits_to_float(__ldg(static_cast<const uint16_t*>(x) + idx));
 }
 
+#ifdef MOEV_TC_STATS
+__device__ long long g_rt_stats[32];  // debug builds: phase timestamps of the routing kernels (CTA 0)
+#define MOEV_RT_MARK(i) do { __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) g_rt_stats[i] = clock64(); } while (0)
+#else
+#define MOEV_RT_MARK(i)
+#endif
+
 // part[c, t, e] = sum_{h in slice c} x[t,h] * Wr[e,h]  (fp32, sequential over the slice)
 // part_x2[c, t] = sum_{h in slice c} x[t,h]^2,
 // part_w2max[c, j] = max over the experts of tile j of sum_{h in slice c} Wr[e,h]^2
@@ -149,13 +156,6 @@ __global__ void __launch_bounds__(256) router_partial_kernel(const void* __restr
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-#ifdef MOEV_TC_STATS
-__device__ long long g_rt_stats[32];  // debug builds: phase timestamps of the routing kernels (CTA 0)
-#define MOEV_RT_MARK(i) do { __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) g_rt_stats[i] = clock64(); } while (0)
-#else
-#define MOEV_RT_MARK(i)
-#endif
-
 struct RouteOut {  // optional caller-visible copies (may be null)
   int32_t* topk_ids;
   float* topk_w;
@@ -186,6 +186,11 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   __shared__ double red[kRefineWarps][kRefineCand];
   __shared__ float redf[kRefineWarps], redw[kRefineWarps];
   __shared__ int ncand_s;
+  __shared__ float kth_s;
+  __shared__ int wcnt_s[kRefineWarps];
+  __shared__ __align__(16) float psum[kRefineThreads * 4];  // group sums of the split-K partials
+  __shared__ double sel_v_s[kMaxTopK];
+  __shared__ int sel_e_s[kMaxTopK];
   const int t = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   asm volatile("griddepcontrol.wait;" ::: "memory");               // router partials are complete
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -196,30 +201,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     reinterpret_cast<float4*>(y32 + (size_t)t * H)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 
   MOEV_RT_MARK(1);
-  // ---- fp32 logits of this token (two threads per expert when the block is wide enough)
-  {
-    const int split = (2 * E <= kRefineThreads) ? 2 : 1;
-    const size_t cs = (size_t)gamma * E;
-    for (int base = 0; base < E * split; base += kRefineThreads) {  // one trip when split == 2
-      const int idx = base + tid;
-      const bool act = idx < E * split;
-      const int e = act ? idx / split : 0, half = idx % split;
-      const float* pp = part + (size_t)t * E + e;
-      float s = 0.f;
-      int c = act ? half : n_slices;
-      for (; c + 15 * split < n_slices; c += 16 * split) {
-        float v[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = __ldg(pp + (size_t)(c + i * split) * cs);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) s += v[i];
-      }
-      for (; c < n_slices; c += split) s += __ldg(pp + (size_t)c * cs);
-      if (split == 2) s += __shfl_xor_sync(0xffffffffu, s, 1);  // all lanes reach this point
-      if (act && half == 0) l32[e] = s;
-    }
-  }
-  MOEV_RT_MARK(2);
+  // ---- norms for the error bound (loaded first: their latency overlaps the partial sums below)
   float x2 = 0.f, w2 = 0.f;
   const int n_et = (E + kRouterETile - 1) / kRouterETile;
   for (int c = tid; c < n_slices; c += kRefineThreads) {
@@ -228,55 +210,104 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     for (int j = 0; j < n_et; ++j) m = fmaxf(m, part_w2max[(size_t)c * n_et + j]);
     w2 += m;
   }
+  // ---- fp32 logits of this token: the split-K partials summed over the slices
+  if ((E & 3) == 0 && E / 4 <= kRefineThreads) {
+    // thread (g, q): slices g, g + G, ... of the four experts 4q .. 4q + 3 (one 16-byte load per slice,
+    // eight in flight), then the G group sums are added in a fixed order
+    const int nq = E / 4, G = kRefineThreads / nq;
+    const int q = tid % nq, g = tid / nq;
+    const size_t cs = (size_t)gamma * E;
+    float4 sacc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (g < G) {
+      const float* pp = part + (size_t)t * E + 4 * q;
+      int c = g;
+      for (; c + 7 * G < n_slices; c += 8 * G) {
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = __ldg(reinterpret_cast<const float4*>(pp + (size_t)(c + i * G) * cs));
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { sacc.x += v[i].x; sacc.y += v[i].y; sacc.z += v[i].z; sacc.w += v[i].w; }
+      }
+      for (; c < n_slices; c += G) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(pp + (size_t)c * cs));
+        sacc.x += v.x; sacc.y += v.y; sacc.z += v.z; sacc.w += v.w;
+      }
+      *reinterpret_cast<float4*>(&psum[g * E + 4 * q]) = sacc;
+    }
+    __syncthreads();
+    for (int e = tid; e < E; e += kRefineThreads) {
+      float sum = 0.f;
+      for (int gg = 0; gg < G; ++gg) sum += psum[gg * E + e];
+      l32[e] = sum;
+    }
+  } else {
+    const int split = (2 * E <= kRefineThreads) ? 2 : 1;
+    const size_t cs = (size_t)gamma * E;
+    for (int base = 0; base < E * split; base += kRefineThreads) {  // one trip when split == 2
+      const int idx = base + tid;
+      const bool act = idx < E * split;
+      const int e = act ? idx / split : 0, half = idx % split;
+      const float* pp = part + (size_t)t * E + e;
+      float sum = 0.f;
+      int c = act ? half : n_slices;
+      for (; c + 15 * split < n_slices; c += 16 * split) {
+        float v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = __ldg(pp + (size_t)(c + i * split) * cs);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sum += v[i];
+      }
+      for (; c < n_slices; c += split) sum += __ldg(pp + (size_t)c * cs);
+      if (split == 2) sum += __shfl_xor_sync(0xffffffffu, sum, 1);  // all lanes reach this point
+      if (act && half == 0) l32[e] = sum;
+    }
+  }
+  MOEV_RT_MARK(2);
   x2 = warp_sum(x2);
   w2 = warp_sum(w2);
   if (lane == 0) { redf[warp] = x2; redw[warp] = w2; }
+  __syncthreads();  // l32, redf, redw complete
+  // ---- fp32 top-k by counting: the k-th largest logit is the one preceded by exactly k - 1 others
+  // (larger value, or equal value and lower id); E <= kRefineThreads
+  if (2 * E <= kRefineThreads) {  // two threads per expert, each counts over half of the experts
+    const int e = tid >> 1, hf = tid & 1;
+    const bool act = e < E;
+    const float v = act ? l32[e] : 0.f;
+    int rank = 0;
+    if (act)
+      for (int e2 = hf * (E / 2); e2 < (hf ? E : E / 2); ++e2) {
+        const float u = l32[e2];
+        rank += (u > v || (u == v && e2 < e)) ? 1 : 0;
+      }
+    rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+    if (act && hf == 0 && rank == k - 1) kth_s = v;
+  } else if (tid < E) {
+    const float v = l32[tid];
+    int rank = 0;
+    for (int e2 = 0; e2 < E; ++e2) {
+      const float u = l32[e2];
+      rank += (u > v || (u == v && e2 < tid)) ? 1 : 0;
+    }
+    if (rank == k - 1) kth_s = v;
+  }
   __syncthreads();
-  if (warp == 0) {
+  {
     float xs = 0.f, wm = 0.f;
     for (int w = 0; w < kRefineWarps; ++w) { xs += redf[w]; wm += redw[w]; }
     // |fp32 logit - exact| <= gamma_n * sum|x w| <= n u ||x|| ||w||, n = roundings on the longest path
     // (slice length + number of slices + the norm sums' own error, covered by the factor 1.25)
     const float n_round = (float)(ks + n_slices + 4);
     const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
-    // ---- fp32 top-k: value of the k-th largest logit
-    constexpr int PL = kMaxE / 32;
-    float v[PL];
-    uint32_t taken = 0;
-#pragma unroll
-    for (int i = 0; i < PL; ++i) {
-      int e = i * 32 + lane;
-      if (e < E) v[i] = l32[e];
-      else { v[i] = 0.f; taken |= 1u << i; }
-    }
-    float kth = 0.f;
-    for (int j = 0; j < k; ++j) {
-      float bv = 0.f;
-      int be = 0x7fffffff;
-#pragma unroll
-      for (int i = 0; i < PL; ++i)
-        if (!((taken >> i) & 1u) && (be == 0x7fffffff || v[i] > bv)) { bv = v[i]; be = i * 32 + lane; }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        int oe = __shfl_xor_sync(0xffffffffu, be, o);
-        bool better = (oe != 0x7fffffff) && (be == 0x7fffffff || ov > bv || (ov == bv && oe < be));
-        if (better) { bv = ov; be = oe; }
-      }
-      if ((be & 31) == lane) taken |= 1u << (be >> 5);
-      kth = bv;
-    }
-    // ---- candidates: every expert whose exact logit may be >= the exact k-th largest
-    const float thr = kth - 2.f * eps;
-    int n = 0;
-    for (int e0 = 0; e0 < E; e0 += 32) {
-      int e = e0 + lane;
-      bool in = e < E && l32[e] >= thr;
-      uint32_t m = __ballot_sync(0xffffffffu, in);
-      if (in) cand[n + __popc(m & ((1u << lane) - 1u))] = e;
-      n += __popc(m);
-    }
-    if (lane == 0) ncand_s = n;
+    // ---- candidates: every expert whose exact logit may be >= the exact k-th largest, in ascending id
+    const float thr = kth_s - 2.f * eps;
+    const bool in = tid < E && l32[tid] >= thr;
+    const uint32_t m = __ballot_sync(0xffffffffu, in);
+    if (lane == 0) wcnt_s[warp] = __popc(m);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < kRefineWarps; ++w) { const int cw = wcnt_s[w]; before += w < warp ? cw : 0; total += cw; }
+    if (in) cand[before + __popc(m & ((1u << lane) - 1u))] = tid;
+    if (tid == 0) ncand_s = total;
   }
   __syncthreads();
   const int ncand = ncand_s;
@@ -332,6 +363,17 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     __syncthreads();
   }
   MOEV_RT_MARK(4);
+  // ---- exact ranking by counting: candidate c is preceded by every candidate with a larger
+  // logit and, at equal logits, by those with a lower id (candidates are stored in ascending id)
+  for (int c = tid; c < ncand; c += kRefineThreads) {
+    const double v = L[c];
+    int rank = 0;
+    for (int c2 = 0; c2 < ncand; ++c2) {
+      const double u = L[c2];
+      rank += (u > v || (u == v && c2 < c)) ? 1 : 0;
+    }
+    if (rank < k) { sel_v_s[rank] = v; sel_e_s[rank] = cand[c]; }
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
   if (lane == 0) redf[warp] = amax;
@@ -383,48 +425,27 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
       T.tok_scale[t] = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
     }
-    double sel_v = 0.0;
-    int sel_e = -1;
-    // candidates are stored in ascending id; lane owns candidates lane, lane+32, ...
-    uint32_t taken = 0;  // bit i: candidate lane + 32 i already selected (ncand <= 512 -> 16 bits)
-    for (int j = 0; j < k; ++j) {
-      double bv = 0.0;
-      int be = 0x7fffffff, bi = -1;
-      for (int i = 0; lane + 32 * i < ncand; ++i) {
-        if ((taken >> i) & 1u) continue;
-        double val = L[lane + 32 * i];
-        int e = cand[lane + 32 * i];
-        if (be == 0x7fffffff || val > bv) { bv = val; be = e; bi = i; }
-      }
-      double wv = bv;
-      int we = be;
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        double ov = __shfl_xor_sync(0xffffffffu, wv, o);
-        int oe = __shfl_xor_sync(0xffffffffu, we, o);
-        bool better = (oe != 0x7fffffff) && (we == 0x7fffffff || ov > wv || (ov == wv && oe < we));
-        if (better) { wv = ov; we = oe; }
-      }
-      if (we == be && bi >= 0) taken |= 1u << bi;
-      if (lane == j) { sel_v = wv; sel_e = we; }
-    }
-    double wgt = 0.0;
+    // router weights of the k selected experts (lane j owns the j-th); binary32 is ample for
+    // weights that are compared to 1e-5: the differences are formed in fp64 first
+    const double sel_v = lane < k ? sel_v_s[lane] : 0.0;
+    const int sel_e = lane < k ? sel_e_s[lane] : -1;
+    float wgt = 0.f;
     if (score == MOEV_SCORE_SOFTMAX) {
-      double mx = __shfl_sync(0xffffffffu, sel_v, 0);
-      double ex = lane < k ? exp(sel_v - mx) : 0.0;
-      double den = warp_sum(ex);
+      const double mx = sel_v_s[0];
+      const float ex = lane < k ? expf((float)(sel_v - mx)) : 0.f;
+      const float den = warp_sum(ex);
       wgt = ex / den;
     } else {
-      double sg = lane < k ? 1.0 / (1.0 + exp(-sel_v)) : 0.0;
-      double den = warp_sum(sg);
-      wgt = (double)routed_scale * sg / (den + 1e-20);
+      const float sg = lane < k ? 1.f / (1.f + expf((float)(-sel_v))) : 0.f;
+      const float den = warp_sum(sg);
+      wgt = routed_scale * sg / (den + 1e-20f);
     }
     if (lane < k) {
       int a = t * k + lane;
       T.topk_ids[a] = sel_e;
-      T.topk_w[a] = (float)wgt;
+      T.topk_w[a] = wgt;
       if (O.topk_ids) O.topk_ids[a] = sel_e;
-      if (O.topk_w) O.topk_w[a] = (float)wgt;
+      if (O.topk_w) O.topk_w[a] = wgt;
     }
   }
   MOEV_RT_MARK(6);
