@@ -43,6 +43,8 @@ struct Tables {
   Unit* units;         // [max_units]
   int32_t* n_units;    // [1]
   int32_t* task_counter; // [1] dynamic task scheduler of the tensor-core FFN, zeroed per call
+  int32_t* wide;         // [1] 1 = the call has many tokens per expert: the two-phase FFN kernel runs it (else 0), or null
+  int32_t* unit_done;    // [max_units] per-unit progress counters of the two-phase kernel, zeroed per call, or null
   int32_t* status;     // [1]   kStatusOk / kStatusTimeout
 };
 

@@ -41,6 +41,29 @@
 #include "ptx.cuh"
 
 namespace moev {
+namespace tcw {  // two-phase schedule for calls with many tokens per expert (ffn_tc_wide.cuh)
+struct Params {
+  const Unit* units;
+  const int32_t* n_units;
+  int32_t* task_counter;
+  const int32_t* slot_token;
+  const float* slot_w;
+  const float* tok_scale;
+  const void* x;
+  float* y32;
+  const float *s_gate, *s_up, *s_down;
+  const float *sh_s_gate, *sh_s_up, *sh_s_down;
+  int32_t* status;
+  int32_t gamma, H, I, A;
+  const int32_t* wide;   // [1] written by the grouping kernel: non-zero = this kernel does the work
+  int32_t* unit_done;    // [max_units] phase-1 tasks finished per unit (zeroed by the grouping kernel)
+  uint8_t* hq;           // [max_units][n_slices][64 rows][128 B]: rows 2r / 2r + 1 = hi / lo codes of token r
+  float* hq_f;           // [max_units][n_slices][32]: routing weight * 2^(e_r - 6) of the tile's tokens
+};
+__device__ void wide_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
+                          const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up, const CUtensorMap& tm_sh_down,
+                          const CUtensorMap& tm_hq, const Params& P, uint32_t tmem);
+}  // namespace tcw
 namespace tc {
 
 constexpr int kThreads = 352;  // 11 warps
@@ -70,6 +93,7 @@ struct Params {
   const float *sh_s_gate, *sh_s_up, *sh_s_down;  // fp8 block scales (shared)
   int32_t* status;
   int32_t gamma, H, I, A;
+  const int32_t* wide;  // non-null and non-zero: the two-phase kernel (ffn_tc_wide.cuh) runs this call, this one exits
 #ifdef MOEV_TC_STATS
   unsigned long long* stats;  // [grid][16] cycles the MMA thread spent per wait / issue class (debug builds)
 #endif
@@ -197,7 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_constant__ CUtensorMap tm_up,
                       const __grid_constant__ CUtensorMap tm_down, const __grid_constant__ CUtensorMap tm_sh_gate,
                       const __grid_constant__ CUtensorMap tm_sh_up, const __grid_constant__ CUtensorMap tm_sh_down,
-                      const Params P) {
+                      const __grid_constant__ CUtensorMap tm_hq, const Params P, const __grid_constant__ tcw::Params W) {
   using F = Fmt<WFMT>;
   constexpr bool kFp8 = WFMT == MOEV_W_FP8E4M3_B128;
   constexpr int TPS = F::kDownTilesPerStage;
@@ -244,6 +268,20 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n_units = *P.n_units;
+  if constexpr (WFMT == MOEV_W_FP8E4M3_B128) {
+    if (P.wide && *P.wide) {
+      // many tokens per streamed expert: the two-phase schedule takes the call (same TMEM, its own barriers)
+      tcw::wide_body(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_hq,
+                     W, tmem);
+      ptx::tc_fence_before();
+      __syncthreads();
+      if (warp == 0) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, kTmemCols);
+      }
+      return;
+    }
+  }
   const int n_ids = n_units * ((n_slices + 1) & ~1);
   volatile int* abortp = &S.abort_flag;
 

@@ -8,6 +8,7 @@
 #include "ffn_simt.cuh"
 #include "ffn_tc.cuh"
 #include "ffn_tc_mx.cuh"
+#include "ffn_tc_wide.cuh"
 #include "router.cuh"
 #include "select.cuh"
 
@@ -46,6 +47,10 @@ struct moev_ctx {
   int32_t* host_word = nullptr;  // pinned scratch for status / n_active reads
   TmapSet tmaps[kTmapCache];
   int tmap_next = 0;
+  bool wide_ok = false;   // block-scaled fp8 on tensor cores: the two-phase kernel for many tokens per expert exists
+  uint8_t* hq = nullptr;  // its scratch: quantised h tiles [max_units][n_slices][64][128] ...
+  float* hq_f = nullptr;  // ... and their scales [max_units][n_slices][32]
+  CUtensorMap tm_hq;
   CUtensorMap tm_xq;  // MXFP4 tensor-core path: the [2 * max_tokens, xq_stride] byte array T.xq, box 128 x 2
   int n_sm = 0;
   int unit_cap = 1 << 20;
@@ -111,6 +116,8 @@ cudaError_t dmalloc(T** p, size_t count) {
 }
 
 bool route_use_bitmap(const moev_config& c, int gamma) { return route_bitmap_bytes(c.E, gamma) <= kRouteBitmapBudget; }
+// assignments per streamed expert above which the two-phase FFN kernel takes the call
+constexpr int kWideRatio = 8;
 size_t route_smem(const moev_config& c, int gamma) {
   return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + (route_use_bitmap(c, gamma) ? route_bitmap_bytes(c.E, gamma) : 0);
 }
@@ -237,9 +244,20 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.stats = c->tc_stats;
 #endif
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
+  P.wide = c->wide_ok ? c->T.wide : nullptr;
+  // arguments of the two-phase schedule, which the kernel switches to when the grouping kernel's
+  // flag says that the call has many tokens per streamed expert (fp8 only)
+  tcw::Params W{};
+  W.units = P.units; W.n_units = P.n_units; W.task_counter = P.task_counter; W.slot_token = P.slot_token;
+  W.slot_w = P.slot_w; W.tok_scale = P.tok_scale; W.x = x; W.y32 = P.y32;
+  W.s_gate = P.s_gate; W.s_up = P.s_up; W.s_down = P.s_down;
+  W.sh_s_gate = P.sh_s_gate; W.sh_s_up = P.sh_s_up; W.sh_s_down = P.sh_s_down;
+  W.status = P.status; W.gamma = gamma; W.H = g.H; W.I = g.I; W.A = P.A;
+  W.wide = c->T.wide; W.unit_done = c->T.unit_done; W.hq = c->hq; W.hq_f = c->hq_f;
   launch_k(tc::grouped_ffn_tc_kernel<WFMT>, dim3(c->n_sm), dim3(tc::kThreads), tc::kSmemBytes, st, ev == nullptr,
-           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], P);
+           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], c->wide_ok ? c->tm_hq : tm->map[0], P, W);
   if (ev) cudaEventRecord(ev[4], st);
+  if (ev) cudaEventRecord(ev[5], st);
 }
 
 void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const void* x, int gamma, cudaStream_t st,
@@ -341,6 +359,26 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     const size_t cap = c->unit_cap;
     const size_t max_units = E + A / cap + (size_t)cfg->n_shared * (G / cap + 1) + 8;
     ok = ok && dmalloc(&c->T.units, max_units) == cudaSuccess;
+    const int n_slices = cfg->I / 128;
+    c->wide_ok = c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_FP8E4M3_B128 && n_slices <= tcw::kMaxSlices;
+    if (c->wide_ok) {
+      ok = ok && dmalloc(&c->T.wide, 1) == cudaSuccess;
+      ok = ok && dmalloc(&c->T.unit_done, max_units) == cudaSuccess;
+      ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->hq), max_units * (size_t)n_slices * 8192) == cudaSuccess;
+      ok = ok && dmalloc(&c->hq_f, max_units * (size_t)n_slices * tcw::kMC) == cudaSuccess;
+      EncodeTiledFn fn = encode_tiled_fn();
+      if (ok && fn) {
+        cuuint64_t dims[2] = {128, (cuuint64_t)(max_units * (size_t)n_slices * 64)};
+        cuuint64_t strides[1] = {128};
+        cuuint32_t box[2] = {128, 64};
+        cuuint32_t estr[2] = {1, 1};
+        ok = fn(&c->tm_hq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c->hq, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+      } else {
+        ok = false;
+      }
+    }
   }
   if (c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_MXFP4) {
     // quantised activations (two e4m3 terms per element), loaded by TMA as the MMA's N operand
@@ -407,6 +445,7 @@ moev_status moev_destroy(moev_ctx* c) {
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
   cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->T.task_counter); cudaFree(c->hbuf); cudaFree(c->y32);
+  cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f);
   cudaFree(c->x_stage); cudaFree(c->y_stage);
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)
@@ -483,7 +522,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
              g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale);
   if (ev) cudaEventRecord(ev[2], st);
   launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
-           g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma));
+           g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma), c->wide_ok ? kWideRatio : 0);
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);

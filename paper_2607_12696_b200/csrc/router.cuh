@@ -459,7 +459,8 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
 inline size_t route_bitmap_bytes(int E, int gamma) { return (size_t)E * ((gamma + 31) / 32) * 4; }
 constexpr size_t kRouteBitmapBudget = 96 * 1024;
 __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O, int gamma, int E,
-                                                           int k, int n_shared, int unit_cap, int use_bitmap) {
+                                                           int k, int n_shared, int unit_cap, int use_bitmap,
+                                                           int wide_ratio) {
   extern __shared__ int32_t sm[];
   const int A = gamma * k;
   int32_t* cnt = sm;
@@ -546,7 +547,18 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       un.m = min(unit_cap, m - c * unit_cap); un.shared = shared;
       T.units[first + c] = un;
     }
-    if (tid == blockDim.x - 1) { *T.n_units = base + sc; *T.task_counter = 0; }
+    if (tid == blockDim.x - 1) {
+      *T.n_units = base + sc;
+      *T.task_counter = 0;
+      // many tokens per streamed expert: the two-phase FFN schedule (wide_ratio = 0: not available)
+      if (T.wide) *T.wide = (wide_ratio > 0 && (A + n_shared * gamma) > wide_ratio * (U + n_shared)) ? 1 : 0;
+    }
+    if (T.unit_done) {
+      __shared__ int n_units_s;
+      if (tid == blockDim.x - 1) n_units_s = base + sc;
+      __syncthreads();
+      for (int i = tid; i < n_units_s; i += blockDim.x) T.unit_done[i] = 0;
+    }
   }
 
   MOEV_RT_MARK(11);
