@@ -44,7 +44,7 @@ struct Tables {
   int32_t* n_units;    // [1]
   int32_t* task_counter; // [1] dynamic task scheduler of the tensor-core FFN, zeroed per call
   int32_t* wide;         // [1] 1 = the call has many tokens per expert: the two-phase FFN kernel runs it (else 0), or null
-  int32_t* unit_done;    // [max_units] per-unit progress counters of the two-phase kernel, zeroed per call, or null
+  int32_t* unit_done;    // [2 * max_units] per-unit progress counters, then per-unit gather flags, of the two-phase schedule; zeroed per call; or null
   int32_t* status;     // [1]   kStatusOk / kStatusTimeout
 };
 

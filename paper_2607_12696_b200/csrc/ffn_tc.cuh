@@ -56,13 +56,15 @@ struct Params {
   int32_t* status;
   int32_t gamma, H, I, A;
   const int32_t* wide;   // [1] written by the grouping kernel: non-zero = this kernel does the work
-  int32_t* unit_done;    // [max_units] phase-1 tasks finished per unit (zeroed by the grouping kernel)
+  int32_t* unit_done;    // [2 * max_units], zeroed by the grouping kernel: [u] phase-1 tasks finished of unit u; [n_units + u] 1 once xu[u] is complete
   uint8_t* hq;           // [max_units][n_slices][64 rows][128 B]: rows 2r / 2r + 1 = hi / lo codes of token r
   float* hq_f;           // [max_units][n_slices][32]: routing weight * 2^(e_r - 6) of the tile's tokens
+  const uint8_t* xq;     // [gamma][2][H] e4m3 hi / lo terms of x * tok_scale (written by the routing kernels)
+  uint8_t* xu;           // [max_units][H / 128][64 rows][128 B]: the unit's tokens' rows of xq, one tile per K chunk
 };
 __device__ void wide_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
                           const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up, const CUtensorMap& tm_sh_down,
-                          const CUtensorMap& tm_hq, const Params& P, uint32_t tmem);
+                          const CUtensorMap& tm_hq, const CUtensorMap& tm_xu, const Params& P, uint32_t tmem);
 }  // namespace tcw
 namespace tc {
 
@@ -221,7 +223,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_constant__ CUtensorMap tm_up,
                       const __grid_constant__ CUtensorMap tm_down, const __grid_constant__ CUtensorMap tm_sh_gate,
                       const __grid_constant__ CUtensorMap tm_sh_up, const __grid_constant__ CUtensorMap tm_sh_down,
-                      const __grid_constant__ CUtensorMap tm_hq, const Params P, const __grid_constant__ tcw::Params W) {
+                      const __grid_constant__ CUtensorMap tm_hq, const __grid_constant__ CUtensorMap tm_xu, const Params P,
+                      const __grid_constant__ tcw::Params W) {
   using F = Fmt<WFMT>;
   constexpr bool kFp8 = WFMT == MOEV_W_FP8E4M3_B128;
   constexpr int TPS = F::kDownTilesPerStage;
@@ -271,8 +274,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   if constexpr (WFMT == MOEV_W_FP8E4M3_B128) {
     if (P.wide && *P.wide) {
       // many tokens per streamed expert: the two-phase schedule takes the call (same TMEM, its own barriers)
-      tcw::wide_body(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_hq,
-                     W, tmem);
+      tcw::wide_body(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_hq, tm_xu, W, tmem);
       ptx::tc_fence_before();
       __syncthreads();
       if (warp == 0) {

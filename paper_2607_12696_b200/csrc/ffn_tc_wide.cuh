@@ -1,26 +1,34 @@
-// Tensor-core grouped expert FFN for block-scaled FP8 weights when experts receive MANY tokens
-// (batched verification, few experts shared by all tokens).  Same roles, rings and primitives
-// as ffn_tc.cuh, different schedule.
+// Grouped expert FFN for block-scaled FP8 weights when experts receive MANY tokens (batched
+// verification, few experts shared by all tokens): the two-phase schedule.  Same rings and
+// primitives as ffn_tc.cuh, whose kernel calls wide_body() after its prologue when the flag
+// written by the grouping kernel says that the call has many tokens per streamed expert (one
+// launch per call either way; TMEM is allocated and released by the caller).
 //
-// Why.  ffn_tc.cuh splits the down projection over the 128-wide slices of I, so every task
-// reduce-adds a full [H x m] fp32 tile into the output accumulator: n_slices * A * H * 4 bytes
-// of global reductions per call.  With 2-3 tokens per expert that hides under the weight
-// stream; with 32 tokens per unit the reductions bound the kernel.  Here a unit's work is cut
-// into two kinds of tasks:
-//   phase 1  (unit, slice of I):   gate/up GEMM + SwiGLU exactly as in ffn_tc.cuh, but the
-//            quantised h tile (two e4m3 terms per value, per-token power-of-two scale) goes to
-//            a global scratch array instead of shared memory;
-//   phase 2  (unit, pair of 128-row tiles of H):  streams W_down[tiles, :] (whole rows) and the
-//            unit's h tiles slice by slice, one tensor-core product per (tile, slice), and
-//            accumulates scale * product over all slices in REGISTERS (the 128 x 128 block scale
-//            and the h scale differ per slice, so the sum cannot stay in TMEM); one reduction
-//            per (token, row) at the end: n_slices times fewer global reductions.
+// Why.  ffn_tc.cuh (a) folds the 128 x 128 block scale into the activation operand, which
+// re-quantises the unit's tokens for every (slice, K chunk), and (b) splits the down projection
+// over the 128-wide slices of I, so that every task reduce-adds a full [H x m] fp32 tile into the
+// output accumulator: n_slices * A * H * 4 bytes of global reductions per call.  With 2-3 tokens
+// per expert both hide under the weight stream; with 32 tokens per unit they bound the kernel
+// (conversion throughput and L2 reduction throughput).  Here
+//   * the activation operand is quantised ONCE per token (two e4m3 terms of x * 2^p_t, written
+//     by the routing kernels); at the start every CTA copies the rows of some units' tokens into
+//     per-unit operand tiles (one [64 x 128 B] tile per K chunk), which phase 1 then loads with
+//     one TMA copy per stage; every K chunk's product goes to a TMEM partial
+//     buffer and the epilogue warps add  block scale * partial  into REGISTER accumulators
+//     (gate: warps 2..5, up: warps 6..9 -- there are no activation producers);
+//   * a unit's work is cut into two kinds of tasks:
+//       phase 1 (unit, slice of I):  gate/up + SwiGLU; the quantised h tile (two e4m3 terms per
+//               value, per-token power-of-two scale) goes to a global scratch array;
+//       phase 2 (unit, pair of 128-row tiles of H):  streams W_down[tiles, :] (whole rows) and
+//               the unit's h tiles slice by slice, one product per (tile, slice) into a TMEM
+//               partial buffer, and adds  block scale * h scale * partial  in registers; one
+//               global reduction per (token, row) at the end: n_slices times fewer.
+//     Both phases run the same stage loop (weight tiles + operand tile by TMA, four MMAs per
+//     issuer, partial buffer handed to the two epilogue groups); they differ in what is loaded,
+//     the scale factors and the end of the task.
 // Task ids put every phase-1 task before every phase-2 task, phase-1 tasks unit-major.  A CTA
 // that draws a phase-2 task waits (bounded) until the unit's phase-1 tasks have all finished:
 // those were drawn earlier by CTAs that never wait on another CTA, so the wait always ends.
-// This is not a kernel of its own: ffn_tc.cuh's kernel calls wide_body() after its prologue when
-// the flag written by the grouping kernel says that the call has many tokens per streamed
-// expert (one launch per call either way; TMEM is allocated by the caller).
 #pragma once
 #include <cuda.h>
 
@@ -34,44 +42,40 @@ namespace tcw {
 using tc::kStageBytes;
 using tc::kTaskQ;
 using tc::kWaitBudgetNs;
-using tc::sw128;
 using tc::warp_wait;
 using tc::group_sync;
 using tc::safe_exponent;
 using tc::pow2i;
 
-constexpr int kThreads = 352;  // warps: 0 TMA + scheduler, 1 and 10 MMA issuers, 2..5 epilogue, 6..9 activation producers
+constexpr int kThreads = 352;  // warps: 0 TMA + scheduler, 1 and 10 MMA issuers, 2..5 epilogue group 0, 6..9 group 1
 constexpr int kStages = 5;
-constexpr int kBSlots = 3;                 // phase 1: activation-operand ring, 16 KB slots (gate | up)
-constexpr int kBSlotBytes = 16 * 1024;
-constexpr int kHqTileBytes = 8 * 1024;     // phase 2: one [64 x 128 B] h tile per weight-ring stage (same area)
+constexpr int kBTileBytes = 8 * 1024;      // operand tile of a stage: [64 rows x 128 B], rows 2r / 2r + 1 = hi / lo of token r
 constexpr int kMC = 32;                    // tokens per unit
 constexpr int kMaxSlices = 32;             // I <= 4096 (larger layers keep the ffn_tc.cuh schedule)
-constexpr int kTmemCols = 512;             // G 64 | P 64 | O[2 stage buffers][2 tiles] 64 each
-constexpr int kTileBytes = kStages * kStageBytes + kBSlots * kBSlotBytes;
+constexpr int kMaxChunks = 128;            // H <= 16384
+constexpr int kGath = 8;                   // pieces a unit's operand tiles are gathered in (K ranges)
+constexpr int kColXchg = 256;              // TMEM: partial buffers 2 x (64 | 64) | 32 columns to hand P to the gate group
+constexpr int kTileBytes = kStages * kStageBytes + kStages * kBTileBytes;
 constexpr int kCtlBytes = 12 * 1024;
 constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
-static_assert(kStages * kHqTileBytes <= kBSlots * kBSlotBytes, "phase-2 h tiles fit the activation ring");
 static_assert(kSmemBytes <= tc::kSmemBytes && kThreads == tc::kThreads, "runs inside the launch of ffn_tc.cuh's kernel");
 
 struct Smem {
   uint64_t w_full[kStages], w_empty[kStages];
-  uint64_t b_full[kBSlots], b_empty[kBSlots];
-  uint64_t acc_full, acc_empty;
-  uint64_t d_full[2], d_empty[2];
+  uint64_t p_full[2], p_empty[2];      // TMEM partial buffers: MMA issuers -> both epilogue groups
+  uint64_t x_full, x_empty;            // P values of a phase-1 task: group 1 -> group 0
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
-  uint64_t ep_bar;
+  uint64_t ep_bar;                     // barrier of group 0 (128 threads)
+  uint64_t all_bar;                    // barrier of both groups (256 threads)
   volatile int32_t tq_task[kTaskQ];
   volatile int abort_flag;
-  int32_t p_tok[2][kMC];
-  float p_tscale[2][kMC];
-  float p_sg[2][128], p_su[2][128];
+  // tables, double-buffered by task parity; every warp writes all entries it reads (identical values)
   int32_t e_tok[2][kMC];
   float e_w[2][kMC];
-  float e_inv[2][kMC];
+  float e_inv[2][kMC];                 // 1 / tok_scale
+  float s_tab[2][2][kMaxChunks];       // [parity][group]: phase 1 block scale per K chunk; phase 2 W_down block scale per slice
+  float f2[2][kMaxSlices][kMC];        // phase 2: [slice][token] h scale * routing weight
   uint32_t e_amax[4][kMC];
-  float e_f2[kMaxSlices][kMC];   // phase 2: [slice][token] h scale * routing weight of the unit's tiles
-  float e_sd2[2][kMaxSlices];    // phase 2: [tile of the pair][slice] W_down block scales
 };
 
 struct Task { int unit, slice, hp; bool phase2; };
@@ -114,32 +118,45 @@ __device__ __forceinline__ bool wait_unit_done(const int32_t* ctr, int target, v
   }
 }
 
+// 32 lanes x 32 consecutive 32-bit columns from registers (lane l of the warp -> its TMEM lane)
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};" ::"r"(taddr),
+      "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]), "f"(v[9]),
+      "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]), "f"(v[18]),
+      "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]),
+      "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+      : "memory");
+}
+
 __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
                                        const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up,
-                                       const CUtensorMap& tm_sh_down, const CUtensorMap& tm_hq, const Params& P,
-                                       uint32_t tmem) {
+                                       const CUtensorMap& tm_sh_down, const CUtensorMap& tm_hq,
+                                       const CUtensorMap& tm_xu, const Params& P, uint32_t tmem) {
   constexpr int WFMT = MOEV_W_FP8E4M3_B128;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* w_ring = base;
-  uint8_t* b_ring = w_ring + kStages * kStageBytes;  // phase 1: kBSlots x 16 KB; phase 2: kStages x 8 KB h tiles
+  uint8_t* b_tiles = w_ring + kStages * kStageBytes;
   static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
   Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int H = P.H, I = P.I;
-  const int KC = H / 128;           // K chunks of the gate/up phase
+  const int KC = H / 128;           // K chunks of the gate/up phase = stages of a phase-1 task
   const int HT = H / 128;           // 128-row tiles of W_down
-  const int n_slices = I / 128;
+  const int n_slices = I / 128;     // stages of a phase-2 task
   const int n_hp = (HT + 1) / 2;    // phase-2 tasks per unit: pairs of H tiles
 
+  __syncthreads();  // every thread has left the caller's use of shared memory
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
-    for (int i = 0; i < kBSlots; ++i) { ptx::mbar_init(&S.b_full[i], 128); ptx::mbar_init(&S.b_empty[i], 2); }
-    ptx::mbar_init(&S.acc_full, 2); ptx::mbar_init(&S.acc_empty, 128);
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 128); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 256); }
+    ptx::mbar_init(&S.x_full, 128); ptx::mbar_init(&S.x_empty, 128);
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
+    ptx::mbar_init(&S.all_bar, 256);
     S.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -151,140 +168,169 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
   const int n_ids = n_units * (n_slices + n_hp);
 #endif
   volatile int* abortp = &S.abort_flag;
+  int32_t* gath_done = P.unit_done + n_units;  // the grouping kernel zeroes 2 * n_units counters: progress, then gather flags
+
+  // ---- operand tiles of the units.  Piece (unit, g) = the K chunks [g KC / kGath, (g + 1) KC / kGath) of the
+  // unit; pieces are dealt round-robin to the CTAs.  Rows 2r / 2r + 1 of the tile of K chunk kc =
+  // bytes [128 kc, 128 kc + 128) of the hi / lo rows of the unit's r-th token.
+  for (int pc = blockIdx.x; pc < n_units * kGath; pc += gridDim.x) {
+    const int un = pc / kGath, g = pc % kGath;
+    const Unit u = P.units[un];
+    const int kc0 = g * KC / kGath, kc1 = (g + 1) * KC / kGath;
+    const int n16 = (kc1 - kc0) * 8;  // 16-byte pieces per row in this K range
+    for (int i = tid; i < u.m * 2 * n16; i += kThreads) {
+      const int rr = i / n16, p16 = kc0 * 8 + i % n16;  // rr = 2 r + (0 hi, 1 lo)
+      const int r = rr >> 1;
+      const int tok = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma) + r) : P.slot_token[u.slot0 + r];
+      const uint4 v = *reinterpret_cast<const uint4*>(P.xq + ((size_t)(2 * tok + (rr & 1)) * H) + (size_t)p16 * 16);
+      const int kc = p16 >> 3;
+      *reinterpret_cast<uint4*>(P.xu + (((size_t)un * KC + kc) * 64 + rr) * 128 + (p16 & 7) * 16) = v;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      asm volatile("fence.proxy.async;" ::: "memory");
+      __threadfence();
+      atomicAdd(gath_done + un, 1);
+    }
+  }
 
   if (warp == 0) {
-    // ===================================================== TMA producer + scheduler (one lane)
+    // ===================================================== TMA producer + scheduler (lane 0 does the work; the
+    // warp stays converged)
     if (lane == 0) {
-      ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down); ptx::prefetch_tmap(&tm_hq);
-      uint32_t it = 0, q = 0;
-      bool ok = true, drained = false;
-      auto fetch_publish = [&]() -> int {
-        int id = atomicAdd(P.task_counter, 1);
+      ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
+      ptx::prefetch_tmap(&tm_hq); ptx::prefetch_tmap(&tm_xu);
+    }
+    uint32_t it = 0, q = 0;
+    bool ok = true;
+    auto fetch_publish = [&]() -> int {  // lane 0 draws and publishes; every lane learns the id
+      int id = -2;
+      if (lane == 0) {
+        id = atomicAdd(P.task_counter, 1);
         if (id >= n_ids) id = -1;
         const int slot = q % kTaskQ;
-        ok = ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-        if (!ok) return -2;
-        S.tq_task[slot] = id;
-        ptx::mbar_arrive(&S.tq_full[slot]);
-        ++q;
-        return id;
-      };
-      int id = fetch_publish();
-      while (ok && id >= 0) {
-        const int id_next = fetch_publish();  // published one task ahead: the other roles prepare their tables
+        if (ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs)) {
+          S.tq_task[slot] = id;
+          ptx::mbar_arrive(&S.tq_full[slot]);
+        } else {
+          id = -2;
+        }
+      }
+      ++q;
+      id = __shfl_sync(0xffffffffu, id, 0);
+      if (id == -2) ok = false;
+      return id;
+    };
+    auto wait_stage = [&](int s) {  // lane 0 waits for the stage to be free; the outcome is warp-uniform
+      int w = 1;
+      if (lane == 0)
+        w = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, w, 0) != 0;
+    };
+    int id = fetch_publish();
+    while (ok && id >= 0) {
+      const int id_next = fetch_publish();  // published one task ahead: the other roles prepare their tables
+      if (!ok) break;
+      const Task t = decode(id, n_units, n_slices, n_hp);
+      const Unit u = P.units[t.unit];
+      if (!t.phase2) {
+        const CUtensorMap* mg = u.shared ? &tm_sh_gate : &tm_gate;
+        const CUtensorMap* mu = u.shared ? &tm_sh_up : &tm_up;
+        int w = 1;
+        if (lane == 0) {  // the unit's operand tiles are complete (another CTA's ordinary stores: acquire + proxy fence)
+          w = wait_unit_done(gath_done + t.unit, kGath, abortp, P.status) ? 1 : 0;
+          asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        ok = __shfl_sync(0xffffffffu, w, 0) != 0;
         if (!ok) break;
-        const Task t = decode(id, n_units, n_slices, n_hp);
-        const Unit u = P.units[t.unit];
-        if (!t.phase2) {
-          const CUtensorMap* mg = u.shared ? &tm_sh_gate : &tm_gate;
-          const CUtensorMap* mu = u.shared ? &tm_sh_up : &tm_up;
-          for (int kc = 0; kc < KC && ok; ++kc, ++it) {
-            const int s = it % kStages;
-            ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            if (!ok) break;
+        for (int kc = 0; kc < KC && ok; ++kc, ++it) {
+          const int s = it % kStages;
+          wait_stage(s);
+          if (!ok) break;
+          if (lane == 0) {
             uint8_t* dst = w_ring + s * kStageBytes;
-            ptx::mbar_arrive_expect_tx(&S.w_full[s], kStageBytes);
+            ptx::mbar_arrive_expect_tx(&S.w_full[s], kStageBytes + kBTileBytes);
             ptx::tma_load_3d(dst, mg, &S.w_full[s], kc * 128, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
             ptx::tma_load_3d(dst + 16384, mu, &S.w_full[s], kc * 128, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
-          }
-        } else {
-          const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
-          // the unit's h tiles must be complete (written by other CTAs with ordinary stores, read
-          // here by the TMA unit: acquire, then a cross-proxy fence)
-          ok = wait_unit_done(P.unit_done + t.unit, n_slices, abortp, P.status);
-          if (!ok) break;
-          asm volatile("fence.proxy.async;" ::: "memory");
-          if (!drained) {
-            // The h tiles of phase 2 reuse the shared memory of phase 1's activation ring.  Ids
-            // are monotonic (phase 1 first), so a CTA changes over once: let every MMA of its
-            // phase-1 tasks finish first (all outstanding ring stages consumed).
-            for (uint32_t j = it > (uint32_t)kStages ? it - kStages : 0; j < it && ok; ++j)
-              ok = ptx::bounded_wait(&S.w_empty[j % kStages], (j / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            if (!ok) break;
-            drained = true;
-          }
-          const int nt = (2 * t.hp + 1 < HT) ? 2 : 1;
-          for (int sl = 0; sl < n_slices && ok; ++sl, ++it) {
-            const int s = it % kStages;
-            ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            if (!ok) break;
-            uint8_t* dst = w_ring + s * kStageBytes;
-            ptx::mbar_arrive_expect_tx(&S.w_full[s], 16384 * nt + kHqTileBytes);
-            ptx::tma_load_3d(dst, md, &S.w_full[s], sl * 128, (2 * t.hp) * 128, u.expert, ptx::kPolicyEvictFirst);
-            if (nt == 2)
-              ptx::tma_load_3d(dst + 16384, md, &S.w_full[s], sl * 128, (2 * t.hp + 1) * 128, u.expert, ptx::kPolicyEvictFirst);
-            ptx::tma_load_2d(b_ring + s * kHqTileBytes, &tm_hq, &S.w_full[s], 0, (t.unit * n_slices + sl) * 64,
+            ptx::tma_load_2d(b_tiles + s * kBTileBytes, &tm_xu, &S.w_full[s], 0, (t.unit * KC + kc) * 64,
                              ptx::kPolicyEvictNormal);
           }
         }
-        id = id_next;
+      } else {
+        const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
+        // the unit's h tiles must be complete (written by other CTAs with ordinary stores, read
+        // here by the TMA unit: acquire, then a cross-proxy fence)
+        int w = 1;
+        if (lane == 0) {
+          w = wait_unit_done(P.unit_done + t.unit, n_slices, abortp, P.status) ? 1 : 0;
+          asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        ok = __shfl_sync(0xffffffffu, w, 0) != 0;
+        if (!ok) break;
+        const int nt = (2 * t.hp + 1 < HT) ? 2 : 1;
+        for (int sl = 0; sl < n_slices && ok; ++sl, ++it) {
+          const int s = it % kStages;
+          wait_stage(s);
+          if (!ok) break;
+          if (lane == 0) {
+            uint8_t* dst = w_ring + s * kStageBytes;
+            ptx::mbar_arrive_expect_tx(&S.w_full[s], 16384 * nt + kBTileBytes);
+            ptx::tma_load_3d(dst, md, &S.w_full[s], sl * 128, (2 * t.hp) * 128, u.expert, ptx::kPolicyEvictFirst);
+            if (nt == 2)
+              ptx::tma_load_3d(dst + 16384, md, &S.w_full[s], sl * 128, (2 * t.hp + 1) * 128, u.expert, ptx::kPolicyEvictFirst);
+            ptx::tma_load_2d(b_tiles + s * kBTileBytes, &tm_hq, &S.w_full[s], 0, (t.unit * n_slices + sl) * 64,
+                             ptx::kPolicyEvictNormal);
+          }
+        }
       }
+      id = id_next;
     }
   } else if (warp == 1 || warp == 10) {
-    // ===================================================== MMA issuers (one lane each)
-    const int issuer = warp == 1 ? 0 : 1;  // 0: gate chain / first tile of the pair, 1: up chain / second tile
+    // ===================================================== MMA issuers (one lane each): issuer 0 = gate tile /
+    // first H tile -> columns 0..63 of the partial buffer, issuer 1 = up tile / second H tile -> columns 64..127
+    const int issuer = warp == 1 ? 0 : 1;
     if (lane == 0) {
-      uint32_t it = 0, bit = 0, p1 = 0, dsc = 0, q = 0;
+      uint32_t it = 0, q = 0;
       bool ok = true;
       const uint32_t w_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(w_ring));
-      const uint32_t b_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(b_ring));
+      const uint32_t b_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(b_tiles));
       for (;;) {
         const int id = next_task(S, q, abortp, P.status, false);
         if (id < 0) break;
         const Task t = decode(id, n_units, n_slices, n_hp);
         const Unit u = P.units[t.unit];
-        const uint32_t N = (uint32_t)((2 * u.m + 15) & ~15);
-        const uint32_t idesc = ptx::instr_desc(0, 0, N);
-        if (!t.phase2) {
-          ok = ptx::bounded_wait(&S.acc_empty, (p1 & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+        const uint32_t idesc = ptx::instr_desc(0, 0, (uint32_t)((2 * u.m + 15) & ~15));
+        const int n_st = t.phase2 ? n_slices : KC;
+        const bool mine = !t.phase2 || issuer == 0 || 2 * t.hp + 1 < HT;  // an odd last H tile has no partner
+        for (int st = 0; st < n_st && ok; ++st, ++it) {
+          const int s = it % kStages, pb = it & 1;
+          ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((it >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
           if (!ok) break;
           ptx::tc_fence_after();
-          const uint32_t dacc = tmem + (issuer ? 64 : 0);
-          for (int kc = 0; kc < KC && ok; ++kc, ++it, ++bit) {
-            const int s = it % kStages, sb = bit % kBSlots;
-            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            ok = ok && ptx::bounded_wait(&S.b_full[sb], (bit / kBSlots) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            if (!ok) break;
-            ptx::tc_fence_after();
-            const uint32_t wa = w_lo0 + s * (kStageBytes >> 4) + (issuer ? 1024 : 0);
-            const uint32_t ba = b_lo0 + sb * (kBSlotBytes >> 4) + (issuer ? 512 : 0);
+          if (mine) {
+            const uint32_t wa = w_lo0 + s * (kStageBytes >> 4) + issuer * 1024;
+            const uint32_t ba = b_lo0 + s * (kBTileBytes >> 4);
+            const uint32_t d = tmem + pb * 128 + issuer * 64;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) tc::issue_mma<WFMT>(dacc, wa + 2 * j, ba + 2 * j, idesc, (kc | j) ? 1u : 0u);
-            ptx::mma_commit(&S.w_empty[s]);
-            ptx::mma_commit(&S.b_empty[sb]);
+            for (int j = 0; j < 4; ++j) tc::issue_mma<WFMT>(d, wa + 2 * j, ba + 2 * j, idesc, j ? 1u : 0u);
           }
-          if (!ok) break;
-          ptx::mma_commit(&S.acc_full);
-          ++p1;
-        } else {
-          const int nt = (2 * t.hp + 1 < HT) ? 2 : 1;
-          for (int sl = 0; sl < n_slices && ok; ++sl, ++dsc, ++it) {
-            const int db = dsc & 1, s = it % kStages;
-            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            ok = ok && ptx::bounded_wait(&S.d_empty[db], ((dsc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-            if (!ok) break;
-            ptx::tc_fence_after();
-            if (issuer < nt) {
-              const uint32_t wa = w_lo0 + s * (kStageBytes >> 4) + issuer * 1024;
-              const uint32_t ha = b_lo0 + s * (kHqTileBytes >> 4);
-              const uint32_t d_part = tmem + 128 + (db * 2 + issuer) * 64;
-#pragma unroll
-              for (int j = 0; j < 4; ++j) tc::issue_mma<WFMT>(d_part, wa + 2 * j, ha + 2 * j, idesc, j ? 1u : 0u);
-            }
-            ptx::mma_commit(&S.d_full[db]);
-            ptx::mma_commit(&S.w_empty[s]);
-          }
-          if (!ok) break;
+          ptx::mma_commit(&S.p_full[pb]);
+          ptx::mma_commit(&S.w_empty[s]);
         }
+        if (!ok) break;
       }
     }
   }
-  else if (warp < 6) {
-    // ===================================================== epilogue warps (TMEM lane quarter = warp % 4)
+  else {
+    // ===================================================== epilogue groups: warps 2..5 = group 0 (gate tile / first
+    // H tile), warps 6..9 = group 1 (up tile / second H tile).  TMEM lane quarter = warp % 4 in both.
+    const int grp = warp >= 6 ? 1 : 0;
     const int qd = warp & 3;
     const uint32_t lane_base = (uint32_t)(qd * 32) << 16;
     const int row = qd * 32 + lane;   // row of the 128-row tile this thread owns
-    uint32_t p1 = 0, dsc = 0, gph = 0, q = 0, tcount = 0;
+    uint32_t it = 0, q = 0, tcount = 0, gph = 0, xph = 0, aph = 0;
     bool ok = true;
     for (;; ++tcount) {
       const int id = next_task(S, q, abortp, P.status, true);
@@ -293,6 +339,10 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
       const Unit u = P.units[t.unit];
       const int m = u.m;
       const int par = tcount & 1;
+      const int n_st = t.phase2 ? n_slices : KC;
+      // ---- tables of this task.  Tasks can be as short as two stages, so the partial-buffer barriers do not
+      // keep a fast warp from running a whole task ahead: every epilogue thread has left the previous task first.
+      if (!(ok = group_sync(&S.all_bar, aph, abortp, P.status))) break;
       for (int r = lane; r < m; r += 32) {
         int tok;
         float w;
@@ -302,247 +352,135 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         S.e_w[par][r] = w;
         S.e_inv[par][r] = 1.f / P.tok_scale[tok];
       }
+      bool have_tile = true;  // phase 2: does this group's H tile exist
       if (!t.phase2) {
-        // ---------------- phase 1: SwiGLU of the slice, h tile and its scales to the scratch arrays
-        const int slice = t.slice;
-        const float* sg = (u.shared ? P.sh_s_gate : P.s_gate) + ((size_t)u.expert * n_slices + slice) * KC;
-        const float* su = (u.shared ? P.sh_s_up : P.s_up) + ((size_t)u.expert * n_slices + slice) * KC;
-        float mg = 0.f, mu = 0.f;
-        for (int kc = lane; kc < KC; kc += 32) { mg = fmaxf(mg, fabsf(__ldg(sg + kc))); mu = fmaxf(mu, fabsf(__ldg(su + kc))); }
-        mg = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mg)));
-        mu = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mu)));
-        const float ig = pow2i(safe_exponent(mg)), iu = pow2i(safe_exponent(mu));
-        __syncwarp();
-        ok = warp_wait(&S.acc_full, p1 & 1, abortp, P.status);
+        const float* sc = grp ? (u.shared ? P.sh_s_up : P.s_up) : (u.shared ? P.sh_s_gate : P.s_gate);
+        sc += ((size_t)u.expert * n_slices + t.slice) * KC;
+        for (int kc = lane; kc < KC; kc += 32) S.s_tab[par][grp][kc] = __ldg(sc + kc);
+      } else {
+        ok = wait_unit_done(P.unit_done + t.unit, n_slices, abortp, P.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const int ht = 2 * t.hp + grp;
+        have_tile = ht < HT;
+        const float* sd = u.shared ? P.sh_s_down : P.s_down;
+        for (int sl = lane; sl < n_slices; sl += 32)
+          S.s_tab[par][grp][sl] = have_tile ? __ldg(sd + ((size_t)u.expert * HT + ht) * n_slices + sl) : 0.f;
+        for (int i = lane; i < n_slices * kMC; i += 32) {
+          const int sl = i / kMC, r = i % kMC;
+          S.f2[par][sl][r] = r < m ? __ldcg(P.hq_f + ((size_t)t.unit * n_slices + sl) * kMC + r) : 0.f;
+        }
+      }
+      __syncwarp();
+
+      // ---- stage loop: acc[r] += factor * (hi + lo / 16) of this group's 64 partial columns
+      float acc[kMC];
+#pragma unroll
+      for (int r = 0; r < kMC; ++r) acc[r] = 0.f;
+      for (int st = 0; st < n_st && ok; ++st, ++it) {
+        const int pb = it & 1;
+        ok = warp_wait(&S.p_full[pb], (it >> 1) & 1, abortp, P.status);
         if (!ok) break;
         ptx::tc_fence_after();
-        float hv[kMC];
+        const float sv = S.s_tab[par][grp][st];
+        const uint32_t src = tmem + lane_base + pb * 128 + grp * 64;
 #pragma unroll
         for (int c0 = 0; c0 < 64; c0 += 16) {
           if (c0 < 2 * m) {
-            uint32_t g[16], p[16];
-            ptx::tmem_ld16(tmem + lane_base + c0, g);
-            ptx::tmem_ld16(tmem + lane_base + 64 + c0, p);
+            uint32_t o[16];
+            ptx::tmem_ld16(src + c0, o);
             ptx::tmem_ld_wait();
 #pragma unroll
             for (int r = 0; r < 8; ++r) {
               const int tr = c0 / 2 + r;
-              const float inv = tr < m ? S.e_inv[par][tr] : 0.f;
-              const float gg = (__uint_as_float(g[2 * r]) + __uint_as_float(g[2 * r + 1]) * 0.0625f) * (inv * ig);
-              const float pp = (__uint_as_float(p[2 * r]) + __uint_as_float(p[2 * r + 1]) * 0.0625f) * (inv * iu);
-              hv[tr] = tr < m ? gg / (1.f + __expf(-gg)) * pp : 0.f;
+              const float f = t.phase2 ? sv * S.f2[par][st][tr] : sv;
+              acc[tr] = fmaf(__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f, f, acc[tr]);
             }
-          } else {
-#pragma unroll
-            for (int r = 0; r < 8; ++r) hv[c0 / 2 + r] = 0.f;
           }
         }
         ptx::tc_fence_before();
-        ptx::mbar_arrive(&S.acc_empty);  // G and P are in registers: the next phase-1 task may start
-        ++p1;
-#pragma unroll
-        for (int r = 0; r < kMC; ++r) {
-          if (r < m) {
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hv[r])));
-            if (lane == 0) S.e_amax[warp - 2][r] = mx;
-          }
-        }
-        if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
-        uint8_t* tile = P.hq + ((size_t)t.unit * n_slices + slice) * 8192;  // [64 rows][128 B], row-major
-        float* tf = P.hq_f + ((size_t)t.unit * n_slices + slice) * kMC;
-#pragma unroll
-        for (int r = 0; r < kMC; ++r) {
-          if (r < m) {
-            const uint32_t mx = max(max(S.e_amax[0][r], S.e_amax[1][r]), max(S.e_amax[2][r], S.e_amax[3][r]));
-            const int er = safe_exponent(__uint_as_float(mx));
-            const float v = hv[r] * pow2i(6 - er);
-            const __nv_fp8_storage_t hc = __nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
-            const __half_raw hr = __nv_cvt_fp8_to_halfraw(hc, __NV_E4M3);
-            const float hf = __half2float(*reinterpret_cast<const __half*>(&hr));
-            const __nv_fp8_storage_t lc = __nv_cvt_float_to_fp8((v - hf) * 16.f, __NV_SATFINITE, __NV_E4M3);
-            tile[(2 * r) * 128 + row] = hc;
-            tile[(2 * r + 1) * 128 + row] = lc;
-            if (row == r) tf[r] = S.e_w[par][r] * pow2i(er - 6);
-          }
-        }
-        // publish: every thread's stores, then one release increment of the unit's counter
-        __threadfence();
-        if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
-        if (warp == 2 && lane == 0) {
-          asm volatile("fence.proxy.async;" ::: "memory");
-          __threadfence();
-          atomicAdd(P.unit_done + t.unit, 1);
-        }
-      } else {
-        // ---------------- phase 2: two H tiles, all slices; scaled partial products summed in registers
-        ok = wait_unit_done(P.unit_done + t.unit, n_slices, abortp, P.status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        // the tables below are single-buffered: every epilogue warp has left the previous task
-        if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
-        const int nt = (2 * t.hp + 1 < HT) ? 2 : 1;
-        const float* sd = u.shared ? P.sh_s_down : P.s_down;
-        // tables (every warp writes all entries it reads: identical values, no cross-warp sync)
-        for (int i = lane; i < n_slices * kMC; i += 32) {
-          const int sl = i / kMC, r = i % kMC;
-          S.e_f2[sl][r] = r < m ? __ldcg(P.hq_f + ((size_t)t.unit * n_slices + sl) * kMC + r) : 0.f;
-        }
-        for (int i = lane; i < 2 * n_slices; i += 32) {
-          const int tl = i / n_slices, sl = i % n_slices;
-          const int ht = 2 * t.hp + tl;
-          S.e_sd2[tl][sl] = ht < HT ? __ldg(sd + ((size_t)u.expert * HT + ht) * n_slices + sl) : 0.f;
-        }
-        __syncwarp();
-        float acc[2][kMC];
-#pragma unroll
-        for (int tl = 0; tl < 2; ++tl)
-#pragma unroll
-          for (int r = 0; r < kMC; ++r) acc[tl][r] = 0.f;
-        for (int sl = 0; sl < n_slices && ok; ++sl, ++dsc) {
-          const int db = dsc & 1;
-          ok = warp_wait(&S.d_full[db], (dsc >> 1) & 1, abortp, P.status);
-          if (!ok) break;
-          ptx::tc_fence_after();
-#pragma unroll
-          for (int tl = 0; tl < 2; ++tl) {
-            if (tl < nt) {
-              const float sdv = S.e_sd2[tl][sl];
-#pragma unroll
-              for (int c0 = 0; c0 < 64; c0 += 16) {
-                if (c0 < 2 * m) {
-                  uint32_t o[16];
-                  ptx::tmem_ld16(tmem + lane_base + 128 + (db * 2 + tl) * 64 + c0, o);
-                  ptx::tmem_ld_wait();
-#pragma unroll
-                  for (int r = 0; r < 8; ++r) {
-                    const int tr = c0 / 2 + r;
-                    acc[tl][tr] = fmaf(__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f,
-                                       sdv * S.e_f2[sl][tr], acc[tl][tr]);
-                  }
-                }
-              }
-            }
-          }
-          ptx::tc_fence_before();
-          ptx::mbar_arrive(&S.d_empty[db]);
-        }
-        if (!ok) break;
-#pragma unroll
-        for (int tl = 0; tl < 2; ++tl) {
-          if (tl < nt) {
-            float* ycol = P.y32 + (size_t)(2 * t.hp + tl) * 128 + row;
-#pragma unroll
-            for (int r = 0; r < kMC; ++r)
-              if (r < m) ptx::red_add_f32(ycol + (size_t)S.e_tok[par][r] * H, acc[tl][r]);
-          }
-        }
-      }
-    }
-  }
-  else {
-    // ===================================================== activation producers (4 warps): phase-1 tasks only
-    const int pw = warp - 6;
-    uint32_t bit = 0, q = 0, tcount = 0;
-    bool ok = true;
-    const uint16_t* xb = static_cast<const uint16_t*>(P.x);
-    for (;; ++tcount) {
-      const int id = next_task(S, q, abortp, P.status, true);
-      if (id < 0) break;
-      const Task t = decode(id, n_units, n_slices, n_hp);
-      if (t.phase2) continue;  // phase 2 reads its operand tiles from the scratch array by TMA
-      const Unit u = P.units[t.unit];
-      const int slice = t.slice, m = u.m, par = tcount & 1;
-      for (int r = lane; r < m; r += 32) {
-        const int tok = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma) + r) : P.slot_token[u.slot0 + r];
-        S.p_tok[par][r] = tok;
-        S.p_tscale[par][r] = P.tok_scale[tok];
-      }
-      {
-        // block scales of this task's row block, one per K chunk; common power of two from their max
-        const float* sg = (u.shared ? P.sh_s_gate : P.s_gate) + ((size_t)u.expert * n_slices + slice) * KC;
-        const float* su = (u.shared ? P.sh_s_up : P.s_up) + ((size_t)u.expert * n_slices + slice) * KC;
-        float vg[4], vu[4];
-        float mg = 0.f, mu = 0.f;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int kc = lane + 32 * i;
-          vg[i] = kc < KC ? __ldg(sg + kc) : 0.f;
-          vu[i] = kc < KC ? __ldg(su + kc) : 0.f;
-          mg = fmaxf(mg, fabsf(vg[i]));
-          mu = fmaxf(mu, fabsf(vu[i]));
-        }
-        mg = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mg)));
-        mu = __uint_as_float(__reduce_max_sync(0xffffffffu, __float_as_uint(mu)));
-        const int eg = safe_exponent(mg), eu = safe_exponent(mu);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int kc = lane + 32 * i;
-          if (kc < KC) { S.p_sg[par][kc] = vg[i] * pow2i(-eg); S.p_su[par][kc] = vu[i] * pow2i(-eu); }
-        }
-      }
-      __syncwarp();
-      // warp pw converts token rows pw, pw + 4, ...; a lane owns 4 consecutive elements of the chunk
-      constexpr int kMaxPass = kMC / 4;
-      const int passes = (m - pw + 3) >> 2;
-      uint2 n0[kMaxPass], n1[kMaxPass], n2[kMaxPass];
-      const uint8_t* xrow[kMaxPass];
-#pragma unroll
-      for (int i = 0; i < kMaxPass; ++i) {
-        n0[i] = n1[i] = n2[i] = make_uint2(0, 0);
-        xrow[i] = nullptr;
-        if (i < passes) {
-          xrow[i] = reinterpret_cast<const uint8_t*>(xb + (size_t)S.p_tok[par][pw + 4 * i] * H) + lane * 8;
-          n0[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i]));
-          if (1 < KC) n1[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + 256));
-          if (2 < KC) n2[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + 512));
-        }
-      }
-      for (int kc = 0; kc < KC && ok; ++kc, ++bit) {
-        const int sb = bit % kBSlots;
-        uint2 cur[kMaxPass];
-#pragma unroll
-        for (int i = 0; i < kMaxPass; ++i) {
-          cur[i] = n0[i];
-          n0[i] = n1[i];
-          n1[i] = n2[i];
-          if (i < passes && kc + 3 < KC) n2[i] = __ldg(reinterpret_cast<const uint2*>(xrow[i] + (size_t)(kc + 3) * 256));
-        }
-        ok = warp_wait(&S.b_empty[sb], ((bit / kBSlots) & 1) ^ 1, abortp, P.status);
-        if (!ok) break;
-        uint8_t* tile = b_ring + sb * kBSlotBytes;
-        const float sgc = S.p_sg[par][kc], suc = S.p_su[par][kc];
-#pragma unroll
-        for (int i = 0; i < kMaxPass; ++i) {
-          if (i < passes) {
-            const int r = pw + 4 * i;
-            const float ts = S.p_tscale[par][r];
-            float v[4], f[4];
-            v[0] = __uint_as_float(cur[i].x << 16) * ts;
-            v[1] = __uint_as_float(cur[i].x & 0xffff0000u) * ts;
-            v[2] = __uint_as_float(cur[i].y << 16) * ts;
-            v[3] = __uint_as_float(cur[i].y & 0xffff0000u) * ts;
-            uint32_t hi, lo;
-            const uint32_t off_hi = sw128(2 * r, lane >> 2) + (lane & 3) * 4;
-            const uint32_t off_lo = sw128(2 * r + 1, lane >> 2) + (lane & 3) * 4;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) f[e] = v[e] * sgc;
-            split4_e4m3(f, hi, lo);
-            *reinterpret_cast<uint32_t*>(tile + off_hi) = hi;
-            *reinterpret_cast<uint32_t*>(tile + off_lo) = lo;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) f[e] = v[e] * suc;
-            split4_e4m3(f, hi, lo);
-            *reinterpret_cast<uint32_t*>(tile + 8192 + off_hi) = hi;
-            *reinterpret_cast<uint32_t*>(tile + 8192 + off_lo) = lo;
-          }
-        }
-        ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(&S.b_full[sb]);
+        ptx::mbar_arrive(&S.p_empty[pb]);
       }
       if (!ok) break;
+
+      if (t.phase2) {
+        // ---- one reduction per (token, row)
+        if (have_tile) {
+          float* ycol = P.y32 + (size_t)(2 * t.hp + grp) * 128 + row;
+#pragma unroll
+          for (int r = 0; r < kMC; ++r)
+            if (r < m) ptx::red_add_f32(ycol + (size_t)S.e_tok[par][r] * H, acc[r]);
+        }
+        continue;
+      }
+      // ---- phase 1: undo the token scale; group 1 hands P to group 0 through TMEM
+#pragma unroll
+      for (int r = 0; r < kMC; ++r) acc[r] *= (r < m ? S.e_inv[par][r] : 0.f);
+      if (grp == 1) {
+        ok = warp_wait(&S.x_empty, (xph & 1) ^ 1, abortp, P.status);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        tmem_st32(tmem + lane_base + kColXchg, acc);
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&S.x_full);
+        ++xph;
+        continue;
+      }
+      ok = warp_wait(&S.x_full, xph & 1, abortp, P.status);
+      if (!ok) break;
+      ptx::tc_fence_after();
+      float hv[kMC];
+      {
+        uint32_t pv[32];
+        ptx::tmem_ld16(tmem + lane_base + kColXchg, *reinterpret_cast<uint32_t(*)[16]>(&pv[0]));
+        ptx::tmem_ld16(tmem + lane_base + kColXchg + 16, *reinterpret_cast<uint32_t(*)[16]>(&pv[16]));
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&S.x_empty);
+        ++xph;
+#pragma unroll
+        for (int r = 0; r < kMC; ++r) {
+          const float gg = acc[r], pp = __uint_as_float(pv[r]);
+          hv[r] = r < m ? gg / (1.f + __expf(-gg)) * pp : 0.f;
+        }
+      }
+      // per-token power-of-two scale from the amax over the 128 rows of the slice
+#pragma unroll
+      for (int r = 0; r < kMC; ++r) {
+        if (r < m) {
+          const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hv[r])));
+          if (lane == 0) S.e_amax[qd][r] = mx;
+        }
+      }
+      if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
+      uint8_t* tile = P.hq + ((size_t)t.unit * n_slices + t.slice) * 8192;  // [64 rows][128 B], row-major
+      float* tf = P.hq_f + ((size_t)t.unit * n_slices + t.slice) * kMC;
+#pragma unroll
+      for (int r = 0; r < kMC; ++r) {
+        if (r < m) {
+          const uint32_t mx = max(max(S.e_amax[0][r], S.e_amax[1][r]), max(S.e_amax[2][r], S.e_amax[3][r]));
+          const int er = safe_exponent(__uint_as_float(mx));
+          const float v = hv[r] * pow2i(6 - er);
+          const __nv_fp8_storage_t hc = __nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
+          const __half_raw hr = __nv_cvt_fp8_to_halfraw(hc, __NV_E4M3);
+          const float hf = __half2float(*reinterpret_cast<const __half*>(&hr));
+          const __nv_fp8_storage_t lc = __nv_cvt_float_to_fp8((v - hf) * 16.f, __NV_SATFINITE, __NV_E4M3);
+          tile[(2 * r) * 128 + row] = hc;
+          tile[(2 * r + 1) * 128 + row] = lc;
+          if (row == r) tf[r] = S.e_w[par][r] * pow2i(er - 6);
+        }
+      }
+      // publish: every thread's stores, then one release increment of the unit's counter
+      __threadfence();
+      if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
+      if (warp == 2 && lane == 0) {
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __threadfence();
+        atomicAdd(P.unit_done + t.unit, 1);
+      }
     }
   }
-
   // the caller synchronises the CTA and releases TMEM
 }
 

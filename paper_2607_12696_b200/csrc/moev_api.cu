@@ -50,7 +50,9 @@ struct moev_ctx {
   bool wide_ok = false;   // block-scaled fp8 on tensor cores: the two-phase kernel for many tokens per expert exists
   uint8_t* hq = nullptr;  // its scratch: quantised h tiles [max_units][n_slices][64][128] ...
   float* hq_f = nullptr;  // ... and their scales [max_units][n_slices][32]
-  CUtensorMap tm_hq;
+  uint8_t* xu = nullptr;  // per-unit operand tiles [max_units][H / 128][64][128]
+  size_t max_units = 0;
+  CUtensorMap tm_hq, tm_xu;
   CUtensorMap tm_xq;  // MXFP4 tensor-core path: the [2 * max_tokens, xq_stride] byte array T.xq, box 128 x 2
   int n_sm = 0;
   int unit_cap = 1 << 20;
@@ -117,7 +119,7 @@ cudaError_t dmalloc(T** p, size_t count) {
 
 bool route_use_bitmap(const moev_config& c, int gamma) { return route_bitmap_bytes(c.E, gamma) <= kRouteBitmapBudget; }
 // assignments per streamed expert above which the two-phase FFN kernel takes the call
-constexpr int kWideRatio = 8;
+constexpr int kWideRatio = 12;
 size_t route_smem(const moev_config& c, int gamma) {
   return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + (route_use_bitmap(c, gamma) ? route_bitmap_bytes(c.E, gamma) : 0);
 }
@@ -254,8 +256,10 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   W.sh_s_gate = P.sh_s_gate; W.sh_s_up = P.sh_s_up; W.sh_s_down = P.sh_s_down;
   W.status = P.status; W.gamma = gamma; W.H = g.H; W.I = g.I; W.A = P.A;
   W.wide = c->T.wide; W.unit_done = c->T.unit_done; W.hq = c->hq; W.hq_f = c->hq_f;
+  W.xq = c->T.xq; W.xu = c->xu;
   launch_k(tc::grouped_ffn_tc_kernel<WFMT>, dim3(c->n_sm), dim3(tc::kThreads), tc::kSmemBytes, st, ev == nullptr,
-           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], c->wide_ok ? c->tm_hq : tm->map[0], P, W);
+           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], c->wide_ok ? c->tm_hq : tm->map[0],
+           c->wide_ok ? c->tm_xu : tm->map[0], P, W);
   if (ev) cudaEventRecord(ev[4], st);
   if (ev) cudaEventRecord(ev[5], st);
 }
@@ -363,7 +367,9 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     c->wide_ok = c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_FP8E4M3_B128 && n_slices <= tcw::kMaxSlices;
     if (c->wide_ok) {
       ok = ok && dmalloc(&c->T.wide, 1) == cudaSuccess;
-      ok = ok && dmalloc(&c->T.unit_done, max_units) == cudaSuccess;
+      ok = ok && dmalloc(&c->T.unit_done, 2 * max_units) == cudaSuccess;
+      c->max_units = max_units;
+      ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->xu), max_units * (size_t)(cfg->H / 128) * 8192) == cudaSuccess;
       ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->hq), max_units * (size_t)n_slices * 8192) == cudaSuccess;
       ok = ok && dmalloc(&c->hq_f, max_units * (size_t)n_slices * tcw::kMC) == cudaSuccess;
       EncodeTiledFn fn = encode_tiled_fn();
@@ -375,12 +381,16 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
         ok = fn(&c->tm_hq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c->hq, dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+        cuuint64_t dims_u[2] = {128, (cuuint64_t)(max_units * (size_t)(cfg->H / 128) * 64)};
+        ok = ok && fn(&c->tm_xu, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c->xu, dims_u, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
       } else {
         ok = false;
       }
     }
   }
-  if (c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_MXFP4) {
+  if (c->resolved_impl == MOEV_IMPL_TCGEN05 && (cfg->wfmt == MOEV_W_MXFP4 || c->wide_ok)) {
     // quantised activations (two e4m3 terms per element), loaded by TMA as the MMA's N operand
     c->T.xq_stride = cfg->H + (cfg->H % 128 ? 128 : 0);
     ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->T.xq), 2 * G * (size_t)c->T.xq_stride) == cudaSuccess;
@@ -445,7 +455,7 @@ moev_status moev_destroy(moev_ctx* c) {
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
   cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->T.task_counter); cudaFree(c->hbuf); cudaFree(c->y32);
-  cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f);
+  cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f); cudaFree(c->xu);
   cudaFree(c->x_stage); cudaFree(c->y_stage);
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)

@@ -557,7 +557,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       __shared__ int n_units_s;
       if (tid == blockDim.x - 1) n_units_s = base + sc;
       __syncthreads();
-      for (int i = tid; i < n_units_s; i += blockDim.x) T.unit_done[i] = 0;
+      for (int i = tid; i < 2 * n_units_s; i += blockDim.x) T.unit_done[i] = 0;  // and the gather flags behind them
     }
   }
 

@@ -76,6 +76,16 @@ def test_batched_verification_skewed_routing(base, kw, gamma):
     assert counts.max() >= gamma // 2 and ref.n_active <= shape.E
 
 
+@pytest.mark.parametrize("gamma,U,n_shared", [(100, 8, 1), (77, 16, 0), (128, 8, 2), (33, 8, 1)])
+def test_many_tokens_per_expert_two_phase_schedule(gamma, U, n_shared):
+    """FP8 calls with many tokens per streamed expert take the two-phase schedule (gate/up tasks
+    write h tiles to scratch, down tasks own a pair of H tiles): odd number of H tiles (the last
+    down task has one tile), three I slices, token runs that do not fill a unit, shared experts."""
+    shape = small_shape("deepseek", H=640, I=384, E=32, n_shared=n_shared)
+    err, ref = parity_case(shape, gamma, routing="exact", U=U)
+    assert ref.n_active == U
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_topk_equals_E_and_two_shared(impl):
     shape = small_shape("deepseek", H=256, I=128, E=8, top_k=8, n_shared=2)
