@@ -119,7 +119,7 @@ cudaError_t dmalloc(T** p, size_t count) {
 
 bool route_use_bitmap(const moev_config& c, int gamma) { return route_bitmap_bytes(c.E, gamma) <= kRouteBitmapBudget; }
 // assignments per streamed expert above which the two-phase FFN kernel takes the call
-constexpr int kWideRatio = 12;
+constexpr int kWideRatio = 8;
 size_t route_smem(const moev_config& c, int gamma) {
   return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + (route_use_bitmap(c, gamma) ? route_bitmap_bytes(c.E, gamma) : 0);
 }
