@@ -54,6 +54,8 @@ WORKLOADS = {
     # and Qwen-shaped layers with 64 experts
     "deepseek_fp8_E64_g16_profile": ("deepseek", 16, "scattered", {"_E": 64}),
     "qwen_bf16_E64_g16_profile": ("qwen", 16, "iid", {"_E": 64}),
+    # the two-phase schedule (many tokens per expert) at profiling size: 256 rows, skewed routing
+    "deepseek_fp8_E64_b4g64_zipf_profile": ("deepseek", 256, "zipf", {"_E": 64, "alpha": 1.0}),
     # routing kernels at the full router shape (256 experts, gamma 64) with thin experts (0.7 GB)
     "deepseek_router_profile": ("deepseek", 64, "scattered", {"_I": 128}),
 }

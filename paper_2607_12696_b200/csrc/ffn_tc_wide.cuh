@@ -162,11 +162,7 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
   }
   __syncthreads();
   const int n_units = *P.n_units;
-#ifdef MOEV_WIDE_ONLY_PHASE1
-  const int n_ids = n_units * n_slices;  // timing experiment: results are wrong
-#else
   const int n_ids = n_units * (n_slices + n_hp);
-#endif
   volatile int* abortp = &S.abort_flag;
   int32_t* gath_done = P.unit_done + n_units;  // the grouping kernel zeroes 2 * n_units counters: progress, then gather flags
 
