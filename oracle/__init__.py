@@ -20,6 +20,7 @@ _SRC = os.path.join(_HERE, "moe_oracle.c")
 _LIB = os.path.join(_HERE, "libmoe_oracle.so")
 
 W_FP32, W_BF16, W_FP8E4M3_B128, W_MXFP4 = 0, 1, 2, 3
+FFN_SWIGLU, FFN_GPTOSS = 0, 1
 ACT_FP32, ACT_BF16 = 0, 1
 SCORE_SOFTMAX, SCORE_SIGMOID = 0, 1
 
@@ -36,13 +37,14 @@ def build(force: bool = False) -> str:
 class _Cfg(C.Structure):
     _fields_ = [("H", C.c_int32), ("I", C.c_int32), ("E", C.c_int32), ("top_k", C.c_int32),
                 ("n_shared", C.c_int32), ("wfmt", C.c_int32), ("afmt", C.c_int32),
-                ("score", C.c_int32), ("routed_scale", C.c_double)]
+                ("score", C.c_int32), ("routed_scale", C.c_double), ("ffn_kind", C.c_int32),
+                ("reserved", C.c_int32)]
 
 
 class _Layer(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "router_w", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down",
-        "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down")]
+        "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down", "b_gate", "b_up", "b_down")]
 
 
 @dataclass
@@ -56,10 +58,11 @@ class Config:
     afmt: int = ACT_FP32
     score: int = SCORE_SOFTMAX
     routed_scale: float = 1.0
+    ffn_kind: int = 0   # 0 bias-free SwiGLU; 1 GPT-OSS form (clamped, biased; layer keys b_gate / b_up / b_down)
 
     def c(self) -> _Cfg:
         return _Cfg(self.H, self.I, self.E, self.top_k, self.n_shared, self.wfmt, self.afmt,
-                    self.score, self.routed_scale)
+                    self.score, self.routed_scale, self.ffn_kind, 0)
 
 
 _lib = None

@@ -47,6 +47,8 @@ typedef struct {
   int32_t H, I, E, top_k, n_shared;
   int32_t wfmt, afmt, score;
   double routed_scale;
+  int32_t ffn_kind; /* 0: bias-free SwiGLU (the benchmark configurations); 1: GPT-OSS form, see expert_ffn */
+  int32_t reserved;
 } oracle_cfg;
 
 /* All pointers are HOST pointers.  Layouts (K = contraction dim, contiguous):
@@ -62,6 +64,7 @@ typedef struct {
   const void *s_gate, *s_up, *s_down;
   const void *sh_gate, *sh_up, *sh_down;
   const void *sh_s_gate, *sh_s_up, *sh_s_down;
+  const float *b_gate, *b_up, *b_down; /* ffn_kind 1: fp32 biases [E,I], [E,I], [E,H]; NULL = zero */
 } oracle_layer;
 
 /* ---------------------------------------------------------------- decoders */
@@ -248,10 +251,14 @@ int32_t oracle_union_perm(int32_t E, int32_t k, int32_t gamma, const int32_t *id
 
 /* Apply expert e (of the tensor set wg/wu/wd with scales sg/su/sd) to m
  * tokens: xs[m][H] -> out[m][H] with out = Wd * ( silu(Wg x) * (Wu x) ),
- * silu(z) = z / (1 + exp(-z)).  Each weight row is decoded once. */
+ * silu(z) = z / (1 + exp(-z)).  Each weight row is decoded once.
+ * ffn_kind 1 (the published GPT-OSS expert; not in the paper, which does not print the FFN):
+ *   g = min(Wg x + bg, 7),  u = clamp(Wu x + bu, -7, 7),
+ *   h = g * sigmoid(1.702 g) * (u + 1),  out = Wd h + bd          (bg, bu, bd may be NULL = 0). */
 static void expert_ffn(const oracle_cfg *c, const void *wg, const void *wu, const void *wd,
                        const void *sg, const void *su, const void *sd, int64_t e, int m,
-                       const double *xs, double *out) {
+                       const double *xs, double *out, const float *bg, const float *bu,
+                       const float *bd) {
   int64_t H = c->H, I = c->I;
   double *hbuf = (double *)malloc(sizeof(double) * (size_t)m * (size_t)I);
 #pragma omp parallel
@@ -267,7 +274,16 @@ static void expert_ffn(const oracle_cfg *c, const void *wg, const void *wu, cons
         double g = 0.0, p = 0.0;
         for (int64_t h = 0; h < H; ++h) g += rg[h] * xv[h];
         for (int64_t h = 0; h < H; ++h) p += ru[h] * xv[h];
-        hbuf[(int64_t)r * I + i] = g / (1.0 + exp(-g)) * p;
+        if (c->ffn_kind == 1) {
+          if (bg) g += (double)bg[e * I + i];
+          if (bu) p += (double)bu[e * I + i];
+          if (g > 7.0) g = 7.0;
+          if (p > 7.0) p = 7.0;
+          if (p < -7.0) p = -7.0;
+          hbuf[(int64_t)r * I + i] = g / (1.0 + exp(-1.702 * g)) * (p + 1.0);
+        } else {
+          hbuf[(int64_t)r * I + i] = g / (1.0 + exp(-g)) * p;
+        }
       }
     }
 #pragma omp for schedule(static)
@@ -277,6 +293,7 @@ static void expert_ffn(const oracle_cfg *c, const void *wg, const void *wu, cons
         const double *hv = hbuf + (int64_t)r * I;
         double o = 0.0;
         for (int64_t i = 0; i < I; ++i) o += rg[i] * hv[i];
+        if (c->ffn_kind == 1 && bd) o += (double)bd[e * H + n];
         out[(int64_t)r * H + n] = o;
       }
     }
@@ -291,9 +308,10 @@ void oracle_expert_ffn(const oracle_cfg *c, const oracle_layer *L, int32_t share
                        int32_t m, const double *xs, double *out) {
   if (shared)
     expert_ffn(c, L->sh_gate, L->sh_up, L->sh_down, L->sh_s_gate, L->sh_s_up, L->sh_s_down, e, m,
-               xs, out);
+               xs, out, NULL, NULL, NULL);
   else
-    expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, e, m, xs, out);
+    expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, e, m, xs, out, L->b_gate, L->b_up,
+               L->b_down);
 }
 
 /* ------------------------------------------------------------- whole layer */
@@ -346,7 +364,7 @@ int32_t oracle_moe_verify(const oracle_cfg *c, const oracle_layer *L, const void
         memcpy(xs + (int64_t)r * H, xd + (int64_t)t * H, sizeof(double) * (size_t)H);
       }
       expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, uni[u], m, xs,
-                 os);
+                 os, L->b_gate, L->b_up, L->b_down);
       for (int r = 0; r < m; ++r) {
         int a = pm[off[u] + r], t = a / k;
         for (int64_t n = 0; n < H; ++n) y64[(int64_t)t * H + n] += cw[a] * os[(int64_t)r * H + n];
@@ -354,7 +372,7 @@ int32_t oracle_moe_verify(const oracle_cfg *c, const oracle_layer *L, const void
     }
     for (int s = 0; s < c->n_shared; ++s) {
       expert_ffn(c, L->sh_gate, L->sh_up, L->sh_down, L->sh_s_gate, L->sh_s_up, L->sh_s_down, s,
-                 gamma, xd, os);
+                 gamma, xd, os, NULL, NULL, NULL);
       for (int64_t i = 0; i < (int64_t)gamma * H; ++i) y64[i] += os[i];
     }
     free(xd);
@@ -394,12 +412,13 @@ int32_t oracle_moe_dense(const oracle_cfg *c, const oracle_layer *L, const void 
   for (int t = 0; t < gamma; ++t) {
     for (int64_t h = 0; h < H; ++h) xd[h] = decode_act(x, c->afmt, (size_t)(t * H + h));
     for (int e = 0; e < E; ++e) {
-      expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, e, 1, xd, o);
+      expert_ffn(c, L->w_gate, L->w_up, L->w_down, L->s_gate, L->s_up, L->s_down, e, 1, xd, o, L->b_gate, L->b_up,
+                 L->b_down);
       for (int64_t n = 0; n < H; ++n) y64[(int64_t)t * H + n] += gate[(int64_t)t * E + e] * o[n];
     }
     for (int s = 0; s < c->n_shared; ++s) {
       expert_ffn(c, L->sh_gate, L->sh_up, L->sh_down, L->sh_s_gate, L->sh_s_up, L->sh_s_down, s, 1,
-                 xd, o);
+                 xd, o, NULL, NULL, NULL);
       for (int64_t n = 0; n < H; ++n) y64[(int64_t)t * H + n] += o[n];
     }
   }
