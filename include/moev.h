@@ -79,6 +79,12 @@ typedef enum {
   MOEV_IMPL_TCGEN05 = 2 /* tensor-core path; MOEV_EINVAL if the shape does not allow it */
 } moev_impl;
 
+/* Expert form.  The paper does not print the FFN; the benchmark configurations use the bias-free
+ * gated SwiGLU  down(silu(gate x) * (up x)).  MOEV_FFN_GPTOSS is the published GPT-OSS expert:
+ *   g = min(gate x + b_gate, 7),  u = clamp(up x + b_up, -7, 7),
+ *   h = g * sigmoid(1.702 g) * (u + 1),  out = down h + b_down   (weighted by the router weight). */
+typedef enum { MOEV_FFN_SWIGLU = 0, MOEV_FFN_GPTOSS = 1 } moev_ffn_kind;
+
 typedef struct {
   int32_t H;          /* hidden size; multiple of 32 */
   int32_t I;          /* expert intermediate size; multiple of 32 */
@@ -91,6 +97,7 @@ typedef struct {
   int32_t score;      /* moev_score */
   int32_t impl;       /* moev_impl */
   float routed_scale; /* c in the SIGMOID rule; ignored for SOFTMAX */
+  int32_t ffn_kind;   /* moev_ffn_kind; MOEV_FFN_GPTOSS needs n_shared == 0 */
 } moev_config;
 
 /* One layer's parameters.  Layouts, row-major, last index contiguous:
@@ -107,6 +114,7 @@ typedef struct {
   const void *s_gate, *s_up, *s_down;
   const void *sh_gate, *sh_up, *sh_down;
   const void *sh_s_gate, *sh_s_up, *sh_s_down;
+  const float *b_gate, *b_up, *b_down; /* MOEV_FFN_GPTOSS: fp32 biases [E,I], [E,I], [E,H]; NULL = zero */
 } moev_layer;
 
 /* Outputs.  y and n_active are required; the others are diagnostics and may be NULL.

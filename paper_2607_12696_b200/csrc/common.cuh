@@ -53,6 +53,8 @@ struct LayerPtrs {
   const void *s_gate, *s_up, *s_down;
   const void *sh_gate, *sh_up, *sh_down;
   const void *sh_s_gate, *sh_s_up, *sh_s_down;
+  const float *b_gate, *b_up, *b_down;  // MOEV_FFN_GPTOSS biases (routed experts), may be null
+  int ffn_kind;
 };
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
@@ -82,6 +84,17 @@ __device__ __forceinline__ void split4_e4m3(const float (&v)[4], uint32_t& hi, u
     hi |= (uint32_t)hc << (16 * p);
     lo |= (uint32_t)lc << (16 * p);
   }
+}
+
+// h from the gate / up pre-activations (biases already added): bias-free SwiGLU, or the GPT-OSS
+// form  min(g, 7) * sigmoid(1.702 min(g, 7)) * (clamp(u, -7, 7) + 1)
+__device__ __forceinline__ float ffn_act(int kind, float g, float u) {
+  if (kind == MOEV_FFN_GPTOSS) {
+    g = fminf(g, 7.f);
+    u = fminf(fmaxf(u, -7.f), 7.f);
+    return g / (1.f + __expf(-1.702f * g)) * (u + 1.f);
+  }
+  return g / (1.f + __expf(-g)) * u;
 }
 
 // e8m0 scale byte -> float 2^(b-127)  (b = 0 is the subnormal 2^-127)

@@ -152,8 +152,11 @@ __global__ void __launch_bounds__(256) ffn_gateup_simt(LayerPtrs L, Tables T, co
       for (int c = 0; c < kSimtTC; ++c) {
         float gs = warp_sum(ag[c]), us = warp_sum(au[c]);
         if (lane == 0 && tok[c] >= 0) {
-          float hval = gs / (1.f + __expf(-gs)) * us;
-          hbuf[(size_t)(s.slot0 + r0 + c) * I + i] = hval;
+          if (L.ffn_kind == MOEV_FFN_GPTOSS && !s.shared) {
+            if (L.b_gate) gs += __ldg(L.b_gate + (size_t)s.e * I + i);
+            if (L.b_up) us += __ldg(L.b_up + (size_t)s.e * I + i);
+          }
+          hbuf[(size_t)(s.slot0 + r0 + c) * I + i] = ffn_act(L.ffn_kind, gs, us);
         }
       }
     }
@@ -203,6 +206,7 @@ __global__ void __launch_bounds__(256) ffn_down_simt(LayerPtrs L, Tables T, cons
           int slot = s.slot0 + r0 + c;
           int t = s.shared ? (r0 + c) : T.slot_token[slot];
           float w = s.shared ? 1.f : T.slot_w[slot];
+          if (L.ffn_kind == MOEV_FFN_GPTOSS && !s.shared && L.b_down) o += __ldg(L.b_down + (size_t)s.e * H + n);
           atomicAdd(&y32[(size_t)t * H + n], w * o);
         }
       }

@@ -96,6 +96,8 @@ struct Params {
   float* y32;
   const uint8_t *s_gate, *s_up, *s_down;           // e8m0 [E, N, K/32]
   const uint8_t *sh_s_gate, *sh_s_up, *sh_s_down;
+  const float *b_gate, *b_up, *b_down;  // MOEV_FFN_GPTOSS biases of the routed experts (may be null)
+  int32_t ffn_kind;
   int32_t* status;
   int32_t gamma, H, I, A;
 #ifdef MOEV_TC_STATS
@@ -484,6 +486,12 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 
       float hv[kMC];
       const uint32_t gp = tmem + lane_base + par * 64;
+      // GPT-OSS form: biases of this thread's row of the slice (rows past the end of I stay 0, as does h)
+      const int irow = slice * 128 + row;
+      const bool biased = P.ffn_kind == MOEV_FFN_GPTOSS && !u.shared;
+      const float bgv = (biased && P.b_gate && irow < I) ? __ldg(P.b_gate + (size_t)u.expert * I + irow) : 0.f;
+      const float buv = (biased && P.b_up && irow < I) ? __ldg(P.b_up + (size_t)u.expert * I + irow) : 0.f;
+      const int kind = (biased && irow < I) ? MOEV_FFN_GPTOSS : (irow < I ? MOEV_FFN_SWIGLU : -1);
 #pragma unroll
       for (int c0 = 0; c0 < 32; c0 += 16) {
         if (c0 < 2 * m) {
@@ -497,7 +505,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             float inv = tr < m ? S.e_inv[par][tr] : 0.f;
             float gg = (__uint_as_float(g[2 * r]) + __uint_as_float(g[2 * r + 1]) * 0.0625f) * inv;
             float pp = (__uint_as_float(p[2 * r]) + __uint_as_float(p[2 * r + 1]) * 0.0625f) * inv;
-            hv[tr] = tr < m ? gg / (1.f + __expf(-gg)) * pp : 0.f;
+            hv[tr] = (tr < m && kind >= 0) ? ffn_act(kind, gg + bgv, pp + buv) : 0.f;
           }
         } else {
 #pragma unroll
@@ -564,10 +572,13 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           const int hrow = (ds * 2 + tl) * 128 + row;
           if (tl < nt && hrow < H) {
             float* ycol = P.y32 + hrow;
+            // the down bias belongs to the expert's output: added once per (token, expert), by the slice-0 task
+            const float bdv = (biased && slice == 0 && P.b_down) ? __ldg(P.b_down + (size_t)u.expert * H + hrow) : 0.f;
 #pragma unroll
             for (int r = 0; r < kMC; ++r)
               if (r < m) {
-                float val = (__uint_as_float(o[tl][2 * r]) + __uint_as_float(o[tl][2 * r + 1]) * 0.0625f) * S.e_f[r];
+                float val = (__uint_as_float(o[tl][2 * r]) + __uint_as_float(o[tl][2 * r + 1]) * 0.0625f) * S.e_f[r] +
+                            bdv * S.e_w[par][r];
                 ptx::red_add_f32(ycol + (size_t)S.e_tok[par][r] * H, val);
               }
           }

@@ -90,6 +90,8 @@ bool cfg_ok(const moev_config* c, char* why, size_t n) {
   BAD(c->afmt < 0 || c->afmt > MOEV_ACT_BF16, "unknown activation format");
   BAD(c->score < 0 || c->score > MOEV_SCORE_SIGMOID, "unknown score function");
   BAD(c->impl < 0 || c->impl > MOEV_IMPL_TCGEN05, "unknown impl");
+  BAD(c->ffn_kind < 0 || c->ffn_kind > MOEV_FFN_GPTOSS, "unknown ffn_kind");
+  BAD(c->ffn_kind == MOEV_FFN_GPTOSS && c->n_shared != 0, "the GPT-OSS expert form has no shared experts");
 #undef BAD
   return true;
 }
@@ -148,6 +150,7 @@ bool tc_eligible(const moev_config& c) {
            128 * (c.H / 32) <= tcmx::kScStageBytes &&  // a slice's gate/up scale block is staged in shared memory,
            (c.H + 127) / 128 <= tcmx::kDownWords;         // and one word per W_down row
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
+  if (c.ffn_kind != MOEV_FFN_SWIGLU) return false;  // the biased, clamped form: MXFP4 tensor-core kernel or CUDA cores
   if (c.H % 128 || c.I % 128) return false;
   const int bk = c.wfmt == MOEV_W_BF16 ? 64 : 128;
   if (c.H / bk < 4 || c.H / 128 > 128 || c.H / bk > 128 * (128 / bk)) return false;
@@ -274,6 +277,7 @@ void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.s_down = static_cast<const uint8_t*>(L->s_down);
   P.sh_s_gate = static_cast<const uint8_t*>(L->sh_s_gate); P.sh_s_up = static_cast<const uint8_t*>(L->sh_s_up);
   P.sh_s_down = static_cast<const uint8_t*>(L->sh_s_down);
+  P.b_gate = L->b_gate; P.b_up = L->b_up; P.b_down = L->b_down; P.ffn_kind = g.ffn_kind;
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
 #ifdef MOEV_TC_STATS
   P.stats = c->tc_stats;
@@ -505,7 +509,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   LayerPtrs L{layer->w_gate, layer->w_up, layer->w_down, layer->s_gate, layer->s_up, layer->s_down,
               layer->sh_gate, layer->sh_up, layer->sh_down, layer->sh_s_gate, layer->sh_s_up,
-              layer->sh_s_down};
+              layer->sh_s_down, layer->b_gate, layer->b_up, layer->b_down, g.ffn_kind};
   RouteOut O{out->topk_ids, out->topk_w, out->union_ids, out->offsets, out->perm, out->n_active};
   const size_t y_elems = (size_t)gamma * g.H;
 

@@ -37,6 +37,7 @@ def run_gpu(shape, router_w, weights, x, gamma, impl=moev.IMPL_AUTO, max_tokens=
     torch.cuda.synchronize()
     res = {k: t.cpu().numpy() if t.dtype != torch.bfloat16 else t.float().cpu().numpy()
            for k, t in out.items()}
+    res["_impl"] = v.resolved_impl()
     if verifier is None:
         v.close()
     return res
@@ -60,7 +61,7 @@ def compare(shape, res, ref: oracle.Result, gamma, y_ref=None, y_rows=None, tol=
     return err
 
 
-def parity_case(shape, gamma, routing="iid", impl=moev.IMPL_AUTO, layer_id=0, **kw):
+def parity_case(shape, gamma, routing="iid", impl=moev.IMPL_AUTO, layer_id=0, expect_impl=None, **kw):
     dev = "cuda"
     w = synth.make_expert_weights(shape, layer=layer_id, device=dev)
     fn = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
@@ -68,6 +69,8 @@ def parity_case(shape, gamma, routing="iid", impl=moev.IMPL_AUTO, layer_id=0, **
           "zipf": synth.make_zipf_routing}[routing]
     wr, x = fn(shape, gamma, layer=layer_id, device=dev, **kw)
     res = run_gpu(shape, wr, w, x, gamma, impl)
+    if expect_impl is not None:
+        assert res["_impl"] == expect_impl, f"resolved kernels {res['_impl']}, expected {expect_impl}"
     ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), gamma)
     if routing == "iid":
         assert ref.gap.min() > 1e-9, "seed gives a near-tie; pick another layer id"

@@ -39,9 +39,17 @@ def test_deepseek_shaped_reduced(impl, routing):
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("gamma", [1, 8, 19])
 def test_gptoss_shaped_reduced_ragged(impl, gamma):
-    # 736 = 5.75 * 128 and 352 = 2.75 * 128: several tiles and a ragged tail in both dims
+    # 704 = 5.5 * 128 and 320 = 2.5 * 128: several tiles and a ragged tail (half a chunk) in both dims;
+    # the tensor-core kernel needs multiples of 64
+    shape = small_shape("gptoss", H=704, I=320, E=32)
+    parity_case(shape, gamma, impl=impl, expect_impl=moev.IMPL_TCGEN05 if impl == moev.IMPL_AUTO else moev.IMPL_SIMT)
+
+
+@pytest.mark.parametrize("gamma", [3, 19])
+def test_gptoss_shaped_not_multiple_of_64_runs_on_cuda_cores(gamma):
+    # 736 = 5.75 * 128 and 352 = 2.75 * 128: served by the CUDA-core kernels
     shape = small_shape("gptoss", H=736, I=352, E=32)
-    parity_case(shape, gamma, impl=impl)
+    parity_case(shape, gamma, expect_impl=moev.IMPL_SIMT)
 
 
 @pytest.mark.parametrize("impl", IMPLS)
@@ -49,8 +57,9 @@ def test_gptoss_shaped_reduced_ragged(impl, gamma):
 def test_gptoss_shaped_many_tokens_per_expert(impl, gamma, U, n_shared):
     """MXFP4 with more tokens per expert than one work unit holds (runs of 16), with and
     without shared experts, on ragged dimensions."""
-    shape = small_shape("gptoss", H=736, I=352, E=32, n_shared=n_shared)
-    err, ref = parity_case(shape, gamma, routing="exact", impl=impl, U=U)
+    shape = small_shape("gptoss", H=704, I=320, E=32, n_shared=n_shared)
+    err, ref = parity_case(shape, gamma, routing="exact", impl=impl, U=U,
+                           expect_impl=moev.IMPL_TCGEN05 if impl == moev.IMPL_AUTO else moev.IMPL_SIMT)
     assert ref.n_active == U
 
 
@@ -65,7 +74,7 @@ def test_exact_union_cases(impl, gamma, U):
 
 
 @pytest.mark.parametrize("base,kw,gamma", [("deepseek", dict(H=512, I=256, E=64), 512),
-                                           ("gptoss", dict(H=736, I=352, E=32), 200),
+                                           ("gptoss", dict(H=704, I=320, E=32), 200),
                                            ("qwen", dict(H=512, I=256, E=32), 260)])
 def test_batched_verification_skewed_routing(base, kw, gamma):
     """Many rows per call (several requests' trees at once) with Zipf-skewed routing: hot
@@ -107,7 +116,7 @@ def test_exact_logit_ties_break_to_lower_id(impl):
     compare(shape, res, ref, 6)
 
 
-@pytest.mark.parametrize("base,kw", [("deepseek", dict(H=1024, I=512, E=64)), ("gptoss", dict(H=736, I=352, E=32)),
+@pytest.mark.parametrize("base,kw", [("deepseek", dict(H=1024, I=512, E=64)), ("gptoss", dict(H=704, I=320, E=32)),
                                      ("qwen", dict(H=1024, I=384, E=32))])
 def test_pipelined_layers_match_oracle(base, kw):
     """moev_verify_pipeline: three independent layers in one call (the router of layer l + 1
