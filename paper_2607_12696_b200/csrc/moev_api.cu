@@ -39,6 +39,7 @@ struct moev_ctx {
   float* part_w2 = nullptr;  // [n_slices, expert tiles] max over the tile's experts of the slice's squared row norm
   int n_slices = 0;
   int ks = 32;  // columns per split-K slice of the router
+  bool router_mma = false;
 #ifdef MOEV_TC_STATS
   unsigned long long* tc_stats = nullptr;  // [n_sm][16], debug builds only
 #endif
@@ -347,6 +348,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   const size_t act_b = cfg->afmt == MOEV_ACT_FP32 ? 4 : 2;
   bool ok = true;
   c->ks = router_slice_width(cfg->H, prop.multiProcessorCount);
+  c->router_mma = cfg->afmt == MOEV_ACT_BF16;  // split-K partials on the tensor cores (slices of 16 k)
+  if (c->router_mma) c->ks = c->ks <= 16 ? 16 : (c->ks <= 32 ? 32 : (c->ks <= 48 ? 48 : 64));
   c->n_slices = (cfg->H + c->ks - 1) / c->ks;
   ok = ok && dmalloc(&c->part, (size_t)c->n_slices * G * E) == cudaSuccess;
   ok = ok && dmalloc(&c->part_x2, (size_t)c->n_slices * G) == cudaSuccess;
@@ -523,7 +526,8 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
     launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain, x, layer->router_w,
              c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
   else
-    launch_k(router_partial_kernel<MOEV_ACT_BF16>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain, x, layer->router_w,
+    launch_k(router_partial_mma_kernel, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256),
+             router_partial_mma_smem(c->ks), st, pdl && c->chain, static_cast<const uint16_t*>(x), layer->router_w,
              c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
   if (ev) cudaEventRecord(ev[1], st);
   if (g.afmt == MOEV_ACT_FP32)
@@ -533,7 +537,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   else
     launch_k(topk_refine_kernel<MOEV_ACT_BF16>, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x,
              layer->router_w, (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma,
-             g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale);
+             g.H, g.E, g.top_k, c->n_slices, c->router_mma ? 6 * c->ks + c->n_slices + 12 : c->ks, g.score, g.routed_scale);
   if (ev) cudaEventRecord(ev[2], st);
   launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
            g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma), c->wide_ok ? kWideRatio : 0);

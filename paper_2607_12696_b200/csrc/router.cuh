@@ -156,6 +156,149 @@ __global__ void __launch_bounds__(256) router_partial_kernel(const void* __restr
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// The same partials on the tensor cores, for bf16 activations: x is bf16 as it is and every fp32
+// router weight is the exact sum of three bf16 terms (8 + 8 + 8 significand bits), so all products
+// are exact in fp32 and only the accumulation rounds.  mma.sync m16n8k16 (bf16 x bf16 -> fp32);
+// a CTA computes 64 tokens x 64 experts of one K slice (KS a multiple of 16, <= kRouterMaxKS).
+// Warp (wm, wn): token rows 16 wm .., experts 32 wn .. (four n8 tiles).  Same outputs as
+// router_partial_kernel; the error bound of the refinement counts these accumulations instead.
+constexpr int kRouterMmaPad = 8;  // bf16 elements of row padding (16 bytes): conflict-free ldmatrix
+inline size_t router_partial_mma_smem(int ks) { return (size_t)4 * 64 * (ks + kRouterMmaPad) * 2; }
+
+__global__ void __launch_bounds__(256) router_partial_mma_kernel(const uint16_t* __restrict__ x,
+                                                                 const float* __restrict__ router_w,
+                                                                 float* __restrict__ part,
+                                                                 float* __restrict__ part_x2,
+                                                                 float* __restrict__ part_w2max, int gamma,
+                                                                 int H, int E, int KS) {
+  __shared__ float wmax_s[8];
+  __shared__ float sq_s[128];  // [0,64): squared norms of the router rows; [64,128): of the token rows
+  extern __shared__ __align__(16) uint16_t rpm_smem[];
+  const int LD = KS + kRouterMmaPad;           // row stride in elements
+  uint16_t* xs = rpm_smem;                     // [64 tokens][LD]
+  uint16_t* ws = rpm_smem + 64 * LD;           // [3 terms][64 experts][LD]
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int c = blockIdx.x, e0 = blockIdx.y * kRouterETile;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int wm = warp & 3, wn = warp >> 2;
+  const int k0 = c * KS, kn = min(KS, H - k0);  // kn is a multiple of 4
+  if (tid < 128) sq_s[tid] = 0.f;
+  __syncthreads();
+  // ---- router tile: float4 per thread and row, split into the three bf16 terms
+  const int kq4 = KS / 4;
+  const bool k64 = KS == 64;  // 16 lanes per row: shifts instead of divisions, shuffles instead of shared atomics
+  for (int i = tid; i < 64 * kq4; i += 256) {
+    const int er = k64 ? (i >> 4) : i / kq4, kq = (k64 ? (i & 15) : (i % kq4)) * 4;
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (e0 + er < E && kq < kn) v = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)(e0 + er) * H + k0 + kq));
+    const float f[4] = {v.x, v.y, v.z, v.w};
+    uint16_t t1[4], t2[4], t3[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t b1 = __float_as_uint(f[j]) & 0xffff0000u;       // truncation: exact 8-bit significand
+      const float r1 = f[j] - __uint_as_float(b1);                    // exact
+      const uint32_t b2 = __float_as_uint(r1) & 0xffff0000u;
+      const float r2 = r1 - __uint_as_float(b2);                      // exact, at most 8 significant bits left
+      t1[j] = (uint16_t)(b1 >> 16); t2[j] = (uint16_t)(b2 >> 16); t3[j] = (uint16_t)(__float_as_uint(r2) >> 16);
+    }
+    uint16_t* d = ws + er * LD + kq;
+    *reinterpret_cast<uint2*>(d) = make_uint2(t1[0] | ((uint32_t)t1[1] << 16), t1[2] | ((uint32_t)t1[3] << 16));
+    *reinterpret_cast<uint2*>(d + 64 * LD) = make_uint2(t2[0] | ((uint32_t)t2[1] << 16), t2[2] | ((uint32_t)t2[3] << 16));
+    *reinterpret_cast<uint2*>(d + 128 * LD) = make_uint2(t3[0] | ((uint32_t)t3[1] << 16), t3[2] | ((uint32_t)t3[3] << 16));
+    float sq = fmaf(v.x, v.x, fmaf(v.y, v.y, fmaf(v.z, v.z, v.w * v.w)));
+    if (k64) {  // a row is one aligned group of 16 lanes and is visited once
+#pragma unroll
+      for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+      if ((lane & 15) == 0) sq_s[er] = sq;
+    } else {
+      atomicAdd(&sq_s[er], sq);
+    }
+  }
+  for (int t0 = 0; t0 < gamma; t0 += 64) {
+    __syncthreads();  // previous token tile's reads are over (first trip: sq_s zeroed, nothing else pending)
+    if (tid < 64) sq_s[64 + tid] = 0.f;
+    __syncthreads();
+    // ---- token tile: 4 bf16 (8 bytes) per thread and row
+    for (int i = tid; i < 64 * kq4; i += 256) {
+      const int tr = k64 ? (i >> 4) : i / kq4, kq = (k64 ? (i & 15) : (i % kq4)) * 4;
+      uint2 q = make_uint2(0u, 0u);
+      if (t0 + tr < gamma && kq < kn) q = __ldg(reinterpret_cast<const uint2*>(x + (size_t)(t0 + tr) * H + k0 + kq));
+      *reinterpret_cast<uint2*>(xs + tr * LD + kq) = q;
+      const float a = __uint_as_float(q.x << 16), b = __uint_as_float(q.x & 0xffff0000u);
+      const float cc = __uint_as_float(q.y << 16), d = __uint_as_float(q.y & 0xffff0000u);
+      float sq = fmaf(a, a, fmaf(b, b, fmaf(cc, cc, d * d)));
+      if (k64) {
+#pragma unroll
+        for (int o = 8; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+        if ((lane & 15) == 0) sq_s[64 + tr] = sq;
+      } else {
+        atomicAdd(&sq_s[64 + tr], sq);
+      }
+    }
+    __syncthreads();
+    if (blockIdx.y == 0 && tid < 64 && t0 + tid < gamma) part_x2[(size_t)c * gamma + t0 + tid] = sq_s[64 + tid];
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    for (int kk = 0; kk < KS; kk += 16) {
+      uint32_t a[4];
+      {
+        const uint32_t addr = (uint32_t)__cvta_generic_to_shared(xs + (wm * 16 + (lane & 15)) * LD + kk + (lane >> 4) * 8);
+        asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr));
+      }
+#pragma unroll
+      for (int term = 0; term < 3; ++term) {
+#pragma unroll
+        for (int np = 0; np < 2; ++np) {  // two n8 tiles per ldmatrix.x4
+          uint32_t b[4];
+          const int n = wn * 32 + np * 16 + (lane & 7) + ((lane >> 4) << 3);
+          const uint32_t addr = (uint32_t)__cvta_generic_to_shared(ws + (term * 64 + n) * LD + kk + ((lane >> 3) & 1) * 8);
+          asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                       : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]) : "r"(addr));
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {
+            float* cacc = acc[np * 2 + h];
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                         : "+f"(cacc[0]), "+f"(cacc[1]), "+f"(cacc[2]), "+f"(cacc[3])
+                         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[2 * h]), "r"(b[2 * h + 1]));
+          }
+        }
+      }
+    }
+    // ---- C fragments: rows lane / 4 (+ 8), columns 2 (lane % 4) + {0, 1} of each n8 tile
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) {
+      const int e = e0 + wn * 32 + nt * 8 + (lane & 3) * 2;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int t = t0 + wm * 16 + (lane >> 2) + hh * 8;
+        if (t < gamma) {
+          float* dst = part + ((size_t)c * gamma + t) * E + e;
+          if (e + 1 < E && (E & 1) == 0) *reinterpret_cast<float2*>(dst) = make_float2(acc[nt][2 * hh], acc[nt][2 * hh + 1]);
+          else {
+            if (e < E) dst[0] = acc[nt][2 * hh];
+            if (e + 1 < E) dst[1] = acc[nt][2 * hh + 1];
+          }
+        }
+      }
+    }
+  }
+  // max over this tile's experts of the squared norm of this slice of the router rows
+  float w2max = (tid < 64 && e0 + tid < E) ? sq_s[tid] : 0.f;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) w2max = fmaxf(w2max, __shfl_xor_sync(0xffffffffu, w2max, o));
+  if (lane == 0) wmax_s[warp] = w2max;
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < 8; ++w) w2max = fmaxf(w2max, wmax_s[w]);
+    part_w2max[(size_t)c * gridDim.y + blockIdx.y] = w2max;
+  }
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // see router_partial_kernel
+}
+
 struct RouteOut {  // optional caller-visible copies (may be null)
   int32_t* topk_ids;
   float* topk_w;
@@ -295,7 +438,9 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     float xs = 0.f, wm = 0.f;
     for (int w = 0; w < kRefineWarps; ++w) { xs += redf[w]; wm += redw[w]; }
     // |fp32 logit - exact| <= gamma_n * sum|x w| <= n u ||x|| ||w||, n = roundings on the longest path
-    // (slice length + number of slices + the norm sums' own error, covered by the factor 1.25)
+    // (slice length + number of slices + the norm sums' own error, covered by the factor 1.25).  For the
+    // tensor-core partials the caller passes ks = 6 KS + n_slices + 12: three exact-product terms per
+    // element, every accumulation counted twice (the unit's additions may truncate).
     const float n_round = (float)(ks + n_slices + 4);
     const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
     // ---- candidates: every expert whose exact logit may be >= the exact k-th largest, in ascending id
