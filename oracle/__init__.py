@@ -38,13 +38,13 @@ class _Cfg(C.Structure):
     _fields_ = [("H", C.c_int32), ("I", C.c_int32), ("E", C.c_int32), ("top_k", C.c_int32),
                 ("n_shared", C.c_int32), ("wfmt", C.c_int32), ("afmt", C.c_int32),
                 ("score", C.c_int32), ("routed_scale", C.c_double), ("ffn_kind", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("n_group", C.c_int32), ("topk_group", C.c_int32), ("reserved", C.c_int32)]
 
 
 class _Layer(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in (
         "router_w", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down",
-        "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down", "b_gate", "b_up", "b_down")]
+        "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down", "b_gate", "b_up", "b_down", "router_bias")]
 
 
 @dataclass
@@ -59,10 +59,12 @@ class Config:
     score: int = SCORE_SOFTMAX
     routed_scale: float = 1.0
     ffn_kind: int = 0   # 0 bias-free SwiGLU; 1 GPT-OSS form (clamped, biased; layer keys b_gate / b_up / b_down)
+    n_group: int = 0    # > 0: DeepSeek group-limited routing (sigmoid scores; layer key router_bias)
+    topk_group: int = 0
 
     def c(self) -> _Cfg:
         return _Cfg(self.H, self.I, self.E, self.top_k, self.n_shared, self.wfmt, self.afmt,
-                    self.score, self.routed_scale, self.ffn_kind, 0)
+                    self.score, self.routed_scale, self.ffn_kind, self.n_group, self.topk_group, 0)
 
 
 _lib = None
@@ -159,6 +161,19 @@ def topk(cfg: Config, logits: np.ndarray):
     gap = np.empty(gamma, dtype=np.float64)
     c = cfg.c()
     lib().oracle_topk(C.byref(c), _p(logits), C.c_int32(gamma), _p(ids), _p(w), _p(gap))
+    return ids, w, gap
+
+
+def topk_grouped(cfg: Config, logits: np.ndarray, bias=None):
+    gamma = logits.shape[0]
+    logits = np.ascontiguousarray(logits, dtype=np.float64)
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+    ids = np.empty((gamma, cfg.top_k), dtype=np.int32)
+    w = np.empty((gamma, cfg.top_k), dtype=np.float64)
+    gap = np.empty(gamma, dtype=np.float64)
+    c = cfg.c()
+    lib().oracle_topk_grouped(C.byref(c), _p(logits), _p(bias), C.c_int32(gamma), _p(ids), _p(w), _p(gap))
     return ids, w, gap
 
 

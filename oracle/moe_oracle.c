@@ -48,6 +48,8 @@ typedef struct {
   int32_t wfmt, afmt, score;
   double routed_scale;
   int32_t ffn_kind; /* 0: bias-free SwiGLU (the benchmark configurations); 1: GPT-OSS form, see expert_ffn */
+  int32_t n_group;  /* > 0: group-limited routing, see oracle_topk_grouped (score must be sigmoid) */
+  int32_t topk_group;
   int32_t reserved;
 } oracle_cfg;
 
@@ -65,6 +67,7 @@ typedef struct {
   const void *sh_gate, *sh_up, *sh_down;
   const void *sh_s_gate, *sh_s_up, *sh_s_down;
   const float *b_gate, *b_up, *b_down; /* ffn_kind 1: fp32 biases [E,I], [E,I], [E,H]; NULL = zero */
+  const float *router_bias;            /* n_group > 0: fp32 score-correction bias [E]; NULL = zero */
 } oracle_layer;
 
 /* ---------------------------------------------------------------- decoders */
@@ -220,6 +223,74 @@ void oracle_topk(const oracle_cfg *c, const double *logits, int32_t gamma, int32
   }
 }
 
+/* Group-limited routing of the published DeepSeek-V3 models (not in the paper, whose routing is a
+ * plain top-k): s_e = sigmoid(l_e); c_e = s_e + bias_e; the E experts form n_group contiguous
+ * groups; a group's score is the sum of its two largest c (its only c when it has one expert);
+ * the topk_group best groups are kept (score descending, index ascending); among their experts the
+ * top k by (c descending, id ascending) are selected, in that order; weights use the unbiased
+ * scores: w_j = routed_scale * s_j / (sum_j s_j + 1e-20).
+ * gap[t] = the smaller of the two decision margins (k-th vs next c among kept experts; last kept
+ * vs first dropped group score; inf where there is no alternative). */
+void oracle_topk_grouped(const oracle_cfg *c, const double *logits, const float *bias, int32_t gamma,
+                         int32_t *ids, double *w, double *gap) {
+  int E = c->E, k = c->top_k, ng = c->n_group, kg = c->topk_group, gs = E / ng;
+  double *sc = (double *)malloc(sizeof(double) * (size_t)E);
+  double *cc = (double *)malloc(sizeof(double) * (size_t)E);
+  double *G = (double *)malloc(sizeof(double) * (size_t)ng);
+  char *keep = (char *)malloc((size_t)ng);
+  char *taken = (char *)malloc((size_t)E);
+  for (int t = 0; t < gamma; ++t) {
+    const double *l = logits + (int64_t)t * E;
+    for (int e = 0; e < E; ++e) {
+      sc[e] = 1.0 / (1.0 + exp(-l[e]));
+      cc[e] = sc[e] + (bias ? (double)bias[e] : 0.0);
+    }
+    for (int g = 0; g < ng; ++g) {
+      int b1 = -1, b2 = -1;
+      for (int e = g * gs; e < (g + 1) * gs; ++e)
+        if (b1 < 0 || cc[e] > cc[b1]) b1 = e;
+      for (int e = g * gs; e < (g + 1) * gs; ++e)
+        if (e != b1 && (b2 < 0 || cc[e] > cc[b2])) b2 = e;
+      G[g] = cc[b1] + (b2 >= 0 ? cc[b2] : 0.0);
+      keep[g] = 0;
+    }
+    double gmargin = INFINITY;
+    int last_kept = -1;
+    for (int j = 0; j < kg; ++j) {
+      int best = -1;
+      for (int g = 0; g < ng; ++g)
+        if (!keep[g] && (best < 0 || G[g] > G[best])) best = g;
+      keep[best] = 1;
+      last_kept = best;
+    }
+    for (int g = 0; g < ng; ++g)
+      if (!keep[g] && G[last_kept] - G[g] < gmargin) gmargin = G[last_kept] - G[g];
+    memset(taken, 0, (size_t)E);
+    for (int j = 0; j < k; ++j) {
+      int best = -1;
+      for (int e = 0; e < E; ++e) {
+        if (taken[e] || !keep[e / gs]) continue;
+        if (best < 0 || cc[e] > cc[best]) best = e;
+      }
+      taken[best] = 1;
+      ids[t * k + j] = best;
+    }
+    if (gap) {
+      int nxt = -1;
+      for (int e = 0; e < E; ++e) {
+        if (taken[e] || !keep[e / gs]) continue;
+        if (nxt < 0 || cc[e] > cc[nxt]) nxt = e;
+      }
+      double m = (nxt < 0) ? INFINITY : cc[ids[t * k + k - 1]] - cc[nxt];
+      gap[t] = m < gmargin ? m : gmargin;
+    }
+    double den = 0.0;
+    for (int j = 0; j < k; ++j) den += sc[ids[t * k + j]];
+    for (int j = 0; j < k; ++j) w[t * k + j] = c->routed_scale * sc[ids[t * k + j]] / (den + 1e-20);
+  }
+  free(sc); free(cc); free(G); free(keep); free(taken);
+}
+
 /* Eq. 1: the union of the per-token expert sets, and the token->expert
  * grouping.  union_ids ascending [U]; offsets [U+1] exclusive scan of the
  * per-expert token counts in that order; perm[A] lists the assignments
@@ -339,7 +410,8 @@ int32_t oracle_moe_verify(const oracle_cfg *c, const oracle_layer *L, const void
   int32_t *ipm = (int32_t *)malloc(sizeof(int32_t) * (size_t)A);
 
   oracle_router_logits(c, x, L->router_w, gamma, logits);
-  oracle_topk(c, logits, gamma, ids, w, gap);
+  if (c->n_group > 0) oracle_topk_grouped(c, logits, L->router_bias, gamma, ids, w, gap);
+  else oracle_topk(c, logits, gamma, ids, w, gap);
   int U = oracle_union_perm(E, k, gamma, ids, uni, off, pm, ipm);
 
   if (logits_out) memcpy(logits_out, logits, sizeof(double) * (size_t)gamma * (size_t)E);
@@ -403,7 +475,8 @@ int32_t oracle_moe_dense(const oracle_cfg *c, const oracle_layer *L, const void 
   double *w = (double *)malloc(sizeof(double) * (size_t)gamma * (size_t)k);
   double *gate = (double *)calloc((size_t)gamma * (size_t)E, sizeof(double));
   oracle_router_logits(c, x, L->router_w, gamma, logits);
-  oracle_topk(c, logits, gamma, ids, w, NULL);
+  if (c->n_group > 0) oracle_topk_grouped(c, logits, L->router_bias, gamma, ids, w, NULL);
+  else oracle_topk(c, logits, gamma, ids, w, NULL);
   for (int t = 0; t < gamma; ++t)
     for (int j = 0; j < k; ++j) gate[(int64_t)t * E + ids[t * k + j]] = w[t * k + j];
   double *xd = (double *)malloc(sizeof(double) * (size_t)H);
