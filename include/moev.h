@@ -85,6 +85,13 @@ typedef enum {
  *   h = g * sigmoid(1.702 g) * (u + 1),  out = down h + b_down   (weighted by the router weight). */
 typedef enum { MOEV_FFN_SWIGLU = 0, MOEV_FFN_GPTOSS = 1 } moev_ffn_kind;
 
+/* Group-limited routing (n_group > 0), the rule of the published DeepSeek-V3 models; the paper's
+ * routing is the plain top-k.  s_e = sigmoid(logit_e), c_e = s_e + router_bias_e; the E experts
+ * form n_group contiguous groups; a group's score is the sum of its two largest c; the topk_group
+ * best groups are kept (ties: lower index); among their experts the top_k by c (ties: lower id) are
+ * selected and emitted in that order; weights use the unbiased scores:
+ * w_j = routed_scale * s_j / (sum_j s_j + 1e-20). */
+
 typedef struct {
   int32_t H;          /* hidden size; multiple of 32 */
   int32_t I;          /* expert intermediate size; multiple of 32 */
@@ -98,6 +105,8 @@ typedef struct {
   int32_t impl;       /* moev_impl */
   float routed_scale; /* c in the SIGMOID rule; ignored for SOFTMAX */
   int32_t ffn_kind;   /* moev_ffn_kind; MOEV_FFN_GPTOSS needs n_shared == 0 */
+  int32_t n_group;    /* 0 = plain top-k; > 0: group-limited routing (below), needs MOEV_SCORE_SIGMOID, E % n_group == 0 */
+  int32_t topk_group; /* groups kept per token, 1..n_group; top_k <= topk_group * E / n_group */
 } moev_config;
 
 /* One layer's parameters.  Layouts, row-major, last index contiguous:
@@ -115,6 +124,7 @@ typedef struct {
   const void *sh_gate, *sh_up, *sh_down;
   const void *sh_s_gate, *sh_s_up, *sh_s_down;
   const float *b_gate, *b_up, *b_down; /* MOEV_FFN_GPTOSS: fp32 biases [E,I], [E,I], [E,H]; NULL = zero */
+  const float* router_bias;            /* n_group > 0: fp32 score-correction bias [E]; NULL = zero */
 } moev_layer;
 
 /* Outputs.  y and n_active are required; the others are diagnostics and may be NULL.

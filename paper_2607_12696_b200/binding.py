@@ -37,11 +37,12 @@ class _Config(C.Structure):
     _fields_ = [("H", C.c_int32), ("I", C.c_int32), ("E", C.c_int32), ("top_k", C.c_int32),
                 ("n_shared", C.c_int32), ("max_tokens", C.c_int32), ("wfmt", C.c_int32),
                 ("afmt", C.c_int32), ("score", C.c_int32), ("impl", C.c_int32),
-                ("routed_scale", C.c_float), ("ffn_kind", C.c_int32)]
+                ("routed_scale", C.c_float), ("ffn_kind", C.c_int32), ("n_group", C.c_int32),
+                ("topk_group", C.c_int32)]
 
 
 _LAYER_FIELDS = ("router_w", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down",
-                 "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down", "b_gate", "b_up", "b_down")
+                 "sh_gate", "sh_up", "sh_down", "sh_s_gate", "sh_s_up", "sh_s_down", "b_gate", "b_up", "b_down", "router_bias")
 _OUT_FIELDS = ("y", "topk_ids", "topk_w", "union_ids", "offsets", "perm", "n_active")
 
 
@@ -67,10 +68,13 @@ class MoevConfig:
     impl: int = IMPL_AUTO
     routed_scale: float = 1.0
     ffn_kind: int = 0   # FFN_SWIGLU; FFN_GPTOSS = clamped, biased GPT-OSS expert (layer keys b_gate / b_up / b_down)
+    n_group: int = 0    # > 0: DeepSeek group-limited routing (sigmoid scores; layer key router_bias)
+    topk_group: int = 0
 
     def c(self) -> _Config:
         return _Config(self.H, self.I, self.E, self.top_k, self.n_shared, self.max_tokens,
-                       self.wfmt, self.afmt, self.score, self.impl, self.routed_scale, self.ffn_kind)
+                       self.wfmt, self.afmt, self.score, self.impl, self.routed_scale, self.ffn_kind,
+                       self.n_group, self.topk_group)
 
 
 _lib = None

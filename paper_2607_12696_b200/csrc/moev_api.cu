@@ -92,6 +92,10 @@ bool cfg_ok(const moev_config* c, char* why, size_t n) {
   BAD(c->score < 0 || c->score > MOEV_SCORE_SIGMOID, "unknown score function");
   BAD(c->impl < 0 || c->impl > MOEV_IMPL_TCGEN05, "unknown impl");
   BAD(c->ffn_kind < 0 || c->ffn_kind > MOEV_FFN_GPTOSS, "unknown ffn_kind");
+  BAD(c->n_group < 0 || c->topk_group < 0, "n_group and topk_group must be >= 0");
+  BAD(c->n_group > 0 && (c->score != MOEV_SCORE_SIGMOID || c->E % c->n_group || c->topk_group < 1 ||
+                         c->topk_group > c->n_group || c->top_k > c->topk_group * (c->E / c->n_group)),
+      "group-limited routing needs sigmoid scores, E divisible by n_group, 1 <= topk_group <= n_group and top_k <= topk_group * E / n_group");
   BAD(c->ffn_kind == MOEV_FFN_GPTOSS && c->n_shared != 0, "the GPT-OSS expert form has no shared experts");
 #undef BAD
   return true;
@@ -123,6 +127,8 @@ cudaError_t dmalloc(T** p, size_t count) {
 bool route_use_bitmap(const moev_config& c, int gamma) { return route_bitmap_bytes(c.E, gamma) <= kRouteBitmapBudget; }
 // assignments per streamed expert above which the two-phase FFN kernel takes the call
 constexpr int kWideRatio = 8;
+// dynamic shared memory of topk_refine_kernel: three double, three 32-bit and one 8-bit array of E entries
+size_t refine_smem_bytes(int E) { return ((size_t)E * 41 + 15) & ~size_t(15); }
 size_t route_smem(const moev_config& c, int gamma) {
   return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + (route_use_bitmap(c, gamma) ? route_bitmap_bytes(c.E, gamma) : 0);
 }
@@ -519,7 +525,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   cudaEvent_t* ev = nullptr;
   if (c->profile && c->prof_n < kProfSlots) ev = c->ev[c->prof_n++];
   if (ev) cudaEventRecord(ev[0], st);
-  const size_t refine_smem = (size_t)g.E * 16;
+  const size_t refine_smem = refine_smem_bytes(g.E);
   const bool pdl = ev == nullptr;  // event records between the kernels would serialise them anyway
   const size_t rp_smem = router_partial_smem(c->ks);
   if (g.afmt == MOEV_ACT_FP32)
@@ -533,11 +539,12 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   if (g.afmt == MOEV_ACT_FP32)
     launch_k(topk_refine_kernel<MOEV_ACT_FP32>, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x,
              layer->router_w, (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma,
-             g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale);
+             g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale, layer->router_bias, g.n_group, g.topk_group);
   else
     launch_k(topk_refine_kernel<MOEV_ACT_BF16>, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x,
              layer->router_w, (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma,
-             g.H, g.E, g.top_k, c->n_slices, c->router_mma ? 6 * c->ks + c->n_slices + 12 : c->ks, g.score, g.routed_scale);
+             g.H, g.E, g.top_k, c->n_slices, c->router_mma ? 6 * c->ks + c->n_slices + 12 : c->ks, g.score, g.routed_scale,
+             layer->router_bias, g.n_group, g.topk_group);
   if (ev) cudaEventRecord(ev[2], st);
   launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
            g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma), c->wide_ok ? kWideRatio : 0);
@@ -674,7 +681,7 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
   T.tok_scale = tok_scale;
   RouteOut O{};
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const size_t refine_smem = (size_t)cfg->E * 16;
+  const size_t refine_smem = refine_smem_bytes(cfg->E);
   // Nothing has to start at zero: every partial that is read is written by the first kernel of
   // the same call, and the y32 rows are cleared (not accumulated into) by the second.
   const size_t rp_smem = router_partial_smem(ks);  // 17 KB: below the default dynamic limit, no attribute needed
@@ -682,12 +689,14 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
     router_partial_kernel<MOEV_ACT_FP32><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
     topk_refine_kernel<MOEV_ACT_FP32><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
                                                                        gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
-                                                                       cfg->score, cfg->routed_scale);
+                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
+                                                                       cfg->topk_group);
   } else {
     router_partial_kernel<MOEV_ACT_BF16><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
     topk_refine_kernel<MOEV_ACT_BF16><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
                                                                        gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
-                                                                       cfg->score, cfg->routed_scale);
+                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
+                                                                       cfg->topk_group);
   }
   return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
 }

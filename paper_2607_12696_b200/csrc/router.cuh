@@ -321,14 +321,22 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
                                                                      const float* __restrict__ part_w2max,
                                                                      float* __restrict__ y32, int gamma, int H, int E,
                                                                      int k, int n_slices, int ks, int score,
-                                                                     float routed_scale) {
+                                                                     float routed_scale,
+                                                                     const float* __restrict__ router_bias,
+                                                                     int n_group, int topk_group) {
   extern __shared__ double sm_d[];
   double* L = sm_d;                                    // [E] refined logits of the candidates
-  float* l32 = reinterpret_cast<float*>(sm_d + E);     // [E]
-  int32_t* cand = reinterpret_cast<int32_t*>(l32 + E); // [E]
+  double* Cx = sm_d + E;                               // [E] group-limited routing: exact score + bias of the candidates
+  double* Gs = sm_d + 2 * E;                           // [n_group] exact group scores
+  float* l32 = reinterpret_cast<float*>(sm_d + 3 * E); // [E] fp32 logits (group-limited routing: fp32 score + bias)
+  float* v2 = l32 + E;                                 // [n_group] second largest fp32 score + bias of each group
+  int32_t* cand = reinterpret_cast<int32_t*>(v2 + E);  // [E]
+  int32_t* keep = cand + E;                            // [n_group] 1 = group kept
+  uint8_t* inA = reinterpret_cast<uint8_t*>(keep + E); // [E] candidate of the group stage
   __shared__ double red[kRefineWarps][kRefineCand];
   __shared__ float redf[kRefineWarps], redw[kRefineWarps];
   __shared__ int ncand_s;
+  __shared__ unsigned int bmax_s;
   __shared__ float kth_s;
   __shared__ int wcnt_s[kRefineWarps];
   __shared__ __align__(16) float psum[kRefineThreads * 4];  // group sums of the split-K partials
@@ -412,7 +420,9 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   __syncthreads();  // l32, redf, redw complete
   // ---- fp32 top-k by counting: the k-th largest logit is the one preceded by exactly k - 1 others
   // (larger value, or equal value and lower id); E <= kRefineThreads
-  if (2 * E <= kRefineThreads) {  // two threads per expert, each counts over half of the experts
+  if (n_group > 0) {
+    // group-limited routing takes its candidates in two stages, below
+  } else if (2 * E <= kRefineThreads) {  // two threads per expert, each counts over half of the experts
     const int e = tid >> 1, hf = tid & 1;
     const bool act = e < E;
     const float v = act ? l32[e] : 0.f;
@@ -434,6 +444,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     if (rank == k - 1) kth_s = v;
   }
   __syncthreads();
+  float delta = 0.f;  // group-limited routing: error bound of the fp32 score + bias
   {
     float xs = 0.f, wm = 0.f;
     for (int w = 0; w < kRefineWarps; ++w) { xs += redf[w]; wm += redw[w]; }
@@ -443,9 +454,36 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     // element, every accumulation counted twice (the unit's additions may truncate).
     const float n_round = (float)(ks + n_slices + 4);
     const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
-    // ---- candidates: every expert whose exact logit may be >= the exact k-th largest, in ascending id
-    const float thr = kth_s - 2.f * eps;
-    const bool in = tid < E && l32[tid] >= thr;
+    bool in;
+    if (n_group > 0) {
+      // ---- group stage.  c = sigmoid(logit) + bias in fp32 with error <= delta; a group's score is the sum of
+      // its two largest c, so every expert within 2 delta of the group's second largest c is a candidate.
+      const int gsz = E / n_group;
+      const float bv = (tid < E && router_bias) ? __ldg(router_bias + tid) : 0.f;
+      if (tid == 0) bmax_s = 0u;
+      __syncthreads();
+      if (tid < E) atomicMax(&bmax_s, __float_as_uint(fabsf(bv)));
+      const float cv = tid < E ? 1.f / (1.f + expf(-l32[tid])) + bv : 0.f;
+      __syncthreads();
+      if (tid < E) l32[tid] = cv;  // from here on l32 holds c
+      delta = 0.25f * eps + 2e-6f * (1.f + __uint_as_float(bmax_s));
+      __syncthreads();
+      if (tid < E) {
+        const int g = tid / gsz;
+        int rank = 0;
+        for (int e2 = g * gsz; e2 < (g + 1) * gsz; ++e2) {
+          const float u = l32[e2];
+          rank += (u > cv || (u == cv && e2 < tid)) ? 1 : 0;
+        }
+        if (rank == (gsz > 1 ? 1 : 0)) v2[g] = cv;
+      }
+      __syncthreads();
+      in = tid < E && cv >= v2[tid / gsz] - 2.f * delta;
+      if (tid < E) inA[tid] = in ? 1 : 0;
+    } else {
+      // ---- candidates: every expert whose exact logit may be >= the exact k-th largest, in ascending id
+      in = tid < E && l32[tid] >= kth_s - 2.f * eps;
+    }
     const uint32_t m = __ballot_sync(0xffffffffu, in);
     if (lane == 0) wcnt_s[warp] = __popc(m);
     __syncthreads();
@@ -455,16 +493,17 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     if (tid == 0) ncand_s = total;
   }
   __syncthreads();
-  const int ncand = ncand_s;
+  int ncand = ncand_s;
   MOEV_RT_MARK(3);
 
-  // ---- exact (fp64) logits of the candidates, kRefineCand at a time; a thread owns groups of 4 columns
+  // ---- exact (fp64) logits of the candidates [cb, ce), kRefineCand at a time; a thread owns groups of 4 columns
   float amax = 0.f;
-  for (int c0 = 0; c0 < ncand; c0 += kRefineCand) {
+  auto refine_range = [&](int cb, int ce) {
+  for (int c0 = cb; c0 < ce; c0 += kRefineCand) {
     double acc[kRefineCand];
 #pragma unroll
     for (int q = 0; q < kRefineCand; ++q) acc[q] = 0.0;
-    const int nc = min(kRefineCand, ncand - c0);
+    const int nc = min(kRefineCand, ce - c0);
     for (int h4 = tid; h4 < H / 4; h4 += kRefineThreads) {
       double xv[4];
       if constexpr (AFMT == MOEV_ACT_BF16) {
@@ -507,7 +546,75 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     }
     __syncthreads();
   }
+  };
+  refine_range(0, ncand);
   MOEV_RT_MARK(4);
+  if (n_group > 0) {
+    // ---- exact group scores from the group-stage candidates (they contain each group's two largest c)
+    const int gsz = E / n_group, nA = ncand;
+    if (tid < nA) Cx[tid] = 1.0 / (1.0 + exp(-L[tid])) + (router_bias ? (double)__ldg(router_bias + cand[tid]) : 0.0);
+    __syncthreads();
+    if (tid < n_group) {
+      double a1 = 0.0, a2 = 0.0;
+      int n1 = 0;
+      for (int i = 0; i < nA; ++i) {
+        if (cand[i] / gsz != tid) continue;
+        const double v = Cx[i];
+        if (n1 == 0 || v > a1) { a2 = a1; a1 = v; }
+        else if (n1 == 1 || v > a2) a2 = v;
+        ++n1;
+      }
+      Gs[tid] = gsz > 1 ? a1 + a2 : a1;
+    }
+    __syncthreads();
+    if (tid < n_group) {
+      const double v = Gs[tid];
+      int rank = 0;
+      for (int g2 = 0; g2 < n_group; ++g2) rank += (Gs[g2] > v || (Gs[g2] == v && g2 < tid)) ? 1 : 0;
+      keep[tid] = rank < topk_group ? 1 : 0;
+    }
+    __syncthreads();
+    // ---- expert stage: fp32 k-th largest c among the kept groups' experts, then every kept expert within
+    // 2 delta of it that the group stage has not refined already
+    const bool kept = tid < E && keep[tid / gsz] != 0;
+    const float cv = tid < E ? l32[tid] : 0.f;
+    if (kept) {
+      int rank = 0;
+      for (int e2 = 0; e2 < E; ++e2) {
+        if (!keep[e2 / gsz]) continue;
+        const float u = l32[e2];
+        rank += (u > cv || (u == cv && e2 < tid)) ? 1 : 0;
+      }
+      if (rank == k - 1) kth_s = cv;
+    }
+    __syncthreads();
+    const bool in = kept && cv >= kth_s - 2.f * delta && !inA[tid];
+    const uint32_t m = __ballot_sync(0xffffffffu, in);
+    if (lane == 0) wcnt_s[warp] = __popc(m);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < kRefineWarps; ++w) { const int cw = wcnt_s[w]; before += w < warp ? cw : 0; total += cw; }
+    if (in) cand[nA + before + __popc(m & ((1u << lane) - 1u))] = tid;
+    __syncthreads();
+    ncand = nA + total;
+    refine_range(nA, ncand);
+    if (tid >= nA && tid < ncand)
+      Cx[tid] = 1.0 / (1.0 + exp(-L[tid])) + (router_bias ? (double)__ldg(router_bias + cand[tid]) : 0.0);
+    __syncthreads();
+    // ---- exact ranking among the refined experts of the kept groups: larger c first, equal c by lower id
+    for (int c = tid; c < ncand; c += kRefineThreads) {
+      if (!keep[cand[c] / gsz]) continue;
+      const double v = Cx[c];
+      const int e = cand[c];
+      int rank = 0;
+      for (int c2 = 0; c2 < ncand; ++c2) {
+        if (!keep[cand[c2] / gsz]) continue;
+        const double u = Cx[c2];
+        rank += (u > v || (u == v && cand[c2] < e)) ? 1 : 0;
+      }
+      if (rank < k) { sel_v_s[rank] = L[c]; sel_e_s[rank] = e; }
+    }
+  } else {
   // ---- exact ranking by counting: candidate c is preceded by every candidate with a larger
   // logit and, at equal logits, by those with a lower id (candidates are stored in ascending id)
   for (int c = tid; c < ncand; c += kRefineThreads) {
@@ -518,6 +625,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       rank += (u > v || (u == v && c2 < c)) ? 1 : 0;
     }
     if (rank < k) { sel_v_s[rank] = v; sel_e_s[rank] = cand[c]; }
+  }
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
