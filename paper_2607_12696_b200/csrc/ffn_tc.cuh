@@ -66,6 +66,12 @@ __device__ void wide_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, 
                           const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up, const CUtensorMap& tm_sh_down,
                           const CUtensorMap& tm_hq, const CUtensorMap& tm_xu, const Params& P, uint32_t tmem);
 }  // namespace tcw
+namespace tc { struct Params; }
+namespace tcp {  // single-phase schedule without activation producers (ffn_tc_p.cuh)
+__device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
+                             const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up, const CUtensorMap& tm_sh_down,
+                             const CUtensorMap& tm_xq, const tc::Params& P, uint32_t tmem);
+}  // namespace tcp
 namespace tc {
 
 constexpr int kThreads = 352;  // 11 warps
@@ -95,7 +101,8 @@ struct Params {
   const float *sh_s_gate, *sh_s_up, *sh_s_down;  // fp8 block scales (shared)
   int32_t* status;
   int32_t gamma, H, I, A;
-  const int32_t* wide;  // non-null and non-zero: the two-phase kernel (ffn_tc_wide.cuh) runs this call, this one exits
+  const int32_t* wide;  // non-null and non-zero: the two-phase schedule (ffn_tc_wide.cuh) runs this call
+  int32_t xq_ready;     // fp8: the routing kernels wrote the quantised activations: run the schedule of ffn_tc_p.cuh
 #ifdef MOEV_TC_STATS
   unsigned long long* stats;  // [grid][16] cycles the MMA thread spent per wait / issue class (debug builds)
 #endif
@@ -223,7 +230,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_constant__ CUtensorMap tm_up,
                       const __grid_constant__ CUtensorMap tm_down, const __grid_constant__ CUtensorMap tm_sh_gate,
                       const __grid_constant__ CUtensorMap tm_sh_up, const __grid_constant__ CUtensorMap tm_sh_down,
-                      const __grid_constant__ CUtensorMap tm_hq, const __grid_constant__ CUtensorMap tm_xu, const Params P,
+                      const __grid_constant__ CUtensorMap tm_hq, const __grid_constant__ CUtensorMap tm_xu,
+                      const __grid_constant__ CUtensorMap tm_xq, const __grid_constant__ Params P,
                       const __grid_constant__ tcw::Params W) {
   using F = Fmt<WFMT>;
   constexpr bool kFp8 = WFMT == MOEV_W_FP8E4M3_B128;
@@ -283,6 +291,19 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       }
       return;
     }
+#ifndef MOEV_FP8_FOLD_SCALE
+    if (P.xq_ready) {
+      // quantised activations are available: the schedule without activation producers
+      tcp::promote_body(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem);
+      ptx::tc_fence_before();
+      __syncthreads();
+      if (warp == 0) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem, kTmemCols);
+      }
+      return;
+    }
+#endif
   }
   const int n_ids = n_units * ((n_slices + 1) & ~1);
   volatile int* abortp = &S.abort_flag;

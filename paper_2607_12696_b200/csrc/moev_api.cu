@@ -9,6 +9,7 @@
 #include "ffn_tc.cuh"
 #include "ffn_tc_mx.cuh"
 #include "ffn_tc_wide.cuh"
+#include "ffn_tc_p.cuh"
 #include "router.cuh"
 #include "select.cuh"
 
@@ -257,6 +258,7 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
 #endif
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
   P.wide = c->wide_ok ? c->T.wide : nullptr;
+  P.xq_ready = (c->wide_ok && c->T.xq) ? 1 : 0;
   // arguments of the two-phase schedule, which the kernel switches to when the grouping kernel's
   // flag says that the call has many tokens per streamed expert (fp8 only)
   tcw::Params W{};
@@ -269,7 +271,7 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   W.xq = c->T.xq; W.xu = c->xu;
   launch_k(tc::grouped_ffn_tc_kernel<WFMT>, dim3(c->n_sm), dim3(tc::kThreads), tc::kSmemBytes, st, ev == nullptr,
            tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], c->wide_ok ? c->tm_hq : tm->map[0],
-           c->wide_ok ? c->tm_xu : tm->map[0], P, W);
+           c->wide_ok ? c->tm_xu : tm->map[0], c->wide_ok ? c->tm_xq : tm->map[0], P, W);
   if (ev) cudaEventRecord(ev[4], st);
   if (ev) cudaEventRecord(ev[5], st);
 }
