@@ -804,7 +804,12 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       *T.n_units = base + sc;
       *T.task_counter = 0;
       // many tokens per streamed expert: the two-phase FFN schedule (wide_ratio = 0: not available)
-      if (T.wide) *T.wide = (wide_ratio > 0 && (A + n_shared * gamma) > wide_ratio * (U + n_shared)) ? 1 : 0;
+      // (measured switch-over: above 8 assignments per streamed expert for small unions, where the weight stream
+      // is short, above 12 for large ones, where the two-phase schedule's re-streaming per 32-token unit costs more)
+      if (T.wide) {
+        const int ut = U + n_shared, ratio = ut < 100 ? wide_ratio : wide_ratio + wide_ratio / 2;
+        *T.wide = (wide_ratio > 0 && (A + n_shared * gamma) > ratio * ut) ? 1 : 0;
+      }
     }
     if (T.unit_done) {
       __shared__ int n_units_s;
