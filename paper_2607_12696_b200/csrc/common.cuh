@@ -38,8 +38,11 @@ struct Tables {
   float* slot_w;       // [A]   its routing weight
   int32_t* n_active;   // [1]
   float* tok_scale;    // [gamma] power of two bringing the token's max |x| into [64,128)
-  uint8_t* xq;         // [gamma, 2, xq_stride] e4m3 hi / lo terms of x * tok_scale (MXFP4 tensor-core path), or null
-  int32_t xq_stride;   // bytes per row: H, plus a 128-byte tail block when H % 128 != 0
+  uint8_t* xq;         // quantised activations x * tok_scale, written once per token for the tensor-core kernels, or null:
+                       // xq_e2m1 = 0: [gamma, 2, xq_stride] e4m3 hi / lo terms (fp8 weights);
+                       // xq_e2m1 = 1: [gamma, 4, xq_stride] packed e2m1 terms 8^-j (MXFP4 weights)
+  int32_t xq_stride;   // bytes per row: H (e4m3) or H / 2 (e2m1)
+  int32_t xq_e2m1;
   Unit* units;         // [max_units]
   int32_t* n_units;    // [1]
   int32_t* task_counter; // [1] dynamic task scheduler of the tensor-core FFN, zeroed per call
@@ -84,6 +87,22 @@ __device__ __forceinline__ void split4_e4m3(const float (&v)[4], uint32_t& hi, u
     hi |= (uint32_t)hc << (16 * p);
     lo |= (uint32_t)lc << (16 * p);
   }
+}
+
+// Two scaled values (|v| < 4) -> four e2m1 terms each, v ~ q0 + q1 / 8 + q2 / 64 + q3 / 512: byte
+// j of the result holds term j, a in the low nibble and b in the high one.
+__device__ __forceinline__ uint32_t split2_e2m1(float a, float b) {
+  uint32_t out = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const __nv_fp4x2_storage_t c = __nv_cvt_float2_to_fp4x2(make_float2(a, b), __NV_E2M1, cudaRoundNearest);
+    __half2_raw hr = __nv_cvt_fp4x2_to_halfraw2(c, __NV_E2M1);
+    const float2 f = __half22float2(*reinterpret_cast<__half2*>(&hr));
+    a = (a - f.x) * 8.f;
+    b = (b - f.y) * 8.f;
+    out |= (uint32_t)c << (8 * j);
+  }
+  return out;
 }
 
 // h from the gate / up pre-activations (biases already added): bias-free SwiGLU, or the GPT-OSS

@@ -153,10 +153,10 @@ EncodeTiledFn encode_tiled_fn() {
 // Can the tensor-core kernel run this shape?  (Otherwise AUTO resolves to the SIMT kernels.)
 bool tc_eligible(const moev_config& c) {
   if (c.afmt != MOEV_ACT_BF16) return false;
-  if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: K axes in half chunks of 64, >= 4 chunks per row
+  if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: rows of whole 32-byte MMA pieces, >= 2 K chunks per row
     return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 512 && c.I >= 128 &&
            128 * (c.H / 32) <= tcmx::kScStageBytes &&  // a slice's gate/up scale block is staged in shared memory,
-           (c.H + 127) / 128 <= tcmx::kDownWords;         // and one word per W_down row
+           (c.H + 127) / 128 <= tcmx::kDownTiles;         // and the scale words of the W_down rows
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
   if (c.ffn_kind != MOEV_FFN_SWIGLU) return false;  // the biased, clamped form: MXFP4 tensor-core kernel or CUDA cores
   if (c.H % 128 || c.I % 128) return false;
@@ -182,19 +182,19 @@ bool encode_weight_map(CUtensorMap* m, const moev_config& c, const void* ptr, in
   return r == CUDA_SUCCESS;
 }
 
-// MXFP4: [n_mat, N, K] 4-bit codes -> 4-D map {128 elements, half chunks of 64 (stride 32 bytes),
-// rows, matrices} with the "16 x U4 in 16 bytes" element type (expands into the padded layout
-// kind::mxf8f6f4 reads), 128B swizzle.
-bool encode_weight_map_mx(CUtensorMap* m, const void* ptr, int n_mat, int N, int K) {
+// MXFP4: [n_mat, N, K] packed 4-bit codes as bytes -> 3-D map {K / 2 bytes, rows, matrices}; the
+// box is 128 rows x 128 bytes (gate / up, 128-byte swizzle) or 128 rows x 64 bytes (W_down: the
+// 128-column slice of a task, 64-byte swizzle), the layouts kind::mxf4 reads.
+bool encode_weight_map_mx(CUtensorMap* m, const void* ptr, int n_mat, int N, int K, bool down) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
-  cuuint64_t dims[4] = {128, (cuuint64_t)(K / 64 - 1), (cuuint64_t)N, (cuuint64_t)n_mat};
-  cuuint64_t strides[3] = {32, (cuuint64_t)K / 2, (cuuint64_t)K / 2 * (cuuint64_t)N};
-  cuuint32_t box[4] = {128, 1, 128, 1};
-  cuuint32_t estr[4] = {1, 1, 1, 1};
-  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B, 4, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  cuuint64_t dims[3] = {(cuuint64_t)K / 2, (cuuint64_t)N, (cuuint64_t)n_mat};
+  cuuint64_t strides[2] = {(cuuint64_t)K / 2, (cuuint64_t)K / 2 * (cuuint64_t)N};
+  cuuint32_t box[3] = {down ? 64u : 128u, 128, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, down ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
@@ -208,8 +208,9 @@ const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
   t.valid = false;
   const moev_config& g = c->cfg;
   auto enc = [&](CUtensorMap* m, const void* ptr, int n_mat, int N, int K) {
-    if (reinterpret_cast<uintptr_t>(ptr) & 31u) return false;  // the 4-bit element type needs 32-byte alignment
-    return g.wfmt == MOEV_W_MXFP4 ? encode_weight_map_mx(m, ptr, n_mat, N, K) : encode_weight_map(m, g, ptr, n_mat, N, K);
+    if (reinterpret_cast<uintptr_t>(ptr) & 31u) return false;
+    return g.wfmt == MOEV_W_MXFP4 ? encode_weight_map_mx(m, ptr, n_mat, N, K, m == &t.map[2] || m == &t.map[5])
+                                  : encode_weight_map(m, g, ptr, n_mat, N, K);
   };
   bool ok = enc(&t.map[0], L->w_gate, g.E, g.I, g.H) && enc(&t.map[1], L->w_up, g.E, g.I, g.H) &&
             enc(&t.map[2], L->w_down, g.E, g.H, g.I);
@@ -406,14 +407,18 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     }
   }
   if (c->resolved_impl == MOEV_IMPL_TCGEN05 && (cfg->wfmt == MOEV_W_MXFP4 || c->wide_ok)) {
-    // quantised activations (two e4m3 terms per element), loaded by TMA as the MMA's N operand
-    c->T.xq_stride = cfg->H + (cfg->H % 128 ? 128 : 0);
-    ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->T.xq), 2 * G * (size_t)c->T.xq_stride) == cudaSuccess;
+    // quantised activations, loaded by TMA as the MMA's N operand: two e4m3 term rows of H bytes
+    // per token (fp8 weights) or four packed e2m1 term rows of H / 2 bytes (MXFP4 weights)
+    const bool mx = cfg->wfmt == MOEV_W_MXFP4;
+    const size_t rows_per_tok = mx ? 4 : 2;
+    c->T.xq_e2m1 = mx ? 1 : 0;
+    c->T.xq_stride = mx ? cfg->H / 2 : cfg->H;
+    ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->T.xq), rows_per_tok * G * (size_t)c->T.xq_stride) == cudaSuccess;
     EncodeTiledFn fn = encode_tiled_fn();
     if (ok && fn) {
-      cuuint64_t dims[2] = {(cuuint64_t)c->T.xq_stride, (cuuint64_t)(2 * G)};
+      cuuint64_t dims[2] = {(cuuint64_t)c->T.xq_stride, (cuuint64_t)(rows_per_tok * G)};
       cuuint64_t strides[1] = {(cuuint64_t)c->T.xq_stride};
-      cuuint32_t box[2] = {128, 2};
+      cuuint32_t box[2] = {128, (cuuint32_t)rows_per_tok};
       cuuint32_t estr[2] = {1, 1};
       ok = fn(&c->tm_xq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c->T.xq, dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,

@@ -632,39 +632,43 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   if (lane == 0) redf[warp] = amax;
   __syncthreads();
 
-  // ---- MXFP4 tensor-core path: the two e4m3 terms (hi + lo / 16) of x * 2^p_t, the activation
-  // operand of every expert of this call, are formed once per token here (warps other than the
-  // ranking warp).  A ragged last K chunk reads its operand from a tail block after the row:
-  // 64 zeros, then the last 64 elements.
+  // ---- tensor-core paths with a quantised activation operand: x * 2^p_t is split once per
+  // token here (warps other than the ranking warp) into two e4m3 terms hi + lo / 16 (fp8
+  // weights), or into four packed e2m1 terms with weights 8^-j (MXFP4 weights; |x| 2^p_t < 4).
   if (AFMT == MOEV_ACT_BF16 && T.xq != nullptr && warp > 0) {
     float am = 0.f;
     for (int w = 0; w < kRefineWarps; ++w) am = fmaxf(am, redf[w]);
     int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
     ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
-    const float ts = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
+    const float ts = __uint_as_float((uint32_t)((T.xq_e2m1 ? 1 : 6) - ex + 127) << 23);
     const uint16_t* xr = static_cast<const uint16_t*>(x) + (size_t)t * H;
-    uint8_t* hi_row = T.xq + (size_t)(2 * t) * T.xq_stride;
-    uint8_t* lo_row = hi_row + T.xq_stride;
-    const bool tail = T.xq_stride > H;
-    const int n4 = H / 4 + (tail ? 32 : 0);  // groups of 4 elements, then the 128-byte tail block
-    for (int i = tid - 32; i < n4; i += kRefineThreads - 32) {
-      int src = i * 4, dst = i * 4;
-      bool zero = false;
-      if (i >= H / 4) {
-        const int j = i - H / 4;  // 0..31 within the tail block
-        dst = H + j * 4;
-        zero = j < 16;
-        src = H - 64 + (j - 16) * 4;
+    if (T.xq_e2m1) {
+      uint8_t* rows = T.xq + (size_t)(4 * t) * T.xq_stride;
+      for (int i = tid - 32; i < H / 8; i += kRefineThreads - 32) {  // 8 elements -> 4 bytes of every term row
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(xr + i * 8));
+        const uint32_t in[4] = {q.x, q.y, q.z, q.w};
+        uint32_t term[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          const uint32_t sp = split2_e2m1(__uint_as_float(in[p] << 16) * ts, __uint_as_float(in[p] & 0xffff0000u) * ts);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) term[j] |= ((sp >> (8 * j)) & 0xffu) << (8 * p);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) *reinterpret_cast<uint32_t*>(rows + (size_t)j * T.xq_stride + i * 4) = term[j];
       }
-      uint32_t hi = 0, lo = 0;
-      if (!zero) {
-        const uint2 q = __ldg(reinterpret_cast<const uint2*>(xr + src));
+    } else {
+      uint8_t* hi_row = T.xq + (size_t)(2 * t) * T.xq_stride;
+      uint8_t* lo_row = hi_row + T.xq_stride;
+      for (int i = tid - 32; i < H / 4; i += kRefineThreads - 32) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(xr + i * 4));
         float v[4] = {__uint_as_float(q.x << 16) * ts, __uint_as_float(q.x & 0xffff0000u) * ts,
                       __uint_as_float(q.y << 16) * ts, __uint_as_float(q.y & 0xffff0000u) * ts};
+        uint32_t hi, lo;
         split4_e4m3(v, hi, lo);
+        *reinterpret_cast<uint32_t*>(hi_row + i * 4) = hi;
+        *reinterpret_cast<uint32_t*>(lo_row + i * 4) = lo;
       }
-      *reinterpret_cast<uint32_t*>(hi_row + dst) = hi;
-      *reinterpret_cast<uint32_t*>(lo_row + dst) = lo;
     }
   }
 
@@ -676,7 +680,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       for (int w = 0; w < kRefineWarps; ++w) am = fmaxf(am, redf[w]);
       int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
       ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
-      T.tok_scale[t] = __uint_as_float((uint32_t)(6 - ex + 127) << 23);
+      T.tok_scale[t] = __uint_as_float((uint32_t)((T.xq != nullptr && T.xq_e2m1 ? 1 : 6) - ex + 127) << 23);
     }
     // router weights of the k selected experts (lane j owns the j-th); binary32 is ample for
     // weights that are compared to 1e-5: the differences are formed in fp64 first
