@@ -74,19 +74,15 @@ constexpr int kTileBytes = kStages * kStageBytes + kStages * kBTileBytes + kHTil
 constexpr int kCtlBytes = 2 * 1024;
 constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
 
-// Task id -> (unit, slice).  Ids enumerate (slice group, unit, member) with the member fastest:
-// the kGroup slices of a group of one unit are taken back to back by kGroup CTAs, which then read
-// neighbouring 64-byte pieces of the same rows of W_down at about the same time.
-#ifndef MOEV_MX_GROUP
-#define MOEV_MX_GROUP 4
-#endif
-constexpr int kGroup = MOEV_MX_GROUP;
-__device__ __forceinline__ TaskDesc decode_task(int id, int n_units, int n_slices) {
+// Task id -> (unit, slice), unit-major: the slices of one unit are taken back to back by as many
+// CTAs, which then read neighbouring 64-byte pieces of the same rows of W_down (and neighbouring
+// scale words of those rows) at about the same time, so that the sectors and lines they share are
+// fetched from HBM once (ids interleaved over units read 1.25 x the algorithmic bytes).
+__device__ __forceinline__ TaskDesc decode_task(int id, int /*n_units*/, int n_slices) {
   TaskDesc t;
-  const int grp = id / kGroup;
-  t.unit = grp % n_units;
-  t.slice = (grp / n_units) * kGroup + (id % kGroup);
-  t.valid = t.slice < n_slices;
+  t.unit = id / n_slices;
+  t.slice = id - t.unit * n_slices;
+  t.valid = true;
   return t;
 }
 
@@ -248,7 +244,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int n_units = *P.n_units;
-  const int n_ids = n_units * kGroup * ((n_slices + kGroup - 1) / kGroup);
+  const int n_ids = n_units * n_slices;
   volatile int* abortp = &S.abort_flag;
 
   // Phase order of the weight stream, the MMAs and the producers (GU = gate/up phase, D = down
