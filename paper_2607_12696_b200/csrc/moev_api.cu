@@ -53,6 +53,7 @@ struct moev_ctx {
   uint8_t* hq = nullptr;  // its scratch: quantised h tiles [max_units][n_slices][64][128] ...
   float* hq_f = nullptr;  // ... and their scales [max_units][n_slices][32]
   uint8_t* xu = nullptr;  // per-unit operand tiles [max_units][H / 128][64][128]
+  uint8_t* hexp = nullptr;  // MXFP4 tensor-core path: block exponents of h, [max_units * 8][tcmx::kExpStride] (hq holds the h terms)
   size_t max_units = 0;
   CUtensorMap tm_hq, tm_xu;
   CUtensorMap tm_xq;  // MXFP4 tensor-core path: the [2 * max_tokens, xq_stride] byte array T.xq, box 128 x 2
@@ -153,10 +154,9 @@ EncodeTiledFn encode_tiled_fn() {
 // Can the tensor-core kernel run this shape?  (Otherwise AUTO resolves to the SIMT kernels.)
 bool tc_eligible(const moev_config& c) {
   if (c.afmt != MOEV_ACT_BF16) return false;
-  if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: rows of whole 32-byte MMA pieces, >= 2 K chunks per row
-    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 512 && c.I >= 128 &&
-           128 * (c.H / 32) <= tcmx::kScStageBytes &&  // a slice's gate/up scale block is staged in shared memory,
-           (c.H + 127) / 128 <= tcmx::kDownTiles;         // and the scale words of the W_down rows
+  if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: rows of whole 32-byte MMA pieces; a task's scale rows are staged in shared memory
+    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 256 && c.I >= 128 &&
+           128 * (c.H / 32) <= tcmx::kScStageBytes && 128 * (c.I / 32) <= tcmx::kScStageBytes;
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
   if (c.ffn_kind != MOEV_FFN_SWIGLU) return false;  // the biased, clamped form: MXFP4 tensor-core kernel or CUDA cores
   if (c.H % 128 || c.I % 128) return false;
@@ -182,19 +182,18 @@ bool encode_weight_map(CUtensorMap* m, const moev_config& c, const void* ptr, in
   return r == CUDA_SUCCESS;
 }
 
-// MXFP4: [n_mat, N, K] packed 4-bit codes as bytes -> 3-D map {K / 2 bytes, rows, matrices}; the
-// box is 128 rows x 128 bytes (gate / up, 128-byte swizzle) or 128 rows x 64 bytes (W_down: the
-// 128-column slice of a task, 64-byte swizzle), the layouts kind::mxf4 reads.
-bool encode_weight_map_mx(CUtensorMap* m, const void* ptr, int n_mat, int N, int K, bool down) {
+// MXFP4: [n_mat, N, K] packed 4-bit codes as bytes -> 3-D map {K / 2 bytes, rows, matrices}, box
+// 128 rows x 128 bytes with the 128-byte swizzle: the layout kind::mxf4 reads.
+bool encode_weight_map_mx(CUtensorMap* m, const void* ptr, int n_mat, int N, int K) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)K / 2, (cuuint64_t)N, (cuuint64_t)n_mat};
   cuuint64_t strides[2] = {(cuuint64_t)K / 2, (cuuint64_t)K / 2 * (cuuint64_t)N};
-  cuuint32_t box[3] = {down ? 64u : 128u, 128, 1};
+  cuuint32_t box[3] = {128, 128, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, down ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
@@ -209,7 +208,7 @@ const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
   const moev_config& g = c->cfg;
   auto enc = [&](CUtensorMap* m, const void* ptr, int n_mat, int N, int K) {
     if (reinterpret_cast<uintptr_t>(ptr) & 31u) return false;
-    return g.wfmt == MOEV_W_MXFP4 ? encode_weight_map_mx(m, ptr, n_mat, N, K, m == &t.map[2] || m == &t.map[5])
+    return g.wfmt == MOEV_W_MXFP4 ? encode_weight_map_mx(m, ptr, n_mat, N, K)
                                   : encode_weight_map(m, g, ptr, n_mat, N, K);
   };
   bool ok = enc(&t.map[0], L->w_gate, g.E, g.I, g.H) && enc(&t.map[1], L->w_up, g.E, g.I, g.H) &&
@@ -282,7 +281,8 @@ void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   const moev_config& g = c->cfg;
   tcmx::Params P{};
   P.units = c->T.units; P.n_units = c->T.n_units; P.task_counter = c->T.task_counter;
-  P.slot_token = c->T.slot_token; P.slot_w = c->T.slot_w; P.tok_scale = c->T.tok_scale; P.x = x; P.y32 = c->y32;
+  P.slot_token = c->T.slot_token; P.slot_w = c->T.slot_w; P.tok_scale = c->T.tok_scale; P.y32 = c->y32;
+  P.hq = c->hq; P.hexp = c->hexp; P.unit_done = c->T.unit_done; P.hq_stride = g.I / 2;
   P.s_gate = static_cast<const uint8_t*>(L->s_gate); P.s_up = static_cast<const uint8_t*>(L->s_up);
   P.s_down = static_cast<const uint8_t*>(L->s_down);
   P.sh_s_gate = static_cast<const uint8_t*>(L->sh_s_gate); P.sh_s_up = static_cast<const uint8_t*>(L->sh_s_up);
@@ -293,7 +293,7 @@ void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.stats = c->tc_stats;
 #endif
   launch_k(tcmx::grouped_ffn_mx_kernel, dim3(c->n_sm), dim3(tcmx::kThreads), tcmx::kSmemBytes, st, ev == nullptr,
-           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], c->tm_xq, P);
+           tm->map[0], tm->map[1], tm->map[2], tm->map[3], tm->map[4], tm->map[5], c->tm_xq, c->tm_hq, P);
   if (ev) cudaEventRecord(ev[4], st);
 }
 
@@ -381,6 +381,28 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     ok = ok && dmalloc(&c->T.units, max_units) == cudaSuccess;
     const int n_slices = cfg->I / 128;
     c->wide_ok = c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_FP8E4M3_B128 && n_slices <= tcw::kMaxSlices;
+    if (c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_MXFP4) {
+      // two-phase MXFP4 kernel: per-unit progress counters, the h terms ([32 rows per unit, I / 2
+      // bytes], loaded by TMA as the down projection's N operand) and their block exponents
+      ok = ok && dmalloc(&c->T.unit_done, 2 * max_units) == cudaSuccess;
+      c->max_units = max_units;
+      ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->hq), max_units * 32 * (size_t)(cfg->I / 2)) == cudaSuccess;
+      ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->hexp), max_units * 8 * (size_t)tcmx::kExpStride) == cudaSuccess;
+      ok = ok && cudaMemset(c->hq, 0, max_units * 32 * (size_t)(cfg->I / 2)) == cudaSuccess;
+      ok = ok && cudaMemset(c->hexp, 0x7F, max_units * 8 * (size_t)tcmx::kExpStride) == cudaSuccess;
+      EncodeTiledFn fn = encode_tiled_fn();
+      if (ok && fn) {
+        cuuint64_t dims[2] = {(cuuint64_t)(cfg->I / 2), (cuuint64_t)(max_units * 32)};
+        cuuint64_t strides[1] = {(cuuint64_t)(cfg->I / 2)};
+        cuuint32_t box[2] = {128, 32};
+        cuuint32_t estr[2] = {1, 1};
+        ok = fn(&c->tm_hq, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, c->hq, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+      } else {
+        ok = false;
+      }
+    }
     if (c->wide_ok) {
       ok = ok && dmalloc(&c->T.wide, 1) == cudaSuccess;
       ok = ok && dmalloc(&c->T.unit_done, 2 * max_units) == cudaSuccess;
@@ -475,7 +497,7 @@ moev_status moev_destroy(moev_ctx* c) {
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
   cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->T.task_counter); cudaFree(c->hbuf); cudaFree(c->y32);
-  cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f); cudaFree(c->xu);
+  cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f); cudaFree(c->xu); cudaFree(c->hexp);
   cudaFree(c->x_stage); cudaFree(c->y_stage);
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)
