@@ -67,11 +67,12 @@ constexpr int kColSfBx = kColSf + 16 * kStages;
 constexpr int kColSfBh = kColSfBx + 4;
 constexpr int kSfBhCols = 4 * 2 * kMaxChunks;
 static_assert(kColSfBh + 2 * kSfBhCols <= kTmemCols, "TMEM budget");
-// staged scale bytes of a task: [tile 0, tile 1][128 rows x K/32 bytes], double-buffered
+// staged scale bytes of a task: [tile 0, tile 1][128 rows x K/32 bytes], three buffers (the task in
+// progress, the next one, and the one being copied for the task after it)
 constexpr int kScStageBytes = 11776;  // >= 128 * (K / 32) bytes, K <= 2944
 constexpr int kExpStride = 96;        // bytes per (unit, token) row of the h block exponents (I / 32 <= 92, 16-byte multiple)
 constexpr int kSfAtomBytes = 512;     // scale factors of 128 rows x 128 elements as tcgen05.cp reads them: 32 rows of 16 bytes
-constexpr int kTileBytes = kStages * kStageBytes + kStages * kBTileBytes + 4 * kScStageBytes + kStages * 4 * kSfAtomBytes;
+constexpr int kTileBytes = kStages * kStageBytes + kStages * kBTileBytes + 6 * kScStageBytes + kStages * 4 * kSfAtomBytes;
 constexpr int kCtlBytes = 2 * 1024;
 constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
 
@@ -116,7 +117,7 @@ struct Params {
 
 struct Smem {
   uint64_t w_full[kStages], w_empty[kStages];
-  uint64_t aux_full[kStages];  // weight (and, first stage of a phase-2 task, activation) scale factors are in TMEM
+  uint64_t aux_full[kStages];  // the stage's scale-factor atoms are in shared memory (and the task's h scale factors in TMEM)
   uint64_t acc_full[2], acc_empty[2];
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar, pr_bar;
@@ -197,7 +198,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   uint8_t* w_ring = base;
   uint8_t* b_tiles = w_ring + kStages * kStageBytes;
   uint8_t* sc_stage = b_tiles + kStages * kBTileBytes;  // [buffer][tile] scale rows of a task (16-byte aligned)
-  uint8_t* sf_atoms = sc_stage + 4 * kScStageBytes;     // [stage][tile][word] scale-factor atoms
+  uint8_t* sf_atoms = sc_stage + 6 * kScStageBytes;     // [stage][tile][word] scale-factor atoms
   static_assert(kBTileBytes % 1024 == 0 && kStageBytes == 2 * 16384, "tile layout");
   static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
   static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
@@ -215,7 +216,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     // barriers completed by tcgen05.commit of both MMA issuers count 2; barriers completed by a
     // 4-warp role group count 4 (one elected arrival per warp)
     for (int i = 0; i < kStages; ++i) {
-      ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); ptx::mbar_init(&S.aux_full[i], 4);
+      ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); ptx::mbar_init(&S.aux_full[i], 1);
     }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.acc_full[i], 2); ptx::mbar_init(&S.acc_empty[i], 4); }
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
@@ -515,7 +516,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #endif
     // The scale rows of a task's two weight tiles are two contiguous blocks of HBM (128 rows x
     // K/32 bytes each); they are staged in shared memory with 16-byte asynchronous copies one
-    // task ahead (two buffers).
+    // task ahead.
     struct Blocks { const uint8_t* src[2]; int rows[2]; int kb; };
     auto blocks_of = [&](const Task& t) -> Blocks {
       const Unit u = P.units[t.unit];
@@ -537,8 +538,8 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       return b;
     };
     auto stage_scales = [&](int id, int buf) {
-      // every producer thread has finished the task that last used this buffer
-      if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) return;
+      // the buffer was last read by the task three back: every producer thread has finished it,
+      // since all of them have met at the start of the task after it
       const Blocks b = blocks_of(decode_task(id, n_p1, n_slices, n_pairs));
 #pragma unroll
       for (int tl = 0; tl < 2; ++tl) {
@@ -549,76 +550,109 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    auto run = [&](int id, int buf, bool staged_after) {
+    // Activation-side scale factors of a whole phase-2 task: column n = 4 r + j is term j of
+    // token r, scale 2^(e - 1) 8^-j per 32-block of I, two words per K chunk.  Built one task
+    // ahead, when the previous task's stages have been handed over, so that the task's first
+    // stage does not wait for them: the exponent bytes are fetched (after the unit's progress
+    // counter, acquire) and written to TMEM.  `tc` is the task's position in this CTA's sequence; the
+    // columns of its parity are free once the accumulators of the task two back have been drained.
+    uint4 hexp_v[2 * kMaxChunks / 4];
+    auto fetch_exp = [&](int id) {
+      const Task t = decode_task(id, n_p1, n_slices, n_pairs);
+      if (t.phase != 2) return;
+      int w = 0;
+      if (lane == 0) w = wait_unit_done(P.unit_done + t.unit, n_slices, abortp, P.status) ? 1 : 0;
+      ok = __shfl_sync(0xffffffffu, w, 0) != 0;
+      __syncwarp();  // lane 0's acquire orders the other lanes' reads of the exponents too
+      if (!ok) return;
+      const uint4* ep = reinterpret_cast<const uint4*>(P.hexp + (size_t)(8 * t.unit + (lane >> 2)) * kExpStride);
+#pragma unroll
+      for (int v = 0; v < 2 * kMaxChunks / 4; ++v) hexp_v[v] = (16 * v < kb2) ? __ldcg(ep + v) : make_uint4(0, 0, 0, 0);
+    };
+    auto store_sfbh = [&](int id, uint32_t tc) {
+      const Task t = decode_task(id, n_p1, n_slices, n_pairs);
+      if (t.phase != 2) return;
+      const int par = tc & 1;
+#ifdef MOEV_TC_STATS
+      const long long pb0 = clock64();
+#endif
+      ok = warp_wait(&S.acc_empty[par], ((tc >> 1) & 1) ^ 1, abortp, P.status);
+      if (!ok) return;
+      ptx::tc_fence_after();
+      const int r = lane >> 2, j = lane & 3;
+      const int m = P.units[t.unit].m;
+      const uint32_t sub = (uint32_t)(3 * j) * 0x01010101u;
+#pragma unroll
+      for (int v = 0; v < 2 * kMaxChunks / 4; ++v) {
+        const uint32_t in[4] = {hexp_v[v].x, hexp_v[v].y, hexp_v[v].z, hexp_v[v].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int blk = 16 * v + 4 * c;  // kb2 is even: the word's byte pairs lie inside the row or past its end
+          uint32_t x = __vsubus4(in[c], sub);
+          if (blk + 2 >= kb2) x = (x & 0x0000FFFFu) | 0x7F7F0000u;
+          if (blk >= kb2 || r >= m) x = 0x7F7F7F7Fu;
+          tmem_st1(tm_quarter + kColSfBh + par * kSfBhCols + 4 * (4 * v + c), x);
+        }
+      }
+      tmem_st_wait();
+      ptx::tc_fence_before();
+#ifdef MOEV_TC_STATS
+      pst[1] += clock64() - pb0;
+#endif
+    };
+    auto run = [&](int id, int buf, int id_next) {
+      const bool staged_after = id_next >= 0;
       const Task t = decode_task(id, n_p1, n_slices, n_pairs);
       const Blocks b = blocks_of(t);
       const int KC = t.phase == 1 ? KC1 : KC2;
-      const int par = tcount & 1;
       // this task's staged scales have landed (every thread waits for its own copies, then all meet);
       // a copy group committed after them (the next task's) may stay in flight
       if (staged_after) asm volatile("cp.async.wait_group 1;" ::: "memory");
       else asm volatile("cp.async.wait_group 0;" ::: "memory");
       if (!(ok = group_sync(&S.pr_bar, gph, abortp, P.status))) return;
-#ifdef MOEV_TC_STATS
-      const long long pb0 = clock64();
-#endif
-      if (t.phase == 2) {
-        // activation-side scale factors of the whole task: column n = 4 r + j is term j of token
-        // r, scale 2^(e - 1) 8^-j per 32-block of I, two words per K chunk.  The columns of this
-        // parity are free once the accumulators of the task two back have been drained.
-        ok = warp_wait(&S.acc_empty[par], ((tcount >> 1) & 1) ^ 1, abortp, P.status);
-        if (!ok) return;
-        int w = 0;
-        if (lane == 0) w = wait_unit_done(P.unit_done + t.unit, n_slices, abortp, P.status) ? 1 : 0;
-        ok = __shfl_sync(0xffffffffu, w, 0) != 0;
-        __syncwarp();  // lane 0's acquire orders the other lanes' reads of the exponents too
-        if (!ok) return;
-        ptx::tc_fence_after();
-        const int r = lane >> 2, j = lane & 3;
-        const int m = P.units[t.unit].m;
-        const uint4* ep = reinterpret_cast<const uint4*>(P.hexp + (size_t)(8 * t.unit + r) * kExpStride);
-        const uint32_t sub = (uint32_t)(3 * j) * 0x01010101u;
-#pragma unroll
-        for (int v = 0; v < 2 * kMaxChunks / 4; ++v) {
-          uint32_t wv[4] = {0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu, 0x7F7F7F7Fu};
-          if (r < m && 16 * v < kb2) {
-            const uint4 e = __ldcg(ep + v);
-            const uint32_t in[4] = {e.x, e.y, e.z, e.w};
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const int blk = 16 * v + 4 * c;  // kb2 is even: the word's byte pairs lie inside the row or past its end
-              uint32_t x = __vsubus4(in[c], sub);
-              if (blk + 2 >= kb2) x = (x & 0x0000FFFFu) | 0x7F7F0000u;
-              if (blk >= kb2) x = 0x7F7F7F7Fu;
-              wv[c] = x;
-            }
-          }
-#pragma unroll
-          for (int c = 0; c < 4; ++c) tmem_st1(tm_quarter + kColSfBh + par * kSfBhCols + 4 * (4 * v + c), wv[c]);
-        }
-        tmem_st_wait();
-      }
-#ifdef MOEV_TC_STATS
-      pst[1] += clock64() - pb0;
-#endif
-      // Per K chunk each producer warp forms one scale-factor atom: (tile, word) = (wk >> 1, wk & 1),
-      // the word's four K blocks for the tile rows lane, lane + 32, lane + 64, lane + 96, from the
-      // staged block; rows and blocks past the matrix get the unit scale.  The MMA issuers copy
-      // the atoms into TMEM (tcgen05.cp) in front of the stage's MMAs.
-      const int wk = warp & 3, tl = wk >> 1, wd = wk & 1;
-      const uint8_t* stb = sc_stage + (2 * buf + tl) * kScStageBytes;
-      const int rows = b.rows[tl];
+      // The four scale-factor atoms of a K chunk, (tile, word) = (a >> 1, a & 1): the word's four K
+      // blocks for the tile rows lane, lane + 32, lane + 64, lane + 96, from the staged blocks;
+      // rows and blocks past the matrix get the unit scale.  Producer warp k serves the ring
+      // stages it % 4 == k, so the four warps work on four stages at a time.  The MMA issuers
+      // copy the atoms into TMEM (tcgen05.cp) in front of the stage's MMAs.
+      const int wk = warp & 3;
+      const uint8_t* stb = sc_stage + (2 * buf) * kScStageBytes;
+      bool built = false;
       for (int kc = 0; kc < KC && ok; ++kc, ++it) {
+        if (kc == KC / 2 && id_next >= 0) {
+          // halfway: the next task's h scale factors, unless they may depend on this very task
+          // (its unit's progress counter is not complete yet: then they are built at the end)
+          const Task tn = decode_task(id_next, n_p1, n_slices, n_pairs);
+          int ready = 1;
+          if (tn.phase == 2) {
+            if (lane == 0) {
+              int v;
+              asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(P.unit_done + tn.unit) : "memory");
+              ready = v >= n_slices ? 1 : 0;
+            }
+            ready = __shfl_sync(0xffffffffu, ready, 0);
+          }
+          if (ready) {
+            fetch_exp(id_next);
+            if (ok) store_sfbh(id_next, tcount + 1);
+            built = true;
+            if (!ok) break;
+          }
+        }
+        if ((int)(it & 3u) != wk) continue;
         const int s = it % kStages;
-        const int kb = 8 * kc + 4 * wd;
-        uint32_t v[4];
+        uint32_t v[4][4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int r = lane + 32 * i;
-          v[i] = 0x7F7F7F7Fu;
-          if (kb < b.kb && r < rows) {
-            const uint16_t* p = reinterpret_cast<const uint16_t*>(stb + r * b.kb + kb);
-            v[i] = (uint32_t)p[0] | (((kb + 2 < b.kb) ? (uint32_t)p[1] : 0x7F7Fu) << 16);
+        for (int a4 = 0; a4 < 4; ++a4) {
+          const int tl = a4 >> 1, kb = 8 * kc + 4 * (a4 & 1);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int r = lane + 32 * i;
+            v[a4][i] = 0x7F7F7F7Fu;
+            if (kb < b.kb && r < b.rows[tl]) {
+              const uint16_t* p = reinterpret_cast<const uint16_t*>(stb + tl * kScStageBytes + r * b.kb + kb);
+              v[a4][i] = (uint32_t)p[0] | (((kb + 2 < b.kb) ? (uint32_t)p[1] : 0x7F7Fu) << 16);
+            }
           }
         }
 #ifdef MOEV_TC_STATS
@@ -629,31 +663,37 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         pst[0] += clock64() - pw0;
 #endif
         if (!ok) break;
-        *reinterpret_cast<uint4*>(sf_atoms + (4 * s + wk) * kSfAtomBytes + lane * 16) = make_uint4(v[0], v[1], v[2], v[3]);
+#pragma unroll
+        for (int a4 = 0; a4 < 4; ++a4)
+          *reinterpret_cast<uint4*>(sf_atoms + (4 * s + a4) * kSfAtomBytes + lane * 16) = make_uint4(v[a4][0], v[a4][1], v[a4][2], v[a4][3]);
         ptx::fence_proxy_async_smem();
-        ptx::tc_fence_before();  // orders the h scale factors written above (first stage of a phase-2 task)
+        ptx::tc_fence_before();  // orders the h scale factors written earlier (first stage of a phase-2 task)
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&S.aux_full[s]);
       }
+      ok = __all_sync(0xffffffffu, ok);
+      // (not earlier: the next task may wait for this very task's h)
+      if (ok && id_next >= 0 && !built) { fetch_exp(id_next); if (ok) store_sfbh(id_next, tcount + 1); }
     };
     int cur = next_task(S, q, abortp, P.status, true);
-    int buf = 0;
+    int buf = 0;  // cur % 3
     if (cur >= 0) stage_scales(cur, 0);
+    if (ok && cur >= 0) { fetch_exp(cur); if (ok) store_sfbh(cur, 0); }
     while (ok && cur >= 0) {
       const int nxt = next_task(S, q, abortp, P.status, true);
       if (nxt == -2) break;
-      if (nxt >= 0) stage_scales(nxt, buf ^ 1);
+      if (nxt >= 0) stage_scales(nxt, (buf + 1) % 3);
       if (!ok) break;
 #ifdef MOEV_TC_STATS
       const long long pr0 = clock64();
 #endif
-      run(cur, buf, nxt >= 0);
+      run(cur, buf, nxt);
 #ifdef MOEV_TC_STATS
       pst[2] += clock64() - pr0;
 #endif
       ++tcount;
       cur = nxt;
-      buf ^= 1;
+      buf = (buf + 1) % 3;
     }
 #ifdef MOEV_TC_STATS
     if (P.stats && pt == 0)
