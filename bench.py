@@ -66,8 +66,8 @@ DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 # 2.439543 GB + 3.79 MB against 2.422802 GB); traffic grows in proportion to the experts
 # streamed, so the full-size launch is scaled by the same ratio.  Absent = not captured.
 NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.439543e9 + 3.790336e6) / 2.422801920e9,
-                     # profiles/grouped_ffn_mx_gptoss_g64.md: 1.855084 GB + 3.81 MB against 1.454112 GB
-                     ("mxfp4", "tcgen05"): (1.855084e9 + 3.813376e6) / 1.454112e9}
+                     # profiles/grouped_ffn_mx_gptoss_g64.md: 1.518134 GB + 4.46 MB against 1.454112 GB
+                     ("mxfp4", "tcgen05"): (1.518134e9 + 4.463104e6) / 1.454112e9}
 
 ROUTING = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
            "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing,
