@@ -129,15 +129,7 @@ struct Smem {
   float e_inv[2][kMC];
 };
 
-// 16 consecutive 32-bit columns of this warp's TMEM lane quarter from registers: lane l writes
-// TMEM lane (quarter base + l).
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
+// One 32-bit column of this warp's TMEM lane quarter from registers: lane l writes TMEM lane (quarter base + l).
 __device__ __forceinline__ void tmem_st1(uint32_t taddr, uint32_t r0) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x1.b32 [%0], {%1};" ::"r"(taddr), "r"(r0) : "memory");
 }
@@ -180,11 +172,6 @@ __device__ __forceinline__ int next_task(Smem& S, uint32_t& q, volatile int* abo
   ptx::mbar_arrive(&S.tq_empty[slot]);
   ++q;
   return id;
-}
-
-__device__ __forceinline__ void tmem_st4(uint32_t taddr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
-  asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
-               : "memory");
 }
 
 __global__ void __launch_bounds__(kThreads, 1)

@@ -155,7 +155,7 @@ EncodeTiledFn encode_tiled_fn() {
 bool tc_eligible(const moev_config& c) {
   if (c.afmt != MOEV_ACT_BF16) return false;
   if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: rows of whole 32-byte MMA pieces; a task's scale rows are staged in shared memory
-    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 256 && c.I >= 128 &&
+    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 256 && c.I >= 256 &&  // rows of at least one 128-byte box
            128 * (c.H / 32) <= tcmx::kScStageBytes && 128 * (c.I / 32) <= tcmx::kScStageBytes;
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
   if (c.ffn_kind != MOEV_FFN_SWIGLU) return false;  // the biased, clamped form: MXFP4 tensor-core kernel or CUDA cores

@@ -63,6 +63,32 @@ def test_gptoss_shaped_many_tokens_per_expert(impl, gamma, U, n_shared):
     assert ref.n_active == U
 
 
+@pytest.mark.parametrize("H,I,gamma", [(320, 704, 9), (512, 512, 17), (256, 256, 5), (640, 1088, 12), (2880, 2880, 6)])
+def test_gptoss_shapes_two_phase_kernel(H, I, gamma):
+    """Shapes of the MXFP4 tensor-core kernel's two task kinds: I > H (more gate/up slices than
+    W_down tile pairs, ragged last chunk in both phases), scale rows whose length is a multiple of
+    four bytes, the smallest shape it serves (a single K chunk and a single task of each kind per
+    unit), an odd number of 128-row tiles of H, and the full GPT-OSS dimensions with few experts."""
+    shape = small_shape("gptoss", H=H, I=I, E=8 if H == 2880 else 16)
+    err, ref = parity_case(shape, gamma, expect_impl=moev.IMPL_TCGEN05)
+
+
+def test_gptoss_repeated_calls_reuse_scratch():
+    """Two different calls on one context: the h scratch rows and progress counters of the
+    MXFP4 kernel carry nothing over from the previous call."""
+    shape = small_shape("gptoss", H=704, I=320, E=32)
+    dev = "cuda"
+    w = synth.make_expert_weights(shape, layer=0, device=dev)
+    v = moev.MoeVerifier(gcfg(shape, 48))
+    for layer_id, gamma, routing in [(1, 48, synth.make_iid_routing), (2, 7, synth.make_scattered_routing),
+                                     (3, 31, synth.make_iid_routing)]:
+        wr, x = routing(shape, gamma, layer=layer_id, device=dev)
+        res = run_gpu(shape, wr, w, x, gamma, moev.IMPL_AUTO, verifier=v)
+        ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), gamma)
+        compare(shape, res, ref, gamma)
+    v.close()
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("gamma,U", [(1, 8), (8, 8), (8, 64), (32, 40), (128, 8), (128, 64)])
 def test_exact_union_cases(impl, gamma, U):
