@@ -38,7 +38,7 @@ class _Cfg(C.Structure):
     _fields_ = [("H", C.c_int32), ("I", C.c_int32), ("E", C.c_int32), ("top_k", C.c_int32),
                 ("n_shared", C.c_int32), ("wfmt", C.c_int32), ("afmt", C.c_int32),
                 ("score", C.c_int32), ("routed_scale", C.c_double), ("ffn_kind", C.c_int32),
-                ("n_group", C.c_int32), ("topk_group", C.c_int32), ("reserved", C.c_int32)]
+                ("n_group", C.c_int32), ("topk_group", C.c_int32), ("act_quant", C.c_int32)]
 
 
 class _Layer(C.Structure):
@@ -61,10 +61,11 @@ class Config:
     ffn_kind: int = 0   # 0 bias-free SwiGLU; 1 GPT-OSS form (clamped, biased; layer keys b_gate / b_up / b_down)
     n_group: int = 0    # > 0: DeepSeek group-limited routing (sigmoid scores; layer key router_bias)
     topk_group: int = 0
+    act_quant: int = 0  # 1 / 2: FP8 activations with 1x128 scales (binary32 / power-of-two scales) in front of both expert GEMMs
 
     def c(self) -> _Cfg:
         return _Cfg(self.H, self.I, self.E, self.top_k, self.n_shared, self.wfmt, self.afmt,
-                    self.score, self.routed_scale, self.ffn_kind, self.n_group, self.topk_group, 0)
+                    self.score, self.routed_scale, self.ffn_kind, self.n_group, self.topk_group, self.act_quant)
 
 
 _lib = None
@@ -78,6 +79,8 @@ def lib() -> C.CDLL:
         _lib.oracle_decode_bf16.argtypes = [C.c_uint16]
         _lib.oracle_decode_e4m3.restype = C.c_double
         _lib.oracle_decode_e4m3.argtypes = [C.c_uint8]
+        _lib.oracle_encode_e4m3.restype = C.c_uint8
+        _lib.oracle_encode_e4m3.argtypes = [C.c_float]
         _lib.oracle_decode_e2m1.restype = C.c_double
         _lib.oracle_decode_e2m1.argtypes = [C.c_uint8]
         _lib.oracle_decode_e8m0.restype = C.c_double
@@ -114,6 +117,24 @@ def decode_bf16(b: int) -> float:
 
 def decode_e4m3(b: int) -> float:
     return lib().oracle_decode_e4m3(b)
+
+
+def encode_e4m3(f: float) -> int:
+    return lib().oracle_encode_e4m3(f)
+
+
+def act_quant(x: np.ndarray, mode: int = 1):
+    """FP8 1x128 quantisation of the rows of x (float32 [..., n]): (codes uint8 [..., n],
+    scales float32 [..., ceil(n / 128)])."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    n = x.shape[-1]
+    rows = x.reshape(-1, n)
+    codes = np.zeros(rows.shape, dtype=np.uint8)
+    scales = np.zeros((rows.shape[0], (n + 127) // 128), dtype=np.float32)
+    for r in range(rows.shape[0]):
+        lib().oracle_act_quant(C.c_void_p(rows[r].ctypes.data), C.c_int64(n), C.c_int32(mode),
+                               C.c_void_p(codes[r].ctypes.data), C.c_void_p(scales[r].ctypes.data))
+    return codes.reshape(x.shape), scales.reshape(x.shape[:-1] + (scales.shape[1],))
 
 
 def decode_e2m1(b: int) -> float:

@@ -50,7 +50,7 @@ typedef struct {
   int32_t ffn_kind; /* 0: bias-free SwiGLU (the benchmark configurations); 1: GPT-OSS form, see expert_ffn */
   int32_t n_group;  /* > 0: group-limited routing, see oracle_topk_grouped (score must be sigmoid) */
   int32_t topk_group;
-  int32_t reserved;
+  int32_t act_quant; /* 0: activations as given; 1, 2: FP8 activations with 1x128 scales, see oracle_act_quant */
 } oracle_cfg;
 
 /* All pointers are HOST pointers.  Layouts (K = contraction dim, contiguous):
@@ -318,6 +318,68 @@ int32_t oracle_union_perm(int32_t E, int32_t k, int32_t gamma, const int32_t *id
   return U;
 }
 
+/* ------------------------------------------------- FP8 activations (1x128) */
+
+/* Nearest e4m3 code of a finite float, ties to the even code, magnitudes above
+ * 448 saturate to 448.  Written as a search over the 127 finite magnitudes of
+ * the decoder above. */
+uint8_t oracle_encode_e4m3(float f) {
+  double a = fabs((double)f);
+  int lo = 0;
+  if (a >= 448.0) {
+    lo = 0x7E;
+  } else {
+    while (lo < 0x7E && oracle_decode_e4m3((uint8_t)(lo + 1)) <= a) ++lo; /* value(lo) <= a < value(lo + 1) */
+    double dl = a - oracle_decode_e4m3((uint8_t)lo), dh = oracle_decode_e4m3((uint8_t)(lo + 1)) - a;
+    if (dh < dl || (dh == dl && (lo & 1))) ++lo;
+  }
+  return (uint8_t)(lo | (signbit(f) ? 0x80 : 0));
+}
+
+/* Not in the paper (which does not print the expert FFN): deployed DeepSeek-V3
+ * inference feeds every expert GEMM with FP8 activations, quantised on the fly
+ * per token and per block of 128 consecutive elements of the contraction axis:
+ *   amax = max |x_i| over the block,   s = amax / 448   (mode 1, binary32)
+ *                                      s = 2^ceil(log2(amax / 448))   (mode 2, power-of-two scales)
+ *   code_i = e4m3( x_i / s ),   the GEMM sees  decode(code_i) * s.
+ * An all-zero block takes s = 1.  The scale, the division and the rounding are
+ * binary32 operations (the codes are integers decided by floating point, so
+ * the precision is part of the definition); the last block may be shorter. */
+void oracle_act_quant(const float *x, int64_t n, int32_t mode, uint8_t *codes, float *scales) {
+  for (int64_t b0 = 0; b0 < n; b0 += 128) {
+    int64_t b1 = b0 + 128 < n ? b0 + 128 : n;
+    float amax = 0.0f;
+    for (int64_t i = b0; i < b1; ++i) {
+      float a = fabsf(x[i]);
+      if (a > amax) amax = a;
+    }
+    float s = 1.0f;
+    if (amax > 0.0f) {
+      s = amax / 448.0f;
+      if (mode == 2) {
+        int e;
+        float fr = frexpf(s, &e); /* s = fr * 2^e, fr in [0.5, 1) */
+        s = ldexpf(1.0f, fr == 0.5f ? e - 1 : e);
+      }
+    }
+    scales[b0 / 128] = s;
+    for (int64_t i = b0; i < b1; ++i) codes[i] = oracle_encode_e4m3(x[i] / s);
+  }
+}
+
+/* x (length n, values representable in binary32) -> the values the GEMM sees, in place */
+static void act_qdq(double *x, int64_t n, int32_t mode) {
+  float *xf = (float *)malloc(sizeof(float) * (size_t)n);
+  uint8_t *q = (uint8_t *)malloc((size_t)n);
+  float *sc = (float *)malloc(sizeof(float) * (size_t)((n + 127) / 128));
+  for (int64_t i = 0; i < n; ++i) xf[i] = (float)x[i];
+  oracle_act_quant(xf, n, mode, q, sc);
+  for (int64_t i = 0; i < n; ++i) x[i] = oracle_decode_e4m3(q[i]) * (double)sc[i / 128];
+  free(xf);
+  free(q);
+  free(sc);
+}
+
 /* --------------------------------------------------------------- expert FFN */
 
 /* Apply expert e (of the tensor set wg/wu/wd with scales sg/su/sd) to m
@@ -325,13 +387,22 @@ int32_t oracle_union_perm(int32_t E, int32_t k, int32_t gamma, const int32_t *id
  * silu(z) = z / (1 + exp(-z)).  Each weight row is decoded once.
  * ffn_kind 1 (the published GPT-OSS expert; not in the paper, which does not print the FFN):
  *   g = min(Wg x + bg, 7),  u = clamp(Wu x + bu, -7, 7),
- *   h = g * sigmoid(1.702 g) * (u + 1),  out = Wd h + bd          (bg, bu, bd may be NULL = 0). */
+ *   h = g * sigmoid(1.702 g) * (u + 1),  out = Wd h + bd          (bg, bu, bd may be NULL = 0).
+ * act_quant != 0: both GEMM inputs, x and h (rounded to binary32 first), are replaced by their
+ * FP8 1x128 quantisation (oracle_act_quant). */
 static void expert_ffn(const oracle_cfg *c, const void *wg, const void *wu, const void *wd,
                        const void *sg, const void *su, const void *sd, int64_t e, int m,
                        const double *xs, double *out, const float *bg, const float *bu,
                        const float *bd) {
   int64_t H = c->H, I = c->I;
   double *hbuf = (double *)malloc(sizeof(double) * (size_t)m * (size_t)I);
+  double *xq = NULL;
+  if (c->act_quant) {
+    xq = (double *)malloc(sizeof(double) * (size_t)m * (size_t)H);
+    memcpy(xq, xs, sizeof(double) * (size_t)m * (size_t)H);
+    for (int r = 0; r < m; ++r) act_qdq(xq + (int64_t)r * H, H, c->act_quant);
+    xs = xq;
+  }
 #pragma omp parallel
   {
     double *rg = (double *)malloc(sizeof(double) * (size_t)(H > I ? H : I));
@@ -357,6 +428,11 @@ static void expert_ffn(const oracle_cfg *c, const void *wg, const void *wu, cons
         }
       }
     }
+#pragma omp single
+    {
+      if (c->act_quant)
+        for (int r = 0; r < m; ++r) act_qdq(hbuf + (int64_t)r * I, I, c->act_quant);
+    }
 #pragma omp for schedule(static)
     for (int64_t n = 0; n < H; ++n) {
       decode_row(c->wfmt, wd, sd, e, H, I, n, rg);
@@ -372,6 +448,7 @@ static void expert_ffn(const oracle_cfg *c, const void *wg, const void *wu, cons
     free(ru);
   }
   free(hbuf);
+  free(xq);
 }
 
 /* Exposed single-expert FFN on already-decoded double inputs (pins). */
