@@ -159,10 +159,13 @@ def layers_that_fit(shape: synth.Shape, want: int = 4) -> int:
     return max(1, min(want, int((free * 0.85) // per_layer)))
 
 
+ACT_QUANT = 0  # --act-quant: FP8 activations with 1x128 scales in front of both expert GEMMs (a variant, not the headline)
+
+
 def ocfg_of(shape):
     import oracle
     return oracle.Config(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, shape.wfmt,
-                         shape.afmt, shape.score, shape.routed_scale)
+                         shape.afmt, shape.score, shape.routed_scale, act_quant=ACT_QUANT)
 
 
 def time_oracle_sample(shape, layer, gamma_sample: int, repeats: int = 1):
@@ -244,7 +247,7 @@ def run_ours(args):
     shape, gamma, layers = build_workload(args.workload, n_layers, dev, rank)
     impl = {"auto": moev.IMPL_AUTO, "simt": moev.IMPL_SIMT, "tcgen05": moev.IMPL_TCGEN05}[args.kernels]
     cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, gamma, shape.wfmt,
-                          shape.afmt, shape.score, impl, shape.routed_scale)
+                          shape.afmt, shape.score, impl, shape.routed_scale, act_quant=ACT_QUANT)
     v = moev.MoeVerifier(cfg)
     packed = []
     for L in layers:
@@ -367,7 +370,8 @@ def run_ours(args):
                        "unique_experts_per_layer": U, "layers_rotated": n_layers,
                        "l2_policy": "weights of %d layers (%.1f GB) rotated per call, > L2" % (
                            n_layers, n_layers * (shape.E + shape.n_shared) * Wb / 1e9),
-                       "bytes_per_expert": Wb, "kernels": impl_name, "parallelism": "replicas"},
+                       "bytes_per_expert": Wb, "kernels": impl_name, "parallelism": "replicas",
+                       **({"act_quant": ACT_QUANT} if ACT_QUANT else {})},
             "latency_us": 1e3 * ms_total / args.steps,
             "frac_of_8TBps": value / world / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -545,11 +549,15 @@ def main():
     ap.add_argument("--kernels", default="auto", choices=["auto", "simt", "tcgen05"])
     ap.add_argument("--cpu-tokens", type=int, default=0, help="tokens of layer 0 the oracle is timed on (0 = all gamma)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--act-quant", type=int, default=0, choices=[0, 1, 2],
+                    help="FP8 activations with 1x128 scales (1: binary32 scales, 2: power-of-two scales)")
     ap.add_argument("--sweep", action="store_true", help="unique-expert sweep (DeepSeek FP8 shape) instead of the bench line")
     ap.add_argument("--select-demo", action="store_true",
                     help="cost-aware vs acceptance-only draft selection in front of the verification layer")
     ap.add_argument("--p-reuse", type=float, default=0.7, help="expert locality along a tree path (select demo)")
     args = ap.parse_args()
+    global ACT_QUANT
+    ACT_QUANT = args.act_quant
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

@@ -92,6 +92,16 @@ typedef enum { MOEV_FFN_SWIGLU = 0, MOEV_FFN_GPTOSS = 1 } moev_ffn_kind;
  * selected and emitted in that order; weights use the unbiased scores:
  * w_j = routed_scale * s_j / (sum_j s_j + 1e-20). */
 
+/* FP8 activations in front of both expert GEMMs (what deployed DeepSeek-V3 inference does; the
+ * paper does not print the expert FFN).  The input x of the gate / up projections and the input h
+ * of the down projection are quantised on the fly per token and per block of 128 consecutive
+ * elements of the contraction axis: amax = max |v| over the block, s = amax / 448 (binary32; with
+ * POW2 the smallest power of two that is not below it; 1 for an all-zero block), code = e4m3(v / s)
+ * rounded to nearest even, and the GEMM sees decode(code) * s.  The router sees the unquantised x.
+ * Tensor-core kernels: MOEV_W_FP8E4M3_B128 with H <= 8192 and I <= 4096; other configurations run
+ * on the CUDA-core kernels. */
+typedef enum { MOEV_ACTQ_NONE = 0, MOEV_ACTQ_FP8_B128 = 1, MOEV_ACTQ_FP8_B128_POW2 = 2 } moev_act_quant;
+
 typedef struct {
   int32_t H;          /* hidden size; multiple of 32 */
   int32_t I;          /* expert intermediate size; multiple of 32 */
@@ -107,6 +117,7 @@ typedef struct {
   int32_t ffn_kind;   /* moev_ffn_kind; MOEV_FFN_GPTOSS needs n_shared == 0 */
   int32_t n_group;    /* 0 = plain top-k; > 0: group-limited routing (below), needs MOEV_SCORE_SIGMOID, E % n_group == 0 */
   int32_t topk_group; /* groups kept per token, 1..n_group; top_k <= topk_group * E / n_group */
+  int32_t act_quant;  /* moev_act_quant */
 } moev_config;
 
 /* One layer's parameters.  Layouts, row-major, last index contiguous:

@@ -31,6 +31,7 @@ class MoevError(RuntimeError):
 
 
 FFN_SWIGLU, FFN_GPTOSS = 0, 1
+ACTQ_NONE, ACTQ_FP8_B128, ACTQ_FP8_B128_POW2 = 0, 1, 2
 
 
 class _Config(C.Structure):
@@ -38,7 +39,7 @@ class _Config(C.Structure):
                 ("n_shared", C.c_int32), ("max_tokens", C.c_int32), ("wfmt", C.c_int32),
                 ("afmt", C.c_int32), ("score", C.c_int32), ("impl", C.c_int32),
                 ("routed_scale", C.c_float), ("ffn_kind", C.c_int32), ("n_group", C.c_int32),
-                ("topk_group", C.c_int32)]
+                ("topk_group", C.c_int32), ("act_quant", C.c_int32)]
 
 
 _LAYER_FIELDS = ("router_w", "w_gate", "w_up", "w_down", "s_gate", "s_up", "s_down",
@@ -70,11 +71,12 @@ class MoevConfig:
     ffn_kind: int = 0   # FFN_SWIGLU; FFN_GPTOSS = clamped, biased GPT-OSS expert (layer keys b_gate / b_up / b_down)
     n_group: int = 0    # > 0: DeepSeek group-limited routing (sigmoid scores; layer key router_bias)
     topk_group: int = 0
+    act_quant: int = 0  # ACTQ_FP8_B128 / ACTQ_FP8_B128_POW2: FP8 activations with 1x128 scales in front of both expert GEMMs
 
     def c(self) -> _Config:
         return _Config(self.H, self.I, self.E, self.top_k, self.n_shared, self.max_tokens,
                        self.wfmt, self.afmt, self.score, self.impl, self.routed_scale, self.ffn_kind,
-                       self.n_group, self.topk_group)
+                       self.n_group, self.topk_group, self.act_quant)
 
 
 _lib = None

@@ -39,10 +39,13 @@ struct Tables {
   int32_t* n_active;   // [1]
   float* tok_scale;    // [gamma] power of two bringing the token's max |x| into [64,128)
   uint8_t* xq;         // quantised activations x * tok_scale, written once per token for the tensor-core kernels, or null:
-                       // xq_e2m1 = 0: [gamma, 2, xq_stride] e4m3 hi / lo terms (fp8 weights);
-                       // xq_e2m1 = 1: [gamma, 4, xq_stride] packed e2m1 terms 8^-j (MXFP4 weights)
+                       // xq_mode 0: [gamma, 2, xq_stride] e4m3 hi / lo terms (fp8 weights);
+                       // xq_mode 1: [gamma, 4, xq_stride] packed e2m1 terms 8^-j (MXFP4 weights);
+                       // xq_mode 2, 3: moev_act_quant 1, 2: [gamma, 2, xq_stride], first row of a token = its e4m3
+                       //   codes (second row stays zero), block scales in xs, tok_scale = 1
   int32_t xq_stride;   // bytes per row: H (e4m3) or H / 2 (e2m1)
-  int32_t xq_e2m1;
+  int32_t xq_mode;
+  float* xs;           // [gamma, H / 128] block scales of the FP8 1x128 activation quantisation, or null
   Unit* units;         // [max_units]
   int32_t* n_units;    // [1]
   int32_t* task_counter; // [1] dynamic task scheduler of the tensor-core FFN, zeroed per call
@@ -87,6 +90,22 @@ __device__ __forceinline__ void split4_e4m3(const float (&v)[4], uint32_t& hi, u
     hi |= (uint32_t)hc << (16 * p);
     lo |= (uint32_t)lc << (16 * p);
   }
+}
+
+// Scale of one block of the FP8 1x128 activation quantisation (moev_act_quant): amax / 448 in
+// binary32 (mode 1) or the smallest power of two not below it (mode 2); 1 for an all-zero block.
+// The block's codes are e4m3(v / s), round to nearest even, saturating.
+__device__ __forceinline__ float act_scale(float amax, int mode) {
+  if (!(amax > 0.f)) return 1.f;
+  float s = __fdiv_rn(amax, 448.f);
+  if (mode == 2) {
+    const uint32_t b = __float_as_uint(s);
+    s = __uint_as_float(((b >> 23) + ((b & 0x7FFFFFu) ? 1u : 0u)) << 23);
+  }
+  return s;
+}
+__device__ __forceinline__ uint32_t act_code(float v, float s) {
+  return (uint32_t)__nv_cvt_float_to_fp8(__fdiv_rn(v, s), __NV_SATFINITE, __NV_E4M3);
 }
 
 // Two scaled values (|v| < 4) -> four e2m1 terms each, v ~ q0 + q1 / 8 + q2 / 64 + q3 / 512: byte

@@ -234,4 +234,39 @@ __global__ void finalize_kernel(const float* __restrict__ y32, void* __restrict_
   }
 }
 
+// FP8 1x128 activation quantisation (moev_act_quant) for the CUDA-core path: one warp per
+// (row, block of 128): in [rows, n] (AFMT) -> out [rows, n] fp32 holding decode(code) * scale, the
+// values the GEMM sees.  in == out is allowed for fp32 (the h buffer is quantised in place).
+template <int AFMT>
+__global__ void __launch_bounds__(256) act_quant_rows_kernel(const void* in, float* out, int rows, int n,
+                                                             int mode) {
+  const int lane = threadIdx.x & 31;
+  const int nb = (n + 127) / 128;
+  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (wid >= (long long)rows * nb) return;
+  const int r = (int)(wid / nb), b = (int)(wid - (long long)r * nb);
+  float v[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int k = b * 128 + lane * 4 + j;
+    v[j] = 0.f;
+    if (k < n) {
+      if constexpr (AFMT == MOEV_ACT_BF16) v[j] = __uint_as_float((uint32_t)static_cast<const uint16_t*>(in)[(size_t)r * n + k] << 16);
+      else v[j] = static_cast<const float*>(in)[(size_t)r * n + k];
+    }
+  }
+  float bm = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+  const float s = act_scale(bm, mode);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int k = b * 128 + lane * 4 + j;
+    if (k < n) {
+      const __half_raw hr = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)act_code(v[j], s), __NV_E4M3);
+      out[(size_t)r * n + k] = __half2float(*reinterpret_cast<const __half*>(&hr)) * s;
+    }
+  }
+}
+
 }  // namespace moev

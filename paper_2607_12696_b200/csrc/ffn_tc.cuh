@@ -68,7 +68,8 @@ __device__ void wide_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, 
 }  // namespace tcw
 namespace tc { struct Params; }
 namespace tcp {  // single-phase schedule without activation producers (ffn_tc_p.cuh)
-__device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
+template <bool ACTQ>
+__device__ __noinline__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
                              const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up, const CUtensorMap& tm_sh_down,
                              const CUtensorMap& tm_xq, const tc::Params& P, uint32_t tmem);
 }  // namespace tcp
@@ -103,6 +104,8 @@ struct Params {
   int32_t gamma, H, I, A;
   const int32_t* wide;  // non-null and non-zero: the two-phase schedule (ffn_tc_wide.cuh) runs this call
   int32_t xq_ready;     // fp8: the routing kernels wrote the quantised activations: run the schedule of ffn_tc_p.cuh
+  int32_t actq;         // moev_act_quant: FP8 1x128 activations (single e4m3 term, block scales in xs)
+  const float* xs;      // [gamma, H / 128] activation block scales (actq != 0)
 #ifdef MOEV_TC_STATS
   unsigned long long* stats;  // [grid][16] cycles the MMA thread spent per wait / issue class (debug builds)
 #endif
@@ -294,7 +297,8 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #ifndef MOEV_FP8_FOLD_SCALE
     if (P.xq_ready) {
       // quantised activations are available: the schedule without activation producers
-      tcp::promote_body(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem);
+      if (P.actq) tcp::promote_body<true>(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem);
+      else tcp::promote_body<false>(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem);
       ptx::tc_fence_before();
       __syncthreads();
       if (warp == 0) {

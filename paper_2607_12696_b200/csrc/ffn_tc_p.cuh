@@ -8,6 +8,9 @@
 //     (warps 2..5: gate tile, 6..9: up tile) add  block scale * partial  into register accumulators;
 //     P reaches the gate group through 32 TMEM columns;
 //   * in the down phase group g handles tile g of every stage.
+// ACTQ (moev_act_quant): the operand rows hold one e4m3 term per token (the second row of a token
+// is zero) and the activation's 1x128 block scales multiply the partial products per column and
+// K chunk; h gets the same quantisation, its block being the task's 128-wide slice of I.
 // ffn_tc.cuh's kernel calls promote_body() after its prologue (same launch, same TMEM).
 #pragma once
 #include <cuda.h>
@@ -38,7 +41,8 @@ constexpr int kHTileBytes = 8 * 1024;   // h tile, operand of the down phase
 constexpr int kMC = 32;
 constexpr int kColD = 256;              // TMEM: partial buffers 2 x (64 | 64) | O[2 stage buffers][2 tiles] 64 each
 constexpr int kTileBytes = kStages * kStageBytes + kStages * kBTileBytes + kHTileBytes;
-constexpr int kCtlBytes = 8 * 1024;
+constexpr int kCtlBytes = 16 * 1024;
+constexpr int kMaxChunksQ = 64;         // K chunks whose activation block scales fit the table (ACTQ: H <= 8192)
 constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
 static_assert(kSmemBytes <= tc::kSmemBytes, "runs inside the launch of ffn_tc.cuh's kernel");
 
@@ -59,6 +63,7 @@ struct Smem {
   float s_tab[2][2][128];           // [parity][group] gate / up block scale per K chunk
   float e_sd[2][128];               // W_down block scale per H tile
   uint32_t e_amax[4][kMC];
+  float sx[kMC][kMaxChunksQ];      // ACTQ: block scale of the unit's token r for K chunk kc
 };
 
 __device__ __forceinline__ int next_task(Smem& S, uint32_t& q, volatile int* abortp, int* status, bool whole_warp) {
@@ -72,7 +77,8 @@ __device__ __forceinline__ int next_task(Smem& S, uint32_t& q, volatile int* abo
   return id;
 }
 
-__device__ __noinline__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
+template <bool ACTQ>
+__device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
                                           const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up,
                                           const CUtensorMap& tm_sh_down, const CUtensorMap& tm_xq,
                                           const tc::Params& P, uint32_t tmem) {
@@ -280,6 +286,14 @@ __device__ __noinline__ void promote_body(const CUtensorMap& tm_gate, const CUte
         for (int ht = lane; ht < HT; ht += 32) S.e_sd[par][ht] = __ldg(sd + ((size_t)u.expert * HT + ht) * n_slices + slice);
       }
       __syncwarp();
+      if constexpr (ACTQ) {
+        // every warp fills the whole table (identical values), so it reads only what it wrote itself
+        for (int i = lane; i < m * KC; i += 32) {
+          const int r = i / KC, kc = i - r * KC;
+          S.sx[r][kc] = __ldg(P.xs + (size_t)S.e_tok[par][r] * KC + kc);
+        }
+        __syncwarp();
+      }
 
       // ---- gate/up phase: acc[r] += block scale * (hi + lo / 16) of this group's tile
       float acc[kMC];
@@ -299,8 +313,10 @@ __device__ __noinline__ void promote_body(const CUtensorMap& tm_gate, const CUte
           ptx::tc_fence_before();
           ptx::mbar_arrive(&S.p_empty[pb]);
 #pragma unroll
-          for (int r = 0; r < 8; ++r)
-            acc[r] = fmaf(__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f, sv, acc[r]);
+          for (int r = 0; r < 8; ++r) {
+            if constexpr (ACTQ) acc[r] = fmaf(__uint_as_float(o[2 * r]) * (r < m ? S.sx[r][kc] : 0.f), sv, acc[r]);
+            else acc[r] = fmaf(__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f, sv, acc[r]);
+          }
         } else {
 #pragma unroll
           for (int c0 = 0; c0 < 64; c0 += 16) {
@@ -309,8 +325,11 @@ __device__ __noinline__ void promote_body(const CUtensorMap& tm_gate, const CUte
               ptx::tmem_ld16(src + c0, o);
               ptx::tmem_ld_wait();
 #pragma unroll
-              for (int r = 0; r < 8; ++r)
-                acc[c0 / 2 + r] = fmaf(__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f, sv, acc[c0 / 2 + r]);
+              for (int r = 0; r < 8; ++r) {
+                const int tr = c0 / 2 + r;
+                if constexpr (ACTQ) acc[tr] = fmaf(__uint_as_float(o[2 * r]) * (tr < m ? S.sx[tr][kc] : 0.f), sv, acc[tr]);
+                else acc[tr] = fmaf(__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f, sv, acc[tr]);
+              }
             }
           }
           ptx::tc_fence_before();
@@ -363,6 +382,13 @@ __device__ __noinline__ void promote_body(const CUtensorMap& tm_gate, const CUte
         for (int r = 0; r < kMC; ++r) {
           if (r < m) {
             const uint32_t mx = max(max(S.e_amax[0][r], S.e_amax[1][r]), max(S.e_amax[2][r], S.e_amax[3][r]));
+            if constexpr (ACTQ) {  // the slice is one 1x128 block of h: a single e4m3 term with the block's scale
+              const float sh = act_scale(__uint_as_float(mx), P.actq);
+              h_tile[sw128(2 * r, row >> 4) + (row & 15)] = (uint8_t)act_code(hv[r], sh);
+              h_tile[sw128(2 * r + 1, row >> 4) + (row & 15)] = 0;
+              if (row == r) S.e_f[par][r] = S.e_w[par][r] * sh;
+              continue;
+            }
             const int er = safe_exponent(__uint_as_float(mx));
             const float v = hv[r] * pow2i(6 - er);
             const __nv_fp8_storage_t hc = __nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);

@@ -53,6 +53,7 @@ struct moev_ctx {
   uint8_t* hq = nullptr;  // its scratch: quantised h tiles [max_units][n_slices][64][128] ...
   float* hq_f = nullptr;  // ... and their scales [max_units][n_slices][32]
   uint8_t* xu = nullptr;  // per-unit operand tiles [max_units][H / 128][64][128]
+  float* xhat = nullptr;    // CUDA-core path with moev_act_quant: the quantised activations as fp32 [max_tokens, H]
   uint8_t* hexp = nullptr;  // MXFP4 tensor-core path: block exponents of h, [max_units * 8][tcmx::kExpStride] (hq holds the h terms)
   size_t max_units = 0;
   CUtensorMap tm_hq, tm_xu;
@@ -94,6 +95,7 @@ bool cfg_ok(const moev_config* c, char* why, size_t n) {
   BAD(c->score < 0 || c->score > MOEV_SCORE_SIGMOID, "unknown score function");
   BAD(c->impl < 0 || c->impl > MOEV_IMPL_TCGEN05, "unknown impl");
   BAD(c->ffn_kind < 0 || c->ffn_kind > MOEV_FFN_GPTOSS, "unknown ffn_kind");
+  BAD(c->act_quant < 0 || c->act_quant > MOEV_ACTQ_FP8_B128_POW2, "unknown act_quant");
   BAD(c->n_group < 0 || c->topk_group < 0, "n_group and topk_group must be >= 0");
   BAD(c->n_group > 0 && (c->score != MOEV_SCORE_SIGMOID || c->E % c->n_group || c->topk_group < 1 ||
                          c->topk_group > c->n_group || c->top_k > c->topk_group * (c->E / c->n_group)),
@@ -155,10 +157,13 @@ EncodeTiledFn encode_tiled_fn() {
 bool tc_eligible(const moev_config& c) {
   if (c.afmt != MOEV_ACT_BF16) return false;
   if (c.wfmt == MOEV_W_MXFP4)  // block-scaled kernel: rows of whole 32-byte MMA pieces; a task's scale rows are staged in shared memory
-    return c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 256 && c.I >= 256 &&  // rows of at least one 128-byte box
+    return c.act_quant == MOEV_ACTQ_NONE && c.H % 64 == 0 && c.I % 64 == 0 && c.H >= 256 && c.I >= 256 &&  // rows of at least one 128-byte box
            128 * (c.H / 32) <= tcmx::kScStageBytes && 128 * (c.I / 32) <= tcmx::kScStageBytes;
   if (c.wfmt != MOEV_W_BF16 && c.wfmt != MOEV_W_FP8E4M3_B128) return false;
-  if (c.ffn_kind != MOEV_FFN_SWIGLU) return false;  // the biased, clamped form: MXFP4 tensor-core kernel or CUDA cores
+  if (c.ffn_kind != MOEV_FFN_SWIGLU) return false;
+  // FP8 activations: the fp8 schedule that takes its activations from the routing kernels, table of H / 128 block scales
+  if (c.act_quant != MOEV_ACTQ_NONE &&
+      (c.wfmt != MOEV_W_FP8E4M3_B128 || c.I / 128 > tcw::kMaxSlices || c.H / 128 > tcp::kMaxChunksQ)) return false;  // the biased, clamped form: MXFP4 tensor-core kernel or CUDA cores
   if (c.H % 128 || c.I % 128) return false;
   const int bk = c.wfmt == MOEV_W_BF16 ? 64 : 128;
   if (c.H / bk < 4 || c.H / 128 > 128 || c.H / bk > 128 * (128 / bk)) return false;
@@ -259,6 +264,7 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
   P.wide = c->wide_ok ? c->T.wide : nullptr;
   P.xq_ready = (c->wide_ok && c->T.xq) ? 1 : 0;
+  P.actq = g.act_quant; P.xs = c->T.xs;
   // arguments of the two-phase schedule, which the kernel switches to when the grouping kernel's
   // flag says that the call has many tokens per streamed expert (fp8 only)
   tcw::Params W{};
@@ -303,8 +309,19 @@ void launch_simt_ffn(moev_ctx* c, const LayerPtrs& L, const void* x, int gamma, 
   const moev_config& g = c->cfg;
   const int rows = 64;
   dim3 g1(g.E + g.n_shared, (g.I + rows - 1) / rows), g2(g.E + g.n_shared, (g.H + rows - 1) / rows);
-  ffn_gateup_simt<WFMT, AFMT><<<g1, 256, 0, st>>>(L, c->T, x, c->hbuf, gamma, g.H, g.I, g.top_k,
-                                                   g.n_shared, rows);
+  if (g.act_quant != MOEV_ACTQ_NONE) {
+    // FP8 1x128 activations: x -> the values the GEMM sees (fp32), h likewise in place between the two kernels
+    const long long w1 = (long long)gamma * ((g.H + 127) / 128);
+    act_quant_rows_kernel<AFMT><<<(unsigned)((w1 + 7) / 8), 256, 0, st>>>(x, c->xhat, gamma, g.H, g.act_quant);
+    ffn_gateup_simt<WFMT, MOEV_ACT_FP32><<<g1, 256, 0, st>>>(L, c->T, c->xhat, c->hbuf, gamma, g.H, g.I, g.top_k,
+                                                             g.n_shared, rows);
+    const int hrows = gamma * (g.top_k + g.n_shared);
+    const long long w2 = (long long)hrows * ((g.I + 127) / 128);
+    act_quant_rows_kernel<MOEV_ACT_FP32><<<(unsigned)((w2 + 7) / 8), 256, 0, st>>>(c->hbuf, c->hbuf, hrows, g.I, g.act_quant);
+  } else {
+    ffn_gateup_simt<WFMT, AFMT><<<g1, 256, 0, st>>>(L, c->T, x, c->hbuf, gamma, g.H, g.I, g.top_k,
+                                                     g.n_shared, rows);
+  }
   if (ev) cudaEventRecord(ev[4], st);
   ffn_down_simt<WFMT><<<g2, 256, 0, st>>>(L, c->T, c->hbuf, c->y32, gamma, g.H, g.I, g.top_k,
                                            g.n_shared, rows);
@@ -433,9 +450,11 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     // per token (fp8 weights) or four packed e2m1 term rows of H / 2 bytes (MXFP4 weights)
     const bool mx = cfg->wfmt == MOEV_W_MXFP4;
     const size_t rows_per_tok = mx ? 4 : 2;
-    c->T.xq_e2m1 = mx ? 1 : 0;
+    c->T.xq_mode = mx ? 1 : (cfg->act_quant ? 1 + cfg->act_quant : 0);
     c->T.xq_stride = mx ? cfg->H / 2 : cfg->H;
     ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->T.xq), rows_per_tok * G * (size_t)c->T.xq_stride) == cudaSuccess;
+    ok = ok && cudaMemset(c->T.xq, 0, rows_per_tok * G * (size_t)c->T.xq_stride) == cudaSuccess;  // act_quant: the second row of a token stays zero
+    if (cfg->act_quant) ok = ok && dmalloc(&c->T.xs, G * (size_t)(cfg->H / 128)) == cudaSuccess;
     EncodeTiledFn fn = encode_tiled_fn();
     if (ok && fn) {
       cuuint64_t dims[2] = {(cuuint64_t)c->T.xq_stride, (cuuint64_t)(rows_per_tok * G)};
@@ -450,6 +469,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     }
   }
   ok = ok && dmalloc(&c->hbuf, slots * cfg->I) == cudaSuccess;
+  if (cfg->act_quant != MOEV_ACTQ_NONE && c->resolved_impl == MOEV_IMPL_SIMT)
+    ok = ok && dmalloc(&c->xhat, G * cfg->H) == cudaSuccess;
   ok = ok && dmalloc(&c->y32, G * cfg->H) == cudaSuccess;
   ok = ok && cudaMalloc(&c->x_stage, G * cfg->H * act_b) == cudaSuccess;
   ok = ok && cudaMalloc(&c->y_stage, G * cfg->H * act_b) == cudaSuccess;
@@ -497,7 +518,7 @@ moev_status moev_destroy(moev_ctx* c) {
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
   cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->T.task_counter); cudaFree(c->hbuf); cudaFree(c->y32);
-  cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f); cudaFree(c->xu); cudaFree(c->hexp);
+  cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f); cudaFree(c->xu); cudaFree(c->hexp); cudaFree(c->xhat); cudaFree(c->T.xs);
   cudaFree(c->x_stage); cudaFree(c->y_stage);
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)
@@ -510,7 +531,7 @@ moev_status moev_destroy(moev_ctx* c) {
 
 const char* moev_last_error(const moev_ctx* c) { return c ? c->err : "null context"; }
 int32_t moev_launches_per_call(const moev_ctx* c) {
-  return c ? (c->resolved_impl == MOEV_IMPL_TCGEN05 ? 5 : 6) : 0;
+  return c ? (c->resolved_impl == MOEV_IMPL_TCGEN05 ? 5 : (c->cfg.act_quant != MOEV_ACTQ_NONE ? 8 : 6)) : 0;
 }
 int32_t moev_resolved_impl(const moev_ctx* c) { return c ? c->resolved_impl : 0; }
 
@@ -576,7 +597,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
              layer->router_bias, g.n_group, g.topk_group);
   if (ev) cudaEventRecord(ev[2], st);
   launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
-           g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma), c->wide_ok ? kWideRatio : 0);
+           g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma), (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0);
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);

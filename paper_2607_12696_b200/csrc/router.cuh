@@ -640,9 +640,24 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     for (int w = 0; w < kRefineWarps; ++w) am = fmaxf(am, redf[w]);
     int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
     ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
-    const float ts = __uint_as_float((uint32_t)((T.xq_e2m1 ? 1 : 6) - ex + 127) << 23);
+    const float ts = __uint_as_float((uint32_t)((T.xq_mode == 1 ? 1 : 6) - ex + 127) << 23);
     const uint16_t* xr = static_cast<const uint16_t*>(x) + (size_t)t * H;
-    if (T.xq_e2m1) {
+    if (T.xq_mode >= 2) {
+      // FP8 1x128 quantisation: a warp's 32 lanes x 4 elements are one block (H % 128 == 0 here)
+      uint8_t* row = T.xq + (size_t)(2 * t) * T.xq_stride;
+      for (int i = tid - 32; i < H / 4; i += kRefineThreads - 32) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(xr + i * 4));
+        const float v[4] = {__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xffff0000u),
+                            __uint_as_float(q.y << 16), __uint_as_float(q.y & 0xffff0000u)};
+        float bm = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+        const float s = act_scale(bm, T.xq_mode - 1);
+        *reinterpret_cast<uint32_t*>(row + i * 4) =
+            act_code(v[0], s) | (act_code(v[1], s) << 8) | (act_code(v[2], s) << 16) | (act_code(v[3], s) << 24);
+        if (lane == 0) T.xs[(size_t)t * (H / 128) + i / 32] = s;
+      }
+    } else if (T.xq_mode == 1) {
       uint8_t* rows = T.xq + (size_t)(4 * t) * T.xq_stride;
       for (int i = tid - 32; i < H / 8; i += kRefineThreads - 32) {  // 8 elements -> 4 bytes of every term row
         const uint4 q = __ldg(reinterpret_cast<const uint4*>(xr + i * 8));
@@ -680,7 +695,8 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       for (int w = 0; w < kRefineWarps; ++w) am = fmaxf(am, redf[w]);
       int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
       ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
-      T.tok_scale[t] = __uint_as_float((uint32_t)((T.xq != nullptr && T.xq_e2m1 ? 1 : 6) - ex + 127) << 23);
+      T.tok_scale[t] = (T.xq != nullptr && T.xq_mode >= 2) ? 1.f
+                       : __uint_as_float((uint32_t)((T.xq != nullptr && T.xq_mode == 1 ? 1 : 6) - ex + 127) << 23);
     }
     // router weights of the k selected experts (lane j owns the j-th); binary32 is ample for
     // weights that are compared to 1e-5: the differences are formed in fp64 first
