@@ -371,17 +371,16 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     float4 sacc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (g < G) {
       const float* pp = part + (size_t)t * E + 4 * q;
-      int c = g;
-      for (; c + 7 * G < n_slices; c += 8 * G) {
+      // batches of eight loads, the last one predicated (a tail of dependent single loads would
+      // cost one L2 latency each); slices past the end add zero
+      for (int c = g; c < n_slices; c += 8 * G) {
         float4 v[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[i] = __ldg(reinterpret_cast<const float4*>(pp + (size_t)(c + i * G) * cs));
+        for (int i = 0; i < 8; ++i)
+          v[i] = (c + i * G < n_slices) ? __ldg(reinterpret_cast<const float4*>(pp + (size_t)(c + i * G) * cs))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int i = 0; i < 8; ++i) { sacc.x += v[i].x; sacc.y += v[i].y; sacc.z += v[i].z; sacc.w += v[i].w; }
-      }
-      for (; c < n_slices; c += G) {
-        const float4 v = __ldg(reinterpret_cast<const float4*>(pp + (size_t)c * cs));
-        sacc.x += v.x; sacc.y += v.y; sacc.z += v.z; sacc.w += v.w;
       }
       *reinterpret_cast<float4*>(&psum[g * E + 4 * q]) = sacc;
     }
@@ -400,15 +399,13 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       const int e = act ? idx / split : 0, half = idx % split;
       const float* pp = part + (size_t)t * E + e;
       float sum = 0.f;
-      int c = act ? half : n_slices;
-      for (; c + 15 * split < n_slices; c += 16 * split) {
+      for (int c = act ? half : n_slices; c < n_slices; c += 16 * split) {  // batches of sixteen loads, the last one predicated
         float v[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = __ldg(pp + (size_t)(c + i * split) * cs);
+        for (int i = 0; i < 16; ++i) v[i] = (c + i * split < n_slices) ? __ldg(pp + (size_t)(c + i * split) * cs) : 0.f;
 #pragma unroll
         for (int i = 0; i < 16; ++i) sum += v[i];
       }
-      for (; c < n_slices; c += split) sum += __ldg(pp + (size_t)c * cs);
       if (split == 2) sum += __shfl_xor_sync(0xffffffffu, sum, 1);  // all lanes reach this point
       if (act && half == 0) l32[e] = sum;
     }
