@@ -61,6 +61,9 @@ struct Params {
   float* hq_f;           // [max_units][n_slices][32]: routing weight * 2^(e_r - 6) of the tile's tokens
   const uint8_t* xq;     // [gamma][2][H] e4m3 hi / lo terms of x * tok_scale (written by the routing kernels)
   uint8_t* xu;           // [max_units][H / 128][64 rows][128 B]: the unit's tokens' rows of xq, one tile per K chunk
+#ifdef MOEV_TC_STATS
+  unsigned long long* stats;  // [grid][16] cycles MMA issuer 0 spent per wait class (debug builds)
+#endif
 };
 __device__ void wide_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
                           const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up, const CUtensorMap& tm_sh_down,

@@ -291,8 +291,18 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
       bool ok = true;
       const uint32_t w_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(w_ring));
       const uint32_t b_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(b_tiles));
+#ifdef MOEV_TC_STATS
+      unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+      const long long st_begin = clock64();
+#endif
       for (;;) {
-        const int id = next_task(S, q, abortp, P.status, false);
+        int id;
+        { MOEV_STAT_BEGIN();
+          id = next_task(S, q, abortp, P.status, false);
+          MOEV_STAT_END(4); }
+#ifdef MOEV_TC_STATS
+        if (id >= 0) st_acc[7] += 1;
+#endif
         if (id < 0) break;
         const Task t = decode(id, n_units, n_slices, n_hp);
         const Unit u = P.units[t.unit];
@@ -301,8 +311,12 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         const bool mine = !t.phase2 || issuer == 0 || 2 * t.hp + 1 < HT;  // an odd last H tile has no partner
         for (int st = 0; st < n_st && ok; ++st, ++it) {
           const int s = it % kStages, pb = it & 1;
-          ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-          ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((it >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          { MOEV_STAT_BEGIN();
+            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            if (t.phase2) { MOEV_STAT_END(5); } else { MOEV_STAT_END(1); } }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((it >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            if (t.phase2) { MOEV_STAT_END(6); } else { MOEV_STAT_END(3); } }
           if (!ok) break;
           ptx::tc_fence_after();
           if (mine) {
@@ -317,6 +331,11 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         }
         if (!ok) break;
       }
+#ifdef MOEV_TC_STATS
+      st_acc[0] = (unsigned long long)(clock64() - st_begin);
+      if (P.stats && issuer == 0)
+        for (int i = 0; i < 13; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
+#endif
     }
   }
   else {

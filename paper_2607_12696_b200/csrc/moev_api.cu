@@ -273,6 +273,9 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   W.s_gate = P.s_gate; W.s_up = P.s_up; W.s_down = P.s_down;
   W.sh_s_gate = P.sh_s_gate; W.sh_s_up = P.sh_s_up; W.sh_s_down = P.sh_s_down;
   W.status = P.status; W.gamma = gamma; W.H = g.H; W.I = g.I; W.A = P.A;
+#ifdef MOEV_TC_STATS
+  W.stats = c->tc_stats;
+#endif
   W.wide = c->T.wide; W.unit_done = c->T.unit_done; W.hq = c->hq; W.hq_f = c->hq_f;
   W.xq = c->T.xq; W.xu = c->xu;
   launch_k(tc::grouped_ffn_tc_kernel<WFMT>, dim3(c->n_sm), dim3(tc::kThreads), tc::kSmemBytes, st, ev == nullptr,
