@@ -208,6 +208,10 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
       const uint32_t w_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(w_ring));
       const uint32_t b_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(b_tiles));
       const uint32_t h_lo0 = ptx::desc_lo_sw128(ptx::smem_u32(h_tile));
+#ifdef MOEV_TC_STATS
+      unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+      const long long st_begin = clock64();
+#endif
       for (;; ++tcount) {
         const int id = next_task(S, q, abortp, P.status, false);
         if (id < 0) break;
@@ -216,8 +220,12 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
         const uint32_t idesc = ptx::instr_desc(0, 0, (uint32_t)((2 * u.m + 15) & ~15));
         for (int kc = 0; kc < KC && ok; ++kc, ++it, ++pc) {
           const int s = it % kStages, pb = pc & 1;
-          ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-          ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((pc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          { MOEV_STAT_BEGIN();
+            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(1); }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((pc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(3); }
           if (!ok) break;
           ptx::tc_fence_after();
           const uint32_t wa = w_lo0 + s * (kStageBytes >> 4) + issuer * 1024;
@@ -229,13 +237,19 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           ptx::mma_commit(&S.w_empty[s]);
         }
         if (!ok) break;
-        ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+        { MOEV_STAT_BEGIN();
+          ok = ptx::bounded_wait(&S.h_full, tcount & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          MOEV_STAT_END(4); }
         if (!ok) break;
         ptx::tc_fence_after();
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++dsc, ++it) {
           const int db = dsc & 1, s = it % kStages;
-          ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
-          ok = ok && ptx::bounded_wait(&S.d_empty[db], ((dsc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+          { MOEV_STAT_BEGIN();
+            ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(5); }
+          { MOEV_STAT_BEGIN();
+            ok = ok && ptx::bounded_wait(&S.d_empty[db], ((dsc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            MOEV_STAT_END(6); }
           if (!ok) break;
           ptx::tc_fence_after();
           if (issuer == 0 || 2 * ds + 1 < HT) {
@@ -250,6 +264,12 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
       }
+#ifdef MOEV_TC_STATS
+      st_acc[0] = (unsigned long long)(clock64() - st_begin);
+      st_acc[7] = tcount;
+      if (P.stats && issuer == 0)
+        for (int i = 0; i < 13; ++i) P.stats[(size_t)blockIdx.x * 16 + i] = st_acc[i];
+#endif
     }
   }
   else {
