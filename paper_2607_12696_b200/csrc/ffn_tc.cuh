@@ -160,6 +160,14 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
   return __all_sync(0xffffffffu, ok);
 }
 
+// One arrival per warp on a barrier that a whole role group completes (its count is the number
+// of warps): every lane has finished its part (and executed its fences) before lane 0 arrives.
+// 256 single-thread arrivals on one barrier word serialise in shared memory.
+__device__ __forceinline__ void warp_arrive(uint64_t* bar) {
+  __syncwarp();
+  if ((threadIdx.x & 31) == 0) ptx::mbar_arrive(bar);
+}
+
 // Barrier among the 128 threads of one role group, built on an mbarrier so that it is bounded.
 __device__ __forceinline__ bool group_sync(uint64_t* bar, uint32_t& phase, volatile int* abortp, int* status) {
   ptx::mbar_arrive(bar);

@@ -28,6 +28,7 @@ using tc::kTaskQ;
 using tc::kWaitBudgetNs;
 using tc::sw128;
 using tc::warp_wait;
+using tc::warp_arrive;
 using tc::group_sync;
 using tc::safe_exponent;
 using tc::pow2i;
@@ -100,11 +101,11 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
     for (int i = 0; i < 2; ++i) {
-      ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 256);
-      ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 256);
+      ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 8);
+      ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 8);
     }
-    ptx::mbar_init(&S.x_full, 128); ptx::mbar_init(&S.x_empty, 128);
-    ptx::mbar_init(&S.h_full, 128); ptx::mbar_init(&S.h_empty, 2);
+    ptx::mbar_init(&S.x_full, 4); ptx::mbar_init(&S.x_empty, 4);
+    ptx::mbar_init(&S.h_full, 4); ptx::mbar_init(&S.h_empty, 2);
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     ptx::mbar_init(&S.all_bar, 256);
@@ -331,7 +332,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           ptx::tmem_ld16(src, o);
           ptx::tmem_ld_wait();
           ptx::tc_fence_before();
-          ptx::mbar_arrive(&S.p_empty[pb]);
+          warp_arrive(&S.p_empty[pb]);
 #pragma unroll
           for (int r = 0; r < 8; ++r) {
             if constexpr (ACTQ) acc[r] = fmaf(__uint_as_float(o[2 * r]) * (r < m ? S.sx[r][kc] : 0.f), sv, acc[r]);
@@ -353,7 +354,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
             }
           }
           ptx::tc_fence_before();
-          ptx::mbar_arrive(&S.p_empty[pb]);
+          warp_arrive(&S.p_empty[pb]);
         }
       }
       if (!ok) break;
@@ -368,7 +369,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
         tmem_st32(tmem + lane_base + kColD, acc);
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         ptx::tc_fence_before();
-        ptx::mbar_arrive(&S.x_full);
+        warp_arrive(&S.x_full);
       } else {
         ok = warp_wait(&S.x_full, tcount & 1, abortp, P.status);
         if (!ok) break;
@@ -380,7 +381,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           if (m > 16) ptx::tmem_ld16(tmem + lane_base + kColD + 16, *reinterpret_cast<uint32_t(*)[16]>(&pv[16]));
           ptx::tmem_ld_wait();
           ptx::tc_fence_before();
-          ptx::mbar_arrive(&S.x_empty);
+          warp_arrive(&S.x_empty);
 #pragma unroll
           for (int r = 0; r < kMC; ++r) {
             const float gg = acc[r], pp = __uint_as_float(pv[r]);
@@ -421,7 +422,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           }
         }
         ptx::fence_proxy_async_smem();
-        ptx::mbar_arrive(&S.h_full);
+        warp_arrive(&S.h_full);
       }
 
       // ---- down phase: tile `grp` of every stage; block scale * h scale * routing weight, one reduction per token
@@ -438,7 +439,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           if (have) ptx::tmem_ld16(src, o);
           ptx::tmem_ld_wait();
           ptx::tc_fence_before();
-          ptx::mbar_arrive(&S.d_empty[db]);
+          warp_arrive(&S.d_empty[db]);
           if (have) {
             const float sd = S.e_sd[par][ht];
             float* ycol = P.y32 + (size_t)ht * 128 + row;
@@ -469,7 +470,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
             }
           }
           ptx::tc_fence_before();
-          ptx::mbar_arrive(&S.d_empty[db]);
+          warp_arrive(&S.d_empty[db]);
         }
       }
       if (!ok) break;

@@ -43,6 +43,7 @@ using tc::kStageBytes;
 using tc::kTaskQ;
 using tc::kWaitBudgetNs;
 using tc::warp_wait;
+using tc::warp_arrive;
 using tc::group_sync;
 using tc::safe_exponent;
 using tc::pow2i;
@@ -152,8 +153,8 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
   __syncthreads();  // every thread has left the caller's use of shared memory
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 256); }
-    ptx::mbar_init(&S.x_full, 128); ptx::mbar_init(&S.x_empty, 128);
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 8); }
+    ptx::mbar_init(&S.x_full, 4); ptx::mbar_init(&S.x_empty, 4);
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     ptx::mbar_init(&S.all_bar, 256);
@@ -319,6 +320,7 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
             if (t.phase2) { MOEV_STAT_END(6); } else { MOEV_STAT_END(3); } }
           if (!ok) break;
           ptx::tc_fence_after();
+          { MOEV_STAT_BEGIN();
           if (mine) {
             const uint32_t wa = w_lo0 + s * (kStageBytes >> 4) + issuer * 1024;
             const uint32_t ba = b_lo0 + s * (kBTileBytes >> 4);
@@ -326,8 +328,11 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
 #pragma unroll
             for (int j = 0; j < 4; ++j) tc::issue_mma<WFMT>(d, wa + 2 * j, ba + 2 * j, idesc, j ? 1u : 0u);
           }
+          MOEV_STAT_END(8); }
+          { MOEV_STAT_BEGIN();
           ptx::mma_commit(&S.p_full[pb]);
           ptx::mma_commit(&S.w_empty[s]);
+          MOEV_STAT_END(9); }
         }
         if (!ok) break;
       }
@@ -347,6 +352,10 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
     const int row = qd * 32 + lane;   // row of the 128-row tile this thread owns
     uint32_t it = 0, q = 0, tcount = 0, gph = 0, xph = 0, aph = 0;
     bool ok = true;
+#ifdef MOEV_TC_STATS
+    unsigned long long est[3] = {0, 0, 0};
+    const long long est_begin = clock64();
+#endif
     for (;; ++tcount) {
       const int id = next_task(S, q, abortp, P.status, true);
       if (id < 0) break;
@@ -394,27 +403,37 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
       for (int r = 0; r < kMC; ++r) acc[r] = 0.f;
       for (int st = 0; st < n_st && ok; ++st, ++it) {
         const int pb = it & 1;
+#ifdef MOEV_TC_STATS
+        const long long e0 = clock64();
+#endif
         ok = warp_wait(&S.p_full[pb], (it >> 1) & 1, abortp, P.status);
+#ifdef MOEV_TC_STATS
+        est[0] += clock64() - e0;
+        est[2] += 1;
+#endif
         if (!ok) break;
         ptx::tc_fence_after();
         const float sv = S.s_tab[par][grp][st];
         const uint32_t src = tmem + lane_base + pb * 128 + grp * 64;
+        // 32 columns (16 tokens) per TMEM load: two load latencies per stage for a full unit
 #pragma unroll
-        for (int c0 = 0; c0 < 64; c0 += 16) {
+        for (int c0 = 0; c0 < 64; c0 += 32) {
           if (c0 < 2 * m) {
-            uint32_t o[16];
-            ptx::tmem_ld16(src + c0, o);
+            uint32_t o[32];
+            ptx::tmem_ld32(src + c0, o);
             ptx::tmem_ld_wait();
+            if (c0 + 32 >= 2 * m) {  // the last columns of the unit are in registers: hand the buffer back first
+              ptx::tc_fence_before();
+              warp_arrive(&S.p_empty[pb]);
+            }
 #pragma unroll
-            for (int r = 0; r < 8; ++r) {
+            for (int r = 0; r < 16; ++r) {
               const int tr = c0 / 2 + r;
               const float f = t.phase2 ? sv * S.f2[par][st][tr] : sv;
               acc[tr] = fmaf(__uint_as_float(o[2 * r]) + __uint_as_float(o[2 * r + 1]) * 0.0625f, f, acc[tr]);
             }
           }
         }
-        ptx::tc_fence_before();
-        ptx::mbar_arrive(&S.p_empty[pb]);
       }
       if (!ok) break;
 
@@ -438,7 +457,7 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         tmem_st32(tmem + lane_base + kColXchg, acc);
         asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         ptx::tc_fence_before();
-        ptx::mbar_arrive(&S.x_full);
+        warp_arrive(&S.x_full);
         ++xph;
         continue;
       }
@@ -452,7 +471,7 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         ptx::tmem_ld16(tmem + lane_base + kColXchg + 16, *reinterpret_cast<uint32_t(*)[16]>(&pv[16]));
         ptx::tmem_ld_wait();
         ptx::tc_fence_before();
-        ptx::mbar_arrive(&S.x_empty);
+        warp_arrive(&S.x_empty);
         ++xph;
 #pragma unroll
         for (int r = 0; r < kMC; ++r) {
@@ -495,6 +514,13 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         atomicAdd(P.unit_done + t.unit, 1);
       }
     }
+#ifdef MOEV_TC_STATS
+    if (warp == 2 && lane == 0 && P.stats) {  // epilogue group 0: cycles waiting for partial products, total, stages
+      P.stats[(size_t)blockIdx.x * 16 + 13] = est[0];
+      P.stats[(size_t)blockIdx.x * 16 + 14] = (unsigned long long)(clock64() - est_begin);
+      P.stats[(size_t)blockIdx.x * 16 + 15] = est[2];
+    }
+#endif
   }
   // the caller synchronises the CTA and releases TMEM
 }
