@@ -589,15 +589,22 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
              router_partial_mma_smem(c->ks), st, pdl && c->chain, static_cast<const uint16_t*>(x), layer->router_w,
              c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
   if (ev) cudaEventRecord(ev[1], st);
-  if (g.afmt == MOEV_ACT_FP32)
-    launch_k(topk_refine_kernel<MOEV_ACT_FP32>, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x,
-             layer->router_w, (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma,
-             g.H, g.E, g.top_k, c->n_slices, c->ks, g.score, g.routed_scale, layer->router_bias, g.n_group, g.topk_group);
-  else
-    launch_k(topk_refine_kernel<MOEV_ACT_BF16>, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x,
-             layer->router_w, (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma,
-             g.H, g.E, g.top_k, c->n_slices, c->router_mma ? 6 * c->ks + c->n_slices + 12 : c->ks, g.score, g.routed_scale,
-             layer->router_bias, g.n_group, g.topk_group);
+  {
+    // the kernel's code is executed once per CTA, front to back: the plain and the group-limited
+    // routing are separate instantiations so that neither carries the other's instructions
+    const int refine_depth = c->router_mma ? 6 * c->ks + c->n_slices + 12 : c->ks;
+    auto go = [&](auto kern) {
+      launch_k(kern, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x, layer->router_w,
+               (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
+               g.top_k, c->n_slices, g.afmt == MOEV_ACT_FP32 ? c->ks : refine_depth, g.score, g.routed_scale,
+               layer->router_bias, g.n_group, g.topk_group);
+    };
+    if (g.afmt == MOEV_ACT_FP32) {
+      if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_FP32, true>); else go(topk_refine_kernel<MOEV_ACT_FP32, false>);
+    } else {
+      if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_BF16, true>); else go(topk_refine_kernel<MOEV_ACT_BF16, false>);
+    }
+  }
   if (ev) cudaEventRecord(ev[2], st);
   launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
            g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma), (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0);
@@ -740,13 +747,21 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
   const size_t rp_smem = router_partial_smem(ks);  // 17 KB: below the default dynamic limit, no attribute needed
   if (cfg->afmt == MOEV_ACT_FP32) {
     router_partial_kernel<MOEV_ACT_FP32><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
-    topk_refine_kernel<MOEV_ACT_FP32><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+    if (cfg->n_group > 0) topk_refine_kernel<MOEV_ACT_FP32, true><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
+                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
+                                                                       cfg->topk_group);
+    else topk_refine_kernel<MOEV_ACT_FP32, false><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
                                                                        gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
                                                                        cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
                                                                        cfg->topk_group);
   } else {
     router_partial_kernel<MOEV_ACT_BF16><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
-    topk_refine_kernel<MOEV_ACT_BF16><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+    if (cfg->n_group > 0) topk_refine_kernel<MOEV_ACT_BF16, true><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
+                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
+                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
+                                                                       cfg->topk_group);
+    else topk_refine_kernel<MOEV_ACT_BF16, false><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
                                                                        gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
                                                                        cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
                                                                        cfg->topk_group);

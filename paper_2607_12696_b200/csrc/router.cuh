@@ -313,7 +313,7 @@ constexpr int kRefineThreads = 512;
 constexpr int kRefineWarps = kRefineThreads / 32;
 constexpr int kRefineCand = 12;  // candidates re-evaluated per pass over the token's row
 
-template <int AFMT>
+template <int AFMT, bool GROUPED = false>
 __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, RouteOut O, const void* __restrict__ x,
                                                                      const float* __restrict__ router_w,
                                                                      const float* __restrict__ part,
@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   __syncthreads();  // l32, redf, redw complete
   // ---- fp32 top-k by counting: the k-th largest logit is the one preceded by exactly k - 1 others
   // (larger value, or equal value and lower id); E <= kRefineThreads
-  if (n_group > 0) {
+  if constexpr (GROUPED) {
     // group-limited routing takes its candidates in two stages, below
   } else if (2 * E <= kRefineThreads) {  // two threads per expert, each counts over half of the experts
     const int e = tid >> 1, hf = tid & 1;
@@ -452,7 +452,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     const float n_round = (float)(ks + n_slices + 4);
     const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
     bool in;
-    if (n_group > 0) {
+    if constexpr (GROUPED) {
       // ---- group stage.  c = sigmoid(logit) + bias in fp32 with error <= delta; a group's score is the sum of
       // its two largest c, so every expert within 2 delta of the group's second largest c is a candidate.
       const int gsz = E / n_group;
@@ -546,7 +546,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   };
   refine_range(0, ncand);
   MOEV_RT_MARK(4);
-  if (n_group > 0) {
+  if constexpr (GROUPED) {
     // ---- exact group scores from the group-stage candidates (they contain each group's two largest c)
     const int gsz = E / n_group, nA = ncand;
     if (tid < nA) Cx[tid] = 1.0 / (1.0 + exp(-L[tid])) + (router_bias ? (double)__ldg(router_bias + cand[tid]) : 0.0);
@@ -697,6 +697,9 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
     }
     // router weights of the k selected experts (lane j owns the j-th); binary32 is ample for
     // weights that are compared to 1e-5: the differences are formed in fp64 first
+#ifdef MOEV_TC_STATS
+    if (blockIdx.x == 0 && tid == 0) g_rt_stats[20] = clock64();
+#endif
     const double sel_v = lane < k ? sel_v_s[lane] : 0.0;
     const int sel_e = lane < k ? sel_e_s[lane] : -1;
     float wgt = 0.f;
@@ -710,6 +713,9 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       const float den = warp_sum(sg);
       wgt = routed_scale * sg / (den + 1e-20f);
     }
+#ifdef MOEV_TC_STATS
+    if (blockIdx.x == 0 && tid == 0) g_rt_stats[21] = clock64();
+#endif
     if (lane < k) {
       int a = t * k + lane;
       T.topk_ids[a] = sel_e;
@@ -717,6 +723,9 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
       if (O.topk_ids) O.topk_ids[a] = sel_e;
       if (O.topk_w) O.topk_w[a] = wgt;
     }
+#ifdef MOEV_TC_STATS
+    if (blockIdx.x == 0 && tid == 0) g_rt_stats[22] = clock64();
+#endif
   }
   MOEV_RT_MARK(6);
 }
@@ -800,7 +809,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   // finishing times close together (clustered tree workload: FFN kernel 920 -> 895 us), while
   // expert order inside a class keeps concurrently running tasks on neighbouring experts.
   {
-    __shared__ int32_t warp_tot_cls[32];
+    __shared__ int32_t warp_tot_cls[32], tot_unit_s, tot_cls_s;
     const int U = n_union_s;
     const bool sorted = unit_cap <= 64;  // (the CUDA-core path has no cap and no use for the order)
     int e = 0, slot0 = 0, m = 0, shared = 0;
@@ -817,11 +826,19 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
     }
     if (lane == 31) { warp_tot_unit[warp] = sc; warp_tot_cls[warp] = spk; }
     __syncthreads();
-    int base = 0, total1 = 0, bpk = 0, tpk = 0;
-    for (int w = 0; w < 32; ++w) {
-      base += w < warp ? warp_tot_unit[w] : 0; total1 += warp_tot_unit[w];
-      bpk += w < warp ? warp_tot_cls[w] : 0; tpk += warp_tot_cls[w];
+    if (warp == 0) {  // exclusive prefixes of the 32 warp totals (and the grand totals) by one warp
+      const int wu = warp_tot_unit[lane], wc = warp_tot_cls[lane];
+      int su = wu, sk = wc;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int a = __shfl_up_sync(0xffffffffu, su, o), b = __shfl_up_sync(0xffffffffu, sk, o);
+        if (lane >= o) { su += a; sk += b; }
+      }
+      warp_tot_unit[lane] = su - wu; warp_tot_cls[lane] = sk - wc;
+      if (lane == 31) { tot_unit_s = su; tot_cls_s = sk; }
     }
+    __syncthreads();
+    const int base = warp_tot_unit[warp], total1 = tot_unit_s, bpk = warp_tot_cls[warp], tpk = tot_cls_s;
     int first = base + sc - nch;
     for (int c = 0; c < nch; ++c) {
       Unit un;
