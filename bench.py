@@ -67,7 +67,9 @@ DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 # streamed, so the full-size launch is scaled by the same ratio.  Absent = not captured.
 NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.439543e9 + 3.790336e6) / 2.422801920e9,
                      # profiles/grouped_ffn_mx_gptoss_g64.md: 1.518134 GB + 4.46 MB against 1.454112 GB
-                     ("mxfp4", "tcgen05"): (1.518134e9 + 4.463104e6) / 1.454112e9}
+                     ("mxfp4", "tcgen05"): (1.518134e9 + 4.463104e6) / 1.454112e9,
+                     # profiles/grouped_ffn_tc_bf16_E64_g16.md: 2.115337 GB + 3.93 MB against 2.113929 GB
+                     ("bf16", "tcgen05"): (2.115337e9 + 3.926784e6) / 2.113929216e9}
 
 ROUTING = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing,
            "clustered": synth.make_clustered_routing, "exact": synth.make_exact_union_routing,
