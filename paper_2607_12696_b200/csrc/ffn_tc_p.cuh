@@ -282,6 +282,10 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
     const int row = qd * 32 + lane;
     uint32_t pc = 0, dsc = 0, q = 0, tcount = 0, gph = 0, aph = 0;
     bool ok = true;
+#ifdef MOEV_TC_STATS
+    unsigned long long est[3] = {0, 0, 0};
+    long long e_mark = 0;
+#endif
     for (;; ++tcount) {
       const int id = next_task(S, q, abortp, P.status, true);
       if (id < 0) break;
@@ -358,8 +362,17 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
         }
       }
       if (!ok) break;
+#ifdef MOEV_TC_STATS
+      e_mark = clock64();  // the last K chunk has been promoted
+#endif
+      // (token loops below run in blocks of eight under a warp-uniform test: a unit of a tree-sized
+      // call has two or three tokens, and 32 predicated bodies per step cost more than the step)
 #pragma unroll
-      for (int r = 0; r < kMC; ++r) acc[r] *= (r < m ? S.e_inv[par][r] : 0.f);
+      for (int c0 = 0; c0 < kMC; c0 += 8)
+        if (c0 < m) {
+#pragma unroll
+          for (int r = c0; r < c0 + 8; ++r) acc[r] *= (r < m ? S.e_inv[par][r] : 0.f);
+        }
 
       if (grp == 1) {
         // ---- P to the gate group through TMEM (the down-phase accumulators are idle now)
@@ -373,6 +386,9 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
       } else {
         ok = warp_wait(&S.x_full, tcount & 1, abortp, P.status);
         if (!ok) break;
+#ifdef MOEV_TC_STATS
+        { const long long now = clock64(); est[0] += now - e_mark; e_mark = now; }  // waited for the up group's sums
+#endif
         ptx::tc_fence_after();
         float hv[kMC];
         {
@@ -383,24 +399,37 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           ptx::tc_fence_before();
           warp_arrive(&S.x_empty);
 #pragma unroll
-          for (int r = 0; r < kMC; ++r) {
-            const float gg = acc[r], pp = __uint_as_float(pv[r]);
-            hv[r] = r < m ? gg / (1.f + __expf(-gg)) * pp : 0.f;
-          }
+          for (int c0 = 0; c0 < kMC; c0 += 8)
+            if (c0 < m) {
+#pragma unroll
+              for (int r = c0; r < c0 + 8; ++r) {
+                const float gg = acc[r], pp = __uint_as_float(pv[r]);
+                hv[r] = r < m ? gg / (1.f + __expf(-gg)) * pp : 0.f;
+              }
+            }
         }
         // h tile must be free: all down MMAs of the previous task have completed
         ok = warp_wait(&S.h_empty, (tcount & 1) ^ 1, abortp, P.status);
         if (!ok) break;
 #pragma unroll
-        for (int r = 0; r < kMC; ++r) {
-          if (r < m) {
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hv[r])));
-            if (lane == 0) S.e_amax[qd][r] = mx;
-          }
-        }
-        if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
+        for (int c0 = 0; c0 < kMC; c0 += 8)
+          if (c0 < m) {
 #pragma unroll
-        for (int r = 0; r < kMC; ++r) {
+            for (int r = c0; r < c0 + 8; ++r)
+              if (r < m) {
+                const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(hv[r])));
+                if (lane == 0) S.e_amax[qd][r] = mx;
+              }
+          }
+        if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
+#ifdef MOEV_TC_STATS
+        { const long long now = clock64(); est[1] += now - e_mark; e_mark = now; }  // SwiGLU, h_empty, amax exchange
+#endif
+#pragma unroll
+        for (int c0 = 0; c0 < kMC; c0 += 8) {
+        if (c0 >= m) continue;
+#pragma unroll
+        for (int r = c0; r < c0 + 8; ++r) {
           if (r < m) {
             const uint32_t mx = max(max(S.e_amax[0][r], S.e_amax[1][r]), max(S.e_amax[2][r], S.e_amax[3][r]));
             if constexpr (ACTQ) {  // the slice is one 1x128 block of h: a single e4m3 term with the block's scale
@@ -421,8 +450,12 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
             if (row == r) S.e_f[par][r] = S.e_w[par][r] * pow2i(er - 6);
           }
         }
+        }
         ptx::fence_proxy_async_smem();
         warp_arrive(&S.h_full);
+#ifdef MOEV_TC_STATS
+        est[2] += clock64() - e_mark;  // quantise and store h
+#endif
       }
 
       // ---- down phase: tile `grp` of every stage; block scale * h scale * routing weight, one reduction per token
@@ -475,6 +508,10 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
       }
       if (!ok) break;
     }
+#ifdef MOEV_TC_STATS
+    if (warp == 2 && lane == 0 && P.stats)
+      for (int i = 0; i < 3; ++i) P.stats[(size_t)blockIdx.x * 16 + 13 + i] = est[i];
+#endif
   }
   // the caller synchronises the CTA and releases TMEM
 }
