@@ -517,24 +517,37 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
         xv[0] = (double)f.x; xv[1] = (double)f.y; xv[2] = (double)f.z; xv[3] = (double)f.w;
         if (c0 == 0) amax = fmaxf(amax, fmaxf(fmaxf(fabsf(f.x), fabsf(f.y)), fmaxf(fabsf(f.z), fabsf(f.w))));
       }
+      // pairs of candidates under a CTA-uniform test: bodies past nc are skipped, not predicated
+      // (top-4 routing refines five or six candidates per token, top-8 about ten)
       float4 wv[kRefineCand];
 #pragma unroll
-      for (int q = 0; q < kRefineCand; ++q)
-        if (q < nc) wv[q] = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)cand[c0 + q] * H) + h4);
+      for (int q0 = 0; q0 < kRefineCand; q0 += 2)
+        if (q0 < nc) {
 #pragma unroll
-      for (int q = 0; q < kRefineCand; ++q)
-        if (q < nc) {
-          acc[q] = fma(xv[0], (double)wv[q].x, acc[q]); acc[q] = fma(xv[1], (double)wv[q].y, acc[q]);
-          acc[q] = fma(xv[2], (double)wv[q].z, acc[q]); acc[q] = fma(xv[3], (double)wv[q].w, acc[q]);
+          for (int q = q0; q < q0 + 2; ++q)
+            if (q < nc) wv[q] = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)cand[c0 + q] * H) + h4);
+        }
+#pragma unroll
+      for (int q0 = 0; q0 < kRefineCand; q0 += 2)
+        if (q0 < nc) {
+#pragma unroll
+          for (int q = q0; q < q0 + 2; ++q)
+            if (q < nc) {
+              acc[q] = fma(xv[0], (double)wv[q].x, acc[q]); acc[q] = fma(xv[1], (double)wv[q].y, acc[q]);
+              acc[q] = fma(xv[2], (double)wv[q].z, acc[q]); acc[q] = fma(xv[3], (double)wv[q].w, acc[q]);
+            }
         }
     }
 #pragma unroll
-    for (int q = 0; q < kRefineCand; ++q) {
-      if (q < nc) {
-        double a = warp_sum(acc[q]);
-        if (lane == 0) red[warp][q] = a;
+    for (int q0 = 0; q0 < kRefineCand; q0 += 2)
+      if (q0 < nc) {
+#pragma unroll
+        for (int q = q0; q < q0 + 2; ++q)
+          if (q < nc) {
+            double a = warp_sum(acc[q]);
+            if (lane == 0) red[warp][q] = a;
+          }
       }
-    }
     __syncthreads();
     if (tid < nc) {
       double a = 0.0;
