@@ -238,8 +238,11 @@ moev_status moev_verify_pipeline(moev_ctx* ctx, int32_t n_layers, const moev_lay
  *   |E_traj(i)|, buffer not updated.
  * Outputs: selected [gamma] (first min(gamma, n) entries, in selection order), costs [gamma]
  * (cost of each choice when it was made; may be NULL), buffer_out [W] (final B; may be NULL),
- * n_selected [1] (may be NULL).  traj_workspace [n, W] is caller-provided scratch.  All
- * pointers are DEVICE pointers; one kernel is enqueued on cuda_stream; nothing is allocated.
+ * n_selected [1] (may be NULL; -1 if a bounded device wait expired).  traj_workspace is
+ * caller-provided scratch of n * W + 516 32-bit words (the path footprints, then control words).
+ * All pointers are DEVICE pointers; one kernel (for bitmaps too long for one CTA's shared memory:
+ * one memset and one cooperative kernel over several CTAs) is enqueued on cuda_stream; nothing is
+ * allocated.
  * MOEV_EINVAL for n outside 1..4096, W < 1, gamma < 1, eps <= 0, null required pointers, or
  * tables too large for shared memory (3 n + 4 W words above ~50 000). */
 moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, const float* P,

@@ -165,7 +165,7 @@ def select_drafts(parent: torch.Tensor, P: torch.Tensor, pred: torch.Tensor, gam
                   buffer0: torch.Tensor = None, global_cost: bool = False, out: tuple = None):
     """moev_select_drafts: Algorithm 1 on device tensors (parent int32 [n], P float32 [n], pred
     int32/uint32 bitmaps [n, W]).  Returns device tensors (selected [gamma], costs [gamma],
-    buffer [W], n_selected [1], workspace [n, W]); asynchronous on the current stream.  Pass the
+    buffer [W], n_selected [1], workspace [n * W + 516]); asynchronous on the current stream.  Pass the
     tuple a previous call returned as ``out`` to reuse its tensors (no allocation)."""
     n, W = pred.shape
     dev = pred.device
@@ -174,7 +174,7 @@ def select_drafts(parent: torch.Tensor, P: torch.Tensor, pred: torch.Tensor, gam
                torch.zeros(gamma, dtype=torch.int32, device=dev),
                torch.zeros(W, dtype=torch.int32, device=dev),
                torch.zeros(1, dtype=torch.int32, device=dev),
-               torch.empty(n, W, dtype=torch.int32, device=dev))
+               torch.empty(n * W + 516, dtype=torch.int32, device=dev))
     selected, costs, buf, nsel, traj = out
     st = lib().moev_select_drafts(n, W, parent.data_ptr(), P.data_ptr(), pred.data_ptr(), _ptr(buffer0), gamma,
                                   eps, int(global_cost), traj.data_ptr(), selected.data_ptr(), costs.data_ptr(),

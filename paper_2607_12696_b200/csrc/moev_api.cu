@@ -1,4 +1,5 @@
 // Host side of the C ABI declared in include/moev.h: context, validation, launches.
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -776,12 +777,40 @@ moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, cons
   if (n < 1 || n > kSelMaxNodes || W < 1 || gamma < 1 || !parent || !P || !pred || !traj_workspace || !selected)
     return MOEV_EINVAL;
   if (!(eps > 0.f)) return MOEV_EINVAL;  // eps avoids the division by zero (Eq. 9)
-  const size_t fixed = select_fixed_smem_words(n, W) * sizeof(uint32_t);
   constexpr size_t kBudget = 200 * 1024;
-  if (fixed > kBudget) return MOEV_EINVAL;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t fixed = select_fixed_smem_words(n, W) * sizeof(uint32_t);
   // the footprints are copied to shared memory when they fit beside the tables
   const size_t traj_bytes = (size_t)n * (size_t)(W | 1) * sizeof(uint32_t);
-  const int in_smem = fixed + traj_bytes <= kBudget;
+  const bool in_smem = fixed + traj_bytes <= kBudget;
+  if (!in_smem && !global_cost) {
+    // long bitmaps: the footprints spread over the shared memory of several CTAs (cooperative launch)
+    const size_t per_node = (size_t)W * sizeof(uint32_t) + 12;
+    const size_t base = ((size_t)n + 2 * (size_t)W + 64) * sizeof(uint32_t);
+    if (base + per_node > kBudget) return MOEV_EINVAL;
+    const int npc_max = (int)((kBudget - base) / per_node);
+    int G = (n + npc_max - 1) / npc_max;
+    G = std::max(G, std::min(32, (n + 31) / 32));  // also enough CTAs that a round's sweep is short
+    if (G > kSelGridMax) return MOEV_EINVAL;
+    int npc = (n + G - 1) / G;
+    const size_t smem = select_grid_smem_words(n, W, npc) * sizeof(uint32_t);
+    if (cudaFuncSetAttribute(select_drafts_grid_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBudget) !=
+        cudaSuccess) {
+      cudaGetLastError();
+      return MOEV_ECUDA;
+    }
+    uint32_t* ctlw = traj_workspace + (((size_t)n * W + 3) & ~(size_t)3);
+    if (cudaMemsetAsync(ctlw, 0, kSelCtlWords * sizeof(uint32_t), st) != cudaSuccess) return MOEV_ECUDA;
+    void* args[] = {&n, &W, &parent, &P, &pred, &buffer0, &gamma, &eps, &npc, &traj_workspace, &ctlw,
+                    &selected, &costs, &buffer_out, &n_selected};
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(select_drafts_grid_kernel), dim3(G),
+                                    dim3(kSelGridThreads), args, smem, st) != cudaSuccess) {
+      cudaGetLastError();
+      return MOEV_ECUDA;
+    }
+    return MOEV_OK;
+  }
+  if (fixed > kBudget) return MOEV_EINVAL;
   const size_t smem = fixed + (in_smem ? traj_bytes : 0);
   if (smem > 48 * 1024 &&
       cudaFuncSetAttribute(select_drafts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kBudget) != cudaSuccess) {
@@ -790,8 +819,8 @@ moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, cons
   }
   int threads = (n + 31) & ~31;
   threads = threads < 128 ? 128 : (threads > kSelThreads ? kSelThreads : threads);
-  select_drafts_kernel<<<1, threads, smem, static_cast<cudaStream_t>(cuda_stream)>>>(
-      n, W, parent, P, pred, buffer0, gamma, eps, global_cost, in_smem, traj_workspace, selected, costs, buffer_out,
+  select_drafts_kernel<<<1, threads, smem, st>>>(
+      n, W, parent, P, pred, buffer0, gamma, eps, global_cost, in_smem ? 1 : 0, traj_workspace, selected, costs, buffer_out,
       n_selected);
   return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
 }

@@ -40,6 +40,30 @@ def test_selection_matches_oracle(L, E, K, depth, branch, gamma):
         np.testing.assert_array_equal(b, b_ref)
 
 
+@pytest.mark.parametrize("L,E,K,depth,gamma,ties", [
+    (58, 256, 8, 7, 64, False),    # 255 nodes x 464 words: footprints over 8 CTAs' shared memory
+    (58, 256, 8, 9, 128, False),   # 1023 nodes: 32 CTAs
+    (94, 128, 8, 6, 40, True),     # 127 nodes x 376 words, coarse probabilities (many exact score ties), initial buffer
+    (61, 96, 6, 7, 300, False)])   # 183 words (not a multiple of four), budget larger than the tree
+def test_selection_long_bitmaps_several_ctas(L, E, K, depth, gamma, ties):
+    """Bitmaps too long for one CTA's shared memory take the cooperative multi-CTA kernel: same
+    selections, costs and final buffer, bit for bit."""
+    parent, P, pred = synth.make_draft_tree(L, E, K, depth=depth)
+    b0 = None
+    if ties:
+        P = (np.round(P * 8) / 8).astype(np.float32)
+        P[0] = 1.0
+        b0 = np.random.RandomState(5).randint(0, 2 ** 32, size=pred.shape[1], dtype=np.uint64).astype(np.uint32)
+        b0 &= np.random.RandomState(6).randint(0, 2 ** 32, size=pred.shape[1], dtype=np.uint64).astype(np.uint32)
+    eps = 0.5 if ties else 1e-6
+    s_ref, c_ref, b_ref = oracle.select_drafts(parent, P, pred, gamma, eps=eps, buffer0=b0)
+    for rep in range(2):                                     # twice: the control words are reset per call
+        s, c, b = _run(parent, P, pred, gamma, eps=eps, buffer0=b0)
+        np.testing.assert_array_equal(s, s_ref)
+        np.testing.assert_array_equal(c, c_ref)
+        np.testing.assert_array_equal(b, b_ref)
+
+
 def test_selection_with_initial_buffer_and_ties():
     parent, P, pred = synth.make_draft_tree(8, 64, 4, depth=4)
     b0 = np.random.RandomState(3).randint(0, 2 ** 32, size=pred.shape[1], dtype=np.uint64).astype(np.uint32)
