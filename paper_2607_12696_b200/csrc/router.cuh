@@ -824,7 +824,15 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   {
     __shared__ int32_t warp_tot_cls[32], tot_unit_s, tot_cls_s;
     const int U = n_union_s;
-    const bool sorted = unit_cap <= 64;  // (the CUDA-core path has no cap and no use for the order)
+    // many tokens per streamed expert: the two-phase FFN schedule (wide_ratio = 0: not available)
+    // (measured switch-over: above 8 assignments per streamed expert for small unions, where the weight stream
+    // is short, above 12 for large ones, where the two-phase schedule's re-streaming per 32-token unit costs more)
+    const int ut = U + n_shared;
+    const bool wide = T.wide != nullptr && wide_ratio > 0 &&
+                      (A + n_shared * gamma) > (ut < 100 ? wide_ratio : wide_ratio + wide_ratio / 2) * ut;
+    // the order by cost class is for the single-phase schedules; the two-phase one wants an expert's units next to
+    // each other (they re-read its weights through the L2), and the CUDA-core path has no cap and no use for units
+    const bool sorted = unit_cap <= 64 && !wide;
     int e = 0, slot0 = 0, m = 0, shared = 0;
     if (tid < n_shared) { shared = 1; e = tid; slot0 = A + e * gamma; m = gamma; }
     else if (tid < U + n_shared) { e = T.union_ids[tid - n_shared]; slot0 = T.offsets[tid - n_shared]; m = cnt[e]; }
@@ -871,13 +879,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
     if (tid == blockDim.x - 1) {
       *T.n_units = base + sc;
       *T.task_counter = 0;
-      // many tokens per streamed expert: the two-phase FFN schedule (wide_ratio = 0: not available)
-      // (measured switch-over: above 8 assignments per streamed expert for small unions, where the weight stream
-      // is short, above 12 for large ones, where the two-phase schedule's re-streaming per 32-token unit costs more)
-      if (T.wide) {
-        const int ut = U + n_shared, ratio = ut < 100 ? wide_ratio : wide_ratio + wide_ratio / 2;
-        *T.wide = (wide_ratio > 0 && (A + n_shared * gamma) > ratio * ut) ? 1 : 0;
-      }
+      if (T.wide) *T.wide = wide ? 1 : 0;
     }
     if (T.unit_done) {
       __shared__ int n_units_s;
