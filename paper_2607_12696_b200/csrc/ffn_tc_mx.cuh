@@ -473,6 +473,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         __threadfence();
         if (!(ok = group_sync(&S.ep_bar, gph, abortp, P.status))) break;
         if (warp == 2 && lane == 0) {
+          asm volatile("fence.proxy.async;" ::: "memory");  // the readers are TMA copies (async proxy) on other SMs
           __threadfence();
           atomicAdd(P.unit_done + t.unit, 1);
         }
