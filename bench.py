@@ -142,17 +142,135 @@ def workload_shape(name: str) -> synth.Shape:
     return shape
 
 
-def build_workload(name: str, n_layers: int, device, rank: int = 0):
+def build_workload(name: str, n_layers: int, device, rank: int = 0, weights=None):
+    """Inputs of a workload: per rotated layer its expert weights (generated, or taken from
+    ``weights`` when another workload of the same shape already made them), router and x."""
     base, gamma, routing, kw = WORKLOADS[name]
     shape = workload_shape(name)
     kw = {k: v for k, v in kw.items() if not k.startswith("_")}
     layers = []
     for l in range(n_layers):
         lid = rank * 1000 + l
-        w = synth.make_expert_weights(shape, layer=lid, device=device)
+        w = weights[l] if weights is not None else synth.make_expert_weights(shape, layer=lid, device=device)
         wr, x = ROUTING[routing](shape, gamma, layer=lid, device=device, **kw)
         layers.append({"weights": w, "router_w": wr, "x": x})
     return shape, gamma, layers
+
+
+def pack_layers(moev, layers):
+    packed = []
+    for L in layers:
+        d = {"router_w": L["router_w"]}
+        d.update({k: t for k, t in L["weights"].items() if t is not None})
+        packed.append((moev.binding.make_layer(d), d))
+    return packed
+
+
+def time_calls(v, packed, xs, outs, gamma, steps, warmup):
+    """Per-call latency of moev_verify (layers rotated call by call): a CUDA-event pair around
+    every call, then the same calls once more with the per-kernel event records on.  Returns
+    (sorted latencies in us, per-kernel mean us)."""
+    n = len(packed)
+    for i in range(max(warmup, n)):
+        v.verify(packed[i % n][0], xs[i % n], gamma, outs[i % n])
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i, (e0, e1) in enumerate(evs):
+        e0.record()
+        v.verify(packed[i % n][0], xs[i % n], gamma, outs[i % n])
+        e1.record()
+    torch.cuda.synchronize()
+    lat = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
+    v.profile_enable(True)
+    for i in range(steps):
+        v.verify(packed[i % n][0], xs[i % n], gamma, outs[i % n])
+    kern_us, _ = v.profile_read()
+    v.profile_enable(False)
+    v.status_sync()
+    return lat, kern_us
+
+
+def fit_line(pts):
+    """Least-squares latency = a + b U over (U, latency) points; returns None with fewer than two."""
+    if len(pts) < 2:
+        return None
+    u = np.array([p[0] for p in pts], dtype=np.float64)
+    t = np.array([p[1] for p in pts], dtype=np.float64)
+    b, a = np.polyfit(u, t, 1)
+    r2 = 1.0 - ((t - (a + b * u)) ** 2).sum() / max(((t - t.mean()) ** 2).sum(), 1e-30)
+    return {"a_us": float(a), "b_us_per_expert": float(b), "r2": float(r2)}
+
+
+def run_config_entry(moev, name, dev, weights, steps, warmup, peak):
+    """One entry of the bench line's ``configs`` array: a benchmark configuration timed call by
+    call (median of ``steps``), with the FFN kernel's own time and the clocks seen."""
+    n_layers = len(weights)
+    shape, gamma, layers = build_workload(name, n_layers, dev, weights=weights)
+    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, gamma, shape.wfmt,
+                          shape.afmt, shape.score, moev.IMPL_AUTO, shape.routed_scale)
+    v = moev.MoeVerifier(cfg)
+    Wb = moev.expert_bytes(cfg)
+    packed = pack_layers(moev, layers)
+    xs = [L["x"] for L in layers]
+    outs = [v.alloc_out(gamma, diagnostics=False) for _ in layers]
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    lat, kern_us = time_calls(v, packed, xs, outs, gamma, steps, warmup)
+    clocks = sampler.stop()
+    U = [int(o["n_active"].item()) for o in outs]
+    nbytes = (float(np.mean(U)) + shape.n_shared) * Wb
+    med = lat[len(lat) // 2]
+    v.close()
+    return {"workload": name, "gamma": gamma, "U": U, "latency_us": med, "latency_min_us": lat[0],
+            "gbs": nbytes / med / 1e3, "frac_of_8TBps": nbytes / med / 1e3 / NOMINAL_HBM_GBS,
+            "ffn_kernel_us": kern_us[3], "ffn_frac_of_measured": nbytes / kern_us[3] / 1e3 / peak,
+            "routing_us": kern_us[0] + kern_us[1] + kern_us[2], "calls": steps,
+            "clocks": {"sm_mhz": clocks["sm_mhz"], "reasons": clocks["reasons"]}}
+
+
+def run_sweep_cells(moev, dev, weights, gammas, unions, steps, warmup, peak, emit=None):
+    """Unique-expert sweep at the DeepSeek FP8 shape: routing built so that the union is exactly U.
+    Returns (cells, fits per gamma)."""
+    shape = synth.SHAPES["deepseek"]
+    n_layers = len(weights)
+    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, max(gammas), shape.wfmt,
+                          shape.afmt, shape.score, moev.IMPL_AUTO, shape.routed_scale)
+    v = moev.MoeVerifier(cfg)
+    Wb = moev.expert_bytes(cfg)
+    cells, fits = [], {}
+    for gamma in gammas:
+        pts = []
+        for U in unions:
+            cell = {"gamma": gamma, "U": U}
+            if not synth.union_feasible(shape, gamma, U):
+                cell["latency_us"] = "n/a"
+            else:
+                layers = []
+                for l in range(n_layers):
+                    wr, x = synth.make_exact_union_routing(shape, gamma, U, layer=l, device=dev)
+                    layers.append({"weights": weights[l], "router_w": wr, "x": x})
+                packed = pack_layers(moev, layers)
+                xs = [L["x"] for L in layers]
+                outs = [v.alloc_out(gamma, diagnostics=False) for _ in layers]
+                lat, kern_us = time_calls(v, packed, xs, outs, gamma, steps, warmup)
+                assert all(int(o["n_active"].item()) == U for o in outs)
+                med = lat[len(lat) // 2]
+                nbytes = (U + shape.n_shared) * Wb
+                cell.update(latency_us=med, latency_min_us=lat[0], latency_p90_us=lat[int(0.9 * len(lat))],
+                            ffn_kernel_us=kern_us[3], routing_us=kern_us[0] + kern_us[1] + kern_us[2],
+                            bytes=nbytes, gbs=nbytes / med / 1e3,
+                            frac_of_8TBps=nbytes / med / 1e3 / NOMINAL_HBM_GBS,
+                            frac_of_measured=nbytes / med / 1e3 / peak, roofline_us_8TBps=nbytes / 8e6)
+                pts.append((U, med))
+            cells.append(cell)
+            if emit:
+                emit(dict(cell, sweep="unique_experts"))
+        f = fit_line(pts)
+        if f:
+            f["roofline_b_us_per_expert_8TBps"] = Wb / 8e6
+            fits[str(gamma)] = f
+    v.close()
+    return cells, fits
 
 
 def layers_that_fit(shape: synth.Shape, want: int = 4) -> int:
@@ -251,11 +369,7 @@ def run_ours(args):
     cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, gamma, shape.wfmt,
                           shape.afmt, shape.score, impl, shape.routed_scale, act_quant=ACT_QUANT)
     v = moev.MoeVerifier(cfg)
-    packed = []
-    for L in layers:
-        d = {"router_w": L["router_w"]}
-        d.update({k: t for k, t in L["weights"].items() if t is not None})
-        packed.append((moev.binding.make_layer(d), d))
+    packed = pack_layers(moev, layers)
     outs = [v.alloc_out(gamma, diagnostics=False) for _ in layers]
     Wb = moev.expert_bytes(cfg)
 
@@ -358,6 +472,28 @@ def run_ours(args):
             cpu = {"value": cv, "unit": UNIT, "cores": cores, "kind": "oracle",
                    "sample": f"first {n_cpu} of the {gamma} tokens of layer 0 (U={cu}"
                              f"+{shape.n_shared} experts streamed), full layer weights, {cs:.2f} s"}
+        # ---- the other benchmark configurations and the unique-expert sweep, one after another
+        # (default workload on one GPU only; each entry is a median over event-timed calls)
+        configs, sweep_cells, sweep_fit = None, None, None
+        if args.workload == DEFAULT_WORKLOAD and world == 1 and not args.no_configs and ACT_QUANT == 0:
+            cs_, cw = args.config_steps, 5
+            ds_w = [L["weights"] for L in layers]
+            configs = [run_config_entry(moev, "deepseek_fp8_g64_scattered", dev, ds_w, cs_, cw, peak),
+                       run_config_entry(moev, "deepseek_fp8_g64_clustered", dev, ds_w, cs_, cw, peak)]
+            sweep_cells, sweep_fit = run_sweep_cells(moev, dev, ds_w, [1, 4, 8, 32], [8, 16, 32, 64, 128, 256],
+                                                     max(20, cs_ // 2), cw, peak)
+            del ds_w, packed
+            layers.clear()
+            torch.cuda.empty_cache()
+            for base, names in (("qwen", ["qwen_bf16_g16", "qwen_bf16_g32", "qwen_bf16_g64"]),
+                                ("gptoss", ["gptoss_mxfp4_g8", "gptoss_mxfp4_g16", "gptoss_mxfp4_g32",
+                                            "gptoss_mxfp4_g64"])):
+                shp = synth.SHAPES[base]
+                ws = [synth.make_expert_weights(shp, layer=l, device=dev) for l in range(layers_that_fit(shp, 4))]
+                for nm in names:
+                    configs.append(run_config_entry(moev, nm, dev, ws, cs_, cw, peak))
+                del ws
+                torch.cuda.empty_cache()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
@@ -395,6 +531,10 @@ def run_ours(args):
             "gpu_launches": v.launches_per_call() * args.steps,
             "clocks": clocks,
         }
+        if configs is not None:
+            line["configs"] = configs
+            line["sweep"] = sweep_cells
+            line["sweep_fit"] = sweep_fit
         print(json.dumps(line))
     v.close()
     if dist:
@@ -404,7 +544,7 @@ def run_ours(args):
 
 def run_sweep(args):
     """Unique-expert sweep at the DeepSeek FP8 shape: routing built so that the union is exactly
-    U, for gamma in {1, 8, 32, 128}; 4 layers' weights rotated per call.  Prints one JSON line
+    U, for gamma in {1, 4, 8, 32, 128}; 4 layers' weights rotated per call.  Prints one JSON line
     per cell plus a linear fit latency = a + b U per gamma (rank 0, one GPU)."""
     import paper_2607_12696_b200 as moev
     torch.cuda.set_device(0)
@@ -412,63 +552,12 @@ def run_sweep(args):
     shape = synth.SHAPES["deepseek"]
     n_layers = layers_that_fit(shape, args.layers)
     weights = [synth.make_expert_weights(shape, layer=l, device=dev) for l in range(n_layers)]
-    gammas, unions = [1, 8, 32, 128], [8, 16, 32, 64, 128, 256]
-    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, max(gammas), shape.wfmt,
-                          shape.afmt, shape.score, moev.IMPL_AUTO, shape.routed_scale)
-    v = moev.MoeVerifier(cfg)
-    Wb = moev.expert_bytes(cfg)
     peak, peak_src = measured_peaks()
-    fits = {}
-    for gamma in gammas:
-        pts = []
-        for U in unions:
-            cell = {"sweep": "unique_experts", "gamma": gamma, "U": U}
-            if not synth.union_feasible(shape, gamma, U):
-                cell["latency_us"] = "n/a"
-                print(json.dumps(cell))
-                continue
-            packed, xs, outs = [], [], []
-            for l in range(n_layers):
-                wr, x = synth.make_exact_union_routing(shape, gamma, U, layer=l, device=dev)
-                d = {"router_w": wr}
-                d.update({k: t for k, t in weights[l].items() if t is not None})
-                packed.append((moev.binding.make_layer(d), d))
-                xs.append(x)
-                outs.append(v.alloc_out(gamma, diagnostics=False))
-            for i in range(max(args.warmup, n_layers)):
-                v.verify(packed[i % n_layers][0], xs[i % n_layers], gamma, outs[i % n_layers])
-            torch.cuda.synchronize()
-            assert all(int(o["n_active"].item()) == U for o in outs)
-            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                   for _ in range(args.steps)]
-            v.profile_enable(True)
-            for i, (e0, e1) in enumerate(evs):
-                l = i % n_layers
-                e0.record()
-                v.verify(packed[l][0], xs[l], gamma, outs[l])
-                e1.record()
-            torch.cuda.synchronize()
-            kern_us, _ = v.profile_read()
-            v.profile_enable(False)
-            lat = sorted(a.elapsed_time(b) * 1e3 for a, b in evs)
-            med = lat[len(lat) // 2]
-            nbytes = (U + shape.n_shared) * Wb
-            cell.update(latency_us=med, latency_min_us=lat[0], latency_p90_us=lat[int(0.9 * len(lat))],
-                        ffn_kernel_us=kern_us[3], bytes=nbytes, gbs=nbytes / med / 1e3,
-                        frac_of_8TBps=nbytes / med / 1e3 / NOMINAL_HBM_GBS, frac_of_measured=nbytes / med / 1e3 / peak,
-                        roofline_us_8TBps=nbytes / 8e6)
-            print(json.dumps(cell))
-            pts.append((U, med))
-        if len(pts) >= 2:
-            u = np.array([p[0] for p in pts], dtype=np.float64)
-            t = np.array([p[1] for p in pts], dtype=np.float64)
-            b, a = np.polyfit(u, t, 1)
-            r2 = 1.0 - ((t - (a + b * u)) ** 2).sum() / max(((t - t.mean()) ** 2).sum(), 1e-30)
-            fits[gamma] = {"a_us": a, "b_us_per_expert": b, "r2": r2,
-                           "roofline_b_us_per_expert_8TBps": Wb / 8e6}
+    gammas = [int(g) for g in args.sweep_gammas.split(",")]
+    cells, fits = run_sweep_cells(moev, dev, weights, gammas, [8, 16, 32, 64, 128, 256], args.steps,
+                                  args.warmup, peak, emit=lambda c: print(json.dumps(c), flush=True))
     print(json.dumps({"sweep": "unique_experts", "fit_latency_us = a + b*U": fits,
                       "layers_rotated": n_layers, "peak_source": peak_src}))
-    v.close()
 
 
 def run_select_demo(args):
@@ -554,6 +643,10 @@ def main():
     ap.add_argument("--act-quant", type=int, default=0, choices=[0, 1, 2],
                     help="FP8 activations with 1x128 scales (1: binary32 scales, 2: power-of-two scales)")
     ap.add_argument("--sweep", action="store_true", help="unique-expert sweep (DeepSeek FP8 shape) instead of the bench line")
+    ap.add_argument("--sweep-gammas", default="1,4,8,32,128")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="default workload only: skip the other configurations and the sweep behind the headline")
+    ap.add_argument("--config-steps", type=int, default=50, help="timed calls per entry of the configs array")
     ap.add_argument("--select-demo", action="store_true",
                     help="cost-aware vs acceptance-only draft selection in front of the verification layer")
     ap.add_argument("--p-reuse", type=float, default=0.7, help="expert locality along a tree path (select demo)")

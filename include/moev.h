@@ -11,7 +11,8 @@
  * and reports the per-layer active-expert count.
  *
  * Paper passages the operations follow:
- *   - Sec. 1: "a router assigns each token to a small top-k subset of experts".
+ *   - Sec. 1: top-k routing -- the router scores the E experts for every token and the
+ *     token is processed by its k best-scoring experts only.
  *   - Eq. 1 (Sec. 3): the verification footprint is the union over the gamma
  *     verified tokens of their expert sets; its size -- not gamma -- drives the
  *     cost, because the verifier fetches every expert of the union from HBM and
@@ -127,7 +128,9 @@ typedef struct {
  *   s_*   FP8 : float32 [E, ceil(N/128), ceil(K/128)]   (N = rows of the matrix)
  *         MXFP4: uint8  [E, N, K/32]                     else NULL
  *   sh_*  the same for the n_shared shared experts (leading dim n_shared), NULL if none.
- * Every pointer must be 16-byte aligned. */
+ * Every pointer must be 16-byte aligned; on the tensor-core path (moev_resolved_impl ==
+ * MOEV_IMPL_TCGEN05) the six expert weight tensors w_* and sh_* must be 32-byte aligned (they
+ * are read through TMA descriptors).  A misaligned pointer is rejected with MOEV_EINVAL. */
 typedef struct {
   const float* router_w;
   const void *w_gate, *w_up, *w_down;
@@ -239,7 +242,9 @@ moev_status moev_verify_pipeline(moev_ctx* ctx, int32_t n_layers, const moev_lay
  * Outputs: selected [gamma] (first min(gamma, n) entries, in selection order), costs [gamma]
  * (cost of each choice when it was made; may be NULL), buffer_out [W] (final B; may be NULL),
  * n_selected [1] (may be NULL; -1 if a bounded device wait expired).  traj_workspace is
- * caller-provided scratch of n * W + 516 32-bit words (the path footprints, then control words).
+ * caller-provided scratch of n * W + 516 32-bit words (the path footprints, then control words);
+ * it must be 16-byte aligned (the control words are accessed as 64-bit and 128-bit quantities),
+ * otherwise MOEV_EINVAL.
  * All pointers are DEVICE pointers; one kernel (for bitmaps too long for one CTA's shared memory:
  * one memset and one cooperative kernel over several CTAs) is enqueued on cuda_stream; nothing is
  * allocated.
@@ -261,9 +266,11 @@ moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, cons
  * allocates the workspace), but may still want the routing decision of a layer.
  *
  * Computes, for the gamma tokens x [gamma, H] (afmt of cfg), the same topk_ids [gamma, k] and
- * topk_w [gamma, k] that moev_verify writes, using cfg->H, E, top_k, afmt, score,
- * routed_scale and max_tokens (gamma <= max_tokens); all pointers are DEVICE pointers owned by
- * the caller.  The split-K partial logits live in a fixed 20 MiB array compiled into the
+ * topk_w [gamma, k] that moev_verify writes for plain top-k routing.  Of cfg it reads H, E,
+ * top_k, afmt, score, routed_scale and max_tokens (gamma <= max_tokens); the other fields must
+ * merely be valid.  Group-limited routing needs the layer's score-correction bias, which this
+ * entry point does not take: cfg->n_group > 0 is rejected with MOEV_EINVAL.  All pointers are
+ * DEVICE pointers owned by the caller.  The split-K partial logits live in a fixed 20 MiB array compiled into the
  * library (held by every GPU that loads it until the process exits) instead of a context
  * workspace; moev_route_topk_static_scratch_floats() returns how many of its 5 242 880 floats a
  * problem needs, and problems that need more are rejected with MOEV_EINVAL.  The call itself

@@ -166,8 +166,8 @@ int64_t oracle_expert_scale_bytes(const oracle_cfg *c) {
 
 /* ------------------------------------------------------------------ router */
 
-/* logits[t,e] = sum_h x[t,h] * Wr[e,h], summed in index order (Sec. 1: "a
- * router assigns each token to a small top-k subset of experts"). */
+/* logits[t,e] = sum_h x[t,h] * Wr[e,h], summed in index order (Sec. 1: the router's
+ * per-token scores over the E experts, from which each token's top-k experts are taken). */
 void oracle_router_logits(const oracle_cfg *c, const void *x, const float *router_w, int32_t gamma,
                           double *logits) {
   int64_t H = c->H, E = c->E;

@@ -129,13 +129,12 @@ cudaError_t dmalloc(T** p, size_t count) {
   return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
 }
 
-bool route_use_bitmap(const moev_config& c, int gamma) { return route_bitmap_bytes(c.E, gamma) <= kRouteBitmapBudget; }
 // assignments per streamed expert above which the two-phase FFN kernel takes the call
 constexpr int kWideRatio = 8;
 // dynamic shared memory of topk_refine_kernel: three double, three 32-bit and one 8-bit array of E entries
 size_t refine_smem_bytes(int E) { return ((size_t)E * 41 + 15) & ~size_t(15); }
 size_t route_smem(const moev_config& c, int gamma) {
-  return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + (route_use_bitmap(c, gamma) ? route_bitmap_bytes(c.E, gamma) : 0);
+  return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + route_bitmap_bytes(c.E, gamma);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -485,11 +484,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
 #endif
   // opt in to large dynamic shared memory where the shape needs it
   if (ok) {
-    size_t gs = route_smem(*cfg, cfg->max_tokens);
-    {  // the largest gamma that still uses the token bitmaps may need more than max_tokens does
-      const int g_bm = (int)(kRouteBitmapBudget / (4 * (size_t)cfg->E)) * 32;
-      if (g_bm < cfg->max_tokens && g_bm >= 1) gs = gs > route_smem(*cfg, g_bm) ? gs : route_smem(*cfg, g_bm);
-    }
+    const size_t gs = route_smem(*cfg, cfg->max_tokens);
     ok = ok && cudaFuncSetAttribute(router_partial_kernel<MOEV_ACT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)router_partial_smem(kRouterMaxKS)) == cudaSuccess;
     ok = ok && cudaFuncSetAttribute(router_partial_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -566,6 +561,10 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
 
   const TmapSet* tm = nullptr;
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
+    const void* wptrs[] = {layer->w_gate, layer->w_up, layer->w_down, layer->sh_gate, layer->sh_up, layer->sh_down};
+    for (const void* p : wptrs)
+      if (p && (reinterpret_cast<uintptr_t>(p) & 31u))
+        return fail(c, MOEV_EINVAL, "expert weight tensor %p is not 32-byte aligned (tensor-core path)", p);
     tm = get_tmaps(c, layer);
     if (!tm) return fail(c, MOEV_ECUDA, "cuTensorMapEncodeTiled failed for this layer's weight tensors");
   }
@@ -608,7 +607,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   }
   if (ev) cudaEventRecord(ev[2], st);
   launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
-           g.n_shared, c->unit_cap, (int)route_use_bitmap(g, gamma), (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0);
+           g.n_shared, c->unit_cap, (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0);
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);
@@ -719,6 +718,7 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
   if (!cfg_ok(cfg, why, sizeof(why))) return MOEV_EINVAL;
   if (!router_w || !x || !topk_ids || !topk_w || gamma < 1 || gamma > cfg->max_tokens) return MOEV_EINVAL;
   if (!aligned16(router_w) || !aligned16(x)) return MOEV_EINVAL;
+  if (cfg->n_group > 0) return MOEV_EINVAL;  // group-limited routing needs the layer's bias, which this call does not take
   if (moev_route_topk_static_scratch_floats(cfg->H, cfg->E, gamma) > kStaticScratchFloats)
     return MOEV_EINVAL;  // the problem does not fit the fixed scratch array
   float* base = nullptr;
@@ -746,26 +746,17 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
   // Nothing has to start at zero: every partial that is read is written by the first kernel of
   // the same call, and the y32 rows are cleared (not accumulated into) by the second.
   const size_t rp_smem = router_partial_smem(ks);  // 17 KB: below the default dynamic limit, no attribute needed
+  const dim3 pgrid((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile);
   if (cfg->afmt == MOEV_ACT_FP32) {
-    router_partial_kernel<MOEV_ACT_FP32><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
-    if (cfg->n_group > 0) topk_refine_kernel<MOEV_ACT_FP32, true><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
-                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
-                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
-                                                                       cfg->topk_group);
-    else topk_refine_kernel<MOEV_ACT_FP32, false><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
-                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
-                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
-                                                                       cfg->topk_group);
+    router_partial_kernel<MOEV_ACT_FP32><<<pgrid, 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
+    topk_refine_kernel<MOEV_ACT_FP32, false><<<gamma, kRefineThreads, refine_smem, st>>>(
+        T, O, x, router_w, part, part_x2, part_w2, y32, gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks, cfg->score,
+        cfg->routed_scale, nullptr, 0, 0);
   } else {
-    router_partial_kernel<MOEV_ACT_BF16><<<dim3((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile), 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
-    if (cfg->n_group > 0) topk_refine_kernel<MOEV_ACT_BF16, true><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
-                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
-                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
-                                                                       cfg->topk_group);
-    else topk_refine_kernel<MOEV_ACT_BF16, false><<<gamma, kRefineThreads, refine_smem, st>>>(T, O, x, router_w, part, part_x2, part_w2, y32,
-                                                                       gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks,
-                                                                       cfg->score, cfg->routed_scale, nullptr, cfg->n_group,
-                                                                       cfg->topk_group);
+    router_partial_kernel<MOEV_ACT_BF16><<<pgrid, 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
+    topk_refine_kernel<MOEV_ACT_BF16, false><<<gamma, kRefineThreads, refine_smem, st>>>(
+        T, O, x, router_w, part, part_x2, part_w2, y32, gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks, cfg->score,
+        cfg->routed_scale, nullptr, 0, 0);
   }
   return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
 }
@@ -777,6 +768,7 @@ moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, cons
   if (n < 1 || n > kSelMaxNodes || W < 1 || gamma < 1 || !parent || !P || !pred || !traj_workspace || !selected)
     return MOEV_EINVAL;
   if (!(eps > 0.f)) return MOEV_EINVAL;  // eps avoids the division by zero (Eq. 9)
+  if (!aligned16(traj_workspace)) return MOEV_EINVAL;  // the control words behind the footprints are read as 8- and 16-byte quantities
   constexpr size_t kBudget = 200 * 1024;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t fixed = select_fixed_smem_words(n, W) * sizeof(uint32_t);

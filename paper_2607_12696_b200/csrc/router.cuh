@@ -744,15 +744,13 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
 }
 
 // One CTA (1024 threads): per-expert histogram of the selected ids, block scan over the E
-// counts (ascending union and offsets), FFN work units, then one warp per expert walks the
-// assignments in order with ballots and writes the stable permutation.
-// Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A] | (use_bitmap) token bitmaps [E][ceil(gamma/32)].
-// Bytes beyond the bitmaps' budget: the caller passes use_bitmap = 0 and one warp orders the slots.
+// counts (ascending union and offsets), FFN work units, then the stable permutation from
+// per-expert token bitmaps.
+// Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A] | token bitmaps [E][ceil(gamma/32)]
+// (at most 64 KB of bitmaps: E <= 512, gamma <= 1024).
 inline size_t route_bitmap_bytes(int E, int gamma) { return (size_t)E * ((gamma + 31) / 32) * 4; }
-constexpr size_t kRouteBitmapBudget = 96 * 1024;
 __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O, int gamma, int E,
-                                                           int k, int n_shared, int unit_cap, int use_bitmap,
-                                                           int wide_ratio) {
+                                                           int k, int n_shared, int unit_cap, int wide_ratio) {
   extern __shared__ int32_t sm[];
   const int A = gamma * k;
   int32_t* cnt = sm;
@@ -894,7 +892,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
   // assignment (t, e) inside e's run is the number of tokens below t that selected e: a prefix
   // population count over e's token bitmap, one thread per assignment.
   __syncthreads();
-  if (use_bitmap) {
+  {
     const int TW = (gamma + 31) / 32;
     uint32_t* tb = reinterpret_cast<uint32_t*>(sm + 3 * E + 2 * A);  // [E][TW]
     for (int i = tid; i < E * TW; i += blockDim.x) tb[i] = 0u;
@@ -916,32 +914,7 @@ __global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O,
       if (O.perm) O.perm[pos] = a;
     }
     MOEV_RT_MARK(12);
-    return;
   }
-  // Fallback for very large gamma: warp 0 walks the assignments in order, 32 at a time; uidx[]
-  // is reused as the running count of slots already handed out per expert.
-  for (int e = tid; e < E; e += blockDim.x) uidx[e] = 0;
-  __syncthreads();
-  if (warp == 0) {
-    for (int a0 = 0; a0 < A; a0 += 32) {
-      const int a = a0 + lane;
-      const bool valid = a < A;
-      const int e = valid ? ids_s[a] : -1 - lane;  // distinct dummies for idle lanes
-      const uint32_t same = __match_any_sync(0xffffffffu, e);
-      if (valid) {
-        const int before = __popc(same & ((1u << lane) - 1u));
-        const int pos = excl[e] + uidx[e] + before;
-        T.perm[pos] = a;
-        T.slot_token[pos] = a / k;
-        T.slot_w[pos] = w_s[a];
-        if (O.perm) O.perm[pos] = a;
-      }
-      __syncwarp();
-      if (valid && (same & ((1u << lane) - 1u)) == 0) uidx[e] += __popc(same);  // lowest lane of each group
-      __syncwarp();
-    }
-  }
-  MOEV_RT_MARK(12);
 }
 
 }  // namespace moev

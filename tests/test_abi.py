@@ -49,3 +49,28 @@ def test_product_package_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 src = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in src, f"{f} mentions the oracle"
+
+
+def test_select_drafts_rejects_misaligned_workspace_before_any_cuda_call():
+    """Argument validation comes first, so this needs no device: the control words behind the
+    footprints are read as 8- and 16-byte quantities, hence the 16-byte rule of the header."""
+    import ctypes as C
+    L = moev.lib()
+    buf = (C.c_uint32 * 4096)()
+    base = C.addressof(buf)
+    base += (-base) % 16
+    ok_args = dict(n=4, W=1, gamma=2)
+    for off, expect in ((4, 1), (8, 1)):
+        st = L.moev_select_drafts(ok_args["n"], ok_args["W"], base + 1024, base + 2048, base + 3072, None,
+                                  ok_args["gamma"], 1e-6, 0, base + 4096 + off, base + 8192, None, None, None, None)
+        assert st == expect
+
+
+def test_static_router_rejects_group_limited_routing_before_any_cuda_call():
+    import ctypes as C
+    cfg = moev.MoevConfig(256, 128, 16, 2, score=moev.SCORE_SIGMOID, n_group=4, topk_group=2, max_tokens=8).c()
+    buf = (C.c_uint8 * 65536)()
+    base = C.addressof(buf)
+    base += (-base) % 16
+    st = moev.lib().moev_route_topk_static(C.byref(cfg), base, base + 16384, 4, base + 32768, base + 49152, None)
+    assert st == 1

@@ -121,6 +121,15 @@ def test_many_tokens_per_expert_two_phase_schedule(gamma, U, n_shared):
     assert ref.n_active == U
 
 
+@pytest.mark.parametrize("gamma,n_shared", [(5, 0), (40, 1)])
+def test_fp8_wide_intermediate_runs_fold_scale_schedule(gamma, n_shared):
+    """Block-scaled FP8 with I > 4096 (33 slices of 128): the tensor-core kernel has no per-token
+    quantised activations for such shapes and runs the schedule whose producer warps fold the
+    weight block scale into the activations of every K chunk; units of up to 32 tokens."""
+    shape = small_shape("deepseek", H=512, I=4224, E=4, top_k=2, n_shared=n_shared)
+    parity_case(shape, gamma, routing="scattered", expect_impl=moev.IMPL_TCGEN05)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 def test_topk_equals_E_and_two_shared(impl):
     shape = small_shape("deepseek", H=256, I=128, E=8, top_k=8, n_shared=2)
@@ -220,6 +229,14 @@ def test_invalid_arguments_are_rejected_before_launch():
         assert e.value.status == 1
     with pytest.raises(moev.MoevError):  # misaligned x
         v.verify(layer, x.view(-1)[1:257], 1, out)
+    if v.resolved_impl() == moev.IMPL_TCGEN05:  # expert weights at a 16-byte offset: the TMA descriptors need 32
+        off = dict(keep)
+        flat = torch.empty(keep["w_up"].numel() + 8, dtype=keep["w_up"].dtype, device="cuda")
+        off["w_up"] = flat[8:].view_as(keep["w_up"])
+        assert off["w_up"].data_ptr() % 32 == 16
+        with pytest.raises(moev.MoevError) as e:
+            v.verify(moev.binding.make_layer(off), x, 8, out)
+        assert e.value.status == 1
     bad = dict(keep)
     bad.pop("w_up")
     with pytest.raises(moev.MoevError):
