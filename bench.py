@@ -58,6 +58,11 @@ WORKLOADS = {
     "deepseek_fp8_E64_b4g64_zipf_profile": ("deepseek", 256, "zipf", {"_E": 64, "alpha": 1.0}),
     # routing kernels at the full router shape (256 experts, gamma 64) with thin experts (0.7 GB)
     "deepseek_router_profile": ("deepseek", 64, "scattered", {"_I": 128}),
+    "deepseek_router_g8_profile": ("deepseek", 8, "scattered", {"_I": 128}),
+    # tree-sized calls (the paper's operating point: a handful of tokens, 8 - 32 unique experts)
+    "deepseek_fp8_g8_u8": ("deepseek", 8, "exact", {"U": 8}),
+    "deepseek_fp8_g4_u16": ("deepseek", 4, "exact", {"U": 16}),
+    "deepseek_fp8_E64_g8_u16_profile": ("deepseek", 8, "exact", {"_E": 64, "U": 16}),
 }
 DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 
@@ -199,6 +204,43 @@ def fit_line(pts):
     b, a = np.polyfit(u, t, 1)
     r2 = 1.0 - ((t - (a + b * u)) ** 2).sum() / max(((t - t.mean()) ** 2).sum(), 1e-30)
     return {"a_us": float(a), "b_us_per_expert": float(b), "r2": float(r2)}
+
+
+def time_chain(moev, name, dev, weights, steps, warmup):
+    """Dependent layers (layer l + 1 verifies layer l's output): one moev_verify_chain call over the
+    rotated layers against the same layers as separate moev_verify calls on the same inputs."""
+    n_layers = len(weights)
+    shape, gamma, layers = build_workload(name, n_layers, dev, weights=weights)
+    cfg = moev.MoevConfig(shape.H, shape.I, shape.E, shape.top_k, shape.n_shared, gamma, shape.wfmt,
+                          shape.afmt, shape.score, moev.IMPL_AUTO, shape.routed_scale)
+    v = moev.MoeVerifier(cfg)
+    packed = pack_layers(moev, layers)
+    Ls = [p[0] for p in packed]
+    outs = [v.alloc_out(gamma, diagnostics=False) for _ in layers]
+    x0 = layers[0]["x"]
+
+    def separate():
+        for l in range(n_layers):
+            v.verify(Ls[l], x0 if l == 0 else outs[l - 1]["y"], gamma, outs[l])
+
+    res = {}
+    for label, fn in (("chain", lambda: v.verify_chain(Ls, x0, gamma, outs)), ("separate", separate)):
+        for _ in range(max(2, warmup // 2)):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        res[label] = e0.elapsed_time(e1) * 1e3 / (steps * n_layers)
+    v.status_sync()
+    U = [int(o["n_active"].item()) for o in outs]
+    v.close()
+    return {"workload": name, "gamma": gamma, "layers_per_call": n_layers, "U": U,
+            "us_per_layer_chain": res["chain"], "us_per_layer_separate_calls": res["separate"],
+            "note": "moev_verify_chain: x of layer l + 1 = y of layer l (layer 0 as the workload defines it)"}
 
 
 def run_config_entry(moev, name, dev, weights, steps, warmup, peak):
@@ -474,7 +516,7 @@ def run_ours(args):
                              f"+{shape.n_shared} experts streamed), full layer weights, {cs:.2f} s"}
         # ---- the other benchmark configurations and the unique-expert sweep, one after another
         # (default workload on one GPU only; each entry is a median over event-timed calls)
-        configs, sweep_cells, sweep_fit = None, None, None
+        configs, sweep_cells, sweep_fit, chains = None, None, None, None
         if args.workload == DEFAULT_WORKLOAD and world == 1 and not args.no_configs and ACT_QUANT == 0:
             cs_, cw = args.config_steps, 5
             ds_w = [L["weights"] for L in layers]
@@ -482,6 +524,8 @@ def run_ours(args):
                        run_config_entry(moev, "deepseek_fp8_g64_clustered", dev, ds_w, cs_, cw, peak)]
             sweep_cells, sweep_fit = run_sweep_cells(moev, dev, ds_w, [1, 4, 8, 32], [8, 16, 32, 64, 128, 256],
                                                      max(20, cs_ // 2), cw, peak)
+            chains = [time_chain(moev, "deepseek_fp8_g64_scattered", dev, ds_w, max(10, cs_ // 4), cw),
+                      time_chain(moev, "deepseek_fp8_g4_u16", dev, ds_w, max(20, cs_ // 2), cw)]
             del ds_w, packed
             layers.clear()
             torch.cuda.empty_cache()
@@ -535,6 +579,7 @@ def run_ours(args):
             line["configs"] = configs
             line["sweep"] = sweep_cells
             line["sweep_fit"] = sweep_fit
+            line["chain"] = chains
         print(json.dumps(line))
     v.close()
     if dist:

@@ -139,6 +139,13 @@ typedef struct {
   const void *sh_s_gate, *sh_s_up, *sh_s_down;
   const float *b_gate, *b_up, *b_down; /* MOEV_FFN_GPTOSS: fp32 biases [E,I], [E,I], [E,H]; NULL = zero */
   const float* router_bias;            /* n_group > 0: fp32 score-correction bias [E]; NULL = zero */
+  /* Optional prefetch hint (Sec. 4.1, Eq. 4: the predictor's expert set for this layer): DEVICE list of
+   * n_predicted expert ids whose weights the first routing kernel pulls into the L2 while the router
+   * runs, next to the shared experts' (only when moev_prefetch_enable switched the prefetch on).  A wrong prediction costs only
+   * bandwidth; results never depend on the hint.  At most what fits an 80 MB share of the L2 is taken
+   * (the first entries of the list).  NULL / 0 = no hint. */
+  const int32_t* predicted_ids;
+  int32_t n_predicted;
 } moev_layer;
 
 /* Outputs.  y and n_active are required; the others are diagnostics and may be NULL.
@@ -197,8 +204,10 @@ size_t moev_expert_bytes(const moev_config* cfg);
 /* Code bytes only (the paper's 44.04 MB figure). */
 size_t moev_expert_code_bytes(const moev_config* cfg);
 
-/* Number of kernels one moev_verify call launches on this context (for launch accounting),
- * and which FFN implementation it resolved to (a moev_impl value, never AUTO). */
+/* Number of kernels one moev_verify call launches on this context (for launch accounting; calls
+ * of at most 128 tokens with plain top-k routing take two routing launches, others three -- a
+ * context whose max_tokens exceeds 128 reports the larger figure), and which FFN implementation
+ * it resolved to (a moev_impl value, never AUTO). */
 int32_t moev_launches_per_call(const moev_ctx* ctx);
 int32_t moev_resolved_impl(const moev_ctx* ctx);
 
@@ -213,6 +222,14 @@ moev_status moev_profile_enable(moev_ctx* ctx, int32_t on);
 moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[6]*/,
                               int32_t* calls);
 
+/* Weight prefetch by the first routing kernel (off by default): the shared experts' matrices and
+ * those of the layer's predicted_ids are pulled into the L2 while the routing kernels run, so the
+ * expert kernel finds them on chip (Sec. 3: the verification cost is expert-weight traffic from
+ * HBM; what is known to be needed before the router decides need not wait for it).  Measured on
+ * B200 it does not pay: the L2 delivers these bytes only slightly faster than HBM does, and the
+ * prefetch traffic delays the latency-bound routing kernels by more than the expert kernel gains. */
+moev_status moev_prefetch_enable(moev_ctx* ctx, int32_t on);
+
 /* Several independent layers in one call (multi-layer pipelining; the paper has no counterpart:
  * its prototype runs layer by layer).  Equivalent to n_layers calls of moev_verify on the same
  * stream with layers[l], x[l], outs[l] and the same gamma, except that the first kernel of layer
@@ -226,6 +243,18 @@ moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us 
 moev_status moev_verify_pipeline(moev_ctx* ctx, int32_t n_layers, const moev_layer* layers,
                                  const void* const* x, int32_t gamma, const moev_out* outs,
                                  void* cuda_stream);
+
+/* Consecutive dependent layers in one call: layer l + 1 verifies the output of layer l (Sec. 5 /
+ * Table 13: a verification pass runs the model's 36 - 94 MoE layers one after another; the
+ * attention between them is outside this library and is the identity here).  x0 [gamma, H] is the
+ * input of layers[0]; outs[l].y [gamma, H] (afmt, required for every layer) is both the result of
+ * layer l and the input of layer l + 1.  Same results as n_layers calls of moev_verify with those
+ * inputs; every kernel of the call is a programmatic dependent launch of its predecessor, the
+ * first kernel of a layer included: it is scheduled while the previous layer drains, starts the
+ * optional weight prefetch at once, and waits for the previous layer's output before it reads it.
+ * layers / outs are HOST arrays whose pointers are DEVICE pointers.  Errors as moev_verify. */
+moev_status moev_verify_chain(moev_ctx* ctx, int32_t n_layers, const moev_layer* layers, const void* x0,
+                              int32_t gamma, const moev_out* outs, void* cuda_stream);
 
 /* Cost-aware draft selection: Algorithm 1 of the paper (Sec. 4.2, Eqs. 7-10), the step that
  * runs between drafting and verification and decides which gamma draft-tree nodes are verified.

@@ -21,7 +21,7 @@ EXPORTS = ("moev_create", "moev_destroy", "moev_verify", "moev_verify_host", "mo
            "moev_last_error", "moev_expert_bytes", "moev_expert_code_bytes",
            "moev_launches_per_call", "moev_resolved_impl", "moev_profile_enable",
            "moev_profile_read", "moev_route_topk_static", "moev_route_topk_static_scratch_floats", "moev_select_drafts",
-           "moev_verify_pipeline")
+           "moev_verify_pipeline", "moev_prefetch_enable", "moev_verify_chain")
 
 
 class MoevError(RuntimeError):
@@ -48,7 +48,7 @@ _OUT_FIELDS = ("y", "topk_ids", "topk_w", "union_ids", "offsets", "perm", "n_act
 
 
 class _Layer(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in _LAYER_FIELDS]
+    _fields_ = [(n, C.c_void_p) for n in _LAYER_FIELDS] + [("predicted_ids", C.c_void_p), ("n_predicted", C.c_int32)]
 
 
 class _Out(C.Structure):
@@ -104,6 +104,9 @@ def lib() -> C.CDLL:
         L.moev_verify_pipeline.restype = C.c_int
         L.moev_verify_pipeline.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_Layer), C.POINTER(C.c_void_p), C.c_int32,
                                            C.POINTER(_Out), C.c_void_p]
+        L.moev_verify_chain.restype = C.c_int
+        L.moev_verify_chain.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_Layer), C.c_void_p, C.c_int32,
+                                        C.POINTER(_Out), C.c_void_p]
         L.moev_verify_host.restype = C.c_int
         L.moev_verify_host.argtypes = [C.c_void_p, C.POINTER(_Layer), C.c_void_p, C.c_int32,
                                        C.c_void_p, C.c_void_p, C.c_void_p]
@@ -121,6 +124,8 @@ def lib() -> C.CDLL:
         L.moev_resolved_impl.argtypes = [C.c_void_p]
         L.moev_profile_enable.restype = C.c_int
         L.moev_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.moev_prefetch_enable.restype = C.c_int
+        L.moev_prefetch_enable.argtypes = [C.c_void_p, C.c_int32]
         L.moev_profile_read.restype = C.c_int
         L.moev_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_double),
                                         C.POINTER(C.c_int32)]
@@ -200,6 +205,10 @@ def make_layer(tensors: dict) -> _Layer:
         if t is not None:
             assert t.is_cuda and t.is_contiguous(), f"{n} must be a contiguous CUDA tensor"
         setattr(L, n, _ptr(t))
+    pred = tensors.get("predicted_ids")
+    if pred is not None:
+        assert pred.is_cuda and pred.dtype == torch.int32 and pred.is_contiguous()
+        L.predicted_ids, L.n_predicted = pred.data_ptr(), pred.numel()
     return L
 
 
@@ -268,6 +277,17 @@ class MoeVerifier:
                 setattr(OA[i], f, _ptr(out.get(f)))
         self._check(lib().moev_verify_pipeline(self._h, n, LA, XA, gamma, OA, self._stream()))
 
+    def verify_chain(self, layers: list, x0: torch.Tensor, gamma: int, outs: list):
+        """moev_verify_chain: dependent layers, outs[l]["y"] is the input of layer l + 1."""
+        n = len(layers)
+        assert len(outs) == n
+        LA = (_Layer * n)(*layers)
+        OA = (_Out * n)()
+        for i, out in enumerate(outs):
+            for f in _OUT_FIELDS:
+                setattr(OA[i], f, _ptr(out.get(f)))
+        self._check(lib().moev_verify_chain(self._h, n, LA, _ptr(x0), gamma, OA, self._stream()))
+
     def verify_host(self, layer: _Layer, x_host: torch.Tensor, gamma: int, y_host: torch.Tensor,
                     n_active_host: torch.Tensor):
         """moev_verify_host: host x in, host y / n_active out (synchronous)."""
@@ -284,6 +304,10 @@ class MoeVerifier:
 
     def resolved_impl(self) -> int:
         return lib().moev_resolved_impl(self._h)
+
+    def prefetch_enable(self, on: bool):
+        """moev_prefetch_enable: L2 prefetch of shared / predicted experts' weights during routing."""
+        self._check(lib().moev_prefetch_enable(self._h, int(on)))
 
     def profile_enable(self, on: bool):
         self._check(lib().moev_profile_enable(self._h, int(on)))

@@ -12,12 +12,15 @@
 #include "ffn_tc_wide.cuh"
 #include "ffn_tc_p.cuh"
 #include "router.cuh"
+#include "route_fused.cuh"
 #include "select.cuh"
 
 using namespace moev;
 
 namespace {
 constexpr int kProfSlots = 512;
+// expert-weight bytes the first routing kernel may pull into the L2 ahead of the expert kernel (B200: 126 MB of L2)
+constexpr size_t kPrefetchBudgetBytes = 80u * 1024u * 1024u;
 constexpr int kTmapCache = 8;
 
 // The six TMA descriptors of one layer (gate, up, down, shared gate, up, down) and the
@@ -42,6 +45,8 @@ struct moev_ctx {
   int n_slices = 0;
   int ks = 32;  // columns per split-K slice of the router
   bool router_mma = false;
+  FusedScratch fused{};     // two-launch routing of tree-sized calls (route_fused.cuh)
+  size_t fused_smem_max = 0;
 #ifdef MOEV_TC_STATS
   unsigned long long* tc_stats = nullptr;  // [n_sm][16], debug builds only
 #endif
@@ -62,7 +67,10 @@ struct moev_ctx {
   int n_sm = 0;
   int unit_cap = 1 << 20;
   bool profile = false;
-  bool chain = false;  // next moev_verify is a later layer of a pipelined call: its first kernel is a dependent launch
+  bool prefetch = false;  // L2 prefetch of shared / predicted experts' weights by the first routing kernel
+  int chain = 0;  // next moev_verify is a later layer of a multi-layer call: its first kernel is a dependent launch
+                  // (1: independent inputs, the kernel waits for the previous layer at its end; 2: its input is the
+                  // previous layer's output, it waits before reading it)
   cudaEvent_t ev[kProfSlots][7];  // before/after each kernel of a call
   int prof_n = 0;
   bool prof_events_ready = false;
@@ -383,6 +391,19 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && dmalloc(&c->part, (size_t)c->n_slices * G * E) == cudaSuccess;
   ok = ok && dmalloc(&c->part_x2, (size_t)c->n_slices * G) == cudaSuccess;
   ok = ok && dmalloc(&c->part_w2, (size_t)c->n_slices * ((E + kRouterETile - 1) / kRouterETile)) == cudaSuccess;
+  if (cfg->n_group == 0) {
+    // two-launch routing: partial fp64 logits per (token, slice), arrival counters (zero between calls)
+    size_t rows = 0;
+    const int gmax = cfg->max_tokens < kFusedMaxTokens ? cfg->max_tokens : kFusedMaxTokens;
+    for (int g = 1; g <= gmax; ++g) {
+      rows = std::max(rows, (size_t)g * fused_slices(g, cfg->H, prop.multiProcessorCount));
+      c->fused_smem_max = std::max(c->fused_smem_max, route_group_block_smem(cfg->E, g, cfg->top_k));
+    }
+    ok = ok && dmalloc(&c->fused.dpart, rows * E) == cudaSuccess;
+    ok = ok && dmalloc(&c->fused.tok_cnt, (size_t)gmax + 1) == cudaSuccess;
+    ok = ok && cudaMemset(c->fused.tok_cnt, 0, ((size_t)gmax + 1) * sizeof(int32_t)) == cudaSuccess;
+    if (ok) c->fused.done_cnt = c->fused.tok_cnt + gmax;
+  }
   ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.union_ids, E) == cudaSuccess;
@@ -492,6 +513,12 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     if (gs > 48 * 1024)
       ok = ok && cudaFuncSetAttribute(route_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)gs) == cudaSuccess;
+    if (c->fused_smem_max > 20 * 1024) {  // beside about 24 KB of static tables
+      ok = ok && cudaFuncSetAttribute(route_refine_kernel<MOEV_ACT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)c->fused_smem_max) == cudaSuccess;
+      ok = ok && cudaFuncSetAttribute(route_refine_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)c->fused_smem_max) == cudaSuccess;
+    }
     if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
       ok = ok && cudaFuncSetAttribute(tc::grouped_ffn_tc_kernel<MOEV_W_BF16>,
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes) == cudaSuccess;
@@ -513,6 +540,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
 
 moev_status moev_destroy(moev_ctx* c) {
   if (!c) return MOEV_EINVAL;
+  cudaFree(c->fused.dpart); cudaFree(c->fused.tok_cnt);
   cudaFree(c->part); cudaFree(c->part_x2); cudaFree(c->part_w2); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
@@ -530,7 +558,10 @@ moev_status moev_destroy(moev_ctx* c) {
 
 const char* moev_last_error(const moev_ctx* c) { return c ? c->err : "null context"; }
 int32_t moev_launches_per_call(const moev_ctx* c) {
-  return c ? (c->resolved_impl == MOEV_IMPL_TCGEN05 ? 5 : (c->cfg.act_quant != MOEV_ACTQ_NONE ? 8 : 6)) : 0;
+  if (!c) return 0;
+  const int ffn = c->resolved_impl == MOEV_IMPL_TCGEN05 ? 1 : (c->cfg.act_quant != MOEV_ACTQ_NONE ? 4 : 2);
+  const bool fused = c->cfg.n_group == 0 && c->cfg.max_tokens <= kFusedMaxTokens;  // every gamma of this context
+  return (fused ? 2 : 3) + ffn + 1;
 }
 int32_t moev_resolved_impl(const moev_ctx* c) { return c ? c->resolved_impl : 0; }
 
@@ -581,33 +612,70 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   const size_t refine_smem = refine_smem_bytes(g.E);
   const bool pdl = ev == nullptr;  // event records between the kernels would serialise them anyway
   const size_t rp_smem = router_partial_smem(c->ks);
-  if (g.afmt == MOEV_ACT_FP32)
-    launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain, x, layer->router_w,
-             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
-  else
-    launch_k(router_partial_mma_kernel, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256),
-             router_partial_mma_smem(c->ks), st, pdl && c->chain, static_cast<const uint16_t*>(x), layer->router_w,
-             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks);
-  if (ev) cudaEventRecord(ev[1], st);
+  // weights known to be needed before the router has decided: shared experts (and the caller's predicted
+  // experts) go to the L2 while the routing kernels leave the HBM idle
+  PrefetchArgs pf{};
   {
+    const size_t mat_bytes = code_bytes(&g) / 3;
+    const size_t budget = kPrefetchBudgetBytes / (3 * mat_bytes);  // experts that fit the L2 share set aside for this
+    pf.bytes = mat_bytes;
+    pf.sh[0] = static_cast<const uint8_t*>(layer->sh_gate); pf.sh[1] = static_cast<const uint8_t*>(layer->sh_up);
+    pf.sh[2] = static_cast<const uint8_t*>(layer->sh_down);
+    pf.w[0] = static_cast<const uint8_t*>(layer->w_gate); pf.w[1] = static_cast<const uint8_t*>(layer->w_up);
+    pf.w[2] = static_cast<const uint8_t*>(layer->w_down);
+    pf.n_shared = c->prefetch ? (int)std::min<size_t>(g.n_shared, budget) : 0;
+    pf.pred_ids = layer->predicted_ids;
+    pf.n_pred = (c->prefetch && layer->predicted_ids && layer->n_predicted > 0)
+                    ? (int)std::min<size_t>(layer->n_predicted, budget - pf.n_shared) : 0;
+    if (mat_bytes % 16) { pf.n_shared = 0; pf.n_pred = 0; }
+  }
+  if (g.afmt == MOEV_ACT_FP32)
+    launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain != 0, x, layer->router_w,
+             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+  else if (gamma <= 32) {
+    // tree-sized calls: the variant without shared memory (one trip to memory long)
+    auto go = [&](auto kern) {
+      launch_k(kern, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(128), 0, st, pdl && c->chain != 0,
+               static_cast<const uint16_t*>(x), layer->router_w, c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+    };
+    if (gamma <= 8) go(router_partial_small_kernel<1>);
+    else if (gamma <= 16) go(router_partial_small_kernel<2>);
+    else go(router_partial_small_kernel<4>);
+  } else
+    launch_k(router_partial_mma_kernel, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256),
+             router_partial_mma_smem(c->ks), st, pdl && c->chain != 0, static_cast<const uint16_t*>(x), layer->router_w,
+             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+  if (ev) cudaEventRecord(ev[1], st);
+  const int refine_depth = g.afmt == MOEV_ACT_FP32 ? c->ks : 6 * c->ks + c->n_slices + 12;
+  const int wide_ratio = (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0;
+  if (g.n_group == 0 && gamma <= kFusedMaxTokens) {
+    // tree-sized calls: refinement spread over several CTAs per token, grouping by the last one to finish
+    const int S = fused_slices(gamma, g.H, c->n_sm);
+    const size_t gsm = route_group_block_smem(g.E, gamma, g.top_k);
+    auto go = [&](auto kern) {
+      launch_k(kern, dim3(S, gamma), dim3(kFusedThreads), gsm, st, pdl, c->T, O, c->fused, x, layer->router_w,
+               (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
+               g.top_k, c->n_slices, refine_depth, g.score, g.routed_scale, g.n_shared, c->unit_cap, wide_ratio);
+    };
+    if (g.afmt == MOEV_ACT_FP32) go(route_refine_kernel<MOEV_ACT_FP32>); else go(route_refine_kernel<MOEV_ACT_BF16>);
+    if (ev) cudaEventRecord(ev[2], st);
+  } else {
     // the kernel's code is executed once per CTA, front to back: the plain and the group-limited
     // routing are separate instantiations so that neither carries the other's instructions
-    const int refine_depth = c->router_mma ? 6 * c->ks + c->n_slices + 12 : c->ks;
     auto go = [&](auto kern) {
       launch_k(kern, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x, layer->router_w,
                (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
-               g.top_k, c->n_slices, g.afmt == MOEV_ACT_FP32 ? c->ks : refine_depth, g.score, g.routed_scale,
-               layer->router_bias, g.n_group, g.topk_group);
+               g.top_k, c->n_slices, refine_depth, g.score, g.routed_scale, layer->router_bias, g.n_group, g.topk_group);
     };
     if (g.afmt == MOEV_ACT_FP32) {
       if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_FP32, true>); else go(topk_refine_kernel<MOEV_ACT_FP32, false>);
     } else {
       if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_BF16, true>); else go(topk_refine_kernel<MOEV_ACT_BF16, false>);
     }
+    if (ev) cudaEventRecord(ev[2], st);
+    launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
+             g.n_shared, c->unit_cap, wide_ratio);
   }
-  if (ev) cudaEventRecord(ev[2], st);
-  launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
-           g.n_shared, c->unit_cap, (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0);
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
     if (g.wfmt == MOEV_W_BF16) launch_tc_ffn<MOEV_W_BF16>(c, tm, layer, x, gamma, st, ev);
@@ -632,10 +700,25 @@ moev_status moev_verify_pipeline(moev_ctx* c, int32_t n_layers, const moev_layer
   if (n_layers < 1 || !layers || !x || !outs) return fail(c, MOEV_EINVAL, "null argument or n_layers < 1");
   moev_status s = MOEV_OK;
   for (int32_t l = 0; l < n_layers && s == MOEV_OK; ++l) {
-    c->chain = l > 0;
+    c->chain = l > 0 ? 1 : 0;
     s = moev_verify(c, &layers[l], x[l], gamma, &outs[l], cuda_stream);
   }
-  c->chain = false;
+  c->chain = 0;
+  return s;
+}
+
+moev_status moev_verify_chain(moev_ctx* c, int32_t n_layers, const moev_layer* layers, const void* x0, int32_t gamma,
+                              const moev_out* outs, void* cuda_stream) {
+  if (!c) return MOEV_EINVAL;
+  if (n_layers < 1 || !layers || !x0 || !outs) return fail(c, MOEV_EINVAL, "null argument or n_layers < 1");
+  for (int32_t l = 0; l + 1 < n_layers; ++l)
+    if (!outs[l].y) return fail(c, MOEV_EINVAL, "outs[%d].y is the input of layer %d and must not be null", l, l + 1);
+  moev_status s = MOEV_OK;
+  for (int32_t l = 0; l < n_layers && s == MOEV_OK; ++l) {
+    c->chain = l > 0 ? 2 : 0;
+    s = moev_verify(c, &layers[l], l == 0 ? x0 : outs[l - 1].y, gamma, &outs[l], cuda_stream);
+  }
+  c->chain = 0;
   return s;
 }
 
@@ -748,12 +831,12 @@ moev_status moev_route_topk_static(const moev_config* cfg, const float* router_w
   const size_t rp_smem = router_partial_smem(ks);  // 17 KB: below the default dynamic limit, no attribute needed
   const dim3 pgrid((unsigned)ns, (cfg->E + kRouterETile - 1) / kRouterETile);
   if (cfg->afmt == MOEV_ACT_FP32) {
-    router_partial_kernel<MOEV_ACT_FP32><<<pgrid, 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
+    router_partial_kernel<MOEV_ACT_FP32><<<pgrid, 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks, 0, PrefetchArgs{});
     topk_refine_kernel<MOEV_ACT_FP32, false><<<gamma, kRefineThreads, refine_smem, st>>>(
         T, O, x, router_w, part, part_x2, part_w2, y32, gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks, cfg->score,
         cfg->routed_scale, nullptr, 0, 0);
   } else {
-    router_partial_kernel<MOEV_ACT_BF16><<<pgrid, 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks);
+    router_partial_kernel<MOEV_ACT_BF16><<<pgrid, 256, rp_smem, st>>>(x, router_w, part, part_x2, part_w2, gamma, cfg->H, cfg->E, ks, 0, PrefetchArgs{});
     topk_refine_kernel<MOEV_ACT_BF16, false><<<gamma, kRefineThreads, refine_smem, st>>>(
         T, O, x, router_w, part, part_x2, part_w2, y32, gamma, cfg->H, cfg->E, cfg->top_k, (int)ns, ks, cfg->score,
         cfg->routed_scale, nullptr, 0, 0);
@@ -829,6 +912,12 @@ int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*16
   return c->n_sm;
 }
 #endif
+
+moev_status moev_prefetch_enable(moev_ctx* c, int32_t on) {
+  if (!c) return MOEV_EINVAL;
+  c->prefetch = on != 0;
+  return MOEV_OK;
+}
 
 moev_status moev_profile_enable(moev_ctx* c, int32_t on) {
   if (!c) return MOEV_EINVAL;

@@ -1,0 +1,665 @@
+// Routing for tree-sized calls in two launches instead of three, with the per-token work spread
+// over several CTAs.
+//
+//   route_refine_kernel   grid (S, gamma): CTA (s, t) sums the split-K partial logits of token t,
+//                         takes the candidates of the top-k under the rounding-error bound (every
+//                         CTA of a token derives the same list from the same numbers), evaluates
+//                         their exact fp64 logits over its slice s of the hidden dimension and
+//                         publishes the partial sums, and writes its slice of the token's
+//                         quantised activations.  The CTA of a token that arrives last adds the
+//                         S partial sums in a fixed order, ranks the candidates exactly (larger
+//                         logit first, ties to the lower id) and forms the router weights.  The CTA that finishes the last token
+//                         builds the expert union, offsets, permutation and FFN work units
+//                         (route_group_block).  Nothing in the kernel waits: the hand-overs are
+//                         "last arrival continues" counters (release by fence + atomic add,
+//                         acquire by the atomic's result + fence), so there is no spin and no
+//                         co-residency requirement.
+//
+// The results are those of topk_refine_kernel + route_group_kernel: the same candidates, the
+// same fp64 ranking rule, the same tables.  Group-limited routing (two dependent candidate
+// stages) and calls of more than kFusedMaxTokens rows keep the three-kernel path.
+#pragma once
+#include "common.cuh"
+#include "router.cuh"
+
+namespace moev {
+
+#ifdef MOEV_TC_STATS
+#define MOEV_RF_MARK(i, cond) do { if ((cond) && threadIdx.x == 0) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); g_rt_stats[i] = (long long)_t; } } while (0)
+#else
+#define MOEV_RF_MARK(i, cond)
+#endif
+
+constexpr int kFusedThreads = 512;
+constexpr int kFusedWarps = kFusedThreads / 32;
+constexpr int kFusedMaxTokens = 128;   // rows per call served by this path
+constexpr int kFusedMaxSlices = 16;    // CTAs per token
+constexpr int kFusedCand = 12;         // candidates evaluated per pass over the slice
+
+// CTAs per token: one CTA per SM in total (one wave), at most kFusedMaxSlices, slices of at least 256 columns.
+inline int fused_slices(int gamma, int H, int n_sm) {
+  int s = n_sm / gamma;
+  s = s > kFusedMaxSlices ? kFusedMaxSlices : s;
+  const int by_cols = H / 256 < 1 ? 1 : H / 256;
+  s = s > by_cols ? by_cols : s;
+  return s < 1 ? 1 : s;
+}
+
+struct FusedScratch {
+  double* dpart;      // [gamma][S][E] partial fp64 logits of the candidates (candidate order)
+  int32_t* tok_cnt;   // [max_tokens] arrivals per token; zero between calls
+  int32_t* done_cnt;  // [1] finished tokens; zero between calls
+};
+
+// ---------------------------------------------------------------------------------------
+// Exclusive scan of NV integer sequences over the block.  Every thread holds ITEMS consecutive
+// entries of each (blocked layout: thread i owns entries i * ITEMS ..); on return v holds the
+// exclusive prefixes and tot the totals.  ws: NV * 33 ints of shared memory.  Two barriers.
+template <int ITEMS, int NV>
+__device__ __forceinline__ void block_scan(int (&v)[NV][ITEMS], int (&tot)[NV], int32_t* ws) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+  int own[NV], inc[NV];
+#pragma unroll
+  for (int q = 0; q < NV; ++q) {
+    int sa = 0;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) { const int x = v[q][i]; v[q][i] = sa; sa += x; }
+    own[q] = sa; inc[q] = sa;
+  }
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+    for (int q = 0; q < NV; ++q) {
+      const int x = __shfl_up_sync(0xffffffffu, inc[q], o);
+      if (lane >= o) inc[q] += x;
+    }
+  }
+  __syncthreads();  // ws free (previous use over)
+  if (lane == 31) {
+#pragma unroll
+    for (int q = 0; q < NV; ++q) ws[q * 33 + warp] = inc[q];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int q = 0; q < NV; ++q) {
+    int before = 0, total = 0;
+    for (int w = 0; w < nw; ++w) {
+      const int x = ws[q * 33 + w];
+      before += w < warp ? x : 0;
+      total += x;
+    }
+    tot[q] = total;
+    before += inc[q] - own[q];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) v[q][i] += before;
+  }
+}
+
+// Shared memory of route_group_block, in 32-bit words: cnt[E] | excl[E] | ids[A] | w[A] |
+// token bitmaps [E][ceil(gamma / 32)].
+inline size_t route_group_block_smem(int E, int gamma, int k) {
+  return (size_t)(2 * E + 2 * gamma * k) * 4 + route_bitmap_bytes(E, gamma);
+}
+
+// Expert union (ascending, Eq. 1), per-expert token counts and offsets, FFN work units, stable
+// token->expert permutation: the work of route_group_kernel for any block size with
+// blockDim.x * kGroupItems >= E, in four block-wide steps (one scan carries the slot offsets, the
+// union index and both variants of the unit counts).
+constexpr int kGroupItems = 1;
+__device__ __forceinline__ void route_group_block(const Tables& T, const RouteOut& O, int gamma, int E, int k, int n_shared,
+                                                  int unit_cap, int wide_ratio, int32_t* sm) {
+  const int A = gamma * k;
+  int32_t* cnt = sm;
+  int32_t* excl = sm + E;
+  int32_t* ids_s = sm + 2 * E;
+  float* w_s = reinterpret_cast<float*>(sm + 2 * E + A);
+  uint32_t* tb = reinterpret_cast<uint32_t*>(sm + 2 * E + 2 * A);  // [E][TW]
+  __shared__ int32_t scan_ws[5 * 33];
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int TW = (gamma + 31) / 32;
+
+  for (int e = tid; e < E; e += nt) cnt[e] = 0;
+  for (int i = tid; i < E * TW; i += nt) tb[i] = 0u;
+  __syncthreads();
+  for (int a = tid; a < A; a += nt) {
+    const int e = __ldcg(T.topk_ids + a);
+    ids_s[a] = e;
+    w_s[a] = __ldcg(T.topk_w + a);
+    atomicAdd(&cnt[e], 1);
+    const int t = a / k;
+    atomicOr(&tb[e * TW + (t >> 5)], 1u << (t & 31));
+  }
+  __syncthreads();
+  MOEV_RF_MARK(17, true);
+
+  // ---- one scan over the experts: slots before e | active experts before e | units before e and packed counts
+  // of remainder units per class, if remainders are placed behind the full runs | units before e otherwise
+  int v[5][kGroupItems], tot[5], m[kGroupItems];
+#pragma unroll
+  for (int i = 0; i < kGroupItems; ++i) {
+    const int e = tid * kGroupItems + i;
+    m[i] = e < E ? cnt[e] : 0;
+    const int rem = m[i] % unit_cap;
+    const int cls = rem >= 12 ? 0 : (rem >= 6 ? 1 : 2);
+    v[0][i] = m[i];
+    v[1][i] = m[i] > 0 ? 1 : 0;
+    v[2][i] = m[i] / unit_cap;
+    v[3][i] = rem > 0 ? (1 << (10 * cls)) : 0;   // three 10-bit counters (at most 512 experts)
+    v[4][i] = (m[i] + unit_cap - 1) / unit_cap;
+  }
+  block_scan<kGroupItems, 5>(v, tot, scan_ws);
+  MOEV_RF_MARK(18, true);
+  const int U = tot[1];
+  // many tokens per streamed expert: the two-phase FFN schedule (see route_group_kernel)
+  const int ut = U + n_shared;
+  const bool wide = T.wide != nullptr && wide_ratio > 0 &&
+                    (A + n_shared * gamma) > (ut < 100 ? wide_ratio : wide_ratio + wide_ratio / 2) * ut;
+  // Units: every expert's slots cut into runs of at most unit_cap.  Order: the shared experts' units, the full
+  // runs of the routed experts in expert order, then (single-phase tensor-core schedules) the routed experts'
+  // remainders in three classes of decreasing length (>= 12, >= 6, shorter), expert order inside each.
+  const bool sorted = unit_cap <= 64 && !wide;
+  const int sh_each = (gamma + unit_cap - 1) / unit_cap, base = n_shared * sh_each;
+  const int total1 = sorted ? tot[2] : tot[4];
+  const int n0 = sorted ? (tot[3] & 1023) : 0, n1 = sorted ? ((tot[3] >> 10) & 1023) : 0,
+            n2 = sorted ? ((tot[3] >> 20) & 1023) : 0;
+  const int n_units = base + total1 + n0 + n1 + n2;
+  for (int i = tid; i < base; i += nt) {
+    const int sx = i / sh_each, c = i - sx * sh_each;
+    Unit un;
+    un.expert = sx; un.slot0 = A + sx * gamma + c * unit_cap;
+    un.m = min(unit_cap, gamma - c * unit_cap); un.shared = 1;
+    T.units[i] = un;
+  }
+#pragma unroll
+  for (int i = 0; i < kGroupItems; ++i) {
+    const int e = tid * kGroupItems + i;
+    if (e >= E) continue;
+    excl[e] = v[0][i];
+    if (m[i] == 0) continue;
+    const int u = v[1][i], slot0 = v[0][i];
+    T.union_ids[u] = e;
+    T.offsets[u] = slot0;
+    if (O.union_ids) O.union_ids[u] = e;
+    if (O.offsets) O.offsets[u] = slot0;
+    const int rem = sorted ? m[i] % unit_cap : 0;
+    const int nch = sorted ? m[i] / unit_cap : (m[i] + unit_cap - 1) / unit_cap;
+    const int first = base + (sorted ? v[2][i] : v[4][i]);
+    for (int c = 0; c < nch; ++c) {
+      Unit un;
+      un.expert = e; un.slot0 = slot0 + c * unit_cap;
+      un.m = min(unit_cap, m[i] - c * unit_cap); un.shared = 0;
+      T.units[first + c] = un;
+    }
+    if (rem > 0) {
+      const int cls = rem >= 12 ? 0 : (rem >= 6 ? 1 : 2);
+      const int before = (v[3][i] >> (10 * cls)) & 1023;  // earlier experts of the same class
+      Unit un;
+      un.expert = e; un.slot0 = slot0 + (m[i] - rem); un.m = rem; un.shared = 0;
+      T.units[base + total1 + (cls > 0 ? n0 : 0) + (cls > 1 ? n1 : 0) + before] = un;
+    }
+  }
+  if (tid == 0) {
+    T.offsets[U] = A;
+    if (O.offsets) O.offsets[U] = A;
+    *T.n_active = U;
+    if (O.n_active) *O.n_active = U;
+    *T.n_units = n_units;
+    *T.task_counter = 0;
+    if (T.wide) *T.wide = wide ? 1 : 0;
+  }
+  if (T.unit_done)
+    for (int i = tid; i < 2 * n_units; i += nt) T.unit_done[i] = 0;  // progress counters and the gather flags behind them
+  __syncthreads();  // excl complete
+  MOEV_RF_MARK(19, true);
+  // ---- stable permutation.  A token selects an expert at most once, so the slot of assignment (t, e) inside e's
+  // run is the number of tokens below t that selected e: a prefix population count over e's token bitmap.
+  for (int a = tid; a < A; a += nt) {
+    const int t = a / k, e = ids_s[a];
+    const uint32_t* row = tb + e * TW;
+    int rank = __popc(row[t >> 5] & ((1u << (t & 31)) - 1u));
+    for (int w = 0; w < (t >> 5); ++w) rank += __popc(row[w]);
+    const int pos = excl[e] + rank;
+    T.perm[pos] = a;
+    T.slot_token[pos] = t;
+    T.slot_w[pos] = w_s[a];
+    if (O.perm) O.perm[pos] = a;
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Sums of 16 per-lane doubles over the warp by a butterfly that halves the number of entries a lane
+// holds at every step (16 additions per lane instead of 5 per entry): on return lane l holds the
+// warp-wide sum of entry q, both lanes of a pair (l, l ^ 1) the same one.  The order of the additions
+// is fixed.  fp64 additions are the scarce resource here (the fp64 pipe is narrow).
+__device__ __forceinline__ double warp_reduce_scatter16(double (&a)[16], int lane, int& q) {
+#pragma unroll
+  for (int n = 8, o = 16; n >= 1; n >>= 1, o >>= 1) {
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < n; ++i) {
+      const double send = up ? a[i] : a[i + n];
+      const double keep = up ? a[i + n] : a[i];
+      a[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+    }
+  }
+  a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
+  q = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+  return a[0];
+}
+
+template <int AFMT>
+__global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
+    Tables T, RouteOut O, FusedScratch F, const void* __restrict__ x, const float* __restrict__ router_w,
+    const float* __restrict__ part, const float* __restrict__ part_x2, const float* __restrict__ part_w2max,
+    float* __restrict__ y32, int gamma, int H, int E, int k, int n_slices, int ks, int score, float routed_scale,
+    int n_shared, int unit_cap, int wide_ratio) {
+  extern __shared__ __align__(16) int32_t dyn_sm[];  // route_group_block's tables (the last CTA only)
+  __shared__ double L[kMaxE];                        // exact logits of the candidates
+  __shared__ float l32[kMaxE];
+  __shared__ int32_t cand[kMaxE];
+  __shared__ __align__(16) float psum[kFusedThreads * 4];
+  __shared__ double red[kFusedWarps][16];
+  __shared__ float redf[kFusedWarps], redw[kFusedWarps], reda[kFusedWarps];
+  __shared__ int wcnt_s[kFusedWarps];
+  __shared__ float kth_s;
+  __shared__ float top_v[kFusedWarps * kMaxTopK];
+  __shared__ int top_id[kFusedWarps * kMaxTopK];
+  __shared__ int flag_s;
+  __shared__ float sel_v_s[kMaxTopK];
+  __shared__ int sel_e_s[kMaxTopK];
+  const int s = blockIdx.x, S = gridDim.x, t = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // columns of this CTA's slice, in groups of four; slices are whole blocks of 128 columns (the 1 x 128
+  // activation quantisation works on such blocks), so the last slices of a token may be empty
+  const int g4_all = H / 4;
+  const int g4_per = (((g4_all + S - 1) / S) + 31) & ~31;
+  const int g4_lo = min(g4_all, s * g4_per), g4_hi = min(g4_all, g4_lo + g4_per);
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");               // router partials are complete
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  const bool first_cta = s == 0 && t == 0;
+  MOEV_RF_MARK(0, first_cta);
+  // zero this slice of the token's row of the fp32 combine accumulator
+  for (int i = g4_lo + tid; i < g4_hi; i += kFusedThreads)
+    reinterpret_cast<float4*>(y32 + (size_t)t * H)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  // ---- Loads of the first phase, all issued before any is used (one trip to the L2 instead of one per
+  // group of loads): the token's row (for max |x|: every CTA of the token needs the quantisation scale),
+  // the norms for the error bound, and the split-K partial logits.
+  float amax = 0.f;
+  uint2 xa[4];
+  float4 xf[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int i = j * kFusedThreads + tid;
+    if constexpr (AFMT == MOEV_ACT_BF16)
+      xa[j] = i < g4_all ? __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + i)
+                         : make_uint2(0u, 0u);
+    else
+      xf[j] = i < g4_all ? __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + i)
+                         : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  const int n_et = (E + kRouterETile - 1) / kRouterETile;  // at most 8
+  float nx = 0.f, nw[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) nw[j] = 0.f;
+  if (tid < n_slices) {
+    nx = __ldg(part_x2 + (size_t)tid * gamma + t);
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      if (j < n_et) nw[j] = __ldg(part_w2max + (size_t)tid * n_et + j);
+  }
+  // ---- fp32 logits of this token: the split-K partials summed over the slices in a fixed order
+  // (identical in every CTA of the token)
+  if ((E & 3) == 0 && E / 4 <= kFusedThreads) {
+    const int nq = E / 4, G = kFusedThreads / nq;
+    const int q = tid % nq, g = tid / nq;
+    const size_t cs = (size_t)gamma * E;
+    float4 sacc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (g < G) {
+      const float* pp = part + (size_t)t * E + 4 * q;
+      for (int c = g; c < n_slices; c += 16 * G) {  // sixteen 16-byte loads in flight per thread
+        float4 v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          v[i] = (c + i * G < n_slices) ? __ldg(reinterpret_cast<const float4*>(pp + (size_t)(c + i * G) * cs))
+                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { sacc.x += v[i].x; sacc.y += v[i].y; sacc.z += v[i].z; sacc.w += v[i].w; }
+      }
+      *reinterpret_cast<float4*>(&psum[g * E + 4 * q]) = sacc;
+    }
+    MOEV_RF_MARK(14, first_cta);
+    __syncthreads();
+    MOEV_RF_MARK(15, first_cta);
+    for (int e = tid; e < E; e += kFusedThreads) {
+      float sum = 0.f;
+      for (int gg = 0; gg < G; ++gg) sum += psum[gg * E + e];
+      l32[e] = sum;
+    }
+  } else {
+    const size_t cs = (size_t)gamma * E;
+    for (int e = tid; e < E; e += kFusedThreads) {
+      const float* pp = part + (size_t)t * E + e;
+      float sum = 0.f;
+      for (int c = 0; c < n_slices; c += 16) {
+        float v[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = (c + i < n_slices) ? __ldg(pp + (size_t)(c + i) * cs) : 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sum += v[i];
+      }
+      l32[e] = sum;
+    }
+  }
+  // ---- norms and max |x| (rows longer than 4 * kFusedThreads groups and more than kFusedThreads slices: the rest in loops)
+  float x2 = nx, w2 = 0.f;
+  {
+    float mx = 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mx = fmaxf(mx, nw[j]);
+    w2 = mx;
+  }
+  for (int c = tid + kFusedThreads; c < n_slices; c += kFusedThreads) {
+    x2 += __ldg(part_x2 + (size_t)c * gamma + t);
+    float mx = 0.f;
+    for (int j = 0; j < n_et; ++j) mx = fmaxf(mx, __ldg(part_w2max + (size_t)c * n_et + j));
+    w2 += mx;
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    if constexpr (AFMT == MOEV_ACT_BF16)
+      amax = fmaxf(fmaxf(amax, fmaxf(fabsf(__uint_as_float(xa[j].x << 16)), fabsf(__uint_as_float(xa[j].x & 0xffff0000u)))),
+                   fmaxf(fabsf(__uint_as_float(xa[j].y << 16)), fabsf(__uint_as_float(xa[j].y & 0xffff0000u))));
+    else
+      amax = fmaxf(fmaxf(amax, fmaxf(fabsf(xf[j].x), fabsf(xf[j].y))), fmaxf(fabsf(xf[j].z), fabsf(xf[j].w)));
+  }
+  for (int i = 4 * kFusedThreads + tid; i < g4_all; i += kFusedThreads) {
+    if constexpr (AFMT == MOEV_ACT_BF16) {
+      const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + i);
+      amax = fmaxf(fmaxf(amax, fmaxf(fabsf(__uint_as_float(v.x << 16)), fabsf(__uint_as_float(v.x & 0xffff0000u)))),
+                   fmaxf(fabsf(__uint_as_float(v.y << 16)), fabsf(__uint_as_float(v.y & 0xffff0000u))));
+    } else {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + i);
+      amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+  x2 = warp_sum(x2);
+  w2 = warp_sum(w2);
+  if (lane == 0) { redf[warp] = x2; redw[warp] = w2; reda[warp] = amax; }
+  __syncthreads();  // l32, redf, redw, reda complete
+  MOEV_RF_MARK(1, first_cta);
+
+  // ---- the token's power-of-two activation scale, and this slice of the quantised activation operand of the
+  // tensor-core FFN kernels (see topk_refine_kernel): x * 2^p_t as two e4m3 terms hi + lo / 16 (fp8 weights), as
+  // four packed e2m1 terms with weights 8^-j (MXFP4 weights), or as e4m3 codes with 1 x 128 block scales
+  auto quantise_slice = [&](int qt, int qn) {
+  float am = 0.f;
+  for (int w = 0; w < kFusedWarps; ++w) am = fmaxf(am, reda[w]);
+  int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
+  ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
+  if (s == 0 && qt == 0)
+    T.tok_scale[t] = (T.xq != nullptr && T.xq_mode >= 2) ? 1.f
+                     : __uint_as_float((uint32_t)((T.xq != nullptr && T.xq_mode == 1 ? 1 : 6) - ex + 127) << 23);
+  if (AFMT == MOEV_ACT_BF16 && T.xq != nullptr) {
+    const float ts = __uint_as_float((uint32_t)((T.xq_mode == 1 ? 1 : 6) - ex + 127) << 23);
+    const uint16_t* xr = static_cast<const uint16_t*>(x) + (size_t)t * H;
+    if (T.xq_mode >= 2) {
+      // a warp's 32 lanes x 4 elements are one block (slices begin on block boundaries, H % 128 == 0 here)
+      uint8_t* row = T.xq + (size_t)(2 * t) * T.xq_stride;
+      for (int i = g4_lo + qt; i < g4_hi; i += qn) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(xr + i * 4));
+        const float v[4] = {__uint_as_float(q.x << 16), __uint_as_float(q.x & 0xffff0000u),
+                            __uint_as_float(q.y << 16), __uint_as_float(q.y & 0xffff0000u)};
+        float bm = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) bm = fmaxf(bm, __shfl_xor_sync(0xffffffffu, bm, o));
+        const float sc = act_scale(bm, T.xq_mode - 1);
+        *reinterpret_cast<uint32_t*>(row + i * 4) =
+            act_code(v[0], sc) | (act_code(v[1], sc) << 8) | (act_code(v[2], sc) << 16) | (act_code(v[3], sc) << 24);
+        if (lane == 0) T.xs[(size_t)t * (H / 128) + i / 32] = sc;
+      }
+    } else if (T.xq_mode == 1) {
+      uint8_t* rows = T.xq + (size_t)(4 * t) * T.xq_stride;
+      for (int i = g4_lo / 2 + qt; i < g4_hi / 2; i += qn) {  // 8 elements -> 4 bytes of every term row
+        const uint4 q = __ldg(reinterpret_cast<const uint4*>(xr + i * 8));
+        const uint32_t in[4] = {q.x, q.y, q.z, q.w};
+        uint32_t term[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          const uint32_t sp = split2_e2m1(__uint_as_float(in[p] << 16) * ts, __uint_as_float(in[p] & 0xffff0000u) * ts);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) term[j] |= ((sp >> (8 * j)) & 0xffu) << (8 * p);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) *reinterpret_cast<uint32_t*>(rows + (size_t)j * T.xq_stride + i * 4) = term[j];
+      }
+    } else {
+      uint8_t* hi_row = T.xq + (size_t)(2 * t) * T.xq_stride;
+      uint8_t* lo_row = hi_row + T.xq_stride;
+      for (int i = g4_lo + qt; i < g4_hi; i += qn) {
+        const uint2 q = __ldg(reinterpret_cast<const uint2*>(xr + i * 4));
+        float v[4] = {__uint_as_float(q.x << 16) * ts, __uint_as_float(q.x & 0xffff0000u) * ts,
+                      __uint_as_float(q.y << 16) * ts, __uint_as_float(q.y & 0xffff0000u) * ts};
+        uint32_t hi, lo;
+        split4_e4m3(v, hi, lo);
+        *reinterpret_cast<uint32_t*>(hi_row + i * 4) = hi;
+        *reinterpret_cast<uint32_t*>(lo_row + i * 4) = lo;
+      }
+    }
+  }
+  };
+  // ---- fp32 k-th largest logit (larger value, or equal value and lower id, precedes) in two levels: the k
+  // best of each warp's 32 experts, ranked inside the warp by counting over shuffled values, contain the k
+  // best overall; those entries are then ranked by counting, several threads per entry.  (One thread per
+  // expert counting over all E costs E iterations per thread: it was most of this kernel's instructions.)
+  {
+    const int n_pool = (E + 31) >> 5;  // warps that hold experts (E <= 512 = kFusedThreads)
+    const float v = tid < E ? l32[tid] : -INFINITY;
+    int rank = 0;
+    // the warps that hold no experts quantise the slice meanwhile (all warps, afterwards, when every warp holds some)
+    if (n_pool < kFusedWarps) {
+      if (warp >= n_pool) quantise_slice(tid - 32 * n_pool, kFusedThreads - 32 * n_pool);
+    }
+    if (warp < n_pool) {
+      const uint32_t below = (1u << lane) - 1u;  // lanes (= ids) that win ties against this one
+#pragma unroll 8
+      for (int l = 0; l < 32; ++l) {
+        const float u = __shfl_sync(0xffffffffu, v, l);
+        rank += (u > v || (u == v && ((below >> l) & 1u))) ? 1 : 0;
+      }
+    }
+    const int M = n_pool * k;  // <= 512
+    for (int i = tid; i < M; i += kFusedThreads) { top_v[i] = -INFINITY; top_id[i] = 0x7fffffff; }
+    __syncthreads();
+    if (tid < E && rank < k) { top_v[warp * k + rank] = v; top_id[warp * k + rank] = tid; }
+    if (n_pool >= kFusedWarps) quantise_slice(tid, kFusedThreads);
+    __syncthreads();
+    MOEV_RF_MARK(16, first_cta);
+    int TT = 1;
+    while (2 * TT * M <= kFusedThreads && TT < 32) TT <<= 1;  // threads per entry
+    const int i = tid / TT, sub = tid & (TT - 1), per = (M + TT - 1) / TT;
+    int r = 0;
+    float vi = 0.f;
+    if (i < M) {
+      vi = top_v[i];
+      const int idi = top_id[i];
+      const int j1 = min(M, (sub + 1) * per);
+      for (int j = sub * per; j < j1; ++j) {
+        const float u = top_v[j];
+        r += (u > vi || (u == vi && top_id[j] < idi)) ? 1 : 0;
+      }
+    }
+    for (int o = TT >> 1; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+    if (i < M && sub == 0 && r == k - 1) kth_s = vi;
+  }
+  __syncthreads();
+  MOEV_RF_MARK(2, first_cta);
+  // ---- candidates: every expert whose exact logit may reach the exact k-th largest, ascending id
+  // (error bound as in topk_refine_kernel)
+  int ncand = 0;
+  {
+    float xs = 0.f, wm = 0.f;
+    for (int w = 0; w < kFusedWarps; ++w) { xs += redf[w]; wm += redw[w]; }
+    const float n_round = (float)(ks + n_slices + 4);
+    const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
+    const float thr = kth_s - 2.f * eps;
+    const bool in = tid < E && l32[tid] >= thr;  // E <= kFusedThreads
+    const uint32_t mk = __ballot_sync(0xffffffffu, in);
+    if (lane == 0) wcnt_s[warp] = __popc(mk);
+    __syncthreads();
+    int before = 0;
+    for (int w = 0; w < kFusedWarps; ++w) { const int cw = wcnt_s[w]; before += w < warp ? cw : 0; ncand += cw; }
+    if (in) cand[before + __popc(mk & ((1u << lane) - 1u))] = tid;
+    __syncthreads();
+  }
+  MOEV_RF_MARK(3, first_cta);
+
+  MOEV_RF_MARK(4, first_cta);
+
+  // ---- exact (fp64) partial logits of the candidates over this CTA's slice of H, kFusedCand candidates per pass.
+  // Only the warps that own columns of the slice take part; conversions to fp64 are integer operations and
+  // the warp sums use the entry-halving butterfly: the fp64 pipe is narrow, its instructions are the cost.
+  double* dp = F.dpart + ((size_t)t * S + s) * E;
+  const int n_act = min(kFusedWarps, (g4_hi - g4_lo + 31) >> 5);  // warps with columns in the first trip
+  for (int c0 = 0; c0 < ncand; c0 += kFusedCand) {
+    const int nc = min(kFusedCand, ncand - c0);
+    if (warp < n_act) {
+      double acc[16];
+#pragma unroll
+      for (int q = 0; q < 16; ++q) acc[q] = 0.0;
+      for (int h4 = g4_lo + tid; h4 < g4_hi; h4 += kFusedThreads) {
+        double xv[4];
+        if constexpr (AFMT == MOEV_ACT_BF16) {
+          const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + h4);
+          const uint32_t wd[2] = {v.x, v.y};
+#pragma unroll
+          for (int i = 0; i < 2; ++i) {
+            xv[2 * i] = bf16_bits_to_double(wd[i] & 0xffffu);
+            xv[2 * i + 1] = bf16_bits_to_double(wd[i] >> 16);
+          }
+        } else {
+          const float4 f = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + h4);
+          xv[0] = f32_to_double_int(f.x); xv[1] = f32_to_double_int(f.y);
+          xv[2] = f32_to_double_int(f.z); xv[3] = f32_to_double_int(f.w);
+        }
+        float4 wv[kFusedCand];
+#pragma unroll
+        for (int q0 = 0; q0 < kFusedCand; q0 += 2)
+          if (q0 < nc) {
+#pragma unroll
+            for (int q = q0; q < q0 + 2; ++q)
+              if (q < nc) wv[q] = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)cand[c0 + q] * H) + h4);
+          }
+#pragma unroll
+        for (int q0 = 0; q0 < kFusedCand; q0 += 2)
+          if (q0 < nc) {
+#pragma unroll
+            for (int q = q0; q < q0 + 2; ++q)
+              if (q < nc) {
+                acc[q] = fma(xv[0], f32_to_double_int(wv[q].x), acc[q]); acc[q] = fma(xv[1], f32_to_double_int(wv[q].y), acc[q]);
+                acc[q] = fma(xv[2], f32_to_double_int(wv[q].z), acc[q]); acc[q] = fma(xv[3], f32_to_double_int(wv[q].w), acc[q]);
+              }
+          }
+      }
+      int q;
+      const double a = warp_reduce_scatter16(acc, lane, q);
+      if ((lane & 1) == 0) red[warp][q] = a;
+    }
+    __syncthreads();
+    if (tid < nc) {
+      double a = 0.0;
+      for (int w = 0; w < n_act; ++w) a += red[w][tid];
+      dp[c0 + tid] = a;
+    }
+    __syncthreads();
+  }
+
+  MOEV_RF_MARK(5, first_cta);
+  // ---- hand-over: the CTA of this token that arrives last continues
+  __threadfence();
+  __syncthreads();
+  MOEV_RF_MARK(6, first_cta);
+  if (tid == 0) flag_s = (atomicAdd(F.tok_cnt + t, 1) == S - 1) ? 1 : 0;
+  __syncthreads();
+  if (!flag_s) return;
+  __threadfence();
+  MOEV_RF_MARK(7, t == 0);
+
+  // ---- exact logits: the S partial sums of a candidate are fetched by S adjacent lanes (all loads in flight at
+  // once; a loop over the slices would pay one trip to the L2 per slice) and added by a shuffle tree, whose
+  // order is fixed
+  {
+    int P = 1;
+    while (P < S) P <<= 1;  // lanes per candidate (S <= kFusedMaxSlices = 16)
+    const int sub = tid & (P - 1), per_pass = kFusedThreads / P;
+    for (int c0 = 0; c0 < ncand; c0 += per_pass) {
+      const int c = c0 + tid / P;
+      double a = (c < ncand && sub < S) ? __ldcg(F.dpart + ((size_t)t * S + sub) * E + c) : 0.0;
+      for (int o = P >> 1; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+      if (c < ncand && sub == 0) L[c] = a;
+    }
+  }
+  __syncthreads();
+  MOEV_RF_MARK(8, t == 0);
+  // ---- exact ranking by counting (candidates are stored in ascending id)
+  for (int c = tid; c < ncand; c += kFusedThreads) {
+    const double v = L[c];
+    int rank = 0;
+    for (int c2 = 0; c2 < ncand; ++c2) {
+      const double u = L[c2];
+      rank += (u > v || (u == v && c2 < c)) ? 1 : 0;
+    }
+    if (rank < k) { sel_v_s[rank] = (float)v; sel_e_s[rank] = cand[c]; }  // weights from the exact logits rounded to binary32
+  }
+  __syncthreads();
+  MOEV_RF_MARK(13, t == 0);
+
+  // ---- router weights of the k selected experts (warp 0, lane j owns the j-th), in binary32: the exact logits
+  // rounded once (2^-24 relative) leave the weights far inside the 1e-5 they are compared to
+  if (warp == 0) {
+    const float sel_v = lane < k ? sel_v_s[lane] : 0.f;
+    const int sel_e = lane < k ? sel_e_s[lane] : -1;
+    float wgt = 0.f;
+    if (score == MOEV_SCORE_SOFTMAX) {
+      const float mx = sel_v_s[0];
+      const float exv = lane < k ? expf(sel_v - mx) : 0.f;
+      const float den = warp_sum(exv);
+      wgt = exv / den;
+    } else {
+      const float sg = lane < k ? 1.f / (1.f + expf(-sel_v)) : 0.f;
+      const float den = warp_sum(sg);
+      wgt = routed_scale * sg / (den + 1e-20f);
+    }
+    MOEV_RF_MARK(21, t == 0);
+    if (lane < k) {
+      const int a = t * k + lane;
+      T.topk_ids[a] = sel_e;
+      T.topk_w[a] = wgt;
+      if (O.topk_ids) O.topk_ids[a] = sel_e;
+      if (O.topk_w) O.topk_w[a] = wgt;
+    }
+  }
+
+  MOEV_RF_MARK(9, t == 0);
+  // ---- hand-over: the CTA that finishes the last token builds the grouping tables
+  __threadfence();
+  __syncthreads();
+  MOEV_RF_MARK(10, t == 0);
+  if (tid == 0) flag_s = (atomicAdd(F.done_cnt, 1) == gamma - 1) ? 1 : 0;
+  __syncthreads();
+  if (!flag_s) return;
+  __threadfence();
+  MOEV_RF_MARK(11, true);
+  route_group_block(T, O, gamma, E, k, n_shared, unit_cap, wide_ratio, dyn_sm);
+  __syncthreads();
+  MOEV_RF_MARK(12, true);
+  // every CTA has arrived on every counter: clear them for the next call
+  for (int i = tid; i < gamma; i += kFusedThreads) F.tok_cnt[i] = 0;
+  if (tid == 0) *F.done_cnt = 0;
+}
+
+}  // namespace moev

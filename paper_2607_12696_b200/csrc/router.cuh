@@ -49,6 +49,44 @@ __device__ __forceinline__ float load_act1(const void* x, size_t idx) {
   return bf16_bits_to_float(__ldg(static_cast<const uint16_t*>(x) + idx));
 }
 
+// Expert weights that are known to be needed before the router has decided anything -- the
+// always-on shared experts, and experts a caller's predictor expects (an optional list) -- are
+// pulled into the L2 by the first routing kernel: the routing kernels leave the HBM idle, and the
+// expert kernel then finds those bytes on chip.  Three matrices per expert (gate, up, down), each a
+// contiguous range of `bytes` bytes; the ranges are cut into chunks that the CTAs of the grid
+// share out.  cp.async.bulk.prefetch.L2 completes in the background and nothing waits for it.
+struct PrefetchArgs {
+  const uint8_t* sh[3];      // shared experts' gate / up / down matrices (n_shared of each, contiguous), or null
+  const uint8_t* w[3];       // routed experts' matrices [E][...]
+  unsigned long long bytes;  // bytes of one matrix of one expert (a multiple of 16)
+  const int32_t* pred_ids;   // device list of expert ids to prefetch, or null
+  int n_shared, n_pred;      // shared experts to prefetch (0: none), entries of pred_ids used
+};
+constexpr unsigned kPrefetchChunk = 4 * 1024;
+
+__device__ __forceinline__ void prefetch_l2_range(const uint8_t* p, unsigned bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
+// Called by every thread of every CTA of the grid; cta = linear CTA index, n_cta = CTAs in the grid.
+__device__ __forceinline__ void prefetch_expert_weights(const PrefetchArgs& P, int cta, int n_cta) {
+  const int n_exp = P.n_shared + P.n_pred;
+  if (n_exp == 0) return;
+  const unsigned long long per_mat = (P.bytes + kPrefetchChunk - 1) / kPrefetchChunk;  // chunks of one matrix
+  const unsigned long long total = per_mat * 3ull * (unsigned long long)n_exp;
+  for (unsigned long long i = (unsigned long long)cta * blockDim.x + threadIdx.x; i < total;
+       i += (unsigned long long)n_cta * blockDim.x) {
+    const unsigned long long ch = i % per_mat, rest = i / per_mat;
+    const int mat = (int)(rest % 3ull), ex = (int)(rest / 3ull);
+    const uint8_t* base;
+    if (ex < P.n_shared) base = P.sh[mat] + (unsigned long long)ex * P.bytes;
+    else base = P.w[mat] + (unsigned long long)__ldg(P.pred_ids + (ex - P.n_shared)) * P.bytes;
+    const unsigned long long off = ch * kPrefetchChunk;
+    const unsigned long long left = P.bytes - off;
+    prefetch_l2_range(base + off, (unsigned)(left < kPrefetchChunk ? left : kPrefetchChunk));
+  }
+}
+
 #ifdef MOEV_TC_STATS
 __device__ long long g_rt_stats[32];  // debug builds: phase timestamps of the routing kernels (CTA 0)
 #define MOEV_RT_MARK(i) do { __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) g_rt_stats[i] = clock64(); } while (0)
@@ -72,11 +110,15 @@ __global__ void __launch_bounds__(256) router_partial_kernel(const void* __restr
                                                              float* __restrict__ part,
                                                              float* __restrict__ part_x2,
                                                              float* __restrict__ part_w2max, int gamma,
-                                                             int H, int E, int KS) {
+                                                             int H, int E, int KS, int wait_first,
+                                                             PrefetchArgs pf) {
   __shared__ float wmax_s[8];
   extern __shared__ __align__(16) float rp_smem[];
+  prefetch_expert_weights(pf, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
   float (*x_s)[64 + 4] = reinterpret_cast<float (*)[64 + 4]>(rp_smem);            // [k][token]
   float (*w_s)[64 + 1] = reinterpret_cast<float (*)[64 + 1]>(rp_smem + KS * 68);  // [k][expert]
+  // a dependent layer of a chained call reads x written by the previous layer: wait before the loads
+  if (wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int c = blockIdx.x, e0 = blockIdx.y * kRouterETile;
   const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4, lane = tid & 31, warp = tid >> 5;
@@ -153,7 +195,7 @@ __global__ void __launch_bounds__(256) router_partial_kernel(const void* __restr
   // touches nothing the previous layer still uses, but it must not complete before that layer has:
   // the kernels after it (which do reuse the workspace) wait only for this one.  Without the
   // launch attribute the instruction returns at once.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // The same partials on the tensor cores, for bf16 activations: x is bf16 as it is and every fp32
@@ -170,9 +212,12 @@ __global__ void __launch_bounds__(256) router_partial_mma_kernel(const uint16_t*
                                                                  float* __restrict__ part,
                                                                  float* __restrict__ part_x2,
                                                                  float* __restrict__ part_w2max, int gamma,
-                                                                 int H, int E, int KS) {
+                                                                 int H, int E, int KS, int wait_first,
+                                                                 PrefetchArgs pf) {
   __shared__ float wmax_s[8];
-  __shared__ float sq_s[128];  // [0,64): squared norms of the router rows; [64,128): of the token rows
+  __shared__ float sq_s[128];
+  prefetch_expert_weights(pf, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
+  if (wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");  // chained call: x comes from the previous layer  // [0,64): squared norms of the router rows; [64,128): of the token rows
   extern __shared__ __align__(16) uint16_t rpm_smem[];
   const int LD = KS + kRouterMmaPad;           // row stride in elements
   uint16_t* xs = rpm_smem;                     // [64 tokens][LD]
@@ -184,13 +229,31 @@ __global__ void __launch_bounds__(256) router_partial_mma_kernel(const uint16_t*
   const int k0 = c * KS, kn = min(KS, H - k0);  // kn is a multiple of 4
   if (tid < 128) sq_s[tid] = 0.f;
   __syncthreads();
-  // ---- router tile: float4 per thread and row, split into the three bf16 terms
+  // ---- loads first: a thread's (up to four) router float4s and its token uint2s of the first token tile
+  // are all issued before any is used, so the tile costs one trip to memory instead of one per loop trip
   const int kq4 = KS / 4;
   const bool k64 = KS == 64;  // 16 lanes per row: shifts instead of divisions, shuffles instead of shared atomics
-  for (int i = tid; i < 64 * kq4; i += 256) {
+  const int n_it = (64 * kq4 + 255) / 256;  // <= 4
+  float4 wv[4];
+  uint2 xv0[4];
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int i = tid + it * 256;
     const int er = k64 ? (i >> 4) : i / kq4, kq = (k64 ? (i & 15) : (i % kq4)) * 4;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (e0 + er < E && kq < kn) v = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)(e0 + er) * H + k0 + kq));
+    wv[it] = make_float4(0.f, 0.f, 0.f, 0.f);
+    xv0[it] = make_uint2(0u, 0u);
+    if (it < n_it && i < 64 * kq4 && kq < kn) {
+      if (e0 + er < E) wv[it] = __ldg(reinterpret_cast<const float4*>(router_w + (size_t)(e0 + er) * H + k0 + kq));
+      if (er < gamma) xv0[it] = __ldg(reinterpret_cast<const uint2*>(x + (size_t)er * H + k0 + kq));
+    }
+  }
+  // ---- router tile: float4 per thread and row, split into the three bf16 terms
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    const int i = tid + it * 256;
+    if (it >= n_it || i >= 64 * kq4) break;
+    const int er = k64 ? (i >> 4) : i / kq4, kq = (k64 ? (i & 15) : (i % kq4)) * 4;
+    const float4 v = wv[it];
     const float f[4] = {v.x, v.y, v.z, v.w};
     uint16_t t1[4], t2[4], t3[4];
 #pragma unroll
@@ -219,10 +282,14 @@ __global__ void __launch_bounds__(256) router_partial_mma_kernel(const uint16_t*
     if (tid < 64) sq_s[64 + tid] = 0.f;
     __syncthreads();
     // ---- token tile: 4 bf16 (8 bytes) per thread and row
-    for (int i = tid; i < 64 * kq4; i += 256) {
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      const int i = tid + it * 256;
+      if (it >= n_it || i >= 64 * kq4) break;
       const int tr = k64 ? (i >> 4) : i / kq4, kq = (k64 ? (i & 15) : (i % kq4)) * 4;
       uint2 q = make_uint2(0u, 0u);
-      if (t0 + tr < gamma && kq < kn) q = __ldg(reinterpret_cast<const uint2*>(x + (size_t)(t0 + tr) * H + k0 + kq));
+      if (t0 == 0) q = xv0[it];
+      else if (t0 + tr < gamma && kq < kn) q = __ldg(reinterpret_cast<const uint2*>(x + (size_t)(t0 + tr) * H + k0 + kq));
       *reinterpret_cast<uint2*>(xs + tr * LD + kq) = q;
       const float a = __uint_as_float(q.x << 16), b = __uint_as_float(q.x & 0xffff0000u);
       const float cc = __uint_as_float(q.y << 16), d = __uint_as_float(q.y & 0xffff0000u);
@@ -296,7 +363,129 @@ __global__ void __launch_bounds__(256) router_partial_mma_kernel(const uint16_t*
     for (int w = 1; w < 8; ++w) w2max = fmaxf(w2max, wmax_s[w]);
     part_w2max[(size_t)c * gridDim.y + blockIdx.y] = w2max;
   }
-  asm volatile("griddepcontrol.wait;" ::: "memory");  // see router_partial_kernel
+  if (!wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");  // see router_partial_kernel
+}
+
+// The same partials for calls of at most 32 tokens (tree-sized calls), without shared memory:
+// the router weights are the A operand of mma.sync m16n8k16 (16 experts x 16 k per warp and step),
+// loaded from global memory straight into the fragment layout (a lane's two k-neighbours are one
+// 8-byte load) and split into the three exact bf16 terms in registers; the tokens are the B operand
+// (n8 tiles), a lane's two k-neighbours one 4-byte load of x.  All loads of a warp's K slice are
+// issued before the first is used, there is no barrier before the stores, and the kernel is one
+// trip to memory long.  CTA = 4 warps = 64 experts of one K slice (KS a multiple of 16); grid as
+// router_partial_mma_kernel.  NT = n8 tiles of tokens (gamma <= 8 NT).
+template <int NT>
+__global__ void __launch_bounds__(128) router_partial_small_kernel(const uint16_t* __restrict__ x,
+                                                                   const float* __restrict__ router_w,
+                                                                   float* __restrict__ part,
+                                                                   float* __restrict__ part_x2,
+                                                                   float* __restrict__ part_w2max, int gamma,
+                                                                   int H, int E, int KS, int wait_first,
+                                                                   PrefetchArgs pf) {
+  __shared__ float wmax_s[4];
+  // the weights do not depend on the previous layer: their prefetch runs ahead of the wait below
+  prefetch_expert_weights(pf, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
+  // a dependent layer of a chained call reads x written by the previous layer: wait before the loads
+  if (wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int c = blockIdx.x, e0 = blockIdx.y * kRouterETile;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int k0 = c * KS, kn = min(KS, H - k0);  // kn is a multiple of 4
+  const int r0 = e0 + warp * 16 + (lane >> 2), r1 = r0 + 8;  // this lane's two expert rows
+  const int kc = (lane & 3) * 2;                               // its k pair inside every group of 8
+  constexpr int kMaxSteps = kRouterMaxKS / 16;
+  const int n_steps = (KS + 15) / 16;
+  // ---- loads
+  float2 wa[kMaxSteps][4];   // [step][row0 k-lo, row1 k-lo, row0 k-hi, row1 k-hi]
+  uint32_t xb[kMaxSteps][NT][2];
+#pragma unroll
+  for (int st = 0; st < kMaxSteps; ++st) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int kk = st * 16 + h * 8 + kc;
+      const bool kin = st < n_steps && kk < kn;
+      wa[st][2 * h] = (kin && r0 < E) ? __ldg(reinterpret_cast<const float2*>(router_w + (size_t)r0 * H + k0 + kk)) : make_float2(0.f, 0.f);
+      wa[st][2 * h + 1] = (kin && r1 < E) ? __ldg(reinterpret_cast<const float2*>(router_w + (size_t)r1 * H + k0 + kk)) : make_float2(0.f, 0.f);
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const int tok = nt * 8 + (lane >> 2);
+        xb[st][nt][h] = (kin && tok < gamma) ? __ldg(reinterpret_cast<const uint32_t*>(x + (size_t)tok * H + k0 + kk)) : 0u;
+      }
+    }
+  }
+  float acc[NT][4];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[nt][i] = 0.f;
+  float w2a = 0.f, w2b = 0.f;  // squared norms of this lane's pieces of rows r0, r1
+  float x2[NT];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) x2[nt] = 0.f;
+#pragma unroll
+  for (int st = 0; st < kMaxSteps; ++st) {
+    if (st < n_steps) {
+      uint32_t a[3][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float f[2] = {wa[st][i].x, wa[st][i].y};
+        uint32_t t1[2], t2[2], t3[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          const uint32_t b1 = __float_as_uint(f[j]) & 0xffff0000u;   // truncation: exact 8-bit significand
+          const float r1f = f[j] - __uint_as_float(b1);               // exact
+          const uint32_t b2 = __float_as_uint(r1f) & 0xffff0000u;
+          const float r2f = r1f - __uint_as_float(b2);                // exact, at most 8 significant bits left
+          t1[j] = b1 >> 16; t2[j] = b2 >> 16; t3[j] = __float_as_uint(r2f) >> 16;
+        }
+        a[0][i] = t1[0] | (t1[1] << 16); a[1][i] = t2[0] | (t2[1] << 16); a[2][i] = t3[0] | (t3[1] << 16);
+        const float sq = fmaf(f[0], f[0], f[1] * f[1]);
+        if (i & 1) w2b += sq; else w2a += sq;
+      }
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float p = __uint_as_float(xb[st][nt][h] << 16), q = __uint_as_float(xb[st][nt][h] & 0xffff0000u);
+          x2[nt] = fmaf(p, p, fmaf(q, q, x2[nt]));
+        }
+#pragma unroll
+        for (int term = 0; term < 3; ++term)
+          asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                       : "+f"(acc[nt][0]), "+f"(acc[nt][1]), "+f"(acc[nt][2]), "+f"(acc[nt][3])
+                       : "r"(a[term][0]), "r"(a[term][1]), "r"(a[term][2]), "r"(a[term][3]), "r"(xb[st][nt][0]), "r"(xb[st][nt][1]));
+      }
+    }
+  }
+  // ---- C fragments: rows r0 (acc 0, 1) and r1 (acc 2, 3), token columns 2 (lane % 4) + {0, 1} of each n8 tile
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int tok = nt * 8 + (lane & 3) * 2 + (i & 1), e = (i & 2) ? r1 : r0;
+      if (tok < gamma && e < E) part[((size_t)c * gamma + tok) * E + e] = acc[nt][i];
+    }
+  // ---- squared norms: of the token rows over this slice (a token's k pieces lie in the four lanes of a group) ...
+  if (blockIdx.y == 0 && warp == 0) {
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      float v = x2[nt];
+      v += __shfl_xor_sync(0xffffffffu, v, 1);
+      v += __shfl_xor_sync(0xffffffffu, v, 2);
+      const int tok = nt * 8 + (lane >> 2);
+      if ((lane & 3) == 0 && tok < gamma) part_x2[(size_t)c * gamma + tok] = v;
+    }
+  }
+  // ... and the largest one among this tile's router rows
+  w2a += __shfl_xor_sync(0xffffffffu, w2a, 1); w2a += __shfl_xor_sync(0xffffffffu, w2a, 2);
+  w2b += __shfl_xor_sync(0xffffffffu, w2b, 1); w2b += __shfl_xor_sync(0xffffffffu, w2b, 2);
+  float w2max = fmaxf(w2a, w2b);
+#pragma unroll
+  for (int o = 4; o < 32; o <<= 1) w2max = fmaxf(w2max, __shfl_xor_sync(0xffffffffu, w2max, o));
+  if (lane == 0) wmax_s[warp] = w2max;
+  __syncthreads();
+  if (tid == 0) part_w2max[(size_t)c * gridDim.y + blockIdx.y] = fmaxf(fmaxf(wmax_s[0], wmax_s[1]), fmaxf(wmax_s[2], wmax_s[3]));
+  if (!wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");  // see router_partial_kernel
 }
 
 struct RouteOut {  // optional caller-visible copies (may be null)

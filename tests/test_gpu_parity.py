@@ -178,6 +178,53 @@ def test_pipelined_layers_match_oracle(base, kw):
     v.close()
 
 
+@pytest.mark.parametrize("base,kw,gamma,prefetch", [("deepseek", dict(H=1024, I=512, E=64), 24, False),
+                                                    ("deepseek", dict(H=1024, I=512, E=64), 8, True),
+                                                    ("gptoss", dict(H=704, I=320, E=32), 24, False),
+                                                    ("qwen", dict(H=1024, I=384, E=32), 40, True)])
+def test_chained_dependent_layers_match_oracle(base, kw, gamma, prefetch):
+    """moev_verify_chain: four dependent layers in one call, layer l + 1 verifying the output of
+    layer l.  Every layer is checked against the oracle evaluated on the input that layer actually
+    saw (x0, then the previous layer's bf16 output as the device produced it): the routing tables
+    bit for bit, the output within the format's tolerance.  A layer that read its input before the
+    previous one had finished would fail both.  The inputs are rescaled between the layers by the
+    test's own router (logits come from the hidden state itself), so ties and near-ties occur as
+    they fall.  Run twice; with the weight prefetch on, a (partly wrong) expert prediction must not
+    change any result."""
+    shape = small_shape(base, **kw)
+    n = 4
+    v = moev.MoeVerifier(gcfg(shape, gamma))
+    v.prefetch_enable(prefetch)
+    layers, keep, hosts = [], [], []
+    for l in range(n):
+        w = synth.make_expert_weights(shape, layer=l, device="cuda")
+        wr, x = synth.make_iid_routing(shape, gamma, layer=l, device="cuda")
+        wr = wr * 50.0  # the layer outputs are small: keep the logits of later layers well separated
+        d = {"router_w": wr}
+        d.update({k: t for k, t in w.items() if t is not None})
+        if prefetch:
+            d["predicted_ids"] = torch.arange(l, l + 6, dtype=torch.int32, device="cuda") % shape.E
+        layers.append(moev.binding.make_layer(d)); keep.append(d)
+        hosts.append(synth.layer_to_numpy(wr, w))
+        if l == 0:
+            x0 = x
+    for rep in range(2):
+        outs = [v.alloc_out(gamma) for _ in range(n)]
+        v.verify_chain(layers, x0, gamma, outs)
+        v.status_sync()
+        torch.cuda.synchronize()
+        x_in, compared = x0, 0
+        for l in range(n):
+            ref = oracle.moe_verify(ocfg(shape), hosts[l], synth.to_numpy(x_in), gamma)
+            res = {k: (t.float() if t.dtype == torch.bfloat16 else t).cpu().numpy() for k, t in outs[l].items()}
+            if ref.gap.min() > 1e-9:   # (a near-tie in the fp64 logits leaves the ids undefined)
+                compare(shape, res, ref, gamma)
+                compared += 1
+            x_in = outs[l]["y"]
+        assert compared >= n - 1
+    v.close()
+
+
 def test_context_reuse_and_smaller_gamma():
     """One context, several calls with different gamma: workspace state must not leak."""
     shape = small_shape("qwen", H=512, I=256, E=16, top_k=4)
