@@ -16,6 +16,21 @@ constexpr int kMaxTopK = 32;     // one lane per selected expert
 constexpr int kStatusOk = 0;
 constexpr int kStatusTimeout = 1;
 
+// Test builds of the library (-DMOEV_TEST_HOOKS, a second shared object that only the tests load)
+// can make a bounded wait run out on purpose: while g_test_withhold is non-zero the task
+// schedulers of the expert kernels do not publish their final "no more work" message and the grid
+// barrier of the selection kernel expects one arrival too many, so the waiting roles give up when
+// their (millisecond) budget is spent and the kernels leave through their abort paths.  Nothing
+// faults and nothing spins without a bound.  The shipped library has neither the flag nor the code.
+#ifdef MOEV_TEST_HOOKS
+__device__ int g_test_withhold;
+#define MOEV_TEST_WITHHOLD() (*reinterpret_cast<volatile int*>(&g_test_withhold) != 0)
+constexpr unsigned long long kDeviceWaitBudgetNs = 2000000ull;  // 2 ms
+#else
+#define MOEV_TEST_WITHHOLD() false
+constexpr unsigned long long kDeviceWaitBudgetNs = 2000000000ull;  // 2 s per wait
+#endif
+
 // One unit of tensor-core FFN work: an expert and a contiguous run of at most MC of its
 // assignment slots (experts with more tokens are split into several units).
 struct __align__(16) Unit {

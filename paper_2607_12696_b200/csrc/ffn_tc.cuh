@@ -85,7 +85,7 @@ constexpr int kBSlots = 3;                  // activation-operand ring
 constexpr int kNMax = 64;                   // widest N operand
 constexpr int kTaskQ = 4;                   // depth of the task-id queue between the roles
 constexpr int kTmemCols = 512;              // (G 64 | P 64) x 2 task parities | O[2 stages][<=2 tiles] 64 each
-constexpr uint64_t kWaitBudgetNs = 2000000000ull;  // 2 s per wait
+constexpr uint64_t kWaitBudgetNs = kDeviceWaitBudgetNs;  // 2 s per wait (milliseconds in test builds)
 
 // tiles (fp8: 160 + 48 + 8 KB, bf16: 160 + 24 + 16 KB) + 1 KB alignment slack + 8 KB control block
 constexpr int kTileBytes = kStages * kStageBytes + 56 * 1024;
@@ -121,6 +121,8 @@ struct Smem {
   uint64_t d_full[2], d_empty[2];
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar;  // epilogue group barrier (128 threads), bounded like every other wait
+  uint64_t drain_bar[2];  // abort path: one per MMA issuer
+  volatile uint32_t prod_it;  // ring stages the producer armed (read on the abort path)
   volatile int32_t tq_task[kTaskQ];
   uint32_t tmem_base;
   volatile int abort_flag;
@@ -278,6 +280,8 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.d_full[i], 2); ptx::mbar_init(&S.d_empty[i], 128); }
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
+    ptx::mbar_init(&S.drain_bar[0], 1); ptx::mbar_init(&S.drain_bar[1], 1);
+    S.prod_it = 0;
     S.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -343,6 +347,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           if (id >= n_ids) { id = -1; break; }
           td = decode_task(id, n_units, n_slices);
         } while (!td.valid);
+        if (id < 0 && MOEV_TEST_WITHHOLD()) return -1;  // test builds: the final message is withheld
         const int slot = q % kTaskQ;
         ok = ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
         if (!ok) return -2;
@@ -412,6 +417,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         id = id_next; td = td_next;
         id_next = id_nn; td_next = td_nn;
       }
+      S.prod_it = it;
 #ifdef MOEV_TC_STATS
       st_acc[15] = (unsigned long long)(clock64() - st_begin);
       if (P.stats)
@@ -530,6 +536,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         id = id_next;
         idesc = idesc_next;
       }
+      if (*abortp) ptx::drain_issuer(&S.drain_bar[issuer], kWaitBudgetNs);
 #ifdef MOEV_TC_STATS
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
@@ -879,9 +886,14 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     }
   }
 
-  // ---- teardown: everyone arrives; TMEM is released by the warp that allocated it
+  // ---- teardown: everyone arrives; on the abort path the copies still in flight into the ring are
+  // waited for (the issuers have waited for their MMAs); TMEM is released by the warp that allocated it
   ptx::tc_fence_before();
   __syncthreads();
+  if (S.abort_flag) {
+    if (tid == 0) ptx::drain_ring(S.w_full, kStages, S.prod_it, kWaitBudgetNs);
+    __syncthreads();
+  }
   if (warp == 0) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, kTmemCols);

@@ -121,6 +121,8 @@ struct Smem {
   uint64_t acc_full[2], acc_empty[2];
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar, pr_bar;
+  uint64_t drain_bar[2];       // abort path: one per MMA issuer
+  volatile uint32_t prod_it;   // ring stages the producer armed (read on the abort path)
   volatile int32_t tq_task[kTaskQ];
   uint32_t tmem_base;
   volatile int abort_flag;
@@ -209,6 +211,8 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     ptx::mbar_init(&S.pr_bar, 128);
+    ptx::mbar_init(&S.drain_bar[0], 1); ptx::mbar_init(&S.drain_bar[1], 1);
+    S.prod_it = 0;
     S.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -252,6 +256,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       auto fetch_publish = [&]() -> int {
         int id = atomicAdd(P.task_counter, 1);
         if (id >= n_ids) id = -1;
+        if (id < 0 && MOEV_TEST_WITHHOLD()) return -1;  // test builds: the final message is withheld
         const int slot = q % kTaskQ;
         ok = ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
         if (!ok) return -2;
@@ -309,6 +314,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         load(id);
         id = id_next;
       }
+      S.prod_it = it;
     }
   } else if (warp == 1 || warp == 10) {
     // ===================================================== MMA issuers (one lane each): issuer i runs tile i of every stage
@@ -368,6 +374,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         if (!ok) break;
         ptx::mma_commit(&S.acc_full[pb]);
       }
+      if (*abortp) ptx::drain_issuer(&S.drain_bar[issuer], kWaitBudgetNs);
 #ifdef MOEV_TC_STATS
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
@@ -689,8 +696,15 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #endif
   }
 
+  // abort path: the asynchronous copies of the scale rows and the bulk copies still in flight into the ring have
+  // landed before shared memory is given back (the issuers have waited for their MMAs and scale-factor copies)
+  asm volatile("cp.async.wait_all;" ::: "memory");
   ptx::tc_fence_before();
   __syncthreads();
+  if (S.abort_flag) {
+    if (tid == 0) ptx::drain_ring(S.w_full, kStages, S.prod_it, kWaitBudgetNs);
+    __syncthreads();
+  }
   if (warp == 0) {
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, kTmemCols);

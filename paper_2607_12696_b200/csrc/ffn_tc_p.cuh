@@ -55,6 +55,8 @@ struct Smem {
   uint64_t h_full, h_empty;
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar, all_bar;
+  uint64_t drain_bar[2];       // abort path: one per MMA issuer
+  volatile uint32_t prod_it;   // ring stages the producer armed (read on the abort path)
   volatile int32_t tq_task[kTaskQ];
   volatile int abort_flag;
   int32_t e_tok[2][kMC];
@@ -109,6 +111,8 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     ptx::mbar_init(&S.all_bar, 256);
+    ptx::mbar_init(&S.drain_bar[0], 1); ptx::mbar_init(&S.drain_bar[1], 1);
+    S.prod_it = 0;
     S.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -135,7 +139,9 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           td = decode_task(id, n_units, n_slices);
         } while (!td.valid);
         const int slot = q % kTaskQ;
-        if (ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs)) {
+        if (id < 0 && MOEV_TEST_WITHHOLD()) {
+          // test builds: the final message is withheld
+        } else if (ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs)) {
           S.tq_task[slot] = id;
           ptx::mbar_arrive(&S.tq_full[slot]);
         } else {
@@ -199,6 +205,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
       id = id_next;
       td = td_next;
     }
+    if (lane == 0) S.prod_it = it;
   } else if (warp == 1 || warp == 10) {
     // ===================================================== MMA issuers (one lane each): issuer i = gate / up tile of the
     // first phase (columns 64 i of the partial buffer), tile i of every stage of the down phase
@@ -265,6 +272,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
       }
+      if (*abortp) ptx::drain_issuer(&S.drain_bar[issuer], kWaitBudgetNs);
 #ifdef MOEV_TC_STATS
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
@@ -513,7 +521,13 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
       for (int i = 0; i < 3; ++i) P.stats[(size_t)blockIdx.x * 16 + 13 + i] = est[i];
 #endif
   }
-  // the caller synchronises the CTA and releases TMEM
+  // abort path: the copies still in flight into the ring have landed before the shared memory is given back
+  // (the issuers have waited for their MMAs); the caller synchronises the CTA and releases TMEM
+  __syncthreads();
+  if (S.abort_flag) {
+    if (tid == 0) ptx::drain_ring(S.w_full, kStages, S.prod_it, kWaitBudgetNs);
+    __syncthreads();
+  }
 }
 
 }  // namespace tcp

@@ -68,6 +68,8 @@ struct Smem {
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar;                     // barrier of group 0 (128 threads)
   uint64_t all_bar;                    // barrier of both groups (256 threads)
+  uint64_t drain_bar[2];               // abort path: one per MMA issuer
+  volatile uint32_t prod_it;           // ring stages the producer armed (read on the abort path)
   volatile int32_t tq_task[kTaskQ];
   volatile int abort_flag;
   // tables, double-buffered by task parity; every warp writes all entries it reads (identical values)
@@ -158,6 +160,8 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
     ptx::mbar_init(&S.all_bar, 256);
+    ptx::mbar_init(&S.drain_bar[0], 1); ptx::mbar_init(&S.drain_bar[1], 1);
+    S.prod_it = 0;
     S.abort_flag = 0;
     ptx::fence_mbar_init();
   }
@@ -207,7 +211,9 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         id = atomicAdd(P.task_counter, 1);
         if (id >= n_ids) id = -1;
         const int slot = q % kTaskQ;
-        if (ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs)) {
+        if (id < 0 && MOEV_TEST_WITHHOLD()) {
+          // test builds: the final message is withheld
+        } else if (ptx::bounded_wait(&S.tq_empty[slot], ((q / kTaskQ) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs)) {
           S.tq_task[slot] = id;
           ptx::mbar_arrive(&S.tq_full[slot]);
         } else {
@@ -283,6 +289,7 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
       }
       id = id_next;
     }
+    if (lane == 0) S.prod_it = it;
   } else if (warp == 1 || warp == 10) {
     // ===================================================== MMA issuers (one lane each): issuer 0 = gate tile /
     // first H tile -> columns 0..63 of the partial buffer, issuer 1 = up tile / second H tile -> columns 64..127
@@ -336,6 +343,7 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         }
         if (!ok) break;
       }
+      if (*abortp) ptx::drain_issuer(&S.drain_bar[issuer], kWaitBudgetNs);
 #ifdef MOEV_TC_STATS
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       if (P.stats && issuer == 0)
@@ -522,7 +530,13 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
     }
 #endif
   }
-  // the caller synchronises the CTA and releases TMEM
+  // abort path: the copies still in flight into the ring have landed before the shared memory is given back
+  // (the issuers have waited for their MMAs); the caller synchronises the CTA and releases TMEM
+  __syncthreads();
+  if (S.abort_flag) {
+    if (tid == 0) ptx::drain_ring(S.w_full, kStages, S.prod_it, kWaitBudgetNs);
+    __syncthreads();
+  }
 }
 
 }  // namespace tcw

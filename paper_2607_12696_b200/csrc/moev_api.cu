@@ -21,7 +21,7 @@ namespace {
 constexpr int kProfSlots = 512;
 // expert-weight bytes the first routing kernel may pull into the L2 ahead of the expert kernel (B200: 126 MB of L2)
 constexpr size_t kPrefetchBudgetBytes = 80u * 1024u * 1024u;
-constexpr int kTmapCache = 8;
+constexpr int kTmapCache = 256;  // descriptor sets kept per context (a power of two): a model's layers (36 - 94) stay encoded
 
 // The six TMA descriptors of one layer (gate, up, down, shared gate, up, down) and the
 // pointers they were encoded for.
@@ -210,13 +210,22 @@ bool encode_weight_map_mx(CUtensorMap* m, const void* ptr, int n_mat, int N, int
   return r == CUDA_SUCCESS;
 }
 
-// Find or build the descriptors of this layer (cache keyed by the six weight pointers).
+// Find or build the descriptors of this layer.  The cache is a hash table keyed by the six weight
+// pointers (open addressing from a hash of the gate tensor's address, a few probes): a caller that
+// cycles through the layers of a model finds every layer's six descriptors encoded after its first pass.
 const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
   const void* key[6] = {L->w_gate, L->w_up, L->w_down, L->sh_gate, L->sh_up, L->sh_down};
-  for (int i = 0; i < kTmapCache; ++i)
+  constexpr int kProbes = 8;
+  const uintptr_t a = reinterpret_cast<uintptr_t>(L->w_gate) >> 8;
+  const unsigned h0 = (unsigned)((a ^ (a >> 13) ^ (a >> 27)) * 2654435761u);
+  int victim = -1;
+  for (int p = 0; p < kProbes; ++p) {
+    const int i = (int)((h0 + (unsigned)p) & (kTmapCache - 1));
     if (c->tmaps[i].valid && memcmp(c->tmaps[i].key, key, sizeof(key)) == 0) return &c->tmaps[i];
-  TmapSet& t = c->tmaps[c->tmap_next];
-  c->tmap_next = (c->tmap_next + 1) % kTmapCache;
+    if (victim < 0 && !c->tmaps[i].valid) victim = i;
+  }
+  if (victim < 0) victim = (int)((h0 + (unsigned)(c->tmap_next++ % kProbes)) & (kTmapCache - 1));  // all probes taken: replace one in turn
+  TmapSet& t = c->tmaps[victim];
   t.valid = false;
   const moev_config& g = c->cfg;
   auto enc = [&](CUtensorMap* m, const void* ptr, int n_mat, int N, int K) {
@@ -899,6 +908,14 @@ moev_status moev_select_drafts(int32_t n, int32_t W, const int32_t* parent, cons
       n_selected);
   return cudaGetLastError() == cudaSuccess ? MOEV_OK : MOEV_ECUDA;
 }
+
+#ifdef MOEV_TEST_HOOKS
+// Test builds only: while the flag is set, bounded device waits are made to run out (see common.cuh).
+extern "C" int32_t moev_test_withhold(int32_t on) {
+  const int v = on ? 1 : 0;
+  return cudaMemcpyToSymbol(g_test_withhold, &v, sizeof(int)) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 #ifdef MOEV_TC_STATS
 extern "C" int32_t moev_debug_rt_stats(long long* host_out /*[32]*/) {

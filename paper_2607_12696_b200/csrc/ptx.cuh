@@ -65,6 +65,28 @@ __device__ __forceinline__ bool bounded_wait(uint64_t* bar, uint32_t parity, vol
   }
 }
 
+// Abort path only.  Before a CTA that gave up a wait hands back its shared memory and TMEM, what it
+// started asynchronously must have finished: bulk tensor copies still in flight would land in shared
+// memory the next CTA owns, MMAs still running would write TMEM columns that are being freed.
+// drain_wait: bounded wait for a phase of a barrier that changes no status.
+__device__ __forceinline__ bool drain_wait(uint64_t* bar, uint32_t parity, uint64_t budget_ns) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = globaltimer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 0 && globaltimer_ns() - t0 > budget_ns) return false;
+  }
+}
+// drain_ring: the producer armed `it` stages of an n_stages ring (stage = it % n_stages, one arming per
+// use); wait for the last arming of every stage to complete (its copies have landed).
+__device__ __forceinline__ void drain_ring(uint64_t* w_full, int n_stages, uint32_t it, uint64_t budget_ns) {
+  for (int s = 0; s < n_stages; ++s) {
+    if (it <= (uint32_t)s) continue;
+    const uint32_t last = ((it - 1u - (uint32_t)s) / (uint32_t)n_stages) * (uint32_t)n_stages + (uint32_t)s;
+    drain_wait(&w_full[s], (last / (uint32_t)n_stages) & 1u, budget_ns);
+  }
+}
+
 // ---- proxy fences
 __device__ __forceinline__ void fence_proxy_async_smem() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -157,6 +179,11 @@ constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ void mma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
+}
+// drain_issuer: all tensor-core operations this thread has issued (MMAs, tcgen05.cp) have completed.
+__device__ __forceinline__ void drain_issuer(uint64_t* bar, uint64_t budget_ns) {
+  mma_commit(bar);
+  drain_wait(bar, 0u, budget_ns);
 }
 // 32 lanes x 16 consecutive 32-bit columns: thread i of the warp receives lane (base_lane + i).
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
