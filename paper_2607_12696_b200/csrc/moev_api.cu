@@ -643,8 +643,11 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
              c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
   else if (gamma <= 32) {
     // tree-sized calls: the variant without shared memory (one trip to memory long)
+    // (a dependent layer's first kernel is not launched ahead at these sizes: its CTAs, resident and waiting beside
+    // the previous layer's expert kernel, cost that kernel more than the early launch saves -- measured +4 % per
+    // layer at gamma = 4, against -2 % at gamma = 64)
     auto go = [&](auto kern) {
-      launch_k(kern, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(128), 0, st, pdl && c->chain != 0,
+      launch_k(kern, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(128), 0, st, pdl && c->chain == 1,
                static_cast<const uint16_t*>(x), layer->router_w, c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
     };
     if (gamma <= 8) go(router_partial_small_kernel<1>);
