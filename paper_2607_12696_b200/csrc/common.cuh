@@ -69,6 +69,10 @@ struct Tables {
   int32_t* status;     // [1]   kStatusOk / kStatusTimeout
 };
 
+#ifdef MOEV_TC_STATS
+__device__ long long g_rt_stats[32];  // debug builds: phase timestamps (CTA 0) of the routing and expert kernels
+#endif
+
 struct LayerPtrs {
   const void *w_gate, *w_up, *w_down;
   const void *s_gate, *s_up, *s_down;

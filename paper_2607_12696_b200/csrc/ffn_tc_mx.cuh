@@ -194,6 +194,12 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef MOEV_TC_STATS
+#define MOEV_MX_MARK(i) do { if (blockIdx.x == 0) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); g_rt_stats[i] = (long long)_t; } } while (0)
+#else
+#define MOEV_MX_MARK(i)
+#endif
+  if (tid == 0) MOEV_MX_MARK(24);
   const int H = P.H, I = P.I;
   const int KC1 = (H + 255) / 256, KC2 = (I + 255) / 256;  // 256-element K chunks of the two phases (the last may be ragged)
   const int n_slices = (I + 127) / 128;                     // phase-1 tasks per unit
@@ -235,8 +241,10 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
+  if (tid == 0) MOEV_MX_MARK(25);
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (tid == 0) MOEV_MX_MARK(26);
   const int n_units = *P.n_units;
   const int n_p1 = n_units * n_slices;
   const int n_ids = n_p1 + n_units * n_pairs;
@@ -327,6 +335,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #ifdef MOEV_TC_STATS
       unsigned long long st_acc[16] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
       const long long st_begin = clock64();
+      if (issuer == 0) MOEV_MX_MARK(27);
 #endif
       for (;; ++tcount) {
         const int id = next_task(S, q, abortp, P.status, false);
@@ -376,6 +385,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       }
       if (*abortp) ptx::drain_issuer(&S.drain_bar[issuer], kWaitBudgetNs);
 #ifdef MOEV_TC_STATS
+      if (issuer == 0) MOEV_MX_MARK(28);
       st_acc[0] = (unsigned long long)(clock64() - st_begin);
       st_acc[7] = tcount;
       if (P.stats && issuer == 0)
@@ -709,6 +719,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, kTmemCols);
   }
+  if (tid == 0) MOEV_MX_MARK(29);
 }
 
 }  // namespace tcmx

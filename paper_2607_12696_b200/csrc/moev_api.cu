@@ -249,19 +249,35 @@ const TmapSet* get_tmaps(moev_ctx* c, const moev_layer* L) {
 // while its predecessor in the stream drains; it calls griddepcontrol.wait before touching the
 // predecessor's results.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
-                     Args&&... args) {
+cudaError_t launch_kc(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                      int cluster_x, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (cluster_x > 0) {  // thread-block clusters of cluster_x CTAs along x
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x;
+    attr[n].val.clusterDim.y = 1;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
+  cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                     Args&&... args) {
+  return launch_kc(kern, grid, block, smem, st, pdl, 0, static_cast<Args&&>(args)...);
 }
 
 template <int WFMT>
@@ -401,17 +417,12 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && dmalloc(&c->part_x2, (size_t)c->n_slices * G) == cudaSuccess;
   ok = ok && dmalloc(&c->part_w2, (size_t)c->n_slices * ((E + kRouterETile - 1) / kRouterETile)) == cudaSuccess;
   if (cfg->n_group == 0) {
-    // two-launch routing: partial fp64 logits per (token, slice), arrival counters (zero between calls)
-    size_t rows = 0;
+    // two-launch routing: the counter of finished tokens (zero between calls)
     const int gmax = cfg->max_tokens < kFusedMaxTokens ? cfg->max_tokens : kFusedMaxTokens;
-    for (int g = 1; g <= gmax; ++g) {
-      rows = std::max(rows, (size_t)g * fused_slices(g, cfg->H, prop.multiProcessorCount));
+    for (int g = 1; g <= gmax; ++g)
       c->fused_smem_max = std::max(c->fused_smem_max, route_group_block_smem(cfg->E, g, cfg->top_k));
-    }
-    ok = ok && dmalloc(&c->fused.dpart, rows * E) == cudaSuccess;
-    ok = ok && dmalloc(&c->fused.tok_cnt, (size_t)gmax + 1) == cudaSuccess;
-    ok = ok && cudaMemset(c->fused.tok_cnt, 0, ((size_t)gmax + 1) * sizeof(int32_t)) == cudaSuccess;
-    if (ok) c->fused.done_cnt = c->fused.tok_cnt + gmax;
+    ok = ok && dmalloc(&c->fused.done_cnt, 1) == cudaSuccess;
+    ok = ok && cudaMemset(c->fused.done_cnt, 0, sizeof(int32_t)) == cudaSuccess;
   }
   ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
@@ -522,11 +533,11 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     if (gs > 48 * 1024)
       ok = ok && cudaFuncSetAttribute(route_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)gs) == cudaSuccess;
-    if (c->fused_smem_max > 20 * 1024) {  // beside about 24 KB of static tables
+    if (cfg->n_group == 0) {  // its static tables exceed the default limit already
       ok = ok && cudaFuncSetAttribute(route_refine_kernel<MOEV_ACT_FP32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)c->fused_smem_max) == cudaSuccess;
+                                      (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(route_refine_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)c->fused_smem_max) == cudaSuccess;
+                                      (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
     }
     if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
       ok = ok && cudaFuncSetAttribute(tc::grouped_ffn_tc_kernel<MOEV_W_BF16>,
@@ -549,7 +560,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
 
 moev_status moev_destroy(moev_ctx* c) {
   if (!c) return MOEV_EINVAL;
-  cudaFree(c->fused.dpart); cudaFree(c->fused.tok_cnt);
+  cudaFree(c->fused.done_cnt);
   cudaFree(c->part); cudaFree(c->part_x2); cudaFree(c->part_w2); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
@@ -665,7 +676,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
     const int S = fused_slices(gamma, g.H, c->n_sm);
     const size_t gsm = route_group_block_smem(g.E, gamma, g.top_k);
     auto go = [&](auto kern) {
-      launch_k(kern, dim3(S, gamma), dim3(kFusedThreads), gsm, st, pdl, c->T, O, c->fused, x, layer->router_w,
+      launch_kc(kern, dim3(S, gamma), dim3(kFusedThreads), gsm, st, pdl, S, c->T, O, c->fused, x, layer->router_w,
                (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
                g.top_k, c->n_slices, refine_depth, g.score, g.routed_scale, g.n_shared, c->unit_cap, wide_ratio);
     };

@@ -1,24 +1,28 @@
 // Routing for tree-sized calls in two launches instead of three, with the per-token work spread
-// over several CTAs.
+// over a thread-block cluster.
 //
-//   route_refine_kernel   grid (S, gamma): CTA (s, t) sums the split-K partial logits of token t,
-//                         takes the candidates of the top-k under the rounding-error bound (every
-//                         CTA of a token derives the same list from the same numbers), evaluates
-//                         their exact fp64 logits over its slice s of the hidden dimension and
-//                         publishes the partial sums, and writes its slice of the token's
-//                         quantised activations.  The CTA of a token that arrives last adds the
-//                         S partial sums in a fixed order, ranks the candidates exactly (larger
-//                         logit first, ties to the lower id) and forms the router weights.  The CTA that finishes the last token
-//                         builds the expert union, offsets, permutation and FFN work units
-//                         (route_group_block).  Nothing in the kernel waits: the hand-overs are
-//                         "last arrival continues" counters (release by fence + atomic add,
-//                         acquire by the atomic's result + fence), so there is no spin and no
-//                         co-residency requirement.
+//   route_refine_kernel   grid (S, gamma), clusters of S CTAs = one token.  CTA s sums its share of
+//                         the split-K partial logits; the S partial vectors are exchanged through
+//                         distributed shared memory and added in rank order, so every CTA of the
+//                         cluster holds the same fp32 logits; warp 0 finds the k-th largest and the
+//                         candidates of the top-k under the rounding-error bound; the CTA evaluates
+//                         the candidates' exact fp64 logits over its slice s of the hidden
+//                         dimension, writes its slice of the token's quantised activations, and
+//                         stores its partial sums into the shared memory of the cluster's first
+//                         CTA.  That CTA adds them in rank order, ranks the candidates exactly
+//                         (larger logit first, ties to the lower id) and forms the router weights.
+//                         The CTA that finishes the last token builds the expert union, offsets,
+//                         permutation and FFN work units (route_group_block): a "last arrival
+//                         continues" counter (release by fence + atomic add, acquire by the
+//                         atomic's result + fence).  Cluster barriers are the hardware's; nothing
+//                         in the kernel spins.
 //
 // The results are those of topk_refine_kernel + route_group_kernel: the same candidates, the
 // same fp64 ranking rule, the same tables.  Group-limited routing (two dependent candidate
 // stages) and calls of more than kFusedMaxTokens rows keep the three-kernel path.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "router.cuh"
 
@@ -33,28 +37,25 @@ namespace moev {
 constexpr int kFusedThreads = 512;
 constexpr int kFusedWarps = kFusedThreads / 32;
 constexpr int kFusedMaxTokens = 128;   // rows per call served by this path
-constexpr int kFusedMaxSlices = 16;    // CTAs per token
+constexpr int kFusedMaxSlices = 8;     // CTAs per token = cluster size (the portable maximum)
 constexpr int kFusedCand = 12;         // candidates evaluated per pass over the slice
 
-// CTAs per token: one CTA per SM in total (one wave), at most kFusedMaxSlices, slices of at least 256 columns.
+// CTAs per token (a power of two): one CTA per SM in total (one wave), at most kFusedMaxSlices, slices of at
+// least 256 columns.
 inline int fused_slices(int gamma, int H, int n_sm) {
-  int s = n_sm / gamma;
-  s = s > kFusedMaxSlices ? kFusedMaxSlices : s;
-  const int by_cols = H / 256 < 1 ? 1 : H / 256;
-  s = s > by_cols ? by_cols : s;
-  return s < 1 ? 1 : s;
+  int s = 1;
+  while (2 * s <= kFusedMaxSlices && 2 * s * gamma <= n_sm && H / (2 * s) >= 256) s *= 2;
+  return s;
 }
 
 struct FusedScratch {
-  double* dpart;      // [gamma][S][E] partial fp64 logits of the candidates (candidate order)
-  int32_t* tok_cnt;   // [max_tokens] arrivals per token; zero between calls
   int32_t* done_cnt;  // [1] finished tokens; zero between calls
 };
 
 // ---------------------------------------------------------------------------------------
 // Exclusive scan of NV integer sequences over the block.  Every thread holds ITEMS consecutive
 // entries of each (blocked layout: thread i owns entries i * ITEMS ..); on return v holds the
-// exclusive prefixes and tot the totals.  ws: NV * 33 ints of shared memory.  Two barriers.
+// exclusive prefixes and tot the totals.  ws: NV * 33 ints of shared memory.  Three barriers.
 template <int ITEMS, int NV>
 __device__ __forceinline__ void block_scan(int (&v)[NV][ITEMS], int (&tot)[NV], int32_t* ws) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
@@ -80,16 +81,25 @@ __device__ __forceinline__ void block_scan(int (&v)[NV][ITEMS], int (&tot)[NV], 
     for (int q = 0; q < NV; ++q) ws[q * 33 + warp] = inc[q];
   }
   __syncthreads();
+  if (warp == 0) {  // exclusive prefixes of the warp totals (at most 32 warps) and the grand totals, by one warp
+#pragma unroll
+    for (int q = 0; q < NV; ++q) {
+      const int wv = lane < nw ? ws[q * 33 + lane] : 0;
+      int sv = wv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, sv, o);
+        if (lane >= o) sv += x;
+      }
+      ws[q * 33 + lane] = sv - wv;
+      if (lane == 31) ws[q * 33 + 32] = sv;
+    }
+  }
+  __syncthreads();
 #pragma unroll
   for (int q = 0; q < NV; ++q) {
-    int before = 0, total = 0;
-    for (int w = 0; w < nw; ++w) {
-      const int x = ws[q * 33 + w];
-      before += w < warp ? x : 0;
-      total += x;
-    }
-    tot[q] = total;
-    before += inc[q] - own[q];
+    tot[q] = ws[q * 33 + 32];
+    const int before = ws[q * 33 + warp] + inc[q] - own[q];
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) v[q][i] += before;
   }
@@ -132,6 +142,7 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
   __syncthreads();
   MOEV_RF_MARK(17, true);
 
+  const int cap_log2 = 31 - __clz(unit_cap), cap_mask = unit_cap - 1;
   // ---- one scan over the experts: slots before e | active experts before e | units before e and packed counts
   // of remainder units per class, if remainders are placed behind the full runs | units before e otherwise
   int v[5][kGroupItems], tot[5], m[kGroupItems];
@@ -139,13 +150,13 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
   for (int i = 0; i < kGroupItems; ++i) {
     const int e = tid * kGroupItems + i;
     m[i] = e < E ? cnt[e] : 0;
-    const int rem = m[i] % unit_cap;
+    const int rem = m[i] & cap_mask;   // unit_cap is a power of two
     const int cls = rem >= 12 ? 0 : (rem >= 6 ? 1 : 2);
     v[0][i] = m[i];
     v[1][i] = m[i] > 0 ? 1 : 0;
-    v[2][i] = m[i] / unit_cap;
+    v[2][i] = m[i] >> cap_log2;
     v[3][i] = rem > 0 ? (1 << (10 * cls)) : 0;   // three 10-bit counters (at most 512 experts)
-    v[4][i] = (m[i] + unit_cap - 1) / unit_cap;
+    v[4][i] = (m[i] + cap_mask) >> cap_log2;
   }
   block_scan<kGroupItems, 5>(v, tot, scan_ws);
   MOEV_RF_MARK(18, true);
@@ -158,7 +169,7 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
   // runs of the routed experts in expert order, then (single-phase tensor-core schedules) the routed experts'
   // remainders in three classes of decreasing length (>= 12, >= 6, shorter), expert order inside each.
   const bool sorted = unit_cap <= 64 && !wide;
-  const int sh_each = (gamma + unit_cap - 1) / unit_cap, base = n_shared * sh_each;
+  const int sh_each = (gamma + cap_mask) >> cap_log2, base = n_shared * sh_each;
   const int total1 = sorted ? tot[2] : tot[4];
   const int n0 = sorted ? (tot[3] & 1023) : 0, n1 = sorted ? ((tot[3] >> 10) & 1023) : 0,
             n2 = sorted ? ((tot[3] >> 20) & 1023) : 0;
@@ -181,8 +192,8 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
     T.offsets[u] = slot0;
     if (O.union_ids) O.union_ids[u] = e;
     if (O.offsets) O.offsets[u] = slot0;
-    const int rem = sorted ? m[i] % unit_cap : 0;
-    const int nch = sorted ? m[i] / unit_cap : (m[i] + unit_cap - 1) / unit_cap;
+    const int rem = sorted ? (m[i] & cap_mask) : 0;
+    const int nch = sorted ? (m[i] >> cap_log2) : ((m[i] + cap_mask) >> cap_log2);
     const int first = base + (sorted ? v[2][i] : v[4][i]);
     for (int c = 0; c < nch; ++c) {
       Unit un;
@@ -247,33 +258,49 @@ __device__ __forceinline__ double warp_reduce_scatter16(double (&a)[16], int lan
   return a[0];
 }
 
+// float -> unsigned key with the same order (for redux.sync maxima)
+__device__ __forceinline__ uint32_t float_key(float f) {
+  const uint32_t b = __float_as_uint(f);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+constexpr int kFusedEpl = kMaxE / 32;  // experts per lane when one warp holds all logits
+
 template <int AFMT>
 __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
     Tables T, RouteOut O, FusedScratch F, const void* __restrict__ x, const float* __restrict__ router_w,
     const float* __restrict__ part, const float* __restrict__ part_x2, const float* __restrict__ part_w2max,
     float* __restrict__ y32, int gamma, int H, int E, int k, int n_slices, int ks, int score, float routed_scale,
     int n_shared, int unit_cap, int wide_ratio) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
   extern __shared__ __align__(16) int32_t dyn_sm[];  // route_group_block's tables (the last CTA only)
-  __shared__ double L[kMaxE];                        // exact logits of the candidates
+  __shared__ double L[kMaxE];                        // exact logits of the candidates (first CTA of the cluster)
+  __shared__ double dpart_s[kFusedMaxSlices][16];    // first CTA: the partial fp64 logits of every CTA of the cluster (one pass)
+  __shared__ __align__(16) float pv[kMaxE + 4];      // this CTA's partial fp32 logits | x2 | w2 | max |x|
   __shared__ float l32[kMaxE];
   __shared__ int32_t cand[kMaxE];
   __shared__ __align__(16) float psum[kFusedThreads * 4];
   __shared__ double red[kFusedWarps][16];
   __shared__ float redf[kFusedWarps], redw[kFusedWarps], reda[kFusedWarps];
-  __shared__ int wcnt_s[kFusedWarps];
-  __shared__ float kth_s;
-  __shared__ float top_v[kFusedWarps * kMaxTopK];
-  __shared__ int top_id[kFusedWarps * kMaxTopK];
+  __shared__ float bound_s[3];   // x2 | w2 | max |x| of the whole row
+  __shared__ int ncand_s;
   __shared__ int flag_s;
   __shared__ float sel_v_s[kMaxTopK];
   __shared__ int sel_e_s[kMaxTopK];
-  const int s = blockIdx.x, S = gridDim.x, t = blockIdx.y;
+  const int s = blockIdx.x, S = gridDim.x, t = blockIdx.y;   // cluster = the S CTAs of token t, rank = s
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // columns of this CTA's slice, in groups of four; slices are whole blocks of 128 columns (the 1 x 128
   // activation quantisation works on such blocks), so the last slices of a token may be empty
   const int g4_all = H / 4;
   const int g4_per = (((g4_all + S - 1) / S) + 31) & ~31;
   const int g4_lo = min(g4_all, s * g4_per), g4_hi = min(g4_all, g4_lo + g4_per);
+  // split-K slices of the router partials this CTA sums
+  const int sl_per = (n_slices + S - 1) / S;
+  const int sl_lo = min(n_slices, s * sl_per), sl_hi = min(n_slices, sl_lo + sl_per);
 
   asm volatile("griddepcontrol.wait;" ::: "memory");               // router partials are complete
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -284,34 +311,31 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
   for (int i = g4_lo + tid; i < g4_hi; i += kFusedThreads)
     reinterpret_cast<float4*>(y32 + (size_t)t * H)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
 
-  // ---- Loads of the first phase, all issued before any is used (one trip to the L2 instead of one per
-  // group of loads): the token's row (for max |x|: every CTA of the token needs the quantisation scale),
-  // the norms for the error bound, and the split-K partial logits.
-  float amax = 0.f;
-  uint2 xa[4];
-  float4 xf[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const int i = j * kFusedThreads + tid;
+  // ---- Loads of the first phase, all issued before any is used: this thread's first group of the slice of x
+  // (kept for the fp64 products), its share of the norms, and of the split-K partial logits.
+  uint2 xa = make_uint2(0u, 0u);
+  float4 xf = make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool has_x = g4_lo + tid < g4_hi;
+  if (has_x) {
     if constexpr (AFMT == MOEV_ACT_BF16)
-      xa[j] = i < g4_all ? __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + i)
-                         : make_uint2(0u, 0u);
+      xa = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + g4_lo + tid);
     else
-      xf[j] = i < g4_all ? __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + i)
-                         : make_float4(0.f, 0.f, 0.f, 0.f);
+      xf = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + g4_lo + tid);
   }
   const int n_et = (E + kRouterETile - 1) / kRouterETile;  // at most 8
-  float nx = 0.f, nw[8];
+  float x2 = 0.f, w2 = 0.f;
+  for (int c = sl_lo + tid; c < sl_hi; c += kFusedThreads) {
+    float nw[8];
+    const float nx = __ldg(part_x2 + (size_t)c * gamma + t);
 #pragma unroll
-  for (int j = 0; j < 8; ++j) nw[j] = 0.f;
-  if (tid < n_slices) {
-    nx = __ldg(part_x2 + (size_t)tid * gamma + t);
+    for (int j = 0; j < 8; ++j) nw[j] = j < n_et ? __ldg(part_w2max + (size_t)c * n_et + j) : 0.f;
+    float mx = 0.f;
 #pragma unroll
-    for (int j = 0; j < 8; ++j)
-      if (j < n_et) nw[j] = __ldg(part_w2max + (size_t)tid * n_et + j);
+    for (int j = 0; j < 8; ++j) mx = fmaxf(mx, nw[j]);
+    x2 += nx;
+    w2 += mx;
   }
-  // ---- fp32 logits of this token: the split-K partials summed over the slices in a fixed order
-  // (identical in every CTA of the token)
+  // ---- partial fp32 logits of this token over this CTA's split-K slices (fixed order)
   if ((E & 3) == 0 && E / 4 <= kFusedThreads) {
     const int nq = E / 4, G = kFusedThreads / nq;
     const int q = tid % nq, g = tid / nq;
@@ -319,63 +343,46 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
     float4 sacc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (g < G) {
       const float* pp = part + (size_t)t * E + 4 * q;
-      for (int c = g; c < n_slices; c += 16 * G) {  // sixteen 16-byte loads in flight per thread
-        float4 v[16];
+      for (int c = sl_lo + g; c < sl_hi; c += 8 * G) {  // eight 16-byte loads in flight per thread
+        float4 v[8];
 #pragma unroll
-        for (int i = 0; i < 16; ++i)
-          v[i] = (c + i * G < n_slices) ? __ldg(reinterpret_cast<const float4*>(pp + (size_t)(c + i * G) * cs))
-                                        : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < 8; ++i)
+          v[i] = (c + i * G < sl_hi) ? __ldg(reinterpret_cast<const float4*>(pp + (size_t)(c + i * G) * cs))
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) { sacc.x += v[i].x; sacc.y += v[i].y; sacc.z += v[i].z; sacc.w += v[i].w; }
+        for (int i = 0; i < 8; ++i) { sacc.x += v[i].x; sacc.y += v[i].y; sacc.z += v[i].z; sacc.w += v[i].w; }
       }
       *reinterpret_cast<float4*>(&psum[g * E + 4 * q]) = sacc;
     }
-    MOEV_RF_MARK(14, first_cta);
     __syncthreads();
-    MOEV_RF_MARK(15, first_cta);
     for (int e = tid; e < E; e += kFusedThreads) {
       float sum = 0.f;
       for (int gg = 0; gg < G; ++gg) sum += psum[gg * E + e];
-      l32[e] = sum;
+      pv[e] = sum;
     }
   } else {
     const size_t cs = (size_t)gamma * E;
     for (int e = tid; e < E; e += kFusedThreads) {
       const float* pp = part + (size_t)t * E + e;
       float sum = 0.f;
-      for (int c = 0; c < n_slices; c += 16) {
+      for (int c = sl_lo; c < sl_hi; c += 16) {
         float v[16];
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = (c + i < n_slices) ? __ldg(pp + (size_t)(c + i) * cs) : 0.f;
+        for (int i = 0; i < 16; ++i) v[i] = (c + i < sl_hi) ? __ldg(pp + (size_t)(c + i) * cs) : 0.f;
 #pragma unroll
         for (int i = 0; i < 16; ++i) sum += v[i];
       }
-      l32[e] = sum;
+      pv[e] = sum;
     }
   }
-  // ---- norms and max |x| (rows longer than 4 * kFusedThreads groups and more than kFusedThreads slices: the rest in loops)
-  float x2 = nx, w2 = 0.f;
-  {
-    float mx = 0.f;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) mx = fmaxf(mx, nw[j]);
-    w2 = mx;
-  }
-  for (int c = tid + kFusedThreads; c < n_slices; c += kFusedThreads) {
-    x2 += __ldg(part_x2 + (size_t)c * gamma + t);
-    float mx = 0.f;
-    for (int j = 0; j < n_et; ++j) mx = fmaxf(mx, __ldg(part_w2max + (size_t)c * n_et + j));
-    w2 += mx;
-  }
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    if constexpr (AFMT == MOEV_ACT_BF16)
-      amax = fmaxf(fmaxf(amax, fmaxf(fabsf(__uint_as_float(xa[j].x << 16)), fabsf(__uint_as_float(xa[j].x & 0xffff0000u)))),
-                   fmaxf(fabsf(__uint_as_float(xa[j].y << 16)), fabsf(__uint_as_float(xa[j].y & 0xffff0000u))));
-    else
-      amax = fmaxf(fmaxf(amax, fmaxf(fabsf(xf[j].x), fabsf(xf[j].y))), fmaxf(fabsf(xf[j].z), fabsf(xf[j].w)));
-  }
-  for (int i = 4 * kFusedThreads + tid; i < g4_all; i += kFusedThreads) {
+  // max |x| of the slice (further groups of a long slice are read again later)
+  float amax = 0.f;
+  if constexpr (AFMT == MOEV_ACT_BF16)
+    amax = fmaxf(fmaxf(fabsf(__uint_as_float(xa.x << 16)), fabsf(__uint_as_float(xa.x & 0xffff0000u))),
+                 fmaxf(fabsf(__uint_as_float(xa.y << 16)), fabsf(__uint_as_float(xa.y & 0xffff0000u))));
+  else
+    amax = fmaxf(fmaxf(fabsf(xf.x), fabsf(xf.y)), fmaxf(fabsf(xf.z), fabsf(xf.w)));
+  for (int i = g4_lo + tid + kFusedThreads; i < g4_hi; i += kFusedThreads) {
     if constexpr (AFMT == MOEV_ACT_BF16) {
       const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + i);
       amax = fmaxf(fmaxf(amax, fmaxf(fabsf(__uint_as_float(v.x << 16)), fabsf(__uint_as_float(v.x & 0xffff0000u)))),
@@ -390,15 +397,30 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
   x2 = warp_sum(x2);
   w2 = warp_sum(w2);
   if (lane == 0) { redf[warp] = x2; redw[warp] = w2; reda[warp] = amax; }
-  __syncthreads();  // l32, redf, redw, reda complete
+  __syncthreads();
+  if (tid == 0) {
+    float a = 0.f, b = 0.f, c = 0.f;
+    for (int w = 0; w < kFusedWarps; ++w) { a += redf[w]; b += redw[w]; c = fmaxf(c, reda[w]); }
+    pv[E] = a; pv[E + 1] = b; pv[E + 2] = c;
+  }
+  // ---- exchange through distributed shared memory: every CTA adds the S partial vectors in rank order
+  cluster.sync();
+  for (int e = tid; e < E + 3; e += kFusedThreads) {
+    float sum = 0.f;
+    for (int r = 0; r < S; ++r) {
+      const float v = *cluster.map_shared_rank(&pv[e], r);
+      sum = e == E + 2 ? fmaxf(sum, v) : sum + v;
+    }
+    if (e < E) l32[e] = sum; else bound_s[e - E] = sum;
+  }
+  __syncthreads();
   MOEV_RF_MARK(1, first_cta);
 
   // ---- the token's power-of-two activation scale, and this slice of the quantised activation operand of the
   // tensor-core FFN kernels (see topk_refine_kernel): x * 2^p_t as two e4m3 terms hi + lo / 16 (fp8 weights), as
   // four packed e2m1 terms with weights 8^-j (MXFP4 weights), or as e4m3 codes with 1 x 128 block scales
   auto quantise_slice = [&](int qt, int qn) {
-  float am = 0.f;
-  for (int w = 0; w < kFusedWarps; ++w) am = fmaxf(am, reda[w]);
+  const float am = bound_s[2];
   int ex = (am > 0.f && am < 3.0e38f) ? (int)((__float_as_uint(am) >> 23) & 0xffu) - 127 : 6;
   ex = ex < -100 ? -100 : (ex > 100 ? 100 : ex);
   if (s == 0 && qt == 0)
@@ -452,78 +474,59 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
     }
   }
   };
-  // ---- fp32 k-th largest logit (larger value, or equal value and lower id, precedes) in two levels: the k
-  // best of each warp's 32 experts, ranked inside the warp by counting over shuffled values, contain the k
-  // best overall; those entries are then ranked by counting, several threads per entry.  (One thread per
-  // expert counting over all E costs E iterations per thread: it was most of this kernel's instructions.)
-  {
-    const int n_pool = (E + 31) >> 5;  // warps that hold experts (E <= 512 = kFusedThreads)
-    const float v = tid < E ? l32[tid] : -INFINITY;
-    int rank = 0;
-    // the warps that hold no experts quantise the slice meanwhile (all warps, afterwards, when every warp holds some)
-    if (n_pool < kFusedWarps) {
-      if (warp >= n_pool) quantise_slice(tid - 32 * n_pool, kFusedThreads - 32 * n_pool);
+
+  // ---- warp 0: the fp32 k-th largest logit and the candidates, the whole row in its registers (lane l holds the
+  // experts l, l + 32, ...): k rounds of "take the maximum out" (one redux per round; of equal values one
+  // instance goes, so the k-th round's maximum is the k-th largest value), then every expert whose exact logit
+  // may reach the exact k-th largest (error bound as in topk_refine_kernel), in ascending id.  The other
+  // warps quantise the slice meanwhile.
+  if (warp == 0) {
+    uint32_t key[kFusedEpl], work[kFusedEpl];
+#pragma unroll
+    for (int j = 0; j < kFusedEpl; ++j) {
+      const int e = lane + 32 * j;
+      key[j] = e < E ? float_key(l32[e]) : 0u;   // 0 is below every real key
+      work[j] = key[j];
     }
-    if (warp < n_pool) {
-      const uint32_t below = (1u << lane) - 1u;  // lanes (= ids) that win ties against this one
-#pragma unroll 8
-      for (int l = 0; l < 32; ++l) {
-        const float u = __shfl_sync(0xffffffffu, v, l);
-        rank += (u > v || (u == v && ((below >> l) & 1u))) ? 1 : 0;
+    uint32_t kth_key = 0u;
+    for (int r = 0; r < k; ++r) {
+      uint32_t m = 0u;
+#pragma unroll
+      for (int j = 0; j < kFusedEpl; ++j) m = max(m, work[j]);
+      kth_key = __reduce_max_sync(0xffffffffu, m);
+      const uint32_t holders = __ballot_sync(0xffffffffu, m == kth_key);
+      if (lane == __ffs(holders) - 1) {  // one instance of the maximum leaves
+        bool done = false;
+#pragma unroll
+        for (int j = 0; j < kFusedEpl; ++j)
+          if (!done && work[j] == kth_key) { work[j] = 0u; done = true; }
       }
     }
-    const int M = n_pool * k;  // <= 512
-    for (int i = tid; i < M; i += kFusedThreads) { top_v[i] = -INFINITY; top_id[i] = 0x7fffffff; }
-    __syncthreads();
-    if (tid < E && rank < k) { top_v[warp * k + rank] = v; top_id[warp * k + rank] = tid; }
-    if (n_pool >= kFusedWarps) quantise_slice(tid, kFusedThreads);
-    __syncthreads();
-    MOEV_RF_MARK(16, first_cta);
-    int TT = 1;
-    while (2 * TT * M <= kFusedThreads && TT < 32) TT <<= 1;  // threads per entry
-    const int i = tid / TT, sub = tid & (TT - 1), per = (M + TT - 1) / TT;
-    int r = 0;
-    float vi = 0.f;
-    if (i < M) {
-      vi = top_v[i];
-      const int idi = top_id[i];
-      const int j1 = min(M, (sub + 1) * per);
-      for (int j = sub * per; j < j1; ++j) {
-        const float u = top_v[j];
-        r += (u > vi || (u == vi && top_id[j] < idi)) ? 1 : 0;
-      }
+    const float n_round = (float)(ks + n_slices + 4);
+    const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(bound_s[0]) * sqrtf(bound_s[1]) + 1e-30f;
+    const float thr = key_float(kth_key) - 2.f * eps;
+    int n = 0;
+#pragma unroll
+    for (int j = 0; j < kFusedEpl; ++j) {
+      const int e = lane + 32 * j;
+      const bool in = e < E && key_float(key[j]) >= thr;
+      const uint32_t mk = __ballot_sync(0xffffffffu, in);
+      if (in) cand[n + __popc(mk & ((1u << lane) - 1u))] = e;
+      n += __popc(mk);
     }
-    for (int o = TT >> 1; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
-    if (i < M && sub == 0 && r == k - 1) kth_s = vi;
+    if (lane == 0) ncand_s = n;
+  } else {
+    quantise_slice(tid - 32, kFusedThreads - 32);
   }
   __syncthreads();
-  MOEV_RF_MARK(2, first_cta);
-  // ---- candidates: every expert whose exact logit may reach the exact k-th largest, ascending id
-  // (error bound as in topk_refine_kernel)
-  int ncand = 0;
-  {
-    float xs = 0.f, wm = 0.f;
-    for (int w = 0; w < kFusedWarps; ++w) { xs += redf[w]; wm += redw[w]; }
-    const float n_round = (float)(ks + n_slices + 4);
-    const float eps = 1.25f * n_round * 5.9604645e-8f * sqrtf(xs) * sqrtf(wm) + 1e-30f;
-    const float thr = kth_s - 2.f * eps;
-    const bool in = tid < E && l32[tid] >= thr;  // E <= kFusedThreads
-    const uint32_t mk = __ballot_sync(0xffffffffu, in);
-    if (lane == 0) wcnt_s[warp] = __popc(mk);
-    __syncthreads();
-    int before = 0;
-    for (int w = 0; w < kFusedWarps; ++w) { const int cw = wcnt_s[w]; before += w < warp ? cw : 0; ncand += cw; }
-    if (in) cand[before + __popc(mk & ((1u << lane) - 1u))] = tid;
-    __syncthreads();
-  }
+  const int ncand = ncand_s;
   MOEV_RF_MARK(3, first_cta);
-
-  MOEV_RF_MARK(4, first_cta);
 
   // ---- exact (fp64) partial logits of the candidates over this CTA's slice of H, kFusedCand candidates per pass.
   // Only the warps that own columns of the slice take part; conversions to fp64 are integer operations and
   // the warp sums use the entry-halving butterfly: the fp64 pipe is narrow, its instructions are the cost.
-  double* dp = F.dpart + ((size_t)t * S + s) * E;
+  // The sums go to the first CTA of the cluster.
+  double* dp = cluster.map_shared_rank(&dpart_s[s][0], 0);
   const int n_act = min(kFusedWarps, (g4_hi - g4_lo + 31) >> 5);  // warps with columns in the first trip
   for (int c0 = 0; c0 < ncand; c0 += kFusedCand) {
     const int nc = min(kFusedCand, ncand - c0);
@@ -534,7 +537,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
       for (int h4 = g4_lo + tid; h4 < g4_hi; h4 += kFusedThreads) {
         double xv[4];
         if constexpr (AFMT == MOEV_ACT_BF16) {
-          const uint2 v = __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + h4);
+          const uint2 v = h4 == g4_lo + tid ? xa
+                          : __ldg(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(x) + (size_t)t * H) + h4);
           const uint32_t wd[2] = {v.x, v.y};
 #pragma unroll
           for (int i = 0; i < 2; ++i) {
@@ -542,7 +546,8 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
             xv[2 * i + 1] = bf16_bits_to_double(wd[i] >> 16);
           }
         } else {
-          const float4 f = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + h4);
+          const float4 f = h4 == g4_lo + tid ? xf
+                           : __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + h4);
           xv[0] = f32_to_double_int(f.x); xv[1] = f32_to_double_int(f.y);
           xv[2] = f32_to_double_int(f.z); xv[3] = f32_to_double_int(f.w);
         }
@@ -573,66 +578,52 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
     if (tid < nc) {
       double a = 0.0;
       for (int w = 0; w < n_act; ++w) a += red[w][tid];
-      dp[c0 + tid] = a;
+      dp[tid] = a;   // remote store (own shared memory for the first CTA)
     }
-    __syncthreads();
+    // the pass's partial sums of all CTAs of the cluster are in the first CTA's shared memory: it adds them in
+    // rank order; a further pass (more than kFusedCand candidates: rare) reuses the buffer after a second barrier
+    cluster.sync();
+    if (s == 0 && tid < nc) {
+      double a = 0.0;
+      for (int r = 0; r < S; ++r) a += dpart_s[r][tid];
+      L[c0 + tid] = a;
+    }
+    if (c0 + kFusedCand < ncand) cluster.sync();
   }
-
   MOEV_RF_MARK(5, first_cta);
-  // ---- hand-over: the CTA of this token that arrives last continues
-  __threadfence();
+  if (s != 0) return;   // the other CTAs of the cluster are done
   __syncthreads();
-  MOEV_RF_MARK(6, first_cta);
-  if (tid == 0) flag_s = (atomicAdd(F.tok_cnt + t, 1) == S - 1) ? 1 : 0;
-  __syncthreads();
-  if (!flag_s) return;
-  __threadfence();
   MOEV_RF_MARK(7, t == 0);
 
-  // ---- exact logits: the S partial sums of a candidate are fetched by S adjacent lanes (all loads in flight at
-  // once; a loop over the slices would pay one trip to the L2 per slice) and added by a shuffle tree, whose
-  // order is fixed
-  {
-    int P = 1;
-    while (P < S) P <<= 1;  // lanes per candidate (S <= kFusedMaxSlices = 16)
-    const int sub = tid & (P - 1), per_pass = kFusedThreads / P;
-    for (int c0 = 0; c0 < ncand; c0 += per_pass) {
-      const int c = c0 + tid / P;
-      double a = (c < ncand && sub < S) ? __ldcg(F.dpart + ((size_t)t * S + sub) * E + c) : 0.0;
-      for (int o = P >> 1; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-      if (c < ncand && sub == 0) L[c] = a;
-    }
-  }
-  __syncthreads();
-  MOEV_RF_MARK(8, t == 0);
-  // ---- exact ranking by counting (candidates are stored in ascending id)
-  for (int c = tid; c < ncand; c += kFusedThreads) {
-    const double v = L[c];
-    int rank = 0;
-    for (int c2 = 0; c2 < ncand; ++c2) {
-      const double u = L[c2];
-      rank += (u > v || (u == v && c2 < c)) ? 1 : 0;
-    }
-    if (rank < k) { sel_v_s[rank] = (float)v; sel_e_s[rank] = cand[c]; }  // weights from the exact logits rounded to binary32
-  }
-  __syncthreads();
-  MOEV_RF_MARK(13, t == 0);
-
-  // ---- router weights of the k selected experts (warp 0, lane j owns the j-th), in binary32: the exact logits
-  // rounded once (2^-24 relative) leave the weights far inside the 1e-5 they are compared to
+  // ---- warp 0 of the first CTA: exact ranking by counting (candidates are stored in ascending id), router weights
   if (warp == 0) {
+    for (int c = lane; c < ncand; c += 32) {
+      const double v = L[c];
+      int rank = 0;
+      for (int c2 = 0; c2 < ncand; ++c2) {
+        const double u = L[c2];
+        rank += (u > v || (u == v && c2 < c)) ? 1 : 0;
+      }
+      if (rank < k) { sel_v_s[rank] = (float)v; sel_e_s[rank] = cand[c]; }  // weights from the exact logits rounded to binary32
+    }
+    __syncwarp();
+    MOEV_RF_MARK(13, t == 0);
+    // router weights of the k selected experts (lane j owns the j-th), in binary32: the exact logits rounded once
+    // (2^-24 relative) leave the weights far inside the 1e-5 they are compared to
     const float sel_v = lane < k ? sel_v_s[lane] : 0.f;
     const int sel_e = lane < k ? sel_e_s[lane] : -1;
     float wgt = 0.f;
+    // (hardware exponential and division: a few units in the last place at these arguments, |logit| < ~30; one
+    // warp's chain of dependent instructions is this step's whole cost)
     if (score == MOEV_SCORE_SOFTMAX) {
       const float mx = sel_v_s[0];
-      const float exv = lane < k ? expf(sel_v - mx) : 0.f;
+      const float exv = lane < k ? __expf(sel_v - mx) : 0.f;
       const float den = warp_sum(exv);
-      wgt = exv / den;
+      wgt = __fdividef(exv, den);
     } else {
-      const float sg = lane < k ? 1.f / (1.f + expf(-sel_v)) : 0.f;
+      const float sg = lane < k ? __fdividef(1.f, 1.f + __expf(-sel_v)) : 0.f;
       const float den = warp_sum(sg);
-      wgt = routed_scale * sg / (den + 1e-20f);
+      wgt = __fdividef(routed_scale * sg, den + 1e-20f);
     }
     MOEV_RF_MARK(21, t == 0);
     if (lane < k) {
@@ -642,14 +633,12 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
       if (O.topk_ids) O.topk_ids[a] = sel_e;
       if (O.topk_w) O.topk_w[a] = wgt;
     }
+    MOEV_RF_MARK(9, t == 0);
+    // ---- hand-over: the CTA that finishes the last token builds the grouping tables
+    __threadfence();
+    MOEV_RF_MARK(10, t == 0);
+    if (lane == 0) flag_s = (atomicAdd(F.done_cnt, 1) == gamma - 1) ? 1 : 0;
   }
-
-  MOEV_RF_MARK(9, t == 0);
-  // ---- hand-over: the CTA that finishes the last token builds the grouping tables
-  __threadfence();
-  __syncthreads();
-  MOEV_RF_MARK(10, t == 0);
-  if (tid == 0) flag_s = (atomicAdd(F.done_cnt, 1) == gamma - 1) ? 1 : 0;
   __syncthreads();
   if (!flag_s) return;
   __threadfence();
@@ -657,9 +646,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) route_refine_kernel(
   route_group_block(T, O, gamma, E, k, n_shared, unit_cap, wide_ratio, dyn_sm);
   __syncthreads();
   MOEV_RF_MARK(12, true);
-  // every CTA has arrived on every counter: clear them for the next call
-  for (int i = tid; i < gamma; i += kFusedThreads) F.tok_cnt[i] = 0;
-  if (tid == 0) *F.done_cnt = 0;
+  if (tid == 0) *F.done_cnt = 0;  // every token has arrived: clear the counter for the next call
 }
 
 }  // namespace moev

@@ -88,7 +88,6 @@ __device__ __forceinline__ void prefetch_expert_weights(const PrefetchArgs& P, i
 }
 
 #ifdef MOEV_TC_STATS
-__device__ long long g_rt_stats[32];  // debug builds: phase timestamps of the routing kernels (CTA 0)
 #define MOEV_RT_MARK(i) do { __syncthreads(); if (blockIdx.x == 0 && threadIdx.x == 0) g_rt_stats[i] = clock64(); } while (0)
 #else
 #define MOEV_RT_MARK(i)
