@@ -339,11 +339,13 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #endif
       // Task ids are published one task ahead of the loads, so the other roles can prepare
       // their tables (and the first activation tiles) while this task still streams.
+      bool first_draw = true;
       auto fetch_publish = [&](TaskDesc& td) -> int {
         int id;
         td.unit = 0; td.slice = 0; td.valid = false;
         do {
-          id = atomicAdd(P.task_counter, 1);
+          id = first_draw ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(P.task_counter, 1);  // the first draw needs no trip to the counter
+          first_draw = false;
           if (id >= n_ids) { id = -1; break; }
           td = decode_task(id, n_units, n_slices);
         } while (!td.valid);

@@ -261,8 +261,10 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       ptx::prefetch_tmap(&tm_xq); ptx::prefetch_tmap(&tm_hq);
       uint32_t it = 0, q = 0;
       bool ok = true;
+      bool first_draw = true;
       auto fetch_publish = [&]() -> int {
-        int id = atomicAdd(P.task_counter, 1);
+        int id = first_draw ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(P.task_counter, 1);  // the first draw needs no trip to the counter
+        first_draw = false;
         if (id >= n_ids) id = -1;
         if (id < 0 && MOEV_TEST_WITHHOLD()) return -1;  // test builds: the final message is withheld
         const int slot = q % kTaskQ;

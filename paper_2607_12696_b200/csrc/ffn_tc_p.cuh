@@ -129,12 +129,14 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
     }
     uint32_t it = 0, q = 0;
     bool ok = true;
+    bool first_draw = true;
     auto fetch_publish = [&](TaskDesc& td) -> int {
       int id = -2, unit = 0, slice = 0;
       if (lane == 0) {
         td.unit = 0; td.slice = 0; td.valid = false;
         do {
-          id = atomicAdd(P.task_counter, 1);
+          id = first_draw ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(P.task_counter, 1);  // the first draw needs no trip to the counter
+          first_draw = false;
           if (id >= n_ids) { id = -1; break; }
           td = decode_task(id, n_units, n_slices);
         } while (!td.valid);

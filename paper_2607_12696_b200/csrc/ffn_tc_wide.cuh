@@ -205,10 +205,12 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
     }
     uint32_t it = 0, q = 0;
     bool ok = true;
+    bool first_draw = true;
     auto fetch_publish = [&]() -> int {  // lane 0 draws and publishes; every lane learns the id
       int id = -2;
       if (lane == 0) {
-        id = atomicAdd(P.task_counter, 1);
+        id = first_draw ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(P.task_counter, 1);  // the first draw needs no trip to the counter
+        first_draw = false;
         if (id >= n_ids) id = -1;
         const int slot = q % kTaskQ;
         if (id < 0 && MOEV_TEST_WITHHOLD()) {
