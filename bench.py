@@ -676,6 +676,33 @@ def run_select_demo(args):
     v.close()
 
 
+def run_select_bench(args):
+    """Timing of the draft-selection kernels alone (Algorithm 1): the single-CTA kernel (255-node
+    tree, one layer's expert bitmaps) and the cooperative multi-CTA kernel (the same tree with
+    bitmaps over a whole model's 58 layers x 256 experts).  Prints one JSON line."""
+    import paper_2607_12696_b200 as moev
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    out = {"bench": "draft selection kernels", "gamma": 64}
+    for label, n_layers in (("single_cta_1_layer", 1), ("grid_58_layers", 58)):
+        parent, P, pred = synth.make_draft_tree(n_layers, 256, 8, depth=7, branch=2, seed_tag="select-bench")
+        tp, tP = torch.from_numpy(parent).to(dev), torch.from_numpy(P).to(dev)
+        tpred = torch.from_numpy(pred.view(np.int32)).to(dev)
+        o = None
+        for _ in range(max(3, args.warmup)):
+            o = moev.select_drafts(tp, tP, tpred, 64, 1e-6, out=o)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_calls = max(3, min(args.steps, 50))
+        e0.record()
+        for _ in range(n_calls):
+            o = moev.select_drafts(tp, tP, tpred, 64, 1e-6, out=o)
+        e1.record()
+        torch.cuda.synchronize()
+        out[label] = {"nodes": int(len(parent)), "bitmap_words": int(pred.shape[1]),
+                      "us_per_call": e0.elapsed_time(e1) * 1e3 / n_calls, "n_selected": int(o[3].item())}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -696,6 +723,7 @@ def main():
     ap.add_argument("--config-steps", type=int, default=50, help="timed calls per entry of the configs array")
     ap.add_argument("--select-demo", action="store_true",
                     help="cost-aware vs acceptance-only draft selection in front of the verification layer")
+    ap.add_argument("--select-bench", action="store_true", help="time the draft-selection kernels alone")
     ap.add_argument("--p-reuse", type=float, default=0.7, help="expert locality along a tree path (select demo)")
     args = ap.parse_args()
     global ACT_QUANT
@@ -710,6 +738,8 @@ def main():
             run_sweep(args)
         elif args.select_demo:
             run_select_demo(args)
+        elif args.select_bench:
+            run_select_bench(args)
         else:
             run_ours(args)
 
