@@ -205,8 +205,8 @@ size_t moev_expert_bytes(const moev_config* cfg);
 size_t moev_expert_code_bytes(const moev_config* cfg);
 
 /* Number of kernels one moev_verify call launches on this context (for launch accounting; calls
- * of at most 128 tokens with plain top-k routing take two routing launches, others three -- a
- * context whose max_tokens exceeds 128 reports the larger figure), and which FFN implementation
+ * of at most 32 tokens with plain top-k routing take two routing launches, others three -- a
+ * context whose max_tokens exceeds 32 reports the larger figure), and which FFN implementation
  * it resolved to (a moev_impl value, never AUTO). */
 int32_t moev_launches_per_call(const moev_ctx* ctx);
 int32_t moev_resolved_impl(const moev_ctx* ctx);

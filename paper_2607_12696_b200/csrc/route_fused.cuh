@@ -19,7 +19,7 @@
 //
 // The results are those of topk_refine_kernel + route_group_kernel: the same candidates, the
 // same fp64 ranking rule, the same tables.  Group-limited routing (two dependent candidate
-// stages) and calls of more than kFusedMaxTokens rows keep the three-kernel path.
+// stages) and calls of more than kFusedMaxTokens = 32 rows keep the three-kernel path.
 #pragma once
 #include <cooperative_groups.h>
 
@@ -36,7 +36,10 @@ namespace moev {
 
 constexpr int kFusedThreads = 512;
 constexpr int kFusedWarps = kFusedThreads / 32;
-constexpr int kFusedMaxTokens = 128;   // rows per call served by this path
+// Rows per call served by this path.  Measured against the three-kernel path (whole call, dependent launches on):
+// gamma = 8: -8 us, gamma = 32: equal, gamma = 64: +5 to +8 us (one CTA per token without hand-overs wins once
+// the tokens alone fill the machine).
+constexpr int kFusedMaxTokens = 32;
 constexpr int kFusedMaxSlices = 8;     // CTAs per token = cluster size (the portable maximum)
 constexpr int kFusedCand = 12;         // candidates evaluated per pass over the slice
 
