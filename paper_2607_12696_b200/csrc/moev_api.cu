@@ -141,9 +141,7 @@ cudaError_t dmalloc(T** p, size_t count) {
 constexpr int kWideRatio = 8;
 // dynamic shared memory of topk_refine_kernel: three double, three 32-bit and one 8-bit array of E entries
 size_t refine_smem_bytes(int E) { return ((size_t)E * 41 + 15) & ~size_t(15); }
-size_t route_smem(const moev_config& c, int gamma) {
-  return (size_t)(3 * c.E + 2 * gamma * c.top_k) * 4 + route_bitmap_bytes(c.E, gamma);
-}
+size_t route_smem(const moev_config& c, int gamma) { return route_group_block_smem(c.E, gamma, c.top_k); }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -530,7 +528,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
                                     (int)router_partial_smem(kRouterMaxKS)) == cudaSuccess;
     ok = ok && cudaFuncSetAttribute(router_partial_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)router_partial_smem(kRouterMaxKS)) == cudaSuccess;
-    if (gs > 48 * 1024)
+    if (gs > 40 * 1024)
       ok = ok && cudaFuncSetAttribute(route_group_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)gs) == cudaSuccess;
     if (cfg->n_group == 0) {  // its static tables exceed the default limit already
@@ -696,8 +694,8 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
       if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_BF16, true>); else go(topk_refine_kernel<MOEV_ACT_BF16, false>);
     }
     if (ev) cudaEventRecord(ev[2], st);
-    launch_k(route_group_kernel, dim3(1), dim3(1024), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E, g.top_k,
-             g.n_shared, c->unit_cap, wide_ratio);
+    launch_k(route_group_kernel, dim3(1), dim3(kGroupThreads), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E,
+             g.top_k, g.n_shared, c->unit_cap, wide_ratio);
   }
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {

@@ -164,13 +164,21 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
   block_scan<kGroupItems, 5>(v, tot, scan_ws);
   MOEV_RF_MARK(18, true);
   const int U = tot[1];
-  // many tokens per streamed expert: the two-phase FFN schedule (see route_group_kernel)
+  // many tokens per streamed expert: the two-phase FFN schedule (measured switch-over: above 8 assignments per
+  // streamed expert for small unions, where the weight stream is short, above 12 for large ones, where the
+  // two-phase schedule's re-streaming per 32-token unit costs more)
   const int ut = U + n_shared;
   const bool wide = T.wide != nullptr && wide_ratio > 0 &&
                     (A + n_shared * gamma) > (ut < 100 ? wide_ratio : wide_ratio + wide_ratio / 2) * ut;
-  // Units: every expert's slots cut into runs of at most unit_cap.  Order: the shared experts' units, the full
-  // runs of the routed experts in expert order, then (single-phase tensor-core schedules) the routed experts'
-  // remainders in three classes of decreasing length (>= 12, >= 6, shorter), expert order inside each.
+  // Units: every expert's slots cut into runs of at most unit_cap.  Order: the shared experts' units (they see
+  // every token, so their tasks are the longest), the full runs of the routed experts in expert order, then
+  // (single-phase tensor-core schedules) the routed experts' remainders in three classes of decreasing length
+  // (>= 12, >= 6, shorter), expert order inside each.  A task's cost grows with its unit's tokens (one global
+  // reduction per token and output row in the down phase) and tasks are handed out in unit order: the cheap ones
+  // last keeps the CTAs' finishing times close together (clustered tree workload: FFN kernel 920 -> 895 us),
+  // while expert order inside a class keeps concurrently running tasks on neighbouring experts.  The two-phase
+  // schedule wants an expert's units next to each other (they re-read its weights through the L2), and the
+  // CUDA-core path has no cap and no use for units.
   const bool sorted = unit_cap <= 64 && !wide;
   const int sh_each = (gamma + cap_mask) >> cap_log2, base = n_shared * sh_each;
   const int total1 = sorted ? tot[2] : tot[4];
@@ -240,25 +248,15 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
   }
 }
 
-// ---------------------------------------------------------------------------------------
-// Sums of 16 per-lane doubles over the warp by a butterfly that halves the number of entries a lane
-// holds at every step (16 additions per lane instead of 5 per entry): on return lane l holds the
-// warp-wide sum of entry q, both lanes of a pair (l, l ^ 1) the same one.  The order of the additions
-// is fixed.  fp64 additions are the scarce resource here (the fp64 pipe is narrow).
-__device__ __forceinline__ double warp_reduce_scatter16(double (&a)[16], int lane, int& q) {
-#pragma unroll
-  for (int n = 8, o = 16; n >= 1; n >>= 1, o >>= 1) {
-    const bool up = (lane & o) != 0;
-#pragma unroll
-    for (int i = 0; i < n; ++i) {
-      const double send = up ? a[i] : a[i + n];
-      const double keep = up ? a[i + n] : a[i];
-      a[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-    }
-  }
-  a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
-  q = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-  return a[0];
+// The grouping step as a kernel of its own (one CTA), for the three-kernel routing path.
+// Dynamic shared memory: route_group_block_smem(E, gamma, k).
+constexpr int kGroupThreads = 512;
+__global__ void __launch_bounds__(kGroupThreads) route_group_kernel(Tables T, RouteOut O, int gamma, int E, int k,
+                                                                    int n_shared, int unit_cap, int wide_ratio) {
+  extern __shared__ __align__(16) int32_t group_sm[];
+  asm volatile("griddepcontrol.wait;" ::: "memory");               // top-k tables are complete
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  route_group_block(T, O, gamma, E, k, n_shared, unit_cap, wide_ratio, group_sm);
 }
 
 // float -> unsigned key with the same order (for redux.sync maxima)

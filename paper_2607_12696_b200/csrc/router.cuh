@@ -6,8 +6,8 @@
 //                             bound, re-evaluates exactly those logits in fp64 and ranks them
 //                             (larger logit first, exact ties to the lower id), then the router
 //                             weights in fp64;
-//   3. route_group_kernel     one CTA: expert union (Eq. 1), per-expert histogram, offsets,
-//                             stable token->expert permutation, FFN work units.
+//   3. route_group_kernel     (route_fused.cuh) one CTA: expert union (Eq. 1), per-expert histogram,
+//                             offsets, stable token->expert permutation, FFN work units.
 // The selected ids therefore equal the ids an all-fp64 evaluation selects whenever the fp64
 // decision margin exceeds the fp64 rounding error (~1e-12); integer tables are exact.
 #pragma once
@@ -487,6 +487,26 @@ __global__ void __launch_bounds__(128) router_partial_small_kernel(const uint16_
   if (!wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");  // see router_partial_kernel
 }
 
+// Sums of 16 per-lane doubles over the warp by a butterfly that halves the number of entries a lane
+// holds at every step (16 additions per lane instead of 5 per entry): on return lane l holds the
+// warp-wide sum of entry q, both lanes of a pair (l, l ^ 1) the same one.  The order of the additions
+// is fixed.  fp64 additions are the scarce resource here (the fp64 pipe is narrow).
+__device__ __forceinline__ double warp_reduce_scatter16(double (&a)[16], int lane, int& q) {
+#pragma unroll
+  for (int n = 8, o = 16; n >= 1; n >>= 1, o >>= 1) {
+    const bool up = (lane & o) != 0;
+#pragma unroll
+    for (int i = 0; i < n; ++i) {
+      const double send = up ? a[i] : a[i + n];
+      const double keep = up ? a[i + n] : a[i];
+      a[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+    }
+  }
+  a[0] += __shfl_xor_sync(0xffffffffu, a[0], 1);
+  q = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+  return a[0];
+}
+
 struct RouteOut {  // optional caller-visible copies (may be null)
   int32_t* topk_ids;
   float* topk_w;
@@ -685,9 +705,9 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   float amax = 0.f;
   auto refine_range = [&](int cb, int ce) {
   for (int c0 = cb; c0 < ce; c0 += kRefineCand) {
-    double acc[kRefineCand];
+    double acc[16];  // kRefineCand used; 16 for the entry-halving warp reduction
 #pragma unroll
-    for (int q = 0; q < kRefineCand; ++q) acc[q] = 0.0;
+    for (int q = 0; q < 16; ++q) acc[q] = 0.0;
     const int nc = min(kRefineCand, ce - c0);
     for (int h4 = tid; h4 < H / 4; h4 += kRefineThreads) {
       double xv[4];
@@ -702,11 +722,13 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
         }
       } else {
         float4 f = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(x) + (size_t)t * H) + h4);
-        xv[0] = (double)f.x; xv[1] = (double)f.y; xv[2] = (double)f.z; xv[3] = (double)f.w;
+        xv[0] = f32_to_double_int(f.x); xv[1] = f32_to_double_int(f.y);
+        xv[2] = f32_to_double_int(f.z); xv[3] = f32_to_double_int(f.w);
         if (c0 == 0) amax = fmaxf(amax, fmaxf(fmaxf(fabsf(f.x), fabsf(f.y)), fmaxf(fabsf(f.z), fabsf(f.w))));
       }
       // pairs of candidates under a CTA-uniform test: bodies past nc are skipped, not predicated
-      // (top-4 routing refines five or six candidates per token, top-8 about ten)
+      // (top-4 routing refines five or six candidates per token, top-8 about ten); the conversions
+      // to fp64 are integer operations (the fp64 pipe is narrow: its instructions are the cost)
       float4 wv[kRefineCand];
 #pragma unroll
       for (int q0 = 0; q0 < kRefineCand; q0 += 2)
@@ -721,21 +743,16 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
 #pragma unroll
           for (int q = q0; q < q0 + 2; ++q)
             if (q < nc) {
-              acc[q] = fma(xv[0], (double)wv[q].x, acc[q]); acc[q] = fma(xv[1], (double)wv[q].y, acc[q]);
-              acc[q] = fma(xv[2], (double)wv[q].z, acc[q]); acc[q] = fma(xv[3], (double)wv[q].w, acc[q]);
+              acc[q] = fma(xv[0], f32_to_double_int(wv[q].x), acc[q]); acc[q] = fma(xv[1], f32_to_double_int(wv[q].y), acc[q]);
+              acc[q] = fma(xv[2], f32_to_double_int(wv[q].z), acc[q]); acc[q] = fma(xv[3], f32_to_double_int(wv[q].w), acc[q]);
             }
         }
     }
-#pragma unroll
-    for (int q0 = 0; q0 < kRefineCand; q0 += 2)
-      if (q0 < nc) {
-#pragma unroll
-        for (int q = q0; q < q0 + 2; ++q)
-          if (q < nc) {
-            double a = warp_sum(acc[q]);
-            if (lane == 0) red[warp][q] = a;
-          }
-      }
+    {  // warp sums by the entry-halving butterfly (16 fp64 additions per lane instead of 5 per candidate)
+      int q;
+      const double a = warp_reduce_scatter16(acc, lane, q);
+      if ((lane & 1) == 0 && q < kRefineCand) red[warp][q] = a;
+    }
     __syncthreads();
     if (tid < nc) {
       double a = 0.0;
@@ -901,18 +918,20 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
 #ifdef MOEV_TC_STATS
     if (blockIdx.x == 0 && tid == 0) g_rt_stats[20] = clock64();
 #endif
-    const double sel_v = lane < k ? sel_v_s[lane] : 0.0;
+    // binary32 from the exact logits rounded once (2^-24 relative), hardware exponential and division (a few
+    // units in the last place at these arguments): far inside the 1e-5 the weights are compared to
+    const float sel_v = lane < k ? (float)sel_v_s[lane] : 0.f;
     const int sel_e = lane < k ? sel_e_s[lane] : -1;
     float wgt = 0.f;
     if (score == MOEV_SCORE_SOFTMAX) {
-      const double mx = sel_v_s[0];
-      const float ex = lane < k ? expf((float)(sel_v - mx)) : 0.f;
+      const float mx = (float)sel_v_s[0];
+      const float ex = lane < k ? __expf(sel_v - mx) : 0.f;
       const float den = warp_sum(ex);
-      wgt = ex / den;
+      wgt = __fdividef(ex, den);
     } else {
-      const float sg = lane < k ? 1.f / (1.f + expf((float)(-sel_v))) : 0.f;
+      const float sg = lane < k ? __fdividef(1.f, 1.f + __expf(-sel_v)) : 0.f;
       const float den = warp_sum(sg);
-      wgt = routed_scale * sg / (den + 1e-20f);
+      wgt = __fdividef(routed_scale * sg, den + 1e-20f);
     }
 #ifdef MOEV_TC_STATS
     if (blockIdx.x == 0 && tid == 0) g_rt_stats[21] = clock64();
@@ -931,178 +950,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
   MOEV_RT_MARK(6);
 }
 
-// One CTA (1024 threads): per-expert histogram of the selected ids, block scan over the E
-// counts (ascending union and offsets), FFN work units, then the stable permutation from
-// per-expert token bitmaps.
-// Dynamic shared memory: cnt[E] | excl[E] | uidx[E] | ids[A] | w[A] | token bitmaps [E][ceil(gamma/32)]
-// (at most 64 KB of bitmaps: E <= 512, gamma <= 1024).
+// Bytes of the per-expert token bitmaps of the grouping step (at most 64 KB: E <= 512, gamma <= 1024).
 inline size_t route_bitmap_bytes(int E, int gamma) { return (size_t)E * ((gamma + 31) / 32) * 4; }
-__global__ void __launch_bounds__(1024) route_group_kernel(Tables T, RouteOut O, int gamma, int E,
-                                                           int k, int n_shared, int unit_cap, int wide_ratio) {
-  extern __shared__ int32_t sm[];
-  const int A = gamma * k;
-  int32_t* cnt = sm;
-  int32_t* excl = sm + E;
-  int32_t* uidx = sm + 2 * E;
-  int32_t* ids_s = sm + 3 * E;
-  float* w_s = reinterpret_cast<float*>(sm + 3 * E + A);
-  __shared__ int32_t warp_tot_cnt[32], warp_tot_flag[32], warp_tot_unit[32], n_union_s;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  asm volatile("griddepcontrol.wait;" ::: "memory");               // top-k tables are complete
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-  MOEV_RT_MARK(8);
-  for (int e = tid; e < E; e += blockDim.x) cnt[e] = 0;
-  __syncthreads();
-  for (int a = tid; a < A; a += blockDim.x) {
-    int e = T.topk_ids[a];
-    ids_s[a] = e;
-    w_s[a] = T.topk_w[a];
-    atomicAdd(&cnt[e], 1);
-  }
-  __syncthreads();
-
-  MOEV_RT_MARK(9);
-  // ---- phase 2: exclusive scans over experts (E <= 512 <= blockDim)
-  {
-    int c = tid < E ? cnt[tid] : 0, f = c > 0 ? 1 : 0;
-    int sc = c, sf = f;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int a = __shfl_up_sync(0xffffffffu, sc, o), b = __shfl_up_sync(0xffffffffu, sf, o);
-      if (lane >= o) { sc += a; sf += b; }
-    }
-    if (lane == 31) { warp_tot_cnt[warp] = sc; warp_tot_flag[warp] = sf; }
-    __syncthreads();
-    int bc = 0, bf = 0;
-    for (int w = 0; w < warp; ++w) { bc += warp_tot_cnt[w]; bf += warp_tot_flag[w]; }
-    if (tid < E) {
-      excl[tid] = bc + sc - c;
-      uidx[tid] = bf + sf - f;
-      if (f) {
-        int u = bf + sf - f;
-        T.union_ids[u] = tid;
-        T.offsets[u] = bc + sc - c;
-        if (O.union_ids) O.union_ids[u] = tid;
-        if (O.offsets) O.offsets[u] = bc + sc - c;
-      }
-    }
-    if (tid == blockDim.x - 1) {  // totals: this thread's inclusive prefix covers all experts
-      int U = bf + sf;
-      T.offsets[U] = A;
-      if (O.offsets) O.offsets[U] = A;
-      *T.n_active = U;
-      n_union_s = U;
-      if (O.n_active) *O.n_active = U;
-    }
-  }
-  __syncthreads();
-
-  MOEV_RT_MARK(10);
-  // ---- phase 2b: work units for the tensor-core FFN: every expert's slots cut into runs of at
-  // most unit_cap.  Order: the shared experts' units (they see every token, so their tasks are
-  // the longest), then the full runs of the routed experts, then the routed experts' remainders
-  // in three classes of decreasing length (>= 12, >= 6, shorter), expert order inside each.  A
-  // task's cost grows with its unit's tokens (one global reduction per token and output row in
-  // the down phase) and tasks are handed out in unit order: the cheap ones last keeps the CTAs'
-  // finishing times close together (clustered tree workload: FFN kernel 920 -> 895 us), while
-  // expert order inside a class keeps concurrently running tasks on neighbouring experts.
-  {
-    __shared__ int32_t warp_tot_cls[32], tot_unit_s, tot_cls_s;
-    const int U = n_union_s;
-    // many tokens per streamed expert: the two-phase FFN schedule (wide_ratio = 0: not available)
-    // (measured switch-over: above 8 assignments per streamed expert for small unions, where the weight stream
-    // is short, above 12 for large ones, where the two-phase schedule's re-streaming per 32-token unit costs more)
-    const int ut = U + n_shared;
-    const bool wide = T.wide != nullptr && wide_ratio > 0 &&
-                      (A + n_shared * gamma) > (ut < 100 ? wide_ratio : wide_ratio + wide_ratio / 2) * ut;
-    // the order by cost class is for the single-phase schedules; the two-phase one wants an expert's units next to
-    // each other (they re-read its weights through the L2), and the CUDA-core path has no cap and no use for units
-    const bool sorted = unit_cap <= 64 && !wide;
-    int e = 0, slot0 = 0, m = 0, shared = 0;
-    if (tid < n_shared) { shared = 1; e = tid; slot0 = A + e * gamma; m = gamma; }
-    else if (tid < U + n_shared) { e = T.union_ids[tid - n_shared]; slot0 = T.offsets[tid - n_shared]; m = cnt[e]; }
-    const int rem = (sorted && !shared) ? m % unit_cap : 0;   // placed behind the full runs
-    const int cls = rem >= 12 ? 0 : (rem >= 6 ? 1 : 2);
-    int nch = (m - rem + unit_cap - 1) / unit_cap, sc = nch;  // units placed in expert order
-    int pk = rem > 0 ? (1 << (10 * cls)) : 0, spk = pk;       // three 10-bit counters (at most 512 experts)
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      int a = __shfl_up_sync(0xffffffffu, sc, o), b = __shfl_up_sync(0xffffffffu, spk, o);
-      if (lane >= o) { sc += a; spk += b; }
-    }
-    if (lane == 31) { warp_tot_unit[warp] = sc; warp_tot_cls[warp] = spk; }
-    __syncthreads();
-    if (warp == 0) {  // exclusive prefixes of the 32 warp totals (and the grand totals) by one warp
-      const int wu = warp_tot_unit[lane], wc = warp_tot_cls[lane];
-      int su = wu, sk = wc;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int a = __shfl_up_sync(0xffffffffu, su, o), b = __shfl_up_sync(0xffffffffu, sk, o);
-        if (lane >= o) { su += a; sk += b; }
-      }
-      warp_tot_unit[lane] = su - wu; warp_tot_cls[lane] = sk - wc;
-      if (lane == 31) { tot_unit_s = su; tot_cls_s = sk; }
-    }
-    __syncthreads();
-    const int base = warp_tot_unit[warp], total1 = tot_unit_s, bpk = warp_tot_cls[warp], tpk = tot_cls_s;
-    int first = base + sc - nch;
-    for (int c = 0; c < nch; ++c) {
-      Unit un;
-      un.expert = e; un.slot0 = slot0 + c * unit_cap;
-      un.m = min(unit_cap, m - c * unit_cap); un.shared = shared;
-      T.units[first + c] = un;
-    }
-    const int n0 = tpk & 1023, n1 = (tpk >> 10) & 1023, n2 = (tpk >> 20) & 1023;
-    if (rem > 0) {
-      const int before = ((bpk + spk - pk) >> (10 * cls)) & 1023;  // earlier experts of the same class
-      const int pos = total1 + (cls > 0 ? n0 : 0) + (cls > 1 ? n1 : 0) + before;
-      Unit un;
-      un.expert = e; un.slot0 = slot0 + (m - rem); un.m = rem; un.shared = 0;
-      T.units[pos] = un;
-    }
-    sc = total1 + n0 + n1 + n2 - base;  // so that base + sc below is the number of units
-    if (tid == blockDim.x - 1) {
-      *T.n_units = base + sc;
-      *T.task_counter = 0;
-      if (T.wide) *T.wide = wide ? 1 : 0;
-    }
-    if (T.unit_done) {
-      __shared__ int n_units_s;
-      if (tid == blockDim.x - 1) n_units_s = base + sc;
-      __syncthreads();
-      for (int i = tid; i < 2 * n_units_s; i += blockDim.x) T.unit_done[i] = 0;  // and the gather flags behind them
-    }
-  }
-
-  MOEV_RT_MARK(11);
-  // ---- phase 3: stable permutation.  A token selects an expert at most once, so the slot of
-  // assignment (t, e) inside e's run is the number of tokens below t that selected e: a prefix
-  // population count over e's token bitmap, one thread per assignment.
-  __syncthreads();
-  {
-    const int TW = (gamma + 31) / 32;
-    uint32_t* tb = reinterpret_cast<uint32_t*>(sm + 3 * E + 2 * A);  // [E][TW]
-    for (int i = tid; i < E * TW; i += blockDim.x) tb[i] = 0u;
-    __syncthreads();
-    for (int a = tid; a < A; a += blockDim.x) {
-      const int t = a / k;
-      atomicOr(&tb[ids_s[a] * TW + (t >> 5)], 1u << (t & 31));
-    }
-    __syncthreads();
-    for (int a = tid; a < A; a += blockDim.x) {
-      const int t = a / k, e = ids_s[a];
-      const uint32_t* row = tb + e * TW;
-      int rank = __popc(row[t >> 5] & ((1u << (t & 31)) - 1u));
-      for (int w = 0; w < (t >> 5); ++w) rank += __popc(row[w]);
-      const int pos = excl[e] + rank;
-      T.perm[pos] = a;
-      T.slot_token[pos] = t;
-      T.slot_w[pos] = w_s[a];
-      if (O.perm) O.perm[pos] = a;
-    }
-    MOEV_RT_MARK(12);
-  }
-}
 
 }  // namespace moev
