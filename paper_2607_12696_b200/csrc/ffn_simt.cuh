@@ -220,6 +220,9 @@ __global__ void finalize_kernel(const float* __restrict__ y32, void* __restrict_
   // a dependent launch (the first kernel of the next layer of a pipelined call) may be scheduled from here on
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the FFN kernel's reductions are complete
+#ifdef MOEV_TC_STATS
+  if (blockIdx.x == 0 && threadIdx.x == 0) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); g_rt_stats[30] = (long long)_t; }
+#endif
   size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (i >= n) return;
   float4 v = *reinterpret_cast<const float4*>(y32 + i);

@@ -74,7 +74,9 @@ namespace tcp {  // single-phase schedule without activation producers (ffn_tc_p
 template <bool ACTQ>
 __device__ __noinline__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
                              const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up, const CUtensorMap& tm_sh_down,
-                             const CUtensorMap& tm_xq, const tc::Params& P, uint32_t tmem);
+                             const CUtensorMap& tm_xq, const tc::Params& P, uint32_t tmem, const Unit& u_first);
+__device__ __forceinline__ void promote_prologue(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
+                                                 const CUtensorMap& tm_xq);
 }  // namespace tcp
 namespace tc {
 
@@ -109,6 +111,7 @@ struct Params {
   int32_t xq_ready;     // fp8: the routing kernels wrote the quantised activations: run the schedule of ffn_tc_p.cuh
   int32_t actq;         // moev_act_quant: FP8 1x128 activations (single e4m3 term, block scales in xs)
   const float* xs;      // [gamma, H / 128] activation block scales (actq != 0)
+  int32_t units_alloc;  // entries allocated behind `units` (reads ahead of the unit count stay below it)
 #ifdef MOEV_TC_STATS
   unsigned long long* stats;  // [grid][16] cycles the MMA thread spent per wait / issue class (debug builds)
 #endif
@@ -241,6 +244,11 @@ __device__ __forceinline__ int next_task(Smem& S, uint32_t& q, volatile int* abo
   return id;
 }
 
+#ifdef MOEV_TC_STATS
+#define MOEV_TC_MARK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); g_rt_stats[i] = (long long)_t; } } while (0)
+#else
+#define MOEV_TC_MARK(i)
+#endif
 template <int WFMT>
 __global__ void __launch_bounds__(kThreads, 1)
 grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_constant__ CUtensorMap tm_up,
@@ -293,9 +301,25 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem = S.tmem_base;
+  if (tid == 0) { ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down); }
+#ifndef MOEV_FP8_FOLD_SCALE
+  if constexpr (WFMT == MOEV_W_FP8E4M3_B128) {
+    // the schedule that is expected to run sets up its own barriers now (the two-phase schedule, should the
+    // routing result call for it, sets up its own after the wait)
+    if (P.xq_ready) tcp::promote_prologue(tm_gate, tm_up, tm_down, tm_xq);
+  }
+#endif
   // everything above overlapped the tail of the grouping kernel; its tables are needed from here
+  MOEV_TC_MARK(24);
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  MOEV_TC_MARK(25);
+  // (fp8 schedule without producers: the TMA warp asks for the records of the first units, and of the unit this
+  // CTA's first task has in large calls, together with the loads that decide the schedule: one trip to the L2)
+  Unit u_first{};
+  if constexpr (WFMT == MOEV_W_FP8E4M3_B128) {
+    if (P.xq_ready && warp == 0) u_first = P.units[min(lane < 31 ? lane : (int)(blockIdx.x >> 1), P.units_alloc - 1)];
+  }
   const int n_units = *P.n_units;
   if constexpr (WFMT == MOEV_W_FP8E4M3_B128) {
     if (P.wide && *P.wide) {
@@ -312,10 +336,15 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #ifndef MOEV_FP8_FOLD_SCALE
     if (P.xq_ready) {
       // quantised activations are available: the schedule without activation producers
-      if (P.actq) tcp::promote_body<true>(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem);
-      else tcp::promote_body<false>(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem);
+      if (P.actq) tcp::promote_body<true>(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem, u_first);
+      else tcp::promote_body<false>(tm_gate, tm_up, tm_down, tm_sh_gate, tm_sh_up, tm_sh_down, tm_xq, P, tmem, u_first);
       ptx::tc_fence_before();
       __syncthreads();
+      MOEV_TC_MARK(26);
+#ifdef MOEV_TC_STATS
+      if (threadIdx.x == 0) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t));
+        atomicMax(reinterpret_cast<unsigned long long*>(&g_rt_stats[27]), _t); atomicMin(reinterpret_cast<unsigned long long*>(&g_rt_stats[28]), _t); }
+#endif
       if (warp == 0) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, kTmemCols);
@@ -330,7 +359,6 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   if (warp == 0) {
     // ===================================================== TMA producer + scheduler (one lane)
     if (lane == 0) {
-      ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
       uint32_t it = 0, q = 0;
       bool ok = true;
 #ifdef MOEV_TC_STATS
@@ -339,13 +367,14 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
 #endif
       // Task ids are published one task ahead of the loads, so the other roles can prepare
       // their tables (and the first activation tiles) while this task still streams.
-      bool first_draw = true;
+      int draws = 0;
       auto fetch_publish = [&](TaskDesc& td) -> int {
         int id;
         td.unit = 0; td.slice = 0; td.valid = false;
         do {
-          id = first_draw ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(P.task_counter, 1);  // the first draw needs no trip to the counter
-          first_draw = false;
+          // the first two draws need no trip to the counter (two tasks are published before the first loads begin)
+          id = draws < 2 ? (int)(blockIdx.x + draws * gridDim.x) : (int)(2 * gridDim.x) + atomicAdd(P.task_counter, 1);
+          ++draws;
           if (id >= n_ids) { id = -1; break; }
           td = decode_task(id, n_units, n_slices);
         } while (!td.valid);

@@ -242,6 +242,10 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   __syncthreads();
   ptx::tc_fence_after();
   if (tid == 0) MOEV_MX_MARK(25);
+  if (tid == 0) {
+    ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
+    ptx::prefetch_tmap(&tm_xq); ptx::prefetch_tmap(&tm_hq);
+  }
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) MOEV_MX_MARK(26);
@@ -257,14 +261,15 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   if (warp == 0) {
     // ===================================================== TMA producer + scheduler (one lane)
     if (lane == 0) {
-      ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down);
-      ptx::prefetch_tmap(&tm_xq); ptx::prefetch_tmap(&tm_hq);
       uint32_t it = 0, q = 0;
       bool ok = true;
-      bool first_draw = true;
+      int draws = 0;
       auto fetch_publish = [&]() -> int {
-        int id = first_draw ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(P.task_counter, 1);  // the first draw needs no trip to the counter
-        first_draw = false;
+        // the first two draws need no trip to the counter (the second task is published before the first one's
+        // loads begin): ids blockIdx.x and blockIdx.x + gridDim.x.  A task still depends only on phase-1 tasks
+        // with smaller ids, and those wait for nothing.
+        int id = draws < 2 ? (int)(blockIdx.x + draws * gridDim.x) : (int)(2 * gridDim.x) + atomicAdd(P.task_counter, 1);
+        ++draws;
         if (id >= n_ids) id = -1;
         if (id < 0 && MOEV_TEST_WITHHOLD()) return -1;  // test builds: the final message is withheld
         const int slot = q % kTaskQ;

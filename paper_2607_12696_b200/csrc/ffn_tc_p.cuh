@@ -80,27 +80,16 @@ __device__ __forceinline__ int next_task(Smem& S, uint32_t& q, volatile int* abo
   return id;
 }
 
-template <bool ACTQ>
-__device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
-                                          const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up,
-                                          const CUtensorMap& tm_sh_down, const CUtensorMap& tm_xq,
-                                          const tc::Params& P, uint32_t tmem) {
-  constexpr int WFMT = MOEV_W_FP8E4M3_B128;
+// Barriers and flags of promote_body (the same shared memory as the caller's control block: every thread has left
+// that use).  The kernel runs this before it waits for the routing kernels, so that nothing but the loads of the
+// routing result stands between the end of that wait and the first weight copy; ends with a block-wide barrier.
+__device__ __forceinline__ void promote_prologue(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
+                                                 const CUtensorMap& tm_xq) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* w_ring = base;
-  uint8_t* b_tiles = w_ring + kStages * kStageBytes;
-  uint8_t* h_tile = b_tiles + kStages * kBTileBytes;
-  static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
   Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int H = P.H, I = P.I;
-  const int KC = H / 128, HT = H / 128, n_slices = I / 128;
-  const int n_dstage = (HT + 1) / 2;
-
   __syncthreads();
-  if (tid == 0) {
+  if (threadIdx.x == 0) {
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
     for (int i = 0; i < 2; ++i) {
       ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 8);
@@ -115,8 +104,30 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
     S.prod_it = 0;
     S.abort_flag = 0;
     ptx::fence_mbar_init();
+    ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down); ptx::prefetch_tmap(&tm_xq);
   }
   __syncthreads();
+}
+
+template <bool ACTQ>
+__device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_up, const CUtensorMap& tm_down,
+                                          const CUtensorMap& tm_sh_gate, const CUtensorMap& tm_sh_up,
+                                          const CUtensorMap& tm_sh_down, const CUtensorMap& tm_xq,
+                                          const tc::Params& P, uint32_t tmem, const Unit& u_first) {
+  constexpr int WFMT = MOEV_W_FP8E4M3_B128;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* w_ring = base;
+  uint8_t* b_tiles = w_ring + kStages * kStageBytes;
+  uint8_t* h_tile = b_tiles + kStages * kBTileBytes;
+  static_assert(sizeof(Smem) <= kCtlBytes, "control block budget");
+  Smem& S = *reinterpret_cast<Smem*>(base + kTileBytes);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int H = P.H, I = P.I;
+  const int KC = H / 128, HT = H / 128, n_slices = I / 128;
+  const int n_dstage = (HT + 1) / 2;
+
   const int n_units = *P.n_units;
   const int n_ids = n_units * ((n_slices + 1) & ~1);
   volatile int* abortp = &S.abort_flag;
@@ -124,9 +135,8 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
   if (warp == 0) {
     // ===================================================== TMA producer + scheduler (the warp stays converged:
     // lane 0 waits, arms the barriers and loads the weight tiles, lane r loads the operand rows of token r)
-    if (lane == 0) {
-      ptx::prefetch_tmap(&tm_gate); ptx::prefetch_tmap(&tm_up); ptx::prefetch_tmap(&tm_down); ptx::prefetch_tmap(&tm_xq);
-    }
+    // (u_first: lane l < 31 holds the record of unit l, lane 31 that of unit blockIdx.x / 2, requested by the caller
+    // together with the unit count: one trip to the L2 instead of two before the first weight copy)
     uint32_t it = 0, q = 0;
     bool ok = true;
     bool first_draw = true;
@@ -167,10 +177,21 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
     };
     TaskDesc td, td_next;
     int id = fetch_publish(td);
+    bool first_task = true;
+    // the next task is drawn (a trip to the counter) and published while this task's first stages are in flight
+    const int look_kc = KC - 1 < 3 ? KC - 1 : 3;
     while (ok && id >= 0) {
-      const int id_next = fetch_publish(td_next);  // published one task ahead
-      if (!ok) break;
-      const Unit u = P.units[td.unit];
+      int id_next = -1;
+      Unit u;
+      {
+        const int src = td.unit < 31 ? td.unit : 31;
+        uint4 r = *reinterpret_cast<const uint4*>(&u_first);
+        r.x = __shfl_sync(0xffffffffu, r.x, src); r.y = __shfl_sync(0xffffffffu, r.y, src);
+        r.z = __shfl_sync(0xffffffffu, r.z, src); r.w = __shfl_sync(0xffffffffu, r.w, src);
+        const bool hit = first_task && (td.unit < 31 || td.unit == (int)(blockIdx.x >> 1)) && td.unit < P.units_alloc;
+        if (hit) u = *reinterpret_cast<const Unit*>(&r); else u = P.units[td.unit];
+        first_task = false;
+      }
       const int slice = td.slice, m = u.m;
       const CUtensorMap* mg = u.shared ? &tm_sh_gate : &tm_gate;
       const CUtensorMap* mu = u.shared ? &tm_sh_up : &tm_up;
@@ -178,6 +199,10 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
       int tok = 0;
       if (lane < m) tok = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma) + lane) : __ldg(P.slot_token + u.slot0 + lane);
       for (int kc = 0; kc < KC && ok; ++kc, ++it) {
+        if (kc == look_kc) {
+          id_next = fetch_publish(td_next);
+          if (!ok) break;
+        }
         const int s = it % kStages;
         wait_stage(s);
         if (!ok) break;
@@ -233,6 +258,9 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           { MOEV_STAT_BEGIN();
             ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             MOEV_STAT_END(1); }
+#ifdef MOEV_TC_STATS
+          if (it == 0 && blockIdx.x == 0 && warp == 1) { unsigned long long _t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(_t)); g_rt_stats[29] = (long long)_t; }
+#endif
           { MOEV_STAT_BEGIN();
             ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((pc >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             MOEV_STAT_END(3); }

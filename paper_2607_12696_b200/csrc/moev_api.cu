@@ -12,6 +12,7 @@
 #include "ffn_tc_wide.cuh"
 #include "ffn_tc_p.cuh"
 #include "router.cuh"
+#include "route_exact.cuh"
 #include "route_fused.cuh"
 #include "select.cuh"
 
@@ -46,6 +47,8 @@ struct moev_ctx {
   int ks = 32;  // columns per split-K slice of the router
   bool router_mma = false;
   FusedScratch fused{};     // two-launch routing of tree-sized calls (route_fused.cuh)
+  double* logits64 = nullptr;  // [min(max_tokens, kExactMaxTokens), E] exact router logits (route_exact.cuh)
+  bool exact_ok = false;       // the shape is served by the exact-logit routing path
   size_t fused_smem_max = 0;
 #ifdef MOEV_TC_STATS
   unsigned long long* tc_stats = nullptr;  // [n_sm][16], debug builds only
@@ -295,7 +298,7 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
   P.wide = c->wide_ok ? c->T.wide : nullptr;
   P.xq_ready = (c->wide_ok && c->T.xq) ? 1 : 0;
-  P.actq = g.act_quant; P.xs = c->T.xs;
+  P.actq = g.act_quant; P.xs = c->T.xs; P.units_alloc = (int32_t)c->max_units;
   // arguments of the two-phase schedule, which the kernel switches to when the grouping kernel's
   // flag says that the call has many tokens per streamed expert (fp8 only)
   tcw::Params W{};
@@ -421,6 +424,10 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
       c->fused_smem_max = std::max(c->fused_smem_max, route_group_block_smem(cfg->E, g, cfg->top_k));
     ok = ok && dmalloc(&c->fused.done_cnt, 1) == cudaSuccess;
     ok = ok && cudaMemset(c->fused.done_cnt, 0, sizeof(int32_t)) == cudaSuccess;
+    // exact-logit routing of the smallest calls: rows of x staged in shared memory by 16-byte copies
+    c->exact_ok = exact_smem(cfg->H, (int)act_b) <= kExactMaxSmem && (cfg->H * act_b) % 16 == 0 && cfg->H % 4 == 0;
+    if (c->exact_ok)
+      ok = ok && dmalloc(&c->logits64, (size_t)std::min<int>(cfg->max_tokens, kExactMaxTokens) * E) == cudaSuccess;
   }
   ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
@@ -438,6 +445,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     const size_t cap = c->unit_cap;
     const size_t max_units = E + A / cap + (size_t)cfg->n_shared * (G / cap + 1) + 8;
     ok = ok && dmalloc(&c->T.units, max_units) == cudaSuccess;
+    ok = ok && cudaMemset(c->T.units, 0, max_units * sizeof(Unit)) == cudaSuccess;
+    c->max_units = max_units;
     const int n_slices = cfg->I / 128;
     c->wide_ok = c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_FP8E4M3_B128 && n_slices <= tcw::kMaxSlices;
     if (c->resolved_impl == MOEV_IMPL_TCGEN05 && cfg->wfmt == MOEV_W_MXFP4) {
@@ -536,6 +545,20 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
                                       (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(route_refine_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
+      if (c->exact_ok) {
+        const int xs = (int)exact_smem(cfg->H, (int)act_b);
+        if (cfg->afmt == MOEV_ACT_FP32) {
+          ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_FP32, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, xs) == cudaSuccess;
+          ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_FP32, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, xs) == cudaSuccess;
+        } else {
+          ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, xs) == cudaSuccess;
+          ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_BF16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, xs) == cudaSuccess;
+        }
+        ok = ok && cudaFuncSetAttribute(route_select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(route_select_kernel<kMaxE / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
+      }
     }
     if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
       ok = ok && cudaFuncSetAttribute(tc::grouped_ffn_tc_kernel<MOEV_W_BF16>,
@@ -558,7 +581,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
 
 moev_status moev_destroy(moev_ctx* c) {
   if (!c) return MOEV_EINVAL;
-  cudaFree(c->fused.done_cnt);
+  cudaFree(c->fused.done_cnt); cudaFree(c->logits64);
   cudaFree(c->part); cudaFree(c->part_x2); cudaFree(c->part_w2); cudaFree(c->T.topk_ids); cudaFree(c->T.topk_w); cudaFree(c->T.union_ids);
   cudaFree(c->T.offsets); cudaFree(c->T.perm); cudaFree(c->T.slot_token); cudaFree(c->T.slot_w);
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
@@ -647,55 +670,76 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
                     ? (int)std::min<size_t>(layer->n_predicted, budget - pf.n_shared) : 0;
     if (mat_bytes % 16) { pf.n_shared = 0; pf.n_pred = 0; }
   }
-  if (g.afmt == MOEV_ACT_FP32)
-    launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain != 0, x, layer->router_w,
-             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
-  else if (gamma <= 32) {
-    // tree-sized calls: the variant without shared memory (one trip to memory long)
-    // (a dependent layer's first kernel is not launched ahead at these sizes: its CTAs, resident and waiting beside
-    // the previous layer's expert kernel, cost that kernel more than the early launch saves -- measured +4 % per
-    // layer at gamma = 4, against -2 % at gamma = 64)
-    auto go = [&](auto kern) {
-      launch_k(kern, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(128), 0, st, pdl && c->chain == 1,
-               static_cast<const uint16_t*>(x), layer->router_w, c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
-    };
-    if (gamma <= 8) go(router_partial_small_kernel<1>);
-    else if (gamma <= 16) go(router_partial_small_kernel<2>);
-    else go(router_partial_small_kernel<4>);
-  } else
-    launch_k(router_partial_mma_kernel, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256),
-             router_partial_mma_smem(c->ks), st, pdl && c->chain != 0, static_cast<const uint16_t*>(x), layer->router_w,
-             c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
-  if (ev) cudaEventRecord(ev[1], st);
-  const int refine_depth = g.afmt == MOEV_ACT_FP32 ? c->ks : 6 * c->ks + c->n_slices + 12;
   const int wide_ratio = (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0;
-  if (g.n_group == 0 && gamma <= kFusedMaxTokens) {
-    // tree-sized calls: refinement spread over several CTAs per token, grouping by the last one to finish
-    const int S = fused_slices(gamma, g.H, c->n_sm);
-    const size_t gsm = route_group_block_smem(g.E, gamma, g.top_k);
+  if (c->exact_ok && g.n_group == 0 && gamma <= kExactMaxTokens) {
+    // the smallest calls: fp64 logits in one pass, selection and grouping by one CTA (route_exact.cuh)
+    const int epc = exact_epc(g.E, c->n_sm);
+    const dim3 grid((g.E + epc - 1) / epc, (gamma + kExactTok - 1) / kExactTok);
+    const size_t xs = (size_t)std::min(gamma, kExactTok) * g.H * (g.afmt == MOEV_ACT_FP32 ? 4 : 2);
     auto go = [&](auto kern) {
-      launch_kc(kern, dim3(S, gamma), dim3(kFusedThreads), gsm, st, pdl, S, c->T, O, c->fused, x, layer->router_w,
-               (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
-               g.top_k, c->n_slices, refine_depth, g.score, g.routed_scale, g.n_shared, c->unit_cap, wide_ratio);
+      launch_k(kern, grid, dim3(kExactThreads), xs, st, pdl && c->chain == 1, c->T, x, layer->router_w, c->logits64,
+               c->y32, gamma, g.H, g.E, c->chain == 2 ? 1 : 0, pf);
     };
-    if (g.afmt == MOEV_ACT_FP32) go(route_refine_kernel<MOEV_ACT_FP32>); else go(route_refine_kernel<MOEV_ACT_BF16>);
-    if (ev) cudaEventRecord(ev[2], st);
-  } else {
-    // the kernel's code is executed once per CTA, front to back: the plain and the group-limited
-    // routing are separate instantiations so that neither carries the other's instructions
-    auto go = [&](auto kern) {
-      launch_k(kern, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x, layer->router_w,
-               (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
-               g.top_k, c->n_slices, refine_depth, g.score, g.routed_scale, layer->router_bias, g.n_group, g.topk_group);
-    };
-    if (g.afmt == MOEV_ACT_FP32) {
-      if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_FP32, true>); else go(topk_refine_kernel<MOEV_ACT_FP32, false>);
-    } else {
-      if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_BF16, true>); else go(topk_refine_kernel<MOEV_ACT_BF16, false>);
+    if (g.afmt == MOEV_ACT_FP32) { if (epc == 1) go(router_exact_kernel<MOEV_ACT_FP32, 1>); else go(router_exact_kernel<MOEV_ACT_FP32, 2>); }
+    else { if (epc == 1) go(router_exact_kernel<MOEV_ACT_BF16, 1>); else go(router_exact_kernel<MOEV_ACT_BF16, 2>); }
+    if (ev) cudaEventRecord(ev[1], st);
+    {
+      auto sel = g.E <= 256 ? route_select_kernel<8> : route_select_kernel<kMaxE / 32>;
+      launch_k(sel, dim3(1), dim3(kSelectThreads), route_group_block_smem(g.E, gamma, g.top_k), st, pdl, c->T, O,
+               (const double*)c->logits64, gamma, g.E, g.top_k, g.score, g.routed_scale, g.n_shared, c->unit_cap, wide_ratio,
+               pdl ? 1 : 0);
     }
     if (ev) cudaEventRecord(ev[2], st);
-    launch_k(route_group_kernel, dim3(1), dim3(kGroupThreads), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E,
-             g.top_k, g.n_shared, c->unit_cap, wide_ratio);
+  } else {
+    if (g.afmt == MOEV_ACT_FP32)
+      launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain != 0, x, layer->router_w,
+               c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+    else if (gamma <= 32) {
+      // tree-sized calls: the variant without shared memory (one trip to memory long)
+      // (a dependent layer's first kernel is not launched ahead at these sizes: its CTAs, resident and waiting beside
+      // the previous layer's expert kernel, cost that kernel more than the early launch saves -- measured +4 % per
+      // layer at gamma = 4, against -2 % at gamma = 64)
+      auto go = [&](auto kern) {
+        launch_k(kern, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(128), 0, st, pdl && c->chain == 1,
+                 static_cast<const uint16_t*>(x), layer->router_w, c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+      };
+      if (gamma <= 8) go(router_partial_small_kernel<1>);
+      else if (gamma <= 16) go(router_partial_small_kernel<2>);
+      else go(router_partial_small_kernel<4>);
+    } else
+      launch_k(router_partial_mma_kernel, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256),
+               router_partial_mma_smem(c->ks), st, pdl && c->chain != 0, static_cast<const uint16_t*>(x), layer->router_w,
+               c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+    if (ev) cudaEventRecord(ev[1], st);
+    const int refine_depth = g.afmt == MOEV_ACT_FP32 ? c->ks : 6 * c->ks + c->n_slices + 12;
+    if (g.n_group == 0 && gamma <= kFusedMaxTokens) {
+      // tree-sized calls: refinement spread over several CTAs per token, grouping by the last one to finish
+      const int S = fused_slices(gamma, g.H, c->n_sm);
+      const size_t gsm = route_group_block_smem(g.E, gamma, g.top_k);
+      auto go = [&](auto kern) {
+        launch_kc(kern, dim3(S, gamma), dim3(kFusedThreads), gsm, st, pdl, S, c->T, O, c->fused, x, layer->router_w,
+                 (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
+                 g.top_k, c->n_slices, refine_depth, g.score, g.routed_scale, g.n_shared, c->unit_cap, wide_ratio);
+      };
+      if (g.afmt == MOEV_ACT_FP32) go(route_refine_kernel<MOEV_ACT_FP32>); else go(route_refine_kernel<MOEV_ACT_BF16>);
+      if (ev) cudaEventRecord(ev[2], st);
+    } else {
+      // the kernel's code is executed once per CTA, front to back: the plain and the group-limited
+      // routing are separate instantiations so that neither carries the other's instructions
+      auto go = [&](auto kern) {
+        launch_k(kern, dim3(gamma), dim3(kRefineThreads), refine_smem, st, pdl, c->T, O, x, layer->router_w,
+                 (const float*)c->part, (const float*)c->part_x2, (const float*)c->part_w2, c->y32, gamma, g.H, g.E,
+                 g.top_k, c->n_slices, refine_depth, g.score, g.routed_scale, layer->router_bias, g.n_group, g.topk_group);
+      };
+      if (g.afmt == MOEV_ACT_FP32) {
+        if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_FP32, true>); else go(topk_refine_kernel<MOEV_ACT_FP32, false>);
+      } else {
+        if (g.n_group > 0) go(topk_refine_kernel<MOEV_ACT_BF16, true>); else go(topk_refine_kernel<MOEV_ACT_BF16, false>);
+      }
+      if (ev) cudaEventRecord(ev[2], st);
+      launch_k(route_group_kernel, dim3(1), dim3(kGroupThreads), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E,
+               g.top_k, g.n_shared, c->unit_cap, wide_ratio);
+    }
   }
   if (ev) cudaEventRecord(ev[3], st);
   if (c->resolved_impl == MOEV_IMPL_TCGEN05) {

@@ -119,8 +119,13 @@ inline size_t route_group_block_smem(int E, int gamma, int k) {
 // blockDim.x * kGroupItems >= E, in four block-wide steps (one scan carries the slot offsets, the
 // union index and both variants of the unit counts).
 constexpr int kGroupItems = 1;
+// ids_in_smem: the caller has already put the top-k ids and weights into the block's ids / w arrays (sm + 2 E ..).
+// dry: nothing is read from or written to global memory (the tables in shared memory then hold whatever they
+// held); a kernel that is resident before its input is ready runs the routine once this way so that its
+// instructions are in the SM's instruction cache when the real pass starts.
 __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOut& O, int gamma, int E, int k, int n_shared,
-                                                  int unit_cap, int wide_ratio, int32_t* sm) {
+                                                  int unit_cap, int wide_ratio, int32_t* sm, bool ids_in_smem = false,
+                                                  bool dry = false) {
   const int A = gamma * k;
   int32_t* cnt = sm;
   int32_t* excl = sm + E;
@@ -135,9 +140,14 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
   for (int i = tid; i < E * TW; i += nt) tb[i] = 0u;
   __syncthreads();
   for (int a = tid; a < A; a += nt) {
-    const int e = __ldcg(T.topk_ids + a);
-    ids_s[a] = e;
-    w_s[a] = __ldcg(T.topk_w + a);
+    int e;
+    if (ids_in_smem) {
+      e = ids_s[a];
+    } else {
+      e = __ldcg(T.topk_ids + a);
+      ids_s[a] = e;
+      w_s[a] = __ldcg(T.topk_w + a);
+    }
     atomicAdd(&cnt[e], 1);
     const int t = a / k;
     atomicOr(&tb[e * TW + (t >> 5)], 1u << (t & 31));
@@ -190,7 +200,7 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
     Unit un;
     un.expert = sx; un.slot0 = A + sx * gamma + c * unit_cap;
     un.m = min(unit_cap, gamma - c * unit_cap); un.shared = 1;
-    T.units[i] = un;
+    if (!dry) T.units[i] = un;
   }
 #pragma unroll
   for (int i = 0; i < kGroupItems; ++i) {
@@ -199,10 +209,12 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
     excl[e] = v[0][i];
     if (m[i] == 0) continue;
     const int u = v[1][i], slot0 = v[0][i];
-    T.union_ids[u] = e;
-    T.offsets[u] = slot0;
-    if (O.union_ids) O.union_ids[u] = e;
-    if (O.offsets) O.offsets[u] = slot0;
+    if (!dry) {
+      T.union_ids[u] = e;
+      T.offsets[u] = slot0;
+      if (O.union_ids) O.union_ids[u] = e;
+      if (O.offsets) O.offsets[u] = slot0;
+    }
     const int rem = sorted ? (m[i] & cap_mask) : 0;
     const int nch = sorted ? (m[i] >> cap_log2) : ((m[i] + cap_mask) >> cap_log2);
     const int first = base + (sorted ? v[2][i] : v[4][i]);
@@ -210,17 +222,17 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
       Unit un;
       un.expert = e; un.slot0 = slot0 + c * unit_cap;
       un.m = min(unit_cap, m[i] - c * unit_cap); un.shared = 0;
-      T.units[first + c] = un;
+      if (!dry) T.units[first + c] = un;
     }
     if (rem > 0) {
       const int cls = rem >= 12 ? 0 : (rem >= 6 ? 1 : 2);
       const int before = (v[3][i] >> (10 * cls)) & 1023;  // earlier experts of the same class
       Unit un;
       un.expert = e; un.slot0 = slot0 + (m[i] - rem); un.m = rem; un.shared = 0;
-      T.units[base + total1 + (cls > 0 ? n0 : 0) + (cls > 1 ? n1 : 0) + before] = un;
+      if (!dry) T.units[base + total1 + (cls > 0 ? n0 : 0) + (cls > 1 ? n1 : 0) + before] = un;
     }
   }
-  if (tid == 0) {
+  if (tid == 0 && !dry) {
     T.offsets[U] = A;
     if (O.offsets) O.offsets[U] = A;
     *T.n_active = U;
@@ -229,7 +241,7 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
     *T.task_counter = 0;
     if (T.wide) *T.wide = wide ? 1 : 0;
   }
-  if (T.unit_done)
+  if (T.unit_done && !dry)
     for (int i = tid; i < 2 * n_units; i += nt) T.unit_done[i] = 0;  // progress counters and the gather flags behind them
   __syncthreads();  // excl complete
   MOEV_RF_MARK(19, true);
@@ -241,10 +253,12 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
     int rank = __popc(row[t >> 5] & ((1u << (t & 31)) - 1u));
     for (int w = 0; w < (t >> 5); ++w) rank += __popc(row[w]);
     const int pos = excl[e] + rank;
-    T.perm[pos] = a;
-    T.slot_token[pos] = t;
-    T.slot_w[pos] = w_s[a];
-    if (O.perm) O.perm[pos] = a;
+    if (!dry) {
+      T.perm[pos] = a;
+      T.slot_token[pos] = t;
+      T.slot_w[pos] = w_s[a];
+      if (O.perm) O.perm[pos] = a;
+    }
   }
 }
 
