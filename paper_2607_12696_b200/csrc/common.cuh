@@ -71,6 +71,8 @@ struct Tables {
 
 #ifdef MOEV_TC_STATS
 __device__ long long g_rt_stats[32];  // debug builds: phase timestamps (CTA 0) of the routing and expert kernels
+__device__ long long g_task_log[8192][4];  // debug builds: task id | CTA | start | end (global timer) of an expert kernel's tasks
+__device__ __forceinline__ long long debug_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return (long long)t; }
 #endif
 
 struct LayerPtrs {

@@ -57,6 +57,7 @@ constexpr int kStages = 4;     // weight ring of 32 KB stages (two [128 x 128 B]
 constexpr int kMC = 8;         // tokens per unit (four terms each -> N <= 32)
 constexpr int kBTileBytes = 4 * 1024;  // [32 x 128 B] activation tile, one per weight-ring stage
 constexpr int kMaxChunks = 12;         // 256-element K chunks per row: H, I <= 3072
+constexpr int kNormalPolicyUnits = 64; // calls of at least this many units stream the weights with the default L2 policy
 constexpr int kTmemCols = 512;
 // TMEM columns: (tile 0: 32 | tile 1: 32) x 2 task parities | 16 weight scale-factor columns per
 // ring stage | activation scale factors: x (constant), h (two words per K chunk, per task parity).
@@ -264,6 +265,13 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
       uint32_t it = 0, q = 0;
       bool ok = true;
       int draws = 0;
+      // L2 policy of the weight stream.  Rows of K / 2 bytes that are no multiple of 128 bytes (1440 for K = 2880)
+      // make a 128-byte piece of a row share its first and last line with the neighbouring pieces, which the same
+      // CTA fetches a stage later.  Under "evict first" a large call loses many of those lines in between and
+      // reads them twice (gamma = 64, 110 experts: DRAM traffic 1.047 x, kernel 248 us; 234 us with the default
+      // policy); small calls are faster with "evict first" (gamma = 8: 74 against 78 us), which keeps the
+      // activations, the h scratch and the accumulator in the L2.  Measured switch-over between 52 and 78 units.
+      const uint64_t wpol = n_units >= kNormalPolicyUnits ? ptx::kPolicyEvictNormal : ptx::kPolicyEvictFirst;
       auto fetch_publish = [&]() -> int {
         // the first two draws need no trip to the counter (the second task is published before the first one's
         // loads begin): ids blockIdx.x and blockIdx.x + gridDim.x.  A task still depends only on phase-1 tasks
@@ -308,8 +316,8 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           uint8_t* bt = b_tiles + s * kBTileBytes;
           // a box counts its full size, zero-filled parts included
           ptx::mbar_arrive_expect_tx(&S.w_full[s], 2 * 16384 + (t.phase == 1 ? 512 * m : kBTileBytes));
-          ptx::tma_load_3d(dst, m0, &S.w_full[s], kc * 128, row0, u.expert, ptx::kPolicyEvictFirst);
-          ptx::tma_load_3d(dst + 16384, m1, &S.w_full[s], kc * 128, row1, u.expert, ptx::kPolicyEvictFirst);
+          ptx::tma_load_3d(dst, m0, &S.w_full[s], kc * 128, row0, u.expert, wpol);
+          ptx::tma_load_3d(dst + 16384, m1, &S.w_full[s], kc * 128, row1, u.expert, wpol);
           if (t.phase == 1) {
             // activation operand: rows 4 r + j of the stage's tile are the four terms of token r
             for (int r = 0; r < m; ++r) {
@@ -317,7 +325,8 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
               ptx::tma_load_2d(bt + r * 512, &tm_xq, &S.w_full[s], kc * 128, 4 * tok, ptx::kPolicyEvictNormal);
             }
           } else {
-            ptx::tma_load_2d(bt, &tm_hq, &S.w_full[s], kc * 128, 32 * t.unit, ptx::kPolicyEvictNormal);
+            // (the unit's h terms are read by every phase-2 task of the unit: kept in the L2 ahead of the streamed weights)
+            ptx::tma_load_2d(bt, &tm_hq, &S.w_full[s], kc * 128, 32 * t.unit, ptx::kPolicyEvictLast);
           }
         }
       };

@@ -253,6 +253,9 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
         const TaskDesc td = decode_task(id, n_units, n_slices);
         const Unit u = P.units[td.unit];
         const uint32_t idesc = ptx::instr_desc(0, 0, (uint32_t)((2 * u.m + 15) & ~15));
+#ifdef MOEV_TC_STATS
+        if (issuer == 0 && id < 8192) { g_task_log[id][0] = id | ((long long)u.m << 32); g_task_log[id][1] = blockIdx.x; g_task_log[id][2] = debug_gtime(); }
+#endif
         for (int kc = 0; kc < KC && ok; ++kc, ++it, ++pc) {
           const int s = it % kStages, pb = pc & 1;
           { MOEV_STAT_BEGIN();
@@ -301,6 +304,9 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
         }
         if (!ok) break;
         ptx::mma_commit(&S.h_empty);
+#ifdef MOEV_TC_STATS
+        if (issuer == 0 && id < 8192) g_task_log[id][3] = debug_gtime();
+#endif
       }
       if (*abortp) ptx::drain_issuer(&S.drain_bar[issuer], kWaitBudgetNs);
 #ifdef MOEV_TC_STATS

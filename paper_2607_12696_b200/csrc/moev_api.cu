@@ -977,6 +977,9 @@ extern "C" int32_t moev_test_withhold(int32_t on) {
 extern "C" int32_t moev_debug_rt_stats(long long* host_out /*[32]*/) {
   return cudaMemcpyFromSymbol(host_out, g_rt_stats, sizeof(long long) * 32) == cudaSuccess ? 0 : -1;
 }
+extern "C" int32_t moev_debug_task_log(long long* host_out /*[8192*4]*/) {
+  return cudaMemcpyFromSymbol(host_out, g_task_log, sizeof(long long) * 8192 * 4) == cudaSuccess ? 0 : -1;
+}
 // Debug builds: copy the per-CTA wait-cycle counters of the last tensor-core FFN launch.
 int32_t moev_debug_tc_stats(moev_ctx* c, unsigned long long* host_out /*[n_sm*16]*/) {
   if (!c || !host_out) return -1;

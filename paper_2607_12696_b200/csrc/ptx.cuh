@@ -114,6 +114,7 @@ __device__ __forceinline__ void prefetch_tmap(const void* tmap) {
 }
 constexpr uint64_t kPolicyEvictFirst = 0x12F0000000000000ull;
 constexpr uint64_t kPolicyEvictNormal = 0x1000000000000000ull;
+constexpr uint64_t kPolicyEvictLast = 0x14F0000000000000ull;
 
 // ---- tcgen05
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t ncols) {

@@ -135,6 +135,9 @@ __device__ __forceinline__ void route_group_block(const Tables& T, const RouteOu
   __shared__ int32_t scan_ws[5 * 33];
   const int tid = threadIdx.x, nt = blockDim.x;
   const int TW = (gamma + 31) / 32;
+#ifdef MOEV_TC_STATS
+  if (tid == 0) { g_rt_stats[27] = 0; g_rt_stats[28] = 0x7fffffffffffffffll; }
+#endif
 
   for (int e = tid; e < E; e += nt) cnt[e] = 0;
   for (int i = tid; i < E * TW; i += nt) tb[i] = 0u;
