@@ -738,7 +738,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
       }
       if (ev) cudaEventRecord(ev[2], st);
       launch_k(route_group_kernel, dim3(1), dim3(kGroupThreads), route_smem(g, gamma), st, pdl, c->T, O, gamma, g.E,
-               g.top_k, g.n_shared, c->unit_cap, wide_ratio);
+               g.top_k, g.n_shared, c->unit_cap, wide_ratio, pdl ? 1 : 0);
     }
   }
   if (ev) cudaEventRecord(ev[3], st);

@@ -25,23 +25,10 @@ inline int router_slice_width(int H, int n_sm) {
   return ks < 4 ? 4 : (ks > kRouterMaxKS ? kRouterMaxKS : ks);
 }
 
-// bf16 bit pattern -> double without the fp64 conversion unit (exact for normal numbers;
-// zeros / subnormals / non-finite take the conversion instruction).
-__device__ __forceinline__ double bf16_bits_to_double(uint32_t b) {
-  if ((b & 0x7F80u) == 0u || (b & 0x7F80u) == 0x7F80u) return (double)__uint_as_float(b << 16);
-  uint32_t hi = ((b & 0x8000u) << 16) | (((b & 0x7FFFu) << 13) + (896u << 20));
-  return __hiloint2double((int)hi, 0);
-}
-
-// fp32 -> double by integer operations (exact; zeros / subnormals / non-finite take the
-// conversion instruction)
-__device__ __forceinline__ double f32_to_double_int(float f) {
-  const uint32_t b = __float_as_uint(f);
-  const uint32_t e = (b >> 23) & 0xFFu;
-  if (e == 0u || e == 0xFFu) return (double)f;
-  const uint32_t hi = (b & 0x80000000u) | (((b & 0x7FFFFFFFu) >> 3) + (896u << 20));
-  return __hiloint2double((int)hi, (int)(b << 29));
-}
+// bf16 bit pattern / fp32 -> double.  (The hardware conversion: assembling the double by integer operations was
+// measured and is slower -- about 1 us per call in the refinement kernels, 1.5 us in router_exact_kernel.)
+__device__ __forceinline__ double bf16_bits_to_double(uint32_t b) { return (double)__uint_as_float(b << 16); }
+__device__ __forceinline__ double f32_to_double_int(float f) { return (double)f; }
 
 template <int AFMT>
 __device__ __forceinline__ float load_act1(const void* x, size_t idx) {
@@ -727,8 +714,7 @@ __global__ void __launch_bounds__(kRefineThreads) topk_refine_kernel(Tables T, R
         if (c0 == 0) amax = fmaxf(amax, fmaxf(fmaxf(fabsf(f.x), fabsf(f.y)), fmaxf(fabsf(f.z), fabsf(f.w))));
       }
       // pairs of candidates under a CTA-uniform test: bodies past nc are skipped, not predicated
-      // (top-4 routing refines five or six candidates per token, top-8 about ten); the conversions
-      // to fp64 are integer operations (the fp64 pipe is narrow: its instructions are the cost)
+      // (top-4 routing refines five or six candidates per token, top-8 about ten)
       float4 wv[kRefineCand];
 #pragma unroll
       for (int q0 = 0; q0 < kRefineCand; q0 += 2)
