@@ -48,6 +48,10 @@ constexpr int kFusedCand = 12;         // candidates evaluated per pass over the
 inline int fused_slices(int gamma, int H, int n_sm) {
   int s = 1;
   while (2 * s <= kFusedMaxSlices && 2 * s * gamma <= n_sm && H / (2 * s) >= 256) s *= 2;
+  // Clusters of eight only while they fill at most two thirds of the machine: a cluster needs its SMs in one GPC
+  // at one time, and with 16 clusters of 8 (gamma = 16 on 148 SMs) the launch waited for them -- measured 8 us per
+  // call against clusters of four, which are placed without delay up to a full wave.
+  if (s == 8 && 3 * s * gamma > 2 * n_sm) s = 4;
   return s;
 }
 
