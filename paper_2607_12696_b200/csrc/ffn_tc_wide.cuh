@@ -38,6 +38,7 @@
 
 namespace moev {
 namespace tcw {
+constexpr int kNormalPolicyUnits = 64;  // calls of at least this many units stream the weights with the default L2 policy
 
 using tc::kStageBytes;
 using tc::kTaskQ;
@@ -206,6 +207,12 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
     uint32_t it = 0, q = 0;
     bool ok = true;
     bool first_draw = true;
+    // L2 policy of the weight stream.  An expert with more tokens than a unit holds is streamed once per unit, and
+    // its units are adjacent in the task order: in a large call the default policy lets a later unit find the
+    // expert's weights in the L2 (Zipf routing, 256 rows: expert kernel 1181 -> 1130 us), where "evict first" reads
+    // them again from HBM.  Small calls are faster with "evict first" (gamma = 32, 32 experts: 280 against 303 us): it
+    // keeps the per-unit operand tiles and the h scratch in the L2.
+    const uint64_t wpol = n_units >= kNormalPolicyUnits ? ptx::kPolicyEvictNormal : ptx::kPolicyEvictFirst;
     auto fetch_publish = [&]() -> int {  // lane 0 draws and publishes; every lane learns the id
       int id = -2;
       if (lane == 0) {
@@ -256,8 +263,8 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
           if (lane == 0) {
             uint8_t* dst = w_ring + s * kStageBytes;
             ptx::mbar_arrive_expect_tx(&S.w_full[s], kStageBytes + kBTileBytes);
-            ptx::tma_load_3d(dst, mg, &S.w_full[s], kc * 128, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
-            ptx::tma_load_3d(dst + 16384, mu, &S.w_full[s], kc * 128, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
+            ptx::tma_load_3d(dst, mg, &S.w_full[s], kc * 128, t.slice * 128, u.expert, wpol);
+            ptx::tma_load_3d(dst + 16384, mu, &S.w_full[s], kc * 128, t.slice * 128, u.expert, wpol);
             ptx::tma_load_2d(b_tiles + s * kBTileBytes, &tm_xu, &S.w_full[s], 0, (t.unit * KC + kc) * 64,
                              ptx::kPolicyEvictNormal);
           }
@@ -281,9 +288,9 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
           if (lane == 0) {
             uint8_t* dst = w_ring + s * kStageBytes;
             ptx::mbar_arrive_expect_tx(&S.w_full[s], 16384 * nt + kBTileBytes);
-            ptx::tma_load_3d(dst, md, &S.w_full[s], sl * 128, (2 * t.hp) * 128, u.expert, ptx::kPolicyEvictFirst);
+            ptx::tma_load_3d(dst, md, &S.w_full[s], sl * 128, (2 * t.hp) * 128, u.expert, wpol);
             if (nt == 2)
-              ptx::tma_load_3d(dst + 16384, md, &S.w_full[s], sl * 128, (2 * t.hp + 1) * 128, u.expert, ptx::kPolicyEvictFirst);
+              ptx::tma_load_3d(dst + 16384, md, &S.w_full[s], sl * 128, (2 * t.hp + 1) * 128, u.expert, wpol);
             ptx::tma_load_2d(b_tiles + s * kBTileBytes, &tm_hq, &S.w_full[s], 0, (t.unit * n_slices + sl) * 64,
                              ptx::kPolicyEvictNormal);
           }
