@@ -89,6 +89,34 @@ def test_gptoss_repeated_calls_reuse_scratch():
     v.close()
 
 
+@pytest.mark.parametrize("base,kw,gamma,routing", [
+    ("qwen", dict(H=1024, I=384, E=176, top_k=6), 7, "iid"),        # more experts than SMs: two router rows per CTA; E no multiple of 32
+    ("qwen", dict(H=1024, I=384, E=176, top_k=6), 8, "scattered"),  # exact logits with exact ties
+    ("deepseek", dict(H=512, I=256, E=512), 8, "iid"),              # sixteen experts per lane in the selection
+    ("deepseek", dict(H=512, I=256, E=512), 3, "clustered"),
+    ("deepseek", dict(H=8192, I=256, E=32), 5, "iid"),              # rows of 8192 columns: one full pass of the logit kernel
+    ("gptoss", dict(H=704, I=320, E=32), 2, "iid"),
+    ("tiny", dict(), 8, "iid"), ("tiny", dict(E=24, top_k=24), 4, "iid"),   # fp32 activations; top-k = E
+])
+def test_smallest_calls_fp64_logit_routing(base, kw, gamma, routing):
+    """Calls of at most eight rows take the routing path that evaluates all logits in fp64 (no
+    candidate stage): ids, weights, union, offsets and permutation bit for bit against the oracle,
+    outputs within the format's tolerance, twice on one context (the second call meets the first
+    call's workspace)."""
+    shape = small_shape(base, **kw)
+    w = synth.make_expert_weights(shape, device="cuda")
+    fn = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing, "clustered": synth.make_clustered_routing}[routing]
+    v = moev.MoeVerifier(gcfg(shape, 8))
+    for layer in (0, 1):
+        wr, x = fn(shape, gamma, layer=layer, device="cuda")
+        res = run_gpu(shape, wr, w, x, gamma, verifier=v)
+        ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), gamma)
+        if routing == "iid" and ref.gap.min() <= 1e-9:
+            continue  # a near-tie in the fp64 logits leaves the ids undefined
+        compare(shape, res, ref, gamma)
+    v.close()
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("gamma,U", [(1, 8), (8, 8), (8, 64), (32, 40), (128, 8), (128, 64)])
 def test_exact_union_cases(impl, gamma, U):
