@@ -677,7 +677,9 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
     const dim3 grid((g.E + epc - 1) / epc, (gamma + kExactTok - 1) / kExactTok);
     const size_t xs = (size_t)std::min(gamma, kExactTok) * g.H * (g.afmt == MOEV_ACT_FP32 ? 4 : 2);
     auto go = [&](auto kern) {
-      launch_k(kern, grid, dim3(kExactThreads), xs, st, pdl && c->chain == 1, c->T, x, layer->router_w, c->logits64,
+      // (in a multi-layer call the kernel is launched ahead in both modes: its CTAs need more shared memory than an
+      // expert CTA leaves, so they take their SMs only as that kernel leaves them -- 2 us per layer at gamma = 4)
+      launch_k(kern, grid, dim3(kExactThreads), xs, st, pdl && c->chain != 0, c->T, x, layer->router_w, c->logits64,
                c->y32, gamma, g.H, g.E, c->chain == 2 ? 1 : 0, pf);
     };
     if (g.afmt == MOEV_ACT_FP32) { if (epc == 1) go(router_exact_kernel<MOEV_ACT_FP32, 1>); else go(router_exact_kernel<MOEV_ACT_FP32, 2>); }
