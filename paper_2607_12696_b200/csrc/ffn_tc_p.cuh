@@ -20,6 +20,9 @@
 #include "ffn_tc_wide.cuh"
 #include "ptx.cuh"
 
+#ifndef MOEV_P_LOOK
+#define MOEV_P_LOOK(n) ((n) > 2 ? (n) - 2 : 0)
+#endif
 namespace moev {
 namespace tcp {
 
@@ -178,8 +181,11 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
     TaskDesc td, td_next;
     int id = fetch_publish(td);
     bool first_task = true;
-    // the next task is drawn (a trip to the counter) and published while this task's first stages are in flight
-    const int look_kc = KC - 1 < 3 ? KC - 1 : 3;
+    // The next task is drawn (a trip to the counter) and published while the last stages of this task's down phase
+    // are being requested: early enough for the trip to hide behind them, and as late as possible -- a task bound to a
+    // CTA a whole task ahead waits for that CTA even while others idle at the end of the kernel (clustered tree
+    // workload: the last tasks started 30 us after the other CTAs had run out of work).
+    const int look_ds = MOEV_P_LOOK(n_dstage);
     while (ok && id >= 0) {
       int id_next = -1;
       Unit u;
@@ -199,10 +205,6 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
       int tok = 0;
       if (lane < m) tok = u.shared ? (u.slot0 - (P.A + u.expert * P.gamma) + lane) : __ldg(P.slot_token + u.slot0 + lane);
       for (int kc = 0; kc < KC && ok; ++kc, ++it) {
-        if (kc == look_kc) {
-          id_next = fetch_publish(td_next);
-          if (!ok) break;
-        }
         const int s = it % kStages;
         wait_stage(s);
         if (!ok) break;
@@ -217,6 +219,10 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
           ptx::tma_load_2d(b_tiles + s * kBTileBytes + lane * 256, &tm_xq, &S.w_full[s], kc * 128, 2 * tok, ptx::kPolicyEvictNormal);
       }
       for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
+        if (ds == look_ds) {
+          id_next = fetch_publish(td_next);
+          if (!ok) break;
+        }
         const int s = it % kStages;
         wait_stage(s);
         if (!ok) break;
