@@ -40,6 +40,10 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
+#ifndef MOEV_TC_LOOK
+#define MOEV_TC_LOOK(n) ((n) > 2 ? (n) - 2 : 0)
+#endif
+
 namespace moev {
 namespace tcw {  // two-phase schedule for calls with many tokens per expert (ffn_tc_wide.cuh)
 struct Params {
@@ -403,11 +407,18 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           ptx::tma_load_3d(dst + 16384, mu, &S.w_full[s], kc * F::kBK, t.slice * 128, u.expert, ptx::kPolicyEvictFirst);
         }
       };
-      auto load_down = [&](const TaskDesc& t) {
+      TaskDesc td, td_next, td_nn;
+      int id_nn = -1;
+      auto load_down = [&](const TaskDesc& t, bool draw) {
         const Unit u = P.units[t.unit];
         const int slice = t.slice;
         const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
+        const int look_ds = MOEV_TC_LOOK(n_dstage);
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
+          if (draw && ds == look_ds) {
+            id_nn = fetch_publish(td_nn);
+            if (!ok) break;
+          }
           const int s = it % kStages;
           { MOEV_STAT_BEGIN();
           ok = ptx::bounded_wait(&S.w_empty[s], ((it / kStages) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
@@ -427,9 +438,9 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
           }
         }
       };
-      // Stream order GU(0), GU(1), D(0), GU(2), D(1), ...; task t + 2 is published between the
-      // loads of GU(t + 1) and D(t), one down phase before its own loads begin.
-      TaskDesc td, td_next, td_nn;
+      // Stream order GU(0), GU(1), D(0), GU(2), D(1), ...; task t + 2 is drawn and published while the last stages
+      // of D(t) are requested, just before its own loads begin (as late as the trip to the counter allows: a
+      // task bound to a CTA early waits for that CTA even while others idle at the end of the kernel).
       int id = fetch_publish(td);
       int id_next = -1;
       if (ok && id >= 0) {
@@ -437,14 +448,13 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         if (ok) load_gu(td);
       }
       while (ok && id >= 0) {
-        int id_nn = -1;
+        id_nn = -1;
         if (id_next >= 0) {
           load_gu(td_next);
           if (!ok) break;
-          id_nn = fetch_publish(td_nn);
-          if (!ok) break;
         }
-        load_down(td);
+        load_down(td, id_next >= 0);
+        if (!ok) break;
         id = id_next; td = td_next;
         id_next = id_nn; td_next = td_nn;
       }
