@@ -222,6 +222,19 @@ moev_status moev_profile_enable(moev_ctx* ctx, int32_t on);
 moev_status moev_profile_read(moev_ctx* ctx, void* cuda_stream, double* mean_us /*[6]*/,
                               int32_t* calls);
 
+/* Working time of the tensor-core expert kernel inside a call as the call really runs (the event
+ * records above switch the dependent launches off, so their interval for a kernel includes its
+ * launch gap and its set-up, which a real call hides behind the routing kernels).  With
+ * moev_ffn_span_enable(ctx, 1) every CTA of the expert kernel stores the device's global timer when
+ * the routing kernels release it and when it leaves (two 8-byte stores per CTA and call; nothing
+ * else changes).  moev_ffn_span_read waits for the stream and writes to span_us (host) the time in
+ * microseconds from the earliest release to the latest exit in the most recent call, or 0 when no
+ * tensor-core expert kernel has run with the stamps on (the CUDA-core path does not stamp).  The
+ * paper has no counterpart: a measurement aid for its Fig. 1(a) quantity, latency against the
+ * number of active experts. */
+moev_status moev_ffn_span_enable(moev_ctx* ctx, int32_t on);
+moev_status moev_ffn_span_read(moev_ctx* ctx, void* cuda_stream, double* span_us);
+
 /* Weight prefetch by the first routing kernel (off by default): the shared experts' matrices and
  * those of the layer's predicted_ids are pulled into the L2 while the routing kernels run, so the
  * expert kernel finds them on chip (Sec. 3: the verification cost is expert-weight traffic from

@@ -21,7 +21,8 @@ EXPORTS = ("moev_create", "moev_destroy", "moev_verify", "moev_verify_host", "mo
            "moev_last_error", "moev_expert_bytes", "moev_expert_code_bytes",
            "moev_launches_per_call", "moev_resolved_impl", "moev_profile_enable",
            "moev_profile_read", "moev_route_topk_static", "moev_route_topk_static_scratch_floats", "moev_select_drafts",
-           "moev_verify_pipeline", "moev_prefetch_enable", "moev_verify_chain")
+           "moev_verify_pipeline", "moev_prefetch_enable", "moev_verify_chain", "moev_ffn_span_enable",
+           "moev_ffn_span_read")
 
 
 class MoevError(RuntimeError):
@@ -129,6 +130,10 @@ def lib() -> C.CDLL:
         L.moev_profile_read.restype = C.c_int
         L.moev_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_double),
                                         C.POINTER(C.c_int32)]
+        L.moev_ffn_span_enable.restype = C.c_int
+        L.moev_ffn_span_enable.argtypes = [C.c_void_p, C.c_int32]
+        L.moev_ffn_span_read.restype = C.c_int
+        L.moev_ffn_span_read.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(C.c_double)]
         L.moev_route_topk_static.restype = C.c_int
         L.moev_route_topk_static.argtypes = [C.POINTER(_Config), C.c_void_p, C.c_void_p, C.c_int32,
                                              C.c_void_p, C.c_void_p, C.c_void_p]
@@ -311,6 +316,14 @@ class MoeVerifier:
 
     def profile_enable(self, on: bool):
         self._check(lib().moev_profile_enable(self._h, int(on)))
+
+    def ffn_span_enable(self, on: bool):
+        self._check(lib().moev_ffn_span_enable(self._h, int(on)))
+
+    def ffn_span_read(self) -> float:
+        us = C.c_double()
+        self._check(lib().moev_ffn_span_read(self._h, self._stream(), C.byref(us)))
+        return us.value
 
     def profile_read(self):
         us = (C.c_double * 6)()

@@ -116,6 +116,7 @@ struct Params {
   int32_t actq;         // moev_act_quant: FP8 1x128 activations (single e4m3 term, block scales in xs)
   const float* xs;      // [gamma, H / 128] activation block scales (actq != 0)
   int32_t units_alloc;  // entries allocated behind `units` (reads ahead of the unit count stay below it)
+  unsigned long long* span;  // [grid][2] or null: global-timer stamps of every CTA, released by the routing kernels | leaving
 #ifdef MOEV_TC_STATS
   unsigned long long* stats;  // [grid][16] cycles the MMA thread spent per wait / issue class (debug builds)
 #endif
@@ -318,6 +319,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   MOEV_TC_MARK(25);
+  if (P.span && tid == 0) P.span[2 * blockIdx.x] = ptx::globaltimer_ns();
   // (fp8 schedule without producers: the TMA warp asks for the records of the first units, and of the unit this
   // CTA's first task has in large calls, together with the loads that decide the schedule: one trip to the L2)
   Unit u_first{};
@@ -335,6 +337,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, kTmemCols);
       }
+      if (P.span && tid == 0) P.span[2 * blockIdx.x + 1] = ptx::globaltimer_ns();
       return;
     }
 #ifndef MOEV_FP8_FOLD_SCALE
@@ -353,6 +356,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem, kTmemCols);
       }
+      if (P.span && tid == 0) P.span[2 * blockIdx.x + 1] = ptx::globaltimer_ns();
       return;
     }
 #endif
@@ -939,6 +943,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     ptx::tc_fence_after();
     ptx::tmem_dealloc(tmem, kTmemCols);
   }
+  if (P.span && tid == 0) P.span[2 * blockIdx.x + 1] = ptx::globaltimer_ns();
 }
 
 }  // namespace tc

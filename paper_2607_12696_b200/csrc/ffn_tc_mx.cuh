@@ -109,6 +109,7 @@ struct Params {
   int32_t* unit_done;   // [max_units] phase-1 tasks finished per unit (zeroed per call by the grouping kernel)
   int32_t hq_stride;    // I / 2
   int32_t ffn_kind;
+  unsigned long long* span;  // [grid][2] or null: global-timer stamps of every CTA, released by the routing kernels | leaving
   int32_t* status;
   int32_t gamma, H, I, A;
 #ifdef MOEV_TC_STATS
@@ -250,6 +251,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
   asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (tid == 0) MOEV_MX_MARK(26);
+  if (P.span && tid == 0) P.span[2 * blockIdx.x] = ptx::globaltimer_ns();
   const int n_units = *P.n_units;
   const int n_p1 = n_units * n_slices;
   const int n_ids = n_p1 + n_units * n_pairs;
@@ -736,6 +738,7 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
     ptx::tmem_dealloc(tmem, kTmemCols);
   }
   if (tid == 0) MOEV_MX_MARK(29);
+  if (P.span && tid == 0) P.span[2 * blockIdx.x + 1] = ptx::globaltimer_ns();
 }
 
 }  // namespace tcmx

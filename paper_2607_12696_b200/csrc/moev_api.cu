@@ -70,6 +70,8 @@ struct moev_ctx {
   int n_sm = 0;
   int unit_cap = 1 << 20;
   bool profile = false;
+  bool span_on = false;              // the tensor-core expert kernel stamps its CTAs' release and exit (moev_ffn_span_*)
+  unsigned long long* span = nullptr;  // [n_sm][2] device
   bool prefetch = false;  // L2 prefetch of shared / predicted experts' weights by the first routing kernel
   int chain = 0;  // next moev_verify is a later layer of a multi-layer call: its first kernel is a dependent launch
                   // (1: independent inputs, the kernel waits for the previous layer at its end; 2: its input is the
@@ -299,6 +301,7 @@ void launch_tc_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.wide = c->wide_ok ? c->T.wide : nullptr;
   P.xq_ready = (c->wide_ok && c->T.xq) ? 1 : 0;
   P.actq = g.act_quant; P.xs = c->T.xs; P.units_alloc = (int32_t)c->max_units;
+  P.span = c->span_on ? c->span : nullptr;
   // arguments of the two-phase schedule, which the kernel switches to when the grouping kernel's
   // flag says that the call has many tokens per streamed expert (fp8 only)
   tcw::Params W{};
@@ -331,6 +334,7 @@ void launch_mx_ffn(moev_ctx* c, const TmapSet* tm, const moev_layer* L, const vo
   P.sh_s_gate = static_cast<const uint8_t*>(L->sh_s_gate); P.sh_s_up = static_cast<const uint8_t*>(L->sh_s_up);
   P.sh_s_down = static_cast<const uint8_t*>(L->sh_s_down);
   P.b_gate = L->b_gate; P.b_up = L->b_up; P.b_down = L->b_down; P.ffn_kind = g.ffn_kind;
+  P.span = c->span_on ? c->span : nullptr;
   P.status = c->T.status; P.gamma = gamma; P.H = g.H; P.I = g.I; P.A = gamma * g.top_k;
 #ifdef MOEV_TC_STATS
   P.stats = c->tc_stats;
@@ -526,6 +530,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && cudaMalloc(&c->x_stage, G * cfg->H * act_b) == cudaSuccess;
   ok = ok && cudaMalloc(&c->y_stage, G * cfg->H * act_b) == cudaSuccess;
   ok = ok && cudaMallocHost(reinterpret_cast<void**>(&c->host_word), 4 * sizeof(int32_t)) == cudaSuccess;
+  ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->span), (size_t)c->n_sm * 2 * sizeof(unsigned long long)) == cudaSuccess;
+  ok = ok && cudaMemset(c->span, 0, (size_t)c->n_sm * 2 * sizeof(unsigned long long)) == cudaSuccess;
   if (ok) ok = cudaMemset(c->T.status, 0, sizeof(int32_t)) == cudaSuccess;
 #ifdef MOEV_TC_STATS
   ok = ok && cudaMalloc(reinterpret_cast<void**>(&c->tc_stats), (size_t)c->n_sm * 16 * sizeof(unsigned long long)) == cudaSuccess;
@@ -587,7 +593,7 @@ moev_status moev_destroy(moev_ctx* c) {
   cudaFree(c->T.n_active); cudaFree(c->T.status); cudaFree(c->T.tok_scale); cudaFree(c->T.xq);
   cudaFree(c->T.n_units); cudaFree(c->T.units); cudaFree(c->T.task_counter); cudaFree(c->hbuf); cudaFree(c->y32);
   cudaFree(c->T.wide); cudaFree(c->T.unit_done); cudaFree(c->hq); cudaFree(c->hq_f); cudaFree(c->xu); cudaFree(c->hexp); cudaFree(c->xhat); cudaFree(c->T.xs);
-  cudaFree(c->x_stage); cudaFree(c->y_stage);
+  cudaFree(c->x_stage); cudaFree(c->y_stage); cudaFree(c->span);
   if (c->host_word) cudaFreeHost(c->host_word);
   if (c->prof_events_ready)
     for (int i = 0; i < kProfSlots; ++i)
@@ -1008,6 +1014,31 @@ moev_status moev_profile_enable(moev_ctx* c, int32_t on) {
   }
   c->profile = on != 0;
   c->prof_n = 0;
+  return MOEV_OK;
+}
+
+moev_status moev_ffn_span_enable(moev_ctx* c, int32_t on) {
+  if (!c) return MOEV_EINVAL;
+  c->span_on = on != 0;
+  return MOEV_OK;
+}
+
+moev_status moev_ffn_span_read(moev_ctx* c, void* cuda_stream, double* span_us) {
+  if (!c || !span_us) return MOEV_EINVAL;
+  *span_us = 0.0;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned long long host[2 * 1024];
+  if (c->n_sm > 1024) return fail(c, MOEV_EUNSUPPORTED, "more SMs than the span buffer holds");
+  cudaError_t e = cudaMemcpyAsync(host, c->span, (size_t)c->n_sm * 2 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return fail(c, MOEV_ECUDA, "span read failed: %s", cudaGetErrorString(e));
+  unsigned long long first = ~0ull, last = 0ull;
+  for (int i = 0; i < c->n_sm; ++i) {
+    if (host[2 * i] == 0ull || host[2 * i + 1] == 0ull) continue;  // no tensor-core expert kernel has run with the stamps on
+    first = host[2 * i] < first ? host[2 * i] : first;
+    last = host[2 * i + 1] > last ? host[2 * i + 1] : last;
+  }
+  if (last > first) *span_us = (double)(last - first) * 1e-3;
   return MOEV_OK;
 }
 

@@ -256,6 +256,32 @@ def test_chained_dependent_layers_match_oracle(base, kw, gamma, prefetch):
     v.close()
 
 
+def test_expert_kernel_span_stamps():
+    """moev_ffn_span_*: with the stamps on, the expert kernel's working time of the last call is positive and
+    shorter than the call; the results do not change; off again, the stamps stay as they were."""
+    shape = small_shape("deepseek", H=1024, I=512, E=64)
+    gamma = 8
+    v = moev.MoeVerifier(gcfg(shape, gamma))
+    assert v.ffn_span_read() == 0.0
+    w = synth.make_expert_weights(shape, device="cuda")
+    wr, x = synth.make_iid_routing(shape, gamma, device="cuda")
+    ref = oracle.moe_verify(ocfg(shape), synth.layer_to_numpy(wr, w), synth.to_numpy(x), gamma)
+    v.ffn_span_enable(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    res = run_gpu(shape, wr, w, x, gamma, verifier=v)   # warm-up
+    e0.record()
+    res = run_gpu(shape, wr, w, x, gamma, verifier=v)
+    e1.record()
+    torch.cuda.synchronize()
+    span = v.ffn_span_read()
+    assert 0.0 < span < e0.elapsed_time(e1) * 1e3
+    compare(shape, res, ref, gamma)
+    v.ffn_span_enable(False)
+    run_gpu(shape, wr, w, x, gamma, verifier=v)
+    assert v.ffn_span_read() == span
+    v.close()
+
+
 def test_context_reuse_and_smaller_gamma():
     """One context, several calls with different gamma: workspace state must not leak."""
     shape = small_shape("qwen", H=512, I=256, E=16, top_k=4)
