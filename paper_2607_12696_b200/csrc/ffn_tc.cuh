@@ -40,10 +40,6 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
-#ifndef MOEV_TC_LOOK
-#define MOEV_TC_LOOK(n) ((n) > 2 ? (n) - 2 : 0)
-#endif
-
 namespace moev {
 namespace tcw {  // two-phase schedule for calls with many tokens per expert (ffn_tc_wide.cuh)
 struct Params {
@@ -417,7 +413,7 @@ grouped_ffn_tc_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
         const Unit u = P.units[t.unit];
         const int slice = t.slice;
         const CUtensorMap* md = u.shared ? &tm_sh_down : &tm_down;
-        const int look_ds = MOEV_TC_LOOK(n_dstage);
+        const int look_ds = n_dstage > 2 ? n_dstage - 2 : 0;
         for (int ds = 0; ds < n_dstage && ok; ++ds, ++it) {
           if (draw && ds == look_ds) {
             id_nn = fetch_publish(td_nn);

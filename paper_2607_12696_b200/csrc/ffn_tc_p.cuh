@@ -20,9 +20,6 @@
 #include "ffn_tc_wide.cuh"
 #include "ptx.cuh"
 
-#ifndef MOEV_P_LOOK
-#define MOEV_P_LOOK(n) ((n) > 2 ? (n) - 2 : 0)
-#endif
 namespace moev {
 namespace tcp {
 
@@ -185,7 +182,7 @@ __device__ void promote_body(const CUtensorMap& tm_gate, const CUtensorMap& tm_u
     // are being requested: early enough for the trip to hide behind them, and as late as possible -- a task bound to a
     // CTA a whole task ahead waits for that CTA even while others idle at the end of the kernel (clustered tree
     // workload: the last tasks started 30 us after the other CTAs had run out of work).
-    const int look_ds = MOEV_P_LOOK(n_dstage);
+    const int look_ds = n_dstage > 2 ? n_dstage - 2 : 0;
     while (ok && id >= 0) {
       int id_next = -1;
       Unit u;
