@@ -431,7 +431,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     // exact-logit routing of the smallest calls: rows of x staged in shared memory by 16-byte copies
     c->exact_ok = exact_smem(cfg->H, (int)act_b) <= kExactMaxSmem && (cfg->H * act_b) % 16 == 0 && cfg->H % 4 == 0;
     if (c->exact_ok)
-      ok = ok && dmalloc(&c->logits64, (size_t)std::min<int>(cfg->max_tokens, kExactMaxTokens) * E) == cudaSuccess;
+      ok = ok && dmalloc(&c->logits64, (size_t)std::min<int>(cfg->max_tokens, kExactTokWide) * E) == cudaSuccess;
   }
   ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
@@ -559,6 +559,9 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
         } else {
           ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, xs) == cudaSuccess;
           ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_BF16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, xs) == cudaSuccess;
+          if (exact_tokens_per_cta(kExactTokWide, cfg->H, (int)act_b, cfg->E, c->n_sm) == kExactTokWide)
+            ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_BF16, 1, kExactTokWide>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            (int)exact_smem(cfg->H, (int)act_b, kExactTokWide)) == cudaSuccess;
         }
         ok = ok && cudaFuncSetAttribute(route_select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
@@ -677,18 +680,22 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
     if (mat_bytes % 16) { pf.n_shared = 0; pf.n_pred = 0; }
   }
   const int wide_ratio = (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0;
-  if (c->exact_ok && g.n_group == 0 && gamma <= kExactMaxTokens) {
+  const int act_bytes = g.afmt == MOEV_ACT_FP32 ? 4 : 2;
+  const int exact_tok = (c->exact_ok && g.n_group == 0 && (g.afmt == MOEV_ACT_BF16 || gamma <= kExactMaxTokens))
+                            ? exact_tokens_per_cta(gamma, g.H, act_bytes, g.E, c->n_sm) : 0;
+  if (exact_tok > 0) {
     // the smallest calls: fp64 logits in one pass, selection and grouping by one CTA (route_exact.cuh)
     const int epc = exact_epc(g.E, c->n_sm);
-    const dim3 grid((g.E + epc - 1) / epc, (gamma + kExactTok - 1) / kExactTok);
-    const size_t xs = (size_t)std::min(gamma, kExactTok) * g.H * (g.afmt == MOEV_ACT_FP32 ? 4 : 2);
+    const dim3 grid((g.E + epc - 1) / epc, (gamma + exact_tok - 1) / exact_tok);
+    const size_t xs = (size_t)std::min(gamma, exact_tok) * g.H * act_bytes;
     auto go = [&](auto kern) {
       // (in a multi-layer call the kernel is launched ahead in both modes: its CTAs need more shared memory than an
       // expert CTA leaves, so they take their SMs only as that kernel leaves them -- 2 us per layer at gamma = 4)
       launch_k(kern, grid, dim3(kExactThreads), xs, st, pdl && c->chain != 0, c->T, x, layer->router_w, c->logits64,
                c->y32, gamma, g.H, g.E, c->chain == 2 ? 1 : 0, pf);
     };
-    if (g.afmt == MOEV_ACT_FP32) { if (epc == 1) go(router_exact_kernel<MOEV_ACT_FP32, 1>); else go(router_exact_kernel<MOEV_ACT_FP32, 2>); }
+    if (exact_tok == kExactTokWide) go(router_exact_kernel<MOEV_ACT_BF16, 1, kExactTokWide>);
+    else if (g.afmt == MOEV_ACT_FP32) { if (epc == 1) go(router_exact_kernel<MOEV_ACT_FP32, 1>); else go(router_exact_kernel<MOEV_ACT_FP32, 2>); }
     else { if (epc == 1) go(router_exact_kernel<MOEV_ACT_BF16, 1>); else go(router_exact_kernel<MOEV_ACT_BF16, 2>); }
     if (ev) cudaEventRecord(ev[1], st);
     {

@@ -35,15 +35,24 @@ namespace moev {
 constexpr int kExactThreads = 512;
 constexpr int kExactWarps = kExactThreads / 32;
 constexpr int kExactTok = 8;            // tokens per CTA
+constexpr int kExactTokWide = 16;       // ... when a CTA holds one router row and 16 rows of x fit its shared memory
 constexpr int kExactG = 4;              // 4-column groups per thread and pass: a pass covers 8192 columns
 #ifndef MOEV_EXACT_MAX_TOKENS
 #define MOEV_EXACT_MAX_TOKENS 8
 #endif
-constexpr int kExactMaxTokens = MOEV_EXACT_MAX_TOKENS;   // rows per call served by this path
+constexpr int kExactMaxTokens = MOEV_EXACT_MAX_TOKENS;   // rows per call served by this path (16 with kExactTokWide)
 constexpr size_t kExactMaxSmem = 200 * 1024;
 
 inline int exact_epc(int E, int n_sm) { return E > n_sm ? 2 : 1; }   // router rows per CTA: one wave of CTAs
-inline size_t exact_smem(int H, int act_bytes) { return (size_t)kExactTok * H * act_bytes; }
+inline size_t exact_smem(int H, int act_bytes, int tok = kExactTok) { return (size_t)tok * H * act_bytes; }
+// Rows per CTA for a call of gamma rows, or 0 when the call takes another routing path: 8 rows per CTA up to
+// kExactMaxTokens; 16 rows up to 16 where a CTA holds one router row (E <= SMs) and 16 rows of x fit (measured
+// on the GPT-OSS router shape at gamma = 16 against the cluster path; with two token groups of 8 the cluster path wins).
+inline int exact_tokens_per_cta(int gamma, int H, int act_bytes, int E, int n_sm) {
+  if (gamma <= kExactMaxTokens) return kExactTok;
+  if (gamma <= kExactTokWide && exact_epc(E, n_sm) == 1 && exact_smem(H, act_bytes, kExactTokWide) <= kExactMaxSmem) return kExactTokWide;
+  return 0;
+}
 
 // Four consecutive activations of a staged row as doubles; mag keeps the running maximum of |x| in an integer form
 // that orders like the magnitudes: bf16: two 15-bit magnitudes per word (packed 16-bit maxima); fp32: the bits of |x|.
@@ -68,20 +77,20 @@ __device__ __forceinline__ uint32_t mag_bits(uint32_t mag) {
   else return mag;
 }
 
-template <int AFMT, int EPC>
+template <int AFMT, int EPC, int NT = kExactTok>
 __global__ void __launch_bounds__(kExactThreads, 1) router_exact_kernel(
     Tables T, const void* __restrict__ x, const float* __restrict__ router_w, double* __restrict__ logits,
     float* __restrict__ y32, int gamma, int H, int E, int wait_first, PrefetchArgs pf) {
   extern __shared__ __align__(16) uint8_t xs_raw[];            // [nt][H] activations of this CTA's tokens
   __shared__ double red[kExactWarps][16];
-  __shared__ uint32_t amax_w[kExactWarps][kExactTok];
-  __shared__ float amax_s[kExactTok];
+  __shared__ uint32_t amax_w[kExactWarps][NT];
+  __shared__ float amax_s[NT];
   constexpr int ASZ = AFMT == MOEV_ACT_FP32 ? 4 : 2;
-  constexpr int NA = kExactTok * EPC;                          // accumulators per thread (at most 16)
+  constexpr int NA = NT * EPC;                          // accumulators per thread (at most 16)
   static_assert(NA <= 16, "one reduce-scatter serves all accumulators");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int e0 = blockIdx.x * EPC;
-  const int t0 = blockIdx.y * kExactTok, nt = min(kExactTok, gamma - t0);
+  const int t0 = blockIdx.y * NT, nt = min(NT, gamma - t0);
   const int G4 = H / 4;
   const size_t row_bytes = (size_t)H * ASZ;
 
@@ -108,9 +117,9 @@ __global__ void __launch_bounds__(kExactThreads, 1) router_exact_kernel(
   double acc[16];
 #pragma unroll
   for (int q = 0; q < 16; ++q) acc[q] = 0.0;
-  uint32_t mag[kExactTok];
+  uint32_t mag[NT];
 #pragma unroll
-  for (int t = 0; t < kExactTok; ++t) mag[t] = 0u;
+  for (int t = 0; t < NT; ++t) mag[t] = 0u;
 
   for (int g0 = 0; g0 < G4; g0 += kExactG * kExactThreads) {
     // the thread's router weights of this pass, all loads in flight before the first use
@@ -139,7 +148,7 @@ __global__ void __launch_bounds__(kExactThreads, 1) router_exact_kernel(
           wd[e][2] = (double)wv[e][i].z; wd[e][3] = (double)wv[e][i].w;
         }
 #pragma unroll
-        for (int t = 0; t < kExactTok; ++t) {
+        for (int t = 0; t < NT; ++t) {
           if (t < nt) {   // uniform over the CTA
             double xd[4];
             staged_x4<AFMT>(xs_raw + (size_t)t * row_bytes, g4, xd, mag[t]);
@@ -165,13 +174,13 @@ __global__ void __launch_bounds__(kExactThreads, 1) router_exact_kernel(
     if ((lane & 1) == 0) red[warp][q] = a;
     // (the tokens' max |x| of this CTA's copy of their rows, for the quantisation below)
 #pragma unroll
-    for (int t = 0; t < kExactTok; ++t) {
+    for (int t = 0; t < NT; ++t) {
       const uint32_t m = __reduce_max_sync(0xffffffffu, mag_bits<AFMT>(mag[t]));
       if (lane == 0) amax_w[warp][t] = m;
     }
   }
   __syncthreads();
-  if (tid >= 32 && tid < 32 + kExactTok) {
+  if (tid >= 32 && tid < 32 + NT) {
     uint32_t a = 0u;
 #pragma unroll
     for (int w = 0; w < kExactWarps; ++w) a = max(a, amax_w[w][tid - 32]);

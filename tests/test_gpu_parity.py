@@ -97,16 +97,18 @@ def test_gptoss_repeated_calls_reuse_scratch():
     ("deepseek", dict(H=8192, I=256, E=32), 5, "iid"),              # rows of 8192 columns: one full pass of the logit kernel
     ("gptoss", dict(H=704, I=320, E=32), 2, "iid"),
     ("tiny", dict(), 8, "iid"), ("tiny", dict(E=24, top_k=24), 4, "iid"),   # fp32 activations; top-k = E
+    ("gptoss", dict(H=704, I=320, E=32), 13, "iid"),                # 9 to 16 rows, one router row per CTA: 16 rows of x per CTA
+    ("qwen", dict(H=1024, I=384, E=96), 16, "scattered"),
 ])
 def test_smallest_calls_fp64_logit_routing(base, kw, gamma, routing):
-    """Calls of at most eight rows take the routing path that evaluates all logits in fp64 (no
-    candidate stage): ids, weights, union, offsets and permutation bit for bit against the oracle,
+    """Calls of at most eight rows (sixteen where a CTA holds one router row and the rows fit its
+    shared memory) take the routing path that evaluates all logits in fp64 (no candidate stage): ids, weights, union, offsets and permutation bit for bit against the oracle,
     outputs within the format's tolerance, twice on one context (the second call meets the first
     call's workspace)."""
     shape = small_shape(base, **kw)
     w = synth.make_expert_weights(shape, device="cuda")
     fn = {"iid": synth.make_iid_routing, "scattered": synth.make_scattered_routing, "clustered": synth.make_clustered_routing}[routing]
-    v = moev.MoeVerifier(gcfg(shape, 8))
+    v = moev.MoeVerifier(gcfg(shape, 16))
     for layer in (0, 1):
         wr, x = fn(shape, gamma, layer=layer, device="cuda")
         res = run_gpu(shape, wr, w, x, gamma, verifier=v)
