@@ -119,6 +119,15 @@ def test_smallest_calls_fp64_logit_routing(base, kw, gamma, routing):
     v.close()
 
 
+@pytest.mark.parametrize("gamma,routing", [(10, "iid"), (14, "scattered"), (29, "clustered")])
+def test_cluster_routing_path_with_two_router_rows_per_cta_shape(gamma, routing):
+    """9 to 32 rows on a shape the fp64-logit path does not take beyond 8 rows (more experts than SMs):
+    split-K partials + refinement by a thread-block cluster per token, with clusters of eight (10 rows),
+    of four because eight would not fit two thirds of the machine (14 rows), and of two (29 rows)."""
+    shape = small_shape("deepseek", H=2048, I=256, E=256)
+    parity_case(shape, gamma, routing=routing)
+
+
 @pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("gamma,U", [(1, 8), (8, 8), (8, 64), (32, 40), (128, 8), (128, 64)])
 def test_exact_union_cases(impl, gamma, U):
