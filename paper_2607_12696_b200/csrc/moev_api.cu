@@ -679,6 +679,13 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
                     ? (int)std::min<size_t>(layer->n_predicted, budget - pf.n_shared) : 0;
     if (mat_bytes % 16) { pf.n_shared = 0; pf.n_pred = 0; }
   }
+  // The first kernel of a call.  A later layer of a multi-layer call with independent inputs (chain 1) runs beside
+  // the previous layer's expert kernel and waits for it at its end.  Otherwise the kernel waits before it reads x,
+  // and is launched ahead of its predecessor's end wherever that pays: behind this library's own finalize kernel
+  // (which releases its dependents at once) the launch latency then hides; behind any other kernel the attribute
+  // changes nothing, since a kernel that never releases its dependents does so when it ends.
+  const int wait_first = c->chain == 1 ? 0 : 1;
+  const bool ahead = pdl;   // (single calls too: back-to-back calls on one stream, 215.6 -> 213.0 us per call at gamma = 4)
   const int wide_ratio = (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0;
   const int act_bytes = g.afmt == MOEV_ACT_FP32 ? 4 : 2;
   const int exact_tok = (c->exact_ok && g.n_group == 0 && (g.afmt == MOEV_ACT_BF16 || gamma <= kExactMaxTokens))
@@ -691,8 +698,8 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
     auto go = [&](auto kern) {
       // (in a multi-layer call the kernel is launched ahead in both modes: its CTAs need more shared memory than an
       // expert CTA leaves, so they take their SMs only as that kernel leaves them -- 2 us per layer at gamma = 4)
-      launch_k(kern, grid, dim3(kExactThreads), xs, st, pdl && c->chain != 0, c->T, x, layer->router_w, c->logits64,
-               c->y32, gamma, g.H, g.E, c->chain == 2 ? 1 : 0, pf);
+      launch_k(kern, grid, dim3(kExactThreads), xs, st, ahead, c->T, x, layer->router_w, c->logits64,
+               c->y32, gamma, g.H, g.E, wait_first, pf);
     };
     if (exact_tok == kExactTokWide) go(router_exact_kernel<MOEV_ACT_BF16, 1, kExactTokWide>);
     else if (g.afmt == MOEV_ACT_FP32) { if (epc == 1) go(router_exact_kernel<MOEV_ACT_FP32, 1>); else go(router_exact_kernel<MOEV_ACT_FP32, 2>); }
@@ -707,8 +714,8 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
     if (ev) cudaEventRecord(ev[2], st);
   } else {
     if (g.afmt == MOEV_ACT_FP32)
-      launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, pdl && c->chain != 0, x, layer->router_w,
-               c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+      launch_k(router_partial_kernel<MOEV_ACT_FP32>, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256), rp_smem, st, ahead, x, layer->router_w,
+               c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, wait_first, pf);
     else if (gamma <= 32) {
       // tree-sized calls: the variant without shared memory (one trip to memory long)
       // (a dependent layer's first kernel is not launched ahead at these sizes: its CTAs, resident and waiting beside
@@ -716,15 +723,15 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
       // layer at gamma = 4, against -2 % at gamma = 64)
       auto go = [&](auto kern) {
         launch_k(kern, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(128), 0, st, pdl && c->chain == 1,
-                 static_cast<const uint16_t*>(x), layer->router_w, c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+                 static_cast<const uint16_t*>(x), layer->router_w, c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, wait_first, pf);
       };
       if (gamma <= 8) go(router_partial_small_kernel<1>);
       else if (gamma <= 16) go(router_partial_small_kernel<2>);
       else go(router_partial_small_kernel<4>);
     } else
       launch_k(router_partial_mma_kernel, dim3(c->n_slices, (g.E + kRouterETile - 1) / kRouterETile), dim3(256),
-               router_partial_mma_smem(c->ks), st, pdl && c->chain != 0, static_cast<const uint16_t*>(x), layer->router_w,
-               c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, c->chain == 2 ? 1 : 0, pf);
+               router_partial_mma_smem(c->ks), st, ahead, static_cast<const uint16_t*>(x), layer->router_w,
+               c->part, c->part_x2, c->part_w2, gamma, g.H, g.E, c->ks, wait_first, pf);
     if (ev) cudaEventRecord(ev[1], st);
     const int refine_depth = g.afmt == MOEV_ACT_FP32 ? c->ks : 6 * c->ks + c->n_slices + 12;
     if (g.n_group == 0 && gamma <= kFusedMaxTokens) {
