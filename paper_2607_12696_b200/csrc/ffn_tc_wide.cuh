@@ -56,7 +56,10 @@ constexpr int kMC = 32;                    // tokens per unit
 constexpr int kMaxSlices = 32;             // I <= 4096 (larger layers keep the ffn_tc.cuh schedule)
 constexpr int kMaxChunks = 128;            // H <= 16384
 constexpr int kGath = 8;                   // pieces a unit's operand tiles are gathered in (K ranges)
-constexpr int kColXchg = 256;              // TMEM: partial buffers 2 x (64 | 64) | 32 columns to hand P to the gate group
+constexpr int kPartBufs = 3;               // TMEM partial buffers: the MMA issuers run this many stages ahead of the epilogue groups
+                                           // (three against two: 1 % on the batched workloads -- the epilogue's own TMEM reads bound the stage)
+constexpr int kColXchg = kPartBufs * 128;  // TMEM: partial buffers kPartBufs x (64 | 64) | 32 columns to hand P to the gate group
+static_assert(kColXchg + 32 <= 512, "TMEM budget");
 constexpr int kTileBytes = kStages * kStageBytes + kStages * kBTileBytes;
 constexpr int kCtlBytes = 12 * 1024;
 constexpr int kSmemBytes = kTileBytes + 1024 + kCtlBytes;
@@ -64,7 +67,7 @@ static_assert(kSmemBytes <= tc::kSmemBytes && kThreads == tc::kThreads, "runs in
 
 struct Smem {
   uint64_t w_full[kStages], w_empty[kStages];
-  uint64_t p_full[2], p_empty[2];      // TMEM partial buffers: MMA issuers -> both epilogue groups
+  uint64_t p_full[kPartBufs], p_empty[kPartBufs];      // TMEM partial buffers: MMA issuers -> both epilogue groups
   uint64_t x_full, x_empty;            // P values of a phase-1 task: group 1 -> group 0
   uint64_t tq_full[kTaskQ], tq_empty[kTaskQ];
   uint64_t ep_bar;                     // barrier of group 0 (128 threads)
@@ -156,7 +159,7 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
   __syncthreads();  // every thread has left the caller's use of shared memory
   if (tid == 0) {
     for (int i = 0; i < kStages; ++i) { ptx::mbar_init(&S.w_full[i], 1); ptx::mbar_init(&S.w_empty[i], 2); }
-    for (int i = 0; i < 2; ++i) { ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 8); }
+    for (int i = 0; i < kPartBufs; ++i) { ptx::mbar_init(&S.p_full[i], 2); ptx::mbar_init(&S.p_empty[i], 8); }
     ptx::mbar_init(&S.x_full, 4); ptx::mbar_init(&S.x_empty, 4);
     for (int i = 0; i < kTaskQ; ++i) { ptx::mbar_init(&S.tq_full[i], 1); ptx::mbar_init(&S.tq_empty[i], 258); }
     ptx::mbar_init(&S.ep_bar, 128);
@@ -327,12 +330,12 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
         const int n_st = t.phase2 ? n_slices : KC;
         const bool mine = !t.phase2 || issuer == 0 || 2 * t.hp + 1 < HT;  // an odd last H tile has no partner
         for (int st = 0; st < n_st && ok; ++st, ++it) {
-          const int s = it % kStages, pb = it & 1;
+          const int s = it % kStages, pb = it % kPartBufs;
           { MOEV_STAT_BEGIN();
             ok = ptx::bounded_wait(&S.w_full[s], (it / kStages) & 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             if (t.phase2) { MOEV_STAT_END(5); } else { MOEV_STAT_END(1); } }
           { MOEV_STAT_BEGIN();
-            ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((it >> 1) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
+            ok = ok && ptx::bounded_wait(&S.p_empty[pb], ((it / kPartBufs) & 1) ^ 1, abortp, P.status, kStatusTimeout, kWaitBudgetNs);
             if (t.phase2) { MOEV_STAT_END(6); } else { MOEV_STAT_END(3); } }
           if (!ok) break;
           ptx::tc_fence_after();
@@ -419,11 +422,11 @@ __device__ __noinline__ void wide_body(const CUtensorMap& tm_gate, const CUtenso
 #pragma unroll
       for (int r = 0; r < kMC; ++r) acc[r] = 0.f;
       for (int st = 0; st < n_st && ok; ++st, ++it) {
-        const int pb = it & 1;
+        const int pb = it % kPartBufs;
 #ifdef MOEV_TC_STATS
         const long long e0 = clock64();
 #endif
-        ok = warp_wait(&S.p_full[pb], (it >> 1) & 1, abortp, P.status);
+        ok = warp_wait(&S.p_full[pb], (it / kPartBufs) & 1, abortp, P.status);
 #ifdef MOEV_TC_STATS
         est[0] += clock64() - e0;
         est[2] += 1;
