@@ -68,11 +68,11 @@ DEFAULT_WORKLOAD = "deepseek_fp8_g64_scattered"
 
 # DRAM (read + write) bytes per algorithmic byte of the dominant kernel, from the committed ncu
 # capture of a smaller case of the same kernel (profiles/grouped_ffn_tc_fp8_E64_g16.md:
-# 2.444742 GB + 4.01 MB against 2.422802 GB); traffic grows in proportion to the experts
+# 2.430690 GB + 5.26 MB against 2.422802 GB); traffic grows in proportion to the experts
 # streamed, so the full-size launch is scaled by the same ratio.  Absent = not captured.
-NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.444742e9 + 4.011520e6) / 2.422801920e9,
-                     # profiles/grouped_ffn_mx_gptoss_g64.md: 1.518134 GB + 4.46 MB against 1.454112 GB
-                     ("mxfp4", "tcgen05"): (1.518134e9 + 4.463104e6) / 1.454112e9,
+NCU_TRAFFIC_RATIO = {("fp8_e4m3", "tcgen05"): (2.430690e9 + 5.261312e6) / 2.422801920e9,
+                     # profiles/grouped_ffn_mx_gptoss_g64.md: 1.462642 GB + 6.70 MB against 1.454112 GB
+                     ("mxfp4", "tcgen05"): (1.462642e9 + 6.703872e6) / 1.454112e9,
                      # profiles/grouped_ffn_tc_bf16_E64_g16.md: 2.115337 GB + 3.93 MB against 2.113929 GB
                      ("bf16", "tcgen05"): (2.115337e9 + 3.926784e6) / 2.113929216e9}
 
