@@ -379,6 +379,9 @@ grouped_ffn_mx_kernel(const __grid_constant__ CUtensorMap tm_gate, const __grid_
             if (t.phase == 1) { MOEV_STAT_END(2); } else { MOEV_STAT_END(12); } }
           if (!ok) break;
           ptx::tc_fence_after();
+#ifdef MOEV_TC_STATS
+          if (it == 0 && issuer == 0 && blockIdx.x == 0) g_rt_stats[23] = debug_gtime();
+#endif
           { MOEV_STAT_BEGIN();
           const uint32_t sfa = tmem + kColSf + 16 * s + 8 * issuer;
           const uint32_t atoms = ptx::smem_u32(sf_atoms) + (uint32_t)((4 * s + 2 * issuer) * kSfAtomBytes);
