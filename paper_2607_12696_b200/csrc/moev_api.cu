@@ -421,15 +421,20 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && dmalloc(&c->part, (size_t)c->n_slices * G * E) == cudaSuccess;
   ok = ok && dmalloc(&c->part_x2, (size_t)c->n_slices * G) == cudaSuccess;
   ok = ok && dmalloc(&c->part_w2, (size_t)c->n_slices * ((E + kRouterETile - 1) / kRouterETile)) == cudaSuccess;
-  if (cfg->n_group == 0) {
-    // two-launch routing: the counter of finished tokens (zero between calls)
+  {
+    // tables of the grouping routine when it runs inside a routing kernel (calls of at most kFusedMaxTokens rows)
     const int gmax = cfg->max_tokens < kFusedMaxTokens ? cfg->max_tokens : kFusedMaxTokens;
     for (int g = 1; g <= gmax; ++g)
       c->fused_smem_max = std::max(c->fused_smem_max, route_group_block_smem(cfg->E, g, cfg->top_k));
-    ok = ok && dmalloc(&c->fused.done_cnt, 1) == cudaSuccess;
-    ok = ok && cudaMemset(c->fused.done_cnt, 0, sizeof(int32_t)) == cudaSuccess;
-    // exact-logit routing of the smallest calls: rows of x staged in shared memory by 16-byte copies
-    c->exact_ok = exact_smem(cfg->H, (int)act_b) <= kExactMaxSmem && (cfg->H * act_b) % 16 == 0 && cfg->H % 4 == 0;
+    if (cfg->n_group == 0) {
+      // two-launch cluster routing: the counter of finished tokens (zero between calls)
+      ok = ok && dmalloc(&c->fused.done_cnt, 1) == cudaSuccess;
+      ok = ok && cudaMemset(c->fused.done_cnt, 0, sizeof(int32_t)) == cudaSuccess;
+    }
+    // exact-logit routing of the smallest calls: rows of x staged in shared memory by 16-byte copies; group-limited
+    // routing when its groups are whole 32-expert slots (see route_select_kernel)
+    c->exact_ok = exact_smem(cfg->H, (int)act_b) <= kExactMaxSmem && (cfg->H * act_b) % 16 == 0 && cfg->H % 4 == 0 &&
+                  (cfg->n_group == 0 || (cfg->E / cfg->n_group) % 32 == 0);
     if (c->exact_ok)
       ok = ok && dmalloc(&c->logits64, (size_t)std::min<int>(cfg->max_tokens, kExactTokWide) * E) == cudaSuccess;
   }
@@ -551,6 +556,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
                                       (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
       ok = ok && cudaFuncSetAttribute(route_refine_kernel<MOEV_ACT_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
+    }
+    {
       if (c->exact_ok) {
         const int xs = (int)exact_smem(cfg->H, (int)act_b);
         if (cfg->afmt == MOEV_ACT_FP32) {
@@ -563,10 +570,11 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
             ok = ok && cudaFuncSetAttribute(router_exact_kernel<MOEV_ACT_BF16, 1, kExactTokWide>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)exact_smem(cfg->H, (int)act_b, kExactTokWide)) == cudaSuccess;
         }
-        ok = ok && cudaFuncSetAttribute(route_select_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
-        ok = ok && cudaFuncSetAttribute(route_select_kernel<kMaxE / 32>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)std::max<size_t>(c->fused_smem_max, 1024)) == cudaSuccess;
+        const int ssm = (int)std::max<size_t>(c->fused_smem_max, 1024);
+        ok = ok && cudaFuncSetAttribute(route_select_kernel<8, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ssm) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(route_select_kernel<kMaxE / 32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ssm) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(route_select_kernel<8, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ssm) == cudaSuccess;
+        ok = ok && cudaFuncSetAttribute(route_select_kernel<kMaxE / 32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ssm) == cudaSuccess;
       }
     }
     if (c->resolved_impl == MOEV_IMPL_TCGEN05) {
@@ -688,7 +696,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   const bool ahead = pdl;   // (single calls too: back-to-back calls on one stream, 215.6 -> 213.0 us per call at gamma = 4)
   const int wide_ratio = (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0;
   const int act_bytes = g.afmt == MOEV_ACT_FP32 ? 4 : 2;
-  const int exact_tok = (c->exact_ok && g.n_group == 0 && (g.afmt == MOEV_ACT_BF16 || gamma <= kExactMaxTokens))
+  const int exact_tok = (c->exact_ok && (g.afmt == MOEV_ACT_BF16 || gamma <= kExactMaxTokens))
                             ? exact_tokens_per_cta(gamma, g.H, act_bytes, g.E, c->n_sm) : 0;
   if (exact_tok > 0) {
     // the smallest calls: fp64 logits in one pass, selection and grouping by one CTA (route_exact.cuh)
@@ -706,10 +714,11 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
     else { if (epc == 1) go(router_exact_kernel<MOEV_ACT_BF16, 1>); else go(router_exact_kernel<MOEV_ACT_BF16, 2>); }
     if (ev) cudaEventRecord(ev[1], st);
     {
-      auto sel = g.E <= 256 ? route_select_kernel<8> : route_select_kernel<kMaxE / 32>;
+      auto sel = g.n_group > 0 ? (g.E <= 256 ? route_select_kernel<8, true> : route_select_kernel<kMaxE / 32, true>)
+                               : (g.E <= 256 ? route_select_kernel<8, false> : route_select_kernel<kMaxE / 32, false>);
       launch_k(sel, dim3(1), dim3(kSelectThreads), route_group_block_smem(g.E, gamma, g.top_k), st, pdl, c->T, O,
                (const double*)c->logits64, gamma, g.E, g.top_k, g.score, g.routed_scale, g.n_shared, c->unit_cap, wide_ratio,
-               pdl ? 1 : 0);
+               pdl ? 1 : 0, layer->router_bias, g.n_group, g.topk_group);
     }
     if (ev) cudaEventRecord(ev[2], st);
   } else {

@@ -344,12 +344,28 @@ __device__ __forceinline__ void select_topk_warp(unsigned long long (&key)[EPL],
 // being computed; it spends that time on one pass over its own code with made-up keys and no global memory
 // access, which leaves its instructions in the SM's instruction cache (a single CTA that runs its code once,
 // front to back, otherwise waits for every line of it).
-template <int EPL>
+// Warp-wide maximum of one double per lane (as order-preserving keys); owner = the lowest lane that holds it.
+__device__ __forceinline__ unsigned long long warp_max_key(unsigned long long key, int& owner) {
+  const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+  const uint32_t mhi = __reduce_max_sync(0xffffffffu, hi);
+  const bool c1 = hi == mhi;
+  const uint32_t mlo = __reduce_max_sync(0xffffffffu, c1 ? lo : 0u);
+  owner = __ffs(__ballot_sync(0xffffffffu, c1 && lo == mlo)) - 1;
+  return ((unsigned long long)mhi << 32) | mlo;
+}
+
+// GROUPED: the group-limited routing of the published DeepSeek-V3 models on the exact logits (see
+// topk_refine_kernel<.., true> for the definition): c = sigmoid(logit) + bias in fp64, a group's score = the sum of
+// its two largest c, the topk_group best groups are kept (ties to the lower group), top-k by c among their
+// experts (ties to the lower id), weights from the unbiased scores.  Needs E / n_group to be a multiple of 32:
+// lane l holds the experts l, l + 32, ..., so a group is a run of whole slots in every lane.
+template <int EPL, bool GROUPED = false>
 __global__ void __launch_bounds__(kSelectThreads, 1) route_select_kernel(Tables T, RouteOut O,
                                                                         const double* __restrict__ logits, int gamma,
                                                                         int E, int k, int score, float routed_scale,
                                                                         int n_shared, int unit_cap, int wide_ratio,
-                                                                        int warm) {
+                                                                        int warm, const float* __restrict__ router_bias,
+                                                                        int n_group, int topk_group) {
   extern __shared__ __align__(16) int32_t select_sm[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int A = gamma * k;
@@ -369,13 +385,50 @@ __global__ void __launch_bounds__(kSelectThreads, 1) route_select_kernel(Tables 
 #pragma unroll
       for (int j = 0; j < EPL; ++j) {
         const int e = lane + 32 * j;
-        const double v = dry ? (double)((e * 37 + t) & 63) : (e < E ? __ldcg(logits + (size_t)t * E + e) : 0.0);
+        double v = dry ? (double)((e * 37 + t) & 63) * 0.125 - 3.0 : (e < E ? __ldcg(logits + (size_t)t * E + e) : 0.0);
+        if constexpr (GROUPED)
+          v = 1.0 / (1.0 + exp(-v)) + ((router_bias && !dry && e < E) ? (double)__ldg(router_bias + e) : 0.0);
         key[j] = e < E ? double_key(v) : 0ull;
       }
       MOEV_RF_MARK(7, t == 0 && !dry);
+      if constexpr (GROUPED) {
+        // group scores: the slots of a group are consecutive; every lane keeps the two largest of its own values
+        // of the group, the warp's two largest follow by two maxima (the owner of the first gives up its largest)
+        const int spg = E / n_group / 32;   // slots per group
+        unsigned long long a1 = 0ull, a2 = 0ull, gkey = 0ull;   // key 0 is below every real key
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) {
+          if (32 * j < E) {
+            const unsigned long long v = key[j];
+            if (v > a1) { a2 = a1; a1 = v; } else if (v > a2) a2 = v;
+            if ((j + 1) % spg == 0) {
+              int owner;
+              const unsigned long long m1 = warp_max_key(a1, owner);
+              if (lane == owner) a1 = a2;
+              const unsigned long long m2 = warp_max_key(a1, owner);
+              if (lane == j / spg) gkey = double_key(key_double(m1) + key_double(m2));
+              a1 = 0ull; a2 = 0ull;
+            }
+          }
+        }
+        // rank of the groups by counting (lane g holds group g): larger score first, equal scores by lower index
+        int rank = 0;
+        for (int h = 0; h < n_group; ++h) {
+          const unsigned long long kh = __shfl_sync(0xffffffffu, gkey, h);
+          rank += (kh > gkey || (kh == gkey && h < lane)) ? 1 : 0;
+        }
+        const uint32_t keep = __ballot_sync(0xffffffffu, lane < n_group && rank < topk_group);
+#pragma unroll
+        for (int j = 0; j < EPL; ++j)
+          if (!((keep >> (j / spg)) & 1u)) key[j] = 0ull;
+      }
       float sel_v;
       int sel_e;
       select_topk_warp<EPL>(key, k, lane, sel_v, sel_e);
+      if constexpr (GROUPED) {  // the weights come from the logits of the selected experts, not from c
+        const int e = lane < k ? sel_e : 0;
+        sel_v = dry ? sel_v : (float)__ldcg(logits + (size_t)t * E + e);
+      }
       MOEV_RF_MARK(8, t == 0 && !dry);
       // router weights of the k selected experts (lane j owns the j-th), as route_refine_kernel forms them
       const float top = __shfl_sync(0xffffffffu, sel_v, 0);

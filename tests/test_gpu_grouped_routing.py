@@ -69,6 +69,23 @@ def test_full_router_shape():
     _run(shape, 64, 8, 4, 2.5, "scattered")
 
 
+@pytest.mark.parametrize("E,H,n_group,topk_group,k,gamma,routing,bias_sd", [
+    (256, 7168, 8, 4, 8, 4, "iid", 0.1),          # the published DeepSeek-V3 settings at the paper's gamma
+    (256, 7168, 8, 4, 8, 8, "scattered", 0.1),    # exact logits with exact ties
+    (256, 2048, 8, 4, 8, 1, "clustered", 1.0),    # one row; biases as large as the scores
+    (256, 1024, 1, 1, 8, 7, "iid", 0.1),          # one group of 256: eight slots per group
+    (256, 1024, 2, 1, 6, 5, "iid", 0.3),
+    (512, 1024, 8, 3, 8, 6, "iid", 0.1),          # sixteen experts per lane, two slots per group
+    (128, 1024, 4, 2, 4, 13, "iid", 0.1),         # one router row per CTA: 16 rows per CTA
+    (128, 1024, 4, 4, 8, 16, "scattered", 0.1),
+])
+def test_group_limited_routing_on_fp64_logits(E, H, n_group, topk_group, k, gamma, routing, bias_sd):
+    """Small calls whose groups are whole 32-expert slots take the routing path with fp64 logits from the
+    start; the group rule is applied to those logits by one warp per token."""
+    shape = small_shape("deepseek", H=H, I=256, E=E, top_k=k)
+    _run(shape, gamma, n_group, topk_group, 2.5, routing, bias_sd=bias_sd, seed=gamma)
+
+
 def test_bad_group_configs_are_rejected():
     for ng, kg, score in [(3, 1, synth.SCORE_SIGMOID), (8, 9, synth.SCORE_SIGMOID), (8, 4, synth.SCORE_SOFTMAX),
                           (64, 4, synth.SCORE_SIGMOID)]:
