@@ -20,7 +20,9 @@
 //   route_select_kernel   one CTA: a warp per token takes the k largest logits out one by one
 //                         (64-bit order-preserving keys, ties to the lower expert id), forms the
 //                         router weights as the other paths do, and the CTA builds the expert
-//                         union, offsets, permutation and work units (route_group_block).
+//                         union, offsets, permutation and work units (route_group_block).  The
+//                         GROUPED instantiation applies DeepSeek's group-limited rule to the exact
+//                         logits first (groups of whole 32-expert slots).
 //
 // The selected ids are those of a sequential fp64 evaluation whenever the fp64 decision margin
 // exceeds the difference between two fp64 summation orders (~1e-13 relative), as on the other
