@@ -423,7 +423,8 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
   ok = ok && dmalloc(&c->part_w2, (size_t)c->n_slices * ((E + kRouterETile - 1) / kRouterETile)) == cudaSuccess;
   {
     // tables of the grouping routine when it runs inside a routing kernel (calls of at most kFusedMaxTokens rows)
-    const int gmax = cfg->max_tokens < kFusedMaxTokens ? cfg->max_tokens : kFusedMaxTokens;
+    const int glim = std::max(kFusedMaxTokens, cfg->n_group > 0 ? kExactGroupedMaxTokens : 0);
+    const int gmax = cfg->max_tokens < glim ? cfg->max_tokens : glim;
     for (int g = 1; g <= gmax; ++g)
       c->fused_smem_max = std::max(c->fused_smem_max, route_group_block_smem(cfg->E, g, cfg->top_k));
     if (cfg->n_group == 0) {
@@ -436,7 +437,7 @@ moev_status moev_create(const moev_config* cfg, moev_ctx** out) {
     c->exact_ok = exact_smem(cfg->H, (int)act_b) <= kExactMaxSmem && (cfg->H * act_b) % 16 == 0 && cfg->H % 4 == 0 &&
                   (cfg->n_group == 0 || (cfg->E / cfg->n_group) % 32 == 0);
     if (c->exact_ok)
-      ok = ok && dmalloc(&c->logits64, (size_t)std::min<int>(cfg->max_tokens, kExactTokWide) * E) == cudaSuccess;
+      ok = ok && dmalloc(&c->logits64, (size_t)std::min<int>(cfg->max_tokens, cfg->n_group > 0 ? kExactGroupedMaxTokens : kExactTokWide) * E) == cudaSuccess;
   }
   ok = ok && dmalloc(&c->T.topk_ids, A) == cudaSuccess;
   ok = ok && dmalloc(&c->T.topk_w, A) == cudaSuccess;
@@ -697,7 +698,7 @@ moev_status moev_verify(moev_ctx* c, const moev_layer* layer, const void* x, int
   const int wide_ratio = (c->wide_ok && g.act_quant == MOEV_ACTQ_NONE) ? kWideRatio : 0;
   const int act_bytes = g.afmt == MOEV_ACT_FP32 ? 4 : 2;
   const int exact_tok = (c->exact_ok && (g.afmt == MOEV_ACT_BF16 || gamma <= kExactMaxTokens))
-                            ? exact_tokens_per_cta(gamma, g.H, act_bytes, g.E, c->n_sm) : 0;
+                            ? exact_tokens_per_cta(gamma, g.H, act_bytes, g.E, c->n_sm, g.n_group > 0) : 0;
   if (exact_tok > 0) {
     // the smallest calls: fp64 logits in one pass, selection and grouping by one CTA (route_exact.cuh)
     const int epc = exact_epc(g.E, c->n_sm);

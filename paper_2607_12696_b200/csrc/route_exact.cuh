@@ -50,8 +50,13 @@ inline size_t exact_smem(int H, int act_bytes, int tok = kExactTok) { return (si
 // Rows per CTA for a call of gamma rows, or 0 when the call takes another routing path: 8 rows per CTA up to
 // kExactMaxTokens; 16 rows up to 16 where a CTA holds one router row (E <= SMs) and 16 rows of x fit (measured
 // on the GPT-OSS router shape at gamma = 16 against the cluster path; with two token groups of 8 the cluster path wins).
-inline int exact_tokens_per_cta(int gamma, int H, int act_bytes, int E, int n_sm) {
+// rows per call served with group-limited routing, whose other path needs two candidate stages (measured on the
+// DeepSeek router shape, 8 groups: gamma = 12 / 16: -11 / -13 us per call, gamma = 24: +10 us)
+constexpr int kExactGroupedMaxTokens = 16;
+inline int exact_tokens_per_cta(int gamma, int H, int act_bytes, int E, int n_sm, bool grouped = false) {
   if (gamma <= kExactMaxTokens) return kExactTok;
+  if (grouped && gamma <= kExactGroupedMaxTokens)
+    return (exact_epc(E, n_sm) == 1 && exact_smem(H, act_bytes, kExactTokWide) <= kExactMaxSmem) ? kExactTokWide : kExactTok;
   if (gamma <= kExactTokWide && exact_epc(E, n_sm) == 1 && exact_smem(H, act_bytes, kExactTokWide) <= kExactMaxSmem) return kExactTokWide;
   return 0;
 }

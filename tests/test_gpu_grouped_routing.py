@@ -78,6 +78,8 @@ def test_full_router_shape():
     (512, 1024, 8, 3, 8, 6, "iid", 0.1),          # sixteen experts per lane, two slots per group
     (128, 1024, 4, 2, 4, 13, "iid", 0.1),         # one router row per CTA: 16 rows per CTA
     (128, 1024, 4, 4, 8, 16, "scattered", 0.1),
+    (256, 2048, 8, 4, 8, 12, "iid", 0.1),         # 9 to 16 rows with two router rows per CTA: two token groups of 8
+    (256, 2048, 8, 4, 8, 16, "clustered", 0.1),
 ])
 def test_group_limited_routing_on_fp64_logits(E, H, n_group, topk_group, k, gamma, routing, bias_sd):
     """Small calls whose groups are whole 32-expert slots take the routing path with fp64 logits from the
